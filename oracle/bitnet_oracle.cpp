@@ -1,0 +1,416 @@
+// CPU oracle for the ternary mixed-precision GEMM path (int8 activations x ternary weights).
+//
+// TEST INFRASTRUCTURE ONLY.  Plain, slow, scalar C++17 written from the paper's statement
+// of the method; it shares no code, header, table or constant with the CUDA library and is
+// never on the product path.  Only the tests, the smoke check and the benchmark's CPU
+// baseline may call it.
+//
+// What each function follows:
+//   oracle_quant_act      Alg. 1 Phase 1 ("Quantization"), Sec. 2.1 / Sec. 3.2.2 (int8 absmax
+//                         activation quantisation); rounding and operation order: see below.
+//   oracle_mpgemm_def     Alg. 1 Phase 2 / Eq. 1: R[n,m] = sum_k A_q[n,k] * W[m,k].
+//   oracle_dequant        the "Scale" of I2_S (Sec. 3.2.2): y = acc * act_scale * w_scale.
+//   oracle_pack_i2s       I2_S, 2 bits per weight (Table 1); the byte layout is this build's.
+//   oracle_pack_tl        TL1 codes of Table 4 (Alg. 3 PreprocessWeights); TL2 codes of
+//                         Table 5 with the signed-unsigned split (Sec. 3.1.2, Alg. 4
+//                         PreprocessWeights) and the block-fitting split ThreeK / TwoK.
+//   oracle_tl_build_lut   Alg. 3 / Alg. 4 PreCompute (element-wise LUT, Eq. 3), int16 entries
+//                         kept exact (Sec. 3.2.1, the lossless *_1 variants).
+//   oracle_tl_mpgemm      Alg. 3 / Alg. 4 accumulation by table lookups from the packed blob,
+//                         sign applied per group (caption of Fig. 5).
+//   oracle_i2s_mpgemm     Alg. 1 Phase 2 evaluated straight from the I2_S blob.
+//
+// Readings where the paper is silent (all listed in the design notes):
+//   * activations are quantised per token (row of x); per_tensor != 0 gives the paper's
+//     literal "per-tensor" wording (one absmax over all T*K values);
+//   * amax is floored at 1e-5; s = 127 / amax in binary32; q = clamp(rint(x*s), -128, 127)
+//     with round-half-to-even; act_scale = amax / 127 in binary32;
+//   * TL2 code of a triple: v = 9*w0 + 3*w1 + w2, index = |v|, sign = [v < 0] -- this
+//     reproduces every printed row of Table 5;
+//   * TL1 code of a pair: 3*(w0+1) + (w1+1) -- Table 4.
+//
+// Pins (tests/test_oracle_*.py): closed-form quantiser cases, brute-force enumeration on tiny
+// shapes against numpy, one-hot position probes of every packed bit, Tables 4 and 5 as golden
+// text fixtures, LUT identities, and I2_S == TL1 == TL2 == definition on random inputs.
+// No function here is "parity unpinned".
+
+#include <cmath>
+#include <cstdint>
+#include <cstdlib>
+#include <cstring>
+#include <vector>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+namespace {
+
+constexpr int FMT_I2S = 0;
+constexpr int FMT_TL1 = 1;
+constexpr int FMT_TL2 = 2;
+
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// ---- TL geometry: 32-row tiles; a TL2 tile covers 96 weights (32 triples), a TL1 tile 64 (32 pairs)
+struct TlGeom {
+  int64_t three_k;      // columns handled by TL2 triples
+  int64_t two_k;        // columns handled by TL1 pairs
+  int64_t tiles3;       // TL2 tiles per row block
+  int64_t tiles2;       // TL1 tiles per row block
+  int64_t block_bytes;  // bytes of one 32-row block
+};
+
+bool tl_geom(int fmt, int64_t M, int64_t K, int bk3, TlGeom* g) {
+  if (M <= 0 || K <= 0 || (M % 32) != 0 || (K % 2) != 0) return false;
+  if (bk3 == 0) bk3 = 96;
+  if (bk3 < 0 || (bk3 % 96) != 0) return false;
+  if (fmt == FMT_TL2) {
+    g->three_k = (K / bk3) * bk3;  // ThreeK = floor(K / BK3) * BK3
+    g->two_k = K - g->three_k;     // TwoK = K - ThreeK
+  } else if (fmt == FMT_TL1) {
+    g->three_k = 0;
+    g->two_k = K;
+  } else {
+    return false;
+  }
+  g->tiles3 = g->three_k / 96;
+  g->tiles2 = ceil_div(g->two_k, 64);
+  g->block_bytes = g->tiles3 * 640 + g->tiles2 * 512;
+  return true;
+}
+
+inline int tern_ok(int8_t w) { return w >= -1 && w <= 1; }
+
+}  // namespace
+
+extern "C" {
+
+// ---------------------------------------------------------------------------------------------
+// Quantiser.  x[T][K] fp32 -> q[T][K] int8, act_scale[T], act_sum[T] (nullable).
+int oracle_quant_act(const float* x, int64_t T, int64_t K, int per_tensor, int8_t* q,
+                     float* act_scale, int32_t* act_sum) {
+  if (!x || !q || !act_scale || T < 1 || K < 1) return 1;
+  float tensor_amax = 0.0f;
+  if (per_tensor) {
+    for (int64_t i = 0; i < T * K; ++i) tensor_amax = std::fmax(tensor_amax, std::fabs(x[i]));
+  }
+  for (int64_t t = 0; t < T; ++t) {
+    const float* xr = x + t * K;
+    float amax = 0.0f;
+    if (per_tensor) {
+      amax = tensor_amax;
+    } else {
+      for (int64_t k = 0; k < K; ++k) amax = std::fmax(amax, std::fabs(xr[k]));
+    }
+    const float amax_c = std::fmax(amax, 1e-5f);
+    volatile float s = 127.0f / amax_c;        // one binary32 division
+    volatile float inv = amax_c / 127.0f;      // one binary32 division
+    act_scale[t] = inv;
+    int64_t sum = 0;
+    for (int64_t k = 0; k < K; ++k) {
+      volatile float p = xr[k] * s;            // one binary32 product, no fused multiply-add
+      float r = std::nearbyintf(p);            // round-half-to-even in the default mode
+      if (r > 127.0f) r = 127.0f;
+      if (r < -128.0f) r = -128.0f;
+      const int v = (int)r;
+      q[t * K + k] = (int8_t)v;
+      sum += v;
+    }
+    if (act_sum) act_sum[t] = (int32_t)sum;
+  }
+  return 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Definition (Alg. 1 Phase 2).  acc[t][m] = sum_k q[t][k] * w[m][k].  Returns 2 on int32 overflow.
+// The OpenMP pragma only spreads independent output rows over cores when the file is built with
+// -fopenmp (the timed CPU baseline); the arithmetic is the same scalar loop either way.
+int oracle_mpgemm_def(const int8_t* q, const int8_t* w, int64_t T, int64_t M, int64_t K,
+                      int32_t* acc) {
+  if (!q || !w || !acc || T < 1 || M < 1 || K < 1) return 1;
+  int bad = 0;
+#pragma omp parallel for schedule(static) reduction(| : bad)
+  for (int64_t m = 0; m < M; ++m) {
+    const int8_t* wr = w + m * K;
+    for (int64_t t = 0; t < T; ++t) {
+      const int8_t* qr = q + t * K;
+      int64_t s = 0;
+      for (int64_t k = 0; k < K; ++k) s += (int64_t)qr[k] * (int64_t)wr[k];
+      if (s > INT32_MAX || s < INT32_MIN) bad |= 1;
+      acc[t * M + m] = (int32_t)s;
+    }
+  }
+  return bad ? 2 : 0;
+}
+
+// y[t][m] = acc * act_scale[t] * w_scale, evaluated in double.
+void oracle_dequant(const int32_t* acc, const float* act_scale, float w_scale, int64_t T, int64_t M,
+                    double* y) {
+  for (int64_t t = 0; t < T; ++t)
+    for (int64_t m = 0; m < M; ++m)
+      y[t * M + m] = (double)acc[t * M + m] * (double)act_scale[t] * (double)w_scale;
+}
+
+// ---------------------------------------------------------------------------------------------
+// I2_S.  code = w + 1 (0,1,2), two bits.  A row occupies ceil(K/128)*32 bytes; positions past K
+// hold weight 0 (code 1).  Byte 4j+b of a row carries the weights k = 16j + 4s + b, s = 0..3,
+// the code of slot s in bits [2s, 2s+1].
+size_t oracle_i2s_packed_bytes(int64_t M, int64_t K) {
+  if (M < 1 || K < 1) return 0;
+  return (size_t)M * (size_t)ceil_div(K, 128) * 32;
+}
+
+int oracle_pack_i2s(const int8_t* w, int64_t M, int64_t K, uint8_t* packed) {
+  if (!w || !packed || M < 1 || K < 1) return 1;
+  const int64_t row_bytes = ceil_div(K, 128) * 32;
+  for (int64_t m = 0; m < M; ++m) {
+    for (int64_t byte = 0; byte < row_bytes; ++byte) {
+      const int64_t j = byte / 4, b = byte % 4;
+      unsigned v = 0;
+      for (int s = 0; s < 4; ++s) {
+        const int64_t k = 16 * j + 4 * s + b;
+        int8_t wk = (k < K) ? w[m * K + k] : (int8_t)0;
+        if (!tern_ok(wk)) return 3;
+        v |= (unsigned)(wk + 1) << (2 * s);
+      }
+      packed[m * row_bytes + byte] = (uint8_t)v;
+    }
+  }
+  return 0;
+}
+
+int oracle_unpack_i2s(const uint8_t* packed, int64_t M, int64_t K, int8_t* w) {
+  if (!w || !packed || M < 1 || K < 1) return 1;
+  const int64_t row_bytes = ceil_div(K, 128) * 32;
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t k = 0; k < K; ++k) {
+      const int64_t j = k / 16, s = (k % 16) / 4, b = k % 4;
+      const unsigned code = (packed[m * row_bytes + 4 * j + b] >> (2 * s)) & 3u;
+      if (code == 3u) return 3;
+      w[m * K + k] = (int8_t)((int)code - 1);
+    }
+  return 0;
+}
+
+// Alg. 1 Phase 2 straight from the blob (decodes each weight where it is used).
+int oracle_i2s_mpgemm(const uint8_t* packed, int64_t M, int64_t K, const int8_t* q, int64_t T,
+                      int32_t* acc) {
+  if (!packed || !q || !acc || M < 1 || K < 1 || T < 1) return 1;
+  const int64_t row_bytes = ceil_div(K, 128) * 32;
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t t = 0; t < T; ++t) {
+      int64_t s = 0;
+      for (int64_t k = 0; k < K; ++k) {
+        const unsigned byte = packed[m * row_bytes + 4 * (k / 16) + (k % 4)];
+        const int wv = (int)((byte >> (2 * ((k % 16) / 4))) & 3u) - 1;
+        s += (int64_t)q[t * K + k] * wv;
+      }
+      acc[t * M + m] = (int32_t)s;
+    }
+  return 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// TL codes.
+// Table 4: (w0, w1) -> 3*(w0+1) + (w1+1), 0..8.
+int oracle_tl1_code(int w0, int w1) { return 3 * (w0 + 1) + (w1 + 1); }
+// Table 5: v = 9 w0 + 3 w1 + w2; index |v| (0..13) in bits 0..3, sign [v<0] in bit 4.
+int oracle_tl2_code(int w0, int w1, int w2) {
+  const int v = 9 * w0 + 3 * w1 + w2;
+  return (v < 0 ? 16 : 0) | (v < 0 ? -v : v);
+}
+
+size_t oracle_tl_packed_bytes(int fmt, int64_t M, int64_t K, int bk3) {
+  TlGeom g;
+  if (!tl_geom(fmt, M, K, bk3, &g)) return 0;
+  return (size_t)(M / 32) * (size_t)g.block_bytes;
+}
+
+void oracle_tl_split(int fmt, int64_t K, int bk3, int64_t* three_k, int64_t* two_k) {
+  TlGeom g;
+  if (!tl_geom(fmt, 32, K, bk3, &g)) { *three_k = -1; *two_k = -1; return; }
+  *three_k = g.three_k;
+  *two_k = g.two_k;
+}
+
+// Blob = for each block of 32 rows: tiles3 TL2 tiles, then tiles2 TL1 tiles.
+//  TL2 tile (640 B): row r owns bytes [16r,16r+16) of the 512-byte index plane, byte i = index of
+//    triple 2i in the low nibble and of triple 2i+1 in the high nibble; then a 128-byte sign plane,
+//    row r owns the little-endian uint32 at 512+4r whose bit g is the sign of triple g.
+//  TL1 tile (512 B): same index plane over 32 pairs; pairs past the end of K carry code 4 = (0,0).
+int oracle_pack_tl(int fmt, const int8_t* w, int64_t M, int64_t K, int bk3, uint8_t* packed) {
+  TlGeom g;
+  if (!w || !packed || !tl_geom(fmt, M, K, bk3, &g)) return 1;
+  std::memset(packed, 0, (size_t)(M / 32) * (size_t)g.block_bytes);
+  for (int64_t m = 0; m < M; ++m) {
+    const int64_t rb = m / 32, r = m % 32;
+    uint8_t* blk = packed + rb * g.block_bytes;
+    const int8_t* wr = w + m * K;
+    for (int64_t k = 0; k < K; ++k)
+      if (!tern_ok(wr[k])) return 3;
+    for (int64_t t = 0; t < g.tiles3; ++t) {
+      uint8_t* tile = blk + t * 640;
+      uint32_t signs = 0;
+      for (int grp = 0; grp < 32; ++grp) {
+        const int64_t k = t * 96 + 3 * grp;
+        const int code = oracle_tl2_code(wr[k], wr[k + 1], wr[k + 2]);
+        const int idx = code & 15;
+        if (code & 16) signs |= (1u << grp);
+        tile[16 * r + grp / 2] |= (uint8_t)((grp & 1) ? (idx << 4) : idx);
+      }
+      for (int b = 0; b < 4; ++b) tile[512 + 4 * r + b] = (uint8_t)(signs >> (8 * b));
+    }
+    for (int64_t t = 0; t < g.tiles2; ++t) {
+      uint8_t* tile = blk + g.tiles3 * 640 + t * 512;
+      for (int grp = 0; grp < 32; ++grp) {
+        const int64_t k = g.three_k + t * 64 + 2 * grp;
+        const int idx = (k < K) ? oracle_tl1_code(wr[k], wr[k + 1]) : 4;
+        tile[16 * r + grp / 2] |= (uint8_t)((grp & 1) ? (idx << 4) : idx);
+      }
+    }
+  }
+  return 0;
+}
+
+int oracle_unpack_tl(int fmt, const uint8_t* packed, int64_t M, int64_t K, int bk3, int8_t* w) {
+  TlGeom g;
+  if (!w || !packed || !tl_geom(fmt, M, K, bk3, &g)) return 1;
+  for (int64_t m = 0; m < M; ++m) {
+    const int64_t rb = m / 32, r = m % 32;
+    const uint8_t* blk = packed + rb * g.block_bytes;
+    int8_t* wr = w + m * K;
+    for (int64_t t = 0; t < g.tiles3; ++t) {
+      const uint8_t* tile = blk + t * 640;
+      uint32_t signs = 0;
+      for (int b = 0; b < 4; ++b) signs |= (uint32_t)tile[512 + 4 * r + b] << (8 * b);
+      for (int grp = 0; grp < 32; ++grp) {
+        const uint8_t byte = tile[16 * r + grp / 2];
+        const int idx = (grp & 1) ? (byte >> 4) : (byte & 15);
+        if (idx > 13) return 3;
+        int v = ((signs >> grp) & 1u) ? -idx : idx;
+        if (idx == 0 && ((signs >> grp) & 1u)) return 3;
+        // balanced-ternary digits of v in [-13, 13]
+        int d[3];
+        for (int i = 2; i >= 0; --i) {
+          int rem = ((v % 3) + 3) % 3;  // 0,1,2
+          if (rem == 2) rem = -1;
+          d[i] = rem;
+          v = (v - rem) / 3;
+        }
+        const int64_t k = t * 96 + 3 * grp;
+        wr[k] = (int8_t)d[0];
+        wr[k + 1] = (int8_t)d[1];
+        wr[k + 2] = (int8_t)d[2];
+      }
+    }
+    for (int64_t t = 0; t < g.tiles2; ++t) {
+      const uint8_t* tile = blk + g.tiles3 * 640 + t * 512;
+      for (int grp = 0; grp < 32; ++grp) {
+        const uint8_t byte = tile[16 * r + grp / 2];
+        const int idx = (grp & 1) ? (byte >> 4) : (byte & 15);
+        if (idx > 8) return 3;
+        const int64_t k = g.three_k + t * 64 + 2 * grp;
+        if (k < K) {
+          wr[k] = (int8_t)(idx / 3 - 1);
+          wr[k + 1] = (int8_t)(idx % 3 - 1);
+        } else if (idx != 4) {
+          return 3;
+        }
+      }
+    }
+  }
+  return 0;
+}
+
+// Number of 16-slot tables one token needs: ThreeK/3 triples followed by tiles2*32 pairs
+// (pairs past the end of K are all-zero tables).
+int64_t oracle_tl_num_groups(int fmt, int64_t K, int bk3) {
+  TlGeom g;
+  if (!tl_geom(fmt, 32, K, bk3, &g)) return -1;
+  return g.tiles3 * 32 + g.tiles2 * 32;
+}
+
+// PreCompute of Alg. 3 / Alg. 4 for one token: lut[group][16] int16.
+//  triple group: lut[i] = w0*a0 + w1*a1 + w2*a2 for the triple whose value 9w0+3w1+w2 equals i,
+//    i = 0..13 (the non-negative half after mirror consolidation); slots 14, 15 are zero.
+//  pair group: lut[i] = w0*a0 + w1*a1 with (w0, w1) = (i/3 - 1, i%3 - 1), i = 0..8; slots 9..15 zero.
+int oracle_tl_build_lut(int fmt, const int8_t* q, int64_t K, int bk3, int16_t* lut) {
+  TlGeom g;
+  if (!q || !lut || !tl_geom(fmt, 32, K, bk3, &g)) return 1;
+  const int64_t ng = g.tiles3 * 32 + g.tiles2 * 32;
+  std::memset(lut, 0, (size_t)ng * 16 * sizeof(int16_t));
+  for (int64_t grp = 0; grp < g.tiles3 * 32; ++grp) {
+    const int a0 = q[3 * grp], a1 = q[3 * grp + 1], a2 = q[3 * grp + 2];
+    for (int w0 = -1; w0 <= 1; ++w0)
+      for (int w1 = -1; w1 <= 1; ++w1)
+        for (int w2 = -1; w2 <= 1; ++w2) {
+          const int v = 9 * w0 + 3 * w1 + w2;
+          if (v < 0) continue;
+          lut[grp * 16 + v] = (int16_t)(w0 * a0 + w1 * a1 + w2 * a2);
+        }
+  }
+  for (int64_t p = 0; p < g.tiles2 * 32; ++p) {
+    const int64_t k = g.three_k + 2 * p;
+    if (k >= K) continue;
+    const int a0 = q[k], a1 = q[k + 1];
+    for (int w0 = -1; w0 <= 1; ++w0)
+      for (int w1 = -1; w1 <= 1; ++w1)
+        lut[(g.tiles3 * 32 + p) * 16 + 3 * (w0 + 1) + (w1 + 1)] = (int16_t)(w0 * a0 + w1 * a1);
+  }
+  return 0;
+}
+
+// Accumulation of Alg. 3 / Alg. 4: table lookups by the packed indices, the sign bit of a triple
+// negating the looked-up value.
+int oracle_tl_mpgemm(int fmt, const uint8_t* packed, int64_t M, int64_t K, int bk3, const int8_t* q,
+                     int64_t T, int32_t* acc) {
+  TlGeom g;
+  if (!packed || !q || !acc || T < 1 || !tl_geom(fmt, M, K, bk3, &g)) return 1;
+  const int64_t ng = g.tiles3 * 32 + g.tiles2 * 32;
+  std::vector<int16_t> lut((size_t)ng * 16);
+  for (int64_t t = 0; t < T; ++t) {
+    if (oracle_tl_build_lut(fmt, q + t * K, K, bk3, lut.data())) return 1;
+    for (int64_t m = 0; m < M; ++m) {
+      const int64_t rb = m / 32, r = m % 32;
+      const uint8_t* blk = packed + rb * g.block_bytes;
+      int64_t s = 0;
+      for (int64_t tile_i = 0; tile_i < g.tiles3; ++tile_i) {
+        const uint8_t* tile = blk + tile_i * 640;
+        uint32_t signs = 0;
+        for (int b = 0; b < 4; ++b) signs |= (uint32_t)tile[512 + 4 * r + b] << (8 * b);
+        for (int grp = 0; grp < 32; ++grp) {
+          const uint8_t byte = tile[16 * r + grp / 2];
+          const int idx = (grp & 1) ? (byte >> 4) : (byte & 15);
+          const int val = lut[(tile_i * 32 + grp) * 16 + idx];
+          s += ((signs >> grp) & 1u) ? -val : val;
+        }
+      }
+      for (int64_t tile_i = 0; tile_i < g.tiles2; ++tile_i) {
+        const uint8_t* tile = blk + g.tiles3 * 640 + tile_i * 512;
+        for (int grp = 0; grp < 32; ++grp) {
+          const uint8_t byte = tile[16 * r + grp / 2];
+          const int idx = (grp & 1) ? (byte >> 4) : (byte & 15);
+          s += lut[(g.tiles3 * 32 + tile_i * 32 + grp) * 16 + idx];
+        }
+      }
+      acc[t * M + m] = (int32_t)s;
+    }
+  }
+  return 0;
+}
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+  int n = 1;
+#pragma omp parallel
+  {
+#pragma omp master
+    n = omp_get_num_threads();
+  }
+  return n;
+#else
+  return 1;
+#endif
+}
+
+}  // extern "C"

@@ -1,0 +1,340 @@
+"""Pins of the CPU oracle against things other than itself.
+
+Each test checks the oracle against a fact fixed by the paper or by mathematics: printed table rows
+(golden text fixtures), closed forms, brute force written independently in numpy / pure Python,
+invariants, and cross-format equality (the paper's "lossless" claim for I2_S, TL1_1 and TL2_1).
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+rng = np.random.default_rng(1234)
+
+
+def rand_ternary(M, K, p0=1 / 3):
+    u = rng.random((M, K))
+    return np.where(u < p0, 0, np.where(u < p0 + (1 - p0) / 2, 1, -1)).astype(np.int8)
+
+
+def rand_q(T, K):
+    return rng.integers(-127, 128, size=(T, K)).astype(np.int8)
+
+
+# ----------------------------------------------------------------------------- quantiser (Alg. 1 Phase 1)
+def test_quant_half_even_closed_form():
+    # amax = 127 makes the multiplier exactly 1, so q = rint(x) with ties to even
+    x = np.array([[127.0, 0.5, 1.5, 2.5, -0.5, -1.5, 126.5, -2.5, 3.5]], np.float32)
+    q, sc, sm = oracle.quant_act(x)
+    assert q.tolist() == [[127, 0, 2, 2, 0, -2, 126, -2, 4]]
+    assert sc[0] == np.float32(1.0)
+    assert sm[0] == sum(q[0].tolist())
+
+
+def test_quant_extreme_maps_to_127_and_scale():
+    x = rng.standard_normal((5, 333)).astype(np.float32)
+    q, sc, sm = oracle.quant_act(x)
+    for t in range(5):
+        k = np.argmax(np.abs(x[t]))
+        assert abs(int(q[t, k])) == 127
+        assert np.sign(q[t, k]) == np.sign(x[t, k])
+        assert sc[t] == np.float32(np.abs(x[t]).max()) / np.float32(127.0)
+        assert q[t].min() >= -127
+        assert sm[t] == q[t].astype(np.int64).sum()
+
+
+def test_quant_power_of_two_invariance_and_odd_symmetry():
+    x = rng.standard_normal((3, 257)).astype(np.float32)
+    q0, s0, _ = oracle.quant_act(x)
+    for j in (-7, 3, 11):
+        qj, sj, _ = oracle.quant_act(x * np.float32(2.0 ** j))
+        assert np.array_equal(qj, q0)
+        assert np.array_equal(sj, s0 * np.float32(2.0 ** j))
+    qn, sn, smn = oracle.quant_act(-x)
+    assert np.array_equal(qn, -q0) and np.array_equal(sn, s0)
+
+
+def test_quant_matches_float64_rounding_away_from_ties():
+    # independent evaluation in float64: wherever x*s is further than 1e-3 from a .5 tie the rounded
+    # integer is unambiguous and must agree
+    x = rng.standard_normal((4, 1000)).astype(np.float32)
+    q, sc, _ = oracle.quant_act(x)
+    for t in range(4):
+        amax = np.abs(x[t]).astype(np.float64).max()
+        p = x[t].astype(np.float64) * 127.0 / amax
+        clear = np.abs(p - np.floor(p) - 0.5) > 1e-3
+        assert np.array_equal(q[t][clear], np.rint(p[clear]).astype(np.int8))
+
+
+def test_quant_zero_row_and_per_tensor():
+    x = np.zeros((2, 64), np.float32)
+    x[1, 3] = 2.0
+    q, sc, sm = oracle.quant_act(x)
+    assert not q[0].any() and sc[0] == np.float32(1e-5) / np.float32(127.0) and sm[0] == 0
+    assert q[1, 3] == 127
+    qt, sct, _ = oracle.quant_act(x, per_tensor=True)
+    assert sct[0] == sct[1] == np.float32(2.0) / np.float32(127.0)
+    x2 = rng.standard_normal((3, 100)).astype(np.float32)
+    qa, sa, _ = oracle.quant_act(x2, per_tensor=True)
+    qb, sb, _ = oracle.quant_act(x2.reshape(1, -1))
+    assert np.array_equal(qa.reshape(-1), qb.reshape(-1)) and np.all(sa == sb[0])
+
+
+def test_quant_outlier_recipe_range():
+    # two +-20 outliers among N(0,1) values: amax = 20 so a value |x| <= 6.3 quantises to |q| <= 40
+    x = rng.standard_normal((1, 1536)).astype(np.float32).clip(-6.2, 6.2)
+    x[0, 10], x[0, 900] = 20.0, -20.0
+    q, sc, _ = oracle.quant_act(x)
+    assert q[0, 10] == 127 and q[0, 900] == -127
+    mask = np.ones(1536, bool)
+    mask[[10, 900]] = False
+    assert np.abs(q[0][mask]).max() <= 40
+
+
+# ----------------------------------------------------------------------------- definition (Alg. 1 Phase 2, Eq. 1)
+def test_definition_brute_force_all_rows_tiny():
+    K = 5
+    rows = np.array(list(itertools.product((-1, 0, 1), repeat=K)), np.int8)  # all 3^5 weight rows
+    q = np.array([[1, -2, 3, -4, 5], [127, -128, 127, -128, 0], [0, 0, 0, 0, 0]], np.int8)
+    acc = oracle.mpgemm_def(q, rows)
+    for t in range(q.shape[0]):
+        for m in range(rows.shape[0]):
+            s = 0
+            for k in range(K):
+                s += int(q[t][k]) * int(rows[m][k])
+            assert acc[t, m] == s
+
+
+def test_definition_vs_numpy_matmul_and_not_transposed():
+    T, M, K = 3, 37, 129
+    q, w = rand_q(T, K), rand_ternary(M, K)
+    acc = oracle.mpgemm_def(q, w)
+    assert acc.shape == (T, M)
+    assert np.array_equal(acc, q.astype(np.int64) @ w.astype(np.int64).T)
+
+
+def test_definition_permutation_and_linearity():
+    T, M, K = 2, 16, 96
+    q, w = rand_q(T, K), rand_ternary(M, K)
+    perm = rng.permutation(K)
+    assert np.array_equal(oracle.mpgemm_def(q, w), oracle.mpgemm_def(q[:, perm], w[:, perm]))
+    wa, wb = w.copy(), w.copy()
+    wa[:, K // 2:] = 0
+    wb[:, :K // 2] = 0
+    assert np.array_equal(oracle.mpgemm_def(q, w), oracle.mpgemm_def(q, wa) + oracle.mpgemm_def(q, wb))
+
+
+def test_dequant_closed_form():
+    acc = np.array([[3, -5, 0]], np.int32)
+    y = oracle.dequant(acc, np.array([0.5], np.float32), 0.25)
+    assert y.tolist() == [[0.375, -0.625, 0.0]]
+
+
+# ----------------------------------------------------------------------------- I2_S packing (Table 1: 2 bpw)
+def test_i2s_size_and_bpw():
+    assert oracle.i2s_packed_bytes(1536, 1536) == 1536 * 1536 // 4        # exactly 2 bits per weight
+    assert oracle.i2s_packed_bytes(3200, 8640) == 3200 * 68 * 32          # rows padded to 128 weights
+    assert oracle.i2s_packed_bytes(8192, 28672) * 8 == 2 * 8192 * 28672
+
+
+def test_i2s_round_trip_and_padding_code():
+    for (M, K) in [(3, 128), (5, 192), (7, 64), (2, 8640 // 8)]:
+        w = rand_ternary(M, K)
+        p = oracle.pack_i2s(w)
+        assert p.size == oracle.i2s_packed_bytes(M, K)
+        assert np.array_equal(oracle.unpack_i2s(p, M, K), w)
+    # K = 64: the second half of the 128-weight block is padding = weight 0 = code 1 in every slot
+    w = rand_ternary(1, 64)
+    p = oracle.pack_i2s(w)
+    assert p.size == 32 and np.all(p[16:] == 0b01010101)
+
+
+def test_i2s_documented_bit_positions():
+    # byte 4j+b of a row holds weights 16j + 4s + b in bits [2s, 2s+1]; checked by hand-built bytes
+    K = 128
+    for k in range(K):
+        for val in (-1, 1):
+            w = np.zeros((1, K), np.int8)
+            w[0, k] = val
+            p = oracle.pack_i2s(w)
+            j, s, b = k // 16, (k % 16) // 4, k % 4
+            expect = np.full(32, 0b01010101, np.uint8)
+            expect[4 * j + b] = (0b01010101 & ~(3 << (2 * s))) | ((val + 1) << (2 * s))
+            assert np.array_equal(p, expect)
+
+
+def test_i2s_one_hot_dot_products():
+    # a single +-1 at position k against q[k] = k - 60 returns exactly +-(k - 60)
+    K = 128
+    q = (np.arange(K) - 60).astype(np.int8).reshape(1, K)
+    w = np.zeros((2 * K, K), np.int8)
+    for k in range(K):
+        w[2 * k, k] = 1
+        w[2 * k + 1, k] = -1
+    acc = oracle.i2s_mpgemm(oracle.pack_i2s(w), 2 * K, K, q)
+    for k in range(K):
+        assert acc[0, 2 * k] == k - 60 and acc[0, 2 * k + 1] == -(k - 60)
+
+
+def test_i2s_rejects_non_ternary():
+    w = np.zeros((1, 128), np.int8)
+    w[0, 5] = 2
+    with pytest.raises(ValueError):
+        oracle.pack_i2s(w)
+
+
+# ----------------------------------------------------------------------------- TL codes (Tables 4, 5)
+def _read_rows(name):
+    rows = []
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            rows.append(line.split())
+    return rows
+
+
+def test_tl1_codes_match_table4():
+    rows = _read_rows("tl1_table4.txt")
+    assert len(rows) == 9
+    for w0, w1, code in rows:
+        assert oracle.tl1_code(int(w0), int(w1)) == int(code, 2)
+
+
+def test_tl2_codes_match_table5_and_cover_all_triples():
+    rows = _read_rows("tl2_table5.txt")
+    assert len(rows) == 9
+    for w0, w1, w2, sign, idx in rows:
+        c = oracle.tl2_code(int(w0), int(w1), int(w2))
+        assert c >> 4 == int(sign) and c & 15 == int(idx, 2)
+    seen = {}
+    for t in itertools.product((-1, 0, 1), repeat=3):
+        c = oracle.tl2_code(*t)
+        assert (c & 15) <= 13                              # ceil(27/2) = 14 table entries
+        assert c not in seen
+        seen[c] = t
+        # mirror consolidation: the negated triple has the same index and the opposite sign
+        cn = oracle.tl2_code(*[-v for v in t])
+        assert (cn & 15) == (c & 15)
+        if any(t):
+            assert (cn >> 4) != (c >> 4)
+    assert oracle.tl2_code(0, 0, 0) == 0
+    assert len(seen) == 27
+
+
+def test_tl_block_fitting_split():
+    # ThreeK = floor(K / BK3) * BK3, TwoK = K - ThreeK with BK3 = 96
+    for K, three, two in [(3200, 3168, 32), (4096, 4032, 64), (8192, 8160, 32), (14336, 14304, 32),
+                          (28672, 28608, 64), (1536, 1536, 0), (8640, 8640, 0)]:
+        assert oracle.tl_split("tl2", K) == (three, two)
+    assert oracle.tl_split("tl2", 8192, 192) == (8064, 128)
+    assert oracle.tl_split("tl1", 8192) == (0, 8192)
+
+
+def test_tl_sizes_and_bpw():
+    # TL2: 5 bits per 3 weights, TL1: 4 bits per 2 weights
+    assert oracle.tl_packed_bytes("tl2", 1536, 1536) * 8 * 3 == 5 * 1536 * 1536
+    assert oracle.tl_packed_bytes("tl1", 1536, 1536) * 8 == 2 * 1536 * 1536
+    assert oracle.tl_packed_bytes("tl2", 32, 8192) == 85 * 640 + 512
+    assert oracle.tl_packed_bytes("tl2", 33, 96) == 0 and oracle.tl_packed_bytes("tl2", 32, 97) == 0
+
+
+@pytest.mark.parametrize("fmt,K", [("tl1", 64), ("tl1", 130), ("tl2", 96), ("tl2", 96 * 2 + 32),
+                                   ("tl2", 96 + 64), ("tl2", 34), ("tl2", 96 * 3 + 70)])
+def test_tl_round_trip(fmt, K):
+    w = rand_ternary(64, K)
+    p = oracle.pack_tl(fmt, w)
+    assert p.size == oracle.tl_packed_bytes(fmt, 64, K)
+    assert np.array_equal(oracle.unpack_tl(fmt, p, 64, K), w)
+
+
+def test_tl2_documented_byte_positions():
+    # one TL2 tile (32 rows x 96 weights): row r, triple g -> nibble (g odd: high) of byte 16r + g//2,
+    # sign -> bit g of the little-endian word at 512 + 4r
+    w = np.zeros((32, 96), np.int8)
+    w[5, 3 * 7: 3 * 7 + 3] = (-1, 1, 0)     # v = -9 + 3 = -6 -> index 6, sign 1
+    w[31, 3 * 30: 3 * 30 + 3] = (0, 1, -1)  # v = 2 -> index 2, sign 0
+    p = oracle.pack_tl("tl2", w)
+    expect = np.zeros(640, np.uint8)
+    expect[16 * 5 + 3] = 6 << 4
+    expect[512 + 4 * 5 + 0] = 1 << 7
+    expect[16 * 31 + 15] = 2
+    assert np.array_equal(p, expect)
+
+
+def test_tl1_documented_byte_positions_and_padding():
+    w = np.zeros((32, 34), np.int8)         # 17 pairs, tile padded to 32 pairs with code 4
+    w[2, 0:2] = (1, -1)                     # code 6, pair 0 -> low nibble of byte 32
+    w[2, 32:34] = (-1, -1)                  # code 0, pair 16 -> low nibble of byte 40
+    p = oracle.pack_tl("tl1", w)
+    expect = np.full(512, 0x44, np.uint8)
+    expect[16 * 2 + 0] = 0x46
+    expect[16 * 2 + 8] = 0x40
+    assert np.array_equal(p, expect)
+
+
+# ----------------------------------------------------------------------------- LUT build (Alg. 3 / Alg. 4 PreCompute)
+def test_lut_identities():
+    q = rand_q(1, 96 * 2 + 64)[0]
+    lut = oracle.tl_build_lut("tl2", q)
+    assert lut.shape == (64 + 32, 16)
+    for g in range(64):
+        a0, a1, a2 = (int(v) for v in q[3 * g: 3 * g + 3])
+        e = lut[g]
+        assert e[0] == 0 and e[1] == a2 and e[3] == a1 and e[9] == a0 and e[13] == a0 + a1 + a2
+        assert e[2] == a1 - a2 and e[4] == a1 + a2 and e[14] == 0 and e[15] == 0
+        assert np.abs(e).max() <= 384
+        for i in range(14):                  # every entry = dot with the balanced-ternary digits of i
+            d0 = round(i / 9)
+            d1 = round((i - 9 * d0) / 3)
+            d2 = i - 9 * d0 - 3 * d1
+            assert {d0, d1, d2} <= {-1, 0, 1}
+            assert e[i] == d0 * a0 + d1 * a1 + d2 * a2
+    for p in range(32):
+        a0, a1 = int(q[192 + 2 * p]), int(q[192 + 2 * p + 1])
+        e = lut[64 + p]
+        assert e[4] == 0 and all(e[i] + e[8 - i] == 0 for i in range(9))
+        assert e[8] == a0 + a1 and e[6] == a0 - a1 and e[5] == a1 and e[7] == a0
+        assert not e[9:].any()
+
+
+# ----------------------------------------------------------------------------- whole mpGEMM: invariants, cross-format equality
+@pytest.mark.parametrize("K", [128, 96 * 2 + 32, 96 * 4 + 64, 576])
+def test_all_formats_give_the_definition(K):
+    T, M = 3, 64
+    q, w = rand_q(T, K), rand_ternary(M, K, 0.4)
+    ref = q.astype(np.int64) @ w.astype(np.int64).T
+    assert np.array_equal(oracle.mpgemm_def(q, w), ref)
+    if K % 64 == 0:
+        assert np.array_equal(oracle.i2s_mpgemm(oracle.pack_i2s(w), M, K, q), ref)
+    assert np.array_equal(oracle.tl_mpgemm("tl1", oracle.pack_tl("tl1", w), M, K, q), ref)
+    assert np.array_equal(oracle.tl_mpgemm("tl2", oracle.pack_tl("tl2", w), M, K, q), ref)
+
+
+def test_constant_weight_invariants():
+    T, M, K = 2, 32, 96 * 3 + 32
+    q = rand_q(T, K)
+    sums = q.astype(np.int64).sum(axis=1)
+    for val in (0, 1, -1):
+        w = np.full((M, K), val, np.int8)
+        for acc in (oracle.mpgemm_def(q, w),
+                    oracle.tl_mpgemm("tl2", oracle.pack_tl("tl2", w), M, K, q),
+                    oracle.tl_mpgemm("tl1", oracle.pack_tl("tl1", w), M, K, q)):
+            assert np.array_equal(acc, np.repeat((val * sums)[:, None], M, axis=1))
+
+
+def test_tl2_one_hot_across_split_and_tile_boundaries():
+    K = 96 * 2 + 64                      # two TL2 tiles then one TL1 tile
+    q = ((np.arange(K) % 251) - 125).astype(np.int8).reshape(1, K)
+    probes = [0, 1, 2, 94, 95, 96, 97, 191, 192, 193, 254, 255]
+    w = np.zeros((32, K), np.int8)
+    for i, k in enumerate(probes):
+        w[i, k] = 1 if i % 2 == 0 else -1
+    acc = oracle.tl_mpgemm("tl2", oracle.pack_tl("tl2", w), 32, K, q)
+    for i, k in enumerate(probes):
+        assert acc[0, i] == (1 if i % 2 == 0 else -1) * int(q[0, k])
+    assert not acc[0, len(probes):].any()
