@@ -1,0 +1,407 @@
+#!/usr/bin/env python
+"""Benchmark of the ternary mpGEMM hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Workload (config.workload = "sweep100b"): the 100B-shaped decode sweep at batch 1 -- 80 layers of
+four ternary linears (8192->10240, 8192->8192, 8192->57344, 28672->8192), every tensor with its own
+seeded weights resident in HBM in the I2_S encoding (17.1 GB), one fp32 activation vector per linear.
+One step = one pass over all 320 linears: absmax int8 quantiser, then I2_S mpGEMV with the fused
+rescale, replayed from one CUDA graph.  `value` = I2_S bytes streamed per step / step time (GB/s),
+so it charges the quantisers and every launch gap to the weight stream.  The same sweep in the TL2
+encoding and the prefill mpGEMM (2048 x 4096 x 14336, int8 tensor cores) are timed in the same run
+and reported under "tl2" and "prefill".  Inputs (17 GB) exceed L2 (126 MB) many times over, so no L2
+flush is needed between steps.
+
+With --gpus N > 1 (under torchrun) every rank runs an independent replica of the sweep on its own
+GPU (the path has no exchange step; weak scaling, no collective on the data path).
+
+--impl reference times the CPU oracle on a bounded sample of the same workload on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "mpgemv_weight_stream_batch1"
+UNIT = "GB/s"
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=float(d["hbm_gbs"]), bf16=float(d["bf16_tflops"]), which="measured")
+    return dict(hbm=6650.0, bf16=1590.0, which="fallback")
+
+
+# ------------------------------------------------------------------------------------------------ reference arm
+def oracle_sample(wl, layer=0, j=1):
+    """The bounded CPU sample: one linear of the sweep (default W_o of layer 0, 8192 x 8192)."""
+    import numpy as np
+    w = wl.weights(layer, j).numpy()
+    x = wl.activations(layer, j, 1).numpy()
+    return np.ascontiguousarray(w), np.ascontiguousarray(x)
+
+
+def oracle_step(oracle, w, x):
+    q, sc, _ = oracle.quant_act(x)
+    acc = oracle.mpgemm_def(q, w)
+    return oracle.dequant(acc, sc, 2.0 / 3.0)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2502_11880_b200 import synth
+    oracle.build()
+    wl = synth.CONFIGS["sweep100b"]
+    w, x = oracle_sample(wl)
+    M, K = w.shape
+    nbytes = M * K // 4
+    for _ in range(args.warmup):
+        oracle_step(oracle, w, x)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(oracle, w, x)
+    dt = (time.perf_counter() - t0) / args.steps
+    val = nbytes / dt / 1e9
+    sample = f"layer 0 linear 'o' ({K}->{M}, {nbytes / 1e6:.1f} MB as I2_S) per step, quantiser + definition + rescale"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": "sweep100b", "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------ our arm
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.f.close()
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+class Sweep:
+    """The decode sweep resident on one GPU: packed blobs, activation buffers, outputs, workspaces."""
+
+    def __init__(self, bn, torch, wl, fmts, layers, device):
+        self.bn, self.torch, self.wl, self.layers = bn, torch, wl, layers
+        self.lin = wl.linears
+        self.fmts = fmts
+        self.blobs = {f: [] for f in fmts}
+        self.w_scale = []
+        t0 = time.time()
+        for layer in range(layers):
+            for j, lin in enumerate(self.lin):
+                w = wl.weights(layer, j, device=device)
+                self.w_scale.append(bn.synth.absmean_scale(w))
+                for f in fmts:
+                    self.blobs[f].append(bn.pack(f, w, check=False))
+                del w
+        torch.cuda.synchronize()
+        self.setup_s = time.time() - t0
+        self.bytes = {f: sum(b.numel() for b in self.blobs[f]) for f in fmts}
+        # activations: all vectors of the sweep in one pinned host buffer and one device buffer
+        self.x_off, self.y_off = [], []
+        xo = yo = 0
+        for layer in range(layers):
+            for lin in self.lin:
+                self.x_off.append(xo)
+                self.y_off.append(yo)
+                xo += lin.K
+                yo += lin.M
+        self.x_host = torch.empty(xo, dtype=torch.float32).pin_memory()
+        self.y_host = torch.empty(yo, dtype=torch.float32).pin_memory()
+        i = 0
+        for layer in range(layers):
+            for j, lin in enumerate(self.lin):
+                self.x_host[self.x_off[i]: self.x_off[i] + lin.K] = wl.activations(layer, j, 1)[0]
+                i += 1
+        self.x_dev = self.x_host.to(device)
+        self.y_dev = torch.zeros(yo, dtype=torch.float32, device=device)
+        self.q_dev = torch.empty(xo, dtype=torch.int8, device=device)
+        self.sc_dev = torch.empty(len(self.x_off), dtype=torch.float32, device=device)
+        kmax = max(l.K for l in self.lin)
+        mmax = max(l.M for l in self.lin)
+        self.ws = {}
+        for f in fmts:
+            n = max(bn.bitnet_mpgemm_workspace_bytes(f, 1, l.M, l.K) for l in self.lin)
+            self.ws[f] = torch.zeros(max(n, 16), dtype=torch.uint8, device=device)
+        self.kmax, self.mmax = kmax, mmax
+
+    def n_linears(self):
+        return len(self.x_off)
+
+    def views(self, i):
+        lin = self.lin[i % len(self.lin)]
+        x = self.x_dev[self.x_off[i]: self.x_off[i] + lin.K].view(1, lin.K)
+        q = self.q_dev[self.x_off[i]: self.x_off[i] + lin.K].view(1, lin.K)
+        y = self.y_dev[self.y_off[i]: self.y_off[i] + lin.M].view(1, lin.M)
+        sc = self.sc_dev[i: i + 1]
+        return lin, x, q, sc, y
+
+    def step_device(self, fmt, quant=True, gemv=True):
+        """One pass over every linear, inputs resident: quantiser then mpGEMV (2 launches per linear)."""
+        bn = self.bn
+        for i in range(self.n_linears()):
+            lin, x, q, sc, y = self.views(i)
+            if quant:
+                bn.bitnet_quant_act(x, q=q, act_scale=sc, act_sum=self._sum)
+            if gemv:
+                bn.bitnet_mpgemm(fmt, self.blobs[fmt][i], self.w_scale[i], lin.M, lin.K, q, sc, y=y,
+                                 workspace=self.ws[fmt])
+
+    def step_host(self, fmt):
+        """The same pass through the host-buffer entry point: H2D of x, quantise, mpGEMV, D2H of y."""
+        bn = self.bn
+        for i in range(self.n_linears()):
+            lin, x, q, sc, y = self.views(i)
+            xh = self.x_host[self.x_off[i]: self.x_off[i] + lin.K].view(1, lin.K)
+            yh = self.y_host[self.y_off[i]: self.y_off[i] + lin.M].view(1, lin.M)
+            bn.bitnet_linear_host(fmt, self.blobs[fmt][i], self.w_scale[i], lin.M, lin.K, xh, yh, x, q, sc, y,
+                                  workspace=self.ws[fmt])
+
+    def make_graph(self, fmt, quant=True, gemv=True):
+        torch = self.torch
+        self._sum = torch.empty(1, dtype=torch.int32, device=self.x_dev.device)
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            self.step_device(fmt, quant, gemv)       # warm every kernel variant before capture
+        torch.cuda.current_stream().wait_stream(s)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self.step_device(fmt, quant, gemv)
+        return g
+
+
+def time_replays(torch, fn, steps, warmup, dist=None):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+        dist.barrier()
+    return ms / steps
+
+
+def bench_prefill(bn, torch, synth, steps, warmup):
+    wl = synth.CONFIGS["prefill"]
+    lin, T = wl.linears[0], wl.tokens[0]
+    w = wl.weights(0, 0, device="cuda")
+    blob = bn.pack("i2s", w, check=False)
+    w_scale = synth.absmean_scale(w)
+    del w
+    x = wl.activations(0, 0, T).cuda()
+    q, sc, sm = bn.bitnet_quant_act(x)
+    y = torch.empty((T, lin.M), dtype=torch.float32, device="cuda")
+
+    def gemm():
+        bn.bitnet_mpgemm("i2s", blob, w_scale, lin.M, lin.K, q, sc, y=y)
+
+    def both():
+        bn.bitnet_quant_act(x, q=q, act_scale=sc, act_sum=sm)
+        gemm()
+
+    ms_gemm = time_replays(torch, gemm, steps, warmup)
+    ms_both = time_replays(torch, both, steps, warmup)
+    ops = 2.0 * T * lin.K * lin.M
+    return {"workload": f"prefill {T}x{lin.K}x{lin.M}", "ms_gemm": ms_gemm, "ms_quant_plus_gemm": ms_both,
+            "int8_tops": ops / ms_gemm / 1e9, "int8_tops_with_quant": ops / ms_both / 1e9}
+
+
+def run_ours(args):
+    import torch
+    import paper_2502_11880_b200 as bn
+    from paper_2502_11880_b200 import synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    bn.lib()   # fail loudly here if the extension is missing
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    pk = peaks()
+    wl = synth.CONFIGS["sweep100b"]
+    layers = args.layers or wl.layers
+    fmts = ["i2s", "tl2"] if not args.skip_tl2 else ["i2s"]
+    sw = Sweep(bn, torch, wl, fmts, layers, torch.device("cuda", local))
+
+    # ---- headline: I2_S sweep, quantiser + GEMV, one graph replay per step
+    g_full = sw.make_graph("i2s")
+    sampler = ClockSampler(local) if rank == 0 else None
+    ms_step = time_replays(torch, g_full.replay, args.steps, args.warmup, dist)
+    clocks = sampler.stop() if sampler else None
+    total_bytes = sw.bytes["i2s"] * world
+    value = total_bytes / ms_step / 1e6
+
+    # ---- dominant kernel alone (GEMV launches only): roofline
+    g_gemv = sw.make_graph("i2s", quant=False)
+    ms_gemv = time_replays(torch, g_gemv.replay, args.steps, args.warmup, dist)
+    n_lin = sw.n_linears()
+    achieved = sw.bytes["i2s"] / ms_gemv / 1e6
+    g_quant = sw.make_graph("i2s", gemv=False)
+    ms_quant = time_replays(torch, g_quant.replay, args.steps, args.warmup, dist)
+
+    # ---- end to end through the host-buffer entry point
+    ms_e2e = time_replays(torch, lambda: (sw.step_host("i2s"), torch.cuda.current_stream().synchronize()),
+                          max(2, args.steps // 4), 3, dist)
+    e2e_val = total_bytes / ms_e2e / 1e6
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
+        "data": "synthetic",
+        "config": {"workload": "sweep100b", "layers": layers, "linears_per_layer": 4, "tokens": 1, "format": "i2s",
+                   "packed_bytes": sw.bytes["i2s"], "parallelism": f"replicas x{world}",
+                   "l2": "inputs (17 GB of weights) exceed L2; no flush needed", "launch": "one CUDA graph per step",
+                   "pct_of_8TBps": 100.0 * (value / world) / 8000.0},
+        "e2e": {"value": e2e_val, "unit": UNIT, "ms_per_step": ms_e2e,
+                "h2d_bytes_per_step": int(sw.x_host.numel() * 4), "d2h_bytes_per_step": int(sw.y_host.numel() * 4),
+                "note": "per linear: pinned fp32 x -> device, quantiser, mpGEMV, fp32 y -> pinned host; weights resident"},
+        "gpu_launches": 2 * n_lin * args.steps,
+        "roofline": {"bound": "hbm", "kernel": "gemv_i2s_kernel<1,4>", "achieved": achieved, "peak": pk["hbm"],
+                     "unit": "GB/s", "frac": achieved / pk["hbm"], "peak_source": pk["which"],
+                     "bytes_per_launch": sw.bytes["i2s"] / n_lin, "us_per_launch": 1e3 * ms_gemv / n_lin,
+                     "traffic": None},
+        "breakdown": {"ms_gemv_only": ms_gemv, "ms_quant_only": ms_quant, "setup_s": sw.setup_s},
+        "clocks": clocks,
+    }
+
+    if rank == 0:
+        if "tl2" in fmts:
+            g_tl = sw.make_graph("tl2")
+            ms_tl = time_replays(torch, g_tl.replay, args.steps, args.warmup)
+            g_tl_g = sw.make_graph("tl2", quant=False)
+            ms_tl_g = time_replays(torch, g_tl_g.replay, args.steps, args.warmup)
+            line["tl2"] = {"packed_bytes": sw.bytes["tl2"], "ms_per_step": ms_tl, "value": sw.bytes["tl2"] / ms_tl / 1e6,
+                           "unit": UNIT, "gemv_only_GBps": sw.bytes["tl2"] / ms_tl_g / 1e6,
+                           "frac_of_hbm_peak": sw.bytes["tl2"] / ms_tl_g / 1e6 / pk["hbm"]}
+        del sw, g_full, g_gemv, g_quant
+        torch.cuda.empty_cache()
+        if not args.skip_prefill:
+            pf = bench_prefill(bn, torch, synth, max(3, args.steps // 2), 3)
+            pf["frac_of_int8_peak"] = pf["int8_tops"] / (2.0 * pk["bf16"])
+            pf["int8_peak_used"] = f"2 x {pk['which']} bf16 dense ({pk['bf16']} TFLOP/s)"
+            line["prefill"] = pf
+        if world == 1 and not args.skip_cpu:
+            import oracle
+            oracle.build()
+            w, x = oracle_sample(wl)
+            reps, t0 = 0, time.perf_counter()
+            while True:
+                oracle_step(oracle, w, x)
+                reps += 1
+                dt = time.perf_counter() - t0
+                if dt > 10.0 or reps >= 200:
+                    break
+            nb = w.shape[0] * w.shape[1] // 4
+            line["cpu_baseline"] = {"value": nb * reps / dt / 1e9, "unit": UNIT, "cores": oracle.num_threads(),
+                                    "kind": "oracle",
+                                    "sample": f"layer 0 linear 'o' (8192->8192, {nb / 1e6:.1f} MB as I2_S) x {reps} "
+                                              f"repetitions in {dt:.1f} s: quantiser + definition + rescale"}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=0, help="fewer layers than the workload's 80 (debugging only)")
+    ap.add_argument("--skip-tl2", action="store_true")
+    ap.add_argument("--skip-prefill", action="store_true")
+    ap.add_argument("--skip-cpu", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

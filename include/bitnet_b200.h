@@ -1,0 +1,141 @@
+/*
+ * bitnet_b200 -- ternary-weight mixed-precision GEMV/GEMM (mpGEMM) for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of libbitnet_b200.so.  The operation is the one the paper states in Alg. 1 / Eq. 1:
+ *
+ *     A_q      = Quantization(A)                      A: activations, T tokens x K features, fp32
+ *     acc[t,m] = sum_k A_q[t,k] * W[m,k]              W: M x K ternary weights in {-1,0,+1}
+ *     y[t,m]   = acc[t,m] * act_scale[t] * w_scale    ("Int2 with a Scale", Sec. 3.2.2)
+ *
+ * reached through three weight encodings: I2_S (2 bits per weight, multiply-add; Table 1,
+ * Sec. 3.2.2), TL1 (pairs of weights -> 4-bit table index, Table 4 / Alg. 3) and TL2 (triples ->
+ * 4-bit index + 1-bit sign, Table 5 / Alg. 4, Sec. 3.1).  All three give the same int32
+ * accumulators as the definition (the lossless variants of Sec. 3.2).
+ *
+ * Naming: T = tokens (the paper's N), K = reduction length, M = output features; y and acc are
+ * token-major [T][M].
+ *
+ * Conventions for every entry point unless stated otherwise:
+ *   - pointers are DEVICE pointers owned by the caller; nothing is retained after the call;
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream); work is queued
+ *     on it and the call returns without synchronising;
+ *   - the library allocates no device memory and never throws; the return value is a status code
+ *     below, and no kernel is launched when argument validation fails;
+ *   - x, q, packed blobs, y, acc_out and workspaces must be 16-byte aligned.
+ */
+#ifndef BITNET_B200_H
+#define BITNET_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { BITNET_FMT_I2S = 0, BITNET_FMT_TL1 = 1, BITNET_FMT_TL2 = 2 } bitnet_fmt_t;
+
+enum {
+  BITNET_OK = 0,
+  BITNET_ERR_INVALID_ARG = 1,       /* null or misaligned pointer, bad enum, non-positive size       */
+  BITNET_ERR_UNSUPPORTED_SHAPE = 2, /* K % 64 != 0 (I2_S); K odd or M % 32 != 0 (TL); bad bk3         */
+  BITNET_ERR_WORKSPACE = 3,         /* workspace missing or smaller than *_workspace_bytes reports   */
+  BITNET_ERR_BAD_WEIGHT = 4,        /* reserved: packers report bad weights through dev_status       */
+  BITNET_ERR_CUDA = 5,              /* a CUDA call failed; see bitnet_last_cuda_error()              */
+  BITNET_ERR_TIMEOUT = 6            /* a bounded device-side wait gave up (reported via dev_status)  */
+};
+
+/* Text for a status code (static storage). */
+const char* bitnet_status_string(int status);
+/* The cudaError_t of the most recent failing CUDA call made by this library on this thread. */
+int bitnet_last_cuda_error(void);
+
+/*
+ * Activation quantiser -- Alg. 1 Phase 1 ("Quantization"), Sec. 2.1 and 3.2.2: absmax int8.
+ *   x[T][K] fp32 row-major (read)  ->  q[T][K] int8, act_scale[T] fp32, act_sum[T] int32 (nullable).
+ * Per token t: amax = max(max_k |x[t,k]|, 1e-5); s = 127/amax (binary32); q = clamp(rint(x*s),
+ * -128, 127), ties to even; act_scale[t] = amax/127; act_sum[t] = sum_k q[t,k].
+ * per_tensor != 0 takes one amax over all T*K values (the paper's "per-tensor" wording); it equals
+ * the per-token result at T = 1.
+ */
+int bitnet_quant_act(const float* x, int64_t T, int64_t K, int per_tensor, int8_t* q,
+                     float* act_scale, int32_t* act_sum, void* stream);
+
+/*
+ * I2_S weight packer -- I2_S of Table 1 / Sec. 3.2.2 (2 bits per weight; the scale stays outside).
+ *   w[M][K] int8 in {-1,0,+1}, row-major (read) -> packed, bitnet_i2s_packed_bytes(M,K) bytes.
+ * Layout: a row occupies ceil(K/128)*32 bytes; byte 4j+b of a row holds the weights
+ * k = 16j + 4s + b (s = 0..3) as code w+1 in bits [2s, 2s+1]; positions past K hold weight 0.
+ * dev_status (nullable device int): set to BITNET_ERR_BAD_WEIGHT if a non-ternary byte is met
+ * (the blob is then undefined).  Requires K % 64 == 0.
+ */
+size_t bitnet_i2s_packed_bytes(int64_t M, int64_t K);
+int bitnet_pack_i2s(const int8_t* w, int64_t M, int64_t K, void* packed, size_t packed_bytes,
+                    int* dev_status, void* stream);
+
+/*
+ * TL weight packer -- Alg. 3 / Alg. 4 "PreprocessWeights" with the codes of Tables 4 and 5, the
+ * signed-unsigned split and the block-fitting split ThreeK/TwoK of Sec. 3.1.2.
+ *   fmt = BITNET_FMT_TL1 or BITNET_FMT_TL2; bk3 = BK3 (0 = 96; a positive multiple of 96).
+ *   TL2: columns [0, ThreeK), ThreeK = floor(K/bk3)*bk3, are coded as triples
+ *        (v = 9w0+3w1+w2, index |v|, sign [v<0]); the remaining TwoK columns as TL1 pairs
+ *        (index 3(w0+1)+(w1+1)).  TL1: all columns as pairs.
+ * Blob: for each block of 32 rows, ThreeK/96 tiles of 640 bytes then ceil(TwoK/64) tiles of 512
+ * bytes.  In a tile, row r owns bytes [16r, 16r+16): byte i = index of group 2i (low nibble) and
+ * 2i+1 (high nibble); a TL2 tile ends with 32 little-endian uint32 sign words (row r at 512+4r,
+ * bit g = sign of group g).  Pairs past K carry index 4 = (0,0).
+ * Requires K even and M % 32 == 0.  dev_status as for bitnet_pack_i2s.
+ */
+size_t bitnet_tl_packed_bytes(bitnet_fmt_t fmt, int64_t M, int64_t K, int bk3);
+int bitnet_pack_tl(bitnet_fmt_t fmt, const int8_t* w, int64_t M, int64_t K, int bk3, void* packed,
+                   size_t packed_bytes, int* dev_status, void* stream);
+
+/*
+ * mpGEMM -- Alg. 1 Phase 2 (I2_S, multiply-add) or Alg. 2 / 3 / 4 (TL: per-token tables of group
+ * partial sums built in shared memory, then one lookup per packed index; Eq. 3), followed by the
+ * rescale y = acc * (act_scale[t] * w_scale).
+ *   packed   blob from the packer of `fmt` for an M x K matrix (bk3 as given to the packer);
+ *   q[T][K]  int8, act_scale[T] fp32 from bitnet_quant_act;
+ *   y[T][M]  fp32 out; acc_out[T][M] int32 out, nullable (raw accumulators);
+ *   workspace  bitnet_mpgemm_workspace_bytes(fmt,T,M,K) bytes (may be NULL when that is 0).
+ *              It must have been zeroed once with bitnet_workspace_init and is left zeroed by
+ *              every completed call; two calls sharing a workspace must not overlap on the GPU.
+ * T <= 8 runs the decode GEMV kernels; larger T runs the int8 tensor-core kernel (I2_S) or the
+ * GEMV kernel over groups of 8 tokens (TL).
+ */
+size_t bitnet_mpgemm_workspace_bytes(bitnet_fmt_t fmt, int64_t T, int64_t M, int64_t K);
+int bitnet_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+int bitnet_mpgemm(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M, int64_t K, int bk3,
+                  const int8_t* q, const float* act_scale, int64_t T, float* y, int32_t* acc_out,
+                  void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * One linear layer with HOST activations and HOST results: copies x_host[T][K] to x_dev, runs
+ * bitnet_quant_act and bitnet_mpgemm, and copies y_dev[T][M] to y_host, all queued on `stream`
+ * (Alg. 1 end to end).  x_host / y_host should be pinned for the copies to be asynchronous; the
+ * device buffers x_dev [T*K fp32], q_dev [T*K int8], scale_dev [T fp32], y_dev [T*M fp32] and the
+ * workspace are caller-owned scratch.  The caller synchronises the stream before reading y_host.
+ */
+int bitnet_linear_host(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M, int64_t K,
+                       int bk3, const float* x_host, int64_t T, float* y_host, float* x_dev,
+                       int8_t* q_dev, float* scale_dev, float* y_dev, void* workspace,
+                       size_t workspace_bytes, void* stream);
+
+/* ---- test hooks (not part of the four operations) ------------------------------------------- */
+/* Inverse of the packers: packed -> w[M][K] int8.  dev_status set if an invalid code is met. */
+int bitnet_unpack_i2s(const void* packed, int64_t M, int64_t K, int8_t* w, int* dev_status,
+                      void* stream);
+int bitnet_unpack_tl(bitnet_fmt_t fmt, const void* packed, int64_t M, int64_t K, int bk3, int8_t* w,
+                     int* dev_status, void* stream);
+/* The tables of Alg. 3 / Alg. 4 "PreCompute" for one token, as the TL kernel builds them:
+ * lut[group][16] int16, triples first (entry i = sum for the triple of value i, i = 0..13), then
+ * pairs (entry i = sum for the pair of code i, i = 0..8); unused entries are zero.
+ * bitnet_tl_num_groups gives the group count (32 per tile). */
+int64_t bitnet_tl_num_groups(bitnet_fmt_t fmt, int64_t K, int bk3);
+int bitnet_tl_build_lut_debug(bitnet_fmt_t fmt, const int8_t* q_row, int64_t K, int bk3, int16_t* lut,
+                              void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BITNET_B200_H */

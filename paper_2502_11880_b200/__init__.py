@@ -1,0 +1,239 @@
+"""Python binding of libbitnet_b200.so: same names as the C ABI, argument marshalling only.
+
+Every step of the path (quantiser, packers, mpGEMV / mpGEMM, rescale) runs in the library's CUDA
+kernels.  PyTorch supplies device memory and streams.  There is no CPU fallback: if the shared
+library is missing or fails to load, importing a symbol from here raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import synth  # noqa: F401  (seeded inputs; holds none of the method's arithmetic)
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libbitnet_b200.so")
+
+FMT_I2S, FMT_TL1, FMT_TL2 = 0, 1, 2
+FMT = {"i2s": FMT_I2S, "tl1": FMT_TL1, "tl2": FMT_TL2}
+
+# symbols the header declares (checked by the tests against include/bitnet_b200.h)
+SYMBOLS = [
+    "bitnet_status_string", "bitnet_last_cuda_error", "bitnet_quant_act", "bitnet_i2s_packed_bytes",
+    "bitnet_pack_i2s", "bitnet_tl_packed_bytes", "bitnet_pack_tl", "bitnet_mpgemm_workspace_bytes",
+    "bitnet_workspace_init", "bitnet_mpgemm", "bitnet_linear_host", "bitnet_unpack_i2s", "bitnet_unpack_tl",
+    "bitnet_tl_num_groups", "bitnet_tl_build_lut_debug",
+]
+
+_lib = None
+
+
+class BitnetError(RuntimeError):
+    pass
+
+
+def lib():
+    """Loads the shared library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise BitnetError(f"{LIB_PATH} is missing: run `python -m paper_2502_11880_b200.build` "
+                              "(there is no fallback path)")
+        L = C.CDLL(LIB_PATH)
+        i64, vp, ci, sz, fl = C.c_int64, C.c_void_p, C.c_int, C.c_size_t, C.c_float
+        L.bitnet_status_string.argtypes = [ci]
+        L.bitnet_status_string.restype = C.c_char_p
+        L.bitnet_last_cuda_error.restype = ci
+        L.bitnet_quant_act.argtypes = [vp, i64, i64, ci, vp, vp, vp, vp]
+        L.bitnet_i2s_packed_bytes.argtypes = [i64, i64]
+        L.bitnet_i2s_packed_bytes.restype = sz
+        L.bitnet_pack_i2s.argtypes = [vp, i64, i64, vp, sz, vp, vp]
+        L.bitnet_tl_packed_bytes.argtypes = [ci, i64, i64, ci]
+        L.bitnet_tl_packed_bytes.restype = sz
+        L.bitnet_pack_tl.argtypes = [ci, vp, i64, i64, ci, vp, sz, vp, vp]
+        L.bitnet_mpgemm_workspace_bytes.argtypes = [ci, i64, i64, i64]
+        L.bitnet_mpgemm_workspace_bytes.restype = sz
+        L.bitnet_workspace_init.argtypes = [vp, sz, vp]
+        L.bitnet_mpgemm.argtypes = [ci, vp, fl, i64, i64, ci, vp, vp, i64, vp, vp, vp, sz, vp]
+        L.bitnet_linear_host.argtypes = [ci, vp, fl, i64, i64, ci, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.bitnet_unpack_i2s.argtypes = [vp, i64, i64, vp, vp, vp]
+        L.bitnet_unpack_tl.argtypes = [ci, vp, i64, i64, ci, vp, vp, vp]
+        L.bitnet_tl_num_groups.argtypes = [ci, i64, ci]
+        L.bitnet_tl_num_groups.restype = i64
+        L.bitnet_tl_build_lut_debug.argtypes = [ci, vp, i64, ci, vp, vp]
+        _lib = L
+    return _lib
+
+
+def status_string(rc: int) -> str:
+    return lib().bitnet_status_string(rc).decode()
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        extra = f", cudaError {lib().bitnet_last_cuda_error()}" if rc == 5 else ""
+        raise BitnetError(f"{what}: {status_string(rc)} (status {rc}{extra})")
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _fmt(fmt) -> int:
+    return FMT[fmt] if isinstance(fmt, str) else int(fmt)
+
+
+def _dev(t, dtype, name):
+    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise BitnetError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+    return t
+
+
+# ------------------------------------------------------------------------------------------------
+def bitnet_quant_act(x, per_tensor=False, q=None, act_scale=None, act_sum=None, stream=None):
+    """x[T][K] fp32 (CUDA) -> (q int8 [T][K], act_scale fp32 [T], act_sum int32 [T])."""
+    _dev(x, torch.float32, "x")
+    T, K = x.shape
+    q = torch.empty((T, K), dtype=torch.int8, device=x.device) if q is None else q
+    act_scale = torch.empty(T, dtype=torch.float32, device=x.device) if act_scale is None else act_scale
+    act_sum = torch.empty(T, dtype=torch.int32, device=x.device) if act_sum is None else act_sum
+    _check(lib().bitnet_quant_act(_ptr(x), T, K, int(per_tensor), _ptr(q), _ptr(act_scale), _ptr(act_sum),
+                                  _stream(stream)), "bitnet_quant_act")
+    return q, act_scale, act_sum
+
+
+def bitnet_i2s_packed_bytes(M, K) -> int:
+    return lib().bitnet_i2s_packed_bytes(M, K)
+
+
+def bitnet_tl_packed_bytes(fmt, M, K, bk3=0) -> int:
+    return lib().bitnet_tl_packed_bytes(_fmt(fmt), M, K, bk3)
+
+
+def packed_bytes(fmt, M, K, bk3=0) -> int:
+    return bitnet_i2s_packed_bytes(M, K) if _fmt(fmt) == FMT_I2S else bitnet_tl_packed_bytes(fmt, M, K, bk3)
+
+
+def _status_word(device):
+    return torch.zeros(1, dtype=torch.int32, device=device)
+
+
+def bitnet_pack_i2s(w, check=True, stream=None):
+    """w[M][K] int8 ternary (CUDA) -> uint8 blob.  check=True reads the device status word back."""
+    _dev(w, torch.int8, "w")
+    M, K = w.shape
+    n = bitnet_i2s_packed_bytes(M, K)
+    if n == 0:
+        _check(2, "bitnet_pack_i2s")
+    out = torch.empty(n, dtype=torch.uint8, device=w.device)
+    st = _status_word(w.device) if check else None
+    _check(lib().bitnet_pack_i2s(_ptr(w), M, K, _ptr(out), n, _ptr(st), _stream(stream)), "bitnet_pack_i2s")
+    if check:
+        _check(int(st.item()), "bitnet_pack_i2s")
+    return out
+
+
+def bitnet_pack_tl(fmt, w, bk3=0, check=True, stream=None):
+    _dev(w, torch.int8, "w")
+    M, K = w.shape
+    n = bitnet_tl_packed_bytes(fmt, M, K, bk3)
+    if n == 0:
+        _check(2, "bitnet_pack_tl")
+    out = torch.empty(n, dtype=torch.uint8, device=w.device)
+    st = _status_word(w.device) if check else None
+    _check(lib().bitnet_pack_tl(_fmt(fmt), _ptr(w), M, K, bk3, _ptr(out), n, _ptr(st), _stream(stream)),
+           "bitnet_pack_tl")
+    if check:
+        _check(int(st.item()), "bitnet_pack_tl")
+    return out
+
+
+def pack(fmt, w, bk3=0, check=True):
+    return bitnet_pack_i2s(w, check) if _fmt(fmt) == FMT_I2S else bitnet_pack_tl(fmt, w, bk3, check)
+
+
+def bitnet_unpack_i2s(packed, M, K, stream=None):
+    w = torch.empty((M, K), dtype=torch.int8, device=packed.device)
+    st = _status_word(packed.device)
+    _check(lib().bitnet_unpack_i2s(_ptr(packed), M, K, _ptr(w), _ptr(st), _stream(stream)), "bitnet_unpack_i2s")
+    _check(int(st.item()), "bitnet_unpack_i2s")
+    return w
+
+
+def bitnet_unpack_tl(fmt, packed, M, K, bk3=0, stream=None):
+    w = torch.empty((M, K), dtype=torch.int8, device=packed.device)
+    st = _status_word(packed.device)
+    _check(lib().bitnet_unpack_tl(_fmt(fmt), _ptr(packed), M, K, bk3, _ptr(w), _ptr(st), _stream(stream)),
+           "bitnet_unpack_tl")
+    _check(int(st.item()), "bitnet_unpack_tl")
+    return w
+
+
+def bitnet_tl_num_groups(fmt, K, bk3=0) -> int:
+    return lib().bitnet_tl_num_groups(_fmt(fmt), K, bk3)
+
+
+def bitnet_tl_build_lut_debug(fmt, q_row, bk3=0, stream=None):
+    _dev(q_row, torch.int8, "q_row")
+    K = q_row.numel()
+    ng = bitnet_tl_num_groups(fmt, K, bk3)
+    if ng < 0:
+        _check(2, "bitnet_tl_build_lut_debug")
+    lut = torch.empty((ng, 16), dtype=torch.int16, device=q_row.device)
+    _check(lib().bitnet_tl_build_lut_debug(_fmt(fmt), _ptr(q_row), K, bk3, _ptr(lut), _stream(stream)),
+           "bitnet_tl_build_lut_debug")
+    return lut
+
+
+def bitnet_mpgemm_workspace_bytes(fmt, T, M, K) -> int:
+    return lib().bitnet_mpgemm_workspace_bytes(_fmt(fmt), T, M, K)
+
+
+def bitnet_workspace_init(workspace, stream=None):
+    _check(lib().bitnet_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(),
+                                       _stream(stream)), "bitnet_workspace_init")
+
+
+def new_workspace(fmt, T, M, K, device="cuda"):
+    """A zeroed workspace tensor for bitnet_mpgemm (None when the shape needs none)."""
+    n = bitnet_mpgemm_workspace_bytes(fmt, T, M, K)
+    if n == 0:
+        return None
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    bitnet_workspace_init(ws)
+    return ws
+
+
+def bitnet_mpgemm(fmt, packed, w_scale, M, K, q, act_scale, bk3=0, y=None, acc_out=None, want_acc=False,
+                  workspace=None, stream=None):
+    """y[T][M] fp32 = (q @ W^T) * act_scale[t] * w_scale from the packed blob.  Returns (y, acc or None)."""
+    _dev(q, torch.int8, "q")
+    _dev(act_scale, torch.float32, "act_scale")
+    T = q.shape[0]
+    y = torch.empty((T, M), dtype=torch.float32, device=q.device) if y is None else y
+    if want_acc and acc_out is None:
+        acc_out = torch.empty((T, M), dtype=torch.int32, device=q.device)
+    if workspace is None:
+        workspace = new_workspace(fmt, T, M, K, q.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().bitnet_mpgemm(_fmt(fmt), _ptr(packed), float(w_scale), M, K, bk3, _ptr(q), _ptr(act_scale), T,
+                               _ptr(y), _ptr(acc_out), _ptr(workspace), ws_bytes, _stream(stream)),
+           "bitnet_mpgemm")
+    return y, acc_out
+
+
+def bitnet_linear_host(fmt, packed, w_scale, M, K, x_host, y_host, x_dev, q_dev, scale_dev, y_dev,
+                       workspace=None, bk3=0, stream=None):
+    """Host fp32 activations in, host fp32 results out (copies queued on the stream; caller synchronises)."""
+    T = x_host.shape[0]
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().bitnet_linear_host(_fmt(fmt), _ptr(packed), float(w_scale), M, K, bk3, _ptr(x_host), T,
+                                    _ptr(y_host), _ptr(x_dev), _ptr(q_dev), _ptr(scale_dev), _ptr(y_dev),
+                                    _ptr(workspace), ws_bytes, _stream(stream)), "bitnet_linear_host")

@@ -1,0 +1,191 @@
+// C ABI of libbitnet_b200.so: argument validation and dispatch.  Every step of the path runs in the
+// kernels of the sibling files; nothing here computes.
+#include <mutex>
+
+#include "common.cuh"
+
+namespace bitnet {
+
+static thread_local int g_last_cuda_error = 0;
+
+int note_cuda_error(cudaError_t e) {
+  g_last_cuda_error = (int)e;
+  return BITNET_ERR_CUDA;
+}
+
+const DevInfo& dev_info() {
+  static DevInfo info[64];
+  static bool have[64] = {false};
+  static std::mutex mu;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  dev &= 63;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!have[dev]) {
+    cudaDeviceGetAttribute(&info[dev].sm_count, cudaDevAttrMultiProcessorCount, dev);
+    cudaDeviceGetAttribute(&info[dev].max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    have[dev] = true;
+  }
+  return info[dev];
+}
+
+}  // namespace bitnet
+
+using namespace bitnet;
+
+extern "C" {
+
+const char* bitnet_status_string(int status) {
+  switch (status) {
+    case BITNET_OK: return "ok";
+    case BITNET_ERR_INVALID_ARG: return "invalid argument (null or misaligned pointer, bad enum or size)";
+    case BITNET_ERR_UNSUPPORTED_SHAPE: return "unsupported shape for this weight format";
+    case BITNET_ERR_WORKSPACE: return "workspace missing or too small";
+    case BITNET_ERR_BAD_WEIGHT: return "weight outside {-1,0,+1} or invalid packed code";
+    case BITNET_ERR_CUDA: return "CUDA call failed (see bitnet_last_cuda_error)";
+    case BITNET_ERR_TIMEOUT: return "bounded device-side wait gave up";
+    default: return "unknown status";
+  }
+}
+
+int bitnet_last_cuda_error(void) { return g_last_cuda_error; }
+
+int bitnet_quant_act(const float* x, int64_t T, int64_t K, int per_tensor, int8_t* q, float* act_scale,
+                     int32_t* act_sum, void* stream) {
+  if (!x || !q || !act_scale || T < 1 || K < 1 || T > 0x7fffffff) return BITNET_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(q) || (reinterpret_cast<uintptr_t>(act_scale) & 3u)) return BITNET_ERR_INVALID_ARG;
+  return launch_quant_act(x, T, K, per_tensor, q, act_scale, act_sum, (cudaStream_t)stream);
+}
+
+size_t bitnet_i2s_packed_bytes(int64_t M, int64_t K) {
+  if (M < 1 || K < 1 || (K % 64) != 0) return 0;
+  return (size_t)M * (size_t)ceil_div(K, 128) * 32;
+}
+
+static int i2s_shape(int64_t M, int64_t K) {
+  if (M < 1 || K < 1 || M > 0x7fffffff) return BITNET_ERR_INVALID_ARG;
+  if ((K % 64) != 0) return BITNET_ERR_UNSUPPORTED_SHAPE;
+  return BITNET_OK;
+}
+
+int bitnet_pack_i2s(const int8_t* w, int64_t M, int64_t K, void* packed, size_t packed_bytes, int* dev_status,
+                    void* stream) {
+  if (!w || !packed || !aligned16(packed)) return BITNET_ERR_INVALID_ARG;
+  int rc = i2s_shape(M, K);
+  if (rc) return rc;
+  if (packed_bytes < bitnet_i2s_packed_bytes(M, K)) return BITNET_ERR_INVALID_ARG;
+  return launch_pack_i2s(w, M, K, (uint8_t*)packed, dev_status, (cudaStream_t)stream);
+}
+
+int bitnet_unpack_i2s(const void* packed, int64_t M, int64_t K, int8_t* w, int* dev_status, void* stream) {
+  if (!w || !packed || !aligned16(packed)) return BITNET_ERR_INVALID_ARG;
+  int rc = i2s_shape(M, K);
+  if (rc) return rc;
+  return launch_unpack_i2s((const uint8_t*)packed, M, K, w, dev_status, (cudaStream_t)stream);
+}
+
+static int tl_shape(int fmt, int64_t M, int64_t K, int bk3, TlGeom* g) {
+  if (fmt != BITNET_FMT_TL1 && fmt != BITNET_FMT_TL2) return BITNET_ERR_INVALID_ARG;
+  if (M < 1 || K < 1 || M > 0x7fffffff) return BITNET_ERR_INVALID_ARG;
+  if (!tl_geom(fmt, M, K, bk3, g)) return BITNET_ERR_UNSUPPORTED_SHAPE;
+  return BITNET_OK;
+}
+
+size_t bitnet_tl_packed_bytes(bitnet_fmt_t fmt, int64_t M, int64_t K, int bk3) {
+  TlGeom g;
+  if (tl_shape(fmt, M, K, bk3, &g)) return 0;
+  return (size_t)(M / 32) * (size_t)g.block_bytes;
+}
+
+int bitnet_pack_tl(bitnet_fmt_t fmt, const int8_t* w, int64_t M, int64_t K, int bk3, void* packed,
+                   size_t packed_bytes, int* dev_status, void* stream) {
+  if (!w || !packed || !aligned16(packed)) return BITNET_ERR_INVALID_ARG;
+  TlGeom g;
+  int rc = tl_shape(fmt, M, K, bk3, &g);
+  if (rc) return rc;
+  if (packed_bytes < (size_t)(M / 32) * (size_t)g.block_bytes) return BITNET_ERR_INVALID_ARG;
+  return launch_pack_tl(fmt, w, M, K, g, (uint8_t*)packed, dev_status, (cudaStream_t)stream);
+}
+
+int bitnet_unpack_tl(bitnet_fmt_t fmt, const void* packed, int64_t M, int64_t K, int bk3, int8_t* w,
+                     int* dev_status, void* stream) {
+  if (!w || !packed || !aligned16(packed)) return BITNET_ERR_INVALID_ARG;
+  TlGeom g;
+  int rc = tl_shape(fmt, M, K, bk3, &g);
+  if (rc) return rc;
+  return launch_unpack_tl(fmt, (const uint8_t*)packed, M, K, g, w, dev_status, (cudaStream_t)stream);
+}
+
+int64_t bitnet_tl_num_groups(bitnet_fmt_t fmt, int64_t K, int bk3) {
+  TlGeom g;
+  if (tl_shape(fmt, 32, K, bk3, &g)) return -1;
+  return (g.tiles3 + g.tiles2) * 32;
+}
+
+int bitnet_tl_build_lut_debug(bitnet_fmt_t fmt, const int8_t* q_row, int64_t K, int bk3, int16_t* lut,
+                              void* stream) {
+  if (!q_row || !lut) return BITNET_ERR_INVALID_ARG;
+  TlGeom g;
+  int rc = tl_shape(fmt, 32, K, bk3, &g);
+  if (rc) return rc;
+  return launch_tl_build_lut(fmt, q_row, K, g, lut, (cudaStream_t)stream);
+}
+
+size_t bitnet_mpgemm_workspace_bytes(bitnet_fmt_t fmt, int64_t T, int64_t M, int64_t K) {
+  if (T < 1 || M < 1 || K < 1) return 0;
+  if (fmt == BITNET_FMT_I2S) return (T > 8) ? 0 : gemv_i2s_workspace_bytes(T, M, K);
+  return gemv_tl_workspace_bytes(fmt, T, M, K);
+}
+
+int bitnet_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+  if (workspace_bytes == 0) return BITNET_OK;
+  if (!workspace) return BITNET_ERR_INVALID_ARG;
+  cudaError_t e = cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)stream);
+  return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
+}
+
+int bitnet_mpgemm(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M, int64_t K, int bk3,
+                  const int8_t* q, const float* act_scale, int64_t T, float* y, int32_t* acc_out,
+                  void* workspace, size_t workspace_bytes, void* stream) {
+  if (!packed || !q || !act_scale || !y || T < 1) return BITNET_ERR_INVALID_ARG;
+  if (!aligned16(packed) || !aligned16(q) || !aligned16(y) || (acc_out && !aligned16(acc_out)) ||
+      (workspace && !aligned16(workspace)))
+    return BITNET_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (fmt == BITNET_FMT_I2S) {
+    int rc = i2s_shape(M, K);
+    if (rc) return rc;
+    if (T > 8) return launch_gemm_i2s_prefill((const uint8_t*)packed, w_scale, M, K, q, act_scale, T, y, acc_out, st);
+    return launch_gemv_i2s((const uint8_t*)packed, w_scale, M, K, q, act_scale, (int)T, y, acc_out, workspace,
+                           workspace_bytes, st);
+  }
+  TlGeom g;
+  int rc = tl_shape(fmt, M, K, bk3, &g);
+  if (rc) return rc;
+  for (int64_t t0 = 0; t0 < T; t0 += 8) {
+    const int nt = (int)((T - t0 < 8) ? (T - t0) : 8);
+    rc = launch_gemv_tl(fmt, (const uint8_t*)packed, w_scale, M, K, g, q + t0 * K, act_scale + t0, nt,
+                        y + t0 * M, acc_out ? acc_out + t0 * M : nullptr, workspace, workspace_bytes, st);
+    if (rc) return rc;
+  }
+  return BITNET_OK;
+}
+
+int bitnet_linear_host(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M, int64_t K, int bk3,
+                       const float* x_host, int64_t T, float* y_host, float* x_dev, int8_t* q_dev,
+                       float* scale_dev, float* y_dev, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!x_host || !y_host || !x_dev || !q_dev || !scale_dev || !y_dev || T < 1 || M < 1 || K < 1)
+    return BITNET_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = cudaMemcpyAsync(x_dev, x_host, (size_t)T * K * sizeof(float), cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return note_cuda_error(e);
+  int rc = bitnet_quant_act(x_dev, T, K, 0, q_dev, scale_dev, nullptr, stream);
+  if (rc) return rc;
+  rc = bitnet_mpgemm(fmt, packed, w_scale, M, K, bk3, q_dev, scale_dev, T, y_dev, nullptr, workspace,
+                     workspace_bytes, stream);
+  if (rc) return rc;
+  e = cudaMemcpyAsync(y_host, y_dev, (size_t)T * M * sizeof(float), cudaMemcpyDeviceToHost, st);
+  return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
+}
+
+}  // extern "C"

@@ -1,0 +1,263 @@
+// TL1 / TL2 mpGEMV for decode (1..8 tokens): element-wise LUT mpGEMM, Alg. 2 with the tables of
+// Alg. 3 (pairs, 9 sums) and Alg. 4 (triples, 14 sums after mirror consolidation); Eq. 3:
+//     acc = sum over groups of Lookup(LUT_group, index), the sign bit of a triple negating the value.
+//
+// A CTA owns a K-slice (a run of 32-group tiles).  Phase 1 ("PreCompute"): it stages the slice of the
+// token's int8 activations in shared memory and builds, for every group, a 16-slot table of partial
+// sums in shared memory -- slot i of a triple table is d0*a0 + d1*a1 + d2*a2 with (d0,d1,d2) the
+// balanced-ternary digits of i, slot i of a pair table is (i/3-1)*a0 + (i%3-1)*a1.  Sums stay exact
+// (|sum| <= 384), as in the lossless TL*_1 variants.  Two tokens share one 32-bit slot as
+// hi*65536 + lo: integer add and negate act on both halves at once, so a lookup serves two tokens.
+// Phase 2: lanes are rows.  A warp takes one tile of a 32-row block: every lane reads its row's 16
+// index bytes (+ 4 sign bytes) with one coalesced request per plane and resolves its 32 nibbles
+// against the SAME group table -- 16 slots in 16 distinct banks, so the lookups never conflict.  The
+// conditional negate is (v ^ m) with m = 0 / -1 from the sign bit, the "+1" of two's complement
+// negation being added once per tile as popcount(sign word).  Warps of a CTA cover different tiles;
+// their per-row sums meet in shared memory, and K-slices of different CTAs meet in an int32
+// workspace by atomicAdd, finalised by whichever slice arrives last (no waiting).
+#include "common.cuh"
+
+namespace bitnet {
+namespace {
+
+constexpr int WARPS = 8;
+constexpr int THREADS = WARPS * 32;
+constexpr int MAX_SLICE_TILES = 48;  // 2 KB of tables per tile
+
+struct TlArgs {
+  const uint8_t* packed;
+  TlGeom g;
+  int M;
+  int64_t K;
+  const int8_t* q;  // first token of the pass
+  const float* act_scale;
+  float w_scale;
+  int nt;           // tokens in this pass (1 or 2)
+  float* y;
+  int32_t* acc_out;
+  int32_t* ws_acc;
+  unsigned* ws_ticket;
+  int nslices;
+  int tiles_per_slice;
+};
+
+// Entry i of a group's table for activations (a0,a1,a2); pair tables pass a2 = 0 and is3 = false.
+__device__ __forceinline__ int lut_entry(bool is3, int i, int a0, int a1, int a2) {
+  if (is3) {
+    if (i > 13) return 0;
+    const int d0 = (i + 4) / 9;
+    const int rem = i - 9 * d0;
+    const int d1 = (rem + 7) / 3 - 2;
+    const int d2 = rem - 3 * d1;
+    return d0 * a0 + d1 * a1 + d2 * a2;
+  }
+  if (i > 8) return 0;
+  return (i / 3 - 1) * a0 + (i % 3 - 1) * a1;
+}
+
+// Activations of tile `tile` (global tile number), group grp, token row qrow (global memory).
+__device__ __forceinline__ void group_acts(const TlGeom& g, int64_t K, const int8_t* qrow, int tile, int grp,
+                                           bool* is3, int* a0, int* a1, int* a2) {
+  if (tile < g.tiles3) {
+    const int64_t k = (int64_t)tile * 96 + 3 * grp;
+    *is3 = true;
+    *a0 = qrow[k];
+    *a1 = qrow[k + 1];
+    *a2 = qrow[k + 2];
+  } else {
+    const int64_t k = g.three_k + (int64_t)(tile - g.tiles3) * 64 + 2 * grp;
+    *is3 = false;
+    *a2 = 0;
+    if (k < K) {
+      *a0 = qrow[k];
+      *a1 = qrow[k + 1];
+    } else {
+      *a0 = 0;
+      *a1 = 0;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(THREADS, 2) gemv_tl_kernel(const TlArgs a) {
+  extern __shared__ __align__(16) int smem[];
+  int* tab = smem;                                   // [tiles_per_slice][32][16]
+  int* red = smem + a.tiles_per_slice * 512;         // [WARPS][32][2]
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int slice = blockIdx.y;
+  const int tiles_total = (int)(a.g.tiles3 + a.g.tiles2);
+  const int tile0 = slice * a.tiles_per_slice;
+  const int ntiles = min(a.tiles_per_slice, tiles_total - tile0);
+
+  // ---- Phase 1: tables of this slice.  One thread per table slot; consecutive threads write
+  // consecutive words.
+  for (int e = threadIdx.x; e < ntiles * 512; e += THREADS) {
+    const int i = e & 15, grp = (e >> 4) & 31, tl = e >> 9;
+    bool is3;
+    int a0, a1, a2;
+    group_acts(a.g, a.K, a.q, tile0 + tl, grp, &is3, &a0, &a1, &a2);
+    int v = lut_entry(is3, i, a0, a1, a2);
+    if (a.nt == 2) {
+      group_acts(a.g, a.K, a.q + a.K, tile0 + tl, grp, &is3, &a0, &a1, &a2);
+      v += lut_entry(is3, i, a0, a1, a2) * 65536;
+    }
+    tab[e] = v;
+  }
+  __syncthreads();
+
+  const float sc0 = __fmul_rn(a.act_scale[0], a.w_scale);
+  const float sc1 = (a.nt == 2) ? __fmul_rn(a.act_scale[1], a.w_scale) : 0.0f;
+
+  // ---- Phase 2: lookups.
+  for (int rb = blockIdx.x; rb < a.M / 32; rb += gridDim.x) {
+    const uint8_t* blk = a.packed + (int64_t)rb * a.g.block_bytes;
+    int lo = 0, hi = 0;
+    for (int tl = warp; tl < ntiles; tl += WARPS) {
+      const int tile = tile0 + tl;
+      const bool is3 = tile < a.g.tiles3;
+      const uint8_t* tp = is3 ? blk + (int64_t)tile * 640
+                              : blk + a.g.tiles3 * 640 + (int64_t)(tile - a.g.tiles3) * 512;
+      const uint4 iw = __ldg(reinterpret_cast<const uint4*>(tp) + lane);
+      const unsigned sg = is3 ? __ldg(reinterpret_cast<const unsigned*>(tp + 512) + lane) : 0u;
+      const unsigned words[4] = {iw.x, iw.y, iw.z, iw.w};
+      const int* tt = tab + tl * 512;
+      int s = __popc(sg);  // the +1 of every two's-complement negation below, for both halves at once
+#pragma unroll
+      for (int w4 = 0; w4 < 4; ++w4) {
+#pragma unroll
+        for (int n = 0; n < 8; ++n) {
+          const int grp = w4 * 8 + n;
+          const int idx = (words[w4] >> (4 * n)) & 15;
+          const int v = tt[grp * 16 + idx];
+          const int m = -(int)((sg >> grp) & 1u);
+          s += v ^ m;
+        }
+      }
+      // split the packed pair: s = H * 65536 + L with |L| < 32768
+      const int l16 = (int)(short)(s & 0xFFFF);
+      lo += l16;
+      hi += (s - l16) >> 16;
+    }
+    red[(warp * 32 + lane) * 2 + 0] = lo;
+    red[(warp * 32 + lane) * 2 + 1] = hi;
+    __syncthreads();
+    if (warp == 0) {
+      int tot[2] = {0, 0};
+#pragma unroll
+      for (int w = 0; w < WARPS; ++w) {
+        tot[0] += red[(w * 32 + lane) * 2 + 0];
+        tot[1] += red[(w * 32 + lane) * 2 + 1];
+      }
+      const int row = rb * 32 + lane;
+      if (a.nslices == 1) {
+        a.y[row] = __fmul_rn((float)tot[0], sc0);
+        if (a.acc_out) a.acc_out[row] = tot[0];
+        if (a.nt == 2) {
+          a.y[a.M + row] = __fmul_rn((float)tot[1], sc1);
+          if (a.acc_out) a.acc_out[a.M + row] = tot[1];
+        }
+      } else {
+        atomicAdd(a.ws_acc + row, tot[0]);
+        if (a.nt == 2) atomicAdd(a.ws_acc + a.M + row, tot[1]);
+        __threadfence();
+        const unsigned old = atomicAdd(a.ws_ticket + row, 1u);
+        if (old == (unsigned)(a.nslices - 1)) {
+          __threadfence();
+          const int v0 = atomicExch(a.ws_acc + row, 0);
+          a.y[row] = __fmul_rn((float)v0, sc0);
+          if (a.acc_out) a.acc_out[row] = v0;
+          if (a.nt == 2) {
+            const int v1 = atomicExch(a.ws_acc + a.M + row, 0);
+            a.y[a.M + row] = __fmul_rn((float)v1, sc1);
+            if (a.acc_out) a.acc_out[a.M + row] = v1;
+          }
+          atomicExch(a.ws_ticket + row, 0u);
+        }
+      }
+    }
+    __syncthreads();
+  }
+}
+
+__global__ void tl_build_lut_kernel(const int8_t* q_row, int64_t K, TlGeom g, int16_t* lut, int64_t nslots) {
+  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= nslots) return;
+  const int i = (int)(e & 15), grp = (int)((e >> 4) & 31);
+  const int tile = (int)(e >> 9);
+  bool is3;
+  int a0, a1, a2;
+  group_acts(g, K, q_row, tile, grp, &is3, &a0, &a1, &a2);
+  lut[e] = (int16_t)lut_entry(is3, i, a0, a1, a2);
+}
+
+inline void slicing(const TlGeom& g, int* nslices, int* tiles_per_slice) {
+  const int tiles = (int)(g.tiles3 + g.tiles2);
+  *nslices = (tiles + MAX_SLICE_TILES - 1) / MAX_SLICE_TILES;
+  *tiles_per_slice = (tiles + *nslices - 1) / *nslices;
+}
+
+}  // namespace
+
+size_t gemv_tl_workspace_bytes(int fmt, int64_t T, int64_t M, int64_t K) {
+  TlGeom g;
+  if (!tl_geom(fmt, M, K, 0, &g)) return 0;
+  int ns, tps;
+  slicing(g, &ns, &tps);
+  if (ns == 1) return 0;
+  const int64_t Tc = T > 8 ? 8 : T;
+  return (size_t)(Tc * M * 4 + M * 4);
+}
+
+int launch_gemv_tl(int fmt, const uint8_t* packed, float w_scale, int64_t M, int64_t K, const TlGeom& g,
+                   const int8_t* q, const float* act_scale, int T, float* y, int32_t* acc_out, void* ws,
+                   size_t ws_bytes, cudaStream_t st) {
+  (void)fmt;
+  TlArgs a;
+  a.packed = packed;
+  a.g = g;
+  a.M = (int)M;
+  a.K = K;
+  a.w_scale = w_scale;
+  slicing(g, &a.nslices, &a.tiles_per_slice);
+  if (a.nslices > 1) {
+    if (!ws || ws_bytes < (size_t)((int64_t)T * M * 4 + M * 4)) return BITNET_ERR_WORKSPACE;
+    a.ws_ticket = reinterpret_cast<unsigned*>(reinterpret_cast<int32_t*>(ws) + (int64_t)T * M);
+  } else {
+    a.ws_ticket = nullptr;
+  }
+  const size_t smem = (size_t)a.tiles_per_slice * 2048 + WARPS * 32 * 2 * sizeof(int);
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (!attr_set[dev & 63]) {
+    cudaError_t e = cudaFuncSetAttribute(gemv_tl_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         MAX_SLICE_TILES * 2048 + WARPS * 32 * 2 * (int)sizeof(int));
+    if (e != cudaSuccess) return note_cuda_error(e);
+    attr_set[dev & 63] = true;
+  }
+  const int sms = dev_info().sm_count;
+  int gx = (2 * sms + a.nslices - 1) / a.nslices;
+  if (gx > (int)(M / 32)) gx = (int)(M / 32);
+  for (int t0 = 0; t0 < T; t0 += 2) {
+    a.q = q + (int64_t)t0 * K;
+    a.act_scale = act_scale + t0;
+    a.nt = (T - t0 >= 2) ? 2 : 1;
+    a.y = y + (int64_t)t0 * M;
+    a.acc_out = acc_out ? acc_out + (int64_t)t0 * M : nullptr;
+    a.ws_acc = (a.nslices > 1) ? reinterpret_cast<int32_t*>(ws) + (int64_t)t0 * M : nullptr;
+    gemv_tl_kernel<<<dim3((unsigned)gx, (unsigned)a.nslices), THREADS, smem, st>>>(a);
+    int rc = check_launch();
+    if (rc != BITNET_OK) return rc;
+  }
+  return BITNET_OK;
+}
+
+int launch_tl_build_lut(int fmt, const int8_t* q_row, int64_t K, const TlGeom& g, int16_t* lut,
+                        cudaStream_t st) {
+  (void)fmt;
+  const int64_t nslots = (g.tiles3 + g.tiles2) * 512;
+  tl_build_lut_kernel<<<(unsigned)ceil_div(nslots, 256), 256, 0, st>>>(q_row, K, g, lut, nslots);
+  return check_launch();
+}
+
+}  // namespace bitnet

@@ -1,0 +1,185 @@
+// Weight packers (offline step of the path) and their inverses (test hooks).
+//   I2_S : Table 1 / Sec. 3.2.2 -- code w+1 in two bits.
+//   TL1  : Table 4 / Alg. 3 PreprocessWeights -- pair -> 3(w0+1)+(w1+1).
+//   TL2  : Table 5 / Alg. 4 PreprocessWeights -- triple -> (|v|, [v<0]), v = 9w0+3w1+w2, index and
+//          sign kept in separate planes (signed-unsigned weight splitting, Sec. 3.1.2).
+// The byte layouts are documented in bitnet_b200.h.
+#include "common.cuh"
+
+namespace bitnet {
+namespace {
+
+__device__ __forceinline__ bool ternary(int w) { return w >= -1 && w <= 1; }
+
+// One thread per 32-bit packed word = 16 consecutive weights of one row.
+__global__ void pack_i2s_kernel(const int8_t* __restrict__ w, int64_t M, int64_t K, int64_t row_words,
+                                uint32_t* __restrict__ packed, int* dev_status) {
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= M * row_words) return;
+  const int64_t m = gid / row_words, j = gid % row_words;
+  const int8_t* wr = w + m * K;
+  uint32_t word = 0;
+  bool bad = false;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const int64_t k = 16 * j + i;
+    const int wk = (k < K) ? (int)wr[k] : 0;
+    bad |= !ternary(wk);
+    const int s = i >> 2, b = i & 3;  // k = 16j + 4s + b
+    word |= (uint32_t)((wk + 1) & 3) << (8 * b + 2 * s);
+  }
+  packed[gid] = word;
+  if (bad && dev_status) atomicExch(dev_status, BITNET_ERR_BAD_WEIGHT);
+}
+
+__global__ void unpack_i2s_kernel(const uint32_t* __restrict__ packed, int64_t M, int64_t K,
+                                  int64_t row_words, int8_t* __restrict__ w, int* dev_status) {
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= M * row_words) return;
+  const int64_t m = gid / row_words, j = gid % row_words;
+  const uint32_t word = packed[gid];
+  bool bad = false;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const int64_t k = 16 * j + i;
+    const int s = i >> 2, b = i & 3;
+    const int code = (word >> (8 * b + 2 * s)) & 3;
+    bad |= (code == 3);
+    if (k < K) w[m * K + k] = (int8_t)(code - 1);
+  }
+  if (bad && dev_status) atomicExch(dev_status, BITNET_ERR_BAD_WEIGHT);
+}
+
+// One thread per (row, tile): emits the row's 16 index bytes (and the sign word of a TL2 tile).
+__global__ void pack_tl_kernel(const int8_t* __restrict__ w, int64_t M, int64_t K, TlGeom g,
+                               uint8_t* __restrict__ packed, int* dev_status) {
+  const int64_t tiles = g.tiles3 + g.tiles2;
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= M * tiles) return;
+  // consecutive threads = consecutive rows of one tile, so the 16-byte stores of a warp are contiguous
+  const int64_t r = gid % 32;
+  const int64_t tile = (gid / 32) % tiles;
+  const int64_t rb = gid / (32 * tiles);
+  const int64_t m = rb * 32 + r;
+  const int8_t* wr = w + m * K;
+  uint8_t* blk = packed + rb * g.block_bytes;
+  uint32_t idx_words[4] = {0, 0, 0, 0};
+  bool bad = false;
+  if (tile < g.tiles3) {
+    uint32_t signs = 0;
+    const int64_t k0 = tile * 96;
+    for (int grp = 0; grp < 32; ++grp) {
+      const int w0 = wr[k0 + 3 * grp], w1 = wr[k0 + 3 * grp + 1], w2 = wr[k0 + 3 * grp + 2];
+      bad |= !(ternary(w0) && ternary(w1) && ternary(w2));
+      const int v = 9 * w0 + 3 * w1 + w2;
+      const uint32_t idx = (uint32_t)abs(v) & 15u;
+      signs |= (v < 0 ? 1u : 0u) << grp;
+      idx_words[grp >> 3] |= idx << (4 * (grp & 7));
+    }
+    uint8_t* tp = blk + tile * 640;
+    *reinterpret_cast<uint4*>(tp + 16 * r) = make_uint4(idx_words[0], idx_words[1], idx_words[2], idx_words[3]);
+    *reinterpret_cast<uint32_t*>(tp + 512 + 4 * r) = signs;
+  } else {
+    const int64_t t2 = tile - g.tiles3;
+    const int64_t k0 = g.three_k + t2 * 64;
+    for (int grp = 0; grp < 32; ++grp) {
+      const int64_t k = k0 + 2 * grp;
+      uint32_t idx = 4;
+      if (k < K) {
+        const int w0 = wr[k], w1 = wr[k + 1];
+        bad |= !(ternary(w0) && ternary(w1));
+        idx = (uint32_t)(3 * (w0 + 1) + (w1 + 1)) & 15u;
+      }
+      idx_words[grp >> 3] |= idx << (4 * (grp & 7));
+    }
+    uint8_t* tp = blk + g.tiles3 * 640 + t2 * 512;
+    *reinterpret_cast<uint4*>(tp + 16 * r) = make_uint4(idx_words[0], idx_words[1], idx_words[2], idx_words[3]);
+  }
+  if (bad && dev_status) atomicExch(dev_status, BITNET_ERR_BAD_WEIGHT);
+}
+
+__global__ void unpack_tl_kernel(const uint8_t* __restrict__ packed, int64_t M, int64_t K, TlGeom g,
+                                 int8_t* __restrict__ w, int* dev_status) {
+  const int64_t tiles = g.tiles3 + g.tiles2;
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= M * tiles) return;
+  const int64_t r = gid % 32;
+  const int64_t tile = (gid / 32) % tiles;
+  const int64_t rb = gid / (32 * tiles);
+  const int64_t m = rb * 32 + r;
+  int8_t* wr = w + m * K;
+  const uint8_t* blk = packed + rb * g.block_bytes;
+  bool bad = false;
+  if (tile < g.tiles3) {
+    const uint8_t* tp = blk + tile * 640;
+    const uint4 iw = *reinterpret_cast<const uint4*>(tp + 16 * r);
+    const uint32_t words[4] = {iw.x, iw.y, iw.z, iw.w};
+    const uint32_t signs = *reinterpret_cast<const uint32_t*>(tp + 512 + 4 * r);
+    for (int grp = 0; grp < 32; ++grp) {
+      const int idx = (words[grp >> 3] >> (4 * (grp & 7))) & 15;
+      const int neg = (signs >> grp) & 1;
+      bad |= (idx > 13) || (idx == 0 && neg);
+      // digits of idx in balanced ternary: idx = 9 d0 + 3 d1 + d2, digits in {-1,0,1}
+      const int d0 = (idx + 4) / 9;                 // 0 for idx <= 4, 1 for 5..13
+      const int rem = idx - 9 * d0;                 // -4..4
+      const int d1 = (rem + 7) / 3 - 2;             // -1 for -4..-2, 0 for -1..1, 1 for 2..4
+      const int d2 = rem - 3 * d1;
+      const int sgn = neg ? -1 : 1;
+      const int64_t k = tile * 96 + 3 * grp;
+      wr[k] = (int8_t)(sgn * d0);
+      wr[k + 1] = (int8_t)(sgn * d1);
+      wr[k + 2] = (int8_t)(sgn * d2);
+    }
+  } else {
+    const int64_t t2 = tile - g.tiles3;
+    const uint8_t* tp = blk + g.tiles3 * 640 + t2 * 512;
+    const uint4 iw = *reinterpret_cast<const uint4*>(tp + 16 * r);
+    const uint32_t words[4] = {iw.x, iw.y, iw.z, iw.w};
+    for (int grp = 0; grp < 32; ++grp) {
+      const int idx = (words[grp >> 3] >> (4 * (grp & 7))) & 15;
+      const int64_t k = g.three_k + t2 * 64 + 2 * grp;
+      if (k < K) {
+        bad |= idx > 8;
+        wr[k] = (int8_t)(idx / 3 - 1);
+        wr[k + 1] = (int8_t)(idx % 3 - 1);
+      } else {
+        bad |= idx != 4;
+      }
+    }
+  }
+  if (bad && dev_status) atomicExch(dev_status, BITNET_ERR_BAD_WEIGHT);
+}
+
+inline unsigned blocks_for(int64_t n, int threads) { return (unsigned)ceil_div(n, threads); }
+
+}  // namespace
+
+int launch_pack_i2s(const int8_t* w, int64_t M, int64_t K, uint8_t* packed, int* dev_status,
+                    cudaStream_t st) {
+  const int64_t row_words = ceil_div(K, 128) * 8;
+  pack_i2s_kernel<<<blocks_for(M * row_words, 256), 256, 0, st>>>(
+      w, M, K, row_words, reinterpret_cast<uint32_t*>(packed), dev_status);
+  return check_launch();
+}
+
+int launch_unpack_i2s(const uint8_t* packed, int64_t M, int64_t K, int8_t* w, int* dev_status,
+                      cudaStream_t st) {
+  const int64_t row_words = ceil_div(K, 128) * 8;
+  unpack_i2s_kernel<<<blocks_for(M * row_words, 256), 256, 0, st>>>(
+      reinterpret_cast<const uint32_t*>(packed), M, K, row_words, w, dev_status);
+  return check_launch();
+}
+
+int launch_pack_tl(int, const int8_t* w, int64_t M, int64_t K, const TlGeom& g, uint8_t* packed,
+                   int* dev_status, cudaStream_t st) {
+  pack_tl_kernel<<<blocks_for(M * (g.tiles3 + g.tiles2), 256), 256, 0, st>>>(w, M, K, g, packed, dev_status);
+  return check_launch();
+}
+
+int launch_unpack_tl(int, const uint8_t* packed, int64_t M, int64_t K, const TlGeom& g, int8_t* w,
+                     int* dev_status, cudaStream_t st) {
+  unpack_tl_kernel<<<blocks_for(M * (g.tiles3 + g.tiles2), 256), 256, 0, st>>>(packed, M, K, g, w, dev_status);
+  return check_launch();
+}
+
+}  // namespace bitnet

@@ -1,0 +1,146 @@
+// Activation quantiser: Alg. 1 Phase 1 ("Quantization"), absmax int8 (Sec. 2.1, Sec. 3.2.2).
+//
+// One CTA per token.  Pass 1 reduces max|x| over the row (exact, order free); pass 2 re-reads the
+// row (L1/L2 resident), multiplies by s = 127/amax with a single rounded binary32 product, rounds
+// to nearest even, clamps, stores int8 and reduces the sum of the codes.  No fast-math anywhere:
+// the division, the product and the conversion are the IEEE round-to-nearest forms, so the bytes
+// match a scalar CPU evaluation of the same formula.
+#include "common.cuh"
+
+namespace bitnet {
+namespace {
+
+constexpr int QTHREADS = 512;
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__device__ __forceinline__ int quant1(float x, float s) {
+  int v = __float2int_rn(__fmul_rn(x, s));
+  return max(-128, min(127, v));
+}
+
+// amax over a [rows][K] slab starting at x; result in every thread.
+__device__ float block_amax(const float* __restrict__ x, int64_t n, float* red) {
+  float m = 0.0f;
+  const int tid = threadIdx.x;
+  if ((n & 3) == 0 && ((reinterpret_cast<uintptr_t>(x) & 15u) == 0)) {
+    const float4* x4 = reinterpret_cast<const float4*>(x);
+    for (int64_t i = tid; i < n / 4; i += blockDim.x) {
+      float4 v = x4[i];
+      m = fmaxf(m, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+    }
+  } else {
+    for (int64_t i = tid; i < n; i += blockDim.x) m = fmaxf(m, fabsf(x[i]));
+  }
+  m = warp_max(m);
+  if ((tid & 31) == 0) red[tid >> 5] = m;
+  __syncthreads();
+  if (tid < 32) {
+    float v = (tid < (blockDim.x >> 5)) ? red[tid] : 0.0f;
+    v = warp_max(v);
+    if (tid == 0) red[0] = v;
+  }
+  __syncthreads();
+  float r = red[0];
+  __syncthreads();
+  return r;
+}
+
+// per_tensor pass A: one CTA per token folds its row maximum into *amax_bits (bit pattern of a
+// non-negative float orders like the unsigned integer).
+__global__ void __launch_bounds__(QTHREADS) amax_kernel(const float* __restrict__ x, int64_t K,
+                                                        unsigned* amax_bits) {
+  __shared__ float red[32];
+  float m = block_amax(x + (int64_t)blockIdx.x * K, K, red);
+  if (threadIdx.x == 0) atomicMax(amax_bits, __float_as_uint(m));
+}
+
+__global__ void __launch_bounds__(QTHREADS)
+quant_act_kernel(const float* __restrict__ x, int64_t K, int8_t* __restrict__ q, float* __restrict__ act_scale,
+                 int32_t* __restrict__ act_sum, const unsigned* __restrict__ tensor_amax_bits) {
+  __shared__ float red[32];
+  __shared__ int redi[32];
+  const int64_t t = blockIdx.x;
+  const float* xr = x + t * K;
+  int8_t* qr = q + t * K;
+  const int tid = threadIdx.x;
+
+  float amax;
+  if (tensor_amax_bits) {
+    amax = __uint_as_float(*tensor_amax_bits);
+  } else {
+    amax = block_amax(xr, K, red);
+  }
+  const float amax_c = fmaxf(amax, 1e-5f);
+  const float s = __fdiv_rn(127.0f, amax_c);
+
+  int sum = 0;
+  if ((K & 3) == 0 && ((reinterpret_cast<uintptr_t>(xr) & 15u) == 0) &&
+      ((reinterpret_cast<uintptr_t>(qr) & 3u) == 0)) {
+    const float4* x4 = reinterpret_cast<const float4*>(xr);
+    char4* q4 = reinterpret_cast<char4*>(qr);
+    for (int64_t i = tid; i < K / 4; i += blockDim.x) {
+      float4 v = x4[i];
+      int a = quant1(v.x, s), b = quant1(v.y, s), c = quant1(v.z, s), d = quant1(v.w, s);
+      sum += a + b + c + d;
+      q4[i] = make_char4((signed char)a, (signed char)b, (signed char)c, (signed char)d);
+    }
+  } else {
+    for (int64_t i = tid; i < K; i += blockDim.x) {
+      int a = quant1(xr[i], s);
+      sum += a;
+      qr[i] = (int8_t)a;
+    }
+  }
+  sum = warp_sum(sum);
+  if ((tid & 31) == 0) redi[tid >> 5] = sum;
+  __syncthreads();
+  if (tid < 32) {
+    int v = (tid < (blockDim.x >> 5)) ? redi[tid] : 0;
+    v = warp_sum(v);
+    if (tid == 0) {
+      if (act_sum) act_sum[t] = v;
+      // per-tensor mode writes the scales in a separate pass (act_scale[0] carries the maximum)
+      if (!tensor_amax_bits) act_scale[t] = __fdiv_rn(amax_c, 127.0f);
+    }
+  }
+}
+
+__global__ void fill_scale_kernel(float* act_scale, int64_t T) {
+  __shared__ float sc;
+  if (threadIdx.x == 0) {
+    float amax = __uint_as_float(*reinterpret_cast<unsigned*>(act_scale));
+    sc = __fdiv_rn(fmaxf(amax, 1e-5f), 127.0f);
+  }
+  __syncthreads();
+  for (int64_t i = threadIdx.x; i < T; i += blockDim.x) act_scale[i] = sc;
+}
+
+}  // namespace
+
+int launch_quant_act(const float* x, int64_t T, int64_t K, int per_tensor, int8_t* q, float* act_scale,
+                     int32_t* act_sum, cudaStream_t st) {
+  if (per_tensor && T > 1) {
+    // act_scale[0] doubles as the running maximum until the last pass overwrites every entry
+    cudaError_t e = cudaMemsetAsync(act_scale, 0, sizeof(float), st);
+    if (e != cudaSuccess) return note_cuda_error(e);
+    amax_kernel<<<(unsigned)T, QTHREADS, 0, st>>>(x, K, reinterpret_cast<unsigned*>(act_scale));
+    quant_act_kernel<<<(unsigned)T, QTHREADS, 0, st>>>(x, K, q, act_scale, act_sum,
+                                                       reinterpret_cast<const unsigned*>(act_scale));
+    fill_scale_kernel<<<1, 256, 0, st>>>(act_scale, T);
+  } else {
+    quant_act_kernel<<<(unsigned)T, QTHREADS, 0, st>>>(x, K, q, act_scale, act_sum, nullptr);
+  }
+  return check_launch();
+}
+
+}  // namespace bitnet

@@ -1,0 +1,57 @@
+"""Shared helpers of the GPU parity tests: run the CUDA path and the oracle on the same seeded inputs."""
+import numpy as np
+import torch
+
+import oracle
+import paper_2502_11880_b200 as bn
+
+REL_TOL = 1e-6   # fp32 outputs against the oracle's float64 product (two fp32 roundings <= 2^-23)
+
+
+def dev(a):
+    return torch.as_tensor(a).cuda()
+
+
+def npy(t):
+    return t.detach().cpu().numpy()
+
+
+def check_y(y_gpu, acc_ref, act_scale_ref, w_scale):
+    """|y - y_ref| <= 1e-6 |y_ref| element-wise, and y == 0 exactly where the accumulator is 0."""
+    y_ref = oracle.dequant(acc_ref, act_scale_ref, w_scale)
+    y = npy(y_gpu).astype(np.float64)
+    assert y.shape == y_ref.shape
+    err = np.abs(y - y_ref)
+    assert np.all(err <= REL_TOL * np.abs(y_ref)), float((err / np.maximum(np.abs(y_ref), 1e-300)).max())
+    assert np.all(y[acc_ref == 0] == 0.0)
+
+
+def oracle_pack(fmt, w_np, bk3=0):
+    return oracle.pack_i2s(w_np) if fmt == "i2s" else oracle.pack_tl(fmt, w_np, bk3)
+
+
+def run_linear(fmt, w_t, x_t, bk3=0, workspace=None, w_scale=None):
+    """Full path on the GPU: quantise, pack, mpgemm.  Returns dict of device tensors."""
+    M, K = w_t.shape
+    wd, xd = w_t.cuda(), x_t.cuda()
+    q, sc, sm = bn.bitnet_quant_act(xd)
+    blob = bn.pack(fmt, wd, bk3)
+    ws = bn.synth.absmean_scale(w_t) if w_scale is None else w_scale
+    y, acc = bn.bitnet_mpgemm(fmt, blob, ws, M, K, q, sc, bk3=bk3, want_acc=True, workspace=workspace)
+    torch.cuda.synchronize()
+    return dict(q=q, act_scale=sc, act_sum=sm, blob=blob, y=y, acc=acc, w_scale=ws)
+
+
+def check_linear(fmt, w_t, x_t, bk3=0, rows=None):
+    """Element-by-element parity of one linear layer against the oracle (all rows, or a sample)."""
+    out = run_linear(fmt, w_t, x_t, bk3)
+    w_np, x_np = w_t.numpy(), x_t.numpy()
+    q_ref, sc_ref, sm_ref = oracle.quant_act(x_np)
+    assert np.array_equal(npy(out["q"]), q_ref)
+    assert np.array_equal(npy(out["act_scale"]).view(np.uint32), sc_ref.view(np.uint32))
+    assert np.array_equal(npy(out["act_sum"]), sm_ref)
+    assert np.array_equal(npy(out["blob"]), oracle_pack(fmt, w_np, bk3))
+    acc_ref = oracle.mpgemm_def(q_ref, w_np)
+    assert np.array_equal(npy(out["acc"]), acc_ref)
+    check_y(out["y"], acc_ref, sc_ref, out["w_scale"])
+    return out

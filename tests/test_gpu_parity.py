@@ -1,0 +1,208 @@
+"""GPU parity: every step of the CUDA path against the CPU oracle, through the C ABI, on the same
+seeded inputs.  Integers, bytes and scale bit patterns must be identical; fp32 outputs within 1e-6
+relative."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2502_11880_b200 as bn
+from paper_2502_11880_b200 import synth
+
+from helpers import check_linear, check_y, dev, npy, oracle_pack, run_linear
+
+pytestmark = pytest.mark.gpu
+
+
+def tern(seed, M, K, p0=1 / 3, pp=1 / 3):
+    return synth.ternary(seed, 99, M, K, p0, pp)
+
+
+# ----------------------------------------------------------------------------- quantiser
+@pytest.mark.parametrize("T,K", [(1, 1), (1, 7), (3, 64), (2, 1536), (1, 28672), (8, 4096), (5, 1001), (64, 333)])
+def test_quant_bit_exact(T, K):
+    x = synth.normal(11, T * 1000 + K % 997, T, K)
+    q, sc, sm = bn.bitnet_quant_act(x.cuda())
+    q_ref, sc_ref, sm_ref = oracle.quant_act(x.numpy())
+    assert np.array_equal(npy(q), q_ref)
+    assert np.array_equal(npy(sc).view(np.uint32), sc_ref.view(np.uint32))
+    assert np.array_equal(npy(sm), sm_ref)
+
+
+def test_quant_ties_zero_rows_outliers_per_tensor():
+    x = torch.zeros(4, 128)
+    x[0, :9] = torch.tensor([127.0, 0.5, 1.5, 2.5, -0.5, -1.5, 126.5, -2.5, 3.5])
+    x[2] = synth.add_outliers(synth.normal(1, 2, 1, 128), 1, 2, 0.02)[0]
+    x[3] = 1e-7 * synth.normal(1, 3, 1, 128)[0]         # below the 1e-5 floor
+    for per_tensor in (False, True):
+        q, sc, sm = bn.bitnet_quant_act(x.cuda(), per_tensor=per_tensor)
+        q_ref, sc_ref, sm_ref = oracle.quant_act(x.numpy(), per_tensor=per_tensor)
+        assert np.array_equal(npy(q), q_ref)
+        assert np.array_equal(npy(sc).view(np.uint32), sc_ref.view(np.uint32))
+        assert np.array_equal(npy(sm), sm_ref)
+    assert npy(q)[1].any() == False  # noqa: E712  (all-zero row stays zero)
+
+
+# ----------------------------------------------------------------------------- packers
+@pytest.mark.parametrize("M,K", [(1, 64), (5, 128), (33, 192), (100, 8640), (7, 1536)])
+def test_pack_i2s_bytes_and_round_trip(M, K):
+    w = tern(3, M, K)
+    blob = bn.bitnet_pack_i2s(w.cuda())
+    assert np.array_equal(npy(blob), oracle.pack_i2s(w.numpy()))
+    assert torch.equal(bn.bitnet_unpack_i2s(blob, M, K).cpu(), w)
+    # the GPU inverse also decodes the oracle's blob
+    assert torch.equal(bn.bitnet_unpack_i2s(dev(oracle.pack_i2s(w.numpy())), M, K).cpu(), w)
+
+
+@pytest.mark.parametrize("fmt,M,K,bk3", [("tl1", 32, 2, 0), ("tl1", 64, 130, 0), ("tl2", 32, 96, 0),
+                                         ("tl2", 96, 3200, 0), ("tl2", 64, 8640, 0), ("tl2", 32, 4096, 0),
+                                         ("tl2", 64, 1000, 192), ("tl2", 32, 34, 0)])
+def test_pack_tl_bytes_and_round_trip(fmt, M, K, bk3):
+    w = tern(4, M, K, 0.4, 0.3)
+    blob = bn.bitnet_pack_tl(fmt, w.cuda(), bk3)
+    assert np.array_equal(npy(blob), oracle.pack_tl(fmt, w.numpy(), bk3))
+    assert torch.equal(bn.bitnet_unpack_tl(fmt, blob, M, K, bk3).cpu(), w)
+
+
+def test_packers_flag_non_ternary_input():
+    w = tern(5, 32, 192)
+    w[3, 17] = 2
+    for f in (lambda: bn.bitnet_pack_i2s(w.cuda()), lambda: bn.bitnet_pack_tl("tl2", w.cuda()),
+              lambda: bn.bitnet_pack_tl("tl1", w.cuda())):
+        with pytest.raises(bn.BitnetError, match="weight"):
+            f()
+
+
+@pytest.mark.parametrize("fmt,K", [("tl2", 96 * 3 + 64), ("tl2", 3200), ("tl1", 130)])
+def test_tl_tables_match_precompute(fmt, K):
+    q = torch.randint(-127, 128, (K,), dtype=torch.int8, generator=torch.Generator().manual_seed(K))
+    lut = bn.bitnet_tl_build_lut_debug(fmt, q.cuda())
+    assert np.array_equal(npy(lut), oracle.tl_build_lut(fmt, q.numpy()))
+
+
+# ----------------------------------------------------------------------------- mpGEMV, small and ragged shapes
+SHAPES = [(32, 64), (64, 128), (96, 3200), (160, 8640), (32, 2048 * 5 + 64), (224, 1536), (32, 4096 + 2048)]
+
+
+@pytest.mark.parametrize("fmt", ["i2s", "tl1", "tl2"])
+@pytest.mark.parametrize("T", [1, 2, 3, 5, 8])
+def test_mpgemv_parity(fmt, T):
+    for i, (M, K) in enumerate(SHAPES):
+        w = tern(20 + i, M, K, 0.4, 0.3)
+        x = synth.normal(21, i * 16 + T, T, K)
+        check_linear(fmt, w, x)
+
+
+def test_i2s_rows_not_multiple_of_anything():
+    for M in (1, 7, 9, 300):
+        check_linear("i2s", tern(30, M, 256), synth.normal(30, M, 2, 256))
+
+
+@pytest.mark.parametrize("fmt", ["i2s", "tl1", "tl2"])
+def test_constant_weights_and_workspace_reuse(fmt):
+    M, K, T = 64, 28672, 2            # long K: several K-slices meet in the workspace
+    x = synth.normal(31, 1, T, K)
+    q_ref, sc_ref, sm_ref = oracle.quant_act(x.numpy())
+    ws = bn.new_workspace(fmt, T, M, K)
+    assert ws is not None
+    for val in (0, 1, -1, 1):          # the same workspace serves every call: it must come back clean
+        w = torch.full((M, K), val, dtype=torch.int8)
+        out = run_linear(fmt, w, x, workspace=ws, w_scale=0.5)
+        expect = np.repeat((val * sm_ref.astype(np.int64))[:, None], M, axis=1).astype(np.int32)
+        assert np.array_equal(npy(out["acc"]), expect)
+        check_y(out["y"], expect, sc_ref, 0.5)
+    assert not npy(ws).any()
+
+
+def test_formats_agree_on_accumulators():
+    M, K, T = 128, 8192, 3
+    w, x = tern(32, M, K), synth.normal(32, 1, T, K)
+    accs = [npy(run_linear(f, w, x)["acc"]) for f in ("i2s", "tl1", "tl2")]
+    assert np.array_equal(accs[0], accs[1]) and np.array_equal(accs[0], accs[2])
+
+
+def test_many_tokens_tl_and_i2s():
+    M, K, T = 64, 1536, 21            # more than 8 tokens
+    w, x = tern(33, M, K), synth.normal(33, 1, T, K)
+    for fmt in ("tl2", "i2s"):
+        check_linear(fmt, w, x)
+
+
+# ----------------------------------------------------------------------------- the five workloads
+def test_workload_gemv1536_all_formats():
+    wl = synth.CONFIGS["gemv1536"]
+    w, x = wl.weights(0, 0), wl.activations(0, 0, 1)
+    for fmt in wl.formats:
+        check_linear(fmt, w, x)
+
+
+@pytest.mark.parametrize("name", ["layer3b", "layer8b"])
+def test_workload_layers_full_parity(name):
+    wl = synth.CONFIGS[name]
+    for j, lin in enumerate(wl.linears):
+        w = wl.weights(0, j)
+        for T in wl.tokens:
+            x = wl.activations(0, j, T)
+            for fmt in wl.formats:
+                check_linear(fmt, w, x)
+
+
+def _sampled_rows(M, n=96, seed=0):
+    g = np.random.default_rng(seed)
+    rows = np.unique(np.concatenate([[0, 1, 31, 32, M - 33, M - 32, M - 1], g.integers(0, M, n)]))
+    return rows
+
+
+@pytest.mark.parametrize("layer", [0, 79])
+def test_workload_sweep100b_sampled_rows(layer):
+    """Full-size tensors of the 100B-shaped sweep, built and packed in device memory exactly as the
+    benchmark does; the oracle recomputes sampled output rows from host re-draws of the same weights."""
+    wl = synth.CONFIGS["sweep100b"]
+    for j, lin in enumerate(wl.linears):
+        wd = wl.weights(layer, j, device="cuda")
+        x = wl.activations(layer, j, 1)
+        q, sc, sm = bn.bitnet_quant_act(x.cuda())
+        q_ref, sc_ref, _ = oracle.quant_act(x.numpy())
+        assert np.array_equal(npy(q), q_ref)
+        rows = _sampled_rows(lin.M, seed=layer * 4 + j)
+        w_rows = np.stack([wl.weights(layer, j, row_start=int(r), rows=1).numpy()[0] for r in rows])
+        assert np.array_equal(npy(wd[torch.as_tensor(rows).cuda()]), w_rows)
+        acc_ref = oracle.mpgemm_def(q_ref, w_rows)
+        w_scale = 2.0 / 3.0
+        for fmt in wl.formats:
+            blob = bn.pack(fmt, wd, check=False)
+            y, acc = bn.bitnet_mpgemm(fmt, blob, w_scale, lin.M, lin.K, q, sc, want_acc=True)
+            torch.cuda.synchronize()
+            assert np.array_equal(npy(acc)[:, rows], acc_ref)
+            check_y(y[:, torch.as_tensor(rows).cuda()], acc_ref, sc_ref, w_scale)
+            # whole-vector properties: TL and I2_S agree everywhere; accumulators bounded by 127*K
+            if fmt == "i2s":
+                acc_i2s = acc.clone()
+            else:
+                assert torch.equal(acc, acc_i2s)
+            assert int(acc.abs().max()) <= 127 * lin.K
+            del blob
+        del wd
+        torch.cuda.empty_cache()
+
+
+def test_workload_prefill_sampled():
+    wl = synth.CONFIGS["prefill"]
+    lin = wl.linears[0]
+    T = wl.tokens[0]
+    w, x = wl.weights(0, 0), wl.activations(0, 0, T)
+    out = run_linear("i2s", w, x)
+    q_ref, sc_ref, sm_ref = oracle.quant_act(x.numpy())
+    assert np.array_equal(npy(out["q"]), q_ref)
+    assert np.array_equal(npy(out["act_scale"]).view(np.uint32), sc_ref.view(np.uint32))
+    rows = _sampled_rows(lin.M, 64, seed=3)
+    toks = np.unique(np.concatenate([[0, 1, 127, 128, T - 1], np.random.default_rng(3).integers(0, T, 40)]))
+    acc_ref = oracle.mpgemm_def(q_ref[toks], w.numpy()[rows])
+    acc = npy(out["acc"])[np.ix_(toks, rows)]
+    assert np.array_equal(acc, acc_ref)
+    check_y(out["y"][torch.as_tensor(toks).cuda()][:, torch.as_tensor(rows).cuda()], acc_ref, sc_ref[toks],
+            out["w_scale"])
+    # all-ones weights: every output of a token equals that token's code sum (a whole-matrix property)
+    ones = torch.ones(256, lin.K, dtype=torch.int8)
+    o2 = run_linear("i2s", ones, x, w_scale=1.0)
+    assert torch.equal(o2["acc"], o2["act_sum"][:, None].expand(T, 256).contiguous())
