@@ -121,6 +121,28 @@ int bitnet_linear_host(bitnet_fmt_t fmt, const void* packed, float w_scale, int6
                        int8_t* q_dev, float* scale_dev, float* y_dev, void* workspace,
                        size_t workspace_bytes, void* stream);
 
+/*
+ * Table-lookup mpGEMV without a workspace argument (the paper has no counterpart: this entry point
+ * exists for the sake of callers, not of the method).
+ *
+ * Same operation and arguments as bitnet_mpgemm for fmt = BITNET_FMT_TL1 / BITNET_FMT_TL2 and
+ * T <= 8, but the scratch that joins the K-slices lives in a fixed array inside the library
+ * (BITNET_NOALLOC_MAX_M rows x 9 words = 2.25 MiB, held by every GPU that loads the library until
+ * the process exits).  It is meant for hosts that cannot call cudaMalloc or hand over a workspace:
+ * code running while the device allocator is frozen or its pool is fully committed to weights,
+ * latency-critical loops that must not make calls which can block or fail, and plug-ins that
+ * receive input and output buffers only.  The call itself allocates nothing, on host or device.
+ *   - M > BITNET_NOALLOC_MAX_M or T > 8 returns BITNET_ERR_WORKSPACE and launches nothing.
+ *   - The first call on each device looks up the array's device address (a blocking runtime query);
+ *     make that first call outside any stream capture.
+ *   - Every call on a device shares the one array and clears the part it needs first, on `stream`;
+ *     two calls that may run on the GPU at the same time (different streams) race on it.
+ */
+#define BITNET_NOALLOC_MAX_M 65536
+int bitnet_mpgemv_tl_noalloc(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M, int64_t K,
+                             int bk3, const int8_t* q, const float* act_scale, int64_t T, float* y,
+                             int32_t* acc_out, void* stream);
+
 /* ---- test hooks (not part of the four operations) ------------------------------------------- */
 /* Inverse of the packers: packed -> w[M][K] int8.  dev_status set if an invalid code is met. */
 int bitnet_unpack_i2s(const void* packed, int64_t M, int64_t K, int8_t* w, int* dev_status,

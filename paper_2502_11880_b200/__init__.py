@@ -24,7 +24,7 @@ SYMBOLS = [
     "bitnet_status_string", "bitnet_last_cuda_error", "bitnet_quant_act", "bitnet_i2s_packed_bytes",
     "bitnet_pack_i2s", "bitnet_tl_packed_bytes", "bitnet_pack_tl", "bitnet_mpgemm_workspace_bytes",
     "bitnet_workspace_init", "bitnet_mpgemm", "bitnet_linear_host", "bitnet_unpack_i2s", "bitnet_unpack_tl",
-    "bitnet_tl_num_groups", "bitnet_tl_build_lut_debug",
+    "bitnet_tl_num_groups", "bitnet_tl_build_lut_debug", "bitnet_mpgemv_tl_noalloc",
 ]
 
 _lib = None
@@ -63,6 +63,7 @@ def lib():
         L.bitnet_tl_num_groups.argtypes = [ci, i64, ci]
         L.bitnet_tl_num_groups.restype = i64
         L.bitnet_tl_build_lut_debug.argtypes = [ci, vp, i64, ci, vp, vp]
+        L.bitnet_mpgemv_tl_noalloc.argtypes = [ci, vp, fl, i64, i64, ci, vp, vp, i64, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -237,3 +238,17 @@ def bitnet_linear_host(fmt, packed, w_scale, M, K, x_host, y_host, x_dev, q_dev,
     _check(lib().bitnet_linear_host(_fmt(fmt), _ptr(packed), float(w_scale), M, K, bk3, _ptr(x_host), T,
                                     _ptr(y_host), _ptr(x_dev), _ptr(q_dev), _ptr(scale_dev), _ptr(y_dev),
                                     _ptr(workspace), ws_bytes, _stream(stream)), "bitnet_linear_host")
+
+
+NOALLOC_MAX_M = 65536
+
+
+def bitnet_mpgemv_tl_noalloc(fmt, packed, w_scale, M, K, q, act_scale, y, acc_out=None, bk3=0, stream=None):
+    """TL1/TL2 mpGEMV (T <= 8) for callers that cannot allocate: no workspace argument, and this wrapper
+    creates no tensor either -- y (and acc_out, if wanted) must be supplied.  The scratch is a fixed
+    array inside the library, shared by every call on the device; see the header for the limits."""
+    T = q.shape[0]
+    _check(lib().bitnet_mpgemv_tl_noalloc(_fmt(fmt), _ptr(packed), float(w_scale), M, K, bk3, _ptr(q),
+                                          _ptr(act_scale), T, _ptr(y), _ptr(acc_out), _stream(stream)),
+           "bitnet_mpgemv_tl_noalloc")
+    return y, acc_out
