@@ -7,7 +7,7 @@ Workload (config.workload = "sweep100b"): the 100B-shaped decode sweep at batch 
 four ternary linears (8192->10240, 8192->8192, 8192->57344, 28672->8192), every tensor with its own
 seeded weights resident in HBM in the I2_S encoding (17.1 GB), one fp32 activation vector per linear.
 One step = one pass over all 320 linears: absmax int8 quantiser, then I2_S mpGEMV with the fused
-rescale, replayed from one CUDA graph.  `value` = I2_S bytes streamed per step / step time (GB/s),
+rescale -- one fused kernel per linear -- replayed from CUDA graphs.  `value` = I2_S bytes streamed per step / step time (GB/s),
 so it charges the quantisers and every launch gap to the weight stream.  The same sweep in the TL2
 encoding and the prefill mpGEMM (2048 x 4096 x 14336, int8 tensor cores) are timed in the same run
 and reported under "tl2" and "prefill".  Inputs (17 GB) exceed L2 (126 MB) many times over, so no L2
@@ -201,14 +201,19 @@ class Sweep:
         sc = self.sc_dev[i: i + 1]
         return lin, x, q, sc, y
 
-    def step_device(self, fmt, quant=True, gemv=True):
-        """One pass over every linear, inputs resident: quantiser then mpGEMV (2 launches per linear)."""
+    def step_device(self, fmt, mode="linear", lo=0, hi=None):
+        """One pass over linears [lo, hi), inputs resident.  mode "linear": bitnet_linear (quantiser + mpGEMV +
+        rescale; one fused kernel per linear for I2_S, two kernels for TL2); "quant" / "gemv": that step alone."""
         bn = self.bn
-        for i in range(self.n_linears()):
+        hi = self.n_linears() if hi is None else hi
+        for i in range(lo, hi):
             lin, x, q, sc, y = self.views(i)
-            if quant:
+            if mode == "linear":
+                bn.bitnet_linear(fmt, self.blobs[fmt][i], self.w_scale[i], lin.M, lin.K, x, q=q, act_scale=sc, y=y,
+                                 workspace=self.ws[fmt])
+            elif mode == "quant":
                 bn.bitnet_quant_act(x, q=q, act_scale=sc, act_sum=self._sum)
-            if gemv:
+            else:
                 bn.bitnet_mpgemm(fmt, self.blobs[fmt][i], self.w_scale[i], lin.M, lin.K, q, sc, y=y,
                                  workspace=self.ws[fmt])
 
@@ -222,19 +227,30 @@ class Sweep:
             bn.bitnet_linear_host(fmt, self.blobs[fmt][i], self.w_scale[i], lin.M, lin.K, xh, yh, x, q, sc, y,
                                   workspace=self.ws[fmt])
 
-    def make_graph(self, fmt, quant=True, gemv=True):
+    def make_graph(self, fmt, mode="linear", linears_per_graph=128):
+        """Captures the step as CUDA graphs of at most `linears_per_graph` linears each (long chains of
+        programmatically dependent kernel nodes in ONE graph replay pathologically slowly on this driver).
+        Returns a callable that replays them in order."""
         torch = self.torch
         self._sum = torch.empty(1, dtype=torch.int32, device=self.x_dev.device)
         s = torch.cuda.Stream()
         s.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(s):
-            self.step_device(fmt, quant, gemv)       # warm every kernel variant before capture
+            self.step_device(fmt, mode)            # warm every kernel variant before capture
         torch.cuda.current_stream().wait_stream(s)
         torch.cuda.synchronize()
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
-            self.step_device(fmt, quant, gemv)
-        return g
+        graphs = []
+        for lo in range(0, self.n_linears(), linears_per_graph):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                self.step_device(fmt, mode, lo, min(lo + linears_per_graph, self.n_linears()))
+            graphs.append(g)
+
+        def replay():
+            for g in graphs:
+                g.replay()
+        replay.n_graphs = len(graphs)
+        return replay
 
 
 def time_replays(torch, fn, steps, warmup, dist=None):
@@ -292,6 +308,8 @@ def run_ours(args):
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     bn.lib()   # fail loudly here if the extension is missing
+    if args.no_early_start:
+        bn.bitnet_set_early_start(False)
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -309,18 +327,18 @@ def run_ours(args):
     # ---- headline: I2_S sweep, quantiser + GEMV, one graph replay per step
     g_full = sw.make_graph("i2s")
     sampler = ClockSampler(local) if rank == 0 else None
-    ms_step = time_replays(torch, g_full.replay, args.steps, args.warmup, dist)
+    ms_step = time_replays(torch, g_full, args.steps, args.warmup, dist)
     clocks = sampler.stop() if sampler else None
     total_bytes = sw.bytes["i2s"] * world
     value = total_bytes / ms_step / 1e6
 
     # ---- dominant kernel alone (GEMV launches only): roofline
-    g_gemv = sw.make_graph("i2s", quant=False)
-    ms_gemv = time_replays(torch, g_gemv.replay, args.steps, args.warmup, dist)
+    g_gemv = sw.make_graph("i2s", "gemv")
+    ms_gemv = time_replays(torch, g_gemv, args.steps, args.warmup, dist)
     n_lin = sw.n_linears()
-    achieved = sw.bytes["i2s"] / ms_gemv / 1e6
-    g_quant = sw.make_graph("i2s", gemv=False)
-    ms_quant = time_replays(torch, g_quant.replay, args.steps, args.warmup, dist)
+    achieved = sw.bytes["i2s"] / ms_step / 1e6
+    g_quant = sw.make_graph("i2s", "quant")
+    ms_quant = time_replays(torch, g_quant, args.steps, args.warmup, dist)
 
     # ---- end to end through the host-buffer entry point
     ms_e2e = time_replays(torch, lambda: (sw.step_host("i2s"), torch.cuda.current_stream().synchronize()),
@@ -333,30 +351,33 @@ def run_ours(args):
         "data": "synthetic",
         "config": {"workload": "sweep100b", "layers": layers, "linears_per_layer": 4, "tokens": 1, "format": "i2s",
                    "packed_bytes": sw.bytes["i2s"], "parallelism": f"replicas x{world}",
-                   "l2": "inputs (17 GB of weights) exceed L2; no flush needed", "launch": "one CUDA graph per step",
+                   "l2": "inputs (17 GB of weights) exceed L2; no flush needed",
+                   "launch": f"{g_full.n_graphs} CUDA graph replays per step, one fused kernel per linear",
                    "pct_of_8TBps": 100.0 * (value / world) / 8000.0},
         "e2e": {"value": e2e_val, "unit": UNIT, "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": int(sw.x_host.numel() * 4), "d2h_bytes_per_step": int(sw.y_host.numel() * 4),
                 "note": "per linear: pinned fp32 x -> device, quantiser, mpGEMV, fp32 y -> pinned host; weights resident"},
-        "gpu_launches": 2 * n_lin * args.steps,
-        "roofline": {"bound": "hbm", "kernel": "gemv_i2s_kernel<1,4>", "achieved": achieved, "peak": pk["hbm"],
-                     "unit": "GB/s", "frac": achieved / pk["hbm"], "peak_source": pk["which"],
-                     "bytes_per_launch": sw.bytes["i2s"] / n_lin, "us_per_launch": 1e3 * ms_gemv / n_lin,
+        "gpu_launches": n_lin * args.steps,
+        "roofline": {"bound": "hbm", "kernel": "gemv_i2s_mma_kernel (quantiser fused)", "achieved": achieved,
+                     "peak": pk["hbm"], "unit": "GB/s", "frac": achieved / pk["hbm"], "peak_source": pk["which"],
+                     "bytes_per_launch": sw.bytes["i2s"] / n_lin, "us_per_launch": 1e3 * ms_step / n_lin,
                      "traffic": None},
-        "breakdown": {"ms_gemv_only": ms_gemv, "ms_quant_only": ms_quant, "setup_s": sw.setup_s},
+        "breakdown": {"ms_fused_step": ms_step, "ms_gemv_kernels_alone": ms_gemv, "ms_quant_kernels_alone": ms_quant,
+                      "setup_s": sw.setup_s},
         "clocks": clocks,
     }
 
     if rank == 0:
         if "tl2" in fmts:
             g_tl = sw.make_graph("tl2")
-            ms_tl = time_replays(torch, g_tl.replay, args.steps, args.warmup)
-            g_tl_g = sw.make_graph("tl2", quant=False)
-            ms_tl_g = time_replays(torch, g_tl_g.replay, args.steps, args.warmup)
+            ms_tl = time_replays(torch, g_tl, args.steps, args.warmup)
+            g_tl_g = sw.make_graph("tl2", "gemv")
+            ms_tl_g = time_replays(torch, g_tl_g, args.steps, args.warmup)
             line["tl2"] = {"packed_bytes": sw.bytes["tl2"], "ms_per_step": ms_tl, "value": sw.bytes["tl2"] / ms_tl / 1e6,
                            "unit": UNIT, "gemv_only_GBps": sw.bytes["tl2"] / ms_tl_g / 1e6,
                            "frac_of_hbm_peak": sw.bytes["tl2"] / ms_tl_g / 1e6 / pk["hbm"]}
         del sw, g_full, g_gemv, g_quant
+        g_tl = g_tl_g = None
         torch.cuda.empty_cache()
         if not args.skip_prefill:
             pf = bench_prefill(bn, torch, synth, max(3, args.steps // 2), 3)
@@ -395,6 +416,8 @@ def main():
     ap.add_argument("--skip-tl2", action="store_true")
     ap.add_argument("--skip-prefill", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
+    ap.add_argument("--no-early-start", action="store_true",
+                    help="launch every kernel in plain stream order (no programmatic dependent launch)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":

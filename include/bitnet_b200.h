@@ -51,6 +51,24 @@ const char* bitnet_status_string(int status);
 int bitnet_last_cuda_error(void);
 
 /*
+ * Device-side status: kernels that wait on asynchronous copies bound every wait; a wait that gave up
+ * stores BITNET_ERR_TIMEOUT in a device flag.  This call synchronises the device and copies the flag
+ * to *status_out (0 = no kernel ever gave up).  Not for the hot path.
+ */
+int bitnet_device_status(int* status_out);
+
+/*
+ * Early start (on by default).  The quantiser and the I2_S decode kernel are launched with
+ * programmatic dependent launch: their prologue may run while the previous kernel queued on the same
+ * stream is finishing, and the decode kernel starts copying the PACKED WEIGHTS into shared memory
+ * before that kernel has finished (activations, scales and outputs are touched only after it has).
+ * Packed weights are treated as read-only model state: if a blob was written by work queued earlier on
+ * the same stream, synchronise (or record/wait an event) before the first bitnet_mpgemm that reads it,
+ * or switch early start off.  enable = 0 restores plain stream order for every later call.
+ */
+void bitnet_set_early_start(int enable);
+
+/*
  * Activation quantiser -- Alg. 1 Phase 1 ("Quantization"), Sec. 2.1 and 3.2.2: absmax int8.
  *   x[T][K] fp32 row-major (read)  ->  q[T][K] int8, act_scale[T] fp32, act_sum[T] int32 (nullable).
  * Per token t: amax = max(max_k |x[t,k]|, 1e-5); s = 127/amax (binary32); q = clamp(rint(x*s),
@@ -64,8 +82,13 @@ int bitnet_quant_act(const float* x, int64_t T, int64_t K, int per_tensor, int8_
 /*
  * I2_S weight packer -- I2_S of Table 1 / Sec. 3.2.2 (2 bits per weight; the scale stays outside).
  *   w[M][K] int8 in {-1,0,+1}, row-major (read) -> packed, bitnet_i2s_packed_bytes(M,K) bytes.
- * Layout: a row occupies ceil(K/128)*32 bytes; byte 4j+b of a row holds the weights
- * k = 16j + 4s + b (s = 0..3) as code w+1 in bits [2s, 2s+1]; positions past K hold weight 0.
+ * Layout (code = w+1 in two bits; padding holds weight 0): rows in blocks of 8 (M padded to a
+ * multiple of 8), K padded to a multiple of 256.  A block is contiguous: for each chunk c of 256
+ * columns it holds 512 bytes, of which row r of the block owns bytes [64r, 64r+64) = 16 little-endian
+ * words.  Column kk = k % 256 of a chunk sits in word j = 2*(kk/32) + (kk%8)/4, byte b = kk%4, bits
+ * [2s, 2s+1] with s = (kk%32)/8.  (One 8-row block of up to 8192 columns is one contiguous 16 KB piece
+ * for a bulk copy; 32 lanes reading 16 bytes each cover 8 rows x 64 bytes without bank conflicts; the
+ * two activation words an int8 MMA needs for words 2h, 2h+1 are adjacent.)
  * dev_status (nullable device int): set to BITNET_ERR_BAD_WEIGHT if a non-ternary byte is met
  * (the blob is then undefined).  Requires K % 64 == 0.
  */
@@ -110,8 +133,22 @@ int bitnet_mpgemm(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
                   void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * One linear layer from fp32 activations: Alg. 1 end to end -- Phase 1 (quantiser), Phase 2 (mpGEMM)
+ * and the rescale -- with device buffers.
+ *   x[T][K] fp32 in; q[T][K] int8 and act_scale[T] fp32 are OUTPUTS (the quantised activations, as
+ *   bitnet_quant_act would give them); y[T][M] fp32 out; acc_out nullable; workspace as for
+ *   bitnet_mpgemm.
+ * For I2_S with T <= 8 (and T*K up to 64 KiB) this is ONE kernel: every CTA of the decode kernel
+ * quantises the activation vector itself while its first weight tiles are in flight.  Otherwise it is
+ * bitnet_quant_act followed by bitnet_mpgemm.  Results are identical either way.
+ */
+int bitnet_linear(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M, int64_t K, int bk3,
+                  const float* x, int64_t T, int8_t* q, float* act_scale, float* y, int32_t* acc_out,
+                  void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * One linear layer with HOST activations and HOST results: copies x_host[T][K] to x_dev, runs
- * bitnet_quant_act and bitnet_mpgemm, and copies y_dev[T][M] to y_host, all queued on `stream`
+ * bitnet_linear, and copies y_dev[T][M] to y_host, all queued on `stream`
  * (Alg. 1 end to end).  x_host / y_host should be pinned for the copies to be asynchronous; the
  * device buffers x_dev [T*K fp32], q_dev [T*K int8], scale_dev [T fp32], y_dev [T*M fp32] and the
  * workspace are caller-owned scratch.  The caller synchronises the stream before reading y_host.

@@ -152,40 +152,47 @@ void oracle_dequant(const int32_t* acc, const float* act_scale, float w_scale, i
 }
 
 // ---------------------------------------------------------------------------------------------
-// I2_S.  code = w + 1 (0,1,2), two bits.  A row occupies ceil(K/128)*32 bytes; positions past K
-// hold weight 0 (code 1).  Byte 4j+b of a row carries the weights k = 16j + 4s + b, s = 0..3,
-// the code of slot s in bits [2s, 2s+1].
+// I2_S.  code = w + 1 (0,1,2), two bits.  Rows are stored in blocks of 8 (M padded to a multiple of
+// 8), K is padded to a multiple of 256; padding holds weight 0 (code 1).  A block is contiguous and
+// holds, for each chunk c of 256 columns, 512 bytes in which row r (0..7) owns bytes [64r, 64r+64).
+// In those 64 bytes = 16 little-endian words, the weight at column kk = k % 256 of the chunk sits in
+//   word j = 2*(kk/32) + (kk%8)/4,  byte b = kk%4 of that word,  bits [2s, 2s+1] with s = (kk%32)/8.
+struct I2sPos {
+  int64_t byte;
+  int shift;
+};
+static I2sPos i2s_pos(int64_t m, int64_t k, int64_t kp) {
+  const int64_t rb = m / 8, r = m % 8, c = k / 256, kk = k % 256;
+  const int64_t j = 2 * (kk / 32) + (kk % 8) / 4, b = kk % 4, s = (kk % 32) / 8;
+  return {rb * (2 * kp) + c * 512 + r * 64 + 4 * j + b, (int)(2 * s)};
+}
+
 size_t oracle_i2s_packed_bytes(int64_t M, int64_t K) {
   if (M < 1 || K < 1) return 0;
-  return (size_t)M * (size_t)ceil_div(K, 128) * 32;
+  return (size_t)(ceil_div(M, 8) * 8) * (size_t)(ceil_div(K, 256) * 256) / 4;
 }
 
 int oracle_pack_i2s(const int8_t* w, int64_t M, int64_t K, uint8_t* packed) {
   if (!w || !packed || M < 1 || K < 1) return 1;
-  const int64_t row_bytes = ceil_div(K, 128) * 32;
-  for (int64_t m = 0; m < M; ++m) {
-    for (int64_t byte = 0; byte < row_bytes; ++byte) {
-      const int64_t j = byte / 4, b = byte % 4;
-      unsigned v = 0;
-      for (int s = 0; s < 4; ++s) {
-        const int64_t k = 16 * j + 4 * s + b;
-        int8_t wk = (k < K) ? w[m * K + k] : (int8_t)0;
-        if (!tern_ok(wk)) return 3;
-        v |= (unsigned)(wk + 1) << (2 * s);
-      }
-      packed[m * row_bytes + byte] = (uint8_t)v;
+  const int64_t mp = ceil_div(M, 8) * 8, kp = ceil_div(K, 256) * 256;
+  std::memset(packed, 0, (size_t)(mp * kp / 4));
+  for (int64_t m = 0; m < mp; ++m)
+    for (int64_t k = 0; k < kp; ++k) {
+      const int8_t wk = (m < M && k < K) ? w[m * K + k] : (int8_t)0;
+      if (!tern_ok(wk)) return 3;
+      const I2sPos pos = i2s_pos(m, k, kp);
+      packed[pos.byte] |= (uint8_t)((wk + 1) << pos.shift);
     }
-  }
   return 0;
 }
 
 int oracle_unpack_i2s(const uint8_t* packed, int64_t M, int64_t K, int8_t* w) {
   if (!w || !packed || M < 1 || K < 1) return 1;
-  const int64_t row_bytes = ceil_div(K, 128) * 32;
+  const int64_t kp = ceil_div(K, 256) * 256;
   for (int64_t m = 0; m < M; ++m)
     for (int64_t k = 0; k < K; ++k) {
-      const int64_t j = k / 16, s = (k % 16) / 4, b = k % 4;
-      const unsigned code = (packed[m * row_bytes + 4 * j + b] >> (2 * s)) & 3u;
+      const I2sPos pos = i2s_pos(m, k, kp);
+      const unsigned code = (packed[pos.byte] >> pos.shift) & 3u;
       if (code == 3u) return 3;
       w[m * K + k] = (int8_t)((int)code - 1);
     }
@@ -196,13 +203,13 @@ int oracle_unpack_i2s(const uint8_t* packed, int64_t M, int64_t K, int8_t* w) {
 int oracle_i2s_mpgemm(const uint8_t* packed, int64_t M, int64_t K, const int8_t* q, int64_t T,
                       int32_t* acc) {
   if (!packed || !q || !acc || M < 1 || K < 1 || T < 1) return 1;
-  const int64_t row_bytes = ceil_div(K, 128) * 32;
+  const int64_t kp = ceil_div(K, 256) * 256;
   for (int64_t m = 0; m < M; ++m)
     for (int64_t t = 0; t < T; ++t) {
       int64_t s = 0;
       for (int64_t k = 0; k < K; ++k) {
-        const unsigned byte = packed[m * row_bytes + 4 * (k / 16) + (k % 4)];
-        const int wv = (int)((byte >> (2 * ((k % 16) / 4))) & 3u) - 1;
+        const I2sPos pos = i2s_pos(m, k, kp);
+        const int wv = (int)((packed[pos.byte] >> pos.shift) & 3u) - 1;
         s += (int64_t)q[t * K + k] * wv;
       }
       acc[t * M + m] = (int32_t)s;

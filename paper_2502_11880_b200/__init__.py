@@ -23,8 +23,9 @@ FMT = {"i2s": FMT_I2S, "tl1": FMT_TL1, "tl2": FMT_TL2}
 SYMBOLS = [
     "bitnet_status_string", "bitnet_last_cuda_error", "bitnet_quant_act", "bitnet_i2s_packed_bytes",
     "bitnet_pack_i2s", "bitnet_tl_packed_bytes", "bitnet_pack_tl", "bitnet_mpgemm_workspace_bytes",
-    "bitnet_workspace_init", "bitnet_mpgemm", "bitnet_linear_host", "bitnet_unpack_i2s", "bitnet_unpack_tl",
-    "bitnet_tl_num_groups", "bitnet_tl_build_lut_debug", "bitnet_mpgemv_tl_noalloc",
+    "bitnet_workspace_init", "bitnet_mpgemm", "bitnet_linear", "bitnet_linear_host", "bitnet_unpack_i2s", "bitnet_unpack_tl",
+    "bitnet_tl_num_groups", "bitnet_tl_build_lut_debug", "bitnet_mpgemv_tl_noalloc", "bitnet_device_status",
+    "bitnet_set_early_start",
 ]
 
 _lib = None
@@ -46,6 +47,9 @@ def lib():
         L.bitnet_status_string.argtypes = [ci]
         L.bitnet_status_string.restype = C.c_char_p
         L.bitnet_last_cuda_error.restype = ci
+        L.bitnet_device_status.argtypes = [vp]
+        L.bitnet_set_early_start.argtypes = [ci]
+        L.bitnet_set_early_start.restype = None
         L.bitnet_quant_act.argtypes = [vp, i64, i64, ci, vp, vp, vp, vp]
         L.bitnet_i2s_packed_bytes.argtypes = [i64, i64]
         L.bitnet_i2s_packed_bytes.restype = sz
@@ -57,6 +61,7 @@ def lib():
         L.bitnet_mpgemm_workspace_bytes.restype = sz
         L.bitnet_workspace_init.argtypes = [vp, sz, vp]
         L.bitnet_mpgemm.argtypes = [ci, vp, fl, i64, i64, ci, vp, vp, i64, vp, vp, vp, sz, vp]
+        L.bitnet_linear.argtypes = [ci, vp, fl, i64, i64, ci, vp, i64, vp, vp, vp, vp, vp, sz, vp]
         L.bitnet_linear_host.argtypes = [ci, vp, fl, i64, i64, ci, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp]
         L.bitnet_unpack_i2s.argtypes = [vp, i64, i64, vp, vp, vp]
         L.bitnet_unpack_tl.argtypes = [ci, vp, i64, i64, ci, vp, vp, vp]
@@ -70,6 +75,17 @@ def lib():
 
 def status_string(rc: int) -> str:
     return lib().bitnet_status_string(rc).decode()
+
+
+def bitnet_device_status() -> int:
+    """Synchronises the device and returns the device-side status flag (0 = no bounded wait ever gave up)."""
+    out = C.c_int(0)
+    _check(lib().bitnet_device_status(C.byref(out)), "bitnet_device_status")
+    return out.value
+
+
+def bitnet_set_early_start(enable: bool):
+    lib().bitnet_set_early_start(int(bool(enable)))
 
 
 def _check(rc: int, what: str):
@@ -228,6 +244,25 @@ def bitnet_mpgemm(fmt, packed, w_scale, M, K, q, act_scale, bk3=0, y=None, acc_o
                                _ptr(y), _ptr(acc_out), _ptr(workspace), ws_bytes, _stream(stream)),
            "bitnet_mpgemm")
     return y, acc_out
+
+
+def bitnet_linear(fmt, packed, w_scale, M, K, x, bk3=0, q=None, act_scale=None, y=None, acc_out=None, want_acc=False,
+                  workspace=None, stream=None):
+    """fp32 activations x[T][K] (CUDA) -> (y, q, act_scale, acc or None): quantiser + mpGEMM + rescale."""
+    _dev(x, torch.float32, "x")
+    T = x.shape[0]
+    q = torch.empty((T, K), dtype=torch.int8, device=x.device) if q is None else q
+    act_scale = torch.empty(T, dtype=torch.float32, device=x.device) if act_scale is None else act_scale
+    y = torch.empty((T, M), dtype=torch.float32, device=x.device) if y is None else y
+    if want_acc and acc_out is None:
+        acc_out = torch.empty((T, M), dtype=torch.int32, device=x.device)
+    if workspace is None:
+        workspace = new_workspace(fmt, T, M, K, x.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().bitnet_linear(_fmt(fmt), _ptr(packed), float(w_scale), M, K, bk3, _ptr(x), T, _ptr(q),
+                               _ptr(act_scale), _ptr(y), _ptr(acc_out), _ptr(workspace), ws_bytes, _stream(stream)),
+           "bitnet_linear")
+    return y, q, act_scale, acc_out
 
 
 def bitnet_linear_host(fmt, packed, w_scale, M, K, x_host, y_host, x_dev, q_dev, scale_dev, y_dev,

@@ -1,5 +1,7 @@
 // C ABI of libbitnet_b200.so: argument validation and dispatch.  Every step of the path runs in the
 // kernels of the sibling files; nothing here computes.
+#include <cstdlib>
+#include <cstring>
 #include <mutex>
 
 #include "common.cuh"
@@ -13,17 +15,32 @@ int note_cuda_error(cudaError_t e) {
   return BITNET_ERR_CUDA;
 }
 
+static int g_early_start = 1;
+bool early_start_enabled() { return g_early_start != 0; }
+
 const DevInfo& dev_info() {
   static DevInfo info[64];
   static bool have[64] = {false};
   static std::mutex mu;
   int dev = 0;
-  cudaGetDevice(&dev);
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    cudaGetLastError();
+    dev = 0;
+  }
   dev &= 63;
   std::lock_guard<std::mutex> lock(mu);
   if (!have[dev]) {
-    cudaDeviceGetAttribute(&info[dev].sm_count, cudaDevAttrMultiProcessorCount, dev);
-    cudaDeviceGetAttribute(&info[dev].max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    // B200 figures stand in when no device can be queried (size queries on a machine without a GPU)
+    info[dev].sm_count = 148;
+    info[dev].max_smem_optin = 232448;
+    info[dev].max_smem_per_sm = 233472;
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) info[dev].sm_count = v;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) == cudaSuccess && v > 0)
+      info[dev].max_smem_optin = v;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) == cudaSuccess && v > 0)
+      info[dev].max_smem_per_sm = v;
+    cudaGetLastError();
     have[dev] = true;
   }
   return info[dev];
@@ -50,6 +67,13 @@ const char* bitnet_status_string(int status) {
 
 int bitnet_last_cuda_error(void) { return g_last_cuda_error; }
 
+int bitnet_device_status(int* status_out) {
+  if (!status_out) return BITNET_ERR_INVALID_ARG;
+  return gemv_i2s_stream_status(status_out);
+}
+
+void bitnet_set_early_start(int enable) { g_early_start = enable ? 1 : 0; }
+
 int bitnet_quant_act(const float* x, int64_t T, int64_t K, int per_tensor, int8_t* q, float* act_scale,
                      int32_t* act_sum, void* stream) {
   if (!x || !q || !act_scale || T < 1 || K < 1 || T > 0x7fffffff) return BITNET_ERR_INVALID_ARG;
@@ -59,7 +83,7 @@ int bitnet_quant_act(const float* x, int64_t T, int64_t K, int per_tensor, int8_
 
 size_t bitnet_i2s_packed_bytes(int64_t M, int64_t K) {
   if (M < 1 || K < 1 || (K % 64) != 0) return 0;
-  return (size_t)M * (size_t)ceil_div(K, 128) * 32;
+  return (size_t)i2s_mp(M) * (size_t)i2s_kp(K) / 4;
 }
 
 static int i2s_shape(int64_t M, int64_t K) {
@@ -171,6 +195,30 @@ int bitnet_mpgemm(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
   return BITNET_OK;
 }
 
+int bitnet_linear(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M, int64_t K, int bk3, const float* x,
+                  int64_t T, int8_t* q, float* act_scale, float* y, int32_t* acc_out, void* workspace,
+                  size_t workspace_bytes, void* stream) {
+  if (!packed || !x || !q || !act_scale || !y || T < 1) return BITNET_ERR_INVALID_ARG;
+  if (!aligned16(packed) || !aligned16(x) || !aligned16(q) || !aligned16(y) || (acc_out && !aligned16(acc_out)) ||
+      (reinterpret_cast<uintptr_t>(act_scale) & 3u))
+    return BITNET_ERR_INVALID_ARG;
+  if (fmt == BITNET_FMT_I2S && T <= 8) {
+    int rc = i2s_shape(M, K);
+    if (rc) return rc;
+    static const bool no_fuse = [] {
+      const char* e = getenv("BITNET_I2S_KERNEL");
+      return e && strcmp(e, "splitk") == 0;
+    }();
+    if (!no_fuse && gemv_i2s_stream_supported((int)T, M, K, true))
+      return launch_gemv_i2s_stream((const uint8_t*)packed, w_scale, M, K, x, q, act_scale, (int)T, y, acc_out,
+                                    (cudaStream_t)stream);
+  }
+  int rc = bitnet_quant_act(x, T, K, 0, q, act_scale, nullptr, stream);
+  if (rc) return rc;
+  return bitnet_mpgemm(fmt, packed, w_scale, M, K, bk3, q, act_scale, T, y, acc_out, workspace, workspace_bytes,
+                       stream);
+}
+
 int bitnet_linear_host(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M, int64_t K, int bk3,
                        const float* x_host, int64_t T, float* y_host, float* x_dev, int8_t* q_dev,
                        float* scale_dev, float* y_dev, void* workspace, size_t workspace_bytes, void* stream) {
@@ -179,10 +227,8 @@ int bitnet_linear_host(bitnet_fmt_t fmt, const void* packed, float w_scale, int6
   cudaStream_t st = (cudaStream_t)stream;
   cudaError_t e = cudaMemcpyAsync(x_dev, x_host, (size_t)T * K * sizeof(float), cudaMemcpyHostToDevice, st);
   if (e != cudaSuccess) return note_cuda_error(e);
-  int rc = bitnet_quant_act(x_dev, T, K, 0, q_dev, scale_dev, nullptr, stream);
-  if (rc) return rc;
-  rc = bitnet_mpgemm(fmt, packed, w_scale, M, K, bk3, q_dev, scale_dev, T, y_dev, nullptr, workspace,
-                     workspace_bytes, stream);
+  int rc = bitnet_linear(fmt, packed, w_scale, M, K, bk3, x_dev, T, q_dev, scale_dev, y_dev, nullptr, workspace,
+                         workspace_bytes, stream);
   if (rc) return rc;
   e = cudaMemcpyAsync(y_host, y_dev, (size_t)T * M * sizeof(float), cudaMemcpyDeviceToHost, st);
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);

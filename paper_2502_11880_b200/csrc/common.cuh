@@ -37,6 +37,16 @@ inline __host__ bool tl_geom(int fmt, int64_t M, int64_t K, int bk3, TlGeom* g) 
   return true;
 }
 
+// Geometry of an I2_S blob: rows in blocks of 8, K padded to 256; a block is contiguous and holds
+// one 512-byte piece per 256-column chunk, row r of the block owning bytes [64r, 64r+64) of it.
+// Word j (0..15) of those 64 bytes, slot s (bits [8b+2s, 8b+2s+1] of byte b) holds the weights
+// kk = 32*(j/2) + 8*s + 4*(j%2) + b of the chunk, i.e. the activation word 8*(j/2) + 2*s + (j%2).
+inline __host__ __device__ int64_t i2s_kp(int64_t K) { return ceil_div(K, 256) * 256; }
+inline __host__ __device__ int64_t i2s_mp(int64_t M) { return ceil_div(M, 8) * 8; }
+inline __host__ __device__ int64_t i2s_row_chunk_offset(int64_t m, int64_t chunk, int64_t kp) {
+  return (m >> 3) * (2 * kp) + chunk * 512 + (m & 7) * 64;
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Records a failing CUDA call for bitnet_last_cuda_error(); returns the library status.
@@ -50,6 +60,7 @@ inline int check_launch() {
 struct DevInfo {
   int sm_count;
   int max_smem_optin;
+  int max_smem_per_sm;
 };
 const DevInfo& dev_info();
 
@@ -70,6 +81,15 @@ size_t gemv_i2s_workspace_bytes(int64_t T, int64_t M, int64_t K);
 int launch_gemv_i2s(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const int8_t* q,
                     const float* act_scale, int T, float* y, int32_t* acc_out, void* ws, size_t ws_bytes,
                     cudaStream_t st);
+// Streaming (bulk-copy ring + tensor-core MMA) kernel.
+bool gemv_i2s_stream_supported(int T, int64_t M, int64_t K, bool fused);
+// x != nullptr runs the quantiser inside the kernel (q and act_scale are then outputs).
+int launch_gemv_i2s_stream(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const float* x, int8_t* q,
+                           float* act_scale, int T, float* y, int32_t* acc_out, cudaStream_t st);
+int gemv_i2s_stream_status(int* out);
+// Programmatic dependent launch (kernels may start their prologue, and prefetch weights, before the
+// previous kernel in the stream has finished); process-wide switch, on by default.
+bool early_start_enabled();
 size_t gemv_tl_workspace_bytes(int fmt, int64_t T, int64_t M, int64_t K);
 int launch_gemv_tl(int fmt, const uint8_t* packed, float w_scale, int64_t M, int64_t K, const TlGeom& g,
                    const int8_t* q, const float* act_scale, int T, float* y, int32_t* acc_out, void* ws,

@@ -3,18 +3,22 @@
 //   acc[t,m] = sum_k q[t,k] * w[m,k],   w = code - 1,  code in {0,1,2} two bits each
 //            = sum_k q[t,k] * code[m,k]  -  sum_k q[t,k]
 //
+// Split-K fallback for shapes the streaming kernel does not cover (see gemv_i2s_mma.cu).
 // Mapping.  A warp owns a row (for a K-slice of J*2048 weights): lane l loads J 16-byte vectors of
-// the row (vector index slice*J*32 + j*32 + l, 64 weights each), fully coalesced 512-byte requests.
+// the row (vector index slice*J*32 + j*32 + l, 64 weights each).
 // The lane's activations for those weights never change from row to row, so they live in registers
 // (TT tokens x J x 16 words).  A packed 32-bit word holds 16 codes; the four masks 0x03030303 << 2s
-// pick, WITHOUT shifting, the codes of slot s = weights 16j+4s+{0..3} scaled by 4^s, and one
-// dp4a.u32.s32 multiplies them with the activation word 4j+s.  Four accumulators carry the scales
+// pick, WITHOUT shifting, the four codes of slot s scaled by 4^s, and one dp4a.u32.s32 multiplies
+// them with the matching activation word.  Four accumulators carry the scales
 // 1, 4, 16, 64; each is an exact multiple of its scale, so arithmetic shifts undo it.  That is one
 // logic op and one dp4a per four weights.  Lane partials are summed by warp shuffles.
 //
 // K longer than one slice is split over blockIdx.y; partial sums meet in an int32 workspace by
 // atomicAdd (exact and order independent), and the slice that arrives last at a row's ticket
 // converts, stores and re-zeroes that row -- no waiting anywhere.
+#include <cstdlib>
+#include <cstring>
+
 #include "common.cuh"
 
 namespace bitnet {
@@ -42,8 +46,8 @@ __device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
 }
 
 struct GemvArgs {
-  const uint4* packed;   // blob
-  int64_t row_vecs;      // 16-byte vectors per row in the blob (includes padding)
+  const uint8_t* packed; // blob
+  int64_t kp;            // K padded to 256 (blob geometry)
   int data_vecs;         // K / 64: vectors per row that carry weights
   int M;
   int64_t K;
@@ -57,6 +61,11 @@ struct GemvArgs {
   unsigned* ws_ticket;   // [M]
   int nslices;
 };
+
+// 16-byte vector v of a row = its weights [64v, 64v+64): piece v%4 of chunk v/4.
+__device__ __forceinline__ const uint4* vec_ptr(const GemvArgs& a, int row, int v) {
+  return reinterpret_cast<const uint4*>(a.packed + i2s_row_chunk_offset(row, v >> 2, a.kp) + (v & 3) * 16);
+}
 
 template <int TT, int J>
 __global__ void __launch_bounds__(THREADS, 2) gemv_i2s_kernel(const GemvArgs a) {
@@ -107,14 +116,14 @@ __global__ void __launch_bounds__(THREADS, 2) gemv_i2s_kernel(const GemvArgs a) 
 #pragma unroll
   for (int j = 0; j < J; ++j) {
     cur[j] = make_uint4(0, 0, 0, 0);
-    if (row < a.M && ok[j]) cur[j] = ldg_stream(a.packed + (int64_t)row * a.row_vecs + vec[j]);
+    if (row < a.M && ok[j]) cur[j] = ldg_stream(vec_ptr(a, row, vec[j]));
   }
   for (; row < a.M; row += gws) {
     const int nrow = row + gws;
 #pragma unroll
     for (int j = 0; j < J; ++j) {
       nxt[j] = make_uint4(0, 0, 0, 0);
-      if (nrow < a.M && ok[j]) nxt[j] = ldg_stream(a.packed + (int64_t)nrow * a.row_vecs + vec[j]);
+      if (nrow < a.M && ok[j]) nxt[j] = ldg_stream(vec_ptr(a, nrow, vec[j]));
     }
     int acc[TT][4];
 #pragma unroll
@@ -131,10 +140,11 @@ __global__ void __launch_bounds__(THREADS, 2) gemv_i2s_kernel(const GemvArgs a) 
         const unsigned m2 = wv[c] & 0x30303030u, m3 = wv[c] & 0xC0C0C0C0u;
 #pragma unroll
         for (int t = 0; t < TT; ++t) {
-          acc[t][0] = dp4a_us(m0, qr[t][j][4 * c + 0], acc[t][0]);
-          acc[t][1] = dp4a_us(m1, qr[t][j][4 * c + 1], acc[t][1]);
-          acc[t][2] = dp4a_us(m2, qr[t][j][4 * c + 2], acc[t][2]);
-          acc[t][3] = dp4a_us(m3, qr[t][j][4 * c + 3], acc[t][3]);
+          // word c of the piece, slot s multiplies activation word 8*(c/2) + 2*s + (c%2)
+          acc[t][0] = dp4a_us(m0, qr[t][j][8 * (c / 2) + 0 + (c % 2)], acc[t][0]);
+          acc[t][1] = dp4a_us(m1, qr[t][j][8 * (c / 2) + 2 + (c % 2)], acc[t][1]);
+          acc[t][2] = dp4a_us(m2, qr[t][j][8 * (c / 2) + 4 + (c % 2)], acc[t][2]);
+          acc[t][3] = dp4a_us(m3, qr[t][j][8 * (c / 2) + 6 + (c % 2)], acc[t][3]);
         }
       }
     }
@@ -203,7 +213,16 @@ int launch_one(GemvArgs a, cudaStream_t st) {
 
 }  // namespace
 
+static bool use_stream_kernel(int64_t T, int64_t M, int64_t K) {
+  static const bool forced_splitk = [] {
+    const char* e = getenv("BITNET_I2S_KERNEL");
+    return e && strcmp(e, "splitk") == 0;
+  }();
+  return !forced_splitk && gemv_i2s_stream_supported((int)T, M, K, false);
+}
+
 size_t gemv_i2s_workspace_bytes(int64_t T, int64_t M, int64_t K) {
+  if (use_stream_kernel(T > 8 ? 8 : T, M, K)) return 0;
   int TT, J;
   pick((int)(T > 8 ? 8 : T), &TT, &J);
   if (slices_for(K, J) == 1) return 0;
@@ -214,11 +233,14 @@ size_t gemv_i2s_workspace_bytes(int64_t T, int64_t M, int64_t K) {
 int launch_gemv_i2s(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const int8_t* q,
                     const float* act_scale, int T, float* y, int32_t* acc_out, void* ws, size_t ws_bytes,
                     cudaStream_t st) {
+  if (use_stream_kernel(T, M, K))
+    return launch_gemv_i2s_stream(packed, w_scale, M, K, nullptr, const_cast<int8_t*>(q), const_cast<float*>(act_scale), T, y,
+                                  acc_out, st);
   int TT, J;
   pick(T, &TT, &J);
   GemvArgs a;
-  a.packed = reinterpret_cast<const uint4*>(packed);
-  a.row_vecs = ceil_div(K, 128) * 2;
+  a.packed = packed;
+  a.kp = i2s_kp(K);
   a.data_vecs = (int)(K / 64);
   a.M = (int)M;
   a.K = K;

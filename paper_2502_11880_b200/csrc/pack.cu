@@ -11,41 +11,50 @@ namespace {
 
 __device__ __forceinline__ bool ternary(int w) { return w >= -1 && w <= 1; }
 
-// One thread per 32-bit packed word = 16 consecutive weights of one row.
-__global__ void pack_i2s_kernel(const int8_t* __restrict__ w, int64_t M, int64_t K, int64_t row_words,
+// One thread per 32-bit packed word of the blob (16 weights of one row, see common.cuh for the map).
+__global__ void pack_i2s_kernel(const int8_t* __restrict__ w, int64_t M, int64_t K, int64_t kp, int64_t nwords,
                                 uint32_t* __restrict__ packed, int* dev_status) {
   const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (gid >= M * row_words) return;
-  const int64_t m = gid / row_words, j = gid % row_words;
-  const int8_t* wr = w + m * K;
+  if (gid >= nwords) return;
+  const int64_t block_words = kp / 2;
+  const int64_t rb = gid / block_words, rem = gid % block_words;
+  const int64_t c = rem >> 7, r = (rem >> 4) & 7, j = rem & 15;
+  const int64_t m = rb * 8 + r;
   uint32_t word = 0;
   bool bad = false;
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const int64_t k = 16 * j + i;
-    const int wk = (k < K) ? (int)wr[k] : 0;
-    bad |= !ternary(wk);
-    const int s = i >> 2, b = i & 3;  // k = 16j + 4s + b
-    word |= (uint32_t)((wk + 1) & 3) << (8 * b + 2 * s);
+  for (int s = 0; s < 4; ++s) {
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int64_t k = c * 256 + 32 * (j >> 1) + 8 * s + 4 * (j & 1) + b;
+      const int wk = (m < M && k < K) ? (int)w[m * K + k] : 0;
+      bad |= !ternary(wk);
+      word |= (uint32_t)((wk + 1) & 3) << (8 * b + 2 * s);
+    }
   }
   packed[gid] = word;
   if (bad && dev_status) atomicExch(dev_status, BITNET_ERR_BAD_WEIGHT);
 }
 
-__global__ void unpack_i2s_kernel(const uint32_t* __restrict__ packed, int64_t M, int64_t K,
-                                  int64_t row_words, int8_t* __restrict__ w, int* dev_status) {
+__global__ void unpack_i2s_kernel(const uint32_t* __restrict__ packed, int64_t M, int64_t K, int64_t kp,
+                                  int64_t nwords, int8_t* __restrict__ w, int* dev_status) {
   const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (gid >= M * row_words) return;
-  const int64_t m = gid / row_words, j = gid % row_words;
+  if (gid >= nwords) return;
+  const int64_t block_words = kp / 2;
+  const int64_t rb = gid / block_words, rem = gid % block_words;
+  const int64_t c = rem >> 7, r = (rem >> 4) & 7, j = rem & 15;
+  const int64_t m = rb * 8 + r;
   const uint32_t word = packed[gid];
   bool bad = false;
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const int64_t k = 16 * j + i;
-    const int s = i >> 2, b = i & 3;
-    const int code = (word >> (8 * b + 2 * s)) & 3;
-    bad |= (code == 3);
-    if (k < K) w[m * K + k] = (int8_t)(code - 1);
+  for (int s = 0; s < 4; ++s) {
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int64_t k = c * 256 + 32 * (j >> 1) + 8 * s + 4 * (j & 1) + b;
+      const int code = (word >> (8 * b + 2 * s)) & 3;
+      bad |= (code == 3);
+      if (m < M && k < K) w[m * K + k] = (int8_t)(code - 1);
+    }
   }
   if (bad && dev_status) atomicExch(dev_status, BITNET_ERR_BAD_WEIGHT);
 }
@@ -156,17 +165,17 @@ inline unsigned blocks_for(int64_t n, int threads) { return (unsigned)ceil_div(n
 
 int launch_pack_i2s(const int8_t* w, int64_t M, int64_t K, uint8_t* packed, int* dev_status,
                     cudaStream_t st) {
-  const int64_t row_words = ceil_div(K, 128) * 8;
-  pack_i2s_kernel<<<blocks_for(M * row_words, 256), 256, 0, st>>>(
-      w, M, K, row_words, reinterpret_cast<uint32_t*>(packed), dev_status);
+  const int64_t kp = i2s_kp(K), nwords = i2s_mp(M) * kp / 16;
+  pack_i2s_kernel<<<blocks_for(nwords, 256), 256, 0, st>>>(w, M, K, kp, nwords, reinterpret_cast<uint32_t*>(packed),
+                                                         dev_status);
   return check_launch();
 }
 
 int launch_unpack_i2s(const uint8_t* packed, int64_t M, int64_t K, int8_t* w, int* dev_status,
                       cudaStream_t st) {
-  const int64_t row_words = ceil_div(K, 128) * 8;
-  unpack_i2s_kernel<<<blocks_for(M * row_words, 256), 256, 0, st>>>(
-      reinterpret_cast<const uint32_t*>(packed), M, K, row_words, w, dev_status);
+  const int64_t kp = i2s_kp(K), nwords = i2s_mp(M) * kp / 16;
+  unpack_i2s_kernel<<<blocks_for(nwords, 256), 256, 0, st>>>(reinterpret_cast<const uint32_t*>(packed), M, K, kp,
+                                                           nwords, w, dev_status);
   return check_launch();
 }
 

@@ -35,11 +35,11 @@ __device__ float block_amax(const float* __restrict__ x, int64_t n, float* red) 
   if ((n & 3) == 0 && ((reinterpret_cast<uintptr_t>(x) & 15u) == 0)) {
     const float4* x4 = reinterpret_cast<const float4*>(x);
     for (int64_t i = tid; i < n / 4; i += blockDim.x) {
-      float4 v = x4[i];
+      float4 v = __ldcg(x4 + i);
       m = fmaxf(m, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
     }
   } else {
-    for (int64_t i = tid; i < n; i += blockDim.x) m = fmaxf(m, fabsf(x[i]));
+    for (int64_t i = tid; i < n; i += blockDim.x) m = fmaxf(m, fabsf(__ldcg(x + i)));
   }
   m = warp_max(m);
   if ((tid & 31) == 0) red[tid >> 5] = m;
@@ -74,6 +74,11 @@ quant_act_kernel(const float* __restrict__ x, int64_t K, int8_t* __restrict__ q,
   int8_t* qr = q + t * K;
   const int tid = threadIdx.x;
 
+  // programmatic dependent launch: let the next kernel start its prologue, then wait for the kernel
+  // that produced x (both are no-ops under a plain launch)
+  if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
   float amax;
   if (tensor_amax_bits) {
     amax = __uint_as_float(*tensor_amax_bits);
@@ -89,14 +94,14 @@ quant_act_kernel(const float* __restrict__ x, int64_t K, int8_t* __restrict__ q,
     const float4* x4 = reinterpret_cast<const float4*>(xr);
     char4* q4 = reinterpret_cast<char4*>(qr);
     for (int64_t i = tid; i < K / 4; i += blockDim.x) {
-      float4 v = x4[i];
+      float4 v = __ldcg(x4 + i);
       int a = quant1(v.x, s), b = quant1(v.y, s), c = quant1(v.z, s), d = quant1(v.w, s);
       sum += a + b + c + d;
       q4[i] = make_char4((signed char)a, (signed char)b, (signed char)c, (signed char)d);
     }
   } else {
     for (int64_t i = tid; i < K; i += blockDim.x) {
-      int a = quant1(xr[i], s);
+      int a = quant1(__ldcg(xr + i), s);
       sum += a;
       qr[i] = (int8_t)a;
     }
@@ -138,7 +143,18 @@ int launch_quant_act(const float* x, int64_t T, int64_t K, int per_tensor, int8_
                                                        reinterpret_cast<const unsigned*>(act_scale));
     fill_scale_kernel<<<1, 256, 0, st>>>(act_scale, T);
   } else {
-    quant_act_kernel<<<(unsigned)T, QTHREADS, 0, st>>>(x, K, q, act_scale, act_sum, nullptr);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)T);
+    cfg.blockDim = dim3(QTHREADS);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = early_start_enabled() ? 1 : 0;
+    const unsigned* no_amax = nullptr;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, quant_act_kernel, x, K, q, act_scale, act_sum, no_amax);
+    if (e != cudaSuccess) return note_cuda_error(e);
   }
   return check_launch();
 }
