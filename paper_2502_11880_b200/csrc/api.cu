@@ -69,7 +69,13 @@ int bitnet_last_cuda_error(void) { return g_last_cuda_error; }
 
 int bitnet_device_status(int* status_out) {
   if (!status_out) return BITNET_ERR_INVALID_ARG;
-  return gemv_i2s_stream_status(status_out);
+  int a = 0, b = 0;
+  int rc = gemv_i2s_stream_status(&a);
+  if (rc) return rc;
+  rc = gemm_prefill_status(&b);
+  if (rc) return rc;
+  *status_out = a ? a : b;
+  return BITNET_OK;
 }
 
 void bitnet_set_early_start(int enable) { g_early_start = enable ? 1 : 0; }

@@ -102,4 +102,6 @@ int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int
                             const float* act_scale, int64_t T, float* y, int32_t* acc_out,
                             cudaStream_t st);
 
+int gemm_prefill_status(int* out);
+
 }  // namespace bitnet

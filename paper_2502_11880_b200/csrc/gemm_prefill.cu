@@ -1,7 +1,7 @@
 // Prefill mpGEMM (many tokens), I2_S: Alg. 1 Phase 2 at large T.
 //
-// This file holds the plain dp4a kernel (one thread per output, a reference point for the tensor-core
-// kernel and the path used when BITNET_PREFILL=simt).
+// This file holds the plain dp4a kernel (one thread per output): a reference point for the tensor-core
+// kernel of gemm_prefill_tc.cu and the path taken when BITNET_PREFILL=simt is set in the environment.
 #include <cstdlib>
 #include <cstring>
 
@@ -51,8 +51,8 @@ __global__ void __launch_bounds__(256) gemm_i2s_simt_kernel(const uint8_t* __res
 
 }  // namespace
 
-int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const int8_t* q,
-                            const float* act_scale, int64_t T, float* y, int32_t* acc_out, cudaStream_t st) {
+int launch_gemm_i2s_simt(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const int8_t* q,
+                         const float* act_scale, int64_t T, float* y, int32_t* acc_out, cudaStream_t st) {
   dim3 grid((unsigned)ceil_div(M, 32), (unsigned)ceil_div(T, 8));
   gemm_i2s_simt_kernel<<<grid, dim3(32, 8), 0, st>>>(packed, i2s_kp(K), (int)M, (int)K, q, act_scale, w_scale, (int)T,
                                                     y, acc_out);

@@ -1,0 +1,392 @@
+// Prefill mpGEMM (many tokens), I2_S: Alg. 1 Phase 2 at large T on the int8 tensor cores.
+//
+//   acc[t,m] = sum_k q[t,k] * w[m,k]        (tcgen05.mma kind::i8, s8 x s8 -> s32 in tensor memory)
+//   y[t,m]   = acc[t,m] * act_scale[t] * w_scale
+//
+// The paper does not treat the prefill stage (its Limitations section); the definition is the same
+// as for decode, so the design is this build's.  One persistent CTA per SM walks output tiles of
+// 128 out-features x 256 tokens.  Per 128-column K block:
+//   * warp 0   : one TMA tensor copy brings the 256 x 128 int8 activation tile straight into the
+//                128-byte-swizzled K-major layout the MMA wants (operand B);
+//   * warps 2-5: each thread owns one weight row: it reads the row's 32 packed bytes from the blob
+//                (L2 resident: the whole blob is ~15 MB), expands the 2-bit codes to int8 -1/0/+1 in
+//                registers and writes the row of operand A into shared memory in the same swizzled
+//                layout (8 conflict-free 16-byte stores), then fence.proxy.async + mbarrier arrive;
+//   * warp 1   : one thread issues four tcgen05.mma (M=128, N=256, K=32) per K block, accumulating in
+//                tensor memory, and tcgen05.commit releases the stage to the producers;
+//   * warps 6-9: epilogue -- tcgen05.ld the finished 128 x 256 accumulator (lane = out-feature,
+//                column = token), rescale and store y; a warp's 32 lanes write 32 consecutive
+//                out-features of one token, i.e. 128 contiguous bytes.  Two accumulators (2 x 256 of the
+//                512 tensor-memory columns) let the epilogue of a tile overlap the MMAs of the next.
+// Every mbarrier wait is bounded; a wait that gives up sets a CTA-wide abort flag and the device
+// status word, all roles leave their loops, and the CTA frees its tensor memory before it exits.
+#include <cuda.h>
+
+#include <cstdlib>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace bitnet {
+namespace {
+
+constexpr int TILE_M = 128;     // out-features per tile (MMA M, tensor-memory lanes)
+constexpr int TILE_T = 256;     // tokens per tile (MMA N, tensor-memory columns)
+constexpr int KBLK = 128;       // K columns per pipeline stage = one 128-byte swizzle row of int8
+constexpr int STAGES = 4;
+constexpr int A_BYTES = TILE_M * KBLK;   // 16 KB
+constexpr int B_BYTES = TILE_T * KBLK;   // 32 KB
+constexpr int THREADS = 320;             // warp 0 TMA, warp 1 MMA, warps 2-5 unpack, warps 6-9 epilogue
+constexpr uint32_t WAIT_LIMIT = 1u << 22;
+
+static __device__ int g_prefill_error = 0;
+
+struct PrefillArgs {
+  const uint8_t* packed;
+  int64_t kp;            // K padded to 256 (blob geometry)
+  int M;
+  int K;
+  int T;
+  const float* act_scale;
+  float w_scale;
+  float* y;
+  int32_t* acc_out;
+  int tiles_m, tiles_t, nkb;
+};
+
+struct __align__(8) Barriers {
+  uint64_t full_a[STAGES], full_b[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Bounded wait; false = gave up (or another role already aborted).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  const uint32_t addr = smem_u32(bar);
+  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(addr), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if ((it & 1023u) == 1023u && *abort_flag) return false;
+  }
+  return false;
+}
+
+// Shared-memory matrix descriptor for a K-major operand tile whose rows are 128 bytes, 128-byte
+// swizzle: start address, stride between 8-row groups = 1024 bytes, descriptor version 1.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);          // bits 0-13: start address / 16
+  d |= (uint64_t)1 << 16;                            // bits 16-29: leading byte offset / 16 (unused here)
+  d |= (uint64_t)(1024 >> 4) << 32;                  // bits 32-45: stride byte offset / 16
+  d |= (uint64_t)1 << 46;                            // bits 46-47: descriptor version (tcgen05)
+  d |= (uint64_t)2 << 61;                            // bits 61-63: 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor: D = s32, A = s8, B = s8, both K-major, N = 256, M = 128.
+constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TILE_T >> 3) << 17) |
+                           ((uint32_t)(TILE_M >> 4) << 24);
+
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(IDESC), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+
+// signed bytes (-1, 0, +1) of slot s of a packed word: codes 0,1,2 minus one, without borrows between bytes
+__device__ __forceinline__ uint32_t slot_s8(uint32_t w, int s) {
+  const uint32_t c = ((w >> (2 * s)) & 0x03030303u) | 0x80808080u;
+  return (c - 0x01010101u) ^ 0x80808080u;
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const PrefillArgs a) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* tileA = smem;                               // STAGES x 16 KB
+  uint8_t* tileB = smem + STAGES * A_BYTES;            // STAGES x 32 KB
+  Barriers* bars = reinterpret_cast<Barriers*>(smem + STAGES * (A_BYTES + B_BYTES));
+  volatile int* abort_flag = &bars->abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ntiles = a.tiles_m * a.tiles_t;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&bars->full_a[s], 4);      // one arrival per unpack warp
+      mbar_init(&bars->full_b[s], 1);      // TMA producer (+ transaction bytes)
+      mbar_init(&bars->empty[s], 1);       // tcgen05.commit
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&bars->tmem_full[b], 1);   // tcgen05.commit
+      mbar_init(&bars->tmem_empty[b], 4);  // one arrival per epilogue warp
+    }
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    __syncwarp();
+    // the whole tensor memory of the SM: two 128 x 256 s32 accumulators
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&bars->tmem_base))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = bars->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer: activation tiles (operand B)
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int tile = blockIdx.x; tile < ntiles && !*abort_flag; tile += gridDim.x) {
+        const int t0 = (tile / a.tiles_m) * TILE_T;
+        for (int kb = 0; kb < a.nkb; ++kb, ++it) {
+          const int s = it % STAGES;
+          if (!mbar_wait(&bars->empty[s], ((it / STAGES) & 1u) ^ 1u, abort_flag)) {
+            atomicExch(&g_prefill_error, BITNET_ERR_TIMEOUT);
+            bars->abort_flag = 1;
+            break;
+          }
+          mbar_expect_tx(&bars->full_b[s], B_BYTES);
+          asm volatile(
+              "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+              ::"r"(smem_u32(tileB + s * B_BYTES)), "l"(&qmap), "r"(kb * KBLK), "r"(t0),
+              "r"(smem_u32(&bars->full_b[s]))
+              : "memory");
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t it = 0, nt = 0;
+      for (int tile = blockIdx.x; tile < ntiles && !*abort_flag; tile += gridDim.x, ++nt) {
+        const int buf = nt & 1;
+        bool ok = mbar_wait(&bars->tmem_empty[buf], ((nt >> 1) & 1u) ^ 1u, abort_flag);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t d_tmem = tmem_base + buf * TILE_T;
+        for (int kb = 0; ok && kb < a.nkb; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t par = (it / STAGES) & 1u;
+          ok = mbar_wait(&bars->full_a[s], par, abort_flag) && mbar_wait(&bars->full_b[s], par, abort_flag);
+          if (!ok) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint64_t adesc = make_desc(smem_u32(tileA + s * A_BYTES));
+          const uint64_t bdesc = make_desc(smem_u32(tileB + s * B_BYTES));
+#pragma unroll
+          for (int k4 = 0; k4 < KBLK / 32; ++k4)   // 32 bytes further along K: +2 in the address field
+            umma_i8(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, (kb > 0 || k4 > 0) ? 1u : 0u);
+          umma_commit(&bars->empty[s]);            // stage reusable once these MMAs have read it
+        }
+        if (!ok) {
+          atomicExch(&g_prefill_error, BITNET_ERR_TIMEOUT);
+          bars->abort_flag = 1;
+          break;
+        }
+        umma_commit(&bars->tmem_full[buf]);        // accumulator complete
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------------------ unpackers: weight rows (operand A)
+    const int r = threadIdx.x - 64;                // row of the tile, 0..127
+    uint32_t it = 0;
+    for (int tile = blockIdx.x; tile < ntiles && !*abort_flag; tile += gridDim.x) {
+      const int m = (tile % a.tiles_m) * TILE_M + r;
+      const bool row_ok = m < a.M;
+      const uint8_t* rowp = a.packed + i2s_row_chunk_offset(row_ok ? m : 0, 0, a.kp);
+      uint4 nx0 = make_uint4(0x55555555u, 0x55555555u, 0x55555555u, 0x55555555u), nx1 = nx0;   // code 1 = weight 0
+      if (row_ok) {
+        nx0 = __ldg(reinterpret_cast<const uint4*>(rowp));
+        nx1 = __ldg(reinterpret_cast<const uint4*>(rowp) + 1);
+      }
+      bool ok = true;
+      for (int kb = 0; kb < a.nkb; ++kb, ++it) {
+        const uint4 c0 = nx0, c1 = nx1;
+        if (row_ok && kb + 1 < a.nkb) {
+          // K block kb+1 = half (kb+1)&1 of chunk (kb+1)/2: 32 bytes of this row
+          const uint4* np = reinterpret_cast<const uint4*>(rowp + (int64_t)((kb + 1) >> 1) * 512 + ((kb + 1) & 1) * 32);
+          nx0 = __ldg(np);
+          nx1 = __ldg(np + 1);
+        }
+        const int s = it % STAGES;
+        if (!mbar_wait(&bars->empty[s], ((it / STAGES) & 1u) ^ 1u, abort_flag)) {
+          ok = false;
+          break;
+        }
+        const uint32_t w[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+        uint8_t* rowA = tileA + s * A_BYTES + (r >> 3) * 1024 + (r & 7) * 128;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          // 16 consecutive columns 16c..16c+15 of the block: words 2P, 2P+1 (P = c/2), slots 2h, 2h+1 (h = c%2)
+          const uint32_t w0 = w[2 * (c >> 1)], w1 = w[2 * (c >> 1) + 1];
+          const int h = c & 1;
+          const uint4 o = make_uint4(slot_s8(w0, 2 * h), slot_s8(w1, 2 * h), slot_s8(w0, 2 * h + 1), slot_s8(w1, 2 * h + 1));
+          *reinterpret_cast<uint4*>(rowA + ((c ^ (r & 7)) << 4)) = o;
+        }
+        // make the generic-proxy stores visible to the tensor core (async proxy), then signal
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->full_a[s]);
+      }
+      if (!ok) {
+        atomicExch(&g_prefill_error, BITNET_ERR_TIMEOUT);
+        bars->abort_flag = 1;
+        break;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue
+    const int quarter = warp & 3;                  // tensor-memory lanes 32*quarter .. 32*quarter+31
+    uint32_t nt = 0;
+    for (int tile = blockIdx.x; tile < ntiles && !*abort_flag; tile += gridDim.x, ++nt) {
+      const int buf = nt & 1;
+      const int m = (tile % a.tiles_m) * TILE_M + quarter * 32 + lane;
+      const int t0 = (tile / a.tiles_m) * TILE_T;
+      if (!mbar_wait(&bars->tmem_full[buf], (nt >> 1) & 1u, abort_flag)) {
+        atomicExch(&g_prefill_error, BITNET_ERR_TIMEOUT);
+        bars->abort_flag = 1;
+        break;
+      }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * TILE_T;
+#pragma unroll 1
+      for (int c0 = 0; c0 < TILE_T; c0 += 32) {
+        uint32_t v[32];
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+            "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+            "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+              "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+              "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+              "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+            : "r"(taddr + c0)
+            : "memory");
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (m < a.M) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int t = t0 + c0 + j;
+            if (t < a.T) {
+              const int acc = (int)v[j];
+              a.y[(int64_t)t * a.M + m] = __fmul_rn((float)acc, __fmul_rn(__ldg(a.act_scale + t), a.w_scale));
+              if (a.acc_out) a.acc_out[(int64_t)t * a.M + m] = acc;
+            }
+          }
+        }
+      }
+      // the accumulator has been read: hand the buffer back to the MMA issuer
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);
+    }
+  }
+
+  // ---- teardown: every role has left its loop (all waits are bounded); free the tensor memory
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+}  // namespace
+
+int launch_gemm_i2s_simt(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const int8_t* q,
+                         const float* act_scale, int64_t T, float* y, int32_t* acc_out, cudaStream_t st);
+
+int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const int8_t* q,
+                            const float* act_scale, int64_t T, float* y, int32_t* acc_out, cudaStream_t st) {
+  static const bool force_simt = [] {
+    const char* e = getenv("BITNET_PREFILL");
+    return e && strcmp(e, "simt") == 0;
+  }();
+  if (force_simt) return launch_gemm_i2s_simt(packed, w_scale, M, K, q, act_scale, T, y, acc_out, st);
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return note_cuda_error(cudaErrorNotSupported);
+  CUtensorMap qmap;
+  const cuuint64_t gdim[2] = {(cuuint64_t)K, (cuuint64_t)T};
+  const cuuint64_t gstride[1] = {(cuuint64_t)K};            // bytes between token rows
+  const cuuint32_t box[2] = {KBLK, TILE_T};
+  const cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(&qmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(q), gdim, gstride, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return note_cuda_error(cudaErrorInvalidValue);
+
+  PrefillArgs a;
+  a.packed = packed;
+  a.kp = i2s_kp(K);
+  a.M = (int)M;
+  a.K = (int)K;
+  a.T = (int)T;
+  a.act_scale = act_scale;
+  a.w_scale = w_scale;
+  a.y = y;
+  a.acc_out = acc_out;
+  a.tiles_m = (int)ceil_div(M, TILE_M);
+  a.tiles_t = (int)ceil_div(T, TILE_T);
+  a.nkb = (int)(a.kp / KBLK);
+  const size_t smem = (size_t)STAGES * (A_BYTES + B_BYTES) + sizeof(Barriers) + 1024;
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (!attr_set[dev & 63]) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_i2s_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return note_cuda_error(e);
+    attr_set[dev & 63] = true;
+  }
+  int grid = dev_info().sm_count;
+  const int ntiles = a.tiles_m * a.tiles_t;
+  if (grid > ntiles) grid = ntiles;
+  gemm_i2s_tc_kernel<<<grid, THREADS, smem, st>>>(qmap, a);
+  return check_launch();
+}
+
+int gemm_prefill_status(int* out) {
+  cudaError_t e = cudaMemcpyFromSymbol(out, g_prefill_error, sizeof(int));
+  return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
+}
+
+}  // namespace bitnet
