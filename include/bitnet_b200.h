@@ -120,9 +120,11 @@ int bitnet_pack_tl(bitnet_fmt_t fmt, const int8_t* w, int64_t M, int64_t K, int 
  *   packed   blob from the packer of `fmt` for an M x K matrix (bk3 as given to the packer);
  *   q[T][K]  int8, act_scale[T] fp32 from bitnet_quant_act;
  *   y[T][M]  fp32 out; acc_out[T][M] int32 out, nullable (raw accumulators);
- *   workspace  bitnet_mpgemm_workspace_bytes(fmt,T,M,K) bytes (may be NULL when that is 0).
- *              It must have been zeroed once with bitnet_workspace_init and is left zeroed by
- *              every completed call; two calls sharing a workspace must not overlap on the GPU.
+ *   workspace  bitnet_mpgemm_workspace_bytes(fmt,T,M,K) bytes (may be NULL when that is 0: I2_S needs
+ *              none except for extreme shapes; TL keeps its lookup tables and split-K sums there).
+ *              It must have been zeroed once with bitnet_workspace_init and its head (the sums) is
+ *              left zeroed by every completed call; two calls sharing a workspace must not overlap
+ *              on the GPU.
  * T <= 8 runs the decode GEMV kernels; larger T runs the int8 tensor-core kernel (I2_S) or the
  * GEMV kernel over groups of 8 tokens (TL).
  */
@@ -163,19 +165,21 @@ int bitnet_linear_host(bitnet_fmt_t fmt, const void* packed, float w_scale, int6
  * exists for the sake of callers, not of the method).
  *
  * Same operation and arguments as bitnet_mpgemm for fmt = BITNET_FMT_TL1 / BITNET_FMT_TL2 and
- * T <= 8, but the scratch that joins the K-slices lives in a fixed array inside the library
- * (BITNET_NOALLOC_MAX_M rows x 9 words = 2.25 MiB, held by every GPU that loads the library until
- * the process exits).  It is meant for hosts that cannot call cudaMalloc or hand over a workspace:
+ * T <= 8, but the scratch (the per-token lookup tables and the sums that join the K-slices) lives in
+ * a fixed array inside the library (5.1 MiB, held by every GPU that loads the library until the
+ * process exits).  It is meant for hosts that cannot call cudaMalloc or hand over a workspace:
  * code running while the device allocator is frozen or its pool is fully committed to weights,
  * latency-critical loops that must not make calls which can block or fail, and plug-ins that
  * receive input and output buffers only.  The call itself allocates nothing, on host or device.
- *   - M > BITNET_NOALLOC_MAX_M or T > 8 returns BITNET_ERR_WORKSPACE and launches nothing.
+ *   - M > BITNET_NOALLOC_MAX_M, K > BITNET_NOALLOC_MAX_K or T > 8 returns BITNET_ERR_WORKSPACE and
+ *     launches nothing.
  *   - The first call on each device looks up the array's device address (a blocking runtime query);
  *     make that first call outside any stream capture.
  *   - Every call on a device shares the one array and clears the part it needs first, on `stream`;
  *     two calls that may run on the GPU at the same time (different streams) race on it.
  */
-#define BITNET_NOALLOC_MAX_M 65536
+#define BITNET_NOALLOC_MAX_M 32768
+#define BITNET_NOALLOC_MAX_K 32768
 int bitnet_mpgemv_tl_noalloc(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M, int64_t K,
                              int bk3, const int8_t* q, const float* act_scale, int64_t T, float* y,
                              int32_t* acc_out, void* stream);

@@ -275,7 +275,8 @@ def bitnet_linear_host(fmt, packed, w_scale, M, K, x_host, y_host, x_dev, q_dev,
                                     _ptr(workspace), ws_bytes, _stream(stream)), "bitnet_linear_host")
 
 
-NOALLOC_MAX_M = 65536
+NOALLOC_MAX_M = 32768
+NOALLOC_MAX_K = 32768
 
 
 def bitnet_mpgemv_tl_noalloc(fmt, packed, w_scale, M, K, q, act_scale, y, acc_out=None, bk3=0, stream=None):

@@ -74,7 +74,10 @@ int bitnet_device_status(int* status_out) {
   if (rc) return rc;
   rc = gemm_prefill_status(&b);
   if (rc) return rc;
-  *status_out = a ? a : b;
+  int c = 0;
+  rc = gemv_tl_status(&c);
+  if (rc) return rc;
+  *status_out = a ? a : (b ? b : c);
   return BITNET_OK;
 }
 

@@ -103,5 +103,6 @@ int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int
                             cudaStream_t st);
 
 int gemm_prefill_status(int* out);
+int gemv_tl_status(int* out);
 
 }  // namespace bitnet

@@ -1,20 +1,25 @@
-// TL1 / TL2 mpGEMV for decode (1..8 tokens): element-wise LUT mpGEMM, Alg. 2 with the tables of
+// TL1 / TL2 mpGEMV for decode (1..8 tokens): element-wise LUT mpGEMM, Alg. 2, with the tables of
 // Alg. 3 (pairs, 9 sums) and Alg. 4 (triples, 14 sums after mirror consolidation); Eq. 3:
 //     acc = sum over groups of Lookup(LUT_group, index), the sign bit of a triple negating the value.
 //
-// A CTA owns a K-slice (a run of 32-group tiles).  Phase 1 ("PreCompute"): it stages the slice of the
-// token's int8 activations in shared memory and builds, for every group, a 16-slot table of partial
-// sums in shared memory -- slot i of a triple table is d0*a0 + d1*a1 + d2*a2 with (d0,d1,d2) the
-// balanced-ternary digits of i, slot i of a pair table is (i/3-1)*a0 + (i%3-1)*a1.  Sums stay exact
-// (|sum| <= 384), as in the lossless TL*_1 variants.  Two tokens share one 32-bit slot as
-// hi*65536 + lo: integer add and negate act on both halves at once, so a lookup serves two tokens.
-// Phase 2: lanes are rows.  A warp takes one tile of a 32-row block: every lane reads its row's 16
-// index bytes (+ 4 sign bytes) with one coalesced request per plane and resolves its 32 nibbles
-// against the SAME group table -- 16 slots in 16 distinct banks, so the lookups never conflict.  The
-// conditional negate is (v ^ m) with m = 0 / -1 from the sign bit, the "+1" of two's complement
-// negation being added once per tile as popcount(sign word).  Warps of a CTA cover different tiles;
-// their per-row sums meet in shared memory, and K-slices of different CTAs meet in an int32
-// workspace by atomicAdd, finalised by whichever slice arrives last (no waiting).
+// Phase 1 ("Table-setup" / "PreCompute"): a small kernel enumerates, for every group of the token's
+// int8 activations, the 16-slot table of partial sums -- slot i of a triple table is
+// d0*a0 + d1*a1 + d2*a2 with (d0,d1,d2) the balanced-ternary digits of i, slot i of a pair table is
+// (i/3-1)*a0 + (i%3-1)*a1 -- once, into the workspace (it is the same for every output row; building
+// it in every CTA would cost as much as the lookups of ~16 rows).  Sums stay exact (|sum| <= 384), as
+// in the lossless TL*_1 variants.  Two tokens share one 32-bit slot as hi*65536 + lo: integer add and
+// negate act on both halves at once, so one lookup serves two tokens.
+//
+// Phase 2 (accumulation).  A CTA owns a K-slice (a run of 32-group tiles) and copies the slice of
+// the tables into shared memory with one bulk asynchronous copy.  Lanes are rows: a warp takes one
+// tile of a 32-row block, every lane reads its row's 16 index bytes (+ 4 sign bytes) with one
+// coalesced request per plane (the next tile's words are requested before the current tile is
+// processed) and resolves its 32 nibbles against the SAME group table -- 16 slots in 16 distinct
+// banks, so lookups never conflict.  The conditional negate is v ^ m with m = 0 / -1 taken from the
+// sign bit by one bit-field extract; the "+1" of two's-complement negation is added once per tile as
+// popcount(sign word).  Warps of a CTA cover different tiles; their per-row sums meet in shared
+// memory, and K-slices of different CTAs meet in an int32 workspace by atomicAdd, finalised by
+// whichever slice arrives last (no waiting).
 #include "common.cuh"
 
 namespace bitnet {
@@ -22,17 +27,20 @@ namespace {
 
 constexpr int WARPS = 8;
 constexpr int THREADS = WARPS * 32;
-constexpr int MAX_SLICE_TILES = 48;  // 2 KB of tables per tile
+constexpr int MAX_SLICE_TILES = 48;   // 2 KB of tables per tile and token pair -> 96 KB, two CTAs per SM
+constexpr uint32_t WAIT_LIMIT = 1u << 22;
+
+static __device__ int g_tl_error = 0;
 
 struct TlArgs {
   const uint8_t* packed;
   TlGeom g;
   int M;
   int64_t K;
-  const int8_t* q;  // first token of the pass
+  const int* table;  // [tiles][32 groups][16 slots] of this token pair
   const float* act_scale;
   float w_scale;
-  int nt;           // tokens in this pass (1 or 2)
+  int nt;            // tokens in this pass (1 or 2)
   float* y;
   int32_t* acc_out;
   int32_t* ws_acc;
@@ -78,10 +86,38 @@ __device__ __forceinline__ void group_acts(const TlGeom& g, int64_t K, const int
   }
 }
 
+// Phase 1: one thread per table slot; blockIdx.y = token pair.  table[pair][slot] = lo + 65536 * hi.
+__global__ void tl_table_kernel(const int8_t* __restrict__ q, int T, int64_t K, TlGeom g, int* __restrict__ table,
+                                int64_t nslots) {
+  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= nslots) return;
+  const int i = (int)(e & 15), grp = (int)((e >> 4) & 31);
+  const int tile = (int)(e >> 9);
+  const int t0 = 2 * blockIdx.y;
+  bool is3;
+  int a0, a1, a2;
+  group_acts(g, K, q + (int64_t)t0 * K, tile, grp, &is3, &a0, &a1, &a2);
+  int v = lut_entry(is3, i, a0, a1, a2);
+  if (t0 + 1 < T) {
+    group_acts(g, K, q + (int64_t)(t0 + 1) * K, tile, grp, &is3, &a0, &a1, &a2);
+    v += lut_entry(is3, i, a0, a1, a2) * 65536;
+  }
+  table[(int64_t)blockIdx.y * nslots + e] = v;
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ int sign_mask(unsigned sg, int bit) {   // 0 or -1 from one bit
+  int m;
+  asm("bfe.s32 %0, %1, %2, 1;" : "=r"(m) : "r"(sg), "r"(bit));
+  return m;
+}
+
 __global__ void __launch_bounds__(THREADS, 2) gemv_tl_kernel(const TlArgs a) {
-  extern __shared__ __align__(16) int smem[];
+  extern __shared__ __align__(128) int smem[];
   int* tab = smem;                                   // [tiles_per_slice][32][16]
   int* red = smem + a.tiles_per_slice * 512;         // [WARPS][32][2]
+  uint64_t* bar = reinterpret_cast<uint64_t*>(red + WARPS * 64);
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int slice = blockIdx.y;
@@ -89,55 +125,97 @@ __global__ void __launch_bounds__(THREADS, 2) gemv_tl_kernel(const TlArgs a) {
   const int tile0 = slice * a.tiles_per_slice;
   const int ntiles = min(a.tiles_per_slice, tiles_total - tile0);
 
-  // ---- Phase 1: tables of this slice.  One thread per table slot; consecutive threads write
-  // consecutive words.
-  for (int e = threadIdx.x; e < ntiles * 512; e += THREADS) {
-    const int i = e & 15, grp = (e >> 4) & 31, tl = e >> 9;
-    bool is3;
-    int a0, a1, a2;
-    group_acts(a.g, a.K, a.q, tile0 + tl, grp, &is3, &a0, &a1, &a2);
-    int v = lut_entry(is3, i, a0, a1, a2);
-    if (a.nt == 2) {
-      group_acts(a.g, a.K, a.q + a.K, tile0 + tl, grp, &is3, &a0, &a1, &a2);
-      v += lut_entry(is3, i, a0, a1, a2) * 65536;
-    }
-    tab[e] = v;
+  // ---- the tables of this slice: one bulk copy global -> shared
+  if (threadIdx.x == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(bar)) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const uint32_t bytes = (uint32_t)ntiles * 2048u;
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(tab)), "l"(a.table + (int64_t)tile0 * 512), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
   }
   __syncthreads();
+  {
+    bool got = false;
+    for (uint32_t it = 0; it < WAIT_LIMIT && !got; ++it) {
+      uint32_t ok;
+      asm volatile(
+          "{\n\t.reg .pred p;\n\t"
+          "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
+          "selp.u32 %0, 1, 0, p;\n\t}"
+          : "=r"(ok)
+          : "r"(smem_u32(bar))
+          : "memory");
+      got = ok != 0;
+    }
+    if (!got) {
+      if (threadIdx.x == 0) atomicExch(&g_tl_error, BITNET_ERR_TIMEOUT);
+      return;
+    }
+  }
 
   const float sc0 = __fmul_rn(a.act_scale[0], a.w_scale);
   const float sc1 = (a.nt == 2) ? __fmul_rn(a.act_scale[1], a.w_scale) : 0.0f;
+  const int64_t t3bytes = a.g.tiles3 * 640;
 
-  // ---- Phase 2: lookups.
-  for (int rb = blockIdx.x; rb < a.M / 32; rb += gridDim.x) {
+  // ---- Phase 2: lookups.  The warp's work list is (row block, tile) pairs; the next pair's index and
+  // sign words are requested before the current pair is processed.
+  auto tile_ptr = [&](int rb, int tl) -> const uint8_t* {
+    const int tile = tile0 + tl;
     const uint8_t* blk = a.packed + (int64_t)rb * a.g.block_bytes;
+    return (tile < a.g.tiles3) ? blk + (int64_t)tile * 640 : blk + t3bytes + (int64_t)(tile - a.g.tiles3) * 512;
+  };
+  const int nrb = a.M / 32;
+  int rb = blockIdx.x, tl = warp;
+  uint4 iw = make_uint4(0, 0, 0, 0);
+  unsigned sg = 0;
+  bool have = rb < nrb && tl < ntiles;
+  if (have) {
+    const uint8_t* tp = tile_ptr(rb, tl);
+    iw = __ldg(reinterpret_cast<const uint4*>(tp) + lane);
+    sg = (tile0 + tl < a.g.tiles3) ? __ldg(reinterpret_cast<const unsigned*>(tp + 512) + lane) : 0u;
+  }
+  for (; rb < nrb; rb += gridDim.x) {
     int lo = 0, hi = 0;
-    for (int tl = warp; tl < ntiles; tl += WARPS) {
-      const int tile = tile0 + tl;
-      const bool is3 = tile < a.g.tiles3;
-      const uint8_t* tp = is3 ? blk + (int64_t)tile * 640
-                              : blk + a.g.tiles3 * 640 + (int64_t)(tile - a.g.tiles3) * 512;
-      const uint4 iw = __ldg(reinterpret_cast<const uint4*>(tp) + lane);
-      const unsigned sg = is3 ? __ldg(reinterpret_cast<const unsigned*>(tp + 512) + lane) : 0u;
-      const unsigned words[4] = {iw.x, iw.y, iw.z, iw.w};
-      const int* tt = tab + tl * 512;
-      int s = __popc(sg);  // the +1 of every two's-complement negation below, for both halves at once
+    while (tl < ntiles) {
+      const uint4 ciw = iw;
+      const unsigned csg = sg;
+      const int ctl = tl;
+      // next element of the work list: the next tile of this row block, else this warp's first tile of
+      // the CTA's next row block
+      int nrbi = rb, ntl = tl + WARPS;
+      if (ntl >= ntiles) {
+        nrbi = rb + gridDim.x;
+        ntl = warp;
+      }
+      if (nrbi < nrb && ntl < ntiles) {
+        const uint8_t* tp = tile_ptr(nrbi, ntl);
+        iw = __ldg(reinterpret_cast<const uint4*>(tp) + lane);
+        sg = (tile0 + ntl < a.g.tiles3) ? __ldg(reinterpret_cast<const unsigned*>(tp + 512) + lane) : 0u;
+      }
+      const unsigned words[4] = {ciw.x, ciw.y, ciw.z, ciw.w};
+      const char* tt = reinterpret_cast<const char*>(tab + ctl * 512);
+      int s = __popc(csg);   // the +1 of every two's-complement negation below, for both halves at once
 #pragma unroll
       for (int w4 = 0; w4 < 4; ++w4) {
 #pragma unroll
         for (int n = 0; n < 8; ++n) {
           const int grp = w4 * 8 + n;
-          const int idx = (words[w4] >> (4 * n)) & 15;
-          const int v = tt[grp * 16 + idx];
-          const int m = -(int)((sg >> grp) & 1u);
-          s += v ^ m;
+          // byte offset of the slot: 4 * nibble n of the word
+          const unsigned off = (n == 0) ? ((words[w4] << 2) & 0x3Cu) : ((words[w4] >> (4 * n - 2)) & 0x3Cu);
+          const int v = *reinterpret_cast<const int*>(tt + grp * 64 + off);
+          s += v ^ sign_mask(csg, grp);
         }
       }
       // split the packed pair: s = H * 65536 + L with |L| < 32768
       const int l16 = (int)(short)(s & 0xFFFF);
       lo += l16;
       hi += (s - l16) >> 16;
+      tl += WARPS;
+      if (tl >= ntiles) break;
     }
+    tl = warp;
     red[(warp * 32 + lane) * 2 + 0] = lo;
     red[(warp * 32 + lane) * 2 + 1] = hi;
     __syncthreads();
@@ -196,22 +274,37 @@ inline void slicing(const TlGeom& g, int* nslices, int* tiles_per_slice) {
   *tiles_per_slice = (tiles + *nslices - 1) / *nslices;
 }
 
+// bytes of the accumulator/ticket area and of the table area of the workspace (upper bounds that do
+// not depend on bk3: no format has more than K/64 + 2 tiles)
+inline size_t acc_area_bytes(int64_t T, int64_t M) { return (size_t)((T * M + M) * 4 + 255) & ~(size_t)255; }
+inline size_t table_area_bytes(int64_t T, int64_t K) { return (size_t)((T + 1) / 2) * (size_t)(K / 64 + 2) * 2048; }
+
 }  // namespace
 
 size_t gemv_tl_workspace_bytes(int fmt, int64_t T, int64_t M, int64_t K) {
   TlGeom g;
   if (!tl_geom(fmt, M, K, 0, &g)) return 0;
-  int ns, tps;
-  slicing(g, &ns, &tps);
-  if (ns == 1) return 0;
   const int64_t Tc = T > 8 ? 8 : T;
-  return (size_t)(Tc * M * 4 + M * 4);
+  return acc_area_bytes(Tc, M) + table_area_bytes(Tc, K);
 }
 
 int launch_gemv_tl(int fmt, const uint8_t* packed, float w_scale, int64_t M, int64_t K, const TlGeom& g,
                    const int8_t* q, const float* act_scale, int T, float* y, int32_t* acc_out, void* ws,
                    size_t ws_bytes, cudaStream_t st) {
   (void)fmt;
+  const int64_t tiles = g.tiles3 + g.tiles2;
+  const size_t acc_bytes = acc_area_bytes(T, M);
+  const int npairs = (T + 1) / 2;
+  if (!ws || ws_bytes < acc_bytes + (size_t)npairs * (size_t)tiles * 2048) return BITNET_ERR_WORKSPACE;
+  int* table = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(ws) + acc_bytes);
+
+  // Phase 1: tables of every token pair
+  const int64_t nslots = tiles * 512;
+  tl_table_kernel<<<dim3((unsigned)ceil_div(nslots, 256), (unsigned)npairs), 256, 0, st>>>(q, T, K, g, table, nslots);
+  int rc = check_launch();
+  if (rc != BITNET_OK) return rc;
+
+  // Phase 2: lookups, one launch per token pair
   TlArgs a;
   a.packed = packed;
   a.g = g;
@@ -219,34 +312,30 @@ int launch_gemv_tl(int fmt, const uint8_t* packed, float w_scale, int64_t M, int
   a.K = K;
   a.w_scale = w_scale;
   slicing(g, &a.nslices, &a.tiles_per_slice);
-  if (a.nslices > 1) {
-    if (!ws || ws_bytes < (size_t)((int64_t)T * M * 4 + M * 4)) return BITNET_ERR_WORKSPACE;
-    a.ws_ticket = reinterpret_cast<unsigned*>(reinterpret_cast<int32_t*>(ws) + (int64_t)T * M);
-  } else {
-    a.ws_ticket = nullptr;
-  }
-  const size_t smem = (size_t)a.tiles_per_slice * 2048 + WARPS * 32 * 2 * sizeof(int);
+  a.ws_ticket = reinterpret_cast<unsigned*>(reinterpret_cast<int32_t*>(ws) + (int64_t)T * M);
+  const size_t smem = (size_t)a.tiles_per_slice * 2048 + WARPS * 64 * sizeof(int) + 16;
   static bool attr_set[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
   if (!attr_set[dev & 63]) {
     cudaError_t e = cudaFuncSetAttribute(gemv_tl_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         MAX_SLICE_TILES * 2048 + WARPS * 32 * 2 * (int)sizeof(int));
+                                         MAX_SLICE_TILES * 2048 + WARPS * 64 * (int)sizeof(int) + 16);
     if (e != cudaSuccess) return note_cuda_error(e);
     attr_set[dev & 63] = true;
   }
   const int sms = dev_info().sm_count;
   int gx = (2 * sms + a.nslices - 1) / a.nslices;
   if (gx > (int)(M / 32)) gx = (int)(M / 32);
-  for (int t0 = 0; t0 < T; t0 += 2) {
-    a.q = q + (int64_t)t0 * K;
+  for (int p = 0; p < npairs; ++p) {
+    const int t0 = 2 * p;
+    a.table = table + (int64_t)p * nslots;
     a.act_scale = act_scale + t0;
     a.nt = (T - t0 >= 2) ? 2 : 1;
     a.y = y + (int64_t)t0 * M;
     a.acc_out = acc_out ? acc_out + (int64_t)t0 * M : nullptr;
-    a.ws_acc = (a.nslices > 1) ? reinterpret_cast<int32_t*>(ws) + (int64_t)t0 * M : nullptr;
+    a.ws_acc = reinterpret_cast<int32_t*>(ws) + (int64_t)t0 * M;
     gemv_tl_kernel<<<dim3((unsigned)gx, (unsigned)a.nslices), THREADS, smem, st>>>(a);
-    int rc = check_launch();
+    rc = check_launch();
     if (rc != BITNET_OK) return rc;
   }
   return BITNET_OK;
@@ -258,6 +347,11 @@ int launch_tl_build_lut(int fmt, const int8_t* q_row, int64_t K, const TlGeom& g
   const int64_t nslots = (g.tiles3 + g.tiles2) * 512;
   tl_build_lut_kernel<<<(unsigned)ceil_div(nslots, 256), 256, 0, st>>>(q_row, K, g, lut, nslots);
   return check_launch();
+}
+
+int gemv_tl_status(int* out) {
+  cudaError_t e = cudaMemcpyFromSymbol(out, g_tl_error, sizeof(int));
+  return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
 }
 
 }  // namespace bitnet

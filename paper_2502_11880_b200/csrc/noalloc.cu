@@ -13,10 +13,13 @@
 namespace bitnet {
 namespace {
 
-// Partial sums [T<=8][M] int32 followed by one arrival counter per row, for M up to the stated limit.
+// Partial sums [T<=8][M] int32, one arrival counter per row, then the lookup tables of up to four
+// token pairs (2 KB per 32-group tile), for M and K up to the stated limits.
 constexpr int64_t kNoAllocMaxM = BITNET_NOALLOC_MAX_M;
+constexpr int64_t kNoAllocMaxK = BITNET_NOALLOC_MAX_K;
 constexpr int64_t kNoAllocMaxT = 8;
-constexpr size_t kScratchBytes = (size_t)(kNoAllocMaxT + 1) * 4 * kNoAllocMaxM;
+constexpr size_t kScratchBytes =
+    (size_t)(kNoAllocMaxT + 1) * 4 * kNoAllocMaxM + 4 * (size_t)(kNoAllocMaxK / 64 + 2) * 2048;
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
 
@@ -52,17 +55,19 @@ extern "C" int bitnet_mpgemv_tl_noalloc(bitnet_fmt_t fmt, const void* packed, fl
   if (!packed || !q || !act_scale || !y || T < 1 || M < 1 || K < 1) return BITNET_ERR_INVALID_ARG;
   if (!aligned16(packed) || !aligned16(q) || !aligned16(y) || (acc_out && !aligned16(acc_out)))
     return BITNET_ERR_INVALID_ARG;
-  if (M > kNoAllocMaxM || T > kNoAllocMaxT) return BITNET_ERR_WORKSPACE;  // beyond the built-in scratch
+  if (M > kNoAllocMaxM || K > kNoAllocMaxK || T > kNoAllocMaxT) return BITNET_ERR_WORKSPACE;  // beyond the scratch
   TlGeom g;
   if (!tl_geom(fmt, M, K, bk3, &g)) return BITNET_ERR_UNSUPPORTED_SHAPE;
   void* scratch = nullptr;
   int rc = scratch_address(&scratch);
   if (rc != BITNET_OK) return rc;
   cudaStream_t st = (cudaStream_t)stream;
-  // The array keeps whatever the previous call left; partial sums and arrival counters must start at 0.
-  const size_t need = (size_t)(T + 1) * 4 * (size_t)M;
-  cudaError_t e = cudaMemsetAsync(scratch, 0, need, st);
+  const size_t need = gemv_tl_workspace_bytes(fmt, T, M, K);
+  if (need > kScratchBytes) return BITNET_ERR_WORKSPACE;
+  // The array keeps whatever the previous call left; partial sums and arrival counters must start at 0
+  // (the tables behind them are rewritten in full by every call).
+  cudaError_t e = cudaMemsetAsync(scratch, 0, (size_t)(T + 1) * 4 * (size_t)M, st);
   if (e != cudaSuccess) return note_cuda_error(e);
   return launch_gemv_tl(fmt, (const uint8_t*)packed, w_scale, M, K, g, q, act_scale, (int)T, y, acc_out, scratch,
-                        need, st);
+                        kScratchBytes, st);
 }

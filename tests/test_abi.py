@@ -72,6 +72,7 @@ def test_host_validation_returns_codes_without_a_gpu(L):
     assert L.bitnet_mpgemm(0, fake, 1.0, 64, 128, 0, odd, fake, 1, fake, null, null, 0, null) == 1
     # split-K shape without a workspace
     assert L.bitnet_mpgemm(2, fake, 1.0, 64, 28672, 0, fake, fake, 1, fake, null, null, 0, null) == 3
+    assert L.bitnet_mpgemm(1, fake, 1.0, 32, 64, 0, fake, fake, 1, fake, null, fake, 16, null) == 3   # too small
     assert L.bitnet_mpgemm(0, fake, 1.0, 1 << 22, 1 << 17, 0, fake, fake, 1, fake, null, null, 0, null) == 3
 
 

@@ -129,7 +129,8 @@ def test_constant_weights_and_workspace_reuse(fmt):
         expect = np.repeat((val * sm_ref.astype(np.int64))[:, None], M, axis=1).astype(np.int32)
         assert np.array_equal(npy(out["acc"]), expect)
         check_y(out["y"], expect, sc_ref, 0.5)
-    assert ws is None or not npy(ws).any()
+    # the head of the workspace (split-K sums and arrival counters) must come back zeroed
+    assert ws is None or not npy(ws)[: (T * M + M) * 4].any()
 
 
 def test_i2s_very_long_k_runs_in_phases():

@@ -48,6 +48,8 @@ def test_noalloc_rejects_sizes_beyond_its_scratch():
     y = torch.empty((1, 32), dtype=torch.float32, device="cuda")
     with pytest.raises(bn.BitnetError, match="workspace"):
         bn.bitnet_mpgemv_tl_noalloc("tl2", blob, 1.0, bn.NOALLOC_MAX_M + 32, 96, q, sc, y)
+    with pytest.raises(bn.BitnetError, match="workspace"):
+        bn.bitnet_mpgemv_tl_noalloc("tl2", blob, 1.0, 32, bn.NOALLOC_MAX_K + 96, q, sc, y)
     q9 = torch.zeros((9, 96), dtype=torch.int8, device="cuda")
     sc9 = torch.ones(9, dtype=torch.float32, device="cuda")
     y9 = torch.empty((9, 32), dtype=torch.float32, device="cuda")
