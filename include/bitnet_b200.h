@@ -82,13 +82,13 @@ int bitnet_quant_act(const float* x, int64_t T, int64_t K, int per_tensor, int8_
 /*
  * I2_S weight packer -- I2_S of Table 1 / Sec. 3.2.2 (2 bits per weight; the scale stays outside).
  *   w[M][K] int8 in {-1,0,+1}, row-major (read) -> packed, bitnet_i2s_packed_bytes(M,K) bytes.
- * Layout (code = w+1 in two bits; padding holds weight 0): rows in blocks of 8 (M padded to a
- * multiple of 8), K padded to a multiple of 256.  A block is contiguous: for each chunk c of 256
- * columns it holds 512 bytes, of which row r of the block owns bytes [64r, 64r+64) = 16 little-endian
+ * Layout (code = w+1 in two bits; padding holds weight 0): rows in blocks of 16 (M padded to a
+ * multiple of 16), K padded to a multiple of 256.  A block is contiguous: for each chunk c of 256
+ * columns it holds 1024 bytes, of which row r of the block owns bytes [64r, 64r+64) = 16 little-endian
  * words.  Column kk = k % 256 of a chunk sits in word j = 2*(kk/32) + (kk%8)/4, byte b = kk%4, bits
- * [2s, 2s+1] with s = (kk%32)/8.  (One 8-row block of up to 8192 columns is one contiguous 16 KB piece
- * for a bulk copy; 32 lanes reading 16 bytes each cover 8 rows x 64 bytes without bank conflicts; the
- * two activation words an int8 MMA needs for words 2h, 2h+1 are adjacent.)
+ * [2s, 2s+1] with s = (kk%32)/8.  (Any K-slab of a 16-row block -- the tile of one int8 MMA -- is one
+ * contiguous piece for a bulk copy; 32 lanes reading 16 bytes each cover 8 rows x 64 bytes without
+ * bank conflicts; the two activation words an MMA needs for words 2h, 2h+1 are adjacent.)
  * dev_status (nullable device int): set to BITNET_ERR_BAD_WEIGHT if a non-ternary byte is met
  * (the blob is then undefined).  Requires K % 64 == 0.
  */

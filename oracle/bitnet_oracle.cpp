@@ -152,9 +152,9 @@ void oracle_dequant(const int32_t* acc, const float* act_scale, float w_scale, i
 }
 
 // ---------------------------------------------------------------------------------------------
-// I2_S.  code = w + 1 (0,1,2), two bits.  Rows are stored in blocks of 8 (M padded to a multiple of
-// 8), K is padded to a multiple of 256; padding holds weight 0 (code 1).  A block is contiguous and
-// holds, for each chunk c of 256 columns, 512 bytes in which row r (0..7) owns bytes [64r, 64r+64).
+// I2_S.  code = w + 1 (0,1,2), two bits.  Rows are stored in blocks of 16 (M padded to a multiple of
+// 16), K is padded to a multiple of 256; padding holds weight 0 (code 1).  A block is contiguous and
+// holds, for each chunk c of 256 columns, 1024 bytes in which row r (0..15) owns bytes [64r, 64r+64).
 // In those 64 bytes = 16 little-endian words, the weight at column kk = k % 256 of the chunk sits in
 //   word j = 2*(kk/32) + (kk%8)/4,  byte b = kk%4 of that word,  bits [2s, 2s+1] with s = (kk%32)/8.
 struct I2sPos {
@@ -162,19 +162,19 @@ struct I2sPos {
   int shift;
 };
 static I2sPos i2s_pos(int64_t m, int64_t k, int64_t kp) {
-  const int64_t rb = m / 8, r = m % 8, c = k / 256, kk = k % 256;
+  const int64_t rb = m / 16, r = m % 16, c = k / 256, kk = k % 256;
   const int64_t j = 2 * (kk / 32) + (kk % 8) / 4, b = kk % 4, s = (kk % 32) / 8;
-  return {rb * (2 * kp) + c * 512 + r * 64 + 4 * j + b, (int)(2 * s)};
+  return {rb * (4 * kp) + c * 1024 + r * 64 + 4 * j + b, (int)(2 * s)};
 }
 
 size_t oracle_i2s_packed_bytes(int64_t M, int64_t K) {
   if (M < 1 || K < 1) return 0;
-  return (size_t)(ceil_div(M, 8) * 8) * (size_t)(ceil_div(K, 256) * 256) / 4;
+  return (size_t)(ceil_div(M, 16) * 16) * (size_t)(ceil_div(K, 256) * 256) / 4;
 }
 
 int oracle_pack_i2s(const int8_t* w, int64_t M, int64_t K, uint8_t* packed) {
   if (!w || !packed || M < 1 || K < 1) return 1;
-  const int64_t mp = ceil_div(M, 8) * 8, kp = ceil_div(K, 256) * 256;
+  const int64_t mp = ceil_div(M, 16) * 16, kp = ceil_div(K, 256) * 256;
   std::memset(packed, 0, (size_t)(mp * kp / 4));
   for (int64_t m = 0; m < mp; ++m)
     for (int64_t k = 0; k < kp; ++k) {

@@ -37,14 +37,14 @@ inline __host__ bool tl_geom(int fmt, int64_t M, int64_t K, int bk3, TlGeom* g) 
   return true;
 }
 
-// Geometry of an I2_S blob: rows in blocks of 8, K padded to 256; a block is contiguous and holds
-// one 512-byte piece per 256-column chunk, row r of the block owning bytes [64r, 64r+64) of it.
+// Geometry of an I2_S blob: rows in blocks of 16, K padded to 256; a block is contiguous and holds
+// one 1024-byte piece per 256-column chunk, row r of the block owning bytes [64r, 64r+64) of it.
 // Word j (0..15) of those 64 bytes, slot s (bits [8b+2s, 8b+2s+1] of byte b) holds the weights
 // kk = 32*(j/2) + 8*s + 4*(j%2) + b of the chunk, i.e. the activation word 8*(j/2) + 2*s + (j%2).
 inline __host__ __device__ int64_t i2s_kp(int64_t K) { return ceil_div(K, 256) * 256; }
-inline __host__ __device__ int64_t i2s_mp(int64_t M) { return ceil_div(M, 8) * 8; }
+inline __host__ __device__ int64_t i2s_mp(int64_t M) { return ceil_div(M, 16) * 16; }
 inline __host__ __device__ int64_t i2s_row_chunk_offset(int64_t m, int64_t chunk, int64_t kp) {
-  return (m >> 3) * (2 * kp) + chunk * 512 + (m & 7) * 64;
+  return (m >> 4) * (4 * kp) + chunk * 1024 + (m & 15) * 64;
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

@@ -8,13 +8,13 @@
 // 128 out-features x 256 tokens.  Per 128-column K block:
 //   * warp 0   : one TMA tensor copy brings the 256 x 128 int8 activation tile straight into the
 //                128-byte-swizzled K-major layout the MMA wants (operand B);
-//   * warps 2-5: each thread owns one weight row: it reads the row's 32 packed bytes from the blob
+//   * warps 2-9: two threads per weight row: each reads 16 of the row's 32 packed bytes from the blob
 //                (L2 resident: the whole blob is ~15 MB), expands the 2-bit codes to int8 -1/0/+1 in
 //                registers and writes the row of operand A into shared memory in the same swizzled
-//                layout (8 conflict-free 16-byte stores), then fence.proxy.async + mbarrier arrive;
+//                layout (4 conflict-free 16-byte stores), then fence.proxy.async + mbarrier arrive;
 //   * warp 1   : one thread issues four tcgen05.mma (M=128, N=256, K=32) per K block, accumulating in
 //                tensor memory, and tcgen05.commit releases the stage to the producers;
-//   * warps 6-9: epilogue -- tcgen05.ld the finished 128 x 256 accumulator (lane = out-feature,
+//   * warps 10-13: epilogue -- tcgen05.ld the finished 128 x 256 accumulator (lane = out-feature,
 //                column = token), rescale and store y; a warp's 32 lanes write 32 consecutive
 //                out-features of one token, i.e. 128 contiguous bytes.  Two accumulators (2 x 256 of the
 //                512 tensor-memory columns) let the epilogue of a tile overlap the MMAs of the next.
@@ -36,10 +36,19 @@ constexpr int KBLK = 128;       // K columns per pipeline stage = one 128-byte s
 constexpr int STAGES = 4;
 constexpr int A_BYTES = TILE_M * KBLK;   // 16 KB
 constexpr int B_BYTES = TILE_T * KBLK;   // 32 KB
-constexpr int THREADS = 320;             // warp 0 TMA, warp 1 MMA, warps 2-5 unpack, warps 6-9 epilogue
+constexpr int UNPACK_WARPS = 8;           // two threads per weight row
+constexpr int THREADS = (2 + UNPACK_WARPS + 4) * 32;   // warp 0 TMA, warp 1 MMA, warps 2-9 unpack, warps 10-13 epilogue
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 static __device__ int g_prefill_error = 0;
+#ifdef BITNET_PROFILE_PREFILL
+__device__ long long g_pprof[8];   // MMA thread of CTA 0: [0] wait tmem_empty, [1] wait full_a, [2] wait full_b, [3] issue, [4] total
+#define PP_T(v) const long long v = clock64()
+#define PP_ADD(i, x0, x1) if (blockIdx.x == 0) g_pprof[i] += (x1) - (x0)
+#else
+#define PP_T(v)
+#define PP_ADD(i, x0, x1)
+#endif
 
 struct PrefillArgs {
   const uint8_t* packed;
@@ -137,7 +146,7 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const PrefillArgs a
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(&bars->full_a[s], 4);      // one arrival per unpack warp
+      mbar_init(&bars->full_a[s], UNPACK_WARPS);   // one arrival per unpack warp
       mbar_init(&bars->full_b[s], 1);      // TMA producer (+ transaction bytes)
       mbar_init(&bars->empty[s], 1);       // tcgen05.commit
     }
@@ -186,15 +195,25 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const PrefillArgs a
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       uint32_t it = 0, nt = 0;
+      PP_T(pstart);
       for (int tile = blockIdx.x; tile < ntiles && !*abort_flag; tile += gridDim.x, ++nt) {
         const int buf = nt & 1;
+        PP_T(p0);
         bool ok = mbar_wait(&bars->tmem_empty[buf], ((nt >> 1) & 1u) ^ 1u, abort_flag);
+        PP_T(p1);
+        PP_ADD(0, p0, p1);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t d_tmem = tmem_base + buf * TILE_T;
         for (int kb = 0; ok && kb < a.nkb; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t par = (it / STAGES) & 1u;
-          ok = mbar_wait(&bars->full_a[s], par, abort_flag) && mbar_wait(&bars->full_b[s], par, abort_flag);
+          PP_T(q0);
+          ok = mbar_wait(&bars->full_a[s], par, abort_flag);
+          PP_T(q1);
+          ok = ok && mbar_wait(&bars->full_b[s], par, abort_flag);
+          PP_T(q2);
+          PP_ADD(1, q0, q1);
+          PP_ADD(2, q1, q2);
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint64_t adesc = make_desc(smem_u32(tileA + s * A_BYTES));
@@ -203,6 +222,8 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const PrefillArgs a
           for (int k4 = 0; k4 < KBLK / 32; ++k4)   // 32 bytes further along K: +2 in the address field
             umma_i8(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, (kb > 0 || k4 > 0) ? 1u : 0u);
           umma_commit(&bars->empty[s]);            // stage reusable once these MMAs have read it
+          PP_T(q3);
+          PP_ADD(3, q2, q3);
         }
         if (!ok) {
           atomicExch(&g_prefill_error, BITNET_ERR_TIMEOUT);
@@ -211,42 +232,50 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const PrefillArgs a
         }
         umma_commit(&bars->tmem_full[buf]);        // accumulator complete
       }
+      PP_T(pend);
+      PP_ADD(4, pstart, pend);
     }
-  } else if (warp < 6) {
+  } else if (warp < 2 + UNPACK_WARPS) {
     // ------------------------------------------------------------ unpackers: weight rows (operand A)
-    const int r = threadIdx.x - 64;                // row of the tile, 0..127
+    const int u = threadIdx.x - 64;                // 0..255: row u/2 of the tile, half u%2 of its 128 columns
+    const int r = u >> 1, hf = u & 1;
     uint32_t it = 0;
     for (int tile = blockIdx.x; tile < ntiles && !*abort_flag; tile += gridDim.x) {
       const int m = (tile % a.tiles_m) * TILE_M + r;
       const bool row_ok = m < a.M;
-      const uint8_t* rowp = a.packed + i2s_row_chunk_offset(row_ok ? m : 0, 0, a.kp);
-      uint4 nx0 = make_uint4(0x55555555u, 0x55555555u, 0x55555555u, 0x55555555u), nx1 = nx0;   // code 1 = weight 0
-      if (row_ok) {
-        nx0 = __ldg(reinterpret_cast<const uint4*>(rowp));
-        nx1 = __ldg(reinterpret_cast<const uint4*>(rowp) + 1);
-      }
+      // K block kb = half kb&1 of chunk kb/2: 32 bytes of the row, of which this thread takes 16
+      const uint8_t* rowp = a.packed + i2s_row_chunk_offset(row_ok ? m : 0, 0, a.kp) + hf * 16;
+      // packed words of K blocks kb .. kb+PF-1 are kept in flight: an L2 round trip is longer than one block
+      constexpr int PF = 4;
+      const uint4 zero_w = make_uint4(0x55555555u, 0x55555555u, 0x55555555u, 0x55555555u);   // code 1 = weight 0
+      uint4 nx[PF];
+#pragma unroll
+      for (int p = 0; p < PF; ++p)
+        nx[p] = (row_ok && p < a.nkb) ? __ldg(reinterpret_cast<const uint4*>(rowp + (int64_t)(p >> 1) * 1024 + (p & 1) * 32))
+                                      : zero_w;
       bool ok = true;
       for (int kb = 0; kb < a.nkb; ++kb, ++it) {
-        const uint4 c0 = nx0, c1 = nx1;
-        if (row_ok && kb + 1 < a.nkb) {
-          // K block kb+1 = half (kb+1)&1 of chunk (kb+1)/2: 32 bytes of this row
-          const uint4* np = reinterpret_cast<const uint4*>(rowp + (int64_t)((kb + 1) >> 1) * 512 + ((kb + 1) & 1) * 32);
-          nx0 = __ldg(np);
-          nx1 = __ldg(np + 1);
-        }
+        const uint4 cw = nx[0];
+#pragma unroll
+        for (int p = 0; p + 1 < PF; ++p) nx[p] = nx[p + 1];
+        nx[PF - 1] = (row_ok && kb + PF < a.nkb)
+                         ? __ldg(reinterpret_cast<const uint4*>(rowp + (int64_t)((kb + PF) >> 1) * 1024 + ((kb + PF) & 1) * 32))
+                         : zero_w;
         const int s = it % STAGES;
         if (!mbar_wait(&bars->empty[s], ((it / STAGES) & 1u) ^ 1u, abort_flag)) {
           ok = false;
           break;
         }
-        const uint32_t w[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+        const uint32_t w[4] = {cw.x, cw.y, cw.z, cw.w};
         uint8_t* rowA = tileA + s * A_BYTES + (r >> 3) * 1024 + (r & 7) * 128;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          // 16 consecutive columns 16c..16c+15 of the block: words 2P, 2P+1 (P = c/2), slots 2h, 2h+1 (h = c%2)
-          const uint32_t w0 = w[2 * (c >> 1)], w1 = w[2 * (c >> 1) + 1];
-          const int h = c & 1;
+        for (int c4 = 0; c4 < 4; ++c4) {
+          // 16 consecutive columns of the block, chunk c = 4*hf + c4: words 2P, 2P+1 (P = c/2) of the 32
+          // bytes, i.e. words 2*(c4/2), 2*(c4/2)+1 of this thread's 16, slots 2h, 2h+1 (h = c%2)
+          const uint32_t w0 = w[2 * (c4 >> 1)], w1 = w[2 * (c4 >> 1) + 1];
+          const int h = c4 & 1;
           const uint4 o = make_uint4(slot_s8(w0, 2 * h), slot_s8(w1, 2 * h), slot_s8(w0, 2 * h + 1), slot_s8(w1, 2 * h + 1));
+          const int c = 4 * hf + c4;
           *reinterpret_cast<uint4*>(rowA + ((c ^ (r & 7)) << 4)) = o;
         }
         // make the generic-proxy stores visible to the tensor core (async proxy), then signal
@@ -383,6 +412,15 @@ int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int
   gemm_i2s_tc_kernel<<<grid, THREADS, smem, st>>>(qmap, a);
   return check_launch();
 }
+
+#ifdef BITNET_PROFILE_PREFILL
+extern "C" int bitnet_debug_prefill_profile(long long* out, int reset) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(out, g_pprof, sizeof(long long) * 8);
+  if (reset) { long long z[8] = {0}; cudaMemcpyToSymbol(g_pprof, z, sizeof(z)); }
+  return 0;
+}
+#endif
 
 int gemm_prefill_status(int* out) {
   cudaError_t e = cudaMemcpyFromSymbol(out, g_prefill_error, sizeof(int));

@@ -1,31 +1,37 @@
-// I2_S mpGEMV for decode (1..8 tokens), streaming kernel: Alg. 1 Phase 2 from the 2-bit blob.
+// I2_S mpGEMV for decode (1..8 tokens), streaming kernel: Alg. 1 Phase 2 from the 2-bit blob, with
+// the quantiser (Phase 1) optionally fused in.
 //
-// Memory side.  Persistent CTAs, one per SM, whose ring buffer takes the SM's whole shared memory
-// (~220 KB per SM, ~32 MB over the GPU: a small matrix is prefetched completely while the quantiser
-// before it is still running).  The matrix is cut into units of 8 rows;
-// the blob stores a unit contiguously (chunk-major: 512 bytes per 256-column chunk, 64 bytes per
-// row), so one K-slab of a unit (at most 32 chunks = 16 KB) is ONE bulk asynchronous copy
-// (cp.async.bulk global -> shared, completion counted on an mbarrier).  Unit u belongs to CTA
-// u mod gridDim; a ring slot holds two units (one 16-row tile).  There is no producer thread: the
-// warp that is last to finish reading a slot refills it.  Weights never depend on the previous
-// kernel in the stream, so the ring is filled at once under programmatic dependent launch; only the
-// math waits for that kernel (griddepcontrol.wait) before it touches activations.
+// Memory side.  Persistent CTAs, one per SM, whose ring buffer takes the SM's shared memory (~220 KB
+// per SM, ~32 MB over the GPU).  The matrix is cut into units of 16 rows -- the blob stores a unit
+// contiguously and chunk-major (1024 bytes per 256-column chunk, 64 bytes per row), so any K-slab of
+// a unit (at most 32 chunks = 32 KB) is ONE bulk asynchronous copy (cp.async.bulk global -> shared,
+// completion counted on an mbarrier) into a ring slot.  Unit u belongs to CTA u mod gridDim.  Issuing
+// a bulk copy costs the issuing lane a few hundred cycles whatever its size, hence large copies, and
+// there is no producer thread: the warp that is last to finish reading a slot refills it.  Weights
+// never depend on the previous kernel in the stream; under programmatic dependent launch the CTA
+// starts as soon as an SM is free, and only the activation loads wait for that kernel
+// (griddepcontrol.wait).
 //
-// Compute side.  16 warps in groups that work on alternate tiles.  Two units (16 rows) form the A operand of int8 tensor-core
-// MMAs (mma.sync m16n8k32, u8 x s8 -> s32): lane (g = lane/4, t = lane%4) reads 16 bytes = 64 weights
-// of row g of each unit -- the 32 lanes read 512 contiguous bytes, conflict free.  Masking a packed
-// word with 0x03030303 << 2s leaves, without any shift, the four codes of slot s scaled by 4^s:
-// exactly one A register (row g, four consecutive k).  The B operand is the activations: column n of
-// B is token n, so lane (g,t) keeps token g's 64 activations for its k-column in registers, the same
-// for every unit the CTA processes; the blob's word order makes the two activation words of an MMA
-// adjacent.  One MMA does the work of 32 dp4a and the reduction over k happens inside the tensor
-// core, so there are no shuffle reductions, and batches of 1..8 tokens cost the same.  Four
-// accumulator fragments carry the slot scales 1, 4, 16, 64; each is an exact multiple of its scale,
-// so arithmetic shifts undo it, and sum(code*q) - sum(q) = sum(w*q).  The warps of a tile cover
-// different k-steps; their fragments meet in shared memory (atomicAdd + arrival counter) and the
-// last warp rescales and stores y = acc * act_scale[t] * w_scale.  K longer than one slab is
-// processed in phases (slab 0 of every unit, then slab 1, ...) with the partial sums parked in
-// shared memory, so nothing is exchanged between CTAs and no workspace is needed.
+// Compute side.  16 warps in groups that work on alternate units.  A unit is the A operand of int8
+// tensor-core MMAs (mma.sync m16n8k32, u8 x s8 -> s32): lane (g = lane/4, t = lane%4) reads 16 bytes =
+// 64 weights of row g and of row g+8 -- the 32 lanes read 512 contiguous bytes each time, conflict
+// free.  Masking a packed word with 0x03030303 << 2s leaves, without any shift, the four codes of slot
+// s scaled by 4^s: exactly one A register (one row, four consecutive k).  The B operand is the
+// activations: column n of B is token n, so lane (g,t) keeps token g's 64 activations for its
+// k-column in registers, the same for every unit the CTA processes; the blob's word order makes the
+// two activation words of an MMA adjacent.  One MMA does the work of 32 dp4a and the reduction over k
+// happens inside the tensor core, so there are no shuffle reductions, and batches of 1..8 tokens cost
+// the same.  Four accumulator fragments carry the slot scales 1, 4, 16, 64; each is an exact multiple
+// of its scale, so arithmetic shifts undo it, and sum(code*q) - sum(q) = sum(w*q).  The warps of a
+// group cover different chunks; their fragments meet in shared memory (atomicAdd + arrival counter)
+// and the last warp rescales and stores y = acc * act_scale[t] * w_scale.  K longer than one slab
+// is walked slab by slab for the same unit, the accumulators staying in registers and the activation
+// registers being reloaded from shared memory, so nothing is exchanged between CTAs and no workspace
+// is needed.
+//
+// Fused quantiser: with fp32 activations given, every CTA computes the absmax and the int8 codes
+// itself (the row stays in registers between the two passes) while its first weight tiles are in
+// flight; CTA 0 also stores the codes and scales for the caller.
 //
 // Every wait on an mbarrier is bounded; a wait that gives up raises a device flag that
 // bitnet_device_status() reports, and the thread leaves the kernel.
@@ -34,34 +40,19 @@
 namespace bitnet {
 namespace {
 
-#ifndef BITNET_GEMV_CTAS_PER_SM
-#define BITNET_GEMV_CTAS_PER_SM 1
-#endif
-constexpr int CTAS_PER_SM = BITNET_GEMV_CTAS_PER_SM;   // 2: the next kernel's CTA fits beside this one's
-constexpr int CW = 16 / CTAS_PER_SM;     // consumer warps
-constexpr int WPT_MAX = 8;               // warps that share one 16-row tile
-constexpr int THREADS = CW * 32;         // no producer warp: the warp that frees a slot last refills it
-constexpr int MAX_SLOTS = 12;            // ring slots, one PAIR of units (16 rows) each
+constexpr int CW = 16;                   // warps (all consume)
+constexpr int WPT_MAX = 8;               // warps that share one unit
+constexpr int THREADS = CW * 32;
+constexpr int MAX_SLOTS = 12;            // ring slots, one unit-slab (16 rows x up to 32 chunks) each
 constexpr int XREG = 16;                 // float4 registers per thread of the fused quantiser's fast path
-constexpr int EARLY_SLOTS = 3;            // tiles requested before the activations (96 KB per SM)
-constexpr int ACC_RING = 16;             // accumulator entries when a unit pair is finished in one phase
-                                         // (more than the pairs the ring lets warps drift apart)
-constexpr int MAX_ACC_BYTES = 24 * 1024;
+constexpr int ACC_RING = 16;             // cross-warp accumulator entries (more than the units warps can drift apart)
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 static __device__ int g_stream_error = 0;
-#ifdef BITNET_PROFILE_GEMV
-__device__ long long g_prof[12];   // [0] wait, [1] load+mma, [2] release, [3] epilogue, [4] pairs (warp 0 of CTA 0)
-#define PROF_T(var) const long long var = clock64()
-#define PROF_ADD(i, a0, a1) if (blockIdx.x == 0 && warp == 0 && lane == 0) g_prof[i] += (a1) - (a0)
-#else
-#define PROF_T(var)
-#define PROF_ADD(i, a0, a1)
-#endif
 
 struct MmaArgs {
   const uint8_t* packed;
-  int64_t unit_bytes;  // bytes of one 8-row block of the blob = 2 * Kp
+  int64_t unit_bytes;    // bytes of one 16-row block of the blob = 4 * Kp
   int M;
   int64_t K;
   const int8_t* q;       // quantised activations [T][K] (input, or output of the fused quantiser)
@@ -74,15 +65,14 @@ struct MmaArgs {
   int T;
   float* y;
   int32_t* acc_out;
-  int nchunks;         // 256-column chunks per row (Kp / 256)
-  int nq;              // K-slabs = phases
-  int slab_chunks;     // chunks per slab
-  int stage_bytes;     // slab_chunks * 512 = ring slot size
-  int wpt;             // warps per tile (each covers KS chunks)
-  int ngroups;         // warp groups; group g takes unit pairs g, g + ngroups, ...
-  int nunits;          // ceil(M / 8)
-  int slots;           // ring slots (one unit-slab each)
-  int acc_entries;
+  int nchunks;           // 256-column chunks per row (Kp / 256)
+  int nq;                // K-slabs per unit
+  int slab_chunks;       // chunks per slab
+  int stage_bytes;       // slab_chunks * 1024 = ring slot size
+  int wpt;               // warps per unit (each covers KS chunks of a slab)
+  int ngroups;           // warp groups; group g takes the CTA's units g, g + ngroups, ...
+  int nunits;            // ceil(M / 16)
+  int slots;             // ring slots
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -91,9 +81,6 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 // Bounded wait for the phase with the given parity; false = gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
@@ -110,6 +97,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   }
   return false;
 }
+__device__ __forceinline__ void st_release_cta(int* p, int v) {
+  asm volatile("st.release.cta.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
+// Bounded wait until *p == want (acquire).
+__device__ __forceinline__ bool wait_issued(const int* p, int want) {
+  const uint32_t addr = smem_u32(p);
+  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    int v;
+    asm volatile("ld.acquire.cta.shared::cta.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    if (v == want) return true;
+  }
+  return false;
+}
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t pol) {
   asm volatile(
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
@@ -119,88 +119,78 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 // D(16x8, s32) += A(16x32, u8, row) * B(32x8, s8, col).  Lane (g = lane/4, t = lane%4):
 // a0 = row g, k 4t..4t+3; a1 = row g+8, same k; a2, a3 = the same rows, k 16+4t..; b0 = k 4t..4t+3 of
 // column g, b1 = k 16+4t..; c0,c1 = row g, columns 2t, 2t+1; c2,c3 = row g+8.
-#ifndef BITNET_MMA_VARIANT
-#define BITNET_MMA_VARIANT 2
-#endif
-#if BITNET_MMA_VARIANT >= 1
-#define MMA_ASM asm
-#else
-#define MMA_ASM asm volatile
-#endif
 __device__ __forceinline__ void mma_u8s8(int (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, int b0,
                                          int b1) {
-  MMA_ASM(
-      "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ int quant1(float x, float s) {
+  return max(-128, min(127, __float2int_rn(__fmul_rn(x, s))));
+}
+__device__ __forceinline__ int quant4(const float4& v, float s) {
+  return (quant1(v.x, s) & 255) | ((quant1(v.y, s) & 255) << 8) | ((quant1(v.z, s) & 255) << 16) |
+         ((quant1(v.w, s) & 255) << 24);
+}
 
-// KS = chunks (256 weights each) a consumer warp covers per slab.
+// KS = chunks (256 weights each) a warp covers per slab.
 template <int KS>
-__global__ void __launch_bounds__(THREADS, CTAS_PER_SM) gemv_i2s_mma_kernel(const MmaArgs a) {
+__global__ void __launch_bounds__(THREADS, 1) gemv_i2s_mma_kernel(const MmaArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
-  // layout: [full barriers][rcnt: readers done per slot][cnt[acc_entries]][acc[acc_entries][T][16]][ring]
+  // layout: [full barriers][readers-done counters][acc counters][acc sums][quantiser scratch][codes][ring]
   uint64_t* full = reinterpret_cast<uint64_t*>(smem);
   int* rcnt = reinterpret_cast<int*>(full + MAX_SLOTS);
-  int* cnt = rcnt + 2 * MAX_SLOTS;
-  int* acc = cnt + a.acc_entries;
-  const uint32_t head = (uint32_t)((2 * MAX_SLOTS * 8 + a.acc_entries * 4 * (1 + a.T * 16) + 127) & ~127);
-  // [fused-quantiser scratch: 8 scales, 8 x 16 partial maxima][staged activations][ring]
-  float* qscale = reinterpret_cast<float*>(smem + head);
-  float* qred = qscale + 8;
+  int* issued = rcnt + MAX_SLOTS;                              // 1 + the tile last requested into each slot
+  int* cnt = issued + MAX_SLOTS;
+  int* acc = cnt + ACC_RING;                                   // [ACC_RING][T][16]
+  const uint32_t head = (uint32_t)((MAX_SLOTS * 16 + ACC_RING * 4 * (1 + a.T * 16) + 127) & ~127);
+  float* qscale = reinterpret_cast<float*>(smem + head);       // [8] act_scale per token
+  float* qred = qscale + 8;                                    // [8][16] partial maxima / multipliers
   int8_t* qs_mem = reinterpret_cast<int8_t*>(smem + head + 1024);
   const int kp = a.nchunks * 256;
   uint8_t* ring = smem + head + 1024 + (a.use_qs ? ((a.T * kp + 127) & ~127) : 0);
 
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
-  PROF_T(tk0);
   const int n_units = (a.nunits - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-  const int n_pairs = (n_units + 1) / 2;
-  const int total = a.nq * n_pairs;            // tiles this CTA streams, in order: phase-major, then pair
+  const int total = a.nq * n_units;            // tiles this CTA streams, in order: unit-major, then slab
 
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-  // Issues the copies of tile `seq` (one K-slab of two units, each contiguous in the blob) into `slot`.
+  // Issues the copy of tile `seq` (one K-slab of one unit, contiguous in the blob) into `slot`.
   auto fill = [&](int seq, int slot) {
-    const int ph = seq / n_pairs;
-    const int p = seq - ph * n_pairs;
+    const int ul = seq / a.nq;
+    const int ph = seq - ul * a.nq;
     const int c0 = ph * a.slab_chunks;
-    const uint32_t bytes = (uint32_t)min(a.slab_chunks, a.nchunks - c0) * 512u;
-    const bool two = 2 * p + 1 < n_units;
-    const uint8_t* src = a.packed + ((int64_t)blockIdx.x + (int64_t)(2 * p) * gridDim.x) * a.unit_bytes + (int64_t)c0 * 512;
+    const uint32_t bytes = (uint32_t)min(a.slab_chunks, a.nchunks - c0) * 1024u;
+    const uint8_t* src = a.packed + ((int64_t)blockIdx.x + (int64_t)ul * gridDim.x) * a.unit_bytes + (int64_t)c0 * 1024;
     const uint32_t bar = smem_u32(full + slot);
-    const uint32_t dst = smem_u32(ring + (size_t)slot * (2 * a.stage_bytes));
-    mbar_expect_tx(bar, two ? 2 * bytes : bytes);
-    bulk_g2s(dst, src, bytes, bar, pol);
-    if (two) bulk_g2s(dst + a.stage_bytes, src + (int64_t)gridDim.x * a.unit_bytes, bytes, bar, pol);
+    mbar_expect_tx(bar, bytes);
+    bulk_g2s(smem_u32(ring + (size_t)slot * a.stage_bytes), src, bytes, bar, pol);
+    // Publish which tile the slot's barrier now counts for.  A parity wait tells two phases apart only;
+    // a group that has not itself read the slot's previous tile must not mistake that tile's phase
+    // (or the fresh barrier) for this one, so readers first wait for this number.
+    st_release_cta(issued + slot, seq + 1);
   };
 
   if (threadIdx.x == 0) {
-    // let the next kernel in the stream begin its own prologue
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may begin its prologue
     for (int s = 0; s < a.slots; ++s) mbar_init(smem_u32(full + s), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int i = threadIdx.x; i < 2 * MAX_SLOTS + a.acc_entries * (1 + a.T * 16); i += THREADS) rcnt[i] = 0;
+  for (int i = threadIdx.x; i < 2 * MAX_SLOTS + ACC_RING * (1 + a.T * 16); i += THREADS) rcnt[i] = 0;
   __syncthreads();
-  // Weights do not depend on any earlier kernel: start streaming at once.  Only EARLY_SLOTS tiles are
-  // requested before the activations are: a load issued behind a burst of bulk copies waits until
-  // the burst has drained, and the rest of the ring is requested right after the activation loads.
-  const int early = a.x ? 0 : EARLY_SLOTS;   // the fused quantiser requests its activations first
-  if (lane == 0 && warp < early && warp < a.slots && warp < total) fill(warp, warp);
 
   const int group = warp / a.wpt;
   const bool idle = group >= a.ngroups;   // warps that do not fit a whole group only help in the prologue
   const int wk = warp % a.wpt;            // this warp's chunks inside a slab: wk*KS .. wk*KS+KS-1
   const int g = lane >> 2, t = lane & 3;
+  // one warp per slot requests the initial contents of the ring (after the activation loads, if any, are on
+  // their way: the issuing lane is held for a few hundred cycles)
+  const bool my_fill = lane == 0 && warp < a.slots && warp < total;
 
   // ---------------- activations come from the previous kernel in the stream
-  PROF_T(tk1);
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  PROF_T(tk2);
-  PROF_ADD(5, tk0, tk1);
-  PROF_ADD(6, tk1, tk2);
 
   if (a.use_qs) {
     if (a.x && a.T == 1 && a.K <= 4 * XREG * THREADS) {
@@ -215,8 +205,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) gemv_i2s_mma_kernel(cons
         const int i = threadIdx.x + r * THREADS;
         xv[r] = (i < n4) ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
       }
-      // the activation loads have been issued: request the ring behind them
-      if (lane == 0 && warp < a.slots && warp < total) fill(warp, warp);
+      if (my_fill) fill(warp, warp);
       float m = 0.0f;
 #pragma unroll
       for (int r = 0; r < XREG; ++r)
@@ -239,12 +228,8 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) gemv_i2s_mma_kernel(cons
       for (int r = 0; r < XREG; ++r) {
         const int i = threadIdx.x + r * THREADS;
         if (i < kp / 4) {
-          const int q0 = max(-128, min(127, __float2int_rn(__fmul_rn(xv[r].x, sq))));
-          const int q1 = max(-128, min(127, __float2int_rn(__fmul_rn(xv[r].y, sq))));
-          const int q2 = max(-128, min(127, __float2int_rn(__fmul_rn(xv[r].z, sq))));
-          const int q3 = max(-128, min(127, __float2int_rn(__fmul_rn(xv[r].w, sq))));
-          const int word = (q0 & 255) | ((q1 & 255) << 8) | ((q2 & 255) << 16) | ((q3 & 255) << 24);
-          reinterpret_cast<int*>(qs_mem)[i] = word;       // columns K..Kp-1 came in as zeros
+          const int word = quant4(xv[r], sq);                 // columns K..Kp-1 came in as zeros
+          reinterpret_cast<int*>(qs_mem)[i] = word;
           if (blockIdx.x == 0 && a.q_out && i < n4) reinterpret_cast<int*>(a.q_out)[i] = word;
         }
       }
@@ -261,6 +246,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) gemv_i2s_mma_kernel(cons
         for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
         if (lane == 0) qred[tok * CW + warp] = m;
       }
+      if (my_fill) fill(warp, warp);
       __syncthreads();
       if (threadIdx.x < a.T) {
         float m = 0.0f;
@@ -278,39 +264,29 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) gemv_i2s_mma_kernel(cons
         for (int i = threadIdx.x; i < kp / 4; i += THREADS) {
           int word = 0;
           if (i < (int)(a.K / 4)) {
-            const float4 v = __ldcg(x4 + i);
-            const int q0 = max(-128, min(127, __float2int_rn(__fmul_rn(v.x, sq))));
-            const int q1 = max(-128, min(127, __float2int_rn(__fmul_rn(v.y, sq))));
-            const int q2 = max(-128, min(127, __float2int_rn(__fmul_rn(v.z, sq))));
-            const int q3 = max(-128, min(127, __float2int_rn(__fmul_rn(v.w, sq))));
-            word = (q0 & 255) | ((q1 & 255) << 8) | ((q2 & 255) << 16) | ((q3 & 255) << 24);
+            word = quant4(__ldcg(x4 + i), sq);
             if (blockIdx.x == 0 && a.q_out) reinterpret_cast<int*>(a.q_out + (int64_t)tok * a.K)[i] = word;
           }
           reinterpret_cast<int*>(qs_mem + tok * kp)[i] = word;
         }
       }
-      // request the ring once the second pass over the activations has been issued
-      if (lane == 0 && warp < a.slots && warp < total) fill(warp, warp);
     } else {
-      // ---- stage the given codes (zero beyond K) so that every phase reloads them from shared memory
+      // ---- stage the given codes (zero beyond K): every warp and every slab reads them from shared memory
       for (int tok = 0; tok < a.T; ++tok) {
         const int* q4 = reinterpret_cast<const int*>(a.q + (int64_t)tok * a.K);
         for (int i = threadIdx.x; i < kp / 4; i += THREADS)
           reinterpret_cast<int*>(qs_mem + tok * kp)[i] = (i < (int)(a.K / 4)) ? __ldcg(q4 + i) : 0;
       }
       if (threadIdx.x < a.T) qscale[threadIdx.x] = __ldcg(a.act_scale + threadIdx.x);
-      if (lane == 0 && warp >= early && warp < a.slots && warp < total) fill(warp, warp);
+      if (my_fill) fill(warp, warp);
     }
     __syncthreads();
+  } else if (my_fill) {
+    fill(warp, warp);
   }
-  PROF_T(tkq);
-  PROF_ADD(7, tk2, tkq);
-  if (idle) {
-    if (!a.use_qs && lane == 0 && warp >= early && warp < a.slots && warp < total) fill(warp, warp);
-    return;
-  }
+  if (idle) return;
 
-  // rescale factors of the tokens this lane stores when its warp finishes a tile (token (lane>>4) + 2i)
+  // rescale factors of the tokens this lane stores when its warp finishes a unit (token (lane>>4) + 2i)
   float sc[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -318,18 +294,19 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) gemv_i2s_mma_kernel(cons
     const float as = (tok < a.T) ? (a.use_qs ? qscale[tok] : __ldcg(a.act_scale + tok)) : 0.0f;
     sc[i] = __fmul_rn(as, a.w_scale);
   }
-  const int target = a.wpt * a.nq;
-  const int lane_off = (wk * KS) * 512 + g * 64 + t * 16;
-  for (int ph = 0; ph < a.nq; ++ph) {
-    // ---- activations of this phase: token g, the 64 values under this lane's 16-byte weight column
-    int qr[KS][16];
-    bool ksok[KS];
-    int qs = 0;
+  const int lane_off = (wk * KS) * 1024 + g * 64 + t * 16;
+
+  // activations of one slab: token g, the 64 values under this lane's 16-byte weight column, per chunk
+  int qr[KS][16];
+  bool ksok[KS];
+  int qs_even = 0, qs_odd = 0;   // sums of the activations of tokens 2t and 2t+1 over this warp's chunks
+  auto load_q = [&](int ph) {
     const int slab_n = min(a.slab_chunks, a.nchunks - ph * a.slab_chunks);
+    int qs = 0;
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
-      const int cl = wk * KS + ks;                                       // chunk inside the slab
-      const int64_t k0 = (int64_t)(ph * a.slab_chunks + cl) * 256 + t * 64;   // first of the lane's 64 columns
+      const int cl = wk * KS + ks;                                          // chunk inside the slab
+      const int64_t k0 = (int64_t)(ph * a.slab_chunks + cl) * 256 + t * 64;  // first of the lane's 64 columns
       ksok[ks] = cl < slab_n;
       if (ksok[ks] && k0 < a.K && g < a.T) {
         const uint4* qp = a.use_qs ? reinterpret_cast<const uint4*>(qs_mem + g * kp + k0)
@@ -346,64 +323,39 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) gemv_i2s_mma_kernel(cons
 #pragma unroll
         for (int i = 0; i < 16; ++i) qr[ks][i] = 0;
       }
-    }
-    // the activation loads are on their way: request the rest of the ring behind them
-    if (!a.use_qs && ph == 0 && lane == 0 && warp >= early && warp < a.slots && warp < total) fill(warp, warp);
-#pragma unroll
-    for (int ks = 0; ks < KS; ++ks)
 #pragma unroll
       for (int i = 0; i < 16; ++i) qs = __dp4a(qr[ks][i], 0x01010101, qs);
-    // sum of token g's activations over this warp's k-range, then the sums of tokens 2t and 2t+1
+    }
     qs += __shfl_xor_sync(0xffffffffu, qs, 1);
     qs += __shfl_xor_sync(0xffffffffu, qs, 2);
-    const int qs_even = __shfl_sync(0xffffffffu, qs, (2 * t) * 4);
-    const int qs_odd = __shfl_sync(0xffffffffu, qs, (2 * t + 1) * 4);
+    qs_even = __shfl_sync(0xffffffffu, qs, (2 * t) * 4);
+    qs_odd = __shfl_sync(0xffffffffu, qs, (2 * t + 1) * 4);
+  };
+  if (a.nq == 1) load_q(0);
 
-    // ring position of this group's first pair in this phase; afterwards advanced without divisions
-    int slot = (ph * n_pairs + group) % a.slots;
-    uint32_t par = (uint32_t)((ph * n_pairs + group) / a.slots) & 1u;
-    for (int p = group; p < n_pairs; p += a.ngroups) {
-      const bool hasB = 2 * p + 1 < n_units;
-      PROF_T(t0);
-      if (!mbar_wait(smem_u32(full + slot), par)) {
+  for (int ul = group; ul < n_units; ul += a.ngroups) {
+    int seq = ul * a.nq;
+    int slot = seq % a.slots;
+    uint32_t par = (uint32_t)(seq / a.slots) & 1u;
+    int C[4][4];
+#pragma unroll
+    for (int s = 0; s < 4; ++s)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) C[s][i] = 0;
+    int corr_even = 0, corr_odd = 0;
+    for (int ph = 0; ph < a.nq; ++ph, ++seq) {
+      if (a.nq > 1) load_q(ph);
+      corr_even += qs_even;
+      corr_odd += qs_odd;
+      if (!wait_issued(issued + slot, seq + 1) || !mbar_wait(smem_u32(full + slot), par)) {
         if (lane == 0) atomicExch(&g_stream_error, BITNET_ERR_TIMEOUT);
         return;
       }
-      PROF_T(t1);
-      const uint8_t* pa = ring + lane_off + slot * (2 * a.stage_bytes);
-      const uint8_t* pb = pa + a.stage_bytes;
-
-#if BITNET_MMA_VARIANT == 3
-      int C2[2][4][4];
-#pragma unroll
-      for (int u = 0; u < 2; ++u)
-#pragma unroll
-        for (int s = 0; s < 4; ++s)
-#pragma unroll
-          for (int i = 0; i < 4; ++i) C2[u][s][i] = 0;
-#else
-      int C[4][4];
-#pragma unroll
-      for (int s = 0; s < 4; ++s)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) C[s][i] = 0;
-#endif
-#if BITNET_MMA_VARIANT == 2
-      uint4 Wp[KS], Vp[KS];
+      const uint8_t* pa = ring + lane_off + slot * a.stage_bytes;
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
-        Wp[ks] = ksok[ks] ? *reinterpret_cast<const uint4*>(pa + ks * 512) : make_uint4(0, 0, 0, 0);
-        Vp[ks] = (ksok[ks] && hasB) ? *reinterpret_cast<const uint4*>(pb + ks * 512) : make_uint4(0, 0, 0, 0);
-      }
-#endif
-#pragma unroll
-      for (int ks = 0; ks < KS; ++ks) {
-#if BITNET_MMA_VARIANT == 2
-        const uint4 W = Wp[ks], V = Vp[ks];
-#else
-        const uint4 W = ksok[ks] ? *reinterpret_cast<const uint4*>(pa + ks * 512) : make_uint4(0, 0, 0, 0);
-        const uint4 V = (ksok[ks] && hasB) ? *reinterpret_cast<const uint4*>(pb + ks * 512) : make_uint4(0, 0, 0, 0);
-#endif
+        const uint4 W = ksok[ks] ? *reinterpret_cast<const uint4*>(pa + ks * 1024) : make_uint4(0, 0, 0, 0);
+        const uint4 V = ksok[ks] ? *reinterpret_cast<const uint4*>(pa + ks * 1024 + 512) : make_uint4(0, 0, 0, 0);
         const unsigned w4[4] = {W.x, W.y, W.z, W.w};
         const unsigned v4[4] = {V.x, V.y, V.z, V.w};
         // words 2h, 2h+1 of the lane's 16 bytes, slot s: weights 32h + 8s + (0..7) of its 64 columns,
@@ -413,103 +365,77 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) gemv_i2s_mma_kernel(cons
 #pragma unroll
           for (int s = 0; s < 4; ++s) {
             const unsigned m = 0x03030303u << (2 * s);
-#if BITNET_MMA_VARIANT == 3
-            mma_u8s8(C2[h][s], w4[2 * h] & m, v4[2 * h] & m, w4[2 * h + 1] & m, v4[2 * h + 1] & m,
-                     qr[ks][8 * h + 2 * s], qr[ks][8 * h + 2 * s + 1]);
-#else
             mma_u8s8(C[s], w4[2 * h] & m, v4[2 * h] & m, w4[2 * h + 1] & m, v4[2 * h + 1] & m,
                      qr[ks][8 * h + 2 * s], qr[ks][8 * h + 2 * s + 1]);
-#endif
           }
         }
       }
-#if BITNET_MMA_VARIANT == 3
-      int C[4][4];
-#pragma unroll
-      for (int s = 0; s < 4; ++s)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) C[s][i] = C2[0][s][i] + C2[1][s][i];
-#endif
-      PROF_T(t2);
       // Every weight of this warp's share has been read (the values are in registers).  The warp that is
       // last to finish with the slot refills it with the tile that comes `slots` later.
       __syncwarp();
       if (lane == 0) {
         if (atomicAdd(rcnt + slot, 1) == a.wpt - 1) {
           atomicExch(rcnt + slot, 0);
-          const int seq = ph * n_pairs + p;
           if (seq + a.slots < total) {
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             fill(seq + a.slots, slot);
           }
         }
       }
-      PROF_T(t3);
-      // fragment: c[0] = (row g, token 2t), c[1] = (row g, token 2t+1), c[2], c[3] = the same for row g+8
-      int c[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) c[i] = C[0][i] + (C[1][i] >> 2) + (C[2][i] >> 4) + (C[3][i] >> 6);
-      c[0] -= qs_even;
-      c[2] -= qs_even;
-      c[1] -= qs_odd;
-      c[3] -= qs_odd;
-
-      const int uA = (int)blockIdx.x + (2 * p) * (int)gridDim.x;
-      const int uB = uA + (int)gridDim.x;
-      const int e = (a.nq == 1) ? (p % ACC_RING) : p;
-      int* ea = acc + e * a.T * 16;
-      if (2 * t < a.T) {
-        atomicAdd(ea + (2 * t) * 16 + g, c[0]);
-        atomicAdd(ea + (2 * t) * 16 + g + 8, c[2]);
-      }
-      if (2 * t + 1 < a.T) {
-        atomicAdd(ea + (2 * t + 1) * 16 + g, c[1]);
-        atomicAdd(ea + (2 * t + 1) * 16 + g + 8, c[3]);
-      }
-      __syncwarp();
-      int last = 0;
-      if (lane == 0) {
-        __threadfence_block();
-        last = atomicAdd(cnt + e, 1) == target - 1;
-      }
-      last = __shfl_sync(0xffffffffu, last, 0);
-      if (last) {
-        // every warp and phase has delivered: rescale and store the 16 rows of this pair
-        __threadfence_block();
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int idx = lane + 32 * i;
-          if (idx < a.T * 16) {
-            const int tok = idx >> 4, r16 = idx & 15;
-            const int v = atomicExch(ea + idx, 0);
-            const int row = ((r16 < 8) ? uA : uB) * 8 + (r16 & 7);
-            if ((r16 < 8 || hasB) && row < a.M) {
-              a.y[(int64_t)tok * a.M + row] = __fmul_rn((float)v, sc[i]);
-              if (a.acc_out) a.acc_out[(int64_t)tok * a.M + row] = v;
-            }
-          }
-        }
-        if (lane == 0) atomicExch(cnt + e, 0);
-      }
-      PROF_T(t4);
-      PROF_ADD(0, t0, t1);
-      PROF_ADD(1, t1, t2);
-      PROF_ADD(2, t2, t3);
-      PROF_ADD(3, t3, t4);
-      PROF_ADD(4, 0, 1);
-      slot += a.ngroups;
-      while (slot >= a.slots) {
-        slot -= a.slots;
+      if (++slot == a.slots) {
+        slot = 0;
         par ^= 1u;
       }
     }
+    // fragment: c[0] = (row g, token 2t), c[1] = (row g, token 2t+1), c[2], c[3] = the same for row g+8
+    int c[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) c[i] = C[0][i] + (C[1][i] >> 2) + (C[2][i] >> 4) + (C[3][i] >> 6);
+    c[0] -= corr_even;
+    c[2] -= corr_even;
+    c[1] -= corr_odd;
+    c[3] -= corr_odd;
+
+    const int e = ul % ACC_RING;
+    int* ea = acc + e * a.T * 16;
+    if (2 * t < a.T) {
+      atomicAdd(ea + (2 * t) * 16 + g, c[0]);
+      atomicAdd(ea + (2 * t) * 16 + g + 8, c[2]);
+    }
+    if (2 * t + 1 < a.T) {
+      atomicAdd(ea + (2 * t + 1) * 16 + g, c[1]);
+      atomicAdd(ea + (2 * t + 1) * 16 + g + 8, c[3]);
+    }
+    __syncwarp();
+    int last = 0;
+    if (lane == 0) {
+      __threadfence_block();
+      last = atomicAdd(cnt + e, 1) == a.wpt - 1;
+    }
+    last = __shfl_sync(0xffffffffu, last, 0);
+    if (last) {
+      // every warp of the group has delivered: rescale and store the 16 rows of this unit
+      __threadfence_block();
+      const int row0 = ((int)blockIdx.x + ul * (int)gridDim.x) * 16;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int idx = lane + 32 * i;
+        if (idx < a.T * 16) {
+          const int tok = idx >> 4, row = row0 + (idx & 15);
+          const int v = atomicExch(ea + idx, 0);
+          if (row < a.M) {
+            a.y[(int64_t)tok * a.M + row] = __fmul_rn((float)v, sc[i]);
+            if (a.acc_out) a.acc_out[(int64_t)tok * a.M + row] = v;
+          }
+        }
+      }
+      if (lane == 0) atomicExch(cnt + e, 0);
+    }
   }
-  PROF_T(tkend);
-  PROF_ADD(8, tk0, tkend);
 }
 
 struct Plan {
-  int KS, nchunks, nq, slab_chunks, stage_bytes, wpt, ngroups, nunits, slots, acc_entries, grid, use_qs;
+  int KS, nchunks, nq, slab_chunks, stage_bytes, wpt, ngroups, nunits, slots, grid, use_qs;
   size_t smem;
 };
 
@@ -523,25 +449,21 @@ bool make_plan(int T, int64_t M, int64_t K, bool fused, Plan* p) {
   p->KS = (p->slab_chunks + WPT_MAX - 1) / WPT_MAX;
   p->wpt = (p->slab_chunks + p->KS - 1) / p->KS;
   p->ngroups = CW / p->wpt;
-  p->stage_bytes = p->slab_chunks * 512;
-  p->nunits = (int)ceil_div(M, 8);
+  p->stage_bytes = p->slab_chunks * 1024;
+  p->nunits = (int)ceil_div(M, 16);
   p->grid = dev_info().sm_count < p->nunits ? dev_info().sm_count : p->nunits;
-  const int max_pairs = (int)(ceil_div(p->nunits, p->grid) + 1) / 2;
-  p->acc_entries = (p->nq == 1) ? ACC_RING : max_pairs;
-  const size_t acc_bytes = (size_t)p->acc_entries * 4 * (1 + T * 16);
-  if (acc_bytes > (size_t)MAX_ACC_BYTES) return false;
   const size_t qs_bytes = ((size_t)T * p->nchunks * 256 + 127) & ~(size_t)127;
-  // staged activations: always for the fused quantiser, otherwise when K takes several phases
-  p->use_qs = (qs_bytes <= MAX_QS_BYTES && (fused || p->nq > 1)) ? 1 : 0;
+  // staged activations whenever they fit (required by the fused quantiser)
+  p->use_qs = (qs_bytes <= MAX_QS_BYTES) ? 1 : 0;
   if (fused && !p->use_qs) return false;
-  const size_t head = ((2 * MAX_SLOTS * 8 + acc_bytes + 127) & ~(size_t)127) + 1024 + (p->use_qs ? qs_bytes : 0);
-  const size_t budget = (CTAS_PER_SM == 1) ? (size_t)dev_info().max_smem_optin - 1024
-                                           : (size_t)dev_info().max_smem_per_sm / CTAS_PER_SM - 1024;
-  if (head + 2 * 2 * (size_t)p->stage_bytes > budget) return false;
-  int slots = (int)((budget - head) / (2 * (size_t)p->stage_bytes));   // a slot holds a pair of units
+  const size_t head = (((size_t)MAX_SLOTS * 16 + (size_t)ACC_RING * 4 * (1 + T * 16) + 127) & ~(size_t)127) + 1024 +
+                      (p->use_qs ? qs_bytes : 0);
+  const size_t budget = (size_t)dev_info().max_smem_optin - 1024;
+  if (head + 2 * (size_t)p->stage_bytes > budget) return false;
+  int slots = (int)((budget - head) / (size_t)p->stage_bytes);
   if (slots > MAX_SLOTS) slots = MAX_SLOTS;
   p->slots = slots;
-  p->smem = head + (size_t)slots * 2 * p->stage_bytes;
+  p->smem = head + (size_t)slots * p->stage_bytes;
   return true;
 }
 
@@ -552,11 +474,7 @@ int launch_mma(const MmaArgs& a, const Plan& p, cudaStream_t st) {
   cudaGetDevice(&dev);
   if (!attr_set[dev & 63]) {
     cudaError_t e = cudaFuncSetAttribute(gemv_i2s_mma_kernel<KS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (CTAS_PER_SM == 1) ? dev_info().max_smem_optin
-                                                            : dev_info().max_smem_per_sm / CTAS_PER_SM - 1024);
-    if (e != cudaSuccess) return note_cuda_error(e);
-    e = cudaFuncSetAttribute(gemv_i2s_mma_kernel<KS>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                             cudaSharedmemCarveoutMaxShared);
+                                         dev_info().max_smem_optin);
     if (e != cudaSuccess) return note_cuda_error(e);
     attr_set[dev & 63] = true;
   }
@@ -588,7 +506,7 @@ int launch_gemv_i2s_stream(const uint8_t* packed, float w_scale, int64_t M, int6
   if (T < 1 || T > 8 || !make_plan(T, M, K, x != nullptr, &p)) return BITNET_ERR_UNSUPPORTED_SHAPE;
   MmaArgs a;
   a.packed = packed;
-  a.unit_bytes = 2 * i2s_kp(K);
+  a.unit_bytes = 4 * i2s_kp(K);
   a.M = (int)M;
   a.K = K;
   a.q = q;
@@ -609,7 +527,6 @@ int launch_gemv_i2s_stream(const uint8_t* packed, float w_scale, int64_t M, int6
   a.ngroups = p.ngroups;
   a.nunits = p.nunits;
   a.slots = p.slots;
-  a.acc_entries = p.acc_entries;
   switch (p.KS) {
     case 1: return launch_mma<1>(a, p, st);
     case 2: return launch_mma<2>(a, p, st);
@@ -618,15 +535,6 @@ int launch_gemv_i2s_stream(const uint8_t* packed, float w_scale, int64_t M, int6
     default: return BITNET_ERR_UNSUPPORTED_SHAPE;
   }
 }
-
-#ifdef BITNET_PROFILE_GEMV
-extern "C" int bitnet_debug_gemv_profile(long long* out, int reset) {
-  cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(out, g_prof, sizeof(long long) * 12);
-  if (reset) { long long z[12] = {0}; cudaMemcpyToSymbol(g_prof, z, sizeof(z)); }
-  return 0;
-}
-#endif
 
 int gemv_i2s_stream_status(int* out) {
   cudaError_t e = cudaMemcpyFromSymbol(out, g_stream_error, sizeof(int));

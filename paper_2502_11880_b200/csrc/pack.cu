@@ -16,10 +16,10 @@ __global__ void pack_i2s_kernel(const int8_t* __restrict__ w, int64_t M, int64_t
                                 uint32_t* __restrict__ packed, int* dev_status) {
   const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (gid >= nwords) return;
-  const int64_t block_words = kp / 2;
+  const int64_t block_words = kp;            // 16 rows x kp / 16 words
   const int64_t rb = gid / block_words, rem = gid % block_words;
-  const int64_t c = rem >> 7, r = (rem >> 4) & 7, j = rem & 15;
-  const int64_t m = rb * 8 + r;
+  const int64_t c = rem >> 8, r = (rem >> 4) & 15, j = rem & 15;
+  const int64_t m = rb * 16 + r;
   uint32_t word = 0;
   bool bad = false;
 #pragma unroll
@@ -40,10 +40,10 @@ __global__ void unpack_i2s_kernel(const uint32_t* __restrict__ packed, int64_t M
                                   int64_t nwords, int8_t* __restrict__ w, int* dev_status) {
   const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (gid >= nwords) return;
-  const int64_t block_words = kp / 2;
+  const int64_t block_words = kp;
   const int64_t rb = gid / block_words, rem = gid % block_words;
-  const int64_t c = rem >> 7, r = (rem >> 4) & 7, j = rem & 15;
-  const int64_t m = rb * 8 + r;
+  const int64_t c = rem >> 8, r = (rem >> 4) & 15, j = rem & 15;
+  const int64_t m = rb * 16 + r;
   const uint32_t word = packed[gid];
   bool bad = false;
 #pragma unroll

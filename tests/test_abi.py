@@ -42,7 +42,7 @@ def test_status_strings(L):
 def test_size_queries(L):
     assert bn.bitnet_i2s_packed_bytes(1536, 1536) == 1536 * 1536 // 4
     assert bn.bitnet_i2s_packed_bytes(3200, 8640) == 3200 * 8704 // 4
-    assert bn.bitnet_i2s_packed_bytes(3, 64) == 512
+    assert bn.bitnet_i2s_packed_bytes(3, 64) == 1024
     assert bn.bitnet_i2s_packed_bytes(16, 100) == 0                      # K % 64 != 0
     assert bn.bitnet_tl_packed_bytes("tl2", 32, 8192) == 85 * 640 + 512
     assert bn.bitnet_tl_packed_bytes("tl1", 64, 130) == 2 * 3 * 512
@@ -51,7 +51,7 @@ def test_size_queries(L):
     assert bn.bitnet_tl_num_groups("tl2", 8192) == 86 * 32
     assert bn.bitnet_mpgemm_workspace_bytes("i2s", 1, 8192, 8192) == 0
     assert bn.bitnet_mpgemm_workspace_bytes("i2s", 1, 8192, 28672) == 0        # in-CTA reduction
-    assert bn.bitnet_mpgemm_workspace_bytes("i2s", 1, 1 << 22, 1 << 17) >= 2 * (1 << 22) * 4  # falls back to split-K
+    assert bn.bitnet_mpgemm_workspace_bytes("i2s", 8, 1 << 20, 1 << 17) == 0      # long K is walked slab by slab
     assert bn.bitnet_mpgemm_workspace_bytes("tl2", 1, 8192, 28672) >= 2 * 8192 * 4
 
 
@@ -73,7 +73,6 @@ def test_host_validation_returns_codes_without_a_gpu(L):
     # split-K shape without a workspace
     assert L.bitnet_mpgemm(2, fake, 1.0, 64, 28672, 0, fake, fake, 1, fake, null, null, 0, null) == 3
     assert L.bitnet_mpgemm(1, fake, 1.0, 32, 64, 0, fake, fake, 1, fake, null, fake, 16, null) == 3   # too small
-    assert L.bitnet_mpgemm(0, fake, 1.0, 1 << 22, 1 << 17, 0, fake, fake, 1, fake, null, null, 0, null) == 3
 
 
 def test_missing_library_raises(monkeypatch, tmp_path):

@@ -139,6 +139,16 @@ def test_i2s_very_long_k_runs_in_phases():
         check_linear("i2s", tern(34, M, K), synth.normal(34, T, T, K))
 
 
+def test_tl_many_row_blocks_few_tiles():
+    # more row blocks per CTA than the kernel keeps cross-warp sums for, and fewer tiles than warps
+    M, K = 32 * 296 * 70, 96
+    w, x = tern(35, M, K), synth.normal(35, 1, 2, K)
+    for fmt in ("tl2", "tl1"):
+        out = run_linear(fmt, w, x)
+        q_ref, sc_ref, _ = oracle.quant_act(x.numpy())
+        assert np.array_equal(npy(out["acc"]), oracle.mpgemm_def(q_ref, w.numpy()))
+
+
 def test_formats_agree_on_accumulators():
     M, K, T = 128, 8192, 3
     w, x = tern(32, M, K), synth.normal(32, 1, T, K)

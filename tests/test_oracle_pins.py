@@ -139,7 +139,7 @@ def test_i2s_size_and_bpw():
     assert oracle.i2s_packed_bytes(1536, 1536) == 1536 * 1536 // 4        # exactly 2 bits per weight
     assert oracle.i2s_packed_bytes(3200, 8640) == 3200 * 8704 // 4        # K padded to 256 columns
     assert oracle.i2s_packed_bytes(8192, 28672) * 8 == 2 * 8192 * 28672
-    assert oracle.i2s_packed_bytes(3, 64) == 8 * 256 // 4                 # rows padded to 8
+    assert oracle.i2s_packed_bytes(3, 64) == 16 * 256 // 4                # rows padded to 16
 
 
 def test_i2s_round_trip_and_padding_code():
@@ -150,35 +150,36 @@ def test_i2s_round_trip_and_padding_code():
         assert np.array_equal(oracle.unpack_i2s(p, M, K), w)
     # all-zero weights: every 2-bit field, padding included, holds code 1
     p = oracle.pack_i2s(np.zeros((3, 64), np.int8))
-    assert p.size == 512 and np.all(p == 0b01010101)
+    assert p.size == 1024 and np.all(p == 0b01010101)
 
 
 def _i2s_byte_and_shift(m, k, K):
     """The documented position of weight (m, k), written out independently of the oracle."""
     kp = -(-K // 256) * 256
-    rb, r, c, kk = m // 8, m % 8, k // 256, k % 256
+    rb, r, c, kk = m // 16, m % 16, k // 256, k % 256
     word = 2 * (kk // 32) + (kk % 8) // 4
-    return rb * 2 * kp + c * 512 + r * 64 + 4 * word + kk % 4, 2 * ((kk % 32) // 8)
+    return rb * 4 * kp + c * 1024 + r * 64 + 4 * word + kk % 4, 2 * ((kk % 32) // 8)
 
 
 def test_i2s_documented_bit_positions():
     # every column of one chunk plus positions in other rows, row blocks and chunks; checked against
     # hand-built bytes
-    M, K = 11, 512
-    probes = [(0, k) for k in range(256)] + [(3, 5), (7, 255), (8, 0), (10, 300), (9, 511), (1, 256)]
+    M, K = 19, 512
+    probes = [(0, k) for k in range(256)] + [(3, 5), (7, 255), (8, 0), (10, 300), (15, 511), (1, 256), (16, 0), (18, 77)]
     for (m, k) in probes:
         for val in (-1, 1):
             w = np.zeros((M, K), np.int8)
             w[m, k] = val
             p = oracle.pack_i2s(w)
             byte, shift = _i2s_byte_and_shift(m, k, K)
-            expect = np.full(16 * 512 // 4, 0b01010101, np.uint8)
+            expect = np.full(32 * 512 // 4, 0b01010101, np.uint8)
             expect[byte] = (0b01010101 & ~(3 << shift)) | ((val + 1) << shift)
             assert np.array_equal(p, expect), (m, k)
     # spot values of the formula itself: k = 0, 4, 8, 32 of row 0 and k = 0 of row 1
     assert _i2s_byte_and_shift(0, 0, 256) == (0, 0) and _i2s_byte_and_shift(0, 4, 256) == (4, 0)
     assert _i2s_byte_and_shift(0, 8, 256) == (0, 2) and _i2s_byte_and_shift(0, 32, 256) == (8, 0)
     assert _i2s_byte_and_shift(1, 0, 256) == (64, 0) and _i2s_byte_and_shift(8, 0, 256) == (512, 0)
+    assert _i2s_byte_and_shift(16, 0, 256) == (1024, 0) and _i2s_byte_and_shift(0, 256, 512) == (1024, 0)
 
 
 def test_i2s_one_hot_dot_products():
