@@ -359,7 +359,7 @@ def run_ours(args):
                 "h2d_bytes_per_step": int(sw.x_host.numel() * 4), "d2h_bytes_per_step": int(sw.y_host.numel() * 4),
                 "note": "per linear: pinned fp32 x -> device, quantiser, mpGEMV, fp32 y -> pinned host; weights resident"},
         "gpu_launches": n_lin * args.steps,
-        "roofline": {"bound": "hbm", "kernel": "gemv_i2s_mma_kernel (quantiser fused)", "achieved": achieved,
+        "roofline": {"bound": "hbm", "kernel": "gemv_i2s_wring_kernel (quantiser fused)", "achieved": achieved,
                      "peak": pk["hbm"], "unit": "GB/s", "frac": achieved / pk["hbm"], "peak_source": pk["which"],
                      "bytes_per_launch": sw.bytes["i2s"] / n_lin, "us_per_launch": 1e3 * ms_step / n_lin,
                      "traffic": None},

@@ -87,6 +87,10 @@ bool gemv_i2s_stream_supported(int T, int64_t M, int64_t K, bool fused);
 int launch_gemv_i2s_stream(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const float* x, int8_t* q,
                            float* act_scale, int T, float* y, int32_t* acc_out, cudaStream_t st);
 int gemv_i2s_stream_status(int* out);
+// Warp-private cp.async rings + tensor-core MMA; two consecutive kernels' CTAs share an SM.
+bool gemv_i2s_wring_supported(int T, int64_t M, int64_t K);
+int launch_gemv_i2s_wring(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const float* x, int8_t* q,
+                          float* act_scale, int T, float* y, int32_t* acc_out, cudaStream_t st);
 // Programmatic dependent launch (kernels may start their prologue, and prefetch weights, before the
 // previous kernel in the stream has finished); process-wide switch, on by default.
 bool early_start_enabled();

@@ -35,6 +35,9 @@
 //
 // Every wait on an mbarrier is bounded; a wait that gives up raises a device flag that
 // bitnet_device_status() reports, and the thread leaves the kernel.
+#include <cstdlib>
+#include <cstring>
+
 #include "common.cuh"
 
 namespace bitnet {
@@ -49,6 +52,22 @@ constexpr int ACC_RING = 16;             // cross-warp accumulator entries (more
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 static __device__ int g_stream_error = 0;
+
+#ifdef BITNET_PROFILE_GEMV
+// Development aid (never in the shipped build): per launch and CTA, %globaltimer at a few points.
+static __device__ unsigned long long g_tl[256][148][6];
+static int g_tl_launch = 0;
+__device__ __forceinline__ unsigned long long gtime() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define TL_MARK(i) do { if (blockIdx.x < 148) g_tl[a.launch_id & 255][blockIdx.x][i] = gtime(); } while (0)
+#define TL_MAX(i) do { if (blockIdx.x < 148) atomicMax(&g_tl[a.launch_id & 255][blockIdx.x][i], gtime()); } while (0)
+#else
+#define TL_MARK(i) do { } while (0)
+#define TL_MAX(i) do { } while (0)
+#endif
 
 struct MmaArgs {
   const uint8_t* packed;
@@ -73,6 +92,7 @@ struct MmaArgs {
   int ngroups;           // warp groups; group g takes the CTA's units g, g + ngroups, ...
   int nunits;            // ceil(M / 16)
   int slots;             // ring slots
+  int launch_id;         // profiling builds only
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -174,6 +194,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_mma_kernel(const MmaArgs 
   };
 
   if (threadIdx.x == 0) {
+    TL_MARK(0);
+    if (blockIdx.x < 148) { TL_MARK(5); }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may begin its prologue
     for (int s = 0; s < a.slots; ++s) mbar_init(smem_u32(full + s), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -185,12 +207,14 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_mma_kernel(const MmaArgs 
   const bool idle = group >= a.ngroups;   // warps that do not fit a whole group only help in the prologue
   const int wk = warp % a.wpt;            // this warp's chunks inside a slab: wk*KS .. wk*KS+KS-1
   const int g = lane >> 2, t = lane & 3;
-  // one warp per slot requests the initial contents of the ring (after the activation loads, if any, are on
-  // their way: the issuing lane is held for a few hundred cycles)
-  const bool my_fill = lane == 0 && warp < a.slots && warp < total;
+  // One warp per slot requests the initial contents of the ring.  The weights do not depend on the previous
+  // kernel in the stream, so this happens before the wait below: a CTA that starts while that kernel's
+  // last CTAs are still running already streams.
+  if (lane == 0 && warp < a.slots && warp < total) fill(warp, warp);
 
   // ---------------- activations come from the previous kernel in the stream
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (threadIdx.x == 0) TL_MARK(1);
 
   if (a.use_qs) {
     if (a.x && a.T == 1 && a.K <= 4 * XREG * THREADS) {
@@ -205,7 +229,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_mma_kernel(const MmaArgs 
         const int i = threadIdx.x + r * THREADS;
         xv[r] = (i < n4) ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
       }
-      if (my_fill) fill(warp, warp);
       float m = 0.0f;
 #pragma unroll
       for (int r = 0; r < XREG; ++r)
@@ -246,7 +269,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_mma_kernel(const MmaArgs 
         for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
         if (lane == 0) qred[tok * CW + warp] = m;
       }
-      if (my_fill) fill(warp, warp);
       __syncthreads();
       if (threadIdx.x < a.T) {
         float m = 0.0f;
@@ -278,12 +300,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_mma_kernel(const MmaArgs 
           reinterpret_cast<int*>(qs_mem + tok * kp)[i] = (i < (int)(a.K / 4)) ? __ldcg(q4 + i) : 0;
       }
       if (threadIdx.x < a.T) qscale[threadIdx.x] = __ldcg(a.act_scale + threadIdx.x);
-      if (my_fill) fill(warp, warp);
     }
     __syncthreads();
-  } else if (my_fill) {
-    fill(warp, warp);
   }
+  if (threadIdx.x == 0) TL_MARK(2);
   if (idle) return;
 
   // rescale factors of the tokens this lane stores when its warp finishes a unit (token (lane>>4) + 2i)
@@ -351,6 +371,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_mma_kernel(const MmaArgs 
         if (lane == 0) atomicExch(&g_stream_error, BITNET_ERR_TIMEOUT);
         return;
       }
+      if (threadIdx.x == 0 && seq == 0) TL_MARK(3);
       const uint8_t* pa = ring + lane_off + slot * a.stage_bytes;
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
@@ -432,6 +453,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_mma_kernel(const MmaArgs 
       if (lane == 0) atomicExch(cnt + e, 0);
     }
   }
+  if (threadIdx.x == 0) TL_MARK(4);
+  if (lane == 0) TL_MAX(5);
 }
 
 struct Plan {
@@ -494,7 +517,18 @@ int launch_mma(const MmaArgs& a, const Plan& p, cudaStream_t st) {
 
 }  // namespace
 
+// The warp-private-ring kernel is the default; BITNET_I2S_STREAM=ring selects this file's kernel.
+static bool prefer_wring() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("BITNET_I2S_STREAM");
+    v = (e && strcmp(e, "ring") == 0) ? 0 : 1;
+  }
+  return v == 1;
+}
+
 bool gemv_i2s_stream_supported(int T, int64_t M, int64_t K, bool fused) {
+  if (prefer_wring() && gemv_i2s_wring_supported(T, M, K)) return true;
   Plan p;
   return T >= 1 && T <= 8 && make_plan(T, M, K, fused, &p);
 }
@@ -502,6 +536,8 @@ bool gemv_i2s_stream_supported(int T, int64_t M, int64_t K, bool fused) {
 // x != nullptr: fused quantiser (q, act_scale are then outputs); otherwise q, act_scale are inputs.
 int launch_gemv_i2s_stream(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const float* x, int8_t* q,
                            float* act_scale, int T, float* y, int32_t* acc_out, cudaStream_t st) {
+  if (prefer_wring() && gemv_i2s_wring_supported(T, M, K))
+    return launch_gemv_i2s_wring(packed, w_scale, M, K, x, q, act_scale, T, y, acc_out, st);
   Plan p;
   if (T < 1 || T > 8 || !make_plan(T, M, K, x != nullptr, &p)) return BITNET_ERR_UNSUPPORTED_SHAPE;
   MmaArgs a;
@@ -527,6 +563,10 @@ int launch_gemv_i2s_stream(const uint8_t* packed, float w_scale, int64_t M, int6
   a.ngroups = p.ngroups;
   a.nunits = p.nunits;
   a.slots = p.slots;
+  a.launch_id = 0;
+#ifdef BITNET_PROFILE_GEMV
+  a.launch_id = g_tl_launch++;
+#endif
   switch (p.KS) {
     case 1: return launch_mma<1>(a, p, st);
     case 2: return launch_mma<2>(a, p, st);
@@ -540,5 +580,17 @@ int gemv_i2s_stream_status(int* out) {
   cudaError_t e = cudaMemcpyFromSymbol(out, g_stream_error, sizeof(int));
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
 }
+
+#ifdef BITNET_PROFILE_GEMV
+extern "C" int bitnet_debug_timeline(unsigned long long* out, int reset) {
+  if (reset) {
+    g_tl_launch = 0;
+    void* p = nullptr;
+    cudaGetSymbolAddress(&p, g_tl);
+    return (int)cudaMemset(p, 0, sizeof(g_tl));
+  }
+  return (int)cudaMemcpyFromSymbol(out, g_tl, sizeof(g_tl));
+}
+#endif
 
 }  // namespace bitnet

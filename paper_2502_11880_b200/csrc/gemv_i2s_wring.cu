@@ -1,0 +1,515 @@
+// I2_S mpGEMV for decode (1..8 tokens), warp-private rings: Alg. 1 Phase 2 from the 2-bit blob with
+// the quantiser (Phase 1) optionally fused in.
+//
+// Why this shape.  A decode step is a chain of dependent kernels that each stream a few tens of MB once;
+// what decides the chain's speed is how little of the time HBM sits idle between and inside kernels.
+// So the kernel is made small enough that the CTAs of TWO consecutive kernels fit on an SM together
+// (512 threads, at most 64 registers, about half the shared memory): under programmatic dependent launch
+// the next kernel's CTAs become resident while this one still runs, request their first weights -- which
+// depend on nothing -- and only then wait for this kernel to finish.  The gap between kernels, the
+// quantiser prologue and the tail of a kernel are then covered by the neighbour's weight traffic.
+//
+// Memory side.  The blob stores 16-row units contiguously and chunk-major (1024 bytes per 256-column
+// chunk, 64 bytes per row).  A unit is shared by S warps (S a power of two), each owning a K-slice of the
+// unit.  Every warp streams the chunks of its slices through a private ring in shared memory with
+// per-thread asynchronous 16-byte copies (cp.async, L2 evict-first): lane l copies bytes [16l, 16l+16)
+// and [512+16l, ...) of a chunk and later reads back exactly those bytes, so the only synchronisation
+// of the stream is the thread's own cp.async.wait_group -- no barrier, no producer, no handshake.  The
+// ring runs DEPTH chunks ahead and crosses unit boundaries.
+//
+// Work distribution.  Unit u belongs to CTA u mod gridDim; inside the CTA the warp groups take the
+// CTA's units from a shared counter, DEPTH units ahead of use (the prefetcher must know where the
+// stream continues), so a group that falls behind simply takes fewer units.
+//
+// Compute side.  A chunk of a unit is the A operand of 8 int8 tensor-core MMAs (mma.sync m16n8k32,
+// u8 x s8 -> s32): lane (g = lane/4, t = lane%4) holds 64 weights of row g and of row g+8.  Masking a
+// packed word with 0x03030303 << 2s leaves, without a shift, the four codes of slot s scaled by 4^s:
+// one A register.  The B operand is the activations (column n = token n), read from shared memory.
+// Four accumulator fragments carry the scales 1, 4, 16, 64; each is an exact multiple of its scale, so
+// arithmetic shifts undo it, and sum(code*q) - sum(q) = sum(w*q).  The S partial fragments of a unit
+// meet in shared memory at a named barrier of the group; one warp (rotating) adds them, rescales and
+// stores y = acc * act_scale[t] * w_scale.
+//
+// Fused quantiser: with fp32 activations given, every CTA computes absmax and the int8 codes itself,
+// after its first weight copies are in flight; CTA 0 also stores the codes and scales for the caller.
+#include <cstdlib>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace bitnet {
+namespace {
+
+constexpr int CW = 16;                   // warps
+constexpr int THREADS = CW * 32;
+constexpr int JQ = 4;                    // entries of a group's queue of upcoming units
+constexpr int XREG = 16;                 // float4 registers per thread of the fused quantiser's fast path
+constexpr size_t MAX_QS_BYTES = 64 * 1024;   // activations staged in shared memory up to this size
+
+#ifdef BITNET_PROFILE_GEMV
+// Development aid (never in the shipped build): per launch and CTA, %globaltimer at a few points.
+static __device__ unsigned long long g_tl[256][148][6];
+static int g_tl_launch = 0;
+__device__ __forceinline__ unsigned long long gtime() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+static __device__ unsigned long long g_steps[256][4][24];
+#define TL_STEP(i) do { if ((blockIdx.x % 37) == 0 && blockIdx.x < 148 && threadIdx.x == 0 && n == 0 && (i) < 24) g_steps[a.launch_id & 255][blockIdx.x / 37][i] = gtime(); } while (0)
+#define TL_MARK(i) do { if (blockIdx.x < 148) g_tl[a.launch_id & 255][blockIdx.x][i] = gtime(); } while (0)
+#define TL_MAX(i) do { if (blockIdx.x < 148) atomicMax(&g_tl[a.launch_id & 255][blockIdx.x][i], gtime()); } while (0)
+#else
+#define TL_MARK(i) do { } while (0)
+#define TL_MAX(i) do { } while (0)
+#define TL_STEP(i) do { } while (0)
+#endif
+
+struct WArgs {
+  int launch_id;         // profiling builds only
+  const uint8_t* packed;
+  int64_t unit_bytes;    // bytes of one 16-row unit of the blob = 4 * Kp
+  int M;
+  int64_t K;
+  const int8_t* q;       // quantised activations [T][K] (input, or output of the fused quantiser)
+  const float* act_scale;
+  const float* x;        // fp32 activations [T][K]: non-null selects the fused quantiser
+  int8_t* q_out;         // fused mode: CTA 0 stores the codes and scales here
+  float* scale_out;
+  float w_scale;
+  int T;
+  float* y;
+  int32_t* acc_out;
+  int nchunks;           // 256-column chunks per row (Kp / 256)
+  int S;                 // warps per unit
+  int KC;                // chunks per warp and unit (the last warp of a unit may have fewer, or none)
+  int nunits;            // ceil(M / 16)
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp16(uint32_t dst, const void* src, uint64_t pol) {
+  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(pol)
+               : "memory");
+}
+__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void group_barrier(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+// D(16x8, s32) += A(16x32, u8, row) * B(32x8, s8, col).  Lane (g = lane/4, t = lane%4):
+// a0 = row g, k 4t..4t+3; a1 = row g+8, same k; a2, a3 = the same rows, k 16+4t..; b0 = k 4t..4t+3 of
+// column g, b1 = k 16+4t..; c0,c1 = row g, columns 2t, 2t+1; c2,c3 = row g+8.
+__device__ __forceinline__ void mma_u8s8(int (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, int b0,
+                                         int b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ int quant1(float x, float s) {
+  return max(-128, min(127, __float2int_rn(__fmul_rn(x, s))));
+}
+__device__ __forceinline__ int quant4(const float4& v, float s) {
+  return (quant1(v.x, s) & 255) | ((quant1(v.y, s) & 255) << 8) | ((quant1(v.z, s) & 255) << 16) |
+         ((quant1(v.w, s) & 255) << 24);
+}
+
+// shared memory: [unit counter, unit queues, quantiser scratch: 2 KB][partials][codes][rings]
+__host__ __device__ inline size_t red_bytes(int T) { return (size_t)CW * 2 * T * 16 * 4; }
+
+template <int DEPTH>
+__global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs a) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  int* counter = reinterpret_cast<int*>(smem);                 // next unit (index into the CTA's list) to hand out
+  int* jq = reinterpret_cast<int*>(smem + 64);                 // [groups][JQ] upcoming units of each group
+  float* qscale = reinterpret_cast<float*>(smem + 1152);       // [8] act_scale per token
+  float* qred = qscale + 8;                                    // [8][16] partial maxima / multipliers
+  int* red = reinterpret_cast<int*>(smem + 2048);              // [CW][2][T][16] partial sums
+  const int kp = a.nchunks * 256;
+  int8_t* qs_mem = reinterpret_cast<int8_t*>(smem + 2048 + red_bytes(a.T));
+  uint8_t* rings = reinterpret_cast<uint8_t*>(qs_mem) + (((size_t)a.T * kp + 127) & ~(size_t)127);
+
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int G = CW / a.S;                      // groups
+  const int gi = warp / a.S;                   // this warp's group
+  const int wk = warp % a.S;                   // its place in the group = its K-slice
+  const int g = lane >> 2, t = lane & 3;
+  const int n_units = (a.nunits - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+  const int c_lo = wk * a.nchunks / a.S, c_hi = (wk + 1) * a.nchunks / a.S;   // this warp's K-slice, >= DEPTH chunks
+
+  if (threadIdx.x == 0) {
+    TL_MARK(0);
+    TL_MARK(5);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may become resident
+    *counter = 2 * G;
+  }
+  // the first two units of each group are fixed: unit i of group gi is gi + i * G
+  if (threadIdx.x < G * JQ) {
+    const int i = threadIdx.x % JQ;
+    jq[threadIdx.x] = (i <= 1) ? (threadIdx.x / JQ) + i * G : 0x7fffffff;
+  }
+  __syncthreads();
+
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+
+  // ---------------- the warp's stream of chunks: its slice of the group's unit 0, of unit 1, ...
+  // The ring holds DEPTH consecutive chunks of that stream; slot_off is the slot of the chunk consumed next.
+  const uint32_t ring = smem_u32(rings + (size_t)warp * DEPTH * 1024) + lane * 16;
+  const uint8_t* const base = a.packed + (int64_t)blockIdx.x * a.unit_bytes + (int64_t)c_lo * 1024 + lane * 16;
+  const int64_t unit_stride = (int64_t)gridDim.x * a.unit_bytes;
+  const volatile int* my_jq = jq + gi * JQ;
+  const int nw = c_hi - c_lo;
+  uint32_t slot_off = 0;
+  // Weights do not depend on the previous kernel in the stream: request the first DEPTH chunks now.
+  {
+    const int j0 = my_jq[0];
+    const uint8_t* src = base + (int64_t)j0 * unit_stride;
+#pragma unroll
+    for (int d = 0; d < DEPTH; ++d) {
+      if (j0 < n_units) {
+        cp16(ring + d * 1024, src + d * 1024, pol);
+        cp16(ring + d * 1024 + 512, src + d * 1024 + 512, pol);
+      }
+      cp_commit();
+    }
+  }
+
+  // ---------------- activations come from the previous kernel in the stream
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (threadIdx.x == 0) TL_MARK(1);
+
+  if (a.x && a.T == 1 && a.K <= 4 * XREG * THREADS) {
+    // ---- fused quantiser (Alg. 1 Phase 1), one token, one round trip: the row stays in registers
+    // between the amax pass and the rounding pass.  Same operations and order as the stand-alone
+    // kernel: s = 127 / max(amax, 1e-5), q = clamp(rint(x * s)).
+    const float4* x4 = reinterpret_cast<const float4*>(a.x);
+    const int n4 = (int)(a.K / 4);
+    float4 xv[XREG];
+#pragma unroll
+    for (int r = 0; r < XREG; ++r) {
+      const int i = threadIdx.x + r * THREADS;
+      xv[r] = (i < n4) ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    float m = 0.0f;
+#pragma unroll
+    for (int r = 0; r < XREG; ++r)
+      m = fmaxf(m, fmaxf(fmaxf(fabsf(xv[r].x), fabsf(xv[r].y)), fmaxf(fabsf(xv[r].z), fabsf(xv[r].w))));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) qred[warp] = m;
+    __syncthreads();
+    float amax = 0.0f;
+#pragma unroll
+    for (int w2 = 0; w2 < CW; ++w2) amax = fmaxf(amax, qred[w2]);
+    const float amax_c = fmaxf(amax, 1e-5f);
+    const float sq = __fdiv_rn(127.0f, amax_c);
+    if (threadIdx.x == 0) {
+      const float inv = __fdiv_rn(amax_c, 127.0f);
+      qscale[0] = inv;
+      if (blockIdx.x == 0 && a.scale_out) a.scale_out[0] = inv;
+    }
+#pragma unroll
+    for (int r = 0; r < XREG; ++r) {
+      const int i = threadIdx.x + r * THREADS;
+      if (i < kp / 4) {
+        const int word = quant4(xv[r], sq);                 // columns K..Kp-1 came in as zeros
+        reinterpret_cast<int*>(qs_mem)[i] = word;
+        if (blockIdx.x == 0 && a.q_out && i < n4) reinterpret_cast<int*>(a.q_out)[i] = word;
+      }
+    }
+  } else if (a.x) {
+    // ---- fused quantiser, general form: amax per token, then a second pass over x
+    for (int tok = 0; tok < a.T; ++tok) {
+      const float4* x4 = reinterpret_cast<const float4*>(a.x + (int64_t)tok * a.K);
+      float m = 0.0f;
+      for (int i = threadIdx.x; i < (int)(a.K / 4); i += THREADS) {
+        const float4 v = __ldcg(x4 + i);
+        m = fmaxf(m, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      if (lane == 0) qred[tok * CW + warp] = m;
+    }
+    __syncthreads();
+    if (threadIdx.x < a.T) {
+      float m = 0.0f;
+      for (int w2 = 0; w2 < CW; ++w2) m = fmaxf(m, qred[threadIdx.x * CW + w2]);
+      const float amax_c = fmaxf(m, 1e-5f);
+      qred[threadIdx.x * CW] = __fdiv_rn(127.0f, amax_c);
+      const float inv = __fdiv_rn(amax_c, 127.0f);
+      qscale[threadIdx.x] = inv;
+      if (blockIdx.x == 0 && a.scale_out) a.scale_out[threadIdx.x] = inv;
+    }
+    __syncthreads();
+    for (int tok = 0; tok < a.T; ++tok) {
+      const float sq = qred[tok * CW];
+      const float4* x4 = reinterpret_cast<const float4*>(a.x + (int64_t)tok * a.K);
+      for (int i = threadIdx.x; i < kp / 4; i += THREADS) {
+        int word = 0;
+        if (i < (int)(a.K / 4)) {
+          word = quant4(__ldcg(x4 + i), sq);
+          if (blockIdx.x == 0 && a.q_out) reinterpret_cast<int*>(a.q_out + (int64_t)tok * a.K)[i] = word;
+        }
+        reinterpret_cast<int*>(qs_mem + tok * kp)[i] = word;
+      }
+    }
+  } else {
+    // ---- stage the given codes (zero beyond K)
+    for (int tok = 0; tok < a.T; ++tok) {
+      const int* q4 = reinterpret_cast<const int*>(a.q + (int64_t)tok * a.K);
+      for (int i = threadIdx.x; i < kp / 4; i += THREADS)
+        reinterpret_cast<int*>(qs_mem + tok * kp)[i] = (i < (int)(a.K / 4)) ? __ldcg(q4 + i) : 0;
+    }
+    if (threadIdx.x < a.T) qscale[threadIdx.x] = __ldcg(a.act_scale + threadIdx.x);
+  }
+  __syncthreads();
+
+  if (threadIdx.x == 0) TL_MARK(2);
+  // sum of the activations of tokens 2t and 2t+1 over this warp's K-slice (the "- sum(q)" term)
+  int corr_even = 0, corr_odd = 0;
+  for (int tok = 0; tok < a.T; ++tok) {
+    int s = 0, s2 = 0;
+    const uint4* qw = reinterpret_cast<const uint4*>(qs_mem + tok * kp + c_lo * 256);
+    for (int i = lane; i < (c_hi - c_lo) * 16; i += 32) {
+      const uint4 v = qw[i];
+      s = __dp4a((int)v.x, 0x01010101, s);
+      s2 = __dp4a((int)v.y, 0x01010101, s2);
+      s = __dp4a((int)v.z, 0x01010101, s);
+      s2 = __dp4a((int)v.w, 0x01010101, s2);
+    }
+    s += s2;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (tok == 2 * t) corr_even = s;
+    if (tok == 2 * t + 1) corr_odd = s;
+  }
+  // Token g's codes under this lane's 16-byte weight column: 64 bytes per chunk.  Columns of B beyond
+  // the batch produce columns of D nobody stores, so those lanes simply read the last token again.
+  const int8_t* const q_lane = qs_mem + min(g, a.T - 1) * kp + c_lo * 256 + t * 64;
+  const int bar_id = 1 + gi, bar_threads = a.S * 32;
+
+  // One step: wait for the oldest chunk of the ring, put it through the tensor cores, then refill its slot
+  // from `pf` (the chunk DEPTH places further down the stream), if there is one.
+  int C[4][4];
+  const uint4* qp = nullptr;
+  auto step = [&](const uint8_t* pf, bool do_pf) {
+    cp_wait<DEPTH - 1>();
+    unsigned w4[4], v4[4];
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(w4[0]), "=r"(w4[1]), "=r"(w4[2]), "=r"(w4[3])
+                 : "r"(ring + slot_off));
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v4[0]), "=r"(v4[1]), "=r"(v4[2]), "=r"(v4[3])
+                 : "r"(ring + slot_off + 512));
+    // words 2h, 2h+1 of the lane's 16 bytes, slot s: weights 32h + 8s + (0..7) of its 64 columns,
+    // i.e. activation words 8h + 2s and 8h + 2s + 1
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const uint4 qa = qp[2 * h], qb = qp[2 * h + 1];
+      const int qr[8] = {(int)qa.x, (int)qa.y, (int)qa.z, (int)qa.w, (int)qb.x, (int)qb.y, (int)qb.z, (int)qb.w};
+#pragma unroll
+      for (int s = 0; s < 4; ++s) {
+        const unsigned m = 0x03030303u << (2 * s);
+        mma_u8s8(C[s], w4[2 * h] & m, v4[2 * h] & m, w4[2 * h + 1] & m, v4[2 * h + 1] & m, qr[2 * s], qr[2 * s + 1]);
+      }
+    }
+    qp += 16;
+    // the chunk's bytes were in registers before the MMAs above were issued: its slot can be refilled
+    if (do_pf) {
+      cp16(ring + slot_off, pf, pol);
+      cp16(ring + slot_off + 512, pf + 512, pol);
+    }
+    cp_commit();
+    slot_off = (slot_off + 1024 == DEPTH * 1024) ? 0 : slot_off + 1024;
+  };
+
+  for (int n = 0;; ++n) {
+    const int j = my_jq[n & (JQ - 1)];
+    if (j >= n_units) break;
+    const int jn = my_jq[(n + 1) & (JQ - 1)];
+    // The group's first warp draws the unit after the next; the barrier at the end of this unit publishes
+    // it before anyone looks for it.  (A warp's slice is at least as long as its ring, so its requests
+    // never reach beyond the next unit.)
+    if (wk == 0 && lane == 0) jq[gi * JQ + ((n + 2) & (JQ - 1))] = atomicAdd(counter, 1);
+
+#pragma unroll
+    for (int s = 0; s < 4; ++s)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) C[s][i] = 0;
+    qp = reinterpret_cast<const uint4*>(q_lane);
+    TL_STEP(0);
+
+    // chunks 0 .. nw-DEPTH-1 are followed, DEPTH places on, by chunks of the same unit
+    const uint8_t* pf = base + (int64_t)j * unit_stride + DEPTH * 1024;
+#pragma unroll 2
+    for (int left = nw - DEPTH; left > 0; --left, pf += 1024) { step(pf, true); TL_STEP(nw - DEPTH - left + 1); }
+    // the last DEPTH chunks by the first DEPTH chunks of the group's next unit, if there is one
+    pf = base + (int64_t)jn * unit_stride;
+    const bool more = jn < n_units;
+#pragma unroll
+    for (int d = 0; d < DEPTH; ++d) { step(pf + d * 1024, more); TL_STEP(nw - DEPTH + d + 1); }
+
+    if (threadIdx.x == 0 && n == 0) TL_MARK(3);
+    // fragment: c[0] = (row g, token 2t), c[1] = (row g, token 2t+1), c[2], c[3] = the same for row g+8
+    int c[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) c[i] = C[0][i] + (C[1][i] >> 2) + (C[2][i] >> 4) + (C[3][i] >> 6);
+    int* mine = red + ((warp * 2 + (n & 1)) * a.T) * 16;
+    if (2 * t < a.T) {
+      mine[(2 * t) * 16 + g] = c[0] - corr_even;
+      mine[(2 * t) * 16 + g + 8] = c[2] - corr_even;
+    }
+    if (2 * t + 1 < a.T) {
+      mine[(2 * t + 1) * 16 + g] = c[1] - corr_odd;
+      mine[(2 * t + 1) * 16 + g + 8] = c[3] - corr_odd;
+    }
+    if (a.S > 1) group_barrier(bar_id, bar_threads);
+    else __syncwarp();
+    if (wk == (n & (a.S - 1))) {
+      // this unit's turn to be finished by this warp: add the group's partials, rescale, store 16 rows
+      const int row0 = ((int)blockIdx.x + j * (int)gridDim.x) * 16;
+      const int* grp = red + (((gi * a.S) * 2 + (n & 1)) * a.T) * 16;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int idx = lane + 32 * i;
+        if (idx < a.T * 16) {
+          int v = 0;
+          for (int w2 = 0; w2 < a.S; ++w2) v += grp[w2 * 2 * a.T * 16 + idx];
+          const int tok = idx >> 4, row = row0 + (idx & 15);
+          if (row < a.M) {
+            a.y[(int64_t)tok * a.M + row] = __fmul_rn((float)v, __fmul_rn(qscale[tok], a.w_scale));
+            if (a.acc_out) a.acc_out[(int64_t)tok * a.M + row] = v;
+          }
+        }
+      }
+    }
+  }
+  cp_wait<0>();
+  if (threadIdx.x == 0) TL_MARK(4);
+  if (lane == 0) TL_MAX(5);
+}
+
+struct Plan {
+  int nchunks, S, KC, nunits, grid, depth;
+  size_t smem;
+};
+
+int env_int(const char* name, int dflt) {
+  const char* v = getenv(name);
+  return (v && *v) ? atoi(v) : dflt;
+}
+
+bool make_plan(int T, int64_t M, int64_t K, Plan* p) {
+  p->nchunks = (int)(i2s_kp(K) / 256);
+  const int forced = env_int("BITNET_I2S_DEPTH", 0);
+  int depth = (forced == 12 || forced == 8 || forced == 6 || forced == 4) ? forced : 8;
+  while (depth > 4 && 2048 + red_bytes(T) + (((size_t)T * p->nchunks * 256 + 127) & ~(size_t)127) +
+                              (size_t)CW * depth * 1024 > (size_t)dev_info().max_smem_optin)
+    depth -= 2;
+  if (depth == 10) depth = 8;
+  if (p->nchunks < depth) return false;     // a warp's slice is at least as long as the ring
+  // warps per unit: as many as leave every warp about kc_target chunks of a unit (never fewer than the ring)
+  int kc_target = env_int("BITNET_I2S_KC", 16);
+  if (kc_target < depth) kc_target = depth;
+  int S = 1;
+  while (S < CW && p->nchunks / (2 * S) >= kc_target) S *= 2;
+  p->S = S;
+  p->KC = (p->nchunks + S - 1) / S;
+  p->nunits = (int)ceil_div(M, 16);
+  const int ctas = dev_info().sm_count * env_int("BITNET_I2S_CTAS", 1);
+  p->grid = ctas < p->nunits ? ctas : p->nunits;
+  const size_t qs_bytes = ((size_t)T * p->nchunks * 256 + 127) & ~(size_t)127;
+  if (qs_bytes > MAX_QS_BYTES) return false;
+  p->depth = depth;
+  p->smem = 2048 + red_bytes(T) + qs_bytes + (size_t)CW * depth * 1024;
+  return p->smem <= (size_t)dev_info().max_smem_optin;
+}
+
+template <int DEPTH>
+int launch_wring(const WArgs& a, const Plan& p, cudaStream_t st) {
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (!attr_set[dev & 63]) {
+    cudaError_t e = cudaFuncSetAttribute(gemv_i2s_wring_kernel<DEPTH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         dev_info().max_smem_optin);
+    if (e != cudaSuccess) return note_cuda_error(e);
+    attr_set[dev & 63] = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)p.grid);
+  cfg.blockDim = dim3(THREADS);
+  cfg.dynamicSmemBytes = p.smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = early_start_enabled() ? 1 : 0;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_i2s_wring_kernel<DEPTH>, a);
+  return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
+}
+
+}  // namespace
+
+bool gemv_i2s_wring_supported(int T, int64_t M, int64_t K) {
+  Plan p;
+  return T >= 1 && T <= 8 && make_plan(T, M, K, &p);
+}
+
+// x != nullptr: fused quantiser (q, act_scale are then outputs); otherwise q, act_scale are inputs.
+int launch_gemv_i2s_wring(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const float* x, int8_t* q,
+                          float* act_scale, int T, float* y, int32_t* acc_out, cudaStream_t st) {
+  Plan p;
+  if (T < 1 || T > 8 || !make_plan(T, M, K, &p)) return BITNET_ERR_UNSUPPORTED_SHAPE;
+  WArgs a;
+  a.launch_id = 0;
+#ifdef BITNET_PROFILE_GEMV
+  a.launch_id = g_tl_launch++;
+#endif
+  a.packed = packed;
+  a.unit_bytes = 4 * i2s_kp(K);
+  a.M = (int)M;
+  a.K = K;
+  a.q = q;
+  a.act_scale = act_scale;
+  a.x = x;
+  a.q_out = x ? q : nullptr;
+  a.scale_out = x ? act_scale : nullptr;
+  a.w_scale = w_scale;
+  a.T = T;
+  a.y = y;
+  a.acc_out = acc_out;
+  a.nchunks = p.nchunks;
+  a.S = p.S;
+  a.KC = p.KC;
+  a.nunits = p.nunits;
+  switch (p.depth) {
+    case 4: return launch_wring<4>(a, p, st);
+    case 6: return launch_wring<6>(a, p, st);
+    case 12: return launch_wring<12>(a, p, st);
+    case 8: return launch_wring<8>(a, p, st);
+    default: return BITNET_ERR_UNSUPPORTED_SHAPE;
+  }
+}
+
+#ifdef BITNET_PROFILE_GEMV
+extern "C" int bitnet_debug_steps_w(unsigned long long* out) {
+  return (int)cudaMemcpyFromSymbol(out, g_steps, sizeof(g_steps));
+}
+extern "C" int bitnet_debug_timeline_w(unsigned long long* out, int reset) {
+  if (reset) {
+    g_tl_launch = 0;
+    void* p = nullptr;
+    cudaGetSymbolAddress(&p, g_tl);
+    return (int)cudaMemset(p, 0, sizeof(g_tl));
+  }
+  return (int)cudaMemcpyFromSymbol(out, g_tl, sizeof(g_tl));
+}
+#endif
+
+}  // namespace bitnet
