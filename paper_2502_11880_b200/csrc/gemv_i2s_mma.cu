@@ -517,18 +517,20 @@ int launch_mma(const MmaArgs& a, const Plan& p, cudaStream_t st) {
 
 }  // namespace
 
-// The warp-private-ring kernel is the default; BITNET_I2S_STREAM=ring selects this file's kernel.
-static bool prefer_wring() {
+// The warp-private-ring kernel takes batches of up to 4 tokens (it reads the activations from shared
+// memory for every chunk, which costs more the more lanes hold a real token); this file's kernel, which
+// keeps them in registers, takes the rest.  BITNET_I2S_STREAM=ring / =warp forces one of them.
+static bool prefer_wring(int T) {
   static int v = -1;
   if (v < 0) {
     const char* e = getenv("BITNET_I2S_STREAM");
-    v = (e && strcmp(e, "ring") == 0) ? 0 : 1;
+    v = (e && strcmp(e, "ring") == 0) ? 0 : (e && strcmp(e, "warp") == 0) ? 2 : 1;
   }
-  return v == 1;
+  return v == 2 || (v == 1 && T <= 4);
 }
 
 bool gemv_i2s_stream_supported(int T, int64_t M, int64_t K, bool fused) {
-  if (prefer_wring() && gemv_i2s_wring_supported(T, M, K)) return true;
+  if (prefer_wring(T) && gemv_i2s_wring_supported(T, M, K)) return true;
   Plan p;
   return T >= 1 && T <= 8 && make_plan(T, M, K, fused, &p);
 }
@@ -536,7 +538,7 @@ bool gemv_i2s_stream_supported(int T, int64_t M, int64_t K, bool fused) {
 // x != nullptr: fused quantiser (q, act_scale are then outputs); otherwise q, act_scale are inputs.
 int launch_gemv_i2s_stream(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const float* x, int8_t* q,
                            float* act_scale, int T, float* y, int32_t* acc_out, cudaStream_t st) {
-  if (prefer_wring() && gemv_i2s_wring_supported(T, M, K))
+  if (prefer_wring(T) && gemv_i2s_wring_supported(T, M, K))
     return launch_gemv_i2s_wring(packed, w_scale, M, K, x, q, act_scale, T, y, acc_out, st);
   Plan p;
   if (T < 1 || T > 8 || !make_plan(T, M, K, x != nullptr, &p)) return BITNET_ERR_UNSUPPORTED_SHAPE;

@@ -287,15 +287,16 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
     if (tok == 2 * t) corr_even = s;
     if (tok == 2 * t + 1) corr_odd = s;
   }
-  // Token g's codes under this lane's 16-byte weight column: 64 bytes per chunk.  Columns of B beyond
-  // the batch produce columns of D nobody stores, so those lanes simply read the last token again.
-  const int8_t* const q_lane = qs_mem + min(g, a.T - 1) * kp + c_lo * 256 + t * 64;
+  // token g's codes under this lane's 16-byte weight column: 64 bytes per chunk
+  const unsigned has_tok = g < a.T ? 1u : 0u;
+  const uint32_t q_lane = smem_u32(qs_mem + min(g, a.T - 1) * kp + c_lo * 256 + t * 64);
   const int bar_id = 1 + gi, bar_threads = a.S * 32;
 
   // One step: wait for the oldest chunk of the ring, put it through the tensor cores, then refill its slot
   // from `pf` (the chunk DEPTH places further down the stream), if there is one.
   int C[4][4];
-  const uint4* qp = nullptr;
+  uint32_t qp = 0;                 // shared-memory address of the lane's 64 codes of the current chunk
+  int qr[8] = {0, 0, 0, 0, 0, 0, 0, 0};   // B registers; lanes beyond the batch keep these zeros
   auto step = [&](const uint8_t* pf, bool do_pf) {
     cp_wait<DEPTH - 1>();
     unsigned w4[4], v4[4];
@@ -309,15 +310,21 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
     // i.e. activation words 8h + 2s and 8h + 2s + 1
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      const uint4 qa = qp[2 * h], qb = qp[2 * h + 1];
-      const int qr[8] = {(int)qa.x, (int)qa.y, (int)qa.z, (int)qa.w, (int)qb.x, (int)qb.y, (int)qb.z, (int)qb.w};
+      // only the lanes whose B column is a real token load (a load by a few lanes costs the shared-memory
+      // pipe a fraction of a full-warp load); the other columns of D are never stored
+      asm volatile(
+          "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %9, 0;\n\t"
+          "@p ld.shared.v4.u32 {%0,%1,%2,%3}, [%8];\n\t"
+          "@p ld.shared.v4.u32 {%4,%5,%6,%7}, [%8+16];\n\t}"
+          : "+r"(qr[0]), "+r"(qr[1]), "+r"(qr[2]), "+r"(qr[3]), "+r"(qr[4]), "+r"(qr[5]), "+r"(qr[6]), "+r"(qr[7])
+          : "r"(qp + h * 32), "r"(has_tok));
 #pragma unroll
       for (int s = 0; s < 4; ++s) {
         const unsigned m = 0x03030303u << (2 * s);
         mma_u8s8(C[s], w4[2 * h] & m, v4[2 * h] & m, w4[2 * h + 1] & m, v4[2 * h + 1] & m, qr[2 * s], qr[2 * s + 1]);
       }
     }
-    qp += 16;
+    qp += 256;
     // the chunk's bytes were in registers before the MMAs above were issued: its slot can be refilled
     if (do_pf) {
       cp16(ring + slot_off, pf, pol);
@@ -340,7 +347,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
     for (int s = 0; s < 4; ++s)
 #pragma unroll
       for (int i = 0; i < 4; ++i) C[s][i] = 0;
-    qp = reinterpret_cast<const uint4*>(q_lane);
+    qp = q_lane;
     TL_STEP(0);
 
     // chunks 0 .. nw-DEPTH-1 are followed, DEPTH places on, by chunks of the same unit
