@@ -57,12 +57,14 @@ __device__ __forceinline__ unsigned long long gtime() {
 }
 static __device__ unsigned long long g_steps[256][4][24];
 #define TL_STEP(i) do { if ((blockIdx.x % 37) == 0 && blockIdx.x < 148 && threadIdx.x == 0 && n == 0 && (i) < 24) g_steps[a.launch_id & 255][blockIdx.x / 37][i] = gtime(); } while (0)
+#define TL_PRO(i) do { if ((blockIdx.x % 37) == 0 && blockIdx.x < 148 && threadIdx.x == 0) g_steps[a.launch_id & 255][blockIdx.x / 37][i] = gtime(); } while (0)
 #define TL_MARK(i) do { if (blockIdx.x < 148) g_tl[a.launch_id & 255][blockIdx.x][i] = gtime(); } while (0)
 #define TL_MAX(i) do { if (blockIdx.x < 148) atomicMax(&g_tl[a.launch_id & 255][blockIdx.x][i], gtime()); } while (0)
 #else
 #define TL_MARK(i) do { } while (0)
 #define TL_MAX(i) do { } while (0)
 #define TL_STEP(i) do { } while (0)
+#define TL_PRO(i) do { } while (0)
 #endif
 
 struct WArgs {
@@ -84,6 +86,7 @@ struct WArgs {
   int S;                 // warps per unit
   int KC;                // chunks per warp and unit (the last warp of a unit may have fewer, or none)
   int nunits;            // ceil(M / 16)
+  int pre;               // ring slots requested before waiting for the previous kernel
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -164,23 +167,29 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
   const volatile int* my_jq = jq + gi * JQ;
   const int nw = c_hi - c_lo;
   uint32_t slot_off = 0;
-  // Weights do not depend on the previous kernel in the stream: request the first DEPTH chunks now.
-  {
-    const int j0 = my_jq[0];
-    const uint8_t* src = base + (int64_t)j0 * unit_stride;
+  // Weights do not depend on the previous kernel in the stream: request the first chunks now.  Only a.pre
+  // of the DEPTH chunks: the activation loads that follow the wait below queue behind whatever is in flight,
+  // and everything after them waits for the activations.  The rest of the ring is requested right after them.
+  const int j0 = my_jq[0];
+  const uint8_t* const src0 = base + (int64_t)j0 * unit_stride;
+  auto first_fill = [&](bool before_wait) {
 #pragma unroll
     for (int d = 0; d < DEPTH; ++d) {
-      if (j0 < n_units) {
-        cp16(ring + d * 1024, src + d * 1024, pol);
-        cp16(ring + d * 1024 + 512, src + d * 1024 + 512, pol);
+      if ((d < a.pre) == before_wait) {
+        if (j0 < n_units) {
+          cp16(ring + d * 1024, src0 + d * 1024, pol);
+          cp16(ring + d * 1024 + 512, src0 + d * 1024 + 512, pol);
+        }
+        cp_commit();
       }
-      cp_commit();
     }
-  }
+  };
+  first_fill(true);
 
   // ---------------- activations come from the previous kernel in the stream
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (threadIdx.x == 0) TL_MARK(1);
+  TL_PRO(17);
 
   if (a.x && a.T == 1 && a.K <= 4 * XREG * THREADS) {
     // ---- fused quantiser (Alg. 1 Phase 1), one token, one round trip: the row stays in registers
@@ -194,14 +203,18 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
       const int i = threadIdx.x + r * THREADS;
       xv[r] = (i < n4) ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
+    first_fill(false);
+    TL_PRO(18);
     float m = 0.0f;
 #pragma unroll
     for (int r = 0; r < XREG; ++r)
       m = fmaxf(m, fmaxf(fmaxf(fabsf(xv[r].x), fabsf(xv[r].y)), fmaxf(fabsf(xv[r].z), fabsf(xv[r].w))));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    TL_PRO(19);
     if (lane == 0) qred[warp] = m;
     __syncthreads();
+    TL_PRO(20);
     float amax = 0.0f;
 #pragma unroll
     for (int w2 = 0; w2 < CW; ++w2) amax = fmaxf(amax, qred[w2]);
@@ -223,6 +236,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
     }
   } else if (a.x) {
     // ---- fused quantiser, general form: amax per token, then a second pass over x
+    first_fill(false);
     for (int tok = 0; tok < a.T; ++tok) {
       const float4* x4 = reinterpret_cast<const float4*>(a.x + (int64_t)tok * a.K);
       float m = 0.0f;
@@ -258,17 +272,33 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
       }
     }
   } else {
-    // ---- stage the given codes (zero beyond K)
-    for (int tok = 0; tok < a.T; ++tok) {
-      const int* q4 = reinterpret_cast<const int*>(a.q + (int64_t)tok * a.K);
-      for (int i = threadIdx.x; i < kp / 4; i += THREADS)
-        reinterpret_cast<int*>(qs_mem + tok * kp)[i] = (i < (int)(a.K / 4)) ? __ldcg(q4 + i) : 0;
+    // ---- stage the given codes (zero beyond K); the first QREG words per thread are loaded before the
+    // rest of the ring is requested
+    constexpr int QREG = 8;
+    const int nq4 = (int)(a.K / 4), total4 = a.T * (kp / 4);     // words per token, words to stage
+    int qv[QREG];
+#pragma unroll
+    for (int r = 0; r < QREG; ++r) {
+      const int i = threadIdx.x + r * THREADS, tok = i / (kp / 4), col = i - tok * (kp / 4);
+      qv[r] = (i < total4 && col < nq4) ? __ldcg(reinterpret_cast<const int*>(a.q + (int64_t)tok * a.K) + col) : 0;
     }
-    if (threadIdx.x < a.T) qscale[threadIdx.x] = __ldcg(a.act_scale + threadIdx.x);
+    const float my_scale = (threadIdx.x < a.T) ? __ldcg(a.act_scale + threadIdx.x) : 0.0f;
+    first_fill(false);
+#pragma unroll
+    for (int r = 0; r < QREG; ++r) {
+      const int i = threadIdx.x + r * THREADS;
+      if (i < total4) reinterpret_cast<int*>(qs_mem)[i] = qv[r];
+    }
+    for (int i = threadIdx.x + QREG * THREADS; i < total4; i += THREADS) {
+      const int tok = i / (kp / 4), col = i - tok * (kp / 4);
+      reinterpret_cast<int*>(qs_mem)[i] = (col < nq4) ? __ldcg(reinterpret_cast<const int*>(a.q + (int64_t)tok * a.K) + col) : 0;
+    }
+    if (threadIdx.x < a.T) qscale[threadIdx.x] = my_scale;
   }
   __syncthreads();
 
   if (threadIdx.x == 0) TL_MARK(2);
+  TL_PRO(21);
   // sum of the activations of tokens 2t and 2t+1 over this warp's K-slice (the "- sum(q)" term)
   int corr_even = 0, corr_odd = 0;
   for (int tok = 0; tok < a.T; ++tok) {
@@ -287,6 +317,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
     if (tok == 2 * t) corr_even = s;
     if (tok == 2 * t + 1) corr_odd = s;
   }
+  TL_PRO(22);
   // token g's codes under this lane's 16-byte weight column: 64 bytes per chunk
   const unsigned has_tok = g < a.T ? 1u : 0u;
   const uint32_t q_lane = smem_u32(qs_mem + min(g, a.T - 1) * kp + c_lo * 256 + t * 64);
@@ -420,7 +451,7 @@ bool make_plan(int T, int64_t M, int64_t K, Plan* p) {
   if (depth == 10) depth = 8;
   if (p->nchunks < depth) return false;     // a warp's slice is at least as long as the ring
   // warps per unit: as many as leave every warp about kc_target chunks of a unit (never fewer than the ring)
-  int kc_target = env_int("BITNET_I2S_KC", 16);
+  int kc_target = env_int("BITNET_I2S_KC", 8);
   if (kc_target < depth) kc_target = depth;
   int S = 1;
   while (S < CW && p->nchunks / (2 * S) >= kc_target) S *= 2;
@@ -495,6 +526,7 @@ int launch_gemv_i2s_wring(const uint8_t* packed, float w_scale, int64_t M, int64
   a.S = p.S;
   a.KC = p.KC;
   a.nunits = p.nunits;
+  a.pre = env_int("BITNET_I2S_PRE", 4);
   switch (p.depth) {
     case 4: return launch_wring<4>(a, p, st);
     case 6: return launch_wring<6>(a, p, st);
