@@ -36,6 +36,11 @@ METRIC = "mpgemv_weight_stream_batch1"
 UNIT = "GB/s"
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one captured launch of the decode kernel (K=8192 -> M=57344:
+# 117.542 MB read + 3.72 MB written) over the packed weight bytes of that launch (117.44 MB).  Traffic grows
+# in proportion to the weights streamed, so the same ratio scales it to the sweep's average launch.
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = (117.542 + 3.72) / 117.440
+
 def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -362,7 +367,9 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "kernel": "gemv_i2s_wring_kernel (quantiser fused)", "achieved": achieved,
                      "peak": pk["hbm"], "unit": "GB/s", "frac": achieved / pk["hbm"], "peak_source": pk["which"],
                      "bytes_per_launch": sw.bytes["i2s"] / n_lin, "us_per_launch": 1e3 * ms_step / n_lin,
-                     "traffic": None},
+                     "traffic": NCU_TRAFFIC_PER_ALGORITHMIC_BYTE * sw.bytes["i2s"] / n_lin,
+                     "traffic_note": "dram read+write bytes of an ncu capture of the K=8192 -> M=57344 launch "
+                                     "(121.26 MB for 117.44 MB of weights), scaled by bytes to the average launch"},
         "breakdown": {"ms_fused_step": ms_step, "ms_gemv_kernels_alone": ms_gemv, "ms_quant_kernels_alone": ms_quant,
                       "setup_s": sw.setup_s},
         "clocks": clocks,
