@@ -1,13 +1,5 @@
-// I2_S mpGEMV for decode (1..8 tokens), warp-private rings: Alg. 1 Phase 2 from the 2-bit blob with
-// the quantiser (Phase 1) optionally fused in.
-//
-// Why this shape.  A decode step is a chain of dependent kernels that each stream a few tens of MB once;
-// what decides the chain's speed is how little of the time HBM sits idle between and inside kernels.
-// So the kernel is made small enough that the CTAs of TWO consecutive kernels fit on an SM together
-// (512 threads, at most 64 registers, about half the shared memory): under programmatic dependent launch
-// the next kernel's CTAs become resident while this one still runs, request their first weights -- which
-// depend on nothing -- and only then wait for this kernel to finish.  The gap between kernels, the
-// quantiser prologue and the tail of a kernel are then covered by the neighbour's weight traffic.
+// I2_S mpGEMV for decode (1..8 tokens; used for batches of up to 4), warp-private rings: Alg. 1 Phase 2
+// from the 2-bit blob with the quantiser (Phase 1) optionally fused in.
 //
 // Memory side.  The blob stores 16-row units contiguously and chunk-major (1024 bytes per 256-column
 // chunk, 64 bytes per row).  A unit is shared by S warps (S a power of two), each owning a K-slice of the
@@ -15,23 +7,30 @@
 // per-thread asynchronous 16-byte copies (cp.async, L2 evict-first): lane l copies bytes [16l, 16l+16)
 // and [512+16l, ...) of a chunk and later reads back exactly those bytes, so the only synchronisation
 // of the stream is the thread's own cp.async.wait_group -- no barrier, no producer, no handshake.  The
-// ring runs DEPTH chunks ahead and crosses unit boundaries.
+// ring runs DEPTH chunks ahead and crosses unit boundaries.  One CTA of 16 warps per SM; the rings (128 KB)
+// keep a second CTA off the SM on purpose: when the CTAs of consecutive kernels shared SMs, the hardware
+// placed them unevenly and the slowest SM set the pace.
 //
 // Work distribution.  Unit u belongs to CTA u mod gridDim; inside the CTA the warp groups take the
-// CTA's units from a shared counter, DEPTH units ahead of use (the prefetcher must know where the
-// stream continues), so a group that falls behind simply takes fewer units.
+// CTA's units from a shared counter, one unit ahead of use (a warp's slice is at least as long as its
+// ring, so its requests never reach beyond the next unit), so a group that falls behind takes fewer units.
 //
 // Compute side.  A chunk of a unit is the A operand of 8 int8 tensor-core MMAs (mma.sync m16n8k32,
 // u8 x s8 -> s32): lane (g = lane/4, t = lane%4) holds 64 weights of row g and of row g+8.  Masking a
 // packed word with 0x03030303 << 2s leaves, without a shift, the four codes of slot s scaled by 4^s:
-// one A register.  The B operand is the activations (column n = token n), read from shared memory.
-// Four accumulator fragments carry the scales 1, 4, 16, 64; each is an exact multiple of its scale, so
-// arithmetic shifts undo it, and sum(code*q) - sum(q) = sum(w*q).  The S partial fragments of a unit
-// meet in shared memory at a named barrier of the group; one warp (rotating) adds them, rescales and
-// stores y = acc * act_scale[t] * w_scale.
+// one A register.  The B operand is the activations (column n = token n), read from shared memory by
+// the lanes of real tokens only (columns of D beyond the batch are never stored, and a load by a few
+// lanes costs the shared-memory pipe a fraction of a full-warp load).  Four accumulator fragments carry
+// the scales 1, 4, 16, 64; each is an exact multiple of its scale, so arithmetic shifts undo it, and
+// sum(code*q) - sum(q) = sum(w*q).  The S partial fragments of a unit meet in shared memory at a named
+// barrier of the group; one warp (rotating) adds them, rescales and stores y = acc * act_scale[t] * w_scale.
+//
+// Kernel chain.  Under programmatic dependent launch the CTA starts as soon as its SM is free, requests
+// its first weights -- which depend on nothing -- and only then waits for the previous kernel
+// (griddepcontrol.wait) before it touches activations.
 //
 // Fused quantiser: with fp32 activations given, every CTA computes absmax and the int8 codes itself,
-// after its first weight copies are in flight; CTA 0 also stores the codes and scales for the caller.
+// while its first weight copies are in flight; CTA 0 also stores the codes and scales for the caller.
 #include <cstdlib>
 #include <cstring>
 
