@@ -259,6 +259,21 @@ class Sweep:
         return replay
 
 
+def max_over_ranks(torch, dist, ms, device):
+    """The job's time for a region is the slowest rank's device time (every rank gets the same number back)."""
+    if dist is None:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.barrier()
+    return float(t.item())
+
+
+def whole_job_value(bytes_per_replica, world, ms_step):
+    """Replicas only: every rank streams its own copy of the sweep, so the job moves world x the bytes."""
+    return bytes_per_replica * world / ms_step / 1e6
+
+
 def time_replays(torch, fn, steps, warmup, dist=None):
     for _ in range(warmup):
         fn()
@@ -272,12 +287,7 @@ def time_replays(torch, fn, steps, warmup, dist=None):
         fn()
     e1.record()
     torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-        dist.barrier()
+    ms = max_over_ranks(torch, dist, e0.elapsed_time(e1), "cuda")
     return ms / steps
 
 
@@ -335,8 +345,7 @@ def run_ours(args):
     sampler = ClockSampler(local) if rank == 0 else None
     ms_step = time_replays(torch, g_full, args.steps, args.warmup, dist)
     clocks = sampler.stop() if sampler else None
-    total_bytes = sw.bytes["i2s"] * world
-    value = total_bytes / ms_step / 1e6
+    value = whole_job_value(sw.bytes["i2s"], world, ms_step)
 
     # ---- dominant kernel alone (GEMV launches only): roofline
     g_gemv = sw.make_graph("i2s", "gemv")
@@ -349,7 +358,7 @@ def run_ours(args):
     # ---- end to end through the host-buffer entry point
     ms_e2e = time_replays(torch, lambda: (sw.step_host("i2s"), torch.cuda.current_stream().synchronize()),
                           max(2, args.steps // 4), 3, dist)
-    e2e_val = total_bytes / ms_e2e / 1e6
+    e2e_val = whole_job_value(sw.bytes["i2s"], world, ms_e2e)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
