@@ -113,6 +113,16 @@ __device__ __forceinline__ void mma_u8s8(int (&c)[4], unsigned a0, unsigned a1, 
 __device__ __forceinline__ int quant1(float x, float s) {
   return max(-128, min(127, __float2int_rn(__fmul_rn(x, s))));
 }
+// Four codes in one word: round to nearest even, then the saturating pack does the clamp to [-128, 127]
+// (which never fires for |x| <= amax; same result as quant1 on every input).
+__device__ __forceinline__ int quant4_packed(const float4& v, float s) {
+  const int a0 = __float2int_rn(__fmul_rn(v.x, s)), a1 = __float2int_rn(__fmul_rn(v.y, s));
+  const int a2 = __float2int_rn(__fmul_rn(v.z, s)), a3 = __float2int_rn(__fmul_rn(v.w, s));
+  int hi, w;
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(a3), "r"(a2), "r"(0));
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(a1), "r"(a0), "r"(hi));
+  return w;
+}
 __device__ __forceinline__ int quant4(const float4& v, float s) {
   return (quant1(v.x, s) & 255) | ((quant1(v.y, s) & 255) << 8) | ((quant1(v.z, s) & 255) << 16) |
          ((quant1(v.w, s) & 255) << 24);
@@ -196,18 +206,19 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
     // kernel: s = 127 / max(amax, 1e-5), q = clamp(rint(x * s)).
     const float4* x4 = reinterpret_cast<const float4*>(a.x);
     const int n4 = (int)(a.K / 4);
+    const int nrow = (max(n4, kp / 4) + THREADS - 1) / THREADS;     // rows of THREADS words that hold anything
     float4 xv[XREG];
 #pragma unroll
     for (int r = 0; r < XREG; ++r) {
       const int i = threadIdx.x + r * THREADS;
-      xv[r] = (i < n4) ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+      xv[r] = (r < nrow && i < n4) ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     first_fill(false);
     TL_PRO(18);
     float m = 0.0f;
 #pragma unroll
     for (int r = 0; r < XREG; ++r)
-      m = fmaxf(m, fmaxf(fmaxf(fabsf(xv[r].x), fabsf(xv[r].y)), fmaxf(fabsf(xv[r].z), fabsf(xv[r].w))));
+      if (r < nrow) m = fmaxf(m, fmaxf(fmaxf(fabsf(xv[r].x), fabsf(xv[r].y)), fmaxf(fabsf(xv[r].z), fabsf(xv[r].w))));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     TL_PRO(19);
@@ -227,8 +238,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
 #pragma unroll
     for (int r = 0; r < XREG; ++r) {
       const int i = threadIdx.x + r * THREADS;
-      if (i < kp / 4) {
-        const int word = quant4(xv[r], sq);                 // columns K..Kp-1 came in as zeros
+      if (r < nrow && i < kp / 4) {
+        const int word = quant4_packed(xv[r], sq);          // columns K..Kp-1 came in as zeros
         reinterpret_cast<int*>(qs_mem)[i] = word;
         if (blockIdx.x == 0 && a.q_out && i < n4) reinterpret_cast<int*>(a.q_out)[i] = word;
       }
