@@ -42,7 +42,7 @@ namespace {
 constexpr int CW = 16;                   // warps
 constexpr int THREADS = CW * 32;
 constexpr int JQ = 4;                    // entries of a group's queue of upcoming units
-constexpr int XREG = 16;                 // float4 registers per thread of the fused quantiser's fast path
+constexpr int XREG_MAX = 16;                 // float4 registers per thread of the fused quantiser's fast path
 constexpr size_t MAX_QS_BYTES = 64 * 1024;   // activations staged in shared memory up to this size
 
 #ifdef BITNET_PROFILE_GEMV
@@ -131,7 +131,8 @@ __device__ __forceinline__ int quant4(const float4& v, float s) {
 // shared memory: [unit counter, unit queues, quantiser scratch: 2 KB][partials][codes][rings]
 __host__ __device__ inline size_t red_bytes(int T) { return (size_t)CW * 2 * T * 16 * 4; }
 
-template <int DEPTH>
+// XREG: float4 registers per thread of the fused quantiser's fast path (rows of THREADS float4 of x)
+template <int DEPTH, int XREG>
 __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   int* counter = reinterpret_cast<int*>(smem);                 // next unit (index into the CTA's list) to hand out
@@ -477,13 +478,13 @@ bool make_plan(int T, int64_t M, int64_t K, Plan* p) {
   return p->smem <= (size_t)dev_info().max_smem_optin;
 }
 
-template <int DEPTH>
+template <int DEPTH, int XREG>
 int launch_wring(const WArgs& a, const Plan& p, cudaStream_t st) {
   static bool attr_set[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
   if (!attr_set[dev & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(gemv_i2s_wring_kernel<DEPTH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(gemv_i2s_wring_kernel<DEPTH, XREG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          dev_info().max_smem_optin);
     if (e != cudaSuccess) return note_cuda_error(e);
     attr_set[dev & 63] = true;
@@ -498,7 +499,7 @@ int launch_wring(const WArgs& a, const Plan& p, cudaStream_t st) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = early_start_enabled() ? 1 : 0;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_i2s_wring_kernel<DEPTH>, a);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_i2s_wring_kernel<DEPTH, XREG>, a);
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
 }
 
@@ -537,11 +538,13 @@ int launch_gemv_i2s_wring(const uint8_t* packed, float w_scale, int64_t M, int64
   a.KC = p.KC;
   a.nunits = p.nunits;
   a.pre = env_int("BITNET_I2S_PRE", 4);
+  // short rows get the instance whose (fully unrolled) quantiser prologue is a quarter of the code
+  const bool small_x = x != nullptr && T == 1 && K <= 4 * 4 * THREADS;
   switch (p.depth) {
-    case 4: return launch_wring<4>(a, p, st);
-    case 6: return launch_wring<6>(a, p, st);
-    case 12: return launch_wring<12>(a, p, st);
-    case 8: return launch_wring<8>(a, p, st);
+    case 4: return launch_wring<4, XREG_MAX>(a, p, st);
+    case 6: return launch_wring<6, XREG_MAX>(a, p, st);
+    case 12: return launch_wring<12, XREG_MAX>(a, p, st);
+    case 8: return small_x ? launch_wring<8, 4>(a, p, st) : launch_wring<8, XREG_MAX>(a, p, st);
     default: return BITNET_ERR_UNSUPPORTED_SHAPE;
   }
 }
