@@ -220,7 +220,8 @@ int bitnet_linear(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
     }();
     // One token: every CTA of the GEMV quantises the row itself.  More tokens: that redundant work (each
     // CTA reading T rows twice) costs more than a separate quantiser launch.
-    if (!no_fuse && T == 1 && gemv_i2s_stream_supported((int)T, M, K, true))
+    static const int fuse_max = [] { const char* e = getenv("BITNET_FUSE_MAX_T"); return e ? atoi(e) : 2; }();
+    if (!no_fuse && T <= fuse_max && gemv_i2s_stream_supported((int)T, M, K, true))
       return launch_gemv_i2s_stream((const uint8_t*)packed, w_scale, M, K, x, q, act_scale, (int)T, y, acc_out,
                                     (cudaStream_t)stream);
   }

@@ -43,7 +43,7 @@ constexpr int CW = 16;                   // warps
 constexpr int THREADS = CW * 32;
 constexpr int JQ = 4;                    // entries of a group's queue of upcoming units
 constexpr int XREG_MAX = 16;                 // float4 registers per thread of the fused quantiser's fast path
-constexpr size_t MAX_QS_BYTES = 64 * 1024;   // activations staged in shared memory up to this size
+constexpr size_t MAX_QS_BYTES = 68 * 1024;   // activations staged in shared memory up to this size
 
 #ifdef BITNET_PROFILE_GEMV
 // Development aid (never in the shipped build): per launch and CTA, %globaltimer at a few points.
@@ -142,7 +142,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
   int* red = reinterpret_cast<int*>(smem + 2048);              // [CW][2][T][16] partial sums
   const int kp = a.nchunks * 256;
   int8_t* qs_mem = reinterpret_cast<int8_t*>(smem + 2048 + red_bytes(a.T));
-  uint8_t* rings = reinterpret_cast<uint8_t*>(qs_mem) + (((size_t)a.T * kp + 127) & ~(size_t)127);
+  // Token rows are kp + 16 bytes apart: the B loads of one MMA pair read 16 bytes of every token at the same
+  // column, and rows a multiple of 128 bytes apart would all hit the same shared-memory banks.
+  const int qst = kp + 16;
+  uint8_t* rings = reinterpret_cast<uint8_t*>(qs_mem) + (((size_t)a.T * qst + 127) & ~(size_t)127);
 
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
@@ -201,48 +204,51 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
   if (threadIdx.x == 0) TL_MARK(1);
   TL_PRO(17);
 
-  if (a.x && a.T == 1 && a.K <= 4 * XREG * THREADS) {
-    // ---- fused quantiser (Alg. 1 Phase 1), one token, one round trip: the row stays in registers
+  if (a.x && a.K <= 4 * XREG * THREADS) {
+    // ---- fused quantiser (Alg. 1 Phase 1), one round trip per token: the row stays in registers
     // between the amax pass and the rounding pass.  Same operations and order as the stand-alone
     // kernel: s = 127 / max(amax, 1e-5), q = clamp(rint(x * s)).
-    const float4* x4 = reinterpret_cast<const float4*>(a.x);
     const int n4 = (int)(a.K / 4);
     const int nrow = (max(n4, kp / 4) + THREADS - 1) / THREADS;     // rows of THREADS words that hold anything
-    float4 xv[XREG];
+    for (int tok = 0; tok < a.T; ++tok) {
+      const float4* x4 = reinterpret_cast<const float4*>(a.x + (int64_t)tok * a.K);
+      float4 xv[XREG];
 #pragma unroll
-    for (int r = 0; r < XREG; ++r) {
-      const int i = threadIdx.x + r * THREADS;
-      xv[r] = (r < nrow && i < n4) ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    first_fill(false);
-    TL_PRO(18);
-    float m = 0.0f;
+      for (int r = 0; r < XREG; ++r) {
+        const int i = threadIdx.x + r * THREADS;
+        xv[r] = (r < nrow && i < n4) ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+      if (tok == 0) first_fill(false);
+      TL_PRO(18);
+      float m = 0.0f;
 #pragma unroll
-    for (int r = 0; r < XREG; ++r)
-      if (r < nrow) m = fmaxf(m, fmaxf(fmaxf(fabsf(xv[r].x), fabsf(xv[r].y)), fmaxf(fabsf(xv[r].z), fabsf(xv[r].w))));
+      for (int r = 0; r < XREG; ++r)
+        if (r < nrow) m = fmaxf(m, fmaxf(fmaxf(fabsf(xv[r].x), fabsf(xv[r].y)), fmaxf(fabsf(xv[r].z), fabsf(xv[r].w))));
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    TL_PRO(19);
-    if (lane == 0) qred[warp] = m;
-    __syncthreads();
-    TL_PRO(20);
-    float amax = 0.0f;
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      TL_PRO(19);
+      if (tok > 0) __syncthreads();          // everyone has read the previous token's partial maxima
+      if (lane == 0) qred[warp] = m;
+      __syncthreads();
+      TL_PRO(20);
+      float amax = 0.0f;
 #pragma unroll
-    for (int w2 = 0; w2 < CW; ++w2) amax = fmaxf(amax, qred[w2]);
-    const float amax_c = fmaxf(amax, 1e-5f);
-    const float sq = __fdiv_rn(127.0f, amax_c);
-    if (threadIdx.x == 0) {
-      const float inv = __fdiv_rn(amax_c, 127.0f);
-      qscale[0] = inv;
-      if (blockIdx.x == 0 && a.scale_out) a.scale_out[0] = inv;
-    }
+      for (int w2 = 0; w2 < CW; ++w2) amax = fmaxf(amax, qred[w2]);
+      const float amax_c = fmaxf(amax, 1e-5f);
+      const float sq = __fdiv_rn(127.0f, amax_c);
+      if (threadIdx.x == 0) {
+        const float inv = __fdiv_rn(amax_c, 127.0f);
+        qscale[tok] = inv;
+        if (blockIdx.x == 0 && a.scale_out) a.scale_out[tok] = inv;
+      }
 #pragma unroll
-    for (int r = 0; r < XREG; ++r) {
-      const int i = threadIdx.x + r * THREADS;
-      if (r < nrow && i < kp / 4) {
-        const int word = quant4_packed(xv[r], sq);          // columns K..Kp-1 came in as zeros
-        reinterpret_cast<int*>(qs_mem)[i] = word;
-        if (blockIdx.x == 0 && a.q_out && i < n4) reinterpret_cast<int*>(a.q_out)[i] = word;
+      for (int r = 0; r < XREG; ++r) {
+        const int i = threadIdx.x + r * THREADS;
+        if (r < nrow && i < kp / 4) {
+          const int word = quant4_packed(xv[r], sq);          // columns K..Kp-1 came in as zeros
+          reinterpret_cast<int*>(qs_mem + tok * qst)[i] = word;
+          if (blockIdx.x == 0 && a.q_out && i < n4) reinterpret_cast<int*>(a.q_out + (int64_t)tok * a.K)[i] = word;
+        }
       }
     }
   } else if (a.x) {
@@ -279,7 +285,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
           word = quant4(__ldcg(x4 + i), sq);
           if (blockIdx.x == 0 && a.q_out) reinterpret_cast<int*>(a.q_out + (int64_t)tok * a.K)[i] = word;
         }
-        reinterpret_cast<int*>(qs_mem + tok * kp)[i] = word;
+        reinterpret_cast<int*>(qs_mem + tok * qst)[i] = word;
       }
     }
   } else {
@@ -298,11 +304,11 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
 #pragma unroll
     for (int r = 0; r < QREG; ++r) {
       const int i = threadIdx.x + r * THREADS;
-      if (i < total4) reinterpret_cast<int*>(qs_mem)[i] = qv[r];
+      if (i < total4) reinterpret_cast<int*>(qs_mem + (i / (kp / 4)) * qst)[i % (kp / 4)] = qv[r];
     }
     for (int i = threadIdx.x + QREG * THREADS; i < total4; i += THREADS) {
       const int tok = i / (kp / 4), col = i - tok * (kp / 4);
-      reinterpret_cast<int*>(qs_mem)[i] = (col < nq4) ? __ldcg(reinterpret_cast<const int*>(a.q + (int64_t)tok * a.K) + col) : 0;
+      reinterpret_cast<int*>(qs_mem + tok * qst)[col] = (col < nq4) ? __ldcg(reinterpret_cast<const int*>(a.q + (int64_t)tok * a.K) + col) : 0;
     }
     if (threadIdx.x < a.T) qscale[threadIdx.x] = my_scale;
   }
@@ -314,7 +320,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
   int corr_even = 0, corr_odd = 0;
   for (int tok = 0; tok < a.T; ++tok) {
     int s = 0, s2 = 0;
-    const uint4* qw = reinterpret_cast<const uint4*>(qs_mem + tok * kp + c_lo * 256);
+    const uint4* qw = reinterpret_cast<const uint4*>(qs_mem + tok * qst + c_lo * 256);
+#pragma unroll 4
     for (int i = lane; i < (c_hi - c_lo) * 16; i += 32) {
       const uint4 v = qw[i];
       s = __dp4a((int)v.x, 0x01010101, s);
@@ -331,7 +338,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
   TL_PRO(22);
   // token g's codes under this lane's 16-byte weight column: 64 bytes per chunk
   const unsigned has_tok = g < a.T ? 1u : 0u;
-  const uint32_t q_lane = smem_u32(qs_mem + min(g, a.T - 1) * kp + c_lo * 256 + t * 64);
+  const uint32_t q_lane = smem_u32(qs_mem + min(g, a.T - 1) * qst + c_lo * 256 + t * 64);
   const int bar_id = 1 + gi, bar_threads = a.S * 32;
 
   // One step: wait for the oldest chunk of the ring, put it through the tensor cores, then refill its slot
@@ -456,7 +463,7 @@ bool make_plan(int T, int64_t M, int64_t K, Plan* p) {
   p->nchunks = (int)(i2s_kp(K) / 256);
   const int forced = env_int("BITNET_I2S_DEPTH", 0);
   int depth = (forced == 12 || forced == 8 || forced == 6 || forced == 4) ? forced : 8;
-  while (depth > 4 && 2048 + red_bytes(T) + (((size_t)T * p->nchunks * 256 + 127) & ~(size_t)127) +
+  while (depth > 4 && 2048 + red_bytes(T) + (((size_t)T * (p->nchunks * 256 + 16) + 127) & ~(size_t)127) +
                               (size_t)CW * depth * 1024 > (size_t)dev_info().max_smem_optin)
     depth -= 2;
   if (depth == 10) depth = 8;
@@ -471,7 +478,7 @@ bool make_plan(int T, int64_t M, int64_t K, Plan* p) {
   p->nunits = (int)ceil_div(M, 16);
   const int ctas = dev_info().sm_count * env_int("BITNET_I2S_CTAS", 1);
   p->grid = ctas < p->nunits ? ctas : p->nunits;
-  const size_t qs_bytes = ((size_t)T * p->nchunks * 256 + 127) & ~(size_t)127;
+  const size_t qs_bytes = ((size_t)T * (p->nchunks * 256 + 16) + 127) & ~(size_t)127;
   if (qs_bytes > MAX_QS_BYTES) return false;
   p->depth = depth;
   p->smem = 2048 + red_bytes(T) + qs_bytes + (size_t)CW * depth * 1024;
