@@ -517,7 +517,7 @@ int launch_mma(const MmaArgs& a, const Plan& p, cudaStream_t st) {
 
 }  // namespace
 
-// The warp-private-ring kernel takes batches of up to 4 tokens (it reads the activations from shared
+// The warp-private-ring kernel takes batches of up to 6 tokens (it reads the activations from shared
 // memory for every chunk, which costs more the more lanes hold a real token); this file's kernel, which
 // keeps them in registers, takes the rest.  BITNET_I2S_STREAM=ring / =warp forces one of them.
 static bool prefer_wring(int T) {
@@ -526,7 +526,7 @@ static bool prefer_wring(int T) {
     const char* e = getenv("BITNET_I2S_STREAM");
     v = (e && strcmp(e, "ring") == 0) ? 0 : (e && strcmp(e, "warp") == 0) ? 2 : 1;
   }
-  return v == 2 || (v == 1 && T <= 4);
+  return v == 2 || (v == 1 && T <= 6);
 }
 
 bool gemv_i2s_stream_supported(int T, int64_t M, int64_t K, bool fused) {
