@@ -161,6 +161,37 @@ int bitnet_linear_host(bitnet_fmt_t fmt, const void* packed, float w_scale, int6
                        size_t workspace_bytes, void* stream);
 
 /*
+ * A batch of linear layers with HOST activations and HOST results (Alg. 1 end to end per item), with the
+ * copies overlapped with the kernels: item i's x_host is uploaded on an internal stream, its kernel
+ * runs on `stream` once that upload is complete, and its y_host is downloaded on a second internal
+ * stream once the kernel is complete.  Kernels run in item order on `stream`; when the call returns
+ * everything is queued, and `stream` has been made to wait for the last download, so work queued on
+ * `stream` afterwards (or a synchronisation of `stream`) follows every copy of the batch.
+ *   - items[n]: plain structs in host memory, read during the call only.
+ *   - x_host / y_host should be pinned.  The device buffers of different items must not overlap
+ *     (uploads run ahead of the kernels); the workspace may be shared (the kernels are serial).
+ *   - The internal streams and events are created on first use per device and kept.
+ *   - Errors: BITNET_ERR_INVALID_ARG for a null or malformed item (nothing of that item or later ones
+ *     is queued); otherwise the status of the first failing call.
+ */
+typedef struct bitnet_host_linear {
+  int32_t fmt;            /* bitnet_fmt_t */
+  int32_t bk3;
+  const void* packed;
+  float w_scale;
+  int64_t M, K, T;
+  const float* x_host;    /* [T][K] */
+  float* y_host;          /* [T][M] */
+  float* x_dev;           /* scratch [T*K] fp32 */
+  int8_t* q_dev;          /* scratch [T*K] int8 */
+  float* scale_dev;       /* scratch [T] fp32 */
+  float* y_dev;           /* scratch [T*M] fp32 */
+  void* workspace;
+  size_t workspace_bytes;
+} bitnet_host_linear_t;
+int bitnet_linear_host_batch(const bitnet_host_linear_t* items, int64_t n, void* stream);
+
+/*
  * Table-lookup mpGEMV without a workspace argument (the paper has no counterpart: this entry point
  * exists for the sake of callers, not of the method).
  *

@@ -23,7 +23,7 @@ FMT = {"i2s": FMT_I2S, "tl1": FMT_TL1, "tl2": FMT_TL2}
 SYMBOLS = [
     "bitnet_status_string", "bitnet_last_cuda_error", "bitnet_quant_act", "bitnet_i2s_packed_bytes",
     "bitnet_pack_i2s", "bitnet_tl_packed_bytes", "bitnet_pack_tl", "bitnet_mpgemm_workspace_bytes",
-    "bitnet_workspace_init", "bitnet_mpgemm", "bitnet_linear", "bitnet_linear_host", "bitnet_unpack_i2s", "bitnet_unpack_tl",
+    "bitnet_workspace_init", "bitnet_mpgemm", "bitnet_linear", "bitnet_linear_host", "bitnet_linear_host_batch", "bitnet_unpack_i2s", "bitnet_unpack_tl",
     "bitnet_tl_num_groups", "bitnet_tl_build_lut_debug", "bitnet_mpgemv_tl_noalloc", "bitnet_device_status",
     "bitnet_set_early_start",
 ]
@@ -63,6 +63,7 @@ def lib():
         L.bitnet_mpgemm.argtypes = [ci, vp, fl, i64, i64, ci, vp, vp, i64, vp, vp, vp, sz, vp]
         L.bitnet_linear.argtypes = [ci, vp, fl, i64, i64, ci, vp, i64, vp, vp, vp, vp, vp, sz, vp]
         L.bitnet_linear_host.argtypes = [ci, vp, fl, i64, i64, ci, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.bitnet_linear_host_batch.argtypes = [vp, i64, vp]
         L.bitnet_unpack_i2s.argtypes = [vp, i64, i64, vp, vp, vp]
         L.bitnet_unpack_tl.argtypes = [ci, vp, i64, i64, ci, vp, vp, vp]
         L.bitnet_tl_num_groups.argtypes = [ci, i64, ci]
@@ -273,6 +274,37 @@ def bitnet_linear_host(fmt, packed, w_scale, M, K, x_host, y_host, x_dev, q_dev,
     _check(lib().bitnet_linear_host(_fmt(fmt), _ptr(packed), float(w_scale), M, K, bk3, _ptr(x_host), T,
                                     _ptr(y_host), _ptr(x_dev), _ptr(q_dev), _ptr(scale_dev), _ptr(y_dev),
                                     _ptr(workspace), ws_bytes, _stream(stream)), "bitnet_linear_host")
+
+
+class HostLinear(C.Structure):
+    """Mirror of bitnet_host_linear_t."""
+    _fields_ = [("fmt", C.c_int32), ("bk3", C.c_int32), ("packed", C.c_void_p), ("w_scale", C.c_float),
+                ("M", C.c_int64), ("K", C.c_int64), ("T", C.c_int64), ("x_host", C.c_void_p), ("y_host", C.c_void_p),
+                ("x_dev", C.c_void_p), ("q_dev", C.c_void_p), ("scale_dev", C.c_void_p), ("y_dev", C.c_void_p),
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
+def make_host_batch(items):
+    """items: dicts with fmt, packed, w_scale, M, K, x_host, y_host, x_dev, q_dev, scale_dev, y_dev and
+    optionally workspace, bk3 (tensors).  Returns the ctypes array for bitnet_linear_host_batch; the caller
+    keeps the tensors alive."""
+    arr = (HostLinear * len(items))()
+    for a, d in zip(arr, items):
+        ws = d.get("workspace")
+        a.fmt, a.bk3, a.packed, a.w_scale = _fmt(d["fmt"]), int(d.get("bk3", 0)), d["packed"].data_ptr(), float(d["w_scale"])
+        a.M, a.K, a.T = int(d["M"]), int(d["K"]), int(d["x_host"].shape[0])
+        a.x_host, a.y_host = d["x_host"].data_ptr(), d["y_host"].data_ptr()
+        a.x_dev, a.q_dev, a.scale_dev, a.y_dev = (d["x_dev"].data_ptr(), d["q_dev"].data_ptr(),
+                                                  d["scale_dev"].data_ptr(), d["y_dev"].data_ptr())
+        a.workspace = None if ws is None else ws.data_ptr()
+        a.workspace_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    return arr
+
+
+def bitnet_linear_host_batch(batch, stream=None):
+    """Queues a batch made by make_host_batch: uploads, kernels and downloads overlap; the caller
+    synchronises the stream before reading the host results."""
+    _check(lib().bitnet_linear_host_batch(batch, C.c_int64(len(batch)), _stream(stream)), "bitnet_linear_host_batch")
 
 
 NOALLOC_MAX_M = 32768

@@ -4,6 +4,8 @@
 #include <cstring>
 #include <mutex>
 
+#include <vector>
+
 #include "common.cuh"
 
 namespace bitnet {
@@ -248,3 +250,77 @@ int bitnet_linear_host(bitnet_fmt_t fmt, const void* packed, float w_scale, int6
 }
 
 }  // extern "C"
+
+namespace {
+// Side streams and events of bitnet_linear_host_batch, per device, created on first use and kept.
+struct HostPipe {
+  cudaStream_t up = nullptr, down = nullptr;
+  std::vector<cudaEvent_t> ev;
+};
+HostPipe* host_pipe() {
+  static HostPipe pipes[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+  HostPipe* p = &pipes[dev & 63];
+  if (!p->up) {
+    if (cudaStreamCreateWithFlags(&p->up, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithFlags(&p->down, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+  }
+  return p;
+}
+bool grow_events(HostPipe* p, size_t n) {
+  while (p->ev.size() < n) {
+    cudaEvent_t e;
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return false;
+    p->ev.push_back(e);
+  }
+  return true;
+}
+}  // namespace
+
+extern "C" int bitnet_linear_host_batch(const bitnet_host_linear_t* items, int64_t n, void* stream) {
+  if (n < 0 || (n > 0 && !items)) return BITNET_ERR_INVALID_ARG;
+  if (n == 0) return BITNET_OK;
+  for (int64_t i = 0; i < n; ++i) {
+    const bitnet_host_linear_t& d = items[i];
+    if (!d.packed || !d.x_host || !d.y_host || !d.x_dev || !d.q_dev || !d.scale_dev || !d.y_dev || d.T < 1 ||
+        d.M < 1 || d.K < 1)
+      return BITNET_ERR_INVALID_ARG;
+  }
+  HostPipe* p = host_pipe();
+  if (!p || !grow_events(p, (size_t)(2 * n + 2))) return note_cuda_error(cudaErrorUnknown);
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e;
+#define BN_TRY(call) do { e = (call); if (e != cudaSuccess) return note_cuda_error(e); } while (0)
+  // the side streams start after whatever is already queued on `stream` (the staging buffers may be in use)
+  cudaEvent_t e_in = p->ev[2 * n], e_out = p->ev[2 * n + 1];
+  BN_TRY(cudaEventRecord(e_in, st));
+  BN_TRY(cudaStreamWaitEvent(p->up, e_in, 0));
+  BN_TRY(cudaStreamWaitEvent(p->down, e_in, 0));
+  for (int64_t i = 0; i < n; ++i) {
+    const bitnet_host_linear_t& d = items[i];
+    BN_TRY(cudaMemcpyAsync(d.x_dev, d.x_host, (size_t)d.T * d.K * sizeof(float), cudaMemcpyHostToDevice, p->up));
+    BN_TRY(cudaEventRecord(p->ev[2 * i], p->up));
+  }
+  for (int64_t i = 0; i < n; ++i) {
+    const bitnet_host_linear_t& d = items[i];
+    BN_TRY(cudaStreamWaitEvent(st, p->ev[2 * i], 0));
+    int rc = bitnet_linear((bitnet_fmt_t)d.fmt, d.packed, d.w_scale, d.M, d.K, d.bk3, d.x_dev, d.T, d.q_dev, d.scale_dev,
+                           d.y_dev, nullptr, d.workspace, d.workspace_bytes, stream);
+    if (rc) {
+      // join the side streams before reporting, so that nothing of this call is left dangling
+      cudaEventRecord(e_out, p->down);
+      cudaStreamWaitEvent(st, e_out, 0);
+      cudaEventRecord(e_out, p->up);
+      cudaStreamWaitEvent(st, e_out, 0);
+      return rc;
+    }
+    BN_TRY(cudaEventRecord(p->ev[2 * i + 1], st));
+    BN_TRY(cudaStreamWaitEvent(p->down, p->ev[2 * i + 1], 0));
+    BN_TRY(cudaMemcpyAsync(d.y_host, d.y_dev, (size_t)d.T * d.M * sizeof(float), cudaMemcpyDeviceToHost, p->down));
+  }
+  BN_TRY(cudaEventRecord(e_out, p->down));
+  BN_TRY(cudaStreamWaitEvent(st, e_out, 0));
+#undef BN_TRY
+  return BITNET_OK;
+}

@@ -307,3 +307,39 @@ def test_split_k_kernel_variant_in_a_child_process():
 
 def test_zzz_no_device_wait_ever_gave_up():
     assert bn.bitnet_device_status() == 0
+
+
+@pytest.mark.gpu
+def test_linear_host_batch_matches_single_calls():
+    """bitnet_linear_host_batch (overlapped copies) gives what bitnet_linear gives item by item, for a mix
+    of formats, shapes and batch sizes, and leaves the stream joined (two batches back to back)."""
+    shapes = [("i2s", 512, 2048, 1), ("i2s", 96, 8192, 2), ("tl2", 64, 1536, 1), ("i2s", 1040, 4096, 4), ("tl1", 128, 256, 3)]
+    items, keep, refs = [], [], []
+    for n, (fmt, M, K, T) in enumerate(shapes):
+        w = synth.ternary(40 + n, 0, M, K, 1 / 3, 1 / 3)
+        x = synth.normal(40 + n, 1, T, K)
+        blob = bn.pack(fmt, w.cuda())
+        xh = x.clone().pin_memory()
+        yh = torch.zeros((T, M), dtype=torch.float32).pin_memory()
+        xd = torch.empty((T, K), dtype=torch.float32, device="cuda")
+        qd = torch.empty((T, K), dtype=torch.int8, device="cuda")
+        sd = torch.empty(T, dtype=torch.float32, device="cuda")
+        yd = torch.empty((T, M), dtype=torch.float32, device="cuda")
+        ws = bn.new_workspace(fmt, T, M, K)
+        items.append(dict(fmt=fmt, packed=blob, w_scale=0.75, M=M, K=K, x_host=xh, y_host=yh, x_dev=xd, q_dev=qd,
+                          scale_dev=sd, y_dev=yd, workspace=ws))
+        keep.append((blob, xh, yh, xd, qd, sd, yd, ws))
+        q = torch.empty_like(qd)
+        sc = torch.empty_like(sd)
+        y = torch.empty_like(yd)
+        bn.bitnet_linear(fmt, blob, 0.75, M, K, x.cuda(), q=q, act_scale=sc, y=y, workspace=bn.new_workspace(fmt, T, M, K))
+        refs.append(y.cpu())
+    batch = bn.make_host_batch(items)
+    for rep in range(2):
+        for it in items:
+            it["y_host"].zero_()
+        bn.bitnet_linear_host_batch(batch)
+        torch.cuda.current_stream().synchronize()
+        for it, ref in zip(items, refs):
+            assert torch.equal(it["y_host"], ref), (rep, it["fmt"], it["M"], it["K"])
+    assert bn.bitnet_device_status() == 0
