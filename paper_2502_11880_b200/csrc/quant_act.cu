@@ -120,6 +120,76 @@ quant_act_kernel(const float* __restrict__ x, int64_t K, int8_t* __restrict__ q,
   }
 }
 
+// Single-pass variant for rows that fit the CTA's registers (K <= 32 * NT floats): NT threads per token, each
+// keeps 8 float4 of the row between the absmax reduction and the rounding, so x is read from memory once and
+// small rows use small CTAs (many tokens per SM in the prefill case).  Same operations in the same order
+// as quant_act_kernel: the bytes are identical.
+template <int NT>
+__global__ void __launch_bounds__(NT) quant_act_reg_kernel(const float* __restrict__ x, int64_t K, int8_t* __restrict__ q,
+                                                           float* __restrict__ act_scale, int32_t* __restrict__ act_sum) {
+  constexpr int VPT = 8;
+  __shared__ float red[32];
+  __shared__ int redi[32];
+  const int64_t t = blockIdx.x;
+  const float4* x4 = reinterpret_cast<const float4*>(x + t * K);
+  int* q4 = reinterpret_cast<int*>(q + t * K);
+  const int tid = threadIdx.x, n4 = (int)(K / 4);
+  if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  float4 v[VPT];
+#pragma unroll
+  for (int r = 0; r < VPT; ++r) {
+    const int i = tid + r * NT;
+    v[r] = (i < n4) ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  float m = 0.0f;
+#pragma unroll
+  for (int r = 0; r < VPT; ++r)
+    m = fmaxf(m, fmaxf(fmaxf(fabsf(v[r].x), fabsf(v[r].y)), fmaxf(fabsf(v[r].z), fabsf(v[r].w))));
+  m = warp_max(m);
+  if ((tid & 31) == 0) red[tid >> 5] = m;
+  __syncthreads();
+  float amax = 0.0f;
+#pragma unroll
+  for (int w = 0; w < NT / 32; ++w) amax = fmaxf(amax, red[w]);
+  const float amax_c = fmaxf(amax, 1e-5f);
+  const float s = __fdiv_rn(127.0f, amax_c);
+  int sum = 0;
+#pragma unroll
+  for (int r = 0; r < VPT; ++r) {
+    const int i = tid + r * NT;
+    if (i < n4) {
+      const int a = quant1(v[r].x, s), b = quant1(v[r].y, s), c = quant1(v[r].z, s), d = quant1(v[r].w, s);
+      sum += a + b + c + d;
+      q4[i] = (a & 255) | ((b & 255) << 8) | ((c & 255) << 16) | ((d & 255) << 24);
+    }
+  }
+  sum = warp_sum(sum);
+  if ((tid & 31) == 0) redi[tid >> 5] = sum;
+  __syncthreads();
+  if (tid == 0) {
+    int tot = 0;
+#pragma unroll
+    for (int w = 0; w < NT / 32; ++w) tot += redi[w];
+    if (act_sum) act_sum[t] = tot;
+    act_scale[t] = __fdiv_rn(amax_c, 127.0f);
+  }
+}
+
+template <int NT>
+cudaError_t launch_reg(const float* x, int64_t T, int64_t K, int8_t* q, float* act_scale, int32_t* act_sum, cudaStream_t st) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)T);
+  cfg.blockDim = dim3(NT);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = early_start_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, quant_act_reg_kernel<NT>, x, K, q, act_scale, act_sum);
+}
+
 __global__ void fill_scale_kernel(float* act_scale, int64_t T) {
   __shared__ float sc;
   if (threadIdx.x == 0) {
@@ -142,6 +212,14 @@ int launch_quant_act(const float* x, int64_t T, int64_t K, int per_tensor, int8_
     quant_act_kernel<<<(unsigned)T, QTHREADS, 0, st>>>(x, K, q, act_scale, act_sum,
                                                        reinterpret_cast<const unsigned*>(act_scale));
     fill_scale_kernel<<<1, 256, 0, st>>>(act_scale, T);
+  } else if ((K & 3) == 0 && K <= 32 * 1024 && aligned16(x) && (reinterpret_cast<uintptr_t>(q) & 3u) == 0) {
+    // rows are 16-byte aligned when x is and K % 4 == 0
+    cudaError_t e;
+    if (K <= 32 * 128) e = launch_reg<128>(x, T, K, q, act_scale, act_sum, st);
+    else if (K <= 32 * 256) e = launch_reg<256>(x, T, K, q, act_scale, act_sum, st);
+    else if (K <= 32 * 512) e = launch_reg<512>(x, T, K, q, act_scale, act_sum, st);
+    else e = launch_reg<1024>(x, T, K, q, act_scale, act_sum, st);
+    if (e != cudaSuccess) return note_cuda_error(e);
   } else {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)T);
