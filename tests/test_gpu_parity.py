@@ -235,6 +235,56 @@ def test_workload_sweep100b_sampled_rows(layer):
         torch.cuda.empty_cache()
 
 
+def test_sweep100b_layer_in_the_benchmark_launch_configuration():
+    """One full-size layer of the sweep exactly as bench.py runs it: the four linears as fused bitnet_linear
+    calls (fp32 activations in), captured in a CUDA graph with programmatic dependent launch and replayed;
+    sampled output rows against the oracle, twice (the second replay must not depend on the first)."""
+    wl = synth.CONFIGS["sweep100b"]
+    layer = 3
+    blobs, xs, ys, qs, scs, rows_l, refs = [], [], [], [], [], [], []
+    w_scale = 2.0 / 3.0
+    for j, lin in enumerate(wl.linears):
+        wd = wl.weights(layer, j, device="cuda")
+        blobs.append(bn.pack("i2s", wd, check=False))
+        del wd
+        x = wl.activations(layer, j, 1)
+        xs.append(x.cuda())
+        ys.append(torch.zeros((1, lin.M), dtype=torch.float32, device="cuda"))
+        qs.append(torch.empty((1, lin.K), dtype=torch.int8, device="cuda"))
+        scs.append(torch.empty(1, dtype=torch.float32, device="cuda"))
+        rows = _sampled_rows(lin.M, seed=100 + j)
+        w_rows = np.stack([wl.weights(layer, j, row_start=int(r), rows=1).numpy()[0] for r in rows])
+        q_ref, sc_ref, _ = oracle.quant_act(x.numpy())
+        rows_l.append(rows)
+        refs.append((q_ref, sc_ref, oracle.mpgemm_def(q_ref, w_rows)))
+    ws = torch.zeros(64, dtype=torch.uint8, device="cuda")
+
+    def layer_step():
+        for j, lin in enumerate(wl.linears):
+            bn.bitnet_linear("i2s", blobs[j], w_scale, lin.M, lin.K, xs[j], q=qs[j], act_scale=scs[j], y=ys[j], workspace=ws)
+
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        layer_step()
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        layer_step()
+    for rep in range(2):
+        for y in ys:
+            y.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        for j in range(len(wl.linears)):
+            q_ref, sc_ref, acc_ref = refs[j]
+            assert np.array_equal(npy(qs[j]), q_ref), (rep, j)
+            assert np.array_equal(npy(scs[j]).view(np.uint32), sc_ref.view(np.uint32)), (rep, j)
+            check_y(ys[j][:, torch.as_tensor(rows_l[j]).cuda()], acc_ref, sc_ref, w_scale)
+    assert bn.bitnet_device_status() == 0
+
+
 def test_workload_prefill_sampled():
     wl = synth.CONFIGS["prefill"]
     lin = wl.linears[0]
