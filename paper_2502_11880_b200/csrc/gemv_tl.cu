@@ -116,8 +116,8 @@ __device__ __forceinline__ int sign_mask(unsigned sg, int bit) {   // 0 or -1 fr
 __global__ void __launch_bounds__(THREADS, 2) gemv_tl_kernel(const TlArgs a) {
   extern __shared__ __align__(128) int smem[];
   int* tab = smem;                                   // [tiles_per_slice][32][16]
-  int* red = smem + a.tiles_per_slice * 512;         // [WARPS][32][2]
-  uint64_t* bar = reinterpret_cast<uint64_t*>(red + WARPS * 64);
+  int* red = smem + a.tiles_per_slice * 512;         // [2][WARPS][32][2]: the sums of two row blocks in flight
+  uint64_t* bar = reinterpret_cast<uint64_t*>(red + 2 * WARPS * 64);
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int slice = blockIdx.y;
@@ -176,8 +176,9 @@ __global__ void __launch_bounds__(THREADS, 2) gemv_tl_kernel(const TlArgs a) {
     iw = __ldg(reinterpret_cast<const uint4*>(tp) + lane);
     sg = (tile0 + tl < a.g.tiles3) ? __ldg(reinterpret_cast<const unsigned*>(tp + 512) + lane) : 0u;
   }
-  for (; rb < nrb; rb += gridDim.x) {
+  for (int nb = 0; rb < nrb; rb += gridDim.x, ++nb) {
     int lo = 0, hi = 0;
+    int* redb = red + (nb & 1) * (WARPS * 64);
     while (tl < ntiles) {
       const uint4 ciw = iw;
       const unsigned csg = sg;
@@ -216,15 +217,18 @@ __global__ void __launch_bounds__(THREADS, 2) gemv_tl_kernel(const TlArgs a) {
       if (tl >= ntiles) break;
     }
     tl = warp;
-    red[(warp * 32 + lane) * 2 + 0] = lo;
-    red[(warp * 32 + lane) * 2 + 1] = hi;
+    redb[(warp * 32 + lane) * 2 + 0] = lo;
+    redb[(warp * 32 + lane) * 2 + 1] = hi;
+    // One barrier per row block: the warp whose turn it is adds the partial sums while the others go on; the
+    // buffer is written again two row blocks later, after the next barrier, which that warp reaches only when
+    // it has finished reading.
     __syncthreads();
-    if (warp == 0) {
+    if (warp == (nb % WARPS)) {
       int tot[2] = {0, 0};
 #pragma unroll
       for (int w = 0; w < WARPS; ++w) {
-        tot[0] += red[(w * 32 + lane) * 2 + 0];
-        tot[1] += red[(w * 32 + lane) * 2 + 1];
+        tot[0] += redb[(w * 32 + lane) * 2 + 0];
+        tot[1] += redb[(w * 32 + lane) * 2 + 1];
       }
       const int row = rb * 32 + lane;
       if (a.nslices == 1) {
@@ -253,7 +257,6 @@ __global__ void __launch_bounds__(THREADS, 2) gemv_tl_kernel(const TlArgs a) {
         }
       }
     }
-    __syncthreads();
   }
 }
 
@@ -313,13 +316,13 @@ int launch_gemv_tl(int fmt, const uint8_t* packed, float w_scale, int64_t M, int
   a.w_scale = w_scale;
   slicing(g, &a.nslices, &a.tiles_per_slice);
   a.ws_ticket = reinterpret_cast<unsigned*>(reinterpret_cast<int32_t*>(ws) + (int64_t)T * M);
-  const size_t smem = (size_t)a.tiles_per_slice * 2048 + WARPS * 64 * sizeof(int) + 16;
+  const size_t smem = (size_t)a.tiles_per_slice * 2048 + 2 * WARPS * 64 * sizeof(int) + 16;
   static bool attr_set[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
   if (!attr_set[dev & 63]) {
     cudaError_t e = cudaFuncSetAttribute(gemv_tl_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         MAX_SLICE_TILES * 2048 + WARPS * 64 * (int)sizeof(int) + 16);
+                                         MAX_SLICE_TILES * 2048 + 2 * WARPS * 64 * (int)sizeof(int) + 16);
     if (e != cudaSuccess) return note_cuda_error(e);
     attr_set[dev & 63] = true;
   }
