@@ -210,13 +210,24 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
     // kernel: s = 127 / max(amax, 1e-5), q = clamp(rint(x * s)).
     const int n4 = (int)(a.K / 4);
     const int nrow = (max(n4, kp / 4) + THREADS - 1) / THREADS;     // rows of THREADS words that hold anything
-    for (int tok = 0; tok < a.T; ++tok) {
+    // With few registers per row (the short-row instance) the next token's row is requested before this
+    // token's is reduced, so the tokens' round trips overlap.
+    constexpr bool AHEAD = XREG <= 8;
+    float4 xv[XREG], xn[AHEAD ? XREG : 1];
+    auto load_row = [&](float4* dst, int tok) {
       const float4* x4 = reinterpret_cast<const float4*>(a.x + (int64_t)tok * a.K);
-      float4 xv[XREG];
 #pragma unroll
       for (int r = 0; r < XREG; ++r) {
         const int i = threadIdx.x + r * THREADS;
-        xv[r] = (r < nrow && i < n4) ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        dst[r] = (r < nrow && i < n4) ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    };
+    if (AHEAD) load_row(xv, 0);
+    for (int tok = 0; tok < a.T; ++tok) {
+      if (AHEAD) {
+        if (tok + 1 < a.T) load_row(xn, tok + 1);
+      } else {
+        load_row(xv, tok);
       }
       if (tok == 0) first_fill(false);
       TL_PRO(18);
@@ -249,6 +260,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
           reinterpret_cast<int*>(qs_mem + tok * qst)[i] = word;
           if (blockIdx.x == 0 && a.q_out && i < n4) reinterpret_cast<int*>(a.q_out + (int64_t)tok * a.K)[i] = word;
         }
+      }
+      if (AHEAD) {
+#pragma unroll
+        for (int r = 0; r < XREG; ++r) xv[r] = xn[r];
       }
     }
   } else if (a.x) {
@@ -546,7 +561,7 @@ int launch_gemv_i2s_wring(const uint8_t* packed, float w_scale, int64_t M, int64
   a.nunits = p.nunits;
   a.pre = env_int("BITNET_I2S_PRE", 4);
   // short rows get the instance whose (fully unrolled) quantiser prologue is a quarter of the code
-  const bool small_x = x != nullptr && T == 1 && K <= 4 * 4 * THREADS;
+  const bool small_x = x != nullptr && K <= 4 * 4 * THREADS;
   switch (p.depth) {
     case 4: return launch_wring<4, XREG_MAX>(a, p, st);
     case 6: return launch_wring<6, XREG_MAX>(a, p, st);
