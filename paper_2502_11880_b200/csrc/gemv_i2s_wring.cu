@@ -43,7 +43,7 @@ constexpr int CW = 16;                   // warps
 constexpr int THREADS = CW * 32;
 constexpr int JQ = 4;                    // entries of a group's queue of upcoming units
 constexpr int XREG_MAX = 16;                 // float4 registers per thread of the fused quantiser's fast path
-constexpr size_t MAX_QS_BYTES = 116 * 1024;   // activations staged in shared memory up to this size
+constexpr size_t MAX_QS_BYTES = 144 * 1024;   // activations staged in shared memory up to this size
 
 #ifdef BITNET_PROFILE_GEMV
 // Development aid (never in the shipped build): per launch and CTA, %globaltimer at a few points.
