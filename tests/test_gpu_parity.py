@@ -137,8 +137,12 @@ def test_i2s_streaming_kernel_edges():
     """Shapes that stress the warp-ring decode kernel: fewer rows than one 16-row unit, ragged last unit,
     K exactly one ring long (2048), six tokens, and more units per CTA than the fixed first two per warp
     group (20000 rows at K = 8192), the last one both fused (four tokens) and with given codes."""
-    for (M, K, T) in [(1, 4096, 1), (17, 4096, 3), (300, 2048, 6), (33, 2048, 1)]:
-        check_linear("i2s", tern(36, M, K), synth.normal(36, M + T, T, K))
+    for (M, K, T) in [(1, 4096, 1), (17, 4096, 3), (300, 2048, 6), (33, 2048, 1), (48, 28672, 5), (48, 28672, 4)]:
+        w, x = tern(36, M, K), synth.normal(36, M + T, T, K)
+        out = check_linear("i2s", w, x)               # given codes (the last two: a shallower ring makes room for them)
+        y, q, sc, acc = bn.bitnet_linear("i2s", out["blob"], out["w_scale"], M, K, x.cuda(), want_acc=True)   # fused
+        torch.cuda.synchronize()
+        assert torch.equal(acc, out["acc"]) and torch.equal(y, out["y"]) and torch.equal(q, out["q"])
     M, K, T = 20000, 8192, 4
     w, x = tern(37, M, K), synth.normal(37, 1, T, K)
     out = check_linear("i2s", w, x)
