@@ -140,7 +140,7 @@ int bitnet_mpgemm(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
  *   x[T][K] fp32 in; q[T][K] int8 and act_scale[T] fp32 are OUTPUTS (the quantised activations, as
  *   bitnet_quant_act would give them); y[T][M] fp32 out; acc_out nullable; workspace as for
  *   bitnet_mpgemm.
- * For I2_S with T <= 6 (and T*(K+16) up to 144 KiB) this is ONE kernel: every CTA of the decode kernel
+ * For I2_S with T <= 8 (and T*(K+16) up to 144 KiB) this is ONE kernel: every CTA of the decode kernel
  * quantises the activation rows itself while its first weight tiles are in flight.  Otherwise it is
  * bitnet_quant_act followed by bitnet_mpgemm.  Results are identical either way.
  */

@@ -220,10 +220,10 @@ int bitnet_linear(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
       const char* e = getenv("BITNET_I2S_KERNEL");
       return e && strcmp(e, "splitk") == 0;
     }();
-    // Up to six tokens (the range of the warp-ring kernel): every CTA of the GEMV quantises the rows itself
-    // (one pass per row, the row held in registers).  Beyond that the redundant work costs more than a
-    // separate quantiser launch (measured).  BITNET_FUSE_MAX_T overrides the threshold.
-    static const int fuse_max = [] { const char* e = getenv("BITNET_FUSE_MAX_T"); return e ? atoi(e) : 6; }();
+    // Decode batches (up to 8 tokens): every CTA of the GEMV quantises the rows itself (one pass per row, the row
+    // held in registers), which measured faster than a separate quantiser launch at every batch size where the
+    // streaming kernel applies.  BITNET_FUSE_MAX_T lowers the threshold.
+    static const int fuse_max = [] { const char* e = getenv("BITNET_FUSE_MAX_T"); return e ? atoi(e) : 8; }();
     if (!no_fuse && T <= fuse_max && gemv_i2s_stream_supported((int)T, M, K, true))
       return launch_gemv_i2s_stream((const uint8_t*)packed, w_scale, M, K, x, q, act_scale, (int)T, y, acc_out,
                                     (cudaStream_t)stream);

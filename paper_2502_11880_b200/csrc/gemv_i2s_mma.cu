@@ -517,16 +517,16 @@ int launch_mma(const MmaArgs& a, const Plan& p, cudaStream_t st) {
 
 }  // namespace
 
-// The warp-private-ring kernel takes batches of up to 6 tokens (it reads the activations from shared
-// memory for every chunk, which costs more the more lanes hold a real token); this file's kernel, which
-// keeps them in registers, takes the rest.  BITNET_I2S_STREAM=ring / =warp forces one of them.
+// The warp-private-ring kernel takes every shape it supports (measured faster or equal at every batch size up
+// to 8); this file's kernel, which keeps the activations in registers, takes the rest (K below 2048, or
+// more staged activations than the other kernel has room for).  BITNET_I2S_STREAM=ring / =warp forces one of them.
 static bool prefer_wring(int T) {
   static int v = -1;
   if (v < 0) {
     const char* e = getenv("BITNET_I2S_STREAM");
     v = (e && strcmp(e, "ring") == 0) ? 0 : (e && strcmp(e, "warp") == 0) ? 2 : 1;
   }
-  return v == 2 || (v == 1 && T <= 6);
+  return v == 2 || (v == 1 && T <= 8);
 }
 
 bool gemv_i2s_stream_supported(int T, int64_t M, int64_t K, bool fused) {
