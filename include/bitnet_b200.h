@@ -162,11 +162,12 @@ int bitnet_linear_host(bitnet_fmt_t fmt, const void* packed, float w_scale, int6
 
 /*
  * A batch of linear layers with HOST activations and HOST results (Alg. 1 end to end per item), with the
- * copies overlapped with the kernels: item i's x_host is uploaded on an internal stream, its kernel
- * runs on `stream` once that upload is complete, and its y_host is downloaded on a second internal
- * stream once the kernel is complete.  Kernels run in item order on `stream`; when the call returns
- * everything is queued, and `stream` has been made to wait for the last download, so work queued on
- * `stream` afterwards (or a synchronisation of `stream`) follows every copy of the batch.
+ * copies overlapped with the kernels: the x_host of a group of 8 consecutive items are uploaded on an
+ * internal stream, their kernels run on `stream` once those uploads are complete, and their y_host are
+ * downloaded on a second internal stream once the group's kernels are complete, while the next groups'
+ * uploads and kernels proceed.  Kernels run in item order on `stream`; when the call returns everything is
+ * queued, and `stream` has been made to wait for the last download, so work queued on `stream` afterwards
+ * (or a synchronisation of `stream`) follows every copy of the batch.
  *   - items[n]: plain structs in host memory, read during the call only.
  *   - x_host / y_host should be pinned.  The device buffers of different items must not overlap
  *     (uploads run ahead of the kernels); the workspace may be shared (the kernels are serial).

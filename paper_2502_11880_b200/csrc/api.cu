@@ -297,14 +297,18 @@ extern "C" int bitnet_linear_host_batch(const bitnet_host_linear_t* items, int64
   BN_TRY(cudaEventRecord(e_in, st));
   BN_TRY(cudaStreamWaitEvent(p->up, e_in, 0));
   BN_TRY(cudaStreamWaitEvent(p->down, e_in, 0));
+  // Items are handled in groups of GROUP: one event after a group's uploads, one after its kernels.  Fewer
+  // events mean fewer driver calls per item, and the kernels of a group follow one another on `stream`
+  // without a wait in between, which keeps their programmatic dependent launch.
+  constexpr int64_t GROUP = 8;
   for (int64_t i = 0; i < n; ++i) {
     const bitnet_host_linear_t& d = items[i];
     BN_TRY(cudaMemcpyAsync(d.x_dev, d.x_host, (size_t)d.T * d.K * sizeof(float), cudaMemcpyHostToDevice, p->up));
-    BN_TRY(cudaEventRecord(p->ev[2 * i], p->up));
+    if (i % GROUP == GROUP - 1 || i == n - 1) BN_TRY(cudaEventRecord(p->ev[2 * (i / GROUP)], p->up));
   }
   for (int64_t i = 0; i < n; ++i) {
     const bitnet_host_linear_t& d = items[i];
-    BN_TRY(cudaStreamWaitEvent(st, p->ev[2 * i], 0));
+    if (i % GROUP == 0) BN_TRY(cudaStreamWaitEvent(st, p->ev[2 * (i / GROUP)], 0));
     int rc = bitnet_linear((bitnet_fmt_t)d.fmt, d.packed, d.w_scale, d.M, d.K, d.bk3, d.x_dev, d.T, d.q_dev, d.scale_dev,
                            d.y_dev, nullptr, d.workspace, d.workspace_bytes, stream);
     if (rc) {
@@ -315,9 +319,14 @@ extern "C" int bitnet_linear_host_batch(const bitnet_host_linear_t* items, int64
       cudaStreamWaitEvent(st, e_out, 0);
       return rc;
     }
-    BN_TRY(cudaEventRecord(p->ev[2 * i + 1], st));
-    BN_TRY(cudaStreamWaitEvent(p->down, p->ev[2 * i + 1], 0));
-    BN_TRY(cudaMemcpyAsync(d.y_host, d.y_dev, (size_t)d.T * d.M * sizeof(float), cudaMemcpyDeviceToHost, p->down));
+    if (i % GROUP == GROUP - 1 || i == n - 1) {
+      const int64_t g0 = (i / GROUP) * GROUP;
+      BN_TRY(cudaEventRecord(p->ev[2 * (i / GROUP) + 1], st));
+      BN_TRY(cudaStreamWaitEvent(p->down, p->ev[2 * (i / GROUP) + 1], 0));
+      for (int64_t j = g0; j <= i; ++j)
+        BN_TRY(cudaMemcpyAsync(items[j].y_host, items[j].y_dev, (size_t)items[j].T * items[j].M * sizeof(float),
+                               cudaMemcpyDeviceToHost, p->down));
+    }
   }
   BN_TRY(cudaEventRecord(e_out, p->down));
   BN_TRY(cudaStreamWaitEvent(st, e_out, 0));
