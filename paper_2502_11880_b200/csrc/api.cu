@@ -301,32 +301,41 @@ extern "C" int bitnet_linear_host_batch(const bitnet_host_linear_t* items, int64
   // events mean fewer driver calls per item, and the kernels of a group follow one another on `stream`
   // without a wait in between, which keeps their programmatic dependent launch.
   constexpr int64_t GROUP = 8;
-  for (int64_t i = 0; i < n; ++i) {
-    const bitnet_host_linear_t& d = items[i];
-    BN_TRY(cudaMemcpyAsync(d.x_dev, d.x_host, (size_t)d.T * d.K * sizeof(float), cudaMemcpyHostToDevice, p->up));
-    if (i % GROUP == GROUP - 1 || i == n - 1) BN_TRY(cudaEventRecord(p->ev[2 * (i / GROUP)], p->up));
-  }
-  for (int64_t i = 0; i < n; ++i) {
-    const bitnet_host_linear_t& d = items[i];
-    if (i % GROUP == 0) BN_TRY(cudaStreamWaitEvent(st, p->ev[2 * (i / GROUP)], 0));
-    int rc = bitnet_linear((bitnet_fmt_t)d.fmt, d.packed, d.w_scale, d.M, d.K, d.bk3, d.x_dev, d.T, d.q_dev, d.scale_dev,
-                           d.y_dev, nullptr, d.workspace, d.workspace_bytes, stream);
-    if (rc) {
-      // join the side streams before reporting, so that nothing of this call is left dangling
-      cudaEventRecord(e_out, p->down);
-      cudaStreamWaitEvent(st, e_out, 0);
-      cudaEventRecord(e_out, p->up);
-      cudaStreamWaitEvent(st, e_out, 0);
-      return rc;
+  const int64_t ngroups = (n + GROUP - 1) / GROUP;
+  auto upload_group = [&](int64_t g) -> cudaError_t {
+    const int64_t lo = g * GROUP, hi = (lo + GROUP < n) ? lo + GROUP : n;
+    for (int64_t i = lo; i < hi; ++i) {
+      const bitnet_host_linear_t& d = items[i];
+      cudaError_t er = cudaMemcpyAsync(d.x_dev, d.x_host, (size_t)d.T * d.K * sizeof(float), cudaMemcpyHostToDevice, p->up);
+      if (er != cudaSuccess) return er;
     }
-    if (i % GROUP == GROUP - 1 || i == n - 1) {
-      const int64_t g0 = (i / GROUP) * GROUP;
-      BN_TRY(cudaEventRecord(p->ev[2 * (i / GROUP) + 1], st));
-      BN_TRY(cudaStreamWaitEvent(p->down, p->ev[2 * (i / GROUP) + 1], 0));
-      for (int64_t j = g0; j <= i; ++j)
-        BN_TRY(cudaMemcpyAsync(items[j].y_host, items[j].y_dev, (size_t)items[j].T * items[j].M * sizeof(float),
-                               cudaMemcpyDeviceToHost, p->down));
+    return cudaEventRecord(p->ev[2 * g], p->up);
+  };
+  // uploads are queued one group ahead of the kernels, so that the first kernel does not wait for the host to
+  // have queued every upload of the batch
+  BN_TRY(upload_group(0));
+  for (int64_t g = 0; g < ngroups; ++g) {
+    if (g + 1 < ngroups) BN_TRY(upload_group(g + 1));
+    const int64_t lo = g * GROUP, hi = (lo + GROUP < n) ? lo + GROUP : n;
+    BN_TRY(cudaStreamWaitEvent(st, p->ev[2 * g], 0));
+    for (int64_t i = lo; i < hi; ++i) {
+      const bitnet_host_linear_t& d = items[i];
+      int rc = bitnet_linear((bitnet_fmt_t)d.fmt, d.packed, d.w_scale, d.M, d.K, d.bk3, d.x_dev, d.T, d.q_dev,
+                             d.scale_dev, d.y_dev, nullptr, d.workspace, d.workspace_bytes, stream);
+      if (rc) {
+        // join the side streams before reporting, so that nothing of this call is left dangling
+        cudaEventRecord(e_out, p->down);
+        cudaStreamWaitEvent(st, e_out, 0);
+        cudaEventRecord(e_out, p->up);
+        cudaStreamWaitEvent(st, e_out, 0);
+        return rc;
+      }
     }
+    BN_TRY(cudaEventRecord(p->ev[2 * g + 1], st));
+    BN_TRY(cudaStreamWaitEvent(p->down, p->ev[2 * g + 1], 0));
+    for (int64_t i = lo; i < hi; ++i)
+      BN_TRY(cudaMemcpyAsync(items[i].y_host, items[i].y_dev, (size_t)items[i].T * items[i].M * sizeof(float),
+                             cudaMemcpyDeviceToHost, p->down));
   }
   BN_TRY(cudaEventRecord(e_out, p->down));
   BN_TRY(cudaStreamWaitEvent(st, e_out, 0));
