@@ -14,7 +14,8 @@ import torch
 from . import synth  # noqa: F401  (seeded inputs; holds none of the method's arithmetic)
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libbitnet_b200.so")
+# BITNET_B200_LIB points at another build of the library (e.g. one compiled with different flags)
+LIB_PATH = os.environ.get("BITNET_B200_LIB") or os.path.join(_PKG, "libbitnet_b200.so")
 
 FMT_I2S, FMT_TL1, FMT_TL2 = 0, 1, 2
 FMT = {"i2s": FMT_I2S, "tl1": FMT_TL1, "tl2": FMT_TL2}
