@@ -166,9 +166,23 @@ int bitnet_tl_build_lut_debug(bitnet_fmt_t fmt, const int8_t* q_row, int64_t K, 
   return launch_tl_build_lut(fmt, q_row, K, g, lut, (cudaStream_t)stream);
 }
 
+// Batch sizes served by the mid-batch kernel (BITNET_I2S_MID_MIN_T / _MAX_T move the limits; MAX_T = 0: never).
+static bool use_mid(int64_t T, int64_t M, int64_t K) {
+  static const int lo = [] { const char* e = getenv("BITNET_I2S_MID_MIN_T"); return e ? atoi(e) : 9; }();
+  static const int hi = [] { const char* e = getenv("BITNET_I2S_MID_MAX_T"); return e ? atoi(e) : 64; }();
+  return T >= lo && T <= hi && T <= 64 && gemv_i2s_mid_supported((int)T, M, K);
+}
+
 size_t bitnet_mpgemm_workspace_bytes(bitnet_fmt_t fmt, int64_t T, int64_t M, int64_t K) {
   if (T < 1 || M < 1 || K < 1) return 0;
-  if (fmt == BITNET_FMT_I2S) return (T > 8) ? 0 : gemv_i2s_workspace_bytes(T, M, K);
+  if (fmt == BITNET_FMT_I2S) {
+    size_t n = T > 8 ? 0 : gemv_i2s_workspace_bytes(T, M, K);
+    if (use_mid(T, M, K)) {
+      const size_t m = gemv_i2s_mid_workspace_bytes((int)T, M, K);
+      if (m > n) n = m;
+    }
+    return n;
+  }
   return gemv_tl_workspace_bytes(fmt, T, M, K);
 }
 
@@ -190,6 +204,11 @@ int bitnet_mpgemm(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
   if (fmt == BITNET_FMT_I2S) {
     int rc = i2s_shape(M, K);
     if (rc) return rc;
+    // 9 to 64 tokens: the weight scan on mma.sync; it falls back to the prefill kernel when the caller's
+    // workspace is smaller than bitnet_mpgemm_workspace_bytes asked for
+    if (use_mid(T, M, K) && gemv_i2s_mid_workspace_bytes((int)T, M, K) <= (workspace ? workspace_bytes : 0))
+      return launch_gemv_i2s_mid((const uint8_t*)packed, w_scale, M, K, q, act_scale, (int)T, y, acc_out, workspace,
+                                 workspace_bytes, st);
     if (T > 8) return launch_gemm_i2s_prefill((const uint8_t*)packed, w_scale, M, K, q, act_scale, T, y, acc_out, st);
     return launch_gemv_i2s((const uint8_t*)packed, w_scale, M, K, q, act_scale, (int)T, y, acc_out, workspace,
                            workspace_bytes, st);

@@ -91,6 +91,13 @@ int gemv_i2s_stream_status(int* out);
 bool gemv_i2s_wring_supported(int T, int64_t M, int64_t K);
 int launch_gemv_i2s_wring(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const float* x, int8_t* q,
                           float* act_scale, int T, float* y, int32_t* acc_out, cudaStream_t st);
+// Batches of 9 to 64 tokens: mma.sync over K-slices, partial sums through a [T][M] int32 workspace when K is
+// cut into more than one slice (gemv_i2s_mid_workspace_bytes says how much; 0 = none needed).
+bool gemv_i2s_mid_supported(int T, int64_t M, int64_t K);
+size_t gemv_i2s_mid_workspace_bytes(int T, int64_t M, int64_t K);
+int launch_gemv_i2s_mid(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const int8_t* q,
+                        const float* act_scale, int T, float* y, int32_t* acc_out, void* ws, size_t ws_bytes,
+                        cudaStream_t st);
 // Programmatic dependent launch (kernels may start their prologue, and prefetch weights, before the
 // previous kernel in the stream has finished); process-wide switch, on by default.
 bool early_start_enabled();

@@ -167,6 +167,79 @@ def test_tl_many_row_blocks_few_tiles():
         assert np.array_equal(npy(out["acc"]), oracle.mpgemm_def(q_ref, w.numpy()))
 
 
+def test_i2s_mid_batch_kernel_every_tile_count():
+    """9 to 64 tokens (the mma.sync weight scan over K-slices): every number of 8-token tiles, ragged last
+    tiles, odd numbers of 16-row units, K that needs padding, one and many K-slices."""
+    shapes = [(7, 1024), (33, 3200), (300, 8640), (200, 28672), (2000, 2048)]
+    for i, (M, K) in enumerate(shapes):
+        w = tern(40 + i, M, K, 0.4, 0.3)
+        for T in (9, 16, 17, 24, 25, 32, 33, 40, 41, 48, 49, 56, 57, 64):
+            if M * K * T > 400e6 and T not in (9, 32, 57, 64):
+                continue                      # keep the oracle's share of the test to seconds
+            assert bn.bitnet_mpgemm_workspace_bytes("i2s", T, M, K) >= T * M * 4
+            check_linear("i2s", w, synth.normal(41, i * 100 + T, T, K))
+
+
+def test_i2s_mid_batch_workspace_comes_back_clean_and_is_optional():
+    M, K, T = 96, 8192, 40
+    w, x = tern(42, M, K), synth.normal(42, 1, T, K)
+    ws = bn.new_workspace("i2s", T, M, K)
+    first = run_linear("i2s", w, x, workspace=ws)
+    assert not npy(ws).any()
+    again = run_linear("i2s", w, x, workspace=ws)        # the sums of the first call are gone
+    assert torch.equal(first["acc"], again["acc"]) and torch.equal(first["y"], again["y"])
+    acc_ref = oracle.mpgemm_def(oracle.quant_act(x.numpy())[0], w.numpy())
+    assert np.array_equal(npy(again["acc"]), acc_ref)
+    # without a workspace the call still succeeds (the tensor-core prefill kernel takes it): same numbers
+    y2 = torch.empty_like(first["y"])
+    acc2 = torch.empty_like(first["acc"])
+    rc = bn.lib().bitnet_mpgemm(0, first["blob"].data_ptr(), first["w_scale"], M, K, 0, first["q"].data_ptr(),
+                                first["act_scale"].data_ptr(), T, y2.data_ptr(), acc2.data_ptr(), None, 0, None)
+    torch.cuda.synchronize()
+    assert rc == 0
+    assert torch.equal(acc2, first["acc"]) and torch.equal(y2, first["y"])
+
+
+def test_i2s_mid_batch_in_a_graph_with_early_start():
+    """Quantiser, scan and rescale kernels of several linears back to back in one CUDA graph (programmatic
+    dependent launch between them), sharing one workspace: the benchmark-style launch configuration."""
+    T = 24
+    shapes = [(512, 4096), (4096, 2048), (640, 8192)]
+    ws_bytes = max(bn.bitnet_mpgemm_workspace_bytes("i2s", T, M, K) for M, K in shapes)
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device="cuda")
+    items = []
+    for i, (M, K) in enumerate(shapes):
+        w, x = tern(43 + i, M, K), synth.normal(43, i, T, K)
+        items.append(dict(M=M, K=K, w=w, x=x.cuda(), blob=bn.pack("i2s", w.cuda()),
+                          q=torch.empty((T, K), dtype=torch.int8, device="cuda"),
+                          sc=torch.empty(T, dtype=torch.float32, device="cuda"),
+                          y=torch.empty((T, M), dtype=torch.float32, device="cuda"),
+                          acc=torch.empty((T, M), dtype=torch.int32, device="cuda")))
+
+    def run():
+        for d in items:
+            bn.bitnet_linear("i2s", d["blob"], 0.5, d["M"], d["K"], d["x"], q=d["q"], act_scale=d["sc"], y=d["y"],
+                             acc_out=d["acc"], workspace=ws)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        run()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        run()
+    for d in items:
+        d["y"].zero_(), d["acc"].zero_()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    for d in items:
+        q_ref, sc_ref, _ = oracle.quant_act(d["x"].cpu().numpy())
+        acc_ref = oracle.mpgemm_def(q_ref, d["w"].numpy())
+        assert np.array_equal(npy(d["acc"]), acc_ref)
+        check_y(d["y"], acc_ref, sc_ref, 0.5)
+    assert not npy(ws).any()
+
+
 def test_formats_agree_on_accumulators():
     M, K, T = 128, 8192, 3
     w, x = tern(32, M, K), synth.normal(32, 1, T, K)
