@@ -166,11 +166,18 @@ int bitnet_tl_build_lut_debug(bitnet_fmt_t fmt, const int8_t* q_row, int64_t K, 
   return launch_tl_build_lut(fmt, q_row, K, g, lut, (cudaStream_t)stream);
 }
 
-// Batch sizes served by the mid-batch kernel (BITNET_I2S_MID_MIN_T / _MAX_T move the limits; MAX_T = 0: never).
+// Batch sizes served by the mid-batch kernel: 9 to 64 tokens, and decode batches whose codes crowd the decode
+// kernel's shared memory (6 tokens or more, or more than 96 KiB of codes: measured crossover on the 100B
+// shapes).  BITNET_I2S_MID_MAX_T = 0 switches the kernel off, BITNET_I2S_MID_MIN_T raises the lower limit.
 static bool use_mid(int64_t T, int64_t M, int64_t K) {
-  static const int lo = [] { const char* e = getenv("BITNET_I2S_MID_MIN_T"); return e ? atoi(e) : 9; }();
+  static const int lo = [] { const char* e = getenv("BITNET_I2S_MID_MIN_T"); return e ? atoi(e) : 1; }();
   static const int hi = [] { const char* e = getenv("BITNET_I2S_MID_MAX_T"); return e ? atoi(e) : 64; }();
-  return T >= lo && T <= hi && T <= 64 && gemv_i2s_mid_supported((int)T, M, K);
+  if (T < lo || T > hi || T > 64) return false;
+  if (T <= 8 && T < 6 && T * i2s_kp(K) <= 96 * 1024) return false;
+  return gemv_i2s_mid_supported((int)T, M, K);
+}
+static bool mid_takes(int64_t T, int64_t M, int64_t K, const void* workspace, size_t workspace_bytes) {
+  return use_mid(T, M, K) && workspace && gemv_i2s_mid_workspace_bytes((int)T, M, K) <= workspace_bytes;
 }
 
 size_t bitnet_mpgemm_workspace_bytes(bitnet_fmt_t fmt, int64_t T, int64_t M, int64_t K) {
@@ -204,9 +211,9 @@ int bitnet_mpgemm(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
   if (fmt == BITNET_FMT_I2S) {
     int rc = i2s_shape(M, K);
     if (rc) return rc;
-    // 9 to 64 tokens: the weight scan on mma.sync; it falls back to the prefill kernel when the caller's
-    // workspace is smaller than bitnet_mpgemm_workspace_bytes asked for
-    if (use_mid(T, M, K) && gemv_i2s_mid_workspace_bytes((int)T, M, K) <= (workspace ? workspace_bytes : 0))
+    // 9 to 64 tokens (and crowded decode batches): the weight scan on mma.sync; the prefill (or decode) kernel
+    // takes the call when the caller's workspace is smaller than bitnet_mpgemm_workspace_bytes asked for
+    if (mid_takes(T, M, K, workspace, workspace_bytes))
       return launch_gemv_i2s_mid((const uint8_t*)packed, w_scale, M, K, q, act_scale, (int)T, y, acc_out, workspace,
                                  workspace_bytes, st);
     if (T > 8) return launch_gemm_i2s_prefill((const uint8_t*)packed, w_scale, M, K, q, act_scale, T, y, acc_out, st);
@@ -232,7 +239,7 @@ int bitnet_linear(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
   if (!aligned16(packed) || !aligned16(x) || !aligned16(q) || !aligned16(y) || (acc_out && !aligned16(acc_out)) ||
       (reinterpret_cast<uintptr_t>(act_scale) & 3u))
     return BITNET_ERR_INVALID_ARG;
-  if (fmt == BITNET_FMT_I2S && T <= 8) {
+  if (fmt == BITNET_FMT_I2S && T <= 8 && !mid_takes(T, M, K, workspace, workspace_bytes)) {
     int rc = i2s_shape(M, K);
     if (rc) return rc;
     static const bool no_fuse = [] {

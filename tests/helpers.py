@@ -42,9 +42,15 @@ def run_linear(fmt, w_t, x_t, bk3=0, workspace=None, w_scale=None):
     return dict(q=q, act_scale=sc, act_sum=sm, blob=blob, y=y, acc=acc, w_scale=ws)
 
 
-def check_linear(fmt, w_t, x_t, bk3=0, rows=None):
+def no_workspace():
+    """An empty workspace: calls that would use one when offered (the I2_S mid-batch kernel for crowded decode
+    batches) run the kernel that needs none instead."""
+    return torch.empty(0, dtype=torch.uint8, device="cuda")
+
+
+def check_linear(fmt, w_t, x_t, bk3=0, rows=None, workspace=None):
     """Element-by-element parity of one linear layer against the oracle (all rows, or a sample)."""
-    out = run_linear(fmt, w_t, x_t, bk3)
+    out = run_linear(fmt, w_t, x_t, bk3, workspace)
     w_np, x_np = w_t.numpy(), x_t.numpy()
     q_ref, sc_ref, sm_ref = oracle.quant_act(x_np)
     assert np.array_equal(npy(out["q"]), q_ref)

@@ -9,7 +9,7 @@ import oracle
 import paper_2502_11880_b200 as bn
 from paper_2502_11880_b200 import synth
 
-from helpers import check_linear, check_y, dev, npy, oracle_pack, run_linear
+from helpers import check_linear, check_y, dev, no_workspace, npy, oracle_pack, run_linear
 
 pytestmark = pytest.mark.gpu
 
@@ -136,19 +136,23 @@ def test_constant_weights_and_workspace_reuse(fmt):
 def test_i2s_streaming_kernel_edges():
     """Shapes that stress the warp-ring decode kernel: fewer rows than one 16-row unit, ragged last unit,
     K exactly one ring long (2048), six tokens, and more units per CTA than the fixed first two per warp
-    group (20000 rows at K = 8192), the last one both fused (four tokens) and with given codes."""
-    for (M, K, T) in [(1, 4096, 1), (17, 4096, 3), (300, 2048, 6), (33, 2048, 1), (48, 28672, 5), (48, 28672, 4)]:
+    group (20000 rows at K = 8192), each with given codes and fused.  Offered a workspace, the crowded
+    batches (six tokens; five and four at K = 28672) go to the mid-batch kernel instead: both must agree."""
+    shapes = [(1, 4096, 1), (17, 4096, 3), (300, 2048, 6), (33, 2048, 1), (48, 28672, 5), (48, 28672, 4),
+              (20000, 8192, 4)]
+    for (M, K, T) in shapes:
         w, x = tern(36, M, K), synth.normal(36, M + T, T, K)
-        out = check_linear("i2s", w, x)               # given codes (the last two: a shallower ring makes room for them)
-        y, q, sc, acc = bn.bitnet_linear("i2s", out["blob"], out["w_scale"], M, K, x.cuda(), want_acc=True)   # fused
+        out = check_linear("i2s", w, x, workspace=no_workspace())     # given codes, decode kernel
+        y, q, sc, acc = bn.bitnet_linear("i2s", out["blob"], out["w_scale"], M, K, x.cuda(), want_acc=True,
+                                         workspace=no_workspace())    # fused
         torch.cuda.synchronize()
         assert torch.equal(acc, out["acc"]) and torch.equal(y, out["y"]) and torch.equal(q, out["q"])
-    M, K, T = 20000, 8192, 4
-    w, x = tern(37, M, K), synth.normal(37, 1, T, K)
-    out = check_linear("i2s", w, x)
-    y, q, sc, acc = bn.bitnet_linear("i2s", out["blob"], out["w_scale"], M, K, x.cuda(), want_acc=True)
-    torch.cuda.synchronize()
-    assert torch.equal(acc, out["acc"]) and torch.equal(y, out["y"]) and torch.equal(q, out["q"])
+        y, q, sc, acc = bn.bitnet_linear("i2s", out["blob"], out["w_scale"], M, K, x.cuda(), want_acc=True)
+        torch.cuda.synchronize()                                      # with whatever workspace the shape asks for
+        assert torch.equal(acc, out["acc"]) and torch.equal(y, out["y"]) and torch.equal(q, out["q"])
+        if bn.bitnet_mpgemm_workspace_bytes("i2s", T, M, K):
+            assert (T >= 6 or T * K > 96 * 1024)
+            check_linear("i2s", w, x)                                 # given codes, mid-batch kernel
 
 
 def test_i2s_very_long_k_runs_in_phases():
