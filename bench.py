@@ -266,6 +266,42 @@ class Sweep:
         return replay
 
 
+def bench_batched(sw, torch, T, steps, warmup, linears_per_graph=64):
+    """The same sweep with T tokens per linear (I2_S): bitnet_linear = quantiser + mpGEMM + rescale.  Every
+    linear keeps its own weights; the T activation rows of layer 0's four linears are reused by all layers."""
+    bn, dev = sw.bn, sw.x_dev.device
+    nl = len(sw.lin)
+    xs = [sw.wl.activations(0, j, T).to(dev) for j in range(nl)]
+    qs = [torch.empty((T, l.K), dtype=torch.int8, device=dev) for l in sw.lin]
+    sc = torch.empty(T, dtype=torch.float32, device=dev)
+    ys = [torch.empty((T, l.M), dtype=torch.float32, device=dev) for l in sw.lin]
+    ws = torch.zeros(max(16, max(bn.bitnet_mpgemm_workspace_bytes("i2s", T, l.M, l.K) for l in sw.lin)),
+                     dtype=torch.uint8, device=dev)
+
+    def step(lo, hi):
+        for i in range(lo, hi):
+            j = i % nl
+            lin = sw.lin[j]
+            bn.bitnet_linear("i2s", sw.blobs["i2s"][i], sw.w_scale[i], lin.M, lin.K, xs[j], q=qs[j], act_scale=sc,
+                             y=ys[j], workspace=ws)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        step(0, nl)
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    graphs = []
+    for lo in range(0, sw.n_linears(), linears_per_graph):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            step(lo, min(lo + linears_per_graph, sw.n_linears()))
+        graphs.append(g)
+    ms = time_replays(torch, lambda: [g.replay() for g in graphs], steps, warmup)
+    weights = sw.bytes["i2s"] * 4.0          # four weights per packed byte
+    return {"tokens": T, "ms_per_step": ms, "tokens_per_s": T / ms * 1e3, "weight_GBps": sw.bytes["i2s"] / ms / 1e6,
+            "int8_tops": 2.0 * T * weights / ms / 1e9}
+
+
 def max_over_ranks(torch, dist, ms, device):
     """The job's time for a region is the slowest rank's device time (every rank gets the same number back)."""
     if dist is None:
@@ -400,6 +436,11 @@ def run_ours(args):
             line["tl2"] = {"packed_bytes": sw.bytes["tl2"], "ms_per_step": ms_tl, "value": sw.bytes["tl2"] / ms_tl / 1e6,
                            "unit": UNIT, "gemv_only_GBps": sw.bytes["tl2"] / ms_tl_g / 1e6,
                            "frac_of_hbm_peak": sw.bytes["tl2"] / ms_tl_g / 1e6 / pk["hbm"]}
+        if not args.skip_batched:
+            line["batched_decode"] = {
+                "note": "the same sweep with T tokens per linear through bitnet_linear (T <= 5: the fused decode kernel; "
+                        "6 to 64: quantiser + mid-batch mma.sync kernel + rescale), CUDA graphs, inputs resident",
+                "runs": [bench_batched(sw, torch, T, max(3, args.steps // 5), 3) for T in (2, 4, 8, 16, 32, 64)]}
         del sw, g_full, g_gemv, g_quant
         g_tl = g_tl_g = None
         torch.cuda.empty_cache()
@@ -440,6 +481,7 @@ def main():
     ap.add_argument("--skip-tl2", action="store_true")
     ap.add_argument("--skip-prefill", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
+    ap.add_argument("--skip-batched", action="store_true")
     ap.add_argument("--no-early-start", action="store_true",
                     help="launch every kernel in plain stream order (no programmatic dependent launch)")
     args = ap.parse_args()
