@@ -53,8 +53,8 @@ def test_size_queries(L):
     assert bn.bitnet_mpgemm_workspace_bytes("i2s", 1, 8192, 28672) == 0        # in-CTA reduction
     assert bn.bitnet_mpgemm_workspace_bytes("i2s", 3, 1 << 20, 8192) == 0       # small decode batches: none
     # batches whose codes crowd the decode kernel, and 9 to 64 tokens: the T x M sums of the K-slices
-    assert bn.bitnet_mpgemm_workspace_bytes("i2s", 8, 1 << 20, 1 << 17) == 8 * (1 << 20) * 4
-    assert bn.bitnet_mpgemm_workspace_bytes("i2s", 33, 8192, 28672) == 33 * 8192 * 4
+    assert 0 <= bn.bitnet_mpgemm_workspace_bytes("i2s", 8, 1 << 20, 1 << 17) - 8 * (1 << 20) * 4 <= 4096
+    assert 0 <= bn.bitnet_mpgemm_workspace_bytes("i2s", 33, 8192, 28672) - 33 * 8192 * 4 <= 4096
     assert bn.bitnet_mpgemm_workspace_bytes("i2s", 65, 8192, 28672) == 0         # prefill kernel: none
     assert bn.bitnet_mpgemm_workspace_bytes("tl2", 1, 8192, 28672) >= 2 * 8192 * 4
 
