@@ -61,6 +61,7 @@ struct PrefillArgs {
   float* y;
   int32_t* acc_out;
   int tiles_m, tiles_t, nkb;
+  int tma_store;         // y leaves through shared memory and bulk tensor stores (needs M % 4 == 0, no acc_out)
 };
 
 struct __align__(8) Barriers {
@@ -133,7 +134,8 @@ __device__ __forceinline__ uint32_t slot_s8(uint32_t w, int s) {
 }
 
 __global__ void __launch_bounds__(THREADS, 1)
-gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const PrefillArgs a) {
+gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap ymap,
+                   const PrefillArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* tileA = smem;                               // STAGES x 16 KB
@@ -142,6 +144,7 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const PrefillArgs a
   volatile int* abort_flag = &bars->abort_flag;
 
   __shared__ float ep_scale[4][TILE_T];                // epilogue: act_scale[t] * w_scale of the current tile
+  __shared__ __align__(128) float ep_stage[4][32][32]; // epilogue: 32 tokens x 32 rows of y per warp, [token][row]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ntiles = a.tiles_m * a.tiles_t;
@@ -328,7 +331,23 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const PrefillArgs a
             : "r"(taddr + c0)
             : "memory");
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (m < a.M) {
+        if (a.tma_store) {
+          // 32 tokens x 32 rows through shared memory, then one bulk tensor store (rows and tokens beyond M
+          // and T are clipped by the tensor map): one instruction instead of 32 strided 128-byte stores
+          if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // previous box read out
+          __syncwarp();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) ep_stage[quarter][j][lane] = __fmul_rn((float)(int)v[j], my_scale[c0 + j]);
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) {
+            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                         ::"l"(&ymap), "r"((tile % a.tiles_m) * TILE_M + quarter * 32), "r"(t0 + c0),
+                           "r"(smem_u32(&ep_stage[quarter][0][0]))
+                         : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          }
+        } else if (m < a.M) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             const int t = t0 + c0 + j;
@@ -345,6 +364,7 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const PrefillArgs a
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);
     }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // the last boxes have left
   }
 
   // ---- teardown: every role has left its loop (all waits are bounded); free the tensor memory
@@ -375,6 +395,11 @@ EncodeTiledFn encode_fn() {
 int launch_gemm_i2s_simt(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const int8_t* q,
                          const float* act_scale, int64_t T, float* y, int32_t* acc_out, cudaStream_t st);
 
+static bool no_tma_store() {
+  static const bool off = [] { const char* e = getenv("BITNET_PREFILL_TMA_STORE"); return e && atoi(e) == 0; }();
+  return off;
+}
+
 int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const int8_t* q,
                             const float* act_scale, int64_t T, float* y, int32_t* acc_out, cudaStream_t st) {
   static const bool force_simt = [] {
@@ -394,7 +419,20 @@ int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return note_cuda_error(cudaErrorInvalidValue);
 
+  // y[T][M] fp32 as a tensor of 32 x 32 boxes for the epilogue's bulk stores
+  const bool tma_store = acc_out == nullptr && (M % 4) == 0 && !no_tma_store();
+  CUtensorMap ymap = qmap;
+  if (tma_store) {
+    const cuuint64_t ydim[2] = {(cuuint64_t)M, (cuuint64_t)T};
+    const cuuint64_t ystride[1] = {(cuuint64_t)M * 4};
+    const cuuint32_t ybox[2] = {32, 32};
+    r = enc(&ymap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, y, ydim, ystride, ybox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return note_cuda_error(cudaErrorInvalidValue);
+  }
+
   PrefillArgs a;
+  a.tma_store = tma_store ? 1 : 0;
   a.packed = packed;
   a.kp = i2s_kp(K);
   a.M = (int)M;
@@ -419,7 +457,7 @@ int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int
   int grid = dev_info().sm_count;
   const int ntiles = a.tiles_m * a.tiles_t;
   if (grid > ntiles) grid = ntiles;
-  gemm_i2s_tc_kernel<<<grid, THREADS, smem, st>>>(qmap, a);
+  gemm_i2s_tc_kernel<<<grid, THREADS, smem, st>>>(qmap, ymap, a);
   return check_launch();
 }
 

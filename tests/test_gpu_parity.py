@@ -366,6 +366,20 @@ def test_sweep100b_layer_in_the_benchmark_launch_configuration():
     assert bn.bitnet_device_status() == 0
 
 
+def test_prefill_output_paths_agree():
+    """The prefill kernel writes y either with plain stores (when the accumulators are asked for, or M % 4 != 0)
+    or through shared memory and bulk tensor stores: same bits, nothing written outside y, ragged M and T."""
+    for (M, K, T) in [(300, 1024, 70), (128, 512, 256), (1000, 2048, 333), (130, 512, 65)]:
+        w, x = tern(50, M, K), synth.normal(50, M + T, T, K)
+        out = check_linear("i2s", w, x)                       # with accumulators: plain stores, against the oracle
+        guard = torch.full((T + 8, M), 12345.0, dtype=torch.float32, device="cuda")
+        y = guard[4: T + 4]                                   # four rows in: 16-byte aligned for every M
+        bn.bitnet_mpgemm("i2s", out["blob"], out["w_scale"], M, K, out["q"], out["act_scale"], y=y)
+        torch.cuda.synchronize()
+        assert torch.equal(y, out["y"])
+        assert bool((guard[:4] == 12345.0).all()) and bool((guard[T + 4:] == 12345.0).all())
+
+
 def test_workload_prefill_sampled():
     wl = synth.CONFIGS["prefill"]
     lin = wl.linears[0]
