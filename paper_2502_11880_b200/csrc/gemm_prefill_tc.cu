@@ -30,14 +30,37 @@
 namespace bitnet {
 namespace {
 
+#ifndef A_IN_TMEM_
+#define A_IN_TMEM_ 0
+#endif
+// Build-time variant (-DA_IN_TMEM_=1, parity-tested, off): operand A (the unpacked weights) goes from the unpack
+// warps' registers straight into tensor memory (tcgen05.st) instead of a shared-memory tile.  Shared memory
+// is what binds this kernel: per K block the MMAs read 48 KB of operands and the producers write 48 KB,
+// against 128 B/clk; with A's 16 KB of generic stores left out (wrong results, timing only) the kernel ran in 93
+// instead of 115 us, with A's operand reads left out as well in 88.  But the A ring takes 128 of the 512
+// tensor-memory columns, so the two accumulators shrink to 192 tokens, every weight tile is unpacked for a
+// third more token tiles, and a K block through tcgen05.st does not fill faster than one through st.shared
+// (0.46 vs 0.55 us): 129 us against 112.  With one 256-column accumulator the epilogue (8 us per tile, all
+// CTAs writing at once) is exposed: 145 us.
+constexpr bool A_IN_TMEM = A_IN_TMEM_ != 0;
 constexpr int TILE_M = 128;     // out-features per tile (MMA M, tensor-memory lanes)
-constexpr int TILE_T = 256;     // tokens per tile (MMA N, tensor-memory columns)
+constexpr int TILE_T = A_IN_TMEM ? 192 : 256;   // tokens per tile (MMA N, tensor-memory columns)
 constexpr int KBLK = 128;       // K columns per pipeline stage = one 128-byte swizzle row of int8
 constexpr int STAGES = 4;
-constexpr int A_BYTES = TILE_M * KBLK;   // 16 KB
+constexpr int NACC = 2;                          // accumulators of TILE_T columns: the epilogue of a tile overlaps the next tile's MMAs
+constexpr int A_COL0 = NACC * TILE_T;            // first tensor-memory column of the A ring (32 columns per stage)
+static_assert(!A_IN_TMEM || A_COL0 + 32 * 4 <= 512, "tensor memory: accumulators + A ring");
+constexpr int A_BYTES = A_IN_TMEM ? 0 : TILE_M * KBLK;   // shared-memory bytes of a stage's A tile (16 KB)
 constexpr int B_BYTES = TILE_T * KBLK;   // 32 KB
-constexpr int UNPACK_WARPS = 8;           // two threads per weight row
-constexpr int THREADS = (2 + UNPACK_WARPS + 4) * 32;   // warp 0 TMA, warp 1 MMA, warps 2-9 unpack, warps 10-13 epilogue
+constexpr int UNPACK_WARPS = 8;           // warps that fill one stage: two threads per weight row
+#ifndef UNPACK_GROUPS_
+#define UNPACK_GROUPS_ 1
+#endif
+constexpr int UNPACK_GROUPS = UNPACK_GROUPS_;   // group g fills the K blocks kb = g (mod UNPACK_GROUPS); a second group
+                                                // measured no faster (115 vs 112 us): the fill is not latency-bound
+// warp 0 TMA, warp 1 MMA, then the unpack warps, then 4 epilogue warps (their index mod 4 is their lane quarter)
+constexpr int THREADS = (2 + UNPACK_WARPS * UNPACK_GROUPS + 4) * 32;
+static_assert(STAGES % UNPACK_GROUPS == 0, "a stage always belongs to the same group");
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 static __device__ int g_prefill_error = 0;
@@ -122,6 +145,15 @@ __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(IDESC), "r"(accumulate)
       : "memory");
 }
+// the same with operand A in tensor memory (lane = row, 8 columns = 32 int8 along K)
+__device__ __forceinline__ void umma_i8_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(IDESC), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
@@ -202,9 +234,9 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
       uint32_t it = 0, nt = 0;
       PP_T(pstart);
       for (int tile = blockIdx.x; tile < ntiles && !*abort_flag; tile += gridDim.x, ++nt) {
-        const int buf = nt & 1;
+        const int buf = nt % NACC;
         PP_T(p0);
-        bool ok = mbar_wait(&bars->tmem_empty[buf], ((nt >> 1) & 1u) ^ 1u, abort_flag);
+        bool ok = mbar_wait(&bars->tmem_empty[buf], ((nt / NACC) & 1u) ^ 1u, abort_flag);
         PP_T(p1);
         PP_ADD(0, p0, p1);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -224,8 +256,12 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
           const uint64_t adesc = make_desc(smem_u32(tileA + s * A_BYTES));
           const uint64_t bdesc = make_desc(smem_u32(tileB + s * B_BYTES));
 #pragma unroll
-          for (int k4 = 0; k4 < KBLK / 32; ++k4)   // 32 bytes further along K: +2 in the address field
-            umma_i8(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, (kb > 0 || k4 > 0) ? 1u : 0u);
+          for (int k4 = 0; k4 < KBLK / 32; ++k4) {  // 32 bytes further along K: +2 in the address field, +8 columns
+            if (A_IN_TMEM)
+              umma_i8_ta(d_tmem, tmem_base + A_COL0 + s * 32 + 8 * k4, bdesc + 2 * k4, (kb > 0 || k4 > 0) ? 1u : 0u);
+            else
+              umma_i8(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, (kb > 0 || k4 > 0) ? 1u : 0u);
+          }
           umma_commit(&bars->empty[s]);            // stage reusable once these MMAs have read it
           PP_T(q3);
           PP_ADD(3, q2, q3);
@@ -240,11 +276,15 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
       PP_T(pend);
       PP_ADD(4, pstart, pend);
     }
-  } else if (warp < 2 + UNPACK_WARPS) {
+  } else if (warp < 2 + UNPACK_WARPS * UNPACK_GROUPS) {
     // ------------------------------------------------------------ unpackers: weight rows (operand A)
-    const int u = threadIdx.x - 64;                // 0..255: row u/2 of the tile, half u%2 of its 128 columns
-    const int r = u >> 1, hf = u & 1;
-    uint32_t it = 0;
+    const int grp = (threadIdx.x - 64) / (UNPACK_WARPS * 32);
+    const int u = (threadIdx.x - 64) % (UNPACK_WARPS * 32);   // 0..255: row u/2 of the tile, half u%2 of its 128 columns
+    // Through tensor memory a warp can only write the 32 lanes of its quarter (warp index mod 4): lane = row
+    // within the quarter, and the two warps of a group that share a quarter take one half of the K block each.
+    const int r = A_IN_TMEM ? (warp & 3) * 32 + lane : u >> 1;
+    const int hf = A_IN_TMEM ? (u >> 7) : (u & 1);
+    uint32_t it0 = 0;                              // pipeline index of the tile's K block 0 (nkb is even)
     for (int tile = blockIdx.x; tile < ntiles && !*abort_flag; tile += gridDim.x) {
       const int m = (tile % a.tiles_m) * TILE_M + r;
       const bool row_ok = m < a.M;
@@ -252,26 +292,55 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
       const uint8_t* rowp = a.packed + i2s_row_chunk_offset(row_ok ? m : 0, 0, a.kp) + hf * 16;
       // packed words of K blocks kb .. kb+PF-1 are kept in flight: an L2 round trip is longer than one block
       constexpr int PF = 4;
+      constexpr int G = UNPACK_GROUPS;
       const uint4 zero_w = make_uint4(0x55555555u, 0x55555555u, 0x55555555u, 0x55555555u);   // code 1 = weight 0
+      auto fetch = [&](int kb) {
+        return (row_ok && kb < a.nkb)
+                   ? __ldg(reinterpret_cast<const uint4*>(rowp + (int64_t)(kb >> 1) * 1024 + (kb & 1) * 32))
+                   : zero_w;
+      };
       uint4 nx[PF];
 #pragma unroll
-      for (int p = 0; p < PF; ++p)
-        nx[p] = (row_ok && p < a.nkb) ? __ldg(reinterpret_cast<const uint4*>(rowp + (int64_t)(p >> 1) * 1024 + (p & 1) * 32))
-                                      : zero_w;
+      for (int p = 0; p < PF; ++p) nx[p] = fetch(grp + p * G);
       bool ok = true;
-      for (int kb = 0; kb < a.nkb; ++kb, ++it) {
+      for (int kb = grp; kb < a.nkb; kb += G) {
+        const uint32_t it = it0 + (uint32_t)kb;
         const uint4 cw = nx[0];
 #pragma unroll
         for (int p = 0; p + 1 < PF; ++p) nx[p] = nx[p + 1];
-        nx[PF - 1] = (row_ok && kb + PF < a.nkb)
-                         ? __ldg(reinterpret_cast<const uint4*>(rowp + (int64_t)((kb + PF) >> 1) * 1024 + ((kb + PF) & 1) * 32))
-                         : zero_w;
+        nx[PF - 1] = fetch(kb + PF * G);
         const int s = it % STAGES;
         if (!mbar_wait(&bars->empty[s], ((it / STAGES) & 1u) ^ 1u, abort_flag)) {
           ok = false;
           break;
         }
         const uint32_t w[4] = {cw.x, cw.y, cw.z, cw.w};
+        if (A_IN_TMEM) {
+          // 64 int8 of the row in K order = 16 tensor-memory columns: chunk c4 of 16 columns takes words
+          // 2*(c4/2), 2*(c4/2)+1 of the 16 packed bytes, slots 2h, 2h+1 (h = c4 % 2)
+          uint32_t o[16];
+#pragma unroll
+          for (int c4 = 0; c4 < 4; ++c4) {
+            const uint32_t w0 = w[2 * (c4 >> 1)], w1 = w[2 * (c4 >> 1) + 1];
+            const int h = c4 & 1;
+            o[4 * c4 + 0] = slot_s8(w0, 2 * h);
+            o[4 * c4 + 1] = slot_s8(w1, 2 * h);
+            o[4 * c4 + 2] = slot_s8(w0, 2 * h + 1);
+            o[4 * c4 + 3] = slot_s8(w1, 2 * h + 1);
+          }
+          const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + A_COL0 + s * 32 + hf * 16;
+          asm volatile(
+              "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, "
+              "%14, %15, %16};"
+              ::"r"(taddr), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]),
+                "r"(o[8]), "r"(o[9]), "r"(o[10]), "r"(o[11]), "r"(o[12]), "r"(o[13]), "r"(o[14]), "r"(o[15])
+              : "memory");
+          asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars->full_a[s]);
+          continue;
+        }
         uint8_t* rowA = tileA + s * A_BYTES + (r >> 3) * 1024 + (r & 7) * 128;
 #pragma unroll
         for (int c4 = 0; c4 < 4; ++c4) {
@@ -293,13 +362,14 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
         bars->abort_flag = 1;
         break;
       }
+      it0 += (uint32_t)a.nkb;
     }
   } else {
     // ------------------------------------------------------------ epilogue
     const int quarter = warp & 3;                  // tensor-memory lanes 32*quarter .. 32*quarter+31
     uint32_t nt = 0;
     for (int tile = blockIdx.x; tile < ntiles && !*abort_flag; tile += gridDim.x, ++nt) {
-      const int buf = nt & 1;
+      const int buf = nt % NACC;
       const int m = (tile % a.tiles_m) * TILE_M + quarter * 32 + lane;
       const int t0 = (tile / a.tiles_m) * TILE_T;
       // this tile's per-token factors act_scale[t] * w_scale, one copy per epilogue warp, fetched while the
@@ -310,7 +380,7 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
       for (int i = lane; i < TILE_T; i += 32)
         my_scale[i] = (t0 + i < a.T) ? __fmul_rn(__ldg(a.act_scale + t0 + i), a.w_scale) : 0.0f;
       __syncwarp();
-      if (!mbar_wait(&bars->tmem_full[buf], (nt >> 1) & 1u, abort_flag)) {
+      if (!mbar_wait(&bars->tmem_full[buf], (nt / NACC) & 1u, abort_flag)) {
         atomicExch(&g_prefill_error, BITNET_ERR_TIMEOUT);
         bars->abort_flag = 1;
         break;
