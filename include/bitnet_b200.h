@@ -175,6 +175,9 @@ int bitnet_linear_host(bitnet_fmt_t fmt, const void* packed, float w_scale, int6
  *   - items[n]: plain structs in host memory, read during the call only.
  *   - x_host / y_host should be pinned.  The device buffers of different items must not overlap
  *     (uploads run ahead of the kernels); the workspace may be shared (the kernels are serial).
+ *     Neighbouring items of a group whose x_host and x_dev (or y_dev and y_host) both start where the
+ *     previous item's end are copied with one call: keeping the activations of a batch in one pinned
+ *     block and one device block, in item order, saves a driver call per item and direction.
  *   - The internal streams and events are created on first use per device and kept.
  *   - Errors: BITNET_ERR_INVALID_ARG for a null or malformed item (nothing of that item or later ones
  *     is queued); otherwise the status of the first failing call.

@@ -330,10 +330,21 @@ extern "C" int bitnet_linear_host_batch(const bitnet_host_linear_t* items, int64
   const int64_t ngroups = (n + GROUP - 1) / GROUP;
   auto upload_group = [&](int64_t g) -> cudaError_t {
     const int64_t lo = g * GROUP, hi = (lo + GROUP < n) ? lo + GROUP : n;
-    for (int64_t i = lo; i < hi; ++i) {
-      const bitnet_host_linear_t& d = items[i];
-      cudaError_t er = cudaMemcpyAsync(d.x_dev, d.x_host, (size_t)d.T * d.K * sizeof(float), cudaMemcpyHostToDevice, p->up);
+    // neighbouring items whose host and device buffers both continue where the previous item's end travel as
+    // one copy (a caller that keeps its activations in one pinned block gets one copy per group)
+    for (int64_t i = lo; i < hi;) {
+      const char* src = reinterpret_cast<const char*>(items[i].x_host);
+      char* dst = reinterpret_cast<char*>(items[i].x_dev);
+      size_t bytes = (size_t)items[i].T * items[i].K * sizeof(float);
+      int64_t j = i + 1;
+      while (j < hi && reinterpret_cast<const char*>(items[j].x_host) == src + bytes &&
+             reinterpret_cast<char*>(items[j].x_dev) == dst + bytes) {
+        bytes += (size_t)items[j].T * items[j].K * sizeof(float);
+        ++j;
+      }
+      cudaError_t er = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, p->up);
       if (er != cudaSuccess) return er;
+      i = j;
     }
     return cudaEventRecord(p->ev[2 * g], p->up);
   };
@@ -359,9 +370,19 @@ extern "C" int bitnet_linear_host_batch(const bitnet_host_linear_t* items, int64
     }
     BN_TRY(cudaEventRecord(p->ev[2 * g + 1], st));
     BN_TRY(cudaStreamWaitEvent(p->down, p->ev[2 * g + 1], 0));
-    for (int64_t i = lo; i < hi; ++i)
-      BN_TRY(cudaMemcpyAsync(items[i].y_host, items[i].y_dev, (size_t)items[i].T * items[i].M * sizeof(float),
-                             cudaMemcpyDeviceToHost, p->down));
+    for (int64_t i = lo; i < hi;) {
+      char* dst = reinterpret_cast<char*>(items[i].y_host);
+      const char* src = reinterpret_cast<const char*>(items[i].y_dev);
+      size_t bytes = (size_t)items[i].T * items[i].M * sizeof(float);
+      int64_t j = i + 1;
+      while (j < hi && reinterpret_cast<char*>(items[j].y_host) == dst + bytes &&
+             reinterpret_cast<const char*>(items[j].y_dev) == src + bytes) {
+        bytes += (size_t)items[j].T * items[j].M * sizeof(float);
+        ++j;
+      }
+      BN_TRY(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, p->down));
+      i = j;
+    }
   }
   BN_TRY(cudaEventRecord(e_out, p->down));
   BN_TRY(cudaStreamWaitEvent(st, e_out, 0));

@@ -502,3 +502,47 @@ def test_linear_host_batch_matches_single_calls():
         for it, ref in zip(items, refs):
             assert torch.equal(it["y_host"], ref), (rep, it["fmt"], it["M"], it["K"])
     assert bn.bitnet_device_status() == 0
+
+
+@pytest.mark.gpu
+def test_linear_host_batch_merges_neighbouring_buffers():
+    """Items whose host and device buffers continue one another (one pinned block, one device block) travel as
+    one copy per group; items 3 and 4 break the chain on the host side only, item 11 has 24 tokens (mid-batch
+    kernel).  Same results as item-by-item calls, nothing outside the buffers touched."""
+    specs = [(256, 1024, 1)] * 3 + [(512, 2048, 2)] * 8 + [(320, 4096, 24)]
+    nx = sum(T * K for M, K, T in specs)
+    ny = sum(T * M for M, K, T in specs)
+    xh_all = torch.empty(nx + 64, dtype=torch.float32).pin_memory()
+    yh_all = torch.full((ny + 64,), -7.0, dtype=torch.float32).pin_memory()
+    xd_all = torch.empty(nx, dtype=torch.float32, device="cuda")
+    yd_all = torch.empty(ny, dtype=torch.float32, device="cuda")
+    items, refs, keep = [], [], []
+    xo = xd_o = yo = 0
+    for n, (M, K, T) in enumerate(specs):
+        w = synth.ternary(60 + n, 0, M, K, 1 / 3, 1 / 3)
+        x = synth.normal(60 + n, 1, T, K)
+        blob = bn.pack("i2s", w.cuda())
+        gap = 32 if n in (3, 4) else 0                     # a hole in the host block: no merging across it
+        xh = xh_all[xo + gap: xo + gap + T * K].view(T, K)
+        xh.copy_(x)
+        yh = yh_all[yo: yo + T * M].view(T, M)
+        xd = xd_all[xd_o: xd_o + T * K].view(T, K)
+        yd = yd_all[yo: yo + T * M].view(T, M)
+        xo += T * K + gap
+        xd_o += T * K
+        yo += T * M
+        qd = torch.empty((T, K), dtype=torch.int8, device="cuda")
+        sd = torch.empty(T, dtype=torch.float32, device="cuda")
+        ws = bn.new_workspace("i2s", T, M, K)
+        items.append(dict(fmt="i2s", packed=blob, w_scale=0.5, M=M, K=K, x_host=xh, y_host=yh, x_dev=xd, q_dev=qd,
+                          scale_dev=sd, y_dev=yd, workspace=ws))
+        keep.append((blob, qd, sd, ws))
+        y, _, _, _ = bn.bitnet_linear("i2s", blob, 0.5, M, K, x.cuda())
+        refs.append(y.cpu())
+    assert xo <= nx + 64
+    bn.bitnet_linear_host_batch(bn.make_host_batch(items))
+    torch.cuda.current_stream().synchronize()
+    for it, ref in zip(items, refs):
+        assert torch.equal(it["y_host"], ref)
+    assert bool((yh_all[ny:] == -7.0).all())
+    assert bn.bitnet_device_status() == 0
