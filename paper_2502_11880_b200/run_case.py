@@ -4,8 +4,9 @@ small, self-contained workload the ncu captures under profiles/ are taken on).
     python -m paper_2502_11880_b200.run_case FMT K M T [N] [--two-kernel]
 
 FMT = i2s | tl1 | tl2.  Weights and activations are seeded synthetic tensors; N launches (default 6) over
-three distinct copies of the packed blob.  T <= 8 runs the decode path (one fused kernel for I2_S unless
---two-kernel), larger T the prefill path.
+three distinct copies of the packed blob.  T <= 8 runs the decode path through bitnet_linear (one fused kernel
+for I2_S up to 5 tokens unless --two-kernel); larger T runs the quantiser and bitnet_mpgemm: the mid-batch
+kernel up to 64 tokens, the prefill kernel beyond.
 """
 import sys
 
