@@ -4,9 +4,9 @@
 // m16n8k32, u8 x s8), not HBM, become the limit from about 24 tokens on.  Differences to the decode kernel:
 //   * NT = ceil(T / 8) token tiles per weight fragment; the 2-bit fields are shifted down to plain codes so that
 //     all four slots of a word add into one accumulator per token tile (a decode kernel keeps one per slot);
-//   * the B fragments (activations) of a token tile are read from shared memory once for RU = 2 adjacent 16-row
-//     units: at one unit per load the shared-memory pipe, which delivers the 256 B of B per MMA in exactly the
-//     two cycles the MMA takes, would bind before the tensor pipe does;
+//   * up to two token tiles, the B fragments (activations) of a tile are read from shared memory once for
+//     RU = 2 adjacent 16-row units (one MMA needs 256 B of B, exactly what the shared-memory pipe delivers in the
+//     MMA's two cycles); from three tiles on, one unit per step with the cheaper field extraction measured faster;
 //   * T x K codes do not fit in shared memory, so K is cut into NS slices; a CTA stages the codes of one slice
 //     and runs the (slice, unit pair) items of a contiguous range, one item per warp at a time, each warp
 //     streaming its item's weights through a private cp.async ring.  With NS > 1 the int32 partial sums meet in
@@ -344,20 +344,25 @@ __global__ void __launch_bounds__(256) finish_mid_kernel(int32_t* __restrict__ w
   }
 }
 
-int env_int(const char* name, int dflt) {
-  const char* v = getenv(name);
-  return (v && *v) ? atoi(v) : dflt;
-}
 
 // bytes of the [T][M] sums at the head of the workspace; one arrival counter per CTA of a slice follows
 constexpr size_t MID_WS_COUNTERS = 1024;
 inline size_t mid_ws_sums(int T, int64_t M) { return (((size_t)T * (size_t)M * 4) + 15) & ~(size_t)15; }
 
+int env_int(const char* name, int dflt) {
+  const char* v = getenv(name);
+  return (v && *v) ? atoi(v) : dflt;
+}
+
 struct MidCfg { int NT, RU, DEPTH; };
+// Measured on the 100B shapes (us per layer, RU 2 vs 1): NT = 2: 91 vs 91 (ring of 8) or 106 (ring of 4); NT = 3:
+// 117 vs 114; NT = 4: 145 vs 132 (ring of 8): from three token tiles on, one unit per step with the cheaper
+// two-set field extraction wins over sharing the B loads between two units.
 inline MidCfg mid_cfg(int T) {
   const int NT = (T + 7) / 8;
   if (NT <= 2) return {NT, 2, 4};
-  if (NT <= 4) return {NT, 2, 3};
+  if (NT == 3) return {NT, 1, 4};
+  if (NT == 4) return {NT, 1, 8};
   return {NT, 1, 4};
 }
 
@@ -467,8 +472,8 @@ int launch_gemv_i2s_mid(const uint8_t* packed, float w_scale, int64_t M, int64_t
   switch (p.c.NT) {
     case 1: rc = launch_mid<1, 2, 4, 4>(a, p, st); break;
     case 2: rc = launch_mid<2, 2, 4, 2>(a, p, st); break;
-    case 3: rc = launch_mid<3, 2, 3, 1>(a, p, st); break;
-    case 4: rc = launch_mid<4, 2, 3, 1>(a, p, st); break;
+    case 3: rc = launch_mid<3, 1, 4, 2>(a, p, st); break;
+    case 4: rc = launch_mid<4, 1, 8, 2>(a, p, st); break;
     case 5: rc = launch_mid<5, 1, 4, 1>(a, p, st); break;
     case 6: rc = launch_mid<6, 1, 4, 1>(a, p, st); break;
     case 7: rc = launch_mid<7, 1, 4, 1>(a, p, st); break;
