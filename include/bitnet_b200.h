@@ -121,15 +121,17 @@ int bitnet_pack_tl(bitnet_fmt_t fmt, const int8_t* w, int64_t M, int64_t K, int 
  *   q[T][K]  int8, act_scale[T] fp32 from bitnet_quant_act;
  *   y[T][M]  fp32 out; acc_out[T][M] int32 out, nullable (raw accumulators);
  *   workspace  bitnet_mpgemm_workspace_bytes(fmt,T,M,K) bytes (may be NULL when that is 0: I2_S with
- *              T <= 8 needs none except for extreme shapes; I2_S with 9 <= T <= 64 keeps the T*M int32
- *              sums of its K-slices there; TL keeps its lookup tables and split-K sums there).
+ *              T <= 8 needs none except for extreme shapes; I2_S with 9 <= T <= 64, and with more tokens
+ *              when the output has fewer 128 x 256 tiles than three quarters of the SMs, keeps the T*M
+ *              int32 sums of its K-slices there; TL keeps its lookup tables and split-K sums there).
  *              It must have been zeroed once with bitnet_workspace_init and its head (the sums) is
  *              left zeroed by every completed call; two calls sharing a workspace must not overlap
  *              on the GPU, and a workspace last used by a TL call is initialised again before an
  *              I2_S call uses it.
  * I2_S: T <= 8 runs the decode GEMV kernel; 9 <= T <= 64 a scan of the weights on mma.sync tensor-core
  * tiles over K-slices followed by a rescale kernel (when the workspace is missing or too small, the
- * prefill kernel takes the call instead); larger T the tcgen05 prefill kernel.  TL runs its GEMV kernel
+ * prefill kernel takes the call instead); larger T the tcgen05 prefill kernel (whole tiles per CTA; parts
+ * of a tile's K per CTA when there are few tiles and the workspace is there).  TL runs its GEMV kernel
  * over groups of 8 tokens.  The integer results do not depend on which kernel ran.
  */
 size_t bitnet_mpgemm_workspace_bytes(bitnet_fmt_t fmt, int64_t T, int64_t M, int64_t K);

@@ -183,7 +183,7 @@ static bool mid_takes(int64_t T, int64_t M, int64_t K, const void* workspace, si
 size_t bitnet_mpgemm_workspace_bytes(bitnet_fmt_t fmt, int64_t T, int64_t M, int64_t K) {
   if (T < 1 || M < 1 || K < 1) return 0;
   if (fmt == BITNET_FMT_I2S) {
-    size_t n = T > 8 ? 0 : gemv_i2s_workspace_bytes(T, M, K);
+    size_t n = T > 8 ? gemm_i2s_prefill_workspace_bytes(T, M, K) : gemv_i2s_workspace_bytes(T, M, K);
     if (use_mid(T, M, K)) {
       const size_t m = gemv_i2s_mid_workspace_bytes((int)T, M, K);
       if (m > n) n = m;
@@ -216,7 +216,9 @@ int bitnet_mpgemm(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
     if (mid_takes(T, M, K, workspace, workspace_bytes))
       return launch_gemv_i2s_mid((const uint8_t*)packed, w_scale, M, K, q, act_scale, (int)T, y, acc_out, workspace,
                                  workspace_bytes, st);
-    if (T > 8) return launch_gemm_i2s_prefill((const uint8_t*)packed, w_scale, M, K, q, act_scale, T, y, acc_out, st);
+    if (T > 8)
+      return launch_gemm_i2s_prefill((const uint8_t*)packed, w_scale, M, K, q, act_scale, T, y, acc_out, workspace,
+                                     workspace_bytes, st);
     return launch_gemv_i2s((const uint8_t*)packed, w_scale, M, K, q, act_scale, (int)T, y, acc_out, workspace,
                            workspace_bytes, st);
   }

@@ -108,9 +108,15 @@ int launch_gemv_tl(int fmt, const uint8_t* packed, float w_scale, int64_t M, int
 int launch_tl_build_lut(int fmt, const int8_t* q_row, int64_t K, const TlGeom& g, int16_t* lut,
                         cudaStream_t st);
 
-// Prefill GEMM (I2_S, int8 tensor cores).
+// y = float(sums) * (act_scale[t] * w_scale) over a [T][M] int32 array of finished sums, which is left zeroed.
+int launch_rescale_sums(int32_t* sums, const float* act_scale, float w_scale, int64_t T, int64_t M, float* y,
+                        int32_t* acc_out, cudaStream_t st);
+
+// Prefill GEMM (I2_S, int8 tensor cores).  With few output tiles for the SMs it cuts every tile's K into parts
+// that meet in `ws` (zeroed [T][M] int32, gemm_i2s_prefill_workspace_bytes; without it: whole tiles only).
+size_t gemm_i2s_prefill_workspace_bytes(int64_t T, int64_t M, int64_t K);
 int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const int8_t* q,
-                            const float* act_scale, int64_t T, float* y, int32_t* acc_out,
+                            const float* act_scale, int64_t T, float* y, int32_t* acc_out, void* ws, size_t ws_bytes,
                             cudaStream_t st);
 
 int gemm_prefill_status(int* out);

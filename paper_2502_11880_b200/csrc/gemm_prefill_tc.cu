@@ -85,6 +85,8 @@ struct PrefillArgs {
   int32_t* acc_out;
   int tiles_m, tiles_t, nkb;
   int tma_store;         // y leaves through shared memory and bulk tensor stores (needs M % 4 == 0, no acc_out)
+  int ksplit;            // > 1: an item is 1/ksplit of a tile's K blocks; partial sums go to ws with integer atomics
+  int32_t* ws;           // [T][M] sums, zero on entry (ksplit > 1); a second kernel rescales them
 };
 
 struct __align__(8) Barriers {
@@ -180,6 +182,10 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ntiles = a.tiles_m * a.tiles_t;
+  // Work items: tile `item % ntiles`, K blocks [kb_lo, kb_hi) = part `item / ntiles` of ksplit (even bounds).
+  const int nitems = ntiles * a.ksplit;
+  auto kb_lo_of = [&](int item) { return 2 * (int)((int64_t)(item / ntiles) * (a.nkb / 2) / a.ksplit); };
+  auto kb_hi_of = [&](int item) { return 2 * (int)((int64_t)(item / ntiles + 1) * (a.nkb / 2) / a.ksplit); };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -210,9 +216,10 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
     // ------------------------------------------------------------ TMA producer: activation tiles (operand B)
     if (lane == 0) {
       uint32_t it = 0;
-      for (int tile = blockIdx.x; tile < ntiles && !*abort_flag; tile += gridDim.x) {
+      for (int item = blockIdx.x; item < nitems && !*abort_flag; item += gridDim.x) {
+        const int tile = item % ntiles;
         const int t0 = (tile / a.tiles_m) * TILE_T;
-        for (int kb = 0; kb < a.nkb; ++kb, ++it) {
+        for (int kb = kb_lo_of(item), kb_end = kb_hi_of(item); kb < kb_end; ++kb, ++it) {
           const int s = it % STAGES;
           if (!mbar_wait(&bars->empty[s], ((it / STAGES) & 1u) ^ 1u, abort_flag)) {
             atomicExch(&g_prefill_error, BITNET_ERR_TIMEOUT);
@@ -233,15 +240,16 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
     if (lane == 0) {
       uint32_t it = 0, nt = 0;
       PP_T(pstart);
-      for (int tile = blockIdx.x; tile < ntiles && !*abort_flag; tile += gridDim.x, ++nt) {
+      for (int item = blockIdx.x; item < nitems && !*abort_flag; item += gridDim.x, ++nt) {
         const int buf = nt % NACC;
+        const int kb_lo = kb_lo_of(item), kb_hi = kb_hi_of(item);
         PP_T(p0);
         bool ok = mbar_wait(&bars->tmem_empty[buf], ((nt / NACC) & 1u) ^ 1u, abort_flag);
         PP_T(p1);
         PP_ADD(0, p0, p1);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t d_tmem = tmem_base + buf * TILE_T;
-        for (int kb = 0; ok && kb < a.nkb; ++kb, ++it) {
+        for (int kb = kb_lo; ok && kb < kb_hi; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t par = (it / STAGES) & 1u;
           PP_T(q0);
@@ -258,9 +266,9 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
 #pragma unroll
           for (int k4 = 0; k4 < KBLK / 32; ++k4) {  // 32 bytes further along K: +2 in the address field, +8 columns
             if (A_IN_TMEM)
-              umma_i8_ta(d_tmem, tmem_base + A_COL0 + s * 32 + 8 * k4, bdesc + 2 * k4, (kb > 0 || k4 > 0) ? 1u : 0u);
+              umma_i8_ta(d_tmem, tmem_base + A_COL0 + s * 32 + 8 * k4, bdesc + 2 * k4, (kb > kb_lo || k4 > 0) ? 1u : 0u);
             else
-              umma_i8(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, (kb > 0 || k4 > 0) ? 1u : 0u);
+              umma_i8(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, (kb > kb_lo || k4 > 0) ? 1u : 0u);
           }
           umma_commit(&bars->empty[s]);            // stage reusable once these MMAs have read it
           PP_T(q3);
@@ -285,7 +293,9 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
     const int r = A_IN_TMEM ? (warp & 3) * 32 + lane : u >> 1;
     const int hf = A_IN_TMEM ? (u >> 7) : (u & 1);
     uint32_t it0 = 0;                              // pipeline index of the tile's K block 0 (nkb is even)
-    for (int tile = blockIdx.x; tile < ntiles && !*abort_flag; tile += gridDim.x) {
+    for (int item = blockIdx.x; item < nitems && !*abort_flag; item += gridDim.x) {
+      const int tile = item % ntiles;
+      const int kb_lo = kb_lo_of(item), kb_hi = kb_hi_of(item);
       const int m = (tile % a.tiles_m) * TILE_M + r;
       const bool row_ok = m < a.M;
       // K block kb = half kb&1 of chunk kb/2: 32 bytes of the row, of which this thread takes 16
@@ -295,16 +305,16 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
       constexpr int G = UNPACK_GROUPS;
       const uint4 zero_w = make_uint4(0x55555555u, 0x55555555u, 0x55555555u, 0x55555555u);   // code 1 = weight 0
       auto fetch = [&](int kb) {
-        return (row_ok && kb < a.nkb)
+        return (row_ok && kb < kb_hi)
                    ? __ldg(reinterpret_cast<const uint4*>(rowp + (int64_t)(kb >> 1) * 1024 + (kb & 1) * 32))
                    : zero_w;
       };
       uint4 nx[PF];
 #pragma unroll
-      for (int p = 0; p < PF; ++p) nx[p] = fetch(grp + p * G);
+      for (int p = 0; p < PF; ++p) nx[p] = fetch(kb_lo + grp + p * G);
       bool ok = true;
-      for (int kb = grp; kb < a.nkb; kb += G) {
-        const uint32_t it = it0 + (uint32_t)kb;
+      for (int kb = kb_lo + grp; kb < kb_hi; kb += G) {
+        const uint32_t it = it0 + (uint32_t)(kb - kb_lo);
         const uint4 cw = nx[0];
 #pragma unroll
         for (int p = 0; p + 1 < PF; ++p) nx[p] = nx[p + 1];
@@ -362,13 +372,14 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
         bars->abort_flag = 1;
         break;
       }
-      it0 += (uint32_t)a.nkb;
+      it0 += (uint32_t)(kb_hi - kb_lo);
     }
   } else {
     // ------------------------------------------------------------ epilogue
     const int quarter = warp & 3;                  // tensor-memory lanes 32*quarter .. 32*quarter+31
     uint32_t nt = 0;
-    for (int tile = blockIdx.x; tile < ntiles && !*abort_flag; tile += gridDim.x, ++nt) {
+    for (int item = blockIdx.x; item < nitems && !*abort_flag; item += gridDim.x, ++nt) {
+      const int tile = item % ntiles;
       const int buf = nt % NACC;
       const int m = (tile % a.tiles_m) * TILE_M + quarter * 32 + lane;
       const int t0 = (tile / a.tiles_m) * TILE_T;
@@ -416,6 +427,15 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
                            "r"(smem_u32(&ep_stage[quarter][0][0]))
                          : "memory");
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          }
+        } else if (a.ksplit > 1) {
+          // part of a tile's K: add the raw sums (integers: any order gives the same); rescaled afterwards
+          if (m < a.M) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int t = t0 + c0 + j;
+              if (t < a.T) atomicAdd(a.ws + (int64_t)t * a.M + m, (int)v[j]);
+            }
           }
         } else if (m < a.M) {
 #pragma unroll
@@ -470,13 +490,35 @@ static bool no_tma_store() {
   return off;
 }
 
+// Parts per tile's K: with fewer tiles than SMs (short prompts, small layers) whole tiles leave SMs idle and
+// the time is that of one tile's K blocks; parts of at least 8 K blocks fill the machine instead.
+static int prefill_ksplit(int64_t T, int64_t M, int64_t K) {
+  static const int forced = [] { const char* e = getenv("BITNET_PREFILL_KSPLIT"); return e ? atoi(e) : 0; }();
+  const int64_t ntiles = ceil_div(M, TILE_M) * ceil_div(T, TILE_T);
+  const int64_t nkb = i2s_kp(K) / KBLK;
+  const int sms = dev_info().sm_count;
+  int64_t ks = 1;
+  if (forced > 0) ks = forced;
+  else if (ntiles * 4 <= sms * 3) ks = sms / ntiles;          // at most three quarters of the SMs would work
+  // (with more tiles than that the atomics and the rescale pass over T x M cost more than the idle SMs)
+  if (ks > nkb / 8) ks = nkb / 8;
+  return ks < 1 ? 1 : (int)ks;
+}
+
+size_t gemm_i2s_prefill_workspace_bytes(int64_t T, int64_t M, int64_t K) {
+  return prefill_ksplit(T, M, K) > 1 ? (size_t)T * (size_t)M * 4 : 0;
+}
+
 int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const int8_t* q,
-                            const float* act_scale, int64_t T, float* y, int32_t* acc_out, cudaStream_t st) {
+                            const float* act_scale, int64_t T, float* y, int32_t* acc_out, void* ws, size_t ws_bytes,
+                            cudaStream_t st) {
   static const bool force_simt = [] {
     const char* e = getenv("BITNET_PREFILL");
     return e && strcmp(e, "simt") == 0;
   }();
   if (force_simt) return launch_gemm_i2s_simt(packed, w_scale, M, K, q, act_scale, T, y, acc_out, st);
+  int ksplit = prefill_ksplit(T, M, K);
+  if (ksplit > 1 && (!ws || ws_bytes < (size_t)T * (size_t)M * 4)) ksplit = 1;
   EncodeTiledFn enc = encode_fn();
   if (!enc) return note_cuda_error(cudaErrorNotSupported);
   CUtensorMap qmap;
@@ -490,7 +532,7 @@ int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int
   if (r != CUDA_SUCCESS) return note_cuda_error(cudaErrorInvalidValue);
 
   // y[T][M] fp32 as a tensor of 32 x 32 boxes for the epilogue's bulk stores
-  const bool tma_store = acc_out == nullptr && (M % 4) == 0 && !no_tma_store();
+  const bool tma_store = ksplit == 1 && acc_out == nullptr && (M % 4) == 0 && !no_tma_store();
   CUtensorMap ymap = qmap;
   if (tma_store) {
     const cuuint64_t ydim[2] = {(cuuint64_t)M, (cuuint64_t)T};
@@ -503,6 +545,8 @@ int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int
 
   PrefillArgs a;
   a.tma_store = tma_store ? 1 : 0;
+  a.ksplit = ksplit;
+  a.ws = reinterpret_cast<int32_t*>(ws);
   a.packed = packed;
   a.kp = i2s_kp(K);
   a.M = (int)M;
@@ -525,10 +569,12 @@ int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int
     attr_set[dev & 63] = true;
   }
   int grid = dev_info().sm_count;
-  const int ntiles = a.tiles_m * a.tiles_t;
-  if (grid > ntiles) grid = ntiles;
+  const int nitems = a.tiles_m * a.tiles_t * ksplit;
+  if (grid > nitems) grid = nitems;
   gemm_i2s_tc_kernel<<<grid, THREADS, smem, st>>>(qmap, ymap, a);
-  return check_launch();
+  int rc = check_launch();
+  if (rc || ksplit == 1) return rc;
+  return launch_rescale_sums(a.ws, act_scale, w_scale, T, M, y, acc_out, st);
 }
 
 #ifdef BITNET_PROFILE_PREFILL

@@ -432,6 +432,24 @@ int launch_mid(const MArgs& a, const MidPlan& p, cudaStream_t st) {
 
 }  // namespace
 
+// y = float(sums) * (act_scale[t] * w_scale) over a [T][M] int32 array, which is left zeroed.
+int launch_rescale_sums(int32_t* sums, const float* act_scale, float w_scale, int64_t T, int64_t M, float* y,
+                        int32_t* acc_out, cudaStream_t st) {
+  const int64_t n4 = (T * M + 3) / 4;
+  const int64_t want = (n4 + 255) / 256;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(want < 8 * 148 ? want : 8 * 148));
+  cfg.blockDim = dim3(256);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = early_start_enabled() ? 1 : 0;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, finish_mid_kernel, sums, act_scale, w_scale, (int)T, (int)M, y, acc_out);
+  return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
+}
+
 bool gemv_i2s_mid_supported(int T, int64_t M, int64_t K) {
   MidPlan p;
   return make_mid_plan(T, M, K, &p);
@@ -481,19 +499,7 @@ int launch_gemv_i2s_mid(const uint8_t* packed, float w_scale, int64_t M, int64_t
     default: return BITNET_ERR_UNSUPPORTED_SHAPE;
   }
   if (rc || p.c.NT <= FINISH_IN_KERNEL_MAX_NT) return rc;
-  const int64_t n4 = ((int64_t)T * M + 3) / 4;
-  const int64_t want = (n4 + 255) / 256;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(want < 8 * 148 ? want : 8 * 148));
-  cfg.blockDim = dim3(256);
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = early_start_enabled() ? 1 : 0;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, finish_mid_kernel, a.ws, act_scale, w_scale, T, (int)M, y, acc_out);
-  return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
+  return launch_rescale_sums(a.ws, act_scale, w_scale, T, M, y, acc_out, st);
 }
 
 }  // namespace bitnet

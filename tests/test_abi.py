@@ -55,7 +55,10 @@ def test_size_queries(L):
     # batches whose codes crowd the decode kernel, and 9 to 64 tokens: the T x M sums of the K-slices
     assert 0 <= bn.bitnet_mpgemm_workspace_bytes("i2s", 8, 1 << 20, 1 << 17) - 8 * (1 << 20) * 4 <= 4096
     assert 0 <= bn.bitnet_mpgemm_workspace_bytes("i2s", 33, 8192, 28672) - 33 * 8192 * 4 <= 4096
-    assert bn.bitnet_mpgemm_workspace_bytes("i2s", 65, 8192, 28672) == 0         # prefill kernel: none
+    # prefill kernel: none when the output tiles fill the SMs, the T x M sums when K is cut to fill them
+    assert bn.bitnet_mpgemm_workspace_bytes("i2s", 2048, 14336, 4096) == 0
+    assert bn.bitnet_mpgemm_workspace_bytes("i2s", 65, 57344, 8192) == 0
+    assert bn.bitnet_mpgemm_workspace_bytes("i2s", 65, 8192, 28672) == 65 * 8192 * 4
     assert bn.bitnet_mpgemm_workspace_bytes("tl2", 1, 8192, 28672) >= 2 * 8192 * 4
 
 

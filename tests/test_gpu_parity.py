@@ -380,6 +380,22 @@ def test_prefill_output_paths_agree():
         assert bool((guard[:4] == 12345.0).all()) and bool((guard[T + 4:] == 12345.0).all())
 
 
+def test_prefill_few_tiles_split_k():
+    """More than 64 tokens on a layer with fewer output tiles than SMs: every tile's K is cut into parts that
+    meet in the workspace (integer atomics) and a second kernel rescales; long K, ragged M and T, and the same
+    call without a workspace (whole tiles) must agree."""
+    for (M, K, T) in [(300, 8192, 70), (1000, 28672, 130), (130, 4096, 65)]:
+        w, x = tern(52, M, K), synth.normal(52, M + T, T, K)
+        assert bn.bitnet_mpgemm_workspace_bytes("i2s", T, M, K) >= T * M * 4
+        ws = bn.new_workspace("i2s", T, M, K)
+        out = check_linear("i2s", w, x, workspace=ws)
+        assert not npy(ws).any()
+        again = run_linear("i2s", w, x, workspace=ws)
+        assert torch.equal(again["acc"], out["acc"]) and torch.equal(again["y"], out["y"])
+        whole = run_linear("i2s", w, x, workspace=no_workspace())
+        assert torch.equal(whole["acc"], out["acc"]) and torch.equal(whole["y"], out["y"])
+
+
 def test_workload_prefill_sampled():
     wl = synth.CONFIGS["prefill"]
     lin = wl.linears[0]
