@@ -65,7 +65,7 @@ constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 static __device__ int g_prefill_error = 0;
 #ifdef BITNET_PROFILE_PREFILL
-__device__ long long g_pprof[8];   // MMA thread of CTA 0: [0] wait tmem_empty, [1] wait full_a, [2] wait full_b, [3] issue, [4] total
+__device__ long long g_pprof[8];   // MMA thread of CTA 0: [0] wait tmem_empty, [1] wait for the stage's operands, [2] unused, [3] issue, [4] total
 #define PP_T(v) const long long v = clock64()
 #define PP_ADD(i, x0, x1) if (blockIdx.x == 0) g_pprof[i] += (x1) - (x0)
 #else
@@ -90,7 +90,7 @@ struct PrefillArgs {
 };
 
 struct __align__(8) Barriers {
-  uint64_t full_a[STAGES], full_b[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2];
+  uint64_t full_a[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -189,8 +189,8 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(&bars->full_a[s], UNPACK_WARPS);   // one arrival per unpack warp
-      mbar_init(&bars->full_b[s], 1);      // TMA producer (+ transaction bytes)
+      // one barrier per stage for both operands: an arrival per unpack warp, one of the TMA producer (+ its bytes)
+      mbar_init(&bars->full_a[s], UNPACK_WARPS + 1);
       mbar_init(&bars->empty[s], 1);       // tcgen05.commit
     }
     for (int b = 0; b < 2; ++b) {
@@ -226,11 +226,11 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
             bars->abort_flag = 1;
             break;
           }
-          mbar_expect_tx(&bars->full_b[s], B_BYTES);
+          mbar_expect_tx(&bars->full_a[s], B_BYTES);
           asm volatile(
               "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
               ::"r"(smem_u32(tileB + s * B_BYTES)), "l"(&qmap), "r"(kb * KBLK), "r"(t0),
-              "r"(smem_u32(&bars->full_b[s]))
+              "r"(smem_u32(&bars->full_a[s]))
               : "memory");
         }
       }
@@ -253,14 +253,12 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
           const int s = it % STAGES;
           const uint32_t par = (it / STAGES) & 1u;
           PP_T(q0);
-          ok = mbar_wait(&bars->full_a[s], par, abort_flag);
+          ok = mbar_wait(&bars->full_a[s], par, abort_flag);   // weights unpacked and activations landed
           PP_T(q1);
-          ok = ok && mbar_wait(&bars->full_b[s], par, abort_flag);
           PP_T(q2);
           PP_ADD(1, q0, q1);
           PP_ADD(2, q1, q2);
           if (!ok) break;
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint64_t adesc = make_desc(smem_u32(tileA + s * A_BYTES));
           const uint64_t bdesc = make_desc(smem_u32(tileB + s * B_BYTES));
 #pragma unroll
