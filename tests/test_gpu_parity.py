@@ -480,6 +480,29 @@ def test_split_k_kernel_variant_in_a_child_process():
     assert out.returncode == 0 and "ok" in out.stdout, out.stderr[-2000:]
 
 
+def test_prefill_forced_split_and_mid_batch_off_in_child_processes():
+    """Read-once switches: BITNET_PREFILL_KSPLIT forces the number of K parts per tile (here 3 and 8, on shapes
+    with several tiles per SM round and a ragged last part), BITNET_I2S_MID_MAX_T=0 sends 9 to 64 tokens to the
+    prefill kernel.  Each must still agree with the oracle."""
+    import os
+    import subprocess
+    import sys
+    code = (
+        "import sys; sys.path.insert(0, 'tests'); import numpy as np, torch\n"
+        "from paper_2502_11880_b200 import synth\n"
+        "import paper_2502_11880_b200 as bn\n"
+        "from helpers import check_linear\n"
+        "for (M, K, T) in [(700, 5120, 70), (130, 28672, 300), (2000, 2048, 33), (64, 8192, 12)]:\n"
+        "    check_linear('i2s', synth.ternary(61, 1, M, K, 1/3, 1/3), synth.normal(61, T, T, K))\n"
+        "assert bn.bitnet_device_status() == 0\n"
+        "print('ok')\n")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    for extra in (dict(BITNET_PREFILL_KSPLIT="3"), dict(BITNET_PREFILL_KSPLIT="8"), dict(BITNET_I2S_MID_MAX_T="0")):
+        env = dict(os.environ, **extra)
+        out = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
+        assert out.returncode == 0 and "ok" in out.stdout, (extra, out.stderr[-2000:])
+
+
 def test_zzz_no_device_wait_ever_gave_up():
     assert bn.bitnet_device_status() == 0
 
