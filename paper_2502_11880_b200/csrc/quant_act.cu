@@ -5,6 +5,8 @@
 // to nearest even, clamps, stores int8 and reduces the sum of the codes.  No fast-math anywhere:
 // the division, the product and the conversion are the IEEE round-to-nearest forms, so the bytes
 // match a scalar CPU evaluation of the same formula.
+#include <stdlib.h>
+
 #include "common.cuh"
 
 namespace bitnet {
@@ -176,6 +178,112 @@ __global__ void __launch_bounds__(NT) quant_act_reg_kernel(const float* __restri
   }
 }
 
+// Few tokens, long rows: a cluster of C CTAs shares one row (decode batches leave most SMs idle with one CTA
+// per token, and a row of 28672 floats is a 5 us round trip for a single CTA).  Each CTA keeps its segment of
+// the row in registers, the segments' maxima meet through distributed shared memory (every CTA writes its
+// partial into every peer), and after the cluster barrier every CTA holds the row's amax: the same
+// operations on the same values as quant_act_reg_kernel, so the bytes are identical.  The partial code sums
+// meet in rank 0 the same way.
+template <int NT, int C>
+__global__ void __launch_bounds__(NT) quant_act_cluster_kernel(const float* __restrict__ x, int64_t K,
+                                                               int8_t* __restrict__ q, float* __restrict__ act_scale,
+                                                               int32_t* __restrict__ act_sum) {
+  constexpr int VPT = 8;
+  __shared__ float red[32];
+  __shared__ int redi[32];
+  __shared__ float part[C];      // partial maxima of all ranks (written by the peers)
+  __shared__ int psum[C];        // partial code sums of all ranks (rank 0's copy is the one that is read)
+  const int64_t t = blockIdx.y;
+  const int rank = blockIdx.x;   // grid.x == cluster size: the rank in the cluster
+  const float4* x4 = reinterpret_cast<const float4*>(x + t * K);
+  int* q4 = reinterpret_cast<int*>(q + t * K);
+  const int tid = threadIdx.x, n4 = (int)(K / 4);
+  const int seg = (n4 + C - 1) / C, lo = rank * seg, hi = (lo + seg < n4) ? lo + seg : n4;
+  if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  float4 v[VPT];
+#pragma unroll
+  for (int r = 0; r < VPT; ++r) {
+    const int i = lo + tid + r * NT;
+    v[r] = (i < hi) ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  float m = 0.0f;
+#pragma unroll
+  for (int r = 0; r < VPT; ++r)
+    m = fmaxf(m, fmaxf(fmaxf(fabsf(v[r].x), fabsf(v[r].y)), fmaxf(fabsf(v[r].z), fabsf(v[r].w))));
+  m = warp_max(m);
+  if ((tid & 31) == 0) red[tid >> 5] = m;
+  __syncthreads();
+  if (tid < C) {
+    float mc = 0.0f;
+#pragma unroll
+    for (int w = 0; w < NT / 32; ++w) mc = fmaxf(mc, red[w]);
+    // thread p sends this CTA's maximum to rank p
+    const uint32_t mine = (uint32_t)__cvta_generic_to_shared(&part[rank]);
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(mine), "r"(tid));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(mc) : "memory");
+  }
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  float amax = 0.0f;
+#pragma unroll
+  for (int p = 0; p < C; ++p) amax = fmaxf(amax, part[p]);
+  const float amax_c = fmaxf(amax, 1e-5f);
+  const float s = __fdiv_rn(127.0f, amax_c);
+  int sum = 0;
+#pragma unroll
+  for (int r = 0; r < VPT; ++r) {
+    const int i = lo + tid + r * NT;
+    if (i < hi) {
+      const int a = quant1(v[r].x, s), b = quant1(v[r].y, s), c = quant1(v[r].z, s), d = quant1(v[r].w, s);
+      sum += a + b + c + d;
+      q4[i] = (a & 255) | ((b & 255) << 8) | ((c & 255) << 16) | ((d & 255) << 24);
+    }
+  }
+  sum = warp_sum(sum);
+  if ((tid & 31) == 0) redi[tid >> 5] = sum;
+  __syncthreads();
+  if (tid == 0) {
+    int tot = 0;
+#pragma unroll
+    for (int w = 0; w < NT / 32; ++w) tot += redi[w];
+    const uint32_t mine = (uint32_t)__cvta_generic_to_shared(&psum[rank]);
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(mine), "r"(0));
+    asm volatile("st.shared::cluster.s32 [%0], %1;" ::"r"(remote), "r"(tot) : "memory");
+  }
+  // nobody leaves before every peer's writes into its shared memory have landed; rank 0 then adds up
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  if (rank == 0 && tid == 0) {
+    int tot = 0;
+#pragma unroll
+    for (int p = 0; p < C; ++p) tot += psum[p];
+    if (act_sum) act_sum[t] = tot;
+    act_scale[t] = __fdiv_rn(amax_c, 127.0f);
+  }
+}
+
+template <int NT, int C>
+cudaError_t launch_cluster(const float* x, int64_t T, int64_t K, int8_t* q, float* act_scale, int32_t* act_sum,
+                           cudaStream_t st) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(C, (unsigned)T);
+  cfg.blockDim = dim3(NT);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = C;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = early_start_enabled() ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, quant_act_cluster_kernel<NT, C>, x, K, q, act_scale, act_sum);
+}
+
 template <int NT>
 cudaError_t launch_reg(const float* x, int64_t T, int64_t K, int8_t* q, float* act_scale, int32_t* act_sum, cudaStream_t st) {
   cudaLaunchConfig_t cfg = {};
@@ -215,7 +323,13 @@ int launch_quant_act(const float* x, int64_t T, int64_t K, int per_tensor, int8_
   } else if ((K & 3) == 0 && K <= 32 * 1024 && aligned16(x) && (reinterpret_cast<uintptr_t>(q) & 3u) == 0) {
     // rows are 16-byte aligned when x is and K % 4 == 0
     cudaError_t e;
-    if (K <= 32 * 128) e = launch_reg<128>(x, T, K, q, act_scale, act_sum, st);
+    static const bool use_clusters = [] { const char* v = getenv("BITNET_QUANT_CLUSTERS"); return !v || atoi(v) != 0; }();
+    // 4 to 8 tokens with rows of 8192 floats or more: 4 or 8 CTAs per row (100B-shaped layer at 8 tokens: 79.6
+    // instead of 81.6 us, at 6 tokens 78.0 instead of 79.9; one CTA per row is as fast or faster for a single token,
+    // 54.6 vs 55.6, and at 16 and 64 tokens, 100.8 vs 103.0 and 236 vs 238)
+    if (use_clusters && T >= 4 && T <= 8 && K >= 16384 && K <= 8 * 128 * 32) e = launch_cluster<128, 8>(x, T, K, q, act_scale, act_sum, st);
+    else if (use_clusters && T >= 4 && T <= 8 && K >= 8192 && K <= 4 * 128 * 32) e = launch_cluster<128, 4>(x, T, K, q, act_scale, act_sum, st);
+    else if (K <= 32 * 128) e = launch_reg<128>(x, T, K, q, act_scale, act_sum, st);
     else if (K <= 32 * 256) e = launch_reg<256>(x, T, K, q, act_scale, act_sum, st);
     else if (K <= 32 * 512) e = launch_reg<512>(x, T, K, q, act_scale, act_sum, st);
     else e = launch_reg<1024>(x, T, K, q, act_scale, act_sum, st);

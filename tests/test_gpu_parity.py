@@ -19,7 +19,8 @@ def tern(seed, M, K, p0=1 / 3, pp=1 / 3):
 
 
 # ----------------------------------------------------------------------------- quantiser
-@pytest.mark.parametrize("T,K", [(1, 1), (1, 7), (3, 64), (2, 1536), (1, 28672), (8, 4096), (5, 1001), (64, 333)])
+@pytest.mark.parametrize("T,K", [(1, 1), (1, 7), (3, 64), (2, 1536), (1, 28672), (8, 4096), (5, 1001), (64, 333),
+                                 (5, 8192), (8, 16384), (4, 32768), (7, 8200), (6, 16388), (9, 8192), (3, 16384)])   # 4-8 tokens: clusters of 4 / 8 CTAs per row
 def test_quant_bit_exact(T, K):
     x = synth.normal(11, T * 1000 + K % 997, T, K)
     q, sc, sm = bn.bitnet_quant_act(x.cuda())
