@@ -9,7 +9,7 @@ import oracle
 import paper_2502_11880_b200 as bn
 from paper_2502_11880_b200 import synth
 
-from helpers import check_linear, check_y, dev, no_workspace, npy, oracle_pack, run_linear
+from helpers import check_linear, check_y, dev, no_workspace, npy, oracle_pack, run_fused, run_linear
 
 pytestmark = pytest.mark.gpu
 
@@ -102,8 +102,7 @@ def test_linear_from_fp32_matches_oracle(fmt, T):
         w = tern(70 + i, M, K)
         x = synth.normal(71, i * 16 + T, T, K)
         blob = bn.pack(fmt, w.cuda())
-        y, q, sc, acc = bn.bitnet_linear(fmt, blob, 0.75, M, K, x.cuda(), want_acc=True)
-        torch.cuda.synchronize()
+        y, q, sc, acc = run_fused(fmt, blob, 0.75, M, K, x.cuda())
         q_ref, sc_ref, _ = oracle.quant_act(x.numpy())
         assert np.array_equal(npy(q), q_ref)
         assert np.array_equal(npy(sc).view(np.uint32), sc_ref.view(np.uint32))
@@ -144,12 +143,10 @@ def test_i2s_streaming_kernel_edges():
     for (M, K, T) in shapes:
         w, x = tern(36, M, K), synth.normal(36, M + T, T, K)
         out = check_linear("i2s", w, x, workspace=no_workspace())     # given codes, decode kernel
-        y, q, sc, acc = bn.bitnet_linear("i2s", out["blob"], out["w_scale"], M, K, x.cuda(), want_acc=True,
-                                         workspace=no_workspace())    # fused
-        torch.cuda.synchronize()
+        y, q, sc, acc = run_fused("i2s", out["blob"], out["w_scale"], M, K, x.cuda(), workspace=no_workspace())   # fused
         assert torch.equal(acc, out["acc"]) and torch.equal(y, out["y"]) and torch.equal(q, out["q"])
-        y, q, sc, acc = bn.bitnet_linear("i2s", out["blob"], out["w_scale"], M, K, x.cuda(), want_acc=True)
-        torch.cuda.synchronize()                                      # with whatever workspace the shape asks for
+        y, q, sc, acc = run_fused("i2s", out["blob"], out["w_scale"], M, K, x.cuda())
+        # (with whatever workspace the shape asks for)
         assert torch.equal(acc, out["acc"]) and torch.equal(y, out["y"]) and torch.equal(q, out["q"])
         if bn.bitnet_mpgemm_workspace_bytes("i2s", T, M, K):
             assert (T >= 6 or T * K > 96 * 1024)
