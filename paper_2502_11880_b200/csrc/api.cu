@@ -2,6 +2,8 @@
 // kernels of the sibling files; nothing here computes.
 #include <cstdlib>
 #include <cstring>
+#include <cstdarg>
+#include <cstdio>
 #include <mutex>
 
 #include <vector>
@@ -19,6 +21,20 @@ int note_cuda_error(cudaError_t e) {
 
 static int g_early_start = 1;
 bool early_start_enabled() { return g_early_start != 0; }
+
+bool log_enabled() {
+  static const bool on = [] { const char* e = getenv("BITNET_LOG"); return e && atoi(e) != 0; }();
+  return on;
+}
+void log_launch(const char* fmt, ...) {
+  if (!log_enabled()) return;
+  va_list ap;
+  va_start(ap, fmt);
+  fputs("[bitnet_b200] ", stderr);
+  vfprintf(stderr, fmt, ap);
+  fputc('\n', stderr);
+  va_end(ap);
+}
 
 const DevInfo& dev_info() {
   static DevInfo info[64];

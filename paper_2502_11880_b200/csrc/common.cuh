@@ -56,6 +56,10 @@ inline int check_launch() {
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(cudaGetLastError());
 }
 
+// BITNET_LOG=1: one line on stderr per kernel launch (which kernel, shape, grid, plan).  Read once.
+bool log_enabled();
+void log_launch(const char* fmt, ...);
+
 // Device properties looked up once per device.
 struct DevInfo {
   int sm_count;

@@ -569,6 +569,9 @@ int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int
   int grid = dev_info().sm_count;
   const int nitems = a.tiles_m * a.tiles_t * ksplit;
   if (grid > nitems) grid = nitems;
+  log_launch("gemm_i2s_tc_kernel T=%lld M=%lld K=%lld grid=%d tiles=%d K-parts=%d output=%s%s", (long long)T, (long long)M,
+             (long long)K, grid, a.tiles_m * a.tiles_t, ksplit, tma_store ? "bulk tensor stores" : "plain stores",
+             ksplit > 1 ? " + finish_mid_kernel" : "");
   gemm_i2s_tc_kernel<<<grid, THREADS, smem, st>>>(qmap, ymap, a);
   int rc = check_launch();
   if (rc || ksplit == 1) return rc;

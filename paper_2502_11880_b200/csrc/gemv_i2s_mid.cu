@@ -486,6 +486,9 @@ int launch_gemv_i2s_mid(const uint8_t* packed, float w_scale, int64_t M, int64_t
   a.cps = p.cps;
   a.nunits = p.nunits;
   a.qst = p.qst;
+  log_launch("gemv_i2s_mid_kernel<NT=%d,RU=%d,DEPTH=%d> T=%d M=%lld K=%lld grid=%d K-slices=%d CTAs/slice=%d smem=%zu%s",
+             p.c.NT, p.c.RU, p.c.DEPTH, T, (long long)M, (long long)K, p.grid, p.NS, p.cps, p.smem,
+             p.c.NT <= FINISH_IN_KERNEL_MAX_NT ? "" : " + finish_mid_kernel");
   int rc;
   switch (p.c.NT) {
     case 1: rc = launch_mid<1, 2, 4, 4>(a, p, st); break;

@@ -561,6 +561,8 @@ int launch_gemv_i2s_wring(const uint8_t* packed, float w_scale, int64_t M, int64
   a.nunits = p.nunits;
   a.pre = env_int("BITNET_I2S_PRE", 4);
   // short rows get the instance whose (fully unrolled) quantiser prologue is a quarter of the code
+  log_launch("gemv_i2s_wring_kernel%s T=%d M=%lld K=%lld grid=%d warps/unit=%d ring=%d smem=%zu", x ? " (fused quantiser)" : "",
+             T, (long long)M, (long long)K, p.grid, p.S, p.depth, p.smem);
   const bool small_x = x != nullptr && K <= 4 * 4 * THREADS;
   switch (p.depth) {
     case 4: return launch_wring<4, XREG_MAX>(a, p, st);

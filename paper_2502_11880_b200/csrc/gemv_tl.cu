@@ -337,6 +337,8 @@ int launch_gemv_tl(int fmt, const uint8_t* packed, float w_scale, int64_t M, int
     a.y = y + (int64_t)t0 * M;
     a.acc_out = acc_out ? acc_out + (int64_t)t0 * M : nullptr;
     a.ws_acc = reinterpret_cast<int32_t*>(ws) + (int64_t)t0 * M;
+    log_launch("gemv_tl_kernel fmt=%d tokens=%d M=%lld K=%lld grid=%lld x %d K-slices smem=%zu", fmt, a.nt, (long long)M,
+               (long long)K, (long long)gx, a.nslices, (size_t)smem);
     gemv_tl_kernel<<<dim3((unsigned)gx, (unsigned)a.nslices), THREADS, smem, st>>>(a);
     rc = check_launch();
     if (rc != BITNET_OK) return rc;

@@ -327,6 +327,7 @@ int launch_quant_act(const float* x, int64_t T, int64_t K, int per_tensor, int8_
     // 4 to 8 tokens with rows of 8192 floats or more: 4 or 8 CTAs per row (100B-shaped layer at 8 tokens: 79.6
     // instead of 81.6 us, at 6 tokens 78.0 instead of 79.9; one CTA per row is as fast or faster for a single token,
     // 54.6 vs 55.6, and at 16 and 64 tokens, 100.8 vs 103.0 and 236 vs 238)
+    if (log_enabled()) log_launch("quant_act T=%lld K=%lld", (long long)T, (long long)K);
     if (use_clusters && T >= 4 && T <= 8 && K >= 16384 && K <= 8 * 128 * 32) e = launch_cluster<128, 8>(x, T, K, q, act_scale, act_sum, st);
     else if (use_clusters && T >= 4 && T <= 8 && K >= 8192 && K <= 4 * 128 * 32) e = launch_cluster<128, 4>(x, T, K, q, act_scale, act_sum, st);
     else if (K <= 32 * 128) e = launch_reg<128>(x, T, K, q, act_scale, act_sum, st);
