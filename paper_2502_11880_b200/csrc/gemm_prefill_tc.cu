@@ -15,9 +15,13 @@
 //   * warp 1   : one thread issues four tcgen05.mma (M=128, N=256, K=32) per K block, accumulating in
 //                tensor memory, and tcgen05.commit releases the stage to the producers;
 //   * warps 10-13: epilogue -- tcgen05.ld the finished 128 x 256 accumulator (lane = out-feature,
-//                column = token), rescale and store y; a warp's 32 lanes write 32 consecutive
-//                out-features of one token, i.e. 128 contiguous bytes.  Two accumulators (2 x 256 of the
-//                512 tensor-memory columns) let the epilogue of a tile overlap the MMAs of the next.
+//                column = token), rescale with the tile's per-token factors (staged in shared memory while the
+//                MMAs still run), and hand 32 x 32 boxes of y to bulk tensor stores through a 4 KB staging
+//                buffer per warp (plain stores when the raw accumulators are wanted or M % 4 != 0; integer
+//                atomics into the workspace when a tile's K is cut into parts).  Two accumulators (2 x 256 of
+//                the 512 tensor-memory columns) let the epilogue of a tile overlap the MMAs of the next.
+// Work items are whole tiles, or, when the output has fewer tiles than three quarters of the SMs, parts of a
+// tile's K whose sums meet in the workspace and are rescaled by a second kernel.
 // Every mbarrier wait is bounded; a wait that gives up sets a CTA-wide abort flag and the device
 // status word, all roles leave their loops, and the CTA frees its tensor memory before it exits.
 #include <cuda.h>

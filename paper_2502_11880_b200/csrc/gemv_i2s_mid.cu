@@ -1,17 +1,21 @@
-// I2_S mpGEMM for batches of 9 to 64 tokens (Alg. 1, Phase 2, between decode and prefill).
+// I2_S mpGEMM for batches of 6 to 64 tokens (Alg. 1, Phase 2, between decode and prefill).
 //
 // Still a scan of the packed weights, but with T tokens per weight byte the int8 tensor cores (mma.sync
 // m16n8k32, u8 x s8), not HBM, become the limit from about 24 tokens on.  Differences to the decode kernel:
-//   * NT = ceil(T / 8) token tiles per weight fragment; the 2-bit fields are shifted down to plain codes so that
-//     all four slots of a word add into one accumulator per token tile (a decode kernel keeps one per slot);
+//   * NT = ceil(T / 8) token tiles per weight fragment; from two tiles on the 2-bit fields are shifted down so
+//     that slots share accumulators (two sets, or one from five tiles on; a decode kernel keeps one per slot);
 //   * up to two token tiles, the B fragments (activations) of a tile are read from shared memory once for
 //     RU = 2 adjacent 16-row units (one MMA needs 256 B of B, exactly what the shared-memory pipe delivers in the
 //     MMA's two cycles); from three tiles on, one unit per step with the cheaper field extraction measured faster;
-//   * T x K codes do not fit in shared memory, so K is cut into NS slices; a CTA stages the codes of one slice
-//     and runs the (slice, unit pair) items of a contiguous range, one item per warp at a time, each warp
-//     streaming its item's weights through a private cp.async ring.  With NS > 1 the int32 partial sums meet in
-//     a zeroed [T][M] workspace through integer atomics (order-independent, hence bit-exact), and a second
-//     kernel rescales them (fused rescale of Alg. 1's last line); with NS == 1 the warp stores y itself.
+//   * the staged codes are stored transposed within each 256-column chunk, token rows 64 bytes apart mod 128:
+//     the four lanes of a B load read 64 consecutive bytes and every quarter-warp covers all banks once;
+//   * T x K codes do not fit in shared memory, so K is cut into NS slices.  CTAs [sl * cps, (sl + 1) * cps) own
+//     slice sl, stage its codes once, and CTA j of them owns an equal share of the units; the CTA's sequence of
+//     (unit group, chunk) steps is cut into sixteen equal runs, one per warp, whatever units that cuts, and each
+//     warp streams its run through a private cp.async ring.  The int32 partial sums meet in a zeroed [T][M]
+//     workspace through integer atomics (order-independent, hence bit-exact);
+//   * closing rescale (Alg. 1's last line): up to 8 tokens the last-arriving CTA of a row range does it, beyond
+//     that a second kernel over all SMs; either way the workspace is left zeroed.
 // The "- sum(q)" term of the code = w + 1 representation is subtracted per slice before the atomics.
 #include <cuda_runtime.h>
 #include <stdint.h>
