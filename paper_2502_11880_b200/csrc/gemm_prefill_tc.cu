@@ -216,9 +216,13 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = bars->tmem_base;
 
+  // Early start (programmatic dependent launch): the weight unpackers and the MMA issuer touch nothing that an
+  // earlier kernel in the stream writes; the TMA producer (codes) and the epilogue (scales, y, workspace) wait.
+  if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer: activation tiles (operand B)
     if (lane == 0) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       uint32_t it = 0;
       for (int item = blockIdx.x; item < nitems && !*abort_flag; item += gridDim.x) {
         const int tile = item % ntiles;
@@ -378,6 +382,7 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
     }
   } else {
     // ------------------------------------------------------------ epilogue
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int quarter = warp & 3;                  // tensor-memory lanes 32*quarter .. 32*quarter+31
     uint32_t nt = 0;
     for (int item = blockIdx.x; item < nitems && !*abort_flag; item += gridDim.x, ++nt) {
@@ -576,8 +581,18 @@ int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int
   log_launch("gemm_i2s_tc_kernel T=%lld M=%lld K=%lld grid=%d tiles=%d K-parts=%d output=%s%s", (long long)T, (long long)M,
              (long long)K, grid, a.tiles_m * a.tiles_t, ksplit, tma_store ? "bulk tensor stores" : "plain stores",
              ksplit > 1 ? " + finish_mid_kernel" : "");
-  gemm_i2s_tc_kernel<<<grid, THREADS, smem, st>>>(qmap, ymap, a);
-  int rc = check_launch();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = early_start_enabled() ? 1 : 0;
+  cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_i2s_tc_kernel, qmap, ymap, a);
+  int rc = le == cudaSuccess ? BITNET_OK : note_cuda_error(le);
   if (rc || ksplit == 1) return rc;
   return launch_rescale_sums(a.ws, act_scale, w_scale, T, M, y, acc_out, st);
 }
