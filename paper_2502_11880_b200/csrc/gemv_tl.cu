@@ -89,6 +89,9 @@ __device__ __forceinline__ void group_acts(const TlGeom& g, int64_t K, const int
 // Phase 1: one thread per table slot; blockIdx.y = token pair.  table[pair][slot] = lo + 65536 * hi.
 __global__ void tl_table_kernel(const int8_t* __restrict__ q, int T, int64_t K, TlGeom g, int* __restrict__ table,
                                 int64_t nslots) {
+  // early start: resident before the previous kernel (the quantiser) has finished, reads its codes after the wait
+  if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= nslots) return;
   const int i = (int)(e & 15), grp = (int)((e >> 4) & 31);
@@ -125,6 +128,10 @@ __global__ void __launch_bounds__(THREADS, 2) gemv_tl_kernel(const TlArgs a) {
   const int tile0 = slice * a.tiles_per_slice;
   const int ntiles = min(a.tiles_per_slice, tiles_total - tile0);
 
+  // early start: everything this kernel reads besides the weights (tables, scales) and everything it writes
+  // (y, the split-K sums and tickets) belongs to earlier kernels until the wait returns
+  if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   // ---- the tables of this slice: one bulk copy global -> shared
   if (threadIdx.x == 0) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(bar)) : "memory");
@@ -303,8 +310,17 @@ int launch_gemv_tl(int fmt, const uint8_t* packed, float w_scale, int64_t M, int
 
   // Phase 1: tables of every token pair
   const int64_t nslots = tiles * 512;
-  tl_table_kernel<<<dim3((unsigned)ceil_div(nslots, 256), (unsigned)npairs), 256, 0, st>>>(q, T, K, g, table, nslots);
-  int rc = check_launch();
+  cudaLaunchAttribute pdl[1];
+  pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  pdl[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t tcfg = {};
+  tcfg.gridDim = dim3((unsigned)ceil_div(nslots, 256), (unsigned)npairs);
+  tcfg.blockDim = dim3(256);
+  tcfg.stream = st;
+  tcfg.attrs = pdl;
+  tcfg.numAttrs = early_start_enabled() ? 1 : 0;
+  cudaError_t le = cudaLaunchKernelEx(&tcfg, tl_table_kernel, q, T, K, g, table, nslots);
+  int rc = le == cudaSuccess ? BITNET_OK : note_cuda_error(le);
   if (rc != BITNET_OK) return rc;
 
   // Phase 2: lookups, one launch per token pair
@@ -339,8 +355,15 @@ int launch_gemv_tl(int fmt, const uint8_t* packed, float w_scale, int64_t M, int
     a.ws_acc = reinterpret_cast<int32_t*>(ws) + (int64_t)t0 * M;
     log_launch("gemv_tl_kernel fmt=%d tokens=%d M=%lld K=%lld grid=%lld x %d K-slices smem=%zu", fmt, a.nt, (long long)M,
                (long long)K, (long long)gx, a.nslices, (size_t)smem);
-    gemv_tl_kernel<<<dim3((unsigned)gx, (unsigned)a.nslices), THREADS, smem, st>>>(a);
-    rc = check_launch();
+    cudaLaunchConfig_t gcfg = {};
+    gcfg.gridDim = dim3((unsigned)gx, (unsigned)a.nslices);
+    gcfg.blockDim = dim3(THREADS);
+    gcfg.dynamicSmemBytes = smem;
+    gcfg.stream = st;
+    gcfg.attrs = pdl;
+    gcfg.numAttrs = early_start_enabled() ? 1 : 0;
+    le = cudaLaunchKernelEx(&gcfg, gemv_tl_kernel, a);
+    rc = le == cudaSuccess ? BITNET_OK : note_cuda_error(le);
     if (rc != BITNET_OK) return rc;
   }
   return BITNET_OK;
