@@ -124,10 +124,11 @@ int bitnet_pack_tl(bitnet_fmt_t fmt, const int8_t* w, int64_t M, int64_t K, int 
  *              T <= 8 needs none except for extreme shapes; I2_S with 9 <= T <= 64, and with more tokens
  *              when the output has fewer 128 x 256 tiles than three quarters of the SMs, keeps the T*M
  *              int32 sums of its K-slices there; TL keeps its lookup tables and split-K sums there).
- *              It must have been zeroed once with bitnet_workspace_init and its head (the sums) is
- *              left zeroed by every completed call; two calls sharing a workspace must not overlap
- *              on the GPU, and a workspace last used by a TL call is initialised again before an
- *              I2_S call uses it.
+ *              TL calls clear what they rely on themselves: their workspace may hold anything.  For the
+ *              I2_S kernels that keep sums there, the workspace must have been zeroed once with
+ *              bitnet_workspace_init; its head (the sums) is left zeroed by every completed I2_S call, and a
+ *              workspace last used by a TL call is initialised again before an I2_S call uses it.  Two
+ *              calls sharing a workspace must not overlap on the GPU.
  * I2_S: T <= 8 runs the decode GEMV kernel; 9 <= T <= 64 a scan of the weights on mma.sync tensor-core
  * tiles over K-slices followed by a rescale kernel (when the workspace is missing or too small, the
  * prefill kernel takes the call instead); larger T the tcgen05 prefill kernel (whole tiles per CTA; parts
@@ -171,19 +172,22 @@ int bitnet_linear_host(bitnet_fmt_t fmt, const void* packed, float w_scale, int6
 
 /*
  * A batch of linear layers with HOST activations and HOST results (Alg. 1 end to end per item), with the
- * copies overlapped with the kernels: the x_host of a group of 8 consecutive items are uploaded on an
- * internal stream, their kernels run on `stream` once those uploads are complete, and their y_host are
- * downloaded on a second internal stream once the group's kernels are complete, while the next groups'
- * uploads and kernels proceed.  Kernels run in item order on `stream`; when the call returns everything is
- * queued, and `stream` has been made to wait for the last download, so work queued on `stream` afterwards
- * (or a synchronisation of `stream`) follows every copy of the batch.
+ * copies overlapped with the kernels.  The batch is cut into about eight groups of consecutive items (one group
+ * up to 16 items); a group's x_host are uploaded on an internal stream, the group runs as one bitnet_linear_group
+ * call on `stream` (one persistent kernel for I2_S decode items) once those uploads are complete, and its y_host
+ * are downloaded on a second internal stream once the group is complete, while the next groups' uploads and
+ * kernels proceed.  The items of a batch must therefore be independent of one another, as for
+ * bitnet_linear_group.  When the call returns everything is queued, and `stream` has been made to wait for the
+ * last download, so work queued on `stream` afterwards (or a synchronisation of `stream`) follows every copy of
+ * the batch.
  *   - items[n]: plain structs in host memory, read during the call only.
  *   - x_host / y_host should be pinned.  The device buffers of different items must not overlap
  *     (uploads run ahead of the kernels); the workspace may be shared (the kernels are serial).
  *     Neighbouring items of a group whose x_host and x_dev (or y_dev and y_host) both start where the
  *     previous item's end are copied with one call: keeping the activations of a batch in one pinned
  *     block and one device block, in item order, saves a driver call per item and direction.
- *   - The internal streams and events are created on first use per device and kept.
+ *   - The internal streams and events are created on first use per device and kept for the life of the
+ *     process; a mutex serialises concurrent calls from several host threads while they queue their work.
  *   - Errors: BITNET_ERR_INVALID_ARG for a null or malformed item (nothing of that item or later ones
  *     is queued); otherwise the status of the first failing call.
  */
@@ -203,6 +207,42 @@ typedef struct bitnet_host_linear {
   size_t workspace_bytes;
 } bitnet_host_linear_t;
 int bitnet_linear_host_batch(const bitnet_host_linear_t* items, int64_t n, void* stream);
+
+/*
+ * A list of linear layers on DEVICE buffers in one call (Alg. 1 end to end per item: Phase 1 quantiser,
+ * Phase 2 mpGEMV, rescale), for linears whose inputs all exist when the call is queued: the Q/K/V or
+ * gate/up projections of one decoder layer, or every linear of a benchmark sweep.  No item may read what
+ * another item of the same call writes.
+ *   - items[n]: plain structs in host memory, read during the call only.  Per item, as for bitnet_linear:
+ *     x[T][K] fp32 in, q[T][K] int8 and act_scale[T] fp32 out, y[T][M] fp32 out, acc_out nullable.
+ *     Items that share an input may share x, q and act_scale (neighbouring I2_S items with the same x, K and
+ *     T are quantised once per CTA).
+ *   - I2_S items with T <= 8, K >= 1024 and T*(K+16) <= 144 KiB run in ONE persistent kernel per run of
+ *     up to 454 consecutive such items: the packed weights of the whole run are one stream, cut into equal
+ *     shares per SM at 16-row borders; a CTA's asynchronous copies run on across the borders between
+ *     linears, and each activation row is quantised by the two or three CTAs whose share touches its linear
+ *     instead of by every CTA of a launch of its own.  The per-launch fixed cost of a decode GEMV (about
+ *     3 us of the 5-20 us a 100B-shaped linear takes) is paid once per run.
+ *   - Every other item (TL formats, more tokens, short K) is run by bitnet_linear in list order, with the
+ *     item's workspace.
+ * Results are identical to calling bitnet_linear per item.  Errors: BITNET_ERR_INVALID_ARG for a null or
+ * malformed item (nothing is queued), otherwise the status of the first failing launch.
+ */
+typedef struct bitnet_group_item {
+  int32_t fmt;            /* bitnet_fmt_t */
+  int32_t bk3;
+  const void* packed;
+  float w_scale;
+  int64_t M, K, T;
+  const float* x;         /* [T][K] fp32, device */
+  int8_t* q;              /* [T][K] int8, device, out */
+  float* act_scale;       /* [T] fp32, device, out */
+  float* y;               /* [T][M] fp32, device, out */
+  int32_t* acc_out;       /* [T][M] int32, device, out, nullable */
+  void* workspace;        /* only used by items the grouped kernel does not take */
+  size_t workspace_bytes;
+} bitnet_group_item_t;
+int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* stream);
 
 /*
  * Table-lookup mpGEMV without a workspace argument (the paper has no counterpart: this entry point

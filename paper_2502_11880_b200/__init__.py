@@ -26,7 +26,7 @@ SYMBOLS = [
     "bitnet_pack_i2s", "bitnet_tl_packed_bytes", "bitnet_pack_tl", "bitnet_mpgemm_workspace_bytes",
     "bitnet_workspace_init", "bitnet_mpgemm", "bitnet_linear", "bitnet_linear_host", "bitnet_linear_host_batch", "bitnet_unpack_i2s", "bitnet_unpack_tl",
     "bitnet_tl_num_groups", "bitnet_tl_build_lut_debug", "bitnet_mpgemv_tl_noalloc", "bitnet_device_status",
-    "bitnet_set_early_start",
+    "bitnet_set_early_start", "bitnet_linear_group",
 ]
 
 _lib = None
@@ -65,6 +65,7 @@ def lib():
         L.bitnet_linear.argtypes = [ci, vp, fl, i64, i64, ci, vp, i64, vp, vp, vp, vp, vp, sz, vp]
         L.bitnet_linear_host.argtypes = [ci, vp, fl, i64, i64, ci, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp]
         L.bitnet_linear_host_batch.argtypes = [vp, i64, vp]
+        L.bitnet_linear_group.argtypes = [vp, i64, vp]
         L.bitnet_unpack_i2s.argtypes = [vp, i64, i64, vp, vp, vp]
         L.bitnet_unpack_tl.argtypes = [ci, vp, i64, i64, ci, vp, vp, vp]
         L.bitnet_tl_num_groups.argtypes = [ci, i64, ci]
@@ -306,6 +307,35 @@ def bitnet_linear_host_batch(batch, stream=None):
     """Queues a batch made by make_host_batch: uploads, kernels and downloads overlap; the caller
     synchronises the stream before reading the host results."""
     _check(lib().bitnet_linear_host_batch(batch, C.c_int64(len(batch)), _stream(stream)), "bitnet_linear_host_batch")
+
+
+class GroupItem(C.Structure):
+    """Mirror of bitnet_group_item_t."""
+    _fields_ = [("fmt", C.c_int32), ("bk3", C.c_int32), ("packed", C.c_void_p), ("w_scale", C.c_float),
+                ("M", C.c_int64), ("K", C.c_int64), ("T", C.c_int64), ("x", C.c_void_p), ("q", C.c_void_p),
+                ("act_scale", C.c_void_p), ("y", C.c_void_p), ("acc_out", C.c_void_p),
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
+def make_group(items):
+    """items: dicts with fmt, packed, w_scale, M, K, x, q, act_scale, y and optionally acc_out, workspace, bk3
+    (CUDA tensors).  Returns the ctypes array for bitnet_linear_group; the caller keeps the tensors alive."""
+    arr = (GroupItem * len(items))()
+    for a, d in zip(arr, items):
+        ws, acc = d.get("workspace"), d.get("acc_out")
+        a.fmt, a.bk3, a.packed, a.w_scale = _fmt(d["fmt"]), int(d.get("bk3", 0)), d["packed"].data_ptr(), float(d["w_scale"])
+        a.M, a.K, a.T = int(d["M"]), int(d["K"]), int(d["x"].shape[0])
+        a.x, a.q, a.act_scale, a.y = d["x"].data_ptr(), d["q"].data_ptr(), d["act_scale"].data_ptr(), d["y"].data_ptr()
+        a.acc_out = None if acc is None else acc.data_ptr()
+        a.workspace = None if ws is None else ws.data_ptr()
+        a.workspace_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    return arr
+
+
+def bitnet_linear_group(group, stream=None):
+    """Queues a list of linears made by make_group (device buffers): one persistent kernel per run of I2_S
+    decode items, bitnet_linear for the others."""
+    _check(lib().bitnet_linear_group(group, C.c_int64(len(group)), _stream(stream)), "bitnet_linear_group")
 
 
 NOALLOC_MAX_M = 32768

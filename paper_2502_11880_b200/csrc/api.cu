@@ -257,9 +257,11 @@ int bitnet_linear(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
   if (!aligned16(packed) || !aligned16(x) || !aligned16(q) || !aligned16(y) || (acc_out && !aligned16(acc_out)) ||
       (reinterpret_cast<uintptr_t>(act_scale) & 3u))
     return BITNET_ERR_INVALID_ARG;
-  if (fmt == BITNET_FMT_I2S && T <= 8 && !mid_takes(T, M, K, workspace, workspace_bytes)) {
-    int rc = i2s_shape(M, K);
+  if (fmt == BITNET_FMT_I2S) {
+    int rc = i2s_shape(M, K);      // before any plan is made from M and K
     if (rc) return rc;
+  }
+  if (fmt == BITNET_FMT_I2S && T <= 8 && !mid_takes(T, M, K, workspace, workspace_bytes)) {
     static const bool no_fuse = [] {
       const char* e = getenv("BITNET_I2S_KERNEL");
       return e && strcmp(e, "splitk") == 0;
@@ -293,14 +295,69 @@ int bitnet_linear_host(bitnet_fmt_t fmt, const void* packed, float w_scale, int6
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
 }
 
+int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* stream) {
+  if (n < 0 || (n > 0 && !items)) return BITNET_ERR_INVALID_ARG;
+  for (int64_t i = 0; i < n; ++i) {
+    const bitnet_group_item_t& d = items[i];
+    if (!d.packed || !d.x || !d.q || !d.act_scale || !d.y || d.T < 1 || d.M < 1 || d.K < 1) return BITNET_ERR_INVALID_ARG;
+    if (!aligned16(d.packed) || !aligned16(d.x) || !aligned16(d.q) || !aligned16(d.y) ||
+        (d.acc_out && !aligned16(d.acc_out)) || (reinterpret_cast<uintptr_t>(d.act_scale) & 3u))
+      return BITNET_ERR_INVALID_ARG;
+    if (d.fmt == BITNET_FMT_I2S) {
+      int rc = i2s_shape(d.M, d.K);
+      if (rc) return rc;
+    } else {
+      TlGeom g;
+      int rc = tl_shape(d.fmt, d.M, d.K, d.bk3, &g);
+      if (rc) return rc;
+    }
+  }
+  static const bool grouped = [] { const char* e = getenv("BITNET_GROUP"); return !(e && atoi(e) == 0); }();
+  auto takes = [&](const bitnet_group_item_t& d) {
+    return grouped && d.fmt == BITNET_FMT_I2S && d.T <= 8 && gemv_i2s_group_item_supported((int)d.T, d.M, d.K);
+  };
+  static thread_local std::vector<GroupLinear> run;
+  for (int64_t i = 0; i < n;) {
+    if (!takes(items[i])) {
+      const bitnet_group_item_t& d = items[i];
+      int rc = bitnet_linear((bitnet_fmt_t)d.fmt, d.packed, d.w_scale, d.M, d.K, d.bk3, d.x, d.T, d.q, d.act_scale, d.y,
+                             d.acc_out, d.workspace, d.workspace_bytes, stream);
+      if (rc) return rc;
+      ++i;
+      continue;
+    }
+    run.clear();
+    for (; i < n && takes(items[i]); ++i) {
+      const bitnet_group_item_t& d = items[i];
+      GroupLinear gl;
+      gl.packed = (const uint8_t*)d.packed;
+      gl.x = d.x;
+      gl.q = d.q;
+      gl.act_scale = d.act_scale;
+      gl.y = d.y;
+      gl.acc_out = d.acc_out;
+      gl.w_scale = d.w_scale;
+      gl.T = (int)d.T;
+      gl.M = d.M;
+      gl.K = d.K;
+      run.push_back(gl);
+    }
+    int rc = launch_gemv_i2s_group(run.data(), (int64_t)run.size(), (cudaStream_t)stream);
+    if (rc) return rc;
+  }
+  return BITNET_OK;
+}
+
 }  // extern "C"
 
 namespace {
-// Side streams and events of bitnet_linear_host_batch, per device, created on first use and kept.
+// Side streams and events of bitnet_linear_host_batch, per device, created on first use and kept.  One mutex
+// serialises the calls of all host threads: the call only queues work, and the events are shared.
 struct HostPipe {
   cudaStream_t up = nullptr, down = nullptr;
   std::vector<cudaEvent_t> ev;
 };
+std::mutex g_host_pipe_mu;
 HostPipe* host_pipe() {
   static HostPipe pipes[64];
   int dev = 0;
@@ -331,21 +388,23 @@ extern "C" int bitnet_linear_host_batch(const bitnet_host_linear_t* items, int64
         d.M < 1 || d.K < 1)
       return BITNET_ERR_INVALID_ARG;
   }
+  std::lock_guard<std::mutex> lock(g_host_pipe_mu);
+  // Items are handled in groups: one event after a group's uploads, one bitnet_linear_group call (for I2_S decode
+  // items: one persistent kernel) per group, one event after it.  About eight groups per batch: enough to hide
+  // all but the first group's uploads and the last group's downloads behind the kernels, few enough that the
+  // fixed cost of a launch stays small against the group's kernel time.
+  const int64_t GROUP = n <= 16 ? n : (n + 7) / 8 < 8 ? 8 : (n + 7) / 8;
+  const int64_t ngroups = (n + GROUP - 1) / GROUP;
   HostPipe* p = host_pipe();
-  if (!p || !grow_events(p, (size_t)(2 * n + 2))) return note_cuda_error(cudaErrorUnknown);
+  if (!p || !grow_events(p, (size_t)(2 * ngroups + 2))) return note_cuda_error(cudaErrorUnknown);
   cudaStream_t st = (cudaStream_t)stream;
   cudaError_t e;
 #define BN_TRY(call) do { e = (call); if (e != cudaSuccess) return note_cuda_error(e); } while (0)
   // the side streams start after whatever is already queued on `stream` (the staging buffers may be in use)
-  cudaEvent_t e_in = p->ev[2 * n], e_out = p->ev[2 * n + 1];
+  cudaEvent_t e_in = p->ev[2 * ngroups], e_out = p->ev[2 * ngroups + 1];
   BN_TRY(cudaEventRecord(e_in, st));
   BN_TRY(cudaStreamWaitEvent(p->up, e_in, 0));
   BN_TRY(cudaStreamWaitEvent(p->down, e_in, 0));
-  // Items are handled in groups of GROUP: one event after a group's uploads, one after its kernels.  Fewer
-  // events mean fewer driver calls per item, and the kernels of a group follow one another on `stream`
-  // without a wait in between, which keeps their programmatic dependent launch.
-  constexpr int64_t GROUP = 8;
-  const int64_t ngroups = (n + GROUP - 1) / GROUP;
   auto upload_group = [&](int64_t g) -> cudaError_t {
     const int64_t lo = g * GROUP, hi = (lo + GROUP < n) ? lo + GROUP : n;
     // neighbouring items whose host and device buffers both continue where the previous item's end travel as
@@ -366,6 +425,7 @@ extern "C" int bitnet_linear_host_batch(const bitnet_host_linear_t* items, int64
     }
     return cudaEventRecord(p->ev[2 * g], p->up);
   };
+  static thread_local std::vector<bitnet_group_item_t> grp;
   // uploads are queued one group ahead of the kernels, so that the first kernel does not wait for the host to
   // have queued every upload of the batch
   BN_TRY(upload_group(0));
@@ -373,18 +433,34 @@ extern "C" int bitnet_linear_host_batch(const bitnet_host_linear_t* items, int64
     if (g + 1 < ngroups) BN_TRY(upload_group(g + 1));
     const int64_t lo = g * GROUP, hi = (lo + GROUP < n) ? lo + GROUP : n;
     BN_TRY(cudaStreamWaitEvent(st, p->ev[2 * g], 0));
+    grp.clear();
     for (int64_t i = lo; i < hi; ++i) {
       const bitnet_host_linear_t& d = items[i];
-      int rc = bitnet_linear((bitnet_fmt_t)d.fmt, d.packed, d.w_scale, d.M, d.K, d.bk3, d.x_dev, d.T, d.q_dev,
-                             d.scale_dev, d.y_dev, nullptr, d.workspace, d.workspace_bytes, stream);
-      if (rc) {
-        // join the side streams before reporting, so that nothing of this call is left dangling
-        cudaEventRecord(e_out, p->down);
-        cudaStreamWaitEvent(st, e_out, 0);
-        cudaEventRecord(e_out, p->up);
-        cudaStreamWaitEvent(st, e_out, 0);
-        return rc;
-      }
+      bitnet_group_item_t gi;
+      gi.fmt = d.fmt;
+      gi.bk3 = d.bk3;
+      gi.packed = d.packed;
+      gi.w_scale = d.w_scale;
+      gi.M = d.M;
+      gi.K = d.K;
+      gi.T = d.T;
+      gi.x = d.x_dev;
+      gi.q = d.q_dev;
+      gi.act_scale = d.scale_dev;
+      gi.y = d.y_dev;
+      gi.acc_out = nullptr;
+      gi.workspace = d.workspace;
+      gi.workspace_bytes = d.workspace_bytes;
+      grp.push_back(gi);
+    }
+    int rc = bitnet_linear_group(grp.data(), (int64_t)grp.size(), stream);
+    if (rc) {
+      // join the side streams before reporting, so that nothing of this call is left dangling
+      cudaEventRecord(e_out, p->down);
+      cudaStreamWaitEvent(st, e_out, 0);
+      cudaEventRecord(e_out, p->up);
+      cudaStreamWaitEvent(st, e_out, 0);
+      return rc;
     }
     BN_TRY(cudaEventRecord(p->ev[2 * g + 1], st));
     BN_TRY(cudaStreamWaitEvent(p->down, p->ev[2 * g + 1], 0));

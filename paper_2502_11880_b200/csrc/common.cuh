@@ -95,6 +95,20 @@ int gemv_i2s_stream_status(int* out);
 bool gemv_i2s_wring_supported(int T, int64_t M, int64_t K);
 int launch_gemv_i2s_wring(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const float* x, int8_t* q,
                           float* act_scale, int T, float* y, int32_t* acc_out, cudaStream_t st);
+// One persistent kernel over a list of I2_S linears (1..8 tokens each) whose inputs exist at launch.
+struct GroupLinear {
+  const uint8_t* packed;
+  const float* x;      // fp32 activations [T][K] (q, act_scale are then outputs); null: q, act_scale are inputs
+  int8_t* q;
+  float* act_scale;
+  float* y;
+  int32_t* acc_out;    // nullable
+  float w_scale;
+  int T;
+  int64_t M, K;
+};
+bool gemv_i2s_group_item_supported(int T, int64_t M, int64_t K);
+int launch_gemv_i2s_group(const GroupLinear* items, int64_t n, cudaStream_t st);
 // Batches of 9 to 64 tokens: mma.sync over K-slices, partial sums through a [T][M] int32 workspace when K is
 // cut into more than one slice (gemv_i2s_mid_workspace_bytes says how much; 0 = none needed).
 bool gemv_i2s_mid_supported(int T, int64_t M, int64_t K);

@@ -1,0 +1,560 @@
+// Grouped I2_S decode (1..8 tokens): Alg. 1, Phases 1 and 2 plus the rescale, for a LIST of linear layers
+// whose inputs are all there at launch, in ONE persistent kernel.
+//
+// Why.  A decode GEMV of a few tens of megabytes lasts 5-20 us, of which about 3 us per launch are fixed
+// (launch release, the quantiser's round trip, the first tile, the tail).  Over a list of linears that fixed
+// part is paid once here: the packed weights of the whole list are one stream of work that is cut into 148
+// equal pieces, one per SM, and a CTA walks its piece from the first byte to the last without ever letting
+// its asynchronous copies run dry, across the borders between linears.
+//
+// Work split.  The unit of work is a 16-row block of one linear (contiguous in the blob: 4*Kp bytes).  The
+// units of all items, in item order, form one sequence; CTA c owns the contiguous range whose packed bytes
+// are the c-th 1/gridDim of the total (found on the device by a binary search over the items' prefix sums,
+// which the host puts into the argument block).  A CTA's range touches two or three items of a long list, so
+// the activation row changes only a few times per CTA.  Inside the CTA the 16 warps form G = 16/S groups;
+// group gi takes the units jb+gi, jb+gi+G, ... of the range, and the S warps of a group split a unit's K
+// into slices (as in the single-linear kernel).  Every warp owns a ring of DEPTH 1-KB chunks in shared
+// memory, filled by per-thread cp.async copies that the same thread reads back: the only synchronisation of
+// the weight stream is cp.async.wait_group.  The prefetch position of a warp is a cursor of its own that runs
+// DEPTH chunks ahead of the consume position through the same sequence of units -- over unit borders, item
+// borders and the CTA-wide barriers of an item change alike.
+//
+// Item change.  When the CTA's range enters a new item, the CTA meets at a barrier, quantises the item's
+// activation rows (fp32 -> int8 by absmax, the row held in registers between the two passes; same operations
+// in the same order as the stand-alone quantiser, so bit-identical) or copies the given codes, into shared
+// memory, and goes on.  An item whose input (x, K, T) equals the previous item's keeps the staged codes: linears
+// that share an input (Q/K/V, gate/up) quantise it once per CTA.  The CTA whose range holds an item's first
+// unit also stores the codes and scales for the caller.
+//
+// Compute side: as in the single-linear kernel -- a packed word under the mask 0x03030303 << 2s is an A
+// register of mma.sync.m16n8k32 (u8 x s8), four accumulators carry the scales 1, 4, 16, 64, and
+// sum(code*q) - sum(q) = sum(w*q); the row sum of the codes is taken once while staging.
+#include <cstdlib>
+#include <cstring>
+
+#include "common.cuh"
+#include "device_utils.cuh"
+
+namespace bitnet {
+namespace {
+
+constexpr int CW = 16;  // warps
+constexpr int THREADS = CW * 32;
+constexpr int XREG = 16;                       // float4 registers per thread of the quantiser's one-pass form
+constexpr int NSMALL = 56, NLARGE = 454;       // items per launch: argument blocks of 4 KB / 32 KB
+constexpr size_t MAX_CODE_BYTES = 144 * 1024;  // staged activation codes of one item
+
+struct GItem {
+  const uint8_t* packed;
+  const float* x;      // fp32 activations [T][K]; null: q and act_scale are inputs
+  int8_t* q;
+  float* act_scale;
+  float* y;
+  int32_t* acc_out;
+  float w_scale;
+  int M, K, T;
+  int first_unit;      // units of the items before this one
+  int first_w;         // 1-KB chunks of the items before this one
+};
+static_assert(sizeof(GItem) == 72, "argument block layout");
+
+template <int NMAX>
+struct GArgs {
+  int n, S, tmax, code_bytes;
+  int total_units, total_w, r0, r1;
+  GItem it[NMAX];
+};
+static_assert(sizeof(GArgs<NSMALL>) <= 4096 && sizeof(GArgs<NLARGE>) <= 32764, "kernel parameter limits");
+
+__device__ __forceinline__ bool same_input(const GItem& p, const GItem& d) {
+  return p.K == d.K && p.T == d.T && (d.x ? p.x == d.x : (p.x == nullptr && p.q == d.q && p.act_scale == d.act_scale));
+}
+
+// Stages the item's activation codes (T rows, kp + 16 bytes apart, zero beyond K) and, per token, the scale
+// and the sum of the codes.  Called by all threads; contains barriers.
+__device__ __forceinline__ void stage_item(const GItem& d, bool owner, int kp, int8_t* qs_mem, float* qscale,
+                                           int* qsum, float* qred) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int qst = kp + 16, n4 = d.K / 4, kw = kp / 4;
+  if (threadIdx.x < 8) qsum[threadIdx.x] = 0;
+  if (d.x && d.K <= 4 * XREG * THREADS) {
+    // Alg. 1 Phase 1, one round trip per token: s = 127 / max(amax, 1e-5), q = clamp(rint(x * s))
+    const int nrow = (kw + THREADS - 1) / THREADS;
+    for (int tok = 0; tok < d.T; ++tok) {
+      const float4* x4 = reinterpret_cast<const float4*>(d.x + (int64_t)tok * d.K);
+      float4 xv[XREG];
+#pragma unroll
+      for (int r = 0; r < XREG; ++r) {
+        const int i = threadIdx.x + r * THREADS;
+        xv[r] = (r < nrow && i < n4) ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+      float m = 0.0f;
+#pragma unroll
+      for (int r = 0; r < XREG; ++r)
+        if (r < nrow) m = fmaxf(m, absmax4(xv[r]));
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      if (tok > 0) __syncthreads();  // everyone has read the previous token's partial maxima
+      if (lane == 0) qred[warp] = m;
+      __syncthreads();
+      float amax = 0.0f;
+#pragma unroll
+      for (int w2 = 0; w2 < CW; ++w2) amax = fmaxf(amax, qred[w2]);
+      const float amax_c = fmaxf(amax, 1e-5f);
+      const float sq = __fdiv_rn(127.0f, amax_c);
+      if (threadIdx.x == 0) {
+        const float inv = __fdiv_rn(amax_c, 127.0f);
+        qscale[tok] = inv;
+        if (owner) d.act_scale[tok] = inv;
+      }
+      int s = 0;
+#pragma unroll
+      for (int r = 0; r < XREG; ++r) {
+        const int i = threadIdx.x + r * THREADS;
+        if (r < nrow && i < kw) {
+          const int word = quant4_packed(xv[r], sq);  // columns K..Kp-1 came in as zeros
+          reinterpret_cast<int*>(qs_mem + tok * qst)[i] = word;
+          s = __dp4a(word, 0x01010101, s);
+          if (owner && i < n4) reinterpret_cast<int*>(d.q + (int64_t)tok * d.K)[i] = word;
+        }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      if (lane == 0) atomicAdd(qsum + tok, s);
+    }
+  } else if (d.x) {
+    // rows too long for the registers: amax per token, then a second pass over x
+    for (int tok = 0; tok < d.T; ++tok) {
+      const float4* x4 = reinterpret_cast<const float4*>(d.x + (int64_t)tok * d.K);
+      float m = 0.0f;
+      for (int i = threadIdx.x; i < n4; i += THREADS) m = fmaxf(m, absmax4(__ldcg(x4 + i)));
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      if (lane == 0) qred[tok * CW + warp] = m;
+    }
+    __syncthreads();
+    if (threadIdx.x < d.T) {
+      float m = 0.0f;
+      for (int w2 = 0; w2 < CW; ++w2) m = fmaxf(m, qred[threadIdx.x * CW + w2]);
+      const float amax_c = fmaxf(m, 1e-5f);
+      const float inv = __fdiv_rn(amax_c, 127.0f);
+      qscale[threadIdx.x] = inv;
+      if (owner) d.act_scale[threadIdx.x] = inv;
+    }
+    __syncthreads();
+    for (int tok = 0; tok < d.T; ++tok) {
+      float m = 0.0f;
+      for (int w2 = 0; w2 < CW; ++w2) m = fmaxf(m, qred[tok * CW + w2]);
+      const float sq = __fdiv_rn(127.0f, fmaxf(m, 1e-5f));
+      const float4* x4 = reinterpret_cast<const float4*>(d.x + (int64_t)tok * d.K);
+      int s = 0;
+      for (int i = threadIdx.x; i < kw; i += THREADS) {
+        int word = 0;
+        if (i < n4) {
+          word = quant4_packed(__ldcg(x4 + i), sq);
+          if (owner) reinterpret_cast<int*>(d.q + (int64_t)tok * d.K)[i] = word;
+        }
+        reinterpret_cast<int*>(qs_mem + tok * qst)[i] = word;
+        s = __dp4a(word, 0x01010101, s);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      if (lane == 0) atomicAdd(qsum + tok, s);
+    }
+  } else {
+    // given codes
+    __syncthreads();  // qsum is zero before the first atomicAdd
+    for (int tok = 0; tok < d.T; ++tok) {
+      const int* qrow = reinterpret_cast<const int*>(d.q + (int64_t)tok * d.K);
+      int s = 0;
+      for (int i = threadIdx.x; i < kw; i += THREADS) {
+        const int word = (i < n4) ? __ldcg(qrow + i) : 0;
+        reinterpret_cast<int*>(qs_mem + tok * qst)[i] = word;
+        s = __dp4a(word, 0x01010101, s);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      if (lane == 0) atomicAdd(qsum + tok, s);
+    }
+    if (threadIdx.x < d.T) qscale[threadIdx.x] = __ldcg(d.act_scale + threadIdx.x);
+  }
+}
+
+template <int DEPTH, int NMAX>
+__global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid_constant__ GArgs<NMAX> a) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  int* hdr = reinterpret_cast<int*>(smem);             // [0] first unit, [1] end unit, [2] first item, [3] last item
+  float* qscale = reinterpret_cast<float*>(smem + 64);  // [8] act_scale per token
+  int* qsum = reinterpret_cast<int*>(smem + 96);        // [8] sum of the codes per token
+  float* qred = reinterpret_cast<float*>(smem + 128);   // [8][16] partial maxima
+  int* red = reinterpret_cast<int*>(smem + 1024);       // [CW][2][tmax][16] partial sums
+  int8_t* qs_mem = reinterpret_cast<int8_t*>(smem + 1024 + CW * 2 * a.tmax * 16 * 4);
+  uint8_t* rings = reinterpret_cast<uint8_t*>(qs_mem) + a.code_bytes;
+
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int S = a.S, G = CW / S, gi = warp / S, wk = warp % S;
+  const int g = lane >> 2, t = lane & 3;
+
+  if (threadIdx.x == 0) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // this CTA's range of the unit sequence: equal shares of the packed bytes, cut at unit borders
+    auto locate = [&](int64_t w, int* item) -> int {
+      int lo = 0, hi = a.n - 1;
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if ((int64_t)a.it[mid].first_w <= w) lo = mid; else hi = mid - 1;
+      }
+      *item = lo;
+      const int nch = (int)(i2s_kp(a.it[lo].K) / 256);
+      return a.it[lo].first_unit + (int)((w - a.it[lo].first_w) / nch);
+    };
+    int ib, ie;
+    const int jb = locate((int64_t)blockIdx.x * a.total_w / gridDim.x, &ib);
+    const int je = locate((int64_t)(blockIdx.x + 1) * a.total_w / gridDim.x, &ie);
+    hdr[0] = jb;
+    hdr[1] = je;
+    hdr[2] = ib;
+    hdr[3] = (je > a.it[ie].first_unit) ? ie : ie - 1;
+  }
+  __syncthreads();
+  const int jb = hdr[0], je = hdr[1], item0 = hdr[2], item1 = hdr[3];
+  if (jb >= je) return;
+
+  const uint64_t pol = policy_evict_first();
+  const uint32_t ring = smem_u32(rings + (size_t)warp * DEPTH * 1024) + lane * 16;
+
+  // ---------------- where the group's next unit lies: a cursor over the items that runs one unit ahead
+  int n_item = item0, n_first = 0, n_end = 0, n_ub = 0;
+  const uint8_t* n_base = nullptr;
+  auto n_load = [&](int i) {
+    const GItem& d = a.it[i];
+    const int kp = (int)i2s_kp(d.K), nch = kp / 256;
+    n_ub = 4 * kp;
+    n_first = d.first_unit;
+    n_end = (i + 1 < a.n) ? a.it[i + 1].first_unit : a.total_units;
+    n_base = d.packed + (int64_t)(wk * nch / S) * 1024 + lane * 16;
+  };
+  // first chunk of this warp's slice of unit `job` (job < je, jobs asked for in ascending order)
+  auto job_ptr = [&](int job) -> const uint8_t* {
+    while (job >= n_end) n_load(++n_item);
+    return n_base + (int64_t)(job - n_first) * n_ub;
+  };
+  n_load(item0);
+  int cj = jb + gi, nloc = 0;
+  const uint8_t* cur = (cj < je) ? job_ptr(cj) : nullptr;
+  // Weights depend on nothing an earlier kernel writes: fill the ring before waiting for that kernel.  Every
+  // slice of every item is at least DEPTH chunks long (the host chooses S and DEPTH that way).
+#pragma unroll
+  for (int d = 0; d < DEPTH; ++d) {
+    if (cur) {
+      cp16(ring + d * 1024, cur + d * 1024, pol);
+      cp16(ring + d * 1024 + 512, cur + d * 1024 + 512, pol);
+    }
+    cp_commit();
+  }
+
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  // ---------------- consume
+  uint32_t slot_off = 0;
+  const int tmax = a.tmax;
+  for (int ci = item0; ci <= item1; ++ci) {
+    const GItem& d = a.it[ci];
+    const int T = d.T, kp = (int)i2s_kp(d.K), nch = kp / 256, qst = kp + 16;
+    const bool owner = jb <= d.first_unit;
+    if (ci == item0 || !same_input(a.it[ci - 1], d)) {
+      if (ci > item0) __syncthreads();  // everyone is done with the previous item's codes
+      stage_item(d, owner, kp, qs_mem, qscale, qsum, qred);
+      __syncthreads();
+    } else if (owner && d.x && d.q != a.it[ci - 1].q) {
+      // same input as the previous item but its own output buffers for the codes
+      for (int tok = 0; tok < T; ++tok)
+        for (int i = threadIdx.x; i < d.K / 4; i += THREADS)
+          reinterpret_cast<int*>(d.q + (int64_t)tok * d.K)[i] = reinterpret_cast<const int*>(qs_mem + tok * qst)[i];
+      if (threadIdx.x < T) d.act_scale[threadIdx.x] = qscale[threadIdx.x];
+    }
+    const int c_lo = wk * nch / S, c_hi = (wk + 1) * nch / S, nw = c_hi - c_lo;
+    const int iend = (ci + 1 < a.n) ? a.it[ci + 1].first_unit : a.total_units;
+    const int cend = je < iend ? je : iend;
+    const int first = d.first_unit, M = d.M;
+    const unsigned has_tok = g < T ? 1u : 0u;
+    const uint32_t q_lane = smem_u32(qs_mem + min(g, T - 1) * qst + c_lo * 256 + t * 64);
+    const float w_scale = d.w_scale;
+    float* const y = d.y;
+    int32_t* const acc_out = d.acc_out;
+
+    for (; cj < cend; cj += G, ++nloc) {
+      int C[4][4];
+#pragma unroll
+      for (int s = 0; s < 4; ++s)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) C[s][i] = 0;
+      uint32_t qp = q_lane;
+      int qr[8] = {0, 0, 0, 0, 0, 0, 0, 0};  // B registers; lanes beyond the batch keep these zeros
+      // One step: wait for the oldest chunk of the ring, put it through the tensor cores, then refill its slot
+      // from `pf` (the chunk DEPTH places further down the warp's stream), if there is one.
+      auto step = [&](const uint8_t* pf, bool do_pf) {
+        cp_wait<DEPTH - 1>();
+        unsigned w4[4], v4[4];
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(w4[0]), "=r"(w4[1]), "=r"(w4[2]), "=r"(w4[3])
+                     : "r"(ring + slot_off));
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(v4[0]), "=r"(v4[1]), "=r"(v4[2]), "=r"(v4[3])
+                     : "r"(ring + slot_off + 512));
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          // only the lanes whose B column is a real token load activations
+          asm volatile(
+              "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %9, 0;\n\t"
+              "@p ld.shared.v4.u32 {%0,%1,%2,%3}, [%8];\n\t"
+              "@p ld.shared.v4.u32 {%4,%5,%6,%7}, [%8+16];\n\t}"
+              : "+r"(qr[0]), "+r"(qr[1]), "+r"(qr[2]), "+r"(qr[3]), "+r"(qr[4]), "+r"(qr[5]), "+r"(qr[6]), "+r"(qr[7])
+              : "r"(qp + h * 32), "r"(has_tok));
+#pragma unroll
+          for (int s = 0; s < 4; ++s) {
+            const unsigned m = 0x03030303u << (2 * s);
+            mma_u8s8(C[s], w4[2 * h] & m, v4[2 * h] & m, w4[2 * h + 1] & m, v4[2 * h + 1] & m, qr[2 * s], qr[2 * s + 1]);
+          }
+        }
+        qp += 256;
+        // the chunk's bytes were in registers before the MMAs were issued: its slot can be refilled
+        if (do_pf) {
+          cp16(ring + slot_off, pf, pol);
+          cp16(ring + slot_off + 512, pf + 512, pol);
+        }
+        cp_commit();
+        slot_off = (slot_off + 1024 == DEPTH * 1024) ? 0 : slot_off + 1024;
+      };
+
+      // chunks 0 .. nw-DEPTH-1 are followed, DEPTH places on, by chunks of the same unit; the last DEPTH chunks by
+      // the first DEPTH chunks of the group's next unit (in this item or a later one), if there is one
+      const int nj = cj + G;
+      const bool more = nj < je;
+      const uint8_t* const nxt = more ? job_ptr(nj) : cur;
+      const uint8_t* pf = cur + DEPTH * 1024;
+#pragma unroll 2
+      for (int left = nw - DEPTH; left > 0; --left, pf += 1024) step(pf, true);
+#pragma unroll
+      for (int dd = 0; dd < DEPTH; ++dd) step(nxt + dd * 1024, more);
+      cur = nxt;
+
+      // fragment: c[0] = (row g, token 2t), c[1] = (row g, token 2t+1), c[2], c[3] = the same for row g+8
+      int c[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) c[i] = C[0][i] + (C[1][i] >> 2) + (C[2][i] >> 4) + (C[3][i] >> 6);
+      int* mine = red + ((warp * 2 + (nloc & 1)) * tmax) * 16;
+      if (2 * t < T) {
+        mine[(2 * t) * 16 + g] = c[0];
+        mine[(2 * t) * 16 + g + 8] = c[2];
+      }
+      if (2 * t + 1 < T) {
+        mine[(2 * t + 1) * 16 + g] = c[1];
+        mine[(2 * t + 1) * 16 + g + 8] = c[3];
+      }
+      if (S > 1) group_barrier(1 + gi, S * 32);
+      else __syncwarp();
+      if (wk == (nloc & (S - 1))) {
+        // this unit's turn to be finished by this warp: add the group's partials, rescale, store 16 rows
+        const int row0 = (cj - first) * 16;
+        const int* grp = red + (((gi * S) * 2 + (nloc & 1)) * tmax) * 16;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int idx = lane + 32 * i;
+          if (idx < T * 16) {
+            int v = 0;
+            for (int w2 = 0; w2 < S; ++w2) v += grp[w2 * 2 * tmax * 16 + idx];
+            const int tok = idx >> 4, row = row0 + (idx & 15);
+            v -= qsum[tok];
+            if (row < M) {
+              y[(int64_t)tok * M + row] = __fmul_rn((float)v, __fmul_rn(qscale[tok], w_scale));
+              if (acc_out) acc_out[(int64_t)tok * M + row] = v;
+            }
+          }
+        }
+      }
+    }
+  }
+  cp_wait<0>();
+  __syncthreads();   // no warp leaves the CTA before the others are done
+}
+
+int env_int_once(const char* name, int dflt) {
+  const char* v = getenv(name);
+  return (v && *v) ? atoi(v) : dflt;
+}
+// Tuning overrides, read once: warps per unit (1, 2 or 4) and ring depth (4, 6, 8 or 12); 0 = the defaults below.
+int forced_s() {
+  static const int s = [] {
+    const int v = env_int_once("BITNET_GROUP_S", 0);
+    return (v == 1 || v == 2 || v == 4 || v == 8) ? v : 0;
+  }();
+  return s;
+}
+int depth_cap() {
+  static const int d = [] {
+    const int v = env_int_once("BITNET_GROUP_DEPTH", 8);
+    return (v == 4 || v == 6 || v == 8 || v == 12) ? v : 8;
+  }();
+  return d;
+}
+
+// Warps per unit and ring depth for a launch whose shortest rows have `nch` chunks: every warp's K-slice must be
+// at least as long as its ring (the prefetch never reaches beyond the next unit), so short rows get fewer warps per
+// unit, then shallower rings.
+struct Shape {
+  int S, depth;
+};
+Shape shape_for(int64_t nch) {
+  int S = forced_s() ? forced_s() : 4;
+  while (S > 1 && nch / S < 8) S >>= 1;
+  const int64_t nw = nch / S;      // the shortest slice
+  int depth = depth_cap();
+  while (depth > 4 && depth > nw) depth = depth == 12 ? 8 : depth - 2;
+  return Shape{S, depth};
+}
+
+size_t code_bytes_of(int T, int64_t K) { return ((size_t)T * (size_t)(i2s_kp(K) + 16) + 127) & ~(size_t)127; }
+size_t smem_of(int tmax, size_t code_bytes, int depth) {
+  return 1024 + (size_t)CW * 2 * tmax * 16 * 4 + code_bytes + (size_t)CW * depth * 1024;
+}
+
+template <int DEPTH, int NMAX>
+int launch_group(const GArgs<NMAX>& a, int grid, size_t smem, cudaStream_t st) {
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (!attr_set[dev & 63]) {
+    cudaError_t e = cudaFuncSetAttribute(gemv_i2s_group_kernel<DEPTH, NMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         dev_info().max_smem_optin);
+    if (e != cudaSuccess) return note_cuda_error(e);
+    attr_set[dev & 63] = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = early_start_enabled() ? 1 : 0;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_i2s_group_kernel<DEPTH, NMAX>, a);
+  return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
+}
+
+template <int NMAX>
+int launch_depth(const GArgs<NMAX>& a, int depth, int grid, size_t smem, cudaStream_t st) {
+  switch (depth) {
+    case 4: return launch_group<4, NMAX>(a, grid, smem, st);
+    case 6: return launch_group<6, NMAX>(a, grid, smem, st);
+    case 8: return launch_group<8, NMAX>(a, grid, smem, st);
+    case 12: return launch_group<12, NMAX>(a, grid, smem, st);
+    default: return BITNET_ERR_UNSUPPORTED_SHAPE;
+  }
+}
+
+// One launch over items of one shape class (the same S and ring depth suit all of them).
+template <int NMAX>
+int launch_run(const GroupLinear* items, int n, Shape shape, cudaStream_t st) {
+  static thread_local GArgs<NMAX> a;   // 32 KB: off the stack
+  a.n = n;
+  a.S = shape.S;
+  a.tmax = 1;
+  size_t code = 0;
+  int64_t units = 0, w = 0;
+  for (int i = 0; i < n; ++i) {
+    const GroupLinear& s = items[i];
+    GItem& d = a.it[i];
+    d.packed = s.packed;
+    d.x = s.x;
+    d.q = s.q;
+    d.act_scale = s.act_scale;
+    d.y = s.y;
+    d.acc_out = s.acc_out;
+    d.w_scale = s.w_scale;
+    d.M = (int)s.M;
+    d.K = (int)s.K;
+    d.T = s.T;
+    d.first_unit = (int)units;
+    d.first_w = (int)w;
+    const int64_t nu = ceil_div(s.M, 16), nch = i2s_kp(s.K) / 256;
+    units += nu;
+    w += nu * nch;
+    if (s.T > a.tmax) a.tmax = s.T;
+    const size_t cb = code_bytes_of(s.T, s.K);
+    if (cb > code) code = cb;
+  }
+  a.total_units = (int)units;
+  a.total_w = (int)w;
+  a.code_bytes = (int)code;
+  a.r0 = a.r1 = 0;
+  const int depth = shape.depth;
+  const size_t smem = smem_of(a.tmax, code, depth);
+  if (smem > (size_t)dev_info().max_smem_optin) return BITNET_ERR_UNSUPPORTED_SHAPE;
+  const int G = CW / a.S;
+  int grid = dev_info().sm_count;
+  if ((int64_t)grid * G > units) grid = (int)ceil_div(units, G);
+  log_launch("gemv_i2s_group_kernel items=%d units=%lld chunks=%lld grid=%d warps/unit=%d ring=%d tmax=%d smem=%zu", n,
+             (long long)units, (long long)w, grid, a.S, depth, a.tmax, smem);
+  return launch_depth<NMAX>(a, depth, grid, smem, st);
+}
+
+// S and ring depth for a launch over items whose shortest rows have `nch` chunks, whose largest batch is `tmax`
+// tokens and whose largest staged codes take `code` bytes; false if they do not fit one SM's shared memory.
+bool launch_shape(int64_t nch, int tmax, size_t code, Shape* out) {
+  if (nch < 4 || code > MAX_CODE_BYTES) return false;
+  Shape sh = shape_for(nch);
+  const size_t cap = (size_t)dev_info().max_smem_optin;
+  while (sh.depth > 4 && smem_of(tmax, code, sh.depth) > cap) sh.depth = sh.depth == 12 ? 8 : sh.depth - 2;
+  if (smem_of(tmax, code, sh.depth) > cap) return false;
+  *out = sh;
+  return true;
+}
+
+}  // namespace
+
+bool gemv_i2s_group_item_supported(int T, int64_t M, int64_t K) {
+  if (T < 1 || T > 8 || M < 1 || K < 1 || (K % 64) != 0 || M > 0x7fffffff) return false;
+  Shape sh;
+  return launch_shape(i2s_kp(K) / 256, T, code_bytes_of(T, K), &sh);
+}
+
+// Launches the grouped kernel over `n` supported items: as few launches as the argument block (NLARGE items,
+// 2^30 chunks) and shared memory (the largest batch and the longest rows of a launch set its code area) allow.
+// A launch runs with the warps per unit and ring depth that suit its shortest rows.
+int launch_gemv_i2s_group(const GroupLinear* items, int64_t n, cudaStream_t st) {
+  int64_t i = 0;
+  while (i < n) {
+    int64_t j = i, w = 0, nch_min = 1 << 30;
+    int tmax = 1;
+    size_t code = 0;
+    Shape sh{1, 4};
+    while (j < n && j - i < NLARGE) {
+      const int64_t nch = i2s_kp(items[j].K) / 256;
+      const int64_t add = ceil_div(items[j].M, 16) * nch;
+      const size_t cb = code_bytes_of(items[j].T, items[j].K);
+      const int tm = items[j].T > tmax ? items[j].T : tmax;
+      const size_t cm = cb > code ? cb : code;
+      const int64_t nm = nch < nch_min ? nch : nch_min;
+      Shape sj;
+      const bool fits = launch_shape(nm, tm, cm, &sj);
+      if (!fits && j == i) return BITNET_ERR_UNSUPPORTED_SHAPE;
+      if (!fits || (j > i && w + add > (1ll << 30))) break;
+      w += add;
+      tmax = tm;
+      code = cm;
+      nch_min = nm;
+      sh = sj;
+      ++j;
+    }
+    const int cnt = (int)(j - i);
+    const int rc = cnt <= NSMALL ? launch_run<NSMALL>(items + i, cnt, sh, st) : launch_run<NLARGE>(items + i, cnt, sh, st);
+    if (rc != BITNET_OK) return rc;
+    i = j;
+  }
+  return BITNET_OK;
+}
+
+}  // namespace bitnet

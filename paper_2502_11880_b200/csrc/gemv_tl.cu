@@ -88,10 +88,15 @@ __device__ __forceinline__ void group_acts(const TlGeom& g, int64_t K, const int
 
 // Phase 1: one thread per table slot; blockIdx.y = token pair.  table[pair][slot] = lo + 65536 * hi.
 __global__ void tl_table_kernel(const int8_t* __restrict__ q, int T, int64_t K, TlGeom g, int* __restrict__ table,
-                                int64_t nslots) {
+                                int64_t nslots, int* __restrict__ head, int64_t head_ints) {
   // early start: resident before the previous kernel (the quantiser) has finished, reads its codes after the wait
   if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  // The split-K sums and arrival counters of this call start at zero whatever an earlier call (of another shape,
+  // whose tables may have lain here) left in the workspace.
+  for (int64_t i = ((int64_t)blockIdx.y * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x; i < head_ints;
+       i += (int64_t)gridDim.x * gridDim.y * blockDim.x)
+    head[i] = 0;
   const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= nslots) return;
   const int i = (int)(e & 15), grp = (int)((e >> 4) & 31);
@@ -319,7 +324,8 @@ int launch_gemv_tl(int fmt, const uint8_t* packed, float w_scale, int64_t M, int
   tcfg.stream = st;
   tcfg.attrs = pdl;
   tcfg.numAttrs = early_start_enabled() ? 1 : 0;
-  cudaError_t le = cudaLaunchKernelEx(&tcfg, tl_table_kernel, q, T, K, g, table, nslots);
+  cudaError_t le = cudaLaunchKernelEx(&tcfg, tl_table_kernel, q, T, K, g, table, nslots, reinterpret_cast<int*>(ws),
+                                      (int64_t)T * M + M);
   int rc = le == cudaSuccess ? BITNET_OK : note_cuda_error(le);
   if (rc != BITNET_OK) return rc;
 

@@ -1,0 +1,158 @@
+"""bitnet_linear_group (a list of linears in one persistent kernel) against the CPU oracle, through the
+C ABI: quantised codes, scale bit patterns and int32 accumulators identical, fp32 outputs within 1e-6."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2502_11880_b200 as bn
+from paper_2502_11880_b200 import synth
+
+from helpers import Guarded, check_y, npy
+
+pytestmark = pytest.mark.gpu
+
+
+def tern(seed, M, K, p0=1 / 3, pp=1 / 3):
+    return synth.ternary(seed, 77, M, K, p0, pp)
+
+
+class Item:
+    """One linear of a group: weights, activations and guarded output buffers."""
+
+    def __init__(self, fmt, M, K, T, seed, x=None, w_scale=0.75):
+        self.fmt, self.M, self.K, self.T, self.w_scale = fmt, M, K, T, w_scale
+        self.w = tern(seed, M, K)
+        self.x = synth.normal(seed, 1000 + T, T, K) if x is None else x
+        self.xd = self.x.cuda()
+        self.blob = bn.pack(fmt, self.w.cuda())
+        self.gq, self.gsc = Guarded((T, K), torch.int8), Guarded((T,), torch.float32)
+        self.gy, self.gacc = Guarded((T, M), torch.float32), Guarded((T, M), torch.int32)
+        self.ws = bn.new_workspace(fmt, T, M, K)
+
+    def desc(self):
+        return dict(fmt=self.fmt, packed=self.blob, w_scale=self.w_scale, M=self.M, K=self.K, x=self.xd, q=self.gq.t,
+                    act_scale=self.gsc.t, y=self.gy.t, acc_out=self.gacc.t, workspace=self.ws)
+
+    def check(self, rows=None):
+        for name, g in (("q", self.gq), ("act_scale", self.gsc), ("y", self.gy), ("acc", self.gacc)):
+            assert g.intact(), f"M={self.M} K={self.K} T={self.T}: bytes outside {name} were written"
+        q_ref, sc_ref, _ = oracle.quant_act(self.x.numpy())
+        assert np.array_equal(npy(self.gq.t), q_ref)
+        assert np.array_equal(npy(self.gsc.t).view(np.uint32), sc_ref.view(np.uint32))
+        w = self.w.numpy()
+        acc, y = npy(self.gacc.t), self.gy.t
+        if rows is not None:
+            w, acc, y = w[rows], acc[:, rows], y[:, rows]
+        acc_ref = oracle.mpgemm_def(q_ref, np.ascontiguousarray(w))
+        assert np.array_equal(acc, acc_ref)
+        check_y(y, acc_ref, sc_ref, self.w_scale)
+
+
+def run_group(items):
+    grp = bn.make_group([it.desc() for it in items])
+    bn.bitnet_linear_group(grp)
+    torch.cuda.synchronize()
+    assert bn.bitnet_device_status() == 0
+
+
+def test_group_small_ragged_list():
+    """Few units for the SMs, ragged row counts, K with a padded last chunk, every token count, one item per
+    shape class; most CTAs get no work or a single unit, and units of neighbouring items share a CTA."""
+    shapes = [(1, 1024, 1), (7, 1536, 2), (300, 3200, 3), (33, 8640, 4), (160, 2048, 5), (48, 28672, 1),
+              (100, 8192, 8), (16, 1024, 6), (17, 4096, 7)]
+    items = [Item("i2s", M, K, T, 100 + i) for i, (M, K, T) in enumerate(shapes)]
+    run_group(items)
+    for it in items:
+        it.check()
+
+
+def test_group_many_units_per_cta_and_shared_inputs():
+    """More units than warp groups (every group walks several units and crosses item borders), Q/K/V-like items
+    that share one activation buffer (quantised once, each item still gets its codes), and an item whose token
+    count differs from its neighbours'."""
+    K = 4096
+    x = synth.normal(7, 1, 2, K)
+    items = [Item("i2s", 6144, K, 2, 200, x=x), Item("i2s", 4096, K, 2, 201, x=x), Item("i2s", 5000, K, 2, 202, x=x),
+             Item("i2s", 4096, 14336, 1, 203), Item("i2s", 9000, 2048, 3, 204)]
+    # the first two share the device input AND the code buffers, the third only the input
+    items[1].xd = items[0].xd
+    items[2].xd = items[0].xd
+    d = [it.desc() for it in items]
+    d[1]["q"], d[1]["act_scale"] = d[0]["q"], d[0]["act_scale"]
+    grp = bn.make_group(d)
+    bn.bitnet_linear_group(grp)
+    torch.cuda.synchronize()
+    items[1].gq, items[1].gsc = items[0].gq, items[0].gsc
+    for it in items:
+        it.check()
+
+
+def test_group_mixed_formats_fall_back_in_order():
+    """TL2 items, a prefill-sized item and a short-K item inside the list are run by bitnet_linear; the I2_S decode
+    items on either side still go through the grouped kernel."""
+    items = [Item("i2s", 64, 2048, 1, 300), Item("tl2", 64, 3200, 2, 301), Item("i2s", 96, 8192, 2, 302),
+             Item("i2s", 32, 256, 1, 303), Item("i2s", 64, 1536, 24, 304), Item("tl1", 32, 130, 1, 305),
+             Item("i2s", 200, 4096, 4, 306)]
+    run_group(items)
+    for it in items:
+        it.check()
+
+
+def test_group_more_items_than_the_small_argument_block():
+    """60 items: the kernel instance with the 32 KB argument block."""
+    items = [Item("i2s", 16 * (1 + i % 5), 1024 + 256 * (i % 3), 1 + i % 2, 400 + i) for i in range(60)]
+    run_group(items)
+    for it in items:
+        it.check()
+
+
+def test_group_equals_single_calls_and_given_workload_layer():
+    """A 100B-shaped decoder layer (8192->10240, 8192->8192, 8192->57344, 28672->8192) at one token through the
+    grouped call: every output row against the oracle."""
+    wl = synth.CONFIGS["sweep100b"]
+    items = []
+    for j, lin in enumerate(wl.linears):
+        it = Item.__new__(Item)
+        it.fmt, it.M, it.K, it.T = "i2s", lin.M, lin.K, 1
+        it.w = wl.weights(3, j)
+        it.w_scale = synth.absmean_scale(it.w)
+        it.x = wl.activations(3, j, 1)
+        it.xd = it.x.cuda()
+        it.blob = bn.pack("i2s", it.w.cuda())
+        it.gq, it.gsc = Guarded((1, lin.K), torch.int8), Guarded((1,), torch.float32)
+        it.gy, it.gacc = Guarded((1, lin.M), torch.float32), Guarded((1, lin.M), torch.int32)
+        it.ws = None
+        items.append(it)
+    run_group(items)
+    for it in items:
+        it.check()
+    # and the same list through bitnet_linear, one call per item: identical bits
+    for it in items:
+        y, q, sc, acc = bn.bitnet_linear("i2s", it.blob, it.w_scale, it.M, it.K, it.xd, want_acc=True)
+        torch.cuda.synchronize()
+        assert torch.equal(y, it.gy.t) and torch.equal(acc, it.gacc.t) and torch.equal(q, it.gq.t)
+
+
+@pytest.mark.parametrize("T", [2, 4])
+def test_group_layer_batched(T):
+    """The 8B-shaped layer at 2 and 4 tokens per linear through the grouped call, sampled rows."""
+    wl = synth.CONFIGS["layer8b"]
+    items = [Item("i2s", lin.M, lin.K, T, 500 + j) for j, lin in enumerate(wl.linears)]
+    run_group(items)
+    rng = np.random.default_rng(5)
+    for it in items:
+        it.check(rows=np.sort(rng.choice(it.M, 200, replace=False)))
+
+
+def test_group_rejects_malformed_items():
+    it = Item("i2s", 32, 1024, 1, 600)
+    d = it.desc()
+    grp = bn.make_group([d])
+    grp[0].K = 1000                      # not a multiple of 64
+    with pytest.raises(bn.BitnetError, match="shape"):
+        bn.bitnet_linear_group(grp)
+    grp = bn.make_group([d])
+    grp[0].y = None
+    with pytest.raises(bn.BitnetError, match="invalid"):
+        bn.bitnet_linear_group(grp)

@@ -583,3 +583,27 @@ def test_linear_host_batch_merges_neighbouring_buffers():
         assert torch.equal(it["y_host"], ref)
     assert bool((yh_all[ny:] == -7.0).all())
     assert bn.bitnet_device_status() == 0
+
+
+@pytest.mark.parametrize("fmt", ["tl1", "tl2"])
+def test_tl_workspace_shared_by_calls_of_different_shapes(fmt):
+    """One workspace serves TL calls of different shapes back to back: the tables of a call with few rows lie
+    where a later call with many rows keeps its split-K sums, so every call must clear what it relies on."""
+    shapes = [(32, 28672, 2), (4096, 8192, 1), (64, 14336, 3), (2048, 28672, 1), (32, 96 * 40, 1)]
+    n = max(bn.bitnet_mpgemm_workspace_bytes(fmt, T, M, K) for M, K, T in shapes)
+    ws = torch.full((n,), 0x5A, dtype=torch.uint8, device="cuda")      # never initialised: garbage on purpose
+    cases = []
+    for i, (M, K, T) in enumerate(shapes):
+        w = tern(90 + i, M, K)
+        x = synth.normal(91, i, T, K)
+        q, sc, _ = bn.bitnet_quant_act(x.cuda())
+        cases.append((M, K, T, w, x, q, sc, bn.pack(fmt, w.cuda())))
+    outs = []
+    for M, K, T, w, x, q, sc, blob in cases + cases[::-1]:             # no synchronisation between the calls
+        outs.append(bn.bitnet_mpgemm(fmt, blob, 0.5, M, K, q, sc, want_acc=True, workspace=ws))
+    torch.cuda.synchronize()
+    for (M, K, T, w, x, q, sc, blob), (y, acc) in zip(cases + cases[::-1], outs):
+        q_ref, sc_ref, _ = oracle.quant_act(x.numpy())
+        acc_ref = oracle.mpgemm_def(q_ref, w.numpy())
+        assert np.array_equal(npy(acc), acc_ref)
+        check_y(y, acc_ref, sc_ref, 0.5)
