@@ -104,9 +104,12 @@ int bitnet_pack_i2s(const int8_t* w, int64_t M, int64_t K, void* packed, size_t 
  *        (v = 9w0+3w1+w2, index |v|, sign [v<0]); the remaining TwoK columns as TL1 pairs
  *        (index 3(w0+1)+(w1+1)).  TL1: all columns as pairs.
  * Blob: for each block of 32 rows, ThreeK/96 tiles of 640 bytes then ceil(TwoK/64) tiles of 512
- * bytes.  In a tile, row r owns bytes [16r, 16r+16): byte i = index of group 2i (low nibble) and
- * 2i+1 (high nibble); a TL2 tile ends with 32 little-endian uint32 sign words (row r at 512+4r,
- * bit g = sign of group g).  Pairs past K carry index 4 = (0,0).
+ * bytes.  A row of a tile has 16 index bytes, byte i = index of group 2i (low nibble) and 2i+1 (high
+ * nibble).  Row r = g + 8u of the block (g = r % 8, u = r / 8) keeps byte i at 64g + 16(i/4) + 4u + i%4 of
+ * the 512-byte index plane: every 16-byte piece holds one 32-bit word of the four rows g, g+8, g+16, g+24
+ * (the rows one lane of a 16x8x32 tensor-core MMA owns in the two halves of the block).  A TL2 tile ends
+ * with the 128-byte sign plane: row r's little-endian uint32 at 512 + 16g + 4u, the sign of group grp
+ * (index byte i = grp/2) in its bit 8(i%4) + 2(i/4) + grp%2.  Pairs past K carry index 4 = (0,0).
  * Requires K even and M % 32 == 0.  dev_status as for bitnet_pack_i2s.
  */
 size_t bitnet_tl_packed_bytes(bitnet_fmt_t fmt, int64_t M, int64_t K, int bk3);

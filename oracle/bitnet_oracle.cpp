@@ -51,32 +51,47 @@ constexpr int FMT_TL2 = 2;
 
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
-// ---- TL geometry: 32-row tiles; a TL2 tile covers 96 weights (32 triples), a TL1 tile 64 (32 pairs)
+// ---- TL geometry (Sec. 3.1.2).  A blob is a sequence of 32-row blocks; each block holds its triple-coded
+// columns as tiles of 32 triples per row (96 weights, 640 bytes) followed by its pair-coded columns as tiles
+// of 32 pairs per row (64 weights, 512 bytes).
 struct TlGeom {
-  int64_t three_k;      // columns handled by TL2 triples
-  int64_t two_k;        // columns handled by TL1 pairs
-  int64_t tiles3;       // TL2 tiles per row block
-  int64_t tiles2;       // TL1 tiles per row block
-  int64_t block_bytes;  // bytes of one 32-row block
+  int64_t three_k;      // ThreeK: columns coded as triples
+  int64_t two_k;        // TwoK: columns coded as pairs
+  int64_t tiles3;       // triple tiles per block
+  int64_t tiles2;       // pair tiles per block
+  int64_t block_bytes;  // bytes per block
 };
 
 bool tl_geom(int fmt, int64_t M, int64_t K, int bk3, TlGeom* g) {
-  if (M <= 0 || K <= 0 || (M % 32) != 0 || (K % 2) != 0) return false;
-  if (bk3 == 0) bk3 = 96;
-  if (bk3 < 0 || (bk3 % 96) != 0) return false;
-  if (fmt == FMT_TL2) {
-    g->three_k = (K / bk3) * bk3;  // ThreeK = floor(K / BK3) * BK3
-    g->two_k = K - g->three_k;     // TwoK = K - ThreeK
-  } else if (fmt == FMT_TL1) {
-    g->three_k = 0;
-    g->two_k = K;
-  } else {
-    return false;
-  }
+  const int64_t BK3 = bk3 ? bk3 : 96;
+  const bool shape_ok = M >= 32 && M % 32 == 0 && K >= 2 && K % 2 == 0 && BK3 > 0 && BK3 % 96 == 0;
+  if (!shape_ok || (fmt != FMT_TL1 && fmt != FMT_TL2)) return false;
+  // block-fitting split: ThreeK = floor(K / BK3) * BK3 columns as triples, the remaining TwoK as pairs;
+  // TL1 codes every column as a pair
+  const int64_t whole_blocks = (fmt == FMT_TL2) ? K / BK3 : 0;
+  g->three_k = whole_blocks * BK3;
+  g->two_k = K - g->three_k;
   g->tiles3 = g->three_k / 96;
-  g->tiles2 = ceil_div(g->two_k, 64);
-  g->block_bytes = g->tiles3 * 640 + g->tiles2 * 512;
+  g->tiles2 = (g->two_k + 63) / 64;
+  g->block_bytes = 640 * g->tiles3 + 512 * g->tiles2;
   return true;
+}
+
+// ---- positions inside a tile (this build's layout; the paper fixes only the codes and the split into an index
+// plane and a sign plane).  Row r = g + 8u of the block (g = r % 8, u = r / 8); its 32 groups are 16 index bytes,
+// byte i holding group 2i in the low nibble and group 2i+1 in the high nibble.
+//   index plane (512 bytes): byte i of row r lies at 64g + 16(i/4) + 4u + i%4, i.e. the four rows g, g+8, g+16,
+//     g+24 interleave word by word, each 16-byte piece holding word i/4 of those four rows;
+//   sign plane of a triple tile (128 bytes at 512): row r owns the little-endian uint32 at 512 + 16g + 4u, and the
+//     sign of group grp (index byte i = grp/2) is its bit 8(i%4) + 2(i/4) + grp%2.
+inline int tl_idx_pos(int r, int grp) {
+  const int i = grp / 2;
+  return 64 * (r % 8) + 16 * (i / 4) + 4 * (r / 8) + (i % 4);
+}
+inline int tl_sign_pos(int r) { return 512 + 16 * (r % 8) + 4 * (r / 8); }
+inline int tl_sign_bit(int grp) {
+  const int i = grp / 2;
+  return 8 * (i % 4) + 2 * (i / 4) + (grp % 2);
 }
 
 inline int tern_ok(int8_t w) { return w >= -1 && w <= 1; }
@@ -241,10 +256,10 @@ void oracle_tl_split(int fmt, int64_t K, int bk3, int64_t* three_k, int64_t* two
 }
 
 // Blob = for each block of 32 rows: tiles3 TL2 tiles, then tiles2 TL1 tiles.
-//  TL2 tile (640 B): row r owns bytes [16r,16r+16) of the 512-byte index plane, byte i = index of
-//    triple 2i in the low nibble and of triple 2i+1 in the high nibble; then a 128-byte sign plane,
-//    row r owns the little-endian uint32 at 512+4r whose bit g is the sign of triple g.
-//  TL1 tile (512 B): same index plane over 32 pairs; pairs past the end of K carry code 4 = (0,0).
+//  TL2 tile (640 B): 512-byte index plane (index of triple 2i in the low nibble of the row's byte i, of triple
+//    2i+1 in the high nibble) then a 128-byte sign plane, one uint32 per row; positions as tl_idx_pos,
+//    tl_sign_pos and tl_sign_bit above give them.
+//  TL1 tile (512 B): the same index plane over 32 pairs; pairs past the end of K carry code 4 = (0,0).
 int oracle_pack_tl(int fmt, const int8_t* w, int64_t M, int64_t K, int bk3, uint8_t* packed) {
   TlGeom g;
   if (!w || !packed || !tl_geom(fmt, M, K, bk3, &g)) return 1;
@@ -262,17 +277,17 @@ int oracle_pack_tl(int fmt, const int8_t* w, int64_t M, int64_t K, int bk3, uint
         const int64_t k = t * 96 + 3 * grp;
         const int code = oracle_tl2_code(wr[k], wr[k + 1], wr[k + 2]);
         const int idx = code & 15;
-        if (code & 16) signs |= (1u << grp);
-        tile[16 * r + grp / 2] |= (uint8_t)((grp & 1) ? (idx << 4) : idx);
+        if (code & 16) signs |= (1u << tl_sign_bit(grp));
+        tile[tl_idx_pos((int)r, grp)] |= (uint8_t)((grp & 1) ? (idx << 4) : idx);
       }
-      for (int b = 0; b < 4; ++b) tile[512 + 4 * r + b] = (uint8_t)(signs >> (8 * b));
+      for (int b = 0; b < 4; ++b) tile[tl_sign_pos((int)r) + b] = (uint8_t)(signs >> (8 * b));
     }
     for (int64_t t = 0; t < g.tiles2; ++t) {
       uint8_t* tile = blk + g.tiles3 * 640 + t * 512;
       for (int grp = 0; grp < 32; ++grp) {
         const int64_t k = g.three_k + t * 64 + 2 * grp;
         const int idx = (k < K) ? oracle_tl1_code(wr[k], wr[k + 1]) : 4;
-        tile[16 * r + grp / 2] |= (uint8_t)((grp & 1) ? (idx << 4) : idx);
+        tile[tl_idx_pos((int)r, grp)] |= (uint8_t)((grp & 1) ? (idx << 4) : idx);
       }
     }
   }
@@ -289,13 +304,14 @@ int oracle_unpack_tl(int fmt, const uint8_t* packed, int64_t M, int64_t K, int b
     for (int64_t t = 0; t < g.tiles3; ++t) {
       const uint8_t* tile = blk + t * 640;
       uint32_t signs = 0;
-      for (int b = 0; b < 4; ++b) signs |= (uint32_t)tile[512 + 4 * r + b] << (8 * b);
+      for (int b = 0; b < 4; ++b) signs |= (uint32_t)tile[tl_sign_pos((int)r) + b] << (8 * b);
       for (int grp = 0; grp < 32; ++grp) {
-        const uint8_t byte = tile[16 * r + grp / 2];
+        const uint8_t byte = tile[tl_idx_pos((int)r, grp)];
         const int idx = (grp & 1) ? (byte >> 4) : (byte & 15);
         if (idx > 13) return 3;
-        int v = ((signs >> grp) & 1u) ? -idx : idx;
-        if (idx == 0 && ((signs >> grp) & 1u)) return 3;
+        const bool neg = ((signs >> tl_sign_bit(grp)) & 1u) != 0;
+        int v = neg ? -idx : idx;
+        if (idx == 0 && neg) return 3;
         // balanced-ternary digits of v in [-13, 13]
         int d[3];
         for (int i = 2; i >= 0; --i) {
@@ -313,7 +329,7 @@ int oracle_unpack_tl(int fmt, const uint8_t* packed, int64_t M, int64_t K, int b
     for (int64_t t = 0; t < g.tiles2; ++t) {
       const uint8_t* tile = blk + g.tiles3 * 640 + t * 512;
       for (int grp = 0; grp < 32; ++grp) {
-        const uint8_t byte = tile[16 * r + grp / 2];
+        const uint8_t byte = tile[tl_idx_pos((int)r, grp)];
         const int idx = (grp & 1) ? (byte >> 4) : (byte & 15);
         if (idx > 8) return 3;
         const int64_t k = g.three_k + t * 64 + 2 * grp;
@@ -384,18 +400,18 @@ int oracle_tl_mpgemm(int fmt, const uint8_t* packed, int64_t M, int64_t K, int b
       for (int64_t tile_i = 0; tile_i < g.tiles3; ++tile_i) {
         const uint8_t* tile = blk + tile_i * 640;
         uint32_t signs = 0;
-        for (int b = 0; b < 4; ++b) signs |= (uint32_t)tile[512 + 4 * r + b] << (8 * b);
+        for (int b = 0; b < 4; ++b) signs |= (uint32_t)tile[tl_sign_pos((int)r) + b] << (8 * b);
         for (int grp = 0; grp < 32; ++grp) {
-          const uint8_t byte = tile[16 * r + grp / 2];
+          const uint8_t byte = tile[tl_idx_pos((int)r, grp)];
           const int idx = (grp & 1) ? (byte >> 4) : (byte & 15);
           const int val = lut[(tile_i * 32 + grp) * 16 + idx];
-          s += ((signs >> grp) & 1u) ? -val : val;
+          s += ((signs >> tl_sign_bit(grp)) & 1u) ? -val : val;
         }
       }
       for (int64_t tile_i = 0; tile_i < g.tiles2; ++tile_i) {
         const uint8_t* tile = blk + g.tiles3 * 640 + tile_i * 512;
         for (int grp = 0; grp < 32; ++grp) {
-          const uint8_t byte = tile[16 * r + grp / 2];
+          const uint8_t byte = tile[tl_idx_pos((int)r, grp)];
           const int idx = (grp & 1) ? (byte >> 4) : (byte & 15);
           s += lut[(g.tiles3 * 32 + tile_i * 32 + grp) * 16 + idx];
         }

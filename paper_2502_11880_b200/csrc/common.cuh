@@ -37,6 +37,16 @@ inline __host__ bool tl_geom(int fmt, int64_t M, int64_t K, int bk3, TlGeom* g) 
   return true;
 }
 
+// Positions inside a TL tile.  Row r = g + 8u of the 32-row block (g = r % 8, u = r / 8) has 16 index bytes (byte i:
+// group 2i in the low nibble, 2i+1 in the high nibble), i.e. four 32-bit words.  Word t of row r lies at
+// 64g + 16t + 4u: every 16-byte piece of the index plane holds word t of the rows g, g+8, g+16, g+24 -- the four
+// rows a lane of an m16n8k32 MMA owns in the two 16-row halves of the block.  A triple tile's sign plane keeps row
+// r's uint32 at 512 + 16g + 4u; the sign of group grp (index byte i = grp/2) is bit 8(i%4) + 2(i/4) + grp%2, so
+// that (signs >> 2t) & 0x03030303 lines the sign pairs of word t's four bytes up with those bytes.
+inline __host__ __device__ int tl_word_off(int r, int t) { return 64 * (r & 7) + 16 * t + 4 * (r >> 3); }
+inline __host__ __device__ int tl_sign_off(int r) { return 512 + 16 * (r & 7) + 4 * (r >> 3); }
+inline __host__ __device__ int tl_sign_bit(int grp) { return 8 * ((grp >> 1) & 3) + 2 * (grp >> 3) + (grp & 1); }
+
 // Geometry of an I2_S blob: rows in blocks of 16, K padded to 256; a block is contiguous and holds
 // one 1024-byte piece per 256-column chunk, row r of the block owning bytes [64r, 64r+64) of it.
 // Word j (0..15) of those 64 bytes, slot s (bits [8b+2s, 8b+2s+1] of byte b) holds the weights

@@ -121,6 +121,12 @@ __device__ __forceinline__ int sign_mask(unsigned sg, int bit) {   // 0 or -1 fr
   return m;
 }
 
+// The four index words of row `r` of a tile (they lie 16 bytes apart: the tile interleaves four rows per piece).
+__device__ __forceinline__ uint4 load_row_words(const uint8_t* tp, int r) {
+  const unsigned* p = reinterpret_cast<const unsigned*>(tp + tl_word_off(r, 0));
+  return make_uint4(__ldg(p), __ldg(p + 4), __ldg(p + 8), __ldg(p + 12));
+}
+
 __global__ void __launch_bounds__(THREADS, 2) gemv_tl_kernel(const TlArgs a) {
   extern __shared__ __align__(128) int smem[];
   int* tab = smem;                                   // [tiles_per_slice][32][16]
@@ -185,8 +191,8 @@ __global__ void __launch_bounds__(THREADS, 2) gemv_tl_kernel(const TlArgs a) {
   bool have = rb < nrb && tl < ntiles;
   if (have) {
     const uint8_t* tp = tile_ptr(rb, tl);
-    iw = __ldg(reinterpret_cast<const uint4*>(tp) + lane);
-    sg = (tile0 + tl < a.g.tiles3) ? __ldg(reinterpret_cast<const unsigned*>(tp + 512) + lane) : 0u;
+    iw = load_row_words(tp, lane);
+    sg = (tile0 + tl < a.g.tiles3) ? __ldg(reinterpret_cast<const unsigned*>(tp + tl_sign_off(lane))) : 0u;
   }
   for (int nb = 0; rb < nrb; rb += gridDim.x, ++nb) {
     int lo = 0, hi = 0;
@@ -204,8 +210,8 @@ __global__ void __launch_bounds__(THREADS, 2) gemv_tl_kernel(const TlArgs a) {
       }
       if (nrbi < nrb && ntl < ntiles) {
         const uint8_t* tp = tile_ptr(nrbi, ntl);
-        iw = __ldg(reinterpret_cast<const uint4*>(tp) + lane);
-        sg = (tile0 + ntl < a.g.tiles3) ? __ldg(reinterpret_cast<const unsigned*>(tp + 512) + lane) : 0u;
+        iw = load_row_words(tp, lane);
+        sg = (tile0 + ntl < a.g.tiles3) ? __ldg(reinterpret_cast<const unsigned*>(tp + tl_sign_off(lane))) : 0u;
       }
       const unsigned words[4] = {ciw.x, ciw.y, ciw.z, ciw.w};
       const char* tt = reinterpret_cast<const char*>(tab + ctl * 512);
@@ -218,7 +224,7 @@ __global__ void __launch_bounds__(THREADS, 2) gemv_tl_kernel(const TlArgs a) {
           // byte offset of the slot: 4 * nibble n of the word
           const unsigned off = (n == 0) ? ((words[w4] << 2) & 0x3Cu) : ((words[w4] >> (4 * n - 2)) & 0x3Cu);
           const int v = *reinterpret_cast<const int*>(tt + grp * 64 + off);
-          s += v ^ sign_mask(csg, grp);
+          s += v ^ sign_mask(csg, tl_sign_bit(grp));
         }
       }
       // split the packed pair: s = H * 65536 + L with |L| < 32768

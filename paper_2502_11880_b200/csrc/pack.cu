@@ -59,13 +59,14 @@ __global__ void unpack_i2s_kernel(const uint32_t* __restrict__ packed, int64_t M
   if (bad && dev_status) atomicExch(dev_status, BITNET_ERR_BAD_WEIGHT);
 }
 
-// One thread per (row, tile): emits the row's 16 index bytes (and the sign word of a TL2 tile).
+// One thread per (row, tile): emits the row's four index words (and the sign word of a TL2 tile) at the
+// positions tl_word_off / tl_sign_off / tl_sign_bit give.
 __global__ void pack_tl_kernel(const int8_t* __restrict__ w, int64_t M, int64_t K, TlGeom g,
                                uint8_t* __restrict__ packed, int* dev_status) {
   const int64_t tiles = g.tiles3 + g.tiles2;
   const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (gid >= M * tiles) return;
-  // consecutive threads = consecutive rows of one tile, so the 16-byte stores of a warp are contiguous
+  // consecutive threads = consecutive rows of one tile: a warp's stores cover the tile's planes completely
   const int64_t r = gid % 32;
   const int64_t tile = (gid / 32) % tiles;
   const int64_t rb = gid / (32 * tiles);
@@ -82,12 +83,13 @@ __global__ void pack_tl_kernel(const int8_t* __restrict__ w, int64_t M, int64_t 
       bad |= !(ternary(w0) && ternary(w1) && ternary(w2));
       const int v = 9 * w0 + 3 * w1 + w2;
       const uint32_t idx = (uint32_t)abs(v) & 15u;
-      signs |= (v < 0 ? 1u : 0u) << grp;
+      signs |= (v < 0 ? 1u : 0u) << tl_sign_bit(grp);
       idx_words[grp >> 3] |= idx << (4 * (grp & 7));
     }
     uint8_t* tp = blk + tile * 640;
-    *reinterpret_cast<uint4*>(tp + 16 * r) = make_uint4(idx_words[0], idx_words[1], idx_words[2], idx_words[3]);
-    *reinterpret_cast<uint32_t*>(tp + 512 + 4 * r) = signs;
+#pragma unroll
+    for (int t = 0; t < 4; ++t) *reinterpret_cast<uint32_t*>(tp + tl_word_off((int)r, t)) = idx_words[t];
+    *reinterpret_cast<uint32_t*>(tp + tl_sign_off((int)r)) = signs;
   } else {
     const int64_t t2 = tile - g.tiles3;
     const int64_t k0 = g.three_k + t2 * 64;
@@ -102,7 +104,8 @@ __global__ void pack_tl_kernel(const int8_t* __restrict__ w, int64_t M, int64_t 
       idx_words[grp >> 3] |= idx << (4 * (grp & 7));
     }
     uint8_t* tp = blk + g.tiles3 * 640 + t2 * 512;
-    *reinterpret_cast<uint4*>(tp + 16 * r) = make_uint4(idx_words[0], idx_words[1], idx_words[2], idx_words[3]);
+#pragma unroll
+    for (int t = 0; t < 4; ++t) *reinterpret_cast<uint32_t*>(tp + tl_word_off((int)r, t)) = idx_words[t];
   }
   if (bad && dev_status) atomicExch(dev_status, BITNET_ERR_BAD_WEIGHT);
 }
@@ -121,12 +124,13 @@ __global__ void unpack_tl_kernel(const uint8_t* __restrict__ packed, int64_t M, 
   bool bad = false;
   if (tile < g.tiles3) {
     const uint8_t* tp = blk + tile * 640;
-    const uint4 iw = *reinterpret_cast<const uint4*>(tp + 16 * r);
-    const uint32_t words[4] = {iw.x, iw.y, iw.z, iw.w};
-    const uint32_t signs = *reinterpret_cast<const uint32_t*>(tp + 512 + 4 * r);
+    uint32_t words[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) words[t] = *reinterpret_cast<const uint32_t*>(tp + tl_word_off((int)r, t));
+    const uint32_t signs = *reinterpret_cast<const uint32_t*>(tp + tl_sign_off((int)r));
     for (int grp = 0; grp < 32; ++grp) {
       const int idx = (words[grp >> 3] >> (4 * (grp & 7))) & 15;
-      const int neg = (signs >> grp) & 1;
+      const int neg = (signs >> tl_sign_bit(grp)) & 1;
       bad |= (idx > 13) || (idx == 0 && neg);
       // digits of idx in balanced ternary: idx = 9 d0 + 3 d1 + d2, digits in {-1,0,1}
       const int d0 = (idx + 4) / 9;                 // 0 for idx <= 4, 1 for 5..13
@@ -142,8 +146,9 @@ __global__ void unpack_tl_kernel(const uint8_t* __restrict__ packed, int64_t M, 
   } else {
     const int64_t t2 = tile - g.tiles3;
     const uint8_t* tp = blk + g.tiles3 * 640 + t2 * 512;
-    const uint4 iw = *reinterpret_cast<const uint4*>(tp + 16 * r);
-    const uint32_t words[4] = {iw.x, iw.y, iw.z, iw.w};
+    uint32_t words[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) words[t] = *reinterpret_cast<const uint32_t*>(tp + tl_word_off((int)r, t));
     for (int grp = 0; grp < 32; ++grp) {
       const int idx = (words[grp >> 3] >> (4 * (grp & 7))) & 15;
       const int64_t k = g.three_k + t2 * 64 + 2 * grp;

@@ -200,6 +200,9 @@ __global__ void __launch_bounds__(NT) quant_act_cluster_kernel(const float* __re
   const int tid = threadIdx.x, n4 = (int)(K / 4);
   const int seg = (n4 + C - 1) / C, lo = rank * seg, hi = (lo + seg < n4) ? lo + seg : n4;
   if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // A peer's shared memory may be written only once that peer is known to be running: every CTA announces itself
+  // here, and the matching wait stands right before the first remote store (it hides behind the loads of x).
+  asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
   float4 v[VPT];
 #pragma unroll
@@ -214,6 +217,7 @@ __global__ void __launch_bounds__(NT) quant_act_cluster_kernel(const float* __re
   m = warp_max(m);
   if ((tid & 31) == 0) red[tid >> 5] = m;
   __syncthreads();
+  asm volatile("barrier.cluster.wait.aligned;" ::: "memory");   // every CTA of the cluster has started
   if (tid < C) {
     float mc = 0.0f;
 #pragma unroll

@@ -182,6 +182,30 @@ def test_i2s_documented_bit_positions():
     assert _i2s_byte_and_shift(16, 0, 256) == (1024, 0) and _i2s_byte_and_shift(0, 256, 512) == (1024, 0)
 
 
+def test_i2s_blob_read_back_by_the_inverse_statement():
+    """The layout stated the other way round: in the 1024-byte piece of 16-row block rb and 256-column chunk c,
+    row r of the block owns bytes [64r, 64r+64); there, 32-bit word j (0..15), byte b, bit pair s (bits 8b+2s,
+    8b+2s+1 of the word) holds code w+1 of column 256c + 32*(j//2) + 8*s + 4*(j%2) + b.  Every field of a random
+    blob (ragged M and K, so padding fields too) is decoded that way."""
+    M, K = 21, 448
+    w = rand_ternary(M, K)
+    p = oracle.pack_i2s(w)
+    kp, mp = 512, 32
+    assert p.size == mp * kp // 4
+    for rb in range(mp // 16):
+        for c in range(kp // 256):
+            piece = p[rb * 4 * kp + c * 1024: rb * 4 * kp + (c + 1) * 1024]
+            for r in range(16):
+                for j in range(16):
+                    word = int.from_bytes(bytes(piece[64 * r + 4 * j: 64 * r + 4 * j + 4]), "little")
+                    for b in range(4):
+                        for s_ in range(4):
+                            code = (word >> (8 * b + 2 * s_)) & 3
+                            m, k = 16 * rb + r, 256 * c + 32 * (j // 2) + 8 * s_ + 4 * (j % 2) + b
+                            want = int(w[m, k]) + 1 if (m < M and k < K) else 1
+                            assert code == want, (m, k)
+
+
 def test_i2s_one_hot_dot_products():
     # a single +-1 at position k against q[k] = k - 60 returns exactly +-(k - 60)
     K = 128
@@ -268,27 +292,48 @@ def test_tl_round_trip(fmt, K):
 
 
 def test_tl2_documented_byte_positions():
-    # one TL2 tile (32 rows x 96 weights): row r, triple g -> nibble (g odd: high) of byte 16r + g//2,
-    # sign -> bit g of the little-endian word at 512 + 4r
+    # one TL2 tile (32 rows x 96 weights).  Row r = g + 8u; triple grp sits in index byte i = grp//2 (grp odd: high
+    # nibble) at 64g + 16(i//4) + 4u + i%4; its sign is bit 8(i%4) + 2(i//4) + grp%2 of the word at 512 + 16g + 4u
     w = np.zeros((32, 96), np.int8)
-    w[5, 3 * 7: 3 * 7 + 3] = (-1, 1, 0)     # v = -9 + 3 = -6 -> index 6, sign 1
-    w[31, 3 * 30: 3 * 30 + 3] = (0, 1, -1)  # v = 2 -> index 2, sign 0
+    w[5, 3 * 7: 3 * 7 + 3] = (-1, 1, 0)     # v = -9 + 3 = -6 -> index 6, sign 1; row 5 = (g 5, u 0), byte i = 3
+    w[31, 3 * 30: 3 * 30 + 3] = (0, 1, -1)  # v = 2 -> index 2, sign 0; row 31 = (g 7, u 3), byte i = 15
     p = oracle.pack_tl("tl2", w)
     expect = np.zeros(640, np.uint8)
-    expect[16 * 5 + 3] = 6 << 4
-    expect[512 + 4 * 5 + 0] = 1 << 7
-    expect[16 * 31 + 15] = 2
+    expect[64 * 5 + 3] = 6 << 4
+    expect[512 + 16 * 5 + 3] = 1 << 1       # bit 8*3 + 2*0 + 1 = 25
+    expect[64 * 7 + 16 * 3 + 4 * 3 + 3] = 2
     assert np.array_equal(p, expect)
+
+
+def test_tl2_tile_read_back_by_the_inverse_statement():
+    """The layout stated the other way round -- which (row, triple) a byte / a sign bit of the tile holds: byte p of
+    the index plane holds index byte 4*((p%64)//16) + p%4 of row p//64 + 8*((p%16)//4); bit b of the sign word at
+    512 + 4*s holds the sign of triple 2*(4*((b%8)//2) + b//8) + b%2 of row s//4 + 8*(s%4).  Every position of a
+    random tile is decoded that way and compared with the codes of Table 5 computed from the weights."""
+    w = rand_ternary(32, 96)
+    p = oracle.pack_tl("tl2", w)
+    v = 9 * w[:, 0::3].astype(int) + 3 * w[:, 1::3] + w[:, 2::3]          # [32][32]
+    for pos in range(512):
+        row, i = pos // 64 + 8 * ((pos % 16) // 4), 4 * ((pos % 64) // 16) + pos % 4
+        assert p[pos] & 15 == abs(v[row, 2 * i]) and p[pos] >> 4 == abs(v[row, 2 * i + 1])
+    for s_ in range(32):
+        word = int.from_bytes(bytes(p[512 + 4 * s_: 516 + 4 * s_]), "little")
+        row = s_ // 4 + 8 * (s_ % 4)
+        for b in range(32):
+            grp = 2 * (4 * ((b % 8) // 2) + b // 8) + b % 2
+            assert (word >> b) & 1 == int(v[row, grp] < 0)
 
 
 def test_tl1_documented_byte_positions_and_padding():
     w = np.zeros((32, 34), np.int8)         # 17 pairs, tile padded to 32 pairs with code 4
-    w[2, 0:2] = (1, -1)                     # code 6, pair 0 -> low nibble of byte 32
-    w[2, 32:34] = (-1, -1)                  # code 0, pair 16 -> low nibble of byte 40
+    w[2, 0:2] = (1, -1)                     # code 6, pair 0 -> low nibble of index byte 0 of row 2 = (g 2, u 0)
+    w[2, 32:34] = (-1, -1)                  # code 0, pair 16 -> low nibble of index byte 8 (word 2, byte 0)
+    w[26, 2:4] = (1, 1)                     # code 8, pair 1 -> high nibble of index byte 0 of row 26 = (g 2, u 3)
     p = oracle.pack_tl("tl1", w)
     expect = np.full(512, 0x44, np.uint8)
-    expect[16 * 2 + 0] = 0x46
-    expect[16 * 2 + 8] = 0x40
+    expect[64 * 2 + 0] = 0x46
+    expect[64 * 2 + 16 * 2 + 0] = 0x40
+    expect[64 * 2 + 4 * 3 + 0] = 0x84
     assert np.array_equal(p, expect)
 
 
