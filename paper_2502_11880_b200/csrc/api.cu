@@ -196,6 +196,13 @@ static bool mid_takes(int64_t T, int64_t M, int64_t K, const void* workspace, si
   return use_mid(T, M, K) && workspace && gemv_i2s_mid_workspace_bytes((int)T, M, K) <= workspace_bytes;
 }
 
+// TL2 decode batches go to the scan kernel (decode table + tensor cores) unless BITNET_TL2=lut asks for the
+// activation-table form of Alg. 2 / Alg. 4, or the shape does not fit it.
+static bool tl2_scan_takes(int fmt, int64_t T, int64_t M, int64_t K, const TlGeom& g) {
+  static const bool lut_only = [] { const char* e = getenv("BITNET_TL2"); return e && strcmp(e, "lut") == 0; }();
+  return !lut_only && fmt == BITNET_FMT_TL2 && T >= 1 && T <= 8 && gemv_tl2_scan_item_supported((int)T, M, K, g);
+}
+
 size_t bitnet_mpgemm_workspace_bytes(bitnet_fmt_t fmt, int64_t T, int64_t M, int64_t K) {
   if (T < 1 || M < 1 || K < 1) return 0;
   if (fmt == BITNET_FMT_I2S) {
@@ -243,8 +250,24 @@ int bitnet_mpgemm(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
   if (rc) return rc;
   for (int64_t t0 = 0; t0 < T; t0 += 8) {
     const int nt = (int)((T - t0 < 8) ? (T - t0) : 8);
-    rc = launch_gemv_tl(fmt, (const uint8_t*)packed, w_scale, M, K, g, q + t0 * K, act_scale + t0, nt,
-                        y + t0 * M, acc_out ? acc_out + t0 * M : nullptr, workspace, workspace_bytes, st);
+    if (tl2_scan_takes(fmt, nt, M, K, g)) {
+      Tl2Linear it;
+      it.packed = (const uint8_t*)packed;
+      it.x = nullptr;
+      it.q = const_cast<int8_t*>(q + t0 * K);
+      it.act_scale = const_cast<float*>(act_scale + t0);
+      it.y = y + t0 * M;
+      it.acc_out = acc_out ? acc_out + t0 * M : nullptr;
+      it.w_scale = w_scale;
+      it.T = nt;
+      it.M = M;
+      it.K = K;
+      it.g = g;
+      rc = launch_gemv_tl2_scan(&it, 1, st);
+    } else {
+      rc = launch_gemv_tl(fmt, (const uint8_t*)packed, w_scale, M, K, g, q + t0 * K, act_scale + t0, nt,
+                          y + t0 * M, acc_out ? acc_out + t0 * M : nullptr, workspace, workspace_bytes, st);
+    }
     if (rc) return rc;
   }
   return BITNET_OK;
@@ -273,6 +296,26 @@ int bitnet_linear(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
     if (!no_fuse && T <= fuse_max && gemv_i2s_stream_supported((int)T, M, K, true))
       return launch_gemv_i2s_stream((const uint8_t*)packed, w_scale, M, K, x, q, act_scale, (int)T, y, acc_out,
                                     (cudaStream_t)stream);
+  }
+  if (fmt == BITNET_FMT_TL2 && T <= 8) {
+    TlGeom g;
+    int rc = tl_shape(fmt, M, K, bk3, &g);
+    if (rc) return rc;
+    if (tl2_scan_takes(fmt, T, M, K, g)) {       // one kernel: quantiser fused
+      Tl2Linear it;
+      it.packed = (const uint8_t*)packed;
+      it.x = x;
+      it.q = q;
+      it.act_scale = act_scale;
+      it.y = y;
+      it.acc_out = acc_out;
+      it.w_scale = w_scale;
+      it.T = (int)T;
+      it.M = M;
+      it.K = K;
+      it.g = g;
+      return launch_gemv_tl2_scan(&it, 1, (cudaStream_t)stream);
+    }
   }
   int rc = bitnet_quant_act(x, T, K, 0, q, act_scale, nullptr, stream);
   if (rc) return rc;
@@ -317,7 +360,35 @@ int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* strea
     return grouped && d.fmt == BITNET_FMT_I2S && d.T <= 8 && gemv_i2s_group_item_supported((int)d.T, d.M, d.K);
   };
   static thread_local std::vector<GroupLinear> run;
+  static thread_local std::vector<Tl2Linear> run2;
+  auto takes2 = [&](const bitnet_group_item_t& d, TlGeom* g) {
+    return grouped && d.fmt == BITNET_FMT_TL2 && tl_shape(d.fmt, d.M, d.K, d.bk3, g) == BITNET_OK &&
+           tl2_scan_takes(d.fmt, d.T, d.M, d.K, *g);
+  };
   for (int64_t i = 0; i < n;) {
+    TlGeom g2;
+    if (takes2(items[i], &g2)) {
+      run2.clear();
+      for (; i < n && takes2(items[i], &g2); ++i) {
+        const bitnet_group_item_t& d = items[i];
+        Tl2Linear it;
+        it.packed = (const uint8_t*)d.packed;
+        it.x = d.x;
+        it.q = d.q;
+        it.act_scale = d.act_scale;
+        it.y = d.y;
+        it.acc_out = d.acc_out;
+        it.w_scale = d.w_scale;
+        it.T = (int)d.T;
+        it.M = d.M;
+        it.K = d.K;
+        it.g = g2;
+        run2.push_back(it);
+      }
+      int rc = launch_gemv_tl2_scan(run2.data(), (int64_t)run2.size(), (cudaStream_t)stream);
+      if (rc) return rc;
+      continue;
+    }
     if (!takes(items[i])) {
       const bitnet_group_item_t& d = items[i];
       int rc = bitnet_linear((bitnet_fmt_t)d.fmt, d.packed, d.w_scale, d.M, d.K, d.bk3, d.x, d.T, d.q, d.act_scale, d.y,

@@ -119,6 +119,22 @@ struct GroupLinear {
 };
 bool gemv_i2s_group_item_supported(int T, int64_t M, int64_t K);
 int launch_gemv_i2s_group(const GroupLinear* items, int64_t n, cudaStream_t st);
+// One persistent kernel over a list of TL2 linears (1..8 tokens each): packed indices decoded through a shared-memory
+// table into tensor-core operands.
+struct Tl2Linear {
+  const uint8_t* packed;
+  const float* x;      // fp32 activations [T][K] (q, act_scale are then outputs); null: q, act_scale are inputs
+  int8_t* q;
+  float* act_scale;
+  float* y;
+  int32_t* acc_out;    // nullable
+  float w_scale;
+  int T;
+  int64_t M, K;
+  TlGeom g;
+};
+bool gemv_tl2_scan_item_supported(int T, int64_t M, int64_t K, const TlGeom& g);
+int launch_gemv_tl2_scan(const Tl2Linear* items, int64_t n, cudaStream_t st);
 // Batches of 9 to 64 tokens: mma.sync over K-slices, partial sums through a [T][M] int32 workspace when K is
 // cut into more than one slice (gemv_i2s_mid_workspace_bytes says how much; 0 = none needed).
 bool gemv_i2s_mid_supported(int T, int64_t M, int64_t K);

@@ -156,3 +156,51 @@ def test_group_rejects_malformed_items():
     grp[0].y = None
     with pytest.raises(bn.BitnetError, match="invalid"):
         bn.bitnet_linear_group(grp)
+
+
+def test_group_tl2_items_through_the_scan_kernel():
+    """TL2 items (decode table + tensor cores): block-fitting splits with no, one and two pair tiles in the tail,
+    every token count, rows a multiple of 32 only, items sharing an input, an I2_S item in between."""
+    x = synth.normal(9, 1, 2, 4096)
+    items = [Item("tl2", 64, 96 * 12, 1, 700), Item("tl2", 320, 3200, 3, 701), Item("tl2", 96, 8640, 4, 702),
+             Item("tl2", 4096, 4096, 2, 703, x=x), Item("tl2", 2048, 4096, 2, 704, x=x), Item("i2s", 64, 2048, 1, 705),
+             Item("tl2", 32, 8192, 8, 706), Item("tl2", 160, 28672, 1, 707), Item("tl2", 64, 96 * 20 + 92, 5, 708)]
+    items[4].xd = items[3].xd
+    run_group(items)
+    for it in items:
+        it.check()
+
+
+def test_group_tl2_workload_layer():
+    """A 100B-shaped decoder layer in the TL2 encoding at one token through the grouped call (one persistent scan
+    kernel): sampled rows of every linear against the oracle, and the whole vectors against the I2_S result."""
+    wl = synth.CONFIGS["sweep100b"]
+    rng = np.random.default_rng(11)
+    for j, lin in enumerate(wl.linears):
+        wd = wl.weights(5, j, device="cuda")
+        x = wl.activations(5, j, 1)
+        rows = np.unique(np.concatenate([[0, 31, 32, lin.M - 1], rng.integers(0, lin.M, 96)]))
+        w_rows = np.stack([wl.weights(5, j, row_start=int(r), rows=1).numpy()[0] for r in rows])
+        outs = {}
+        for fmt in ("tl2", "i2s"):
+            blob = bn.pack(fmt, wd, check=False)
+            q = torch.empty((1, lin.K), dtype=torch.int8, device="cuda")
+            sc = torch.empty(1, dtype=torch.float32, device="cuda")
+            y = torch.empty((1, lin.M), dtype=torch.float32, device="cuda")
+            acc = torch.empty((1, lin.M), dtype=torch.int32, device="cuda")
+            grp = bn.make_group([dict(fmt=fmt, packed=blob, w_scale=0.625, M=lin.M, K=lin.K, x=x.cuda(), q=q, act_scale=sc,
+                                      y=y, acc_out=acc)])
+            bn.bitnet_linear_group(grp)
+            torch.cuda.synchronize()
+            outs[fmt] = (y, acc, q, sc)
+            del blob
+        y, acc, q, sc = outs["tl2"]
+        q_ref, sc_ref, _ = oracle.quant_act(x.numpy())
+        assert np.array_equal(npy(q), q_ref)
+        acc_ref = oracle.mpgemm_def(q_ref, np.ascontiguousarray(w_rows))
+        assert np.array_equal(npy(acc)[:, rows], acc_ref)
+        check_y(y[:, torch.as_tensor(rows).cuda()], acc_ref, sc_ref, 0.625)
+        assert torch.equal(acc, outs["i2s"][1]) and torch.equal(y, outs["i2s"][0])
+        del wd
+        torch.cuda.empty_cache()
+    assert bn.bitnet_device_status() == 0
