@@ -37,10 +37,10 @@ METRIC = "mpgemv_weight_stream_batch1"
 UNIT = "GB/s"
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one captured launch of the decode kernel (K=8192 -> M=57344:
-# 117.542 MB read + 3.72 MB written) over the packed weight bytes of that launch (117.44 MB).  Traffic grows
-# in proportion to the weights streamed, so the same ratio scales it to the sweep's average launch.
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = (117.542 + 3.72) / 117.440
+# dram__bytes_read.sum + dram__bytes_write.sum of one captured launch of the grouped decode kernel over 4 layers of
+# the sweep (856.571 MB read + 4.369 MB written) over the packed weight bytes of that launch (855.638 MB).  Traffic
+# grows in proportion to the weights streamed, so the same ratio scales it to the full launch.
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = (856.571 + 4.369) / 855.638
 
 def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -553,10 +553,20 @@ def run_ours(args):
                                        "launch": f"{g_full.n_graphs} CUDA graph replays per step, one fused kernel per linear"}
         del g_full
         if "tl2" in fmts:
+            # the same sweep in the TL2 encoding: (a) the scan kernel (decode table + tensor cores, one persistent
+            # kernel per step), (b) the activation-table kernel of Alg. 2 (three launches per linear)
             ms_tl = time_replays(torch, lambda: sw.step_group("tl2"), max(5, args.steps // 2), args.warmup)
+            bn.bitnet_set_tl2_lookup(True)
+            ms_lut = time_replays(torch, lambda: sw.step_group("tl2"), max(3, args.steps // 5), args.warmup)
+            bn.bitnet_set_tl2_lookup(False)
             line["tl2"] = {"packed_bytes": sw.bytes["tl2"], "ms_per_step": ms_tl, "value": sw.bytes["tl2"] / ms_tl / 1e6,
                            "unit": UNIT, "frac_of_hbm_peak": sw.bytes["tl2"] / ms_tl / 1e6 / pk["hbm"],
-                           "i2s_equivalent_GBps": sw.bytes["i2s"] / ms_tl / 1e6}
+                           "i2s_equivalent_GBps": sw.bytes["i2s"] / ms_tl / 1e6,
+                           "kernel": "gemv_tl2_scan_kernel (one bitnet_linear_group call per step)",
+                           "lookup_table_kernel": {"ms_per_step": ms_lut, "value": sw.bytes["tl2"] / ms_lut / 1e6,
+                                                   "frac_of_hbm_peak": sw.bytes["tl2"] / ms_lut / 1e6 / pk["hbm"],
+                                                   "kernel": "quantiser + tl_table_kernel + gemv_tl_kernel per linear"}}
+            sw.step_group("tl2")        # the verification below sees the scan kernel's y
         if not args.skip_batched:
             line["batched_decode"] = {
                 "note": "the same sweep with T tokens per linear, one bitnet_linear_group call per step, inputs resident",

@@ -69,6 +69,18 @@ int bitnet_device_status(int* status_out);
 void bitnet_set_early_start(int enable);
 
 /*
+ * Which kernel serves TL2 batches of up to 8 tokens (process-wide; also set by BITNET_TL2=lut in the environment).
+ *   0 (default): the scan kernel -- every packed index byte plus its sign bits is resolved by one shared-memory
+ *      table lookup into the weights it stands for (Table 5), which go through the int8 tensor cores; about
+ *      3.5 times the rate of the other form on a B200.  Shapes it does not take (K not a multiple of 4, fewer
+ *      than three 96-column tiles per warp, more codes than fit beside its 128 KB table) fall back to the other form.
+ *   1: the element-wise lookup-table kernel of Alg. 2 / Alg. 4 as the paper states it -- per-token tables of
+ *      activation partial sums, one lookup, conditional negate and add per packed index.
+ * Both give the same integers.  TL1 always runs the lookup-table kernel.
+ */
+void bitnet_set_tl2_lookup(int enable);
+
+/*
  * Activation quantiser -- Alg. 1 Phase 1 ("Quantization"), Sec. 2.1 and 3.2.2: absmax int8.
  *   x[T][K] fp32 row-major (read)  ->  q[T][K] int8, act_scale[T] fp32, act_sum[T] int32 (nullable).
  * Per token t: amax = max(max_k |x[t,k]|, 1e-5); s = 127/amax (binary32); q = clamp(rint(x*s),

@@ -26,7 +26,7 @@ SYMBOLS = [
     "bitnet_pack_i2s", "bitnet_tl_packed_bytes", "bitnet_pack_tl", "bitnet_mpgemm_workspace_bytes",
     "bitnet_workspace_init", "bitnet_mpgemm", "bitnet_linear", "bitnet_linear_host", "bitnet_linear_host_batch", "bitnet_unpack_i2s", "bitnet_unpack_tl",
     "bitnet_tl_num_groups", "bitnet_tl_build_lut_debug", "bitnet_mpgemv_tl_noalloc", "bitnet_device_status",
-    "bitnet_set_early_start", "bitnet_linear_group",
+    "bitnet_set_early_start", "bitnet_set_tl2_lookup", "bitnet_linear_group",
 ]
 
 _lib = None
@@ -51,6 +51,8 @@ def lib():
         L.bitnet_device_status.argtypes = [vp]
         L.bitnet_set_early_start.argtypes = [ci]
         L.bitnet_set_early_start.restype = None
+        L.bitnet_set_tl2_lookup.argtypes = [ci]
+        L.bitnet_set_tl2_lookup.restype = None
         L.bitnet_quant_act.argtypes = [vp, i64, i64, ci, vp, vp, vp, vp]
         L.bitnet_i2s_packed_bytes.argtypes = [i64, i64]
         L.bitnet_i2s_packed_bytes.restype = sz
@@ -89,6 +91,11 @@ def bitnet_device_status() -> int:
 
 def bitnet_set_early_start(enable: bool):
     lib().bitnet_set_early_start(int(bool(enable)))
+
+
+def bitnet_set_tl2_lookup(enable: bool):
+    """True: TL2 decode batches run the activation-table kernel of Alg. 2 instead of the scan kernel."""
+    lib().bitnet_set_tl2_lookup(int(bool(enable)))
 
 
 def _check(rc: int, what: str):

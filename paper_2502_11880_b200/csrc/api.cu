@@ -20,6 +20,7 @@ int note_cuda_error(cudaError_t e) {
 }
 
 static int g_early_start = 1;
+static int g_tl2_lookup = [] { const char* e = getenv("BITNET_TL2"); return (e && strcmp(e, "lut") == 0) ? 1 : 0; }();
 bool early_start_enabled() { return g_early_start != 0; }
 
 bool log_enabled() {
@@ -100,6 +101,7 @@ int bitnet_device_status(int* status_out) {
 }
 
 void bitnet_set_early_start(int enable) { g_early_start = enable ? 1 : 0; }
+void bitnet_set_tl2_lookup(int enable) { bitnet::g_tl2_lookup = enable ? 1 : 0; }
 
 int bitnet_quant_act(const float* x, int64_t T, int64_t K, int per_tensor, int8_t* q, float* act_scale,
                      int32_t* act_sum, void* stream) {
@@ -199,8 +201,7 @@ static bool mid_takes(int64_t T, int64_t M, int64_t K, const void* workspace, si
 // TL2 decode batches go to the scan kernel (decode table + tensor cores) unless BITNET_TL2=lut asks for the
 // activation-table form of Alg. 2 / Alg. 4, or the shape does not fit it.
 static bool tl2_scan_takes(int fmt, int64_t T, int64_t M, int64_t K, const TlGeom& g) {
-  static const bool lut_only = [] { const char* e = getenv("BITNET_TL2"); return e && strcmp(e, "lut") == 0; }();
-  return !lut_only && fmt == BITNET_FMT_TL2 && T >= 1 && T <= 8 && gemv_tl2_scan_item_supported((int)T, M, K, g);
+  return !bitnet::g_tl2_lookup && fmt == BITNET_FMT_TL2 && T >= 1 && T <= 8 && gemv_tl2_scan_item_supported((int)T, M, K, g);
 }
 
 size_t bitnet_mpgemm_workspace_bytes(bitnet_fmt_t fmt, int64_t T, int64_t M, int64_t K) {

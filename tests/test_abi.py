@@ -77,8 +77,15 @@ def test_host_validation_returns_codes_without_a_gpu(L):
     assert L.bitnet_mpgemm(0, fake, 1.0, 64, 100, 0, fake, fake, 1, fake, null, null, 0, null) == 2
     assert L.bitnet_mpgemm(0, fake, 1.0, 64, 128, 0, fake, fake, 0, fake, null, null, 0, null) == 1
     assert L.bitnet_mpgemm(0, fake, 1.0, 64, 128, 0, odd, fake, 1, fake, null, null, 0, null) == 1
-    # split-K shape without a workspace
-    assert L.bitnet_mpgemm(2, fake, 1.0, 64, 28672, 0, fake, fake, 1, fake, null, null, 0, null) == 3
+    # lookup-table kernel (TL1 always runs it) without the workspace it keeps its tables in
+    assert L.bitnet_mpgemm(1, fake, 1.0, 64, 28672, 0, fake, fake, 1, fake, null, null, 0, null) == 3
+    # bitnet_linear validates the shape before it plans a launch (K = 0 or negative must not reach a division)
+    for T in (1, 6, 8):
+        assert L.bitnet_linear(0, fake, 1.0, 64, 0, 0, fake, T, fake, fake, fake, null, fake, 1 << 20, null) == 1
+        assert L.bitnet_linear(0, fake, 1.0, 64, -16, 0, fake, T, fake, fake, fake, null, fake, 1 << 20, null) == 1
+    # the grouped call rejects a malformed list before anything is queued
+    assert L.bitnet_linear_group(null, 1, null) == 1
+    assert L.bitnet_linear_group(null, 0, null) == 0
     assert L.bitnet_mpgemm(1, fake, 1.0, 32, 64, 0, fake, fake, 1, fake, null, fake, 16, null) == 3   # too small
 
 
