@@ -41,7 +41,7 @@ namespace {
 constexpr int CW = 16;  // warps
 constexpr int THREADS = CW * 32;
 constexpr int XREG = 16;                       // float4 registers per thread of the quantiser's one-pass form
-constexpr int NSMALL = 56, NLARGE = 454;       // items per launch: argument blocks of 4 KB / 32 KB
+constexpr int NSMALL = 50, NLARGE = 409;       // items per launch: argument blocks of 4 KB / 32 KB
 constexpr size_t MAX_CODE_BYTES = 144 * 1024;  // staged activation codes of one item
 
 struct GItem {
@@ -55,8 +55,10 @@ struct GItem {
   int M, K, T;
   int first_unit;      // units of the items before this one
   int first_w;         // 1-KB chunks of the items before this one
+  int nparts;          // K is walked in this many parts (1 unless the staged codes of a whole row do not fit)
+  int pad;
 };
-static_assert(sizeof(GItem) == 72, "argument block layout");
+static_assert(sizeof(GItem) == 80, "argument block layout");
 
 template <int NMAX>
 struct GArgs {
@@ -67,18 +69,22 @@ struct GArgs {
 static_assert(sizeof(GArgs<NSMALL>) <= 4096 && sizeof(GArgs<NLARGE>) <= 32764, "kernel parameter limits");
 
 __device__ __forceinline__ bool same_input(const GItem& p, const GItem& d) {
-  return p.K == d.K && p.T == d.T && (d.x ? p.x == d.x : (p.x == nullptr && p.q == d.q && p.act_scale == d.act_scale));
+  return p.nparts == 1 && d.nparts == 1 && p.K == d.K && p.T == d.T &&
+         (d.x ? p.x == d.x : (p.x == nullptr && p.q == d.q && p.act_scale == d.act_scale));
 }
 
-// Stages the item's activation codes (T rows, kp + 16 bytes apart, zero beyond K) and, per token, the scale
-// and the sum of the codes.  Called by all threads; contains barriers.
-__device__ __forceinline__ void stage_item(const GItem& d, bool owner, int kp, int8_t* qs_mem, float* qscale,
-                                           int* qsum, float* qred) {
+// Stages the activation codes of the item's columns [256 c0, 256 c1) (T rows, qst bytes apart, zero beyond K) and,
+// per token, the scale and the sum of the staged codes.  `first` = the item's first part: the row maximum is taken
+// (Alg. 1 Phase 1) and, in the CTA that owns the item, codes and scales of the WHOLE row go to the caller; later
+// parts reuse the multiplier kept in qmul.  Called by all threads; contains barriers.
+__device__ __forceinline__ void stage_item(const GItem& d, bool owner, bool first, int c0, int c1, int qst, int8_t* qs_mem,
+                                           float* qscale, float* qmul, int* qsum, float* qred) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int qst = kp + 16, n4 = d.K / 4, kw = kp / 4;
+  const int n4 = d.K / 4, w0 = c0 * 64, w1 = c1 * 64;       // staged words [w0, w1) of a row
   if (threadIdx.x < 8) qsum[threadIdx.x] = 0;
-  if (d.x && d.K <= 4 * XREG * THREADS) {
-    // Alg. 1 Phase 1, one round trip per token: s = 127 / max(amax, 1e-5), q = clamp(rint(x * s))
+  if (d.x && first && d.K <= 4 * XREG * THREADS) {
+    // one round trip per token: s = 127 / max(amax, 1e-5), q = clamp(rint(x * s)); the row stays in registers
+    const int kw = (int)(i2s_kp(d.K) / 4);
     const int nrow = (kw + THREADS - 1) / THREADS;
     for (int tok = 0; tok < d.T; ++tok) {
       const float4* x4 = reinterpret_cast<const float4*>(d.x + (int64_t)tok * d.K);
@@ -105,6 +111,7 @@ __device__ __forceinline__ void stage_item(const GItem& d, bool owner, int kp, i
       if (threadIdx.x == 0) {
         const float inv = __fdiv_rn(amax_c, 127.0f);
         qscale[tok] = inv;
+        qmul[tok] = sq;
         if (owner) d.act_scale[tok] = inv;
       }
       int s = 0;
@@ -113,8 +120,10 @@ __device__ __forceinline__ void stage_item(const GItem& d, bool owner, int kp, i
         const int i = threadIdx.x + r * THREADS;
         if (r < nrow && i < kw) {
           const int word = quant4_packed(xv[r], sq);  // columns K..Kp-1 came in as zeros
-          reinterpret_cast<int*>(qs_mem + tok * qst)[i] = word;
-          s = __dp4a(word, 0x01010101, s);
+          if (i >= w0 && i < w1) {
+            reinterpret_cast<int*>(qs_mem + tok * qst)[i - w0] = word;
+            s = __dp4a(word, 0x01010101, s);
+          }
           if (owner && i < n4) reinterpret_cast<int*>(d.q + (int64_t)tok * d.K)[i] = word;
         }
       }
@@ -123,39 +132,44 @@ __device__ __forceinline__ void stage_item(const GItem& d, bool owner, int kp, i
       if (lane == 0) atomicAdd(qsum + tok, s);
     }
   } else if (d.x) {
-    // rows too long for the registers: amax per token, then a second pass over x
-    for (int tok = 0; tok < d.T; ++tok) {
-      const float4* x4 = reinterpret_cast<const float4*>(d.x + (int64_t)tok * d.K);
-      float m = 0.0f;
-      for (int i = threadIdx.x; i < n4; i += THREADS) m = fmaxf(m, absmax4(__ldcg(x4 + i)));
+    if (first) {
+      // rows too long for the registers: amax per token first
+      for (int tok = 0; tok < d.T; ++tok) {
+        const float4* x4 = reinterpret_cast<const float4*>(d.x + (int64_t)tok * d.K);
+        float m = 0.0f;
+        for (int i = threadIdx.x; i < n4; i += THREADS) m = fmaxf(m, absmax4(__ldcg(x4 + i)));
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-      if (lane == 0) qred[tok * CW + warp] = m;
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (lane == 0) qred[tok * CW + warp] = m;
+      }
+      __syncthreads();
+      if (threadIdx.x < d.T) {
+        float m = 0.0f;
+        for (int w2 = 0; w2 < CW; ++w2) m = fmaxf(m, qred[threadIdx.x * CW + w2]);
+        const float amax_c = fmaxf(m, 1e-5f);
+        const float inv = __fdiv_rn(amax_c, 127.0f);
+        qscale[threadIdx.x] = inv;
+        qmul[threadIdx.x] = __fdiv_rn(127.0f, amax_c);
+        if (owner) d.act_scale[threadIdx.x] = inv;
+      }
     }
     __syncthreads();
-    if (threadIdx.x < d.T) {
-      float m = 0.0f;
-      for (int w2 = 0; w2 < CW; ++w2) m = fmaxf(m, qred[threadIdx.x * CW + w2]);
-      const float amax_c = fmaxf(m, 1e-5f);
-      const float inv = __fdiv_rn(amax_c, 127.0f);
-      qscale[threadIdx.x] = inv;
-      if (owner) d.act_scale[threadIdx.x] = inv;
-    }
-    __syncthreads();
+    // quantise: the staged columns into shared memory; in the owning CTA's first part every column for the caller
+    const int lo = (owner && first) ? 0 : w0, hi = (owner && first) ? max(w1, n4) : w1;
     for (int tok = 0; tok < d.T; ++tok) {
-      float m = 0.0f;
-      for (int w2 = 0; w2 < CW; ++w2) m = fmaxf(m, qred[tok * CW + w2]);
-      const float sq = __fdiv_rn(127.0f, fmaxf(m, 1e-5f));
+      const float sq = qmul[tok];
       const float4* x4 = reinterpret_cast<const float4*>(d.x + (int64_t)tok * d.K);
       int s = 0;
-      for (int i = threadIdx.x; i < kw; i += THREADS) {
+      for (int i = lo + threadIdx.x; i < hi; i += THREADS) {
         int word = 0;
         if (i < n4) {
           word = quant4_packed(__ldcg(x4 + i), sq);
-          if (owner) reinterpret_cast<int*>(d.q + (int64_t)tok * d.K)[i] = word;
+          if (owner && first) reinterpret_cast<int*>(d.q + (int64_t)tok * d.K)[i] = word;
         }
-        reinterpret_cast<int*>(qs_mem + tok * qst)[i] = word;
-        s = __dp4a(word, 0x01010101, s);
+        if (i >= w0 && i < w1) {
+          reinterpret_cast<int*>(qs_mem + tok * qst)[i - w0] = word;
+          s = __dp4a(word, 0x01010101, s);
+        }
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
@@ -167,9 +181,9 @@ __device__ __forceinline__ void stage_item(const GItem& d, bool owner, int kp, i
     for (int tok = 0; tok < d.T; ++tok) {
       const int* qrow = reinterpret_cast<const int*>(d.q + (int64_t)tok * d.K);
       int s = 0;
-      for (int i = threadIdx.x; i < kw; i += THREADS) {
+      for (int i = w0 + threadIdx.x; i < w1; i += THREADS) {
         const int word = (i < n4) ? __ldcg(qrow + i) : 0;
-        reinterpret_cast<int*>(qs_mem + tok * qst)[i] = word;
+        reinterpret_cast<int*>(qs_mem + tok * qst)[i - w0] = word;
         s = __dp4a(word, 0x01010101, s);
       }
 #pragma unroll
@@ -185,8 +199,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
   extern __shared__ __align__(128) uint8_t smem[];
   int* hdr = reinterpret_cast<int*>(smem);             // [0] first unit, [1] end unit, [2] first item, [3] last item
   float* qscale = reinterpret_cast<float*>(smem + 64);  // [8] act_scale per token
-  int* qsum = reinterpret_cast<int*>(smem + 96);        // [8] sum of the codes per token
+  int* qsum = reinterpret_cast<int*>(smem + 96);        // [8] sum of the staged codes per token
   float* qred = reinterpret_cast<float*>(smem + 128);   // [8][16] partial maxima
+  float* qmul = reinterpret_cast<float*>(smem + 640);   // [8] 127 / amax per token
   int* red = reinterpret_cast<int*>(smem + 1024);       // [CW][2][tmax][16] partial sums
   int8_t* qs_mem = reinterpret_cast<int8_t*>(smem + 1024 + CW * 2 * a.tmax * 16 * 4);
   uint8_t* rings = reinterpret_cast<uint8_t*>(qs_mem) + a.code_bytes;
@@ -223,27 +238,50 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
   const uint64_t pol = policy_evict_first();
   const uint32_t ring = smem_u32(rings + (size_t)warp * DEPTH * 1024) + lane * 16;
 
-  // ---------------- where the group's next unit lies: a cursor over the items that runs one unit ahead
-  int n_item = item0, n_first = 0, n_end = 0, n_ub = 0;
-  const uint8_t* n_base = nullptr;
-  auto n_load = [&](int i) {
+  // ---------------- the group's sequence of jobs.  Within the CTA's range, item i contributes the units
+  // [max(jb, first_i), min(je, end_i)); the group takes every G-th of them starting at its own index, once per
+  // part of the item's K.  A job is (item, part, unit).
+  auto item_end = [&](int i) { return (i + 1 < a.n) ? a.it[i + 1].first_unit : a.total_units; };
+  auto range_lo = [&](int i) { const int f = a.it[i].first_unit; return (f > jb ? f : jb) + gi; };
+  auto range_hi = [&](int i) { const int e = item_end(i); return e < je ? e : je; };
+  // first chunk of this warp's slice of (item i, part p, unit job)
+  auto job_ptr = [&](int i, int p, int job) -> const uint8_t* {
     const GItem& d = a.it[i];
     const int kp = (int)i2s_kp(d.K), nch = kp / 256;
-    n_ub = 4 * kp;
-    n_first = d.first_unit;
-    n_end = (i + 1 < a.n) ? a.it[i + 1].first_unit : a.total_units;
-    n_base = d.packed + (int64_t)(wk * nch / S) * 1024 + lane * 16;
+    const int c0 = p * nch / d.nparts, npc = (p + 1) * nch / d.nparts - c0;
+    return d.packed + (int64_t)(job - d.first_unit) * (4 * kp) + (int64_t)(c0 + wk * npc / S) * 1024 + lane * 16;
   };
-  // first chunk of this warp's slice of unit `job` (job < je, jobs asked for in ascending order)
-  auto job_ptr = [&](int job) -> const uint8_t* {
-    while (job >= n_end) n_load(++n_item);
-    return n_base + (int64_t)(job - n_first) * n_ub;
+  // the job after (i, p, job) in this group's sequence; false if there is none
+  auto next_job = [&](int& i, int& p, int& job) -> bool {
+    if (job + G < range_hi(i)) {
+      job += G;
+      return true;
+    }
+    if (p + 1 < a.it[i].nparts) {
+      ++p;
+      job = range_lo(i);
+      return true;
+    }
+    for (++i; i <= item1; ++i)
+      if (range_lo(i) < range_hi(i)) {
+        p = 0;
+        job = range_lo(i);
+        return true;
+      }
+    return false;
   };
-  n_load(item0);
-  int cj = jb + gi, nloc = 0;
-  const uint8_t* cur = (cj < je) ? job_ptr(cj) : nullptr;
+  int ni = item0 - 1, np = 0, nj = 0;     // (item, part, unit) of the job whose first chunks enter the ring next
+  bool more = false;
+  for (int i = item0; i <= item1 && !more; ++i)
+    if (range_lo(i) < range_hi(i)) {
+      ni = i;
+      np = 0;
+      nj = range_lo(i);
+      more = true;
+    }
+  const uint8_t* cur = more ? job_ptr(ni, np, nj) : nullptr;
   // Weights depend on nothing an earlier kernel writes: fill the ring before waiting for that kernel.  Every
-  // slice of every item is at least DEPTH chunks long (the host chooses S and DEPTH that way).
+  // slice of every part of every item is at least DEPTH chunks long (the host chooses S and DEPTH that way).
 #pragma unroll
   for (int d = 0; d < DEPTH; ++d) {
     if (cur) {
@@ -257,118 +295,131 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
 
   // ---------------- consume
   uint32_t slot_off = 0;
+  int nloc = 0;
   const int tmax = a.tmax;
+  bool staged_any = false;
   for (int ci = item0; ci <= item1; ++ci) {
     const GItem& d = a.it[ci];
-    const int T = d.T, kp = (int)i2s_kp(d.K), nch = kp / 256, qst = kp + 16;
+    const int T = d.T, kp = (int)i2s_kp(d.K), nch = kp / 256, nparts = d.nparts;
+    const int qst = ((nch + nparts - 1) / nparts) * 256 + 16;
     const bool owner = jb <= d.first_unit;
-    if (ci == item0 || !same_input(a.it[ci - 1], d)) {
-      if (ci > item0) __syncthreads();  // everyone is done with the previous item's codes
-      stage_item(d, owner, kp, qs_mem, qscale, qsum, qred);
-      __syncthreads();
-    } else if (owner && d.x && d.q != a.it[ci - 1].q) {
-      // same input as the previous item but its own output buffers for the codes
-      for (int tok = 0; tok < T; ++tok)
-        for (int i = threadIdx.x; i < d.K / 4; i += THREADS)
-          reinterpret_cast<int*>(d.q + (int64_t)tok * d.K)[i] = reinterpret_cast<const int*>(qs_mem + tok * qst)[i];
-      if (threadIdx.x < T) d.act_scale[threadIdx.x] = qscale[threadIdx.x];
-    }
-    const int c_lo = wk * nch / S, c_hi = (wk + 1) * nch / S, nw = c_hi - c_lo;
-    const int iend = (ci + 1 < a.n) ? a.it[ci + 1].first_unit : a.total_units;
-    const int cend = je < iend ? je : iend;
+    const int jlo = range_lo(ci), jhi = range_hi(ci);
     const int first = d.first_unit, M = d.M;
     const unsigned has_tok = g < T ? 1u : 0u;
-    const uint32_t q_lane = smem_u32(qs_mem + min(g, T - 1) * qst + c_lo * 256 + t * 64);
     const float w_scale = d.w_scale;
     float* const y = d.y;
     int32_t* const acc_out = d.acc_out;
+    for (int part = 0; part < nparts; ++part) {
+      const int c0 = part * nch / nparts, c1 = (part + 1) * nch / nparts, npc = c1 - c0;
+      if (!staged_any || part > 0 || !same_input(a.it[ci - 1], d)) {
+        if (staged_any) __syncthreads();  // everyone is done with the codes staged before (and with y as scratch)
+        stage_item(d, owner, part == 0, c0, c1, qst, qs_mem, qscale, qmul, qsum, qred);
+        __syncthreads();
+        staged_any = true;
+      } else if (owner && d.x && d.q != a.it[ci - 1].q) {
+        // same input as the previous item but its own output buffers for the codes
+        for (int tok = 0; tok < T; ++tok)
+          for (int i = threadIdx.x; i < d.K / 4; i += THREADS)
+            reinterpret_cast<int*>(d.q + (int64_t)tok * d.K)[i] = reinterpret_cast<const int*>(qs_mem + tok * qst)[i];
+        if (threadIdx.x < T) d.act_scale[threadIdx.x] = qscale[threadIdx.x];
+      }
+      const int s_lo = wk * npc / S, nw = (wk + 1) * npc / S - s_lo;
+      const uint32_t q_lane = smem_u32(qs_mem + min(g, T - 1) * qst + s_lo * 256 + t * 64);
+      const bool last_part = part + 1 == nparts;
 
-    for (; cj < cend; cj += G, ++nloc) {
-      int C[4][4];
+      for (int cj = jlo; cj < jhi; cj += G, ++nloc) {
+        int C[4][4];
 #pragma unroll
-      for (int s = 0; s < 4; ++s)
+        for (int s = 0; s < 4; ++s)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) C[s][i] = 0;
-      uint32_t qp = q_lane;
-      int qr[8] = {0, 0, 0, 0, 0, 0, 0, 0};  // B registers; lanes beyond the batch keep these zeros
-      // One step: wait for the oldest chunk of the ring, put it through the tensor cores, then refill its slot
-      // from `pf` (the chunk DEPTH places further down the warp's stream), if there is one.
-      auto step = [&](const uint8_t* pf, bool do_pf) {
-        cp_wait<DEPTH - 1>();
-        unsigned w4[4], v4[4];
-        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                     : "=r"(w4[0]), "=r"(w4[1]), "=r"(w4[2]), "=r"(w4[3])
-                     : "r"(ring + slot_off));
-        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                     : "=r"(v4[0]), "=r"(v4[1]), "=r"(v4[2]), "=r"(v4[3])
-                     : "r"(ring + slot_off + 512));
+          for (int i = 0; i < 4; ++i) C[s][i] = 0;
+        uint32_t qp = q_lane;
+        int qr[8] = {0, 0, 0, 0, 0, 0, 0, 0};  // B registers; lanes beyond the batch keep these zeros
+        // One step: wait for the oldest chunk of the ring, put it through the tensor cores, then refill its slot
+        // from `pf` (the chunk DEPTH places further down the warp's stream), if there is one.
+        auto step = [&](const uint8_t* pf, bool do_pf) {
+          cp_wait<DEPTH - 1>();
+          unsigned w4[4], v4[4];
+          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                       : "=r"(w4[0]), "=r"(w4[1]), "=r"(w4[2]), "=r"(w4[3])
+                       : "r"(ring + slot_off));
+          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                       : "=r"(v4[0]), "=r"(v4[1]), "=r"(v4[2]), "=r"(v4[3])
+                       : "r"(ring + slot_off + 512));
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          // only the lanes whose B column is a real token load activations
-          asm volatile(
-              "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %9, 0;\n\t"
-              "@p ld.shared.v4.u32 {%0,%1,%2,%3}, [%8];\n\t"
-              "@p ld.shared.v4.u32 {%4,%5,%6,%7}, [%8+16];\n\t}"
-              : "+r"(qr[0]), "+r"(qr[1]), "+r"(qr[2]), "+r"(qr[3]), "+r"(qr[4]), "+r"(qr[5]), "+r"(qr[6]), "+r"(qr[7])
-              : "r"(qp + h * 32), "r"(has_tok));
+          for (int h = 0; h < 2; ++h) {
+            // only the lanes whose B column is a real token load activations
+            asm volatile(
+                "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %9, 0;\n\t"
+                "@p ld.shared.v4.u32 {%0,%1,%2,%3}, [%8];\n\t"
+                "@p ld.shared.v4.u32 {%4,%5,%6,%7}, [%8+16];\n\t}"
+                : "+r"(qr[0]), "+r"(qr[1]), "+r"(qr[2]), "+r"(qr[3]), "+r"(qr[4]), "+r"(qr[5]), "+r"(qr[6]), "+r"(qr[7])
+                : "r"(qp + h * 32), "r"(has_tok));
 #pragma unroll
-          for (int s = 0; s < 4; ++s) {
-            const unsigned m = 0x03030303u << (2 * s);
-            mma_u8s8(C[s], w4[2 * h] & m, v4[2 * h] & m, w4[2 * h + 1] & m, v4[2 * h + 1] & m, qr[2 * s], qr[2 * s + 1]);
+            for (int s = 0; s < 4; ++s) {
+              const unsigned m = 0x03030303u << (2 * s);
+              mma_u8s8(C[s], w4[2 * h] & m, v4[2 * h] & m, w4[2 * h + 1] & m, v4[2 * h + 1] & m, qr[2 * s], qr[2 * s + 1]);
+            }
           }
-        }
-        qp += 256;
-        // the chunk's bytes were in registers before the MMAs were issued: its slot can be refilled
-        if (do_pf) {
-          cp16(ring + slot_off, pf, pol);
-          cp16(ring + slot_off + 512, pf + 512, pol);
-        }
-        cp_commit();
-        slot_off = (slot_off + 1024 == DEPTH * 1024) ? 0 : slot_off + 1024;
-      };
+          qp += 256;
+          // the chunk's bytes were in registers before the MMAs were issued: its slot can be refilled
+          if (do_pf) {
+            cp16(ring + slot_off, pf, pol);
+            cp16(ring + slot_off + 512, pf + 512, pol);
+          }
+          cp_commit();
+          slot_off = (slot_off + 1024 == DEPTH * 1024) ? 0 : slot_off + 1024;
+        };
 
-      // chunks 0 .. nw-DEPTH-1 are followed, DEPTH places on, by chunks of the same unit; the last DEPTH chunks by
-      // the first DEPTH chunks of the group's next unit (in this item or a later one), if there is one
-      const int nj = cj + G;
-      const bool more = nj < je;
-      const uint8_t* const nxt = more ? job_ptr(nj) : cur;
-      const uint8_t* pf = cur + DEPTH * 1024;
+        // chunks 0 .. nw-DEPTH-1 are followed, DEPTH places on, by chunks of the same slice; the last DEPTH chunks by
+        // the first DEPTH chunks of the group's next job (this item's next unit or part, or a later item), if any
+        more = next_job(ni, np, nj);
+        const uint8_t* const nxt = more ? job_ptr(ni, np, nj) : cur;
+        const uint8_t* pf = cur + DEPTH * 1024;
 #pragma unroll 2
-      for (int left = nw - DEPTH; left > 0; --left, pf += 1024) step(pf, true);
+        for (int left = nw - DEPTH; left > 0; --left, pf += 1024) step(pf, true);
 #pragma unroll
-      for (int dd = 0; dd < DEPTH; ++dd) step(nxt + dd * 1024, more);
-      cur = nxt;
+        for (int dd = 0; dd < DEPTH; ++dd) step(nxt + dd * 1024, more);
+        cur = nxt;
 
-      // fragment: c[0] = (row g, token 2t), c[1] = (row g, token 2t+1), c[2], c[3] = the same for row g+8
-      int c[4];
+        // fragment: c[0] = (row g, token 2t), c[1] = (row g, token 2t+1), c[2], c[3] = the same for row g+8
+        int c[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) c[i] = C[0][i] + (C[1][i] >> 2) + (C[2][i] >> 4) + (C[3][i] >> 6);
-      int* mine = red + ((warp * 2 + (nloc & 1)) * tmax) * 16;
-      if (2 * t < T) {
-        mine[(2 * t) * 16 + g] = c[0];
-        mine[(2 * t) * 16 + g + 8] = c[2];
-      }
-      if (2 * t + 1 < T) {
-        mine[(2 * t + 1) * 16 + g] = c[1];
-        mine[(2 * t + 1) * 16 + g + 8] = c[3];
-      }
-      if (S > 1) group_barrier(1 + gi, S * 32);
-      else __syncwarp();
-      if (wk == (nloc & (S - 1))) {
-        // this unit's turn to be finished by this warp: add the group's partials, rescale, store 16 rows
-        const int row0 = (cj - first) * 16;
-        const int* grp = red + (((gi * S) * 2 + (nloc & 1)) * tmax) * 16;
+        for (int i = 0; i < 4; ++i) c[i] = C[0][i] + (C[1][i] >> 2) + (C[2][i] >> 4) + (C[3][i] >> 6);
+        int* mine = red + ((warp * 2 + (nloc & 1)) * tmax) * 16;
+        if (2 * t < T) {
+          mine[(2 * t) * 16 + g] = c[0];
+          mine[(2 * t) * 16 + g + 8] = c[2];
+        }
+        if (2 * t + 1 < T) {
+          mine[(2 * t + 1) * 16 + g] = c[1];
+          mine[(2 * t + 1) * 16 + g + 8] = c[3];
+        }
+        if (S > 1) group_barrier(1 + gi, S * 32);
+        else __syncwarp();
+        if (wk == (nloc & (S - 1))) {
+          // this unit's turn to be finished by this warp: add the group's partials; the sums of an item walked in
+          // parts rest in y (as integers) between the parts; the last part rescales and stores 16 rows
+          const int row0 = (cj - first) * 16;
+          const int* grp = red + (((gi * S) * 2 + (nloc & 1)) * tmax) * 16;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int idx = lane + 32 * i;
-          if (idx < T * 16) {
-            int v = 0;
-            for (int w2 = 0; w2 < S; ++w2) v += grp[w2 * 2 * tmax * 16 + idx];
-            const int tok = idx >> 4, row = row0 + (idx & 15);
-            v -= qsum[tok];
-            if (row < M) {
-              y[(int64_t)tok * M + row] = __fmul_rn((float)v, __fmul_rn(qscale[tok], w_scale));
-              if (acc_out) acc_out[(int64_t)tok * M + row] = v;
+          for (int i = 0; i < 4; ++i) {
+            const int idx = lane + 32 * i;
+            if (idx < T * 16) {
+              int v = 0;
+              for (int w2 = 0; w2 < S; ++w2) v += grp[w2 * 2 * tmax * 16 + idx];
+              const int tok = idx >> 4, row = row0 + (idx & 15);
+              v -= qsum[tok];
+              if (row < M) {
+                float* const yp = y + (int64_t)tok * M + row;
+                if (part > 0) v += __ldcg(reinterpret_cast<const int*>(yp));
+                if (last_part) {
+                  *yp = __fmul_rn((float)v, __fmul_rn(qscale[tok], w_scale));
+                  if (acc_out) acc_out[(int64_t)tok * M + row] = v;
+                } else {
+                  *reinterpret_cast<int*>(yp) = v;
+                }
+              }
             }
           }
         }
@@ -414,9 +465,33 @@ Shape shape_for(int64_t nch) {
   return Shape{S, depth};
 }
 
-size_t code_bytes_of(int T, int64_t K) { return ((size_t)T * (size_t)(i2s_kp(K) + 16) + 127) & ~(size_t)127; }
 size_t smem_of(int tmax, size_t code_bytes, int depth) {
   return 1024 + (size_t)CW * 2 * tmax * 16 * 4 + code_bytes + (size_t)CW * depth * 1024;
+}
+
+// How one item is walked: in `nparts` parts of its K (as few as let the staged codes of a part, T rows of at most
+// ceil(nch / nparts) chunks, fit beside a ring of at least 6 chunks per warp -- 4 if nothing else fits); `code` =
+// bytes of the staged codes of its largest part, `npc` = chunks of its smallest part.
+struct ItemPlan {
+  int nparts;
+  size_t code;
+  int64_t npc;
+};
+bool plan_item(int T, int64_t M, int64_t K, ItemPlan* out) {
+  if (T < 1 || T > 8 || M < 1 || K < 1 || (K % 64) != 0 || M > 0x7fffffff) return false;
+  const int64_t nch = i2s_kp(K) / 256;
+  const size_t cap = (size_t)dev_info().max_smem_optin;
+  for (int want_depth = 6; want_depth >= 4; want_depth -= 2)
+    for (int n = 1; n <= 8; ++n) {
+      const int64_t big = ceil_div(nch, n), small = nch / n;
+      if (small < 4) break;
+      const size_t code = ((size_t)T * (size_t)(big * 256 + 16) + 127) & ~(size_t)127;
+      if (code <= MAX_CODE_BYTES && smem_of(T, code, want_depth) <= cap) {
+        *out = ItemPlan{n, code, small};
+        return true;
+      }
+    }
+  return false;
 }
 
 template <int DEPTH, int NMAX>
@@ -455,7 +530,19 @@ int launch_depth(const GArgs<NMAX>& a, int depth, int grid, size_t smem, cudaStr
   }
 }
 
-// One launch over items of one shape class (the same S and ring depth suit all of them).
+// S and ring depth for a launch whose shortest part has `npc` chunks, whose largest batch is `tmax` tokens and
+// whose largest staged codes take `code` bytes; false if they do not fit one SM's shared memory.
+bool launch_shape(int64_t npc, int tmax, size_t code, Shape* out) {
+  if (npc < 4 || code > MAX_CODE_BYTES) return false;
+  Shape sh = shape_for(npc);
+  const size_t cap = (size_t)dev_info().max_smem_optin;
+  while (sh.depth > 4 && smem_of(tmax, code, sh.depth) > cap) sh.depth = sh.depth == 12 ? 8 : sh.depth - 2;
+  if (smem_of(tmax, code, sh.depth) > cap) return false;
+  *out = sh;
+  return true;
+}
+
+// One launch over `n` items with the given shape.
 template <int NMAX>
 int launch_run(const GroupLinear* items, int n, Shape shape, cudaStream_t st) {
   static thread_local GArgs<NMAX> a;   // 32 KB: off the stack
@@ -467,6 +554,8 @@ int launch_run(const GroupLinear* items, int n, Shape shape, cudaStream_t st) {
   for (int i = 0; i < n; ++i) {
     const GroupLinear& s = items[i];
     GItem& d = a.it[i];
+    ItemPlan pl;
+    if (!plan_item(s.T, s.M, s.K, &pl)) return BITNET_ERR_UNSUPPORTED_SHAPE;
     d.packed = s.packed;
     d.x = s.x;
     d.q = s.q;
@@ -479,12 +568,13 @@ int launch_run(const GroupLinear* items, int n, Shape shape, cudaStream_t st) {
     d.T = s.T;
     d.first_unit = (int)units;
     d.first_w = (int)w;
+    d.nparts = pl.nparts;
+    d.pad = 0;
     const int64_t nu = ceil_div(s.M, 16), nch = i2s_kp(s.K) / 256;
     units += nu;
     w += nu * nch;
     if (s.T > a.tmax) a.tmax = s.T;
-    const size_t cb = code_bytes_of(s.T, s.K);
-    if (cb > code) code = cb;
+    if (pl.code > code) code = pl.code;
   }
   a.total_units = (int)units;
   a.total_w = (int)w;
@@ -501,43 +591,31 @@ int launch_run(const GroupLinear* items, int n, Shape shape, cudaStream_t st) {
   return launch_depth<NMAX>(a, depth, grid, smem, st);
 }
 
-// S and ring depth for a launch over items whose shortest rows have `nch` chunks, whose largest batch is `tmax`
-// tokens and whose largest staged codes take `code` bytes; false if they do not fit one SM's shared memory.
-bool launch_shape(int64_t nch, int tmax, size_t code, Shape* out) {
-  if (nch < 4 || code > MAX_CODE_BYTES) return false;
-  Shape sh = shape_for(nch);
-  const size_t cap = (size_t)dev_info().max_smem_optin;
-  while (sh.depth > 4 && smem_of(tmax, code, sh.depth) > cap) sh.depth = sh.depth == 12 ? 8 : sh.depth - 2;
-  if (smem_of(tmax, code, sh.depth) > cap) return false;
-  *out = sh;
-  return true;
-}
-
 }  // namespace
 
 bool gemv_i2s_group_item_supported(int T, int64_t M, int64_t K) {
-  if (T < 1 || T > 8 || M < 1 || K < 1 || (K % 64) != 0 || M > 0x7fffffff) return false;
+  ItemPlan pl;
   Shape sh;
-  return launch_shape(i2s_kp(K) / 256, T, code_bytes_of(T, K), &sh);
+  return plan_item(T, M, K, &pl) && launch_shape(pl.npc, T, pl.code, &sh);
 }
 
 // Launches the grouped kernel over `n` supported items: as few launches as the argument block (NLARGE items,
-// 2^30 chunks) and shared memory (the largest batch and the longest rows of a launch set its code area) allow.
-// A launch runs with the warps per unit and ring depth that suit its shortest rows.
+// 2^30 chunks) and shared memory (the largest batch and the longest part of a launch set its code area) allow.
+// A launch runs with the warps per unit and ring depth that suit its shortest part.
 int launch_gemv_i2s_group(const GroupLinear* items, int64_t n, cudaStream_t st) {
   int64_t i = 0;
   while (i < n) {
-    int64_t j = i, w = 0, nch_min = 1 << 30;
+    int64_t j = i, w = 0, npc_min = 1 << 30;
     int tmax = 1;
     size_t code = 0;
     Shape sh{1, 4};
     while (j < n && j - i < NLARGE) {
-      const int64_t nch = i2s_kp(items[j].K) / 256;
-      const int64_t add = ceil_div(items[j].M, 16) * nch;
-      const size_t cb = code_bytes_of(items[j].T, items[j].K);
+      ItemPlan pl;
+      if (!plan_item(items[j].T, items[j].M, items[j].K, &pl)) return BITNET_ERR_UNSUPPORTED_SHAPE;
+      const int64_t add = ceil_div(items[j].M, 16) * (i2s_kp(items[j].K) / 256);
       const int tm = items[j].T > tmax ? items[j].T : tmax;
-      const size_t cm = cb > code ? cb : code;
-      const int64_t nm = nch < nch_min ? nch : nch_min;
+      const size_t cm = pl.code > code ? pl.code : code;
+      const int64_t nm = pl.npc < npc_min ? pl.npc : npc_min;
       Shape sj;
       const bool fits = launch_shape(nm, tm, cm, &sj);
       if (!fits && j == i) return BITNET_ERR_UNSUPPORTED_SHAPE;
@@ -545,7 +623,7 @@ int launch_gemv_i2s_group(const GroupLinear* items, int64_t n, cudaStream_t st) 
       w += add;
       tmax = tm;
       code = cm;
-      nch_min = nm;
+      npc_min = nm;
       sh = sj;
       ++j;
     }

@@ -204,3 +204,18 @@ def test_group_tl2_workload_layer():
         del wd
         torch.cuda.empty_cache()
     assert bn.bitnet_device_status() == 0
+
+
+def test_group_long_rows_walked_in_parts():
+    """Batches whose staged codes of a whole row do not fit in shared memory: the CTA walks the item's K in two or
+    three parts, the integer sums resting in y between the parts.  Part sizes that do not divide the row evenly, a
+    ragged last 16-row unit, several units per warp group, and neighbours of other shapes on either side."""
+    shapes = [(40, 2048, 2), (1000, 28672, 8), (70, 29440, 8), (520, 28672, 5), (33, 14336, 8), (48, 28672, 6), (64, 8192, 8)]
+    items = [Item("i2s", M, K, T, 800 + i) for i, (M, K, T) in enumerate(shapes)]
+    run_group(items)
+    for it in items:
+        it.check()
+    # the same list once more into the same buffers (y held integer scratch in between: no stale state may survive)
+    run_group(items)
+    for it in items:
+        it.check()
