@@ -68,14 +68,6 @@ static_assert(STAGES % UNPACK_GROUPS == 0, "a stage always belongs to the same g
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 static __device__ int g_prefill_error = 0;
-#ifdef BITNET_PROFILE_PREFILL
-__device__ long long g_pprof[8];   // MMA thread of CTA 0: [0] wait tmem_empty, [1] wait for the stage's operands, [2] unused, [3] issue, [4] total
-#define PP_T(v) const long long v = clock64()
-#define PP_ADD(i, x0, x1) if (blockIdx.x == 0) g_pprof[i] += (x1) - (x0)
-#else
-#define PP_T(v)
-#define PP_ADD(i, x0, x1)
-#endif
 
 struct PrefillArgs {
   const uint8_t* packed;
@@ -247,25 +239,16 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       uint32_t it = 0, nt = 0;
-      PP_T(pstart);
       for (int item = blockIdx.x; item < nitems && !*abort_flag; item += gridDim.x, ++nt) {
         const int buf = nt % NACC;
         const int kb_lo = kb_lo_of(item), kb_hi = kb_hi_of(item);
-        PP_T(p0);
         bool ok = mbar_wait(&bars->tmem_empty[buf], ((nt / NACC) & 1u) ^ 1u, abort_flag);
-        PP_T(p1);
-        PP_ADD(0, p0, p1);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t d_tmem = tmem_base + buf * TILE_T;
         for (int kb = kb_lo; ok && kb < kb_hi; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t par = (it / STAGES) & 1u;
-          PP_T(q0);
           ok = mbar_wait(&bars->full_a[s], par, abort_flag);   // weights unpacked and activations landed
-          PP_T(q1);
-          PP_T(q2);
-          PP_ADD(1, q0, q1);
-          PP_ADD(2, q1, q2);
           if (!ok) break;
           const uint64_t adesc = make_desc(smem_u32(tileA + s * A_BYTES));
           const uint64_t bdesc = make_desc(smem_u32(tileB + s * B_BYTES));
@@ -277,8 +260,6 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
               umma_i8(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, (kb > kb_lo || k4 > 0) ? 1u : 0u);
           }
           umma_commit(&bars->empty[s]);            // stage reusable once these MMAs have read it
-          PP_T(q3);
-          PP_ADD(3, q2, q3);
         }
         if (!ok) {
           atomicExch(&g_prefill_error, BITNET_ERR_TIMEOUT);
@@ -287,8 +268,6 @@ gemm_i2s_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_consta
         }
         umma_commit(&bars->tmem_full[buf]);        // accumulator complete
       }
-      PP_T(pend);
-      PP_ADD(4, pstart, pend);
     }
   } else if (warp < 2 + UNPACK_WARPS * UNPACK_GROUPS) {
     // ------------------------------------------------------------ unpackers: weight rows (operand A)
@@ -597,14 +576,6 @@ int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int
   return launch_rescale_sums(a.ws, act_scale, w_scale, T, M, y, acc_out, st);
 }
 
-#ifdef BITNET_PROFILE_PREFILL
-extern "C" int bitnet_debug_prefill_profile(long long* out, int reset) {
-  cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(out, g_pprof, sizeof(long long) * 8);
-  if (reset) { long long z[8] = {0}; cudaMemcpyToSymbol(g_pprof, z, sizeof(z)); }
-  return 0;
-}
-#endif
 
 int gemm_prefill_status(int* out) {
   cudaError_t e = cudaMemcpyFromSymbol(out, g_prefill_error, sizeof(int));

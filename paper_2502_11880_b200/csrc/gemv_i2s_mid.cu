@@ -377,7 +377,7 @@ struct MidPlan {
 };
 
 bool make_mid_plan(int T, int64_t M, int64_t K, MidPlan* p) {
-  if (T < 1 || T > 64 || (K % 16) != 0 || M < 1) return false;
+  if (T < 1 || T > 64 || K < 16 || (K % 16) != 0 || M < 1) return false;   // (K < 1 would leave no chunk to slice)
   p->c = mid_cfg(T);
   const int TP = p->c.NT * 8;
   p->nchunks = (int)(i2s_kp(K) / 256);
@@ -399,7 +399,7 @@ bool make_mid_plan(int T, int64_t M, int64_t K, MidPlan* p) {
     const int idle = sms - (int)(cps * cand);
     if (idle < best_idle) best_idle = idle, ns = cand;
   }
-  const int forced = env_int("BITNET_MID_NS", 0);
+  static const int forced = env_int("BITNET_MID_NS", 0);   // read once
   if (forced >= ns_min && forced <= p->nchunks && forced <= sms) ns = forced;
   p->NS = ns;
   p->cps = (int)(items < sms / ns ? items : sms / ns);

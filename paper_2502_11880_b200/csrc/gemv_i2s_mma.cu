@@ -53,21 +53,6 @@ constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 static __device__ int g_stream_error = 0;
 
-#ifdef BITNET_PROFILE_GEMV
-// Development aid (never in the shipped build): per launch and CTA, %globaltimer at a few points.
-static __device__ unsigned long long g_tl[256][148][6];
-static int g_tl_launch = 0;
-__device__ __forceinline__ unsigned long long gtime() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-#define TL_MARK(i) do { if (blockIdx.x < 148) g_tl[a.launch_id & 255][blockIdx.x][i] = gtime(); } while (0)
-#define TL_MAX(i) do { if (blockIdx.x < 148) atomicMax(&g_tl[a.launch_id & 255][blockIdx.x][i], gtime()); } while (0)
-#else
-#define TL_MARK(i) do { } while (0)
-#define TL_MAX(i) do { } while (0)
-#endif
 
 struct MmaArgs {
   const uint8_t* packed;
@@ -92,7 +77,6 @@ struct MmaArgs {
   int ngroups;           // warp groups; group g takes the CTA's units g, g + ngroups, ...
   int nunits;            // ceil(M / 16)
   int slots;             // ring slots
-  int launch_id;         // profiling builds only
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -194,8 +178,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_mma_kernel(const MmaArgs 
   };
 
   if (threadIdx.x == 0) {
-    TL_MARK(0);
-    if (blockIdx.x < 148) { TL_MARK(5); }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may begin its prologue
     for (int s = 0; s < a.slots; ++s) mbar_init(smem_u32(full + s), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -214,7 +196,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_mma_kernel(const MmaArgs 
 
   // ---------------- activations come from the previous kernel in the stream
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (threadIdx.x == 0) TL_MARK(1);
 
   if (a.use_qs) {
     if (a.x && a.T == 1 && a.K <= 4 * XREG * THREADS) {
@@ -303,7 +284,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_mma_kernel(const MmaArgs 
     }
     __syncthreads();
   }
-  if (threadIdx.x == 0) TL_MARK(2);
   if (idle) return;
 
   // rescale factors of the tokens this lane stores when its warp finishes a unit (token (lane>>4) + 2i)
@@ -371,7 +351,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_mma_kernel(const MmaArgs 
         if (lane == 0) atomicExch(&g_stream_error, BITNET_ERR_TIMEOUT);
         return;
       }
-      if (threadIdx.x == 0 && seq == 0) TL_MARK(3);
       const uint8_t* pa = ring + lane_off + slot * a.stage_bytes;
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
@@ -453,8 +432,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_mma_kernel(const MmaArgs 
       if (lane == 0) atomicExch(cnt + e, 0);
     }
   }
-  if (threadIdx.x == 0) TL_MARK(4);
-  if (lane == 0) TL_MAX(5);
 }
 
 struct Plan {
@@ -565,10 +542,6 @@ int launch_gemv_i2s_stream(const uint8_t* packed, float w_scale, int64_t M, int6
   a.ngroups = p.ngroups;
   a.nunits = p.nunits;
   a.slots = p.slots;
-  a.launch_id = 0;
-#ifdef BITNET_PROFILE_GEMV
-  a.launch_id = g_tl_launch++;
-#endif
   switch (p.KS) {
     case 1: return launch_mma<1>(a, p, st);
     case 2: return launch_mma<2>(a, p, st);
@@ -583,16 +556,5 @@ int gemv_i2s_stream_status(int* out) {
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
 }
 
-#ifdef BITNET_PROFILE_GEMV
-extern "C" int bitnet_debug_timeline(unsigned long long* out, int reset) {
-  if (reset) {
-    g_tl_launch = 0;
-    void* p = nullptr;
-    cudaGetSymbolAddress(&p, g_tl);
-    return (int)cudaMemset(p, 0, sizeof(g_tl));
-  }
-  return (int)cudaMemcpyFromSymbol(out, g_tl, sizeof(g_tl));
-}
-#endif
 
 }  // namespace bitnet

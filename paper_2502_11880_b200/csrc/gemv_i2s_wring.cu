@@ -45,29 +45,8 @@ constexpr int JQ = 4;                    // entries of a group's queue of upcomi
 constexpr int XREG_MAX = 16;                 // float4 registers per thread of the fused quantiser's fast path
 constexpr size_t MAX_QS_BYTES = 144 * 1024;   // activations staged in shared memory up to this size
 
-#ifdef BITNET_PROFILE_GEMV
-// Development aid (never in the shipped build): per launch and CTA, %globaltimer at a few points.
-static __device__ unsigned long long g_tl[256][148][6];
-static int g_tl_launch = 0;
-__device__ __forceinline__ unsigned long long gtime() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-static __device__ unsigned long long g_steps[256][4][24];
-#define TL_STEP(i) do { if ((blockIdx.x % 37) == 0 && blockIdx.x < 148 && threadIdx.x == 0 && n == 0 && (i) < 24) g_steps[a.launch_id & 255][blockIdx.x / 37][i] = gtime(); } while (0)
-#define TL_PRO(i) do { if ((blockIdx.x % 37) == 0 && blockIdx.x < 148 && threadIdx.x == 0) g_steps[a.launch_id & 255][blockIdx.x / 37][i] = gtime(); } while (0)
-#define TL_MARK(i) do { if (blockIdx.x < 148) g_tl[a.launch_id & 255][blockIdx.x][i] = gtime(); } while (0)
-#define TL_MAX(i) do { if (blockIdx.x < 148) atomicMax(&g_tl[a.launch_id & 255][blockIdx.x][i], gtime()); } while (0)
-#else
-#define TL_MARK(i) do { } while (0)
-#define TL_MAX(i) do { } while (0)
-#define TL_STEP(i) do { } while (0)
-#define TL_PRO(i) do { } while (0)
-#endif
 
 struct WArgs {
-  int launch_id;         // profiling builds only
   const uint8_t* packed;
   int64_t unit_bytes;    // bytes of one 16-row unit of the blob = 4 * Kp
   int M;
@@ -157,8 +136,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
   const int c_lo = wk * a.nchunks / a.S, c_hi = (wk + 1) * a.nchunks / a.S;   // this warp's K-slice, >= DEPTH chunks
 
   if (threadIdx.x == 0) {
-    TL_MARK(0);
-    TL_MARK(5);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may become resident
     *counter = 2 * G;
   }
@@ -201,8 +178,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
 
   // ---------------- activations come from the previous kernel in the stream
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (threadIdx.x == 0) TL_MARK(1);
-  TL_PRO(17);
 
   if (a.x && a.K <= 4 * XREG * THREADS) {
     // ---- fused quantiser (Alg. 1 Phase 1), one round trip per token: the row stays in registers
@@ -230,18 +205,15 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
         load_row(xv, tok);
       }
       if (tok == 0) first_fill(false);
-      TL_PRO(18);
       float m = 0.0f;
 #pragma unroll
       for (int r = 0; r < XREG; ++r)
         if (r < nrow) m = fmaxf(m, fmaxf(fmaxf(fabsf(xv[r].x), fabsf(xv[r].y)), fmaxf(fabsf(xv[r].z), fabsf(xv[r].w))));
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-      TL_PRO(19);
       if (tok > 0) __syncthreads();          // everyone has read the previous token's partial maxima
       if (lane == 0) qred[warp] = m;
       __syncthreads();
-      TL_PRO(20);
       float amax = 0.0f;
 #pragma unroll
       for (int w2 = 0; w2 < CW; ++w2) amax = fmaxf(amax, qred[w2]);
@@ -329,8 +301,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
   }
   __syncthreads();
 
-  if (threadIdx.x == 0) TL_MARK(2);
-  TL_PRO(21);
   // sum of the activations of tokens 2t and 2t+1 over this warp's K-slice (the "- sum(q)" term)
   int corr_even = 0, corr_odd = 0;
   for (int tok = 0; tok < a.T; ++tok) {
@@ -350,7 +320,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
     if (tok == 2 * t) corr_even = s;
     if (tok == 2 * t + 1) corr_odd = s;
   }
-  TL_PRO(22);
   // token g's codes under this lane's 16-byte weight column: 64 bytes per chunk
   const unsigned has_tok = g < a.T ? 1u : 0u;
   const uint32_t q_lane = smem_u32(qs_mem + min(g, a.T - 1) * qst + c_lo * 256 + t * 64);
@@ -412,19 +381,17 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
 #pragma unroll
       for (int i = 0; i < 4; ++i) C[s][i] = 0;
     qp = q_lane;
-    TL_STEP(0);
 
     // chunks 0 .. nw-DEPTH-1 are followed, DEPTH places on, by chunks of the same unit
     const uint8_t* pf = base + (int64_t)j * unit_stride + DEPTH * 1024;
 #pragma unroll 2
-    for (int left = nw - DEPTH; left > 0; --left, pf += 1024) { step(pf, true); TL_STEP(nw - DEPTH - left + 1); }
+    for (int left = nw - DEPTH; left > 0; --left, pf += 1024) { step(pf, true); }
     // the last DEPTH chunks by the first DEPTH chunks of the group's next unit, if there is one
     pf = base + (int64_t)jn * unit_stride;
     const bool more = jn < n_units;
 #pragma unroll
-    for (int d = 0; d < DEPTH; ++d) { step(pf + d * 1024, more); TL_STEP(nw - DEPTH + d + 1); }
+    for (int d = 0; d < DEPTH; ++d) { step(pf + d * 1024, more); }
 
-    if (threadIdx.x == 0 && n == 0) TL_MARK(3);
     // fragment: c[0] = (row g, token 2t), c[1] = (row g, token 2t+1), c[2], c[3] = the same for row g+8
     int c[4];
 #pragma unroll
@@ -460,8 +427,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
     }
   }
   cp_wait<0>();
-  if (threadIdx.x == 0) TL_MARK(4);
-  if (lane == 0) TL_MAX(5);
 }
 
 struct Plan {
@@ -469,14 +434,25 @@ struct Plan {
   size_t smem;
 };
 
-int env_int(const char* name, int dflt) {
-  const char* v = getenv(name);
-  return (v && *v) ? atoi(v) : dflt;
+// Tuning overrides from the environment, read once per process (never on the launch path again).
+struct Tuning {
+  int depth, kc, ctas, pre;
+};
+const Tuning& tuning() {
+  static const Tuning t = [] {
+    auto env_int = [](const char* name, int dflt) {
+      const char* v = getenv(name);
+      return (v && *v) ? atoi(v) : dflt;
+    };
+    return Tuning{env_int("BITNET_I2S_DEPTH", 0), env_int("BITNET_I2S_KC", 8), env_int("BITNET_I2S_CTAS", 1),
+                  env_int("BITNET_I2S_PRE", 4)};
+  }();
+  return t;
 }
 
 bool make_plan(int T, int64_t M, int64_t K, Plan* p) {
   p->nchunks = (int)(i2s_kp(K) / 256);
-  const int forced = env_int("BITNET_I2S_DEPTH", 0);
+  const int forced = tuning().depth;
   int depth = (forced == 12 || forced == 8 || forced == 6 || forced == 4) ? forced : 8;
   while (depth > 4 && 2048 + red_bytes(T) + (((size_t)T * (p->nchunks * 256 + 16) + 127) & ~(size_t)127) +
                               (size_t)CW * depth * 1024 > (size_t)dev_info().max_smem_optin)
@@ -484,14 +460,14 @@ bool make_plan(int T, int64_t M, int64_t K, Plan* p) {
   if (depth == 10) depth = 8;
   if (p->nchunks < depth) return false;     // a warp's slice is at least as long as the ring
   // warps per unit: as many as leave every warp about kc_target chunks of a unit (never fewer than the ring)
-  int kc_target = env_int("BITNET_I2S_KC", 8);
+  int kc_target = tuning().kc;
   if (kc_target < depth) kc_target = depth;
   int S = 1;
   while (S < CW && p->nchunks / (2 * S) >= kc_target) S *= 2;
   p->S = S;
   p->KC = (p->nchunks + S - 1) / S;
   p->nunits = (int)ceil_div(M, 16);
-  const int ctas = dev_info().sm_count * env_int("BITNET_I2S_CTAS", 1);
+  const int ctas = dev_info().sm_count * tuning().ctas;
   p->grid = ctas < p->nunits ? ctas : p->nunits;
   const size_t qs_bytes = ((size_t)T * (p->nchunks * 256 + 16) + 127) & ~(size_t)127;
   if (qs_bytes > MAX_QS_BYTES) return false;
@@ -538,10 +514,6 @@ int launch_gemv_i2s_wring(const uint8_t* packed, float w_scale, int64_t M, int64
   Plan p;
   if (T < 1 || T > 8 || !make_plan(T, M, K, &p)) return BITNET_ERR_UNSUPPORTED_SHAPE;
   WArgs a;
-  a.launch_id = 0;
-#ifdef BITNET_PROFILE_GEMV
-  a.launch_id = g_tl_launch++;
-#endif
   a.packed = packed;
   a.unit_bytes = 4 * i2s_kp(K);
   a.M = (int)M;
@@ -559,7 +531,7 @@ int launch_gemv_i2s_wring(const uint8_t* packed, float w_scale, int64_t M, int64
   a.S = p.S;
   a.KC = p.KC;
   a.nunits = p.nunits;
-  a.pre = env_int("BITNET_I2S_PRE", 4);
+  a.pre = tuning().pre;
   // short rows get the instance whose (fully unrolled) quantiser prologue is a quarter of the code
   log_launch("gemv_i2s_wring_kernel%s T=%d M=%lld K=%lld grid=%d warps/unit=%d ring=%d smem=%zu", x ? " (fused quantiser)" : "",
              T, (long long)M, (long long)K, p.grid, p.S, p.depth, p.smem);
@@ -573,19 +545,5 @@ int launch_gemv_i2s_wring(const uint8_t* packed, float w_scale, int64_t M, int64
   }
 }
 
-#ifdef BITNET_PROFILE_GEMV
-extern "C" int bitnet_debug_steps_w(unsigned long long* out) {
-  return (int)cudaMemcpyFromSymbol(out, g_steps, sizeof(g_steps));
-}
-extern "C" int bitnet_debug_timeline_w(unsigned long long* out, int reset) {
-  if (reset) {
-    g_tl_launch = 0;
-    void* p = nullptr;
-    cudaGetSymbolAddress(&p, g_tl);
-    return (int)cudaMemset(p, 0, sizeof(g_tl));
-  }
-  return (int)cudaMemcpyFromSymbol(out, g_tl, sizeof(g_tl));
-}
-#endif
 
 }  // namespace bitnet

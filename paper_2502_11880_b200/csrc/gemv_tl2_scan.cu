@@ -536,8 +536,15 @@ struct Shape {
 };
 // S and ring depth for a launch whose shortest rows have `t3` triple tiles: every warp's run of triple tiles is at
 // least as long as its ring; the ring is made shallower until everything fits one SM's shared memory.
-bool launch_shape(int t3, int tmax, size_t code, Shape* out) {
-  int S = forced_s() ? forced_s() : 4;
+bool launch_shape(int t3, int tmax, size_t code, int64_t units, Shape* out) {
+  // Warps per 32-row block: one when the launch has enough blocks to keep the 16 warps of every SM busy with
+  // blocks of their own (no partial sums to join: 3.4 TB/s against 3.1 with four on the 100B sweep), more when
+  // it has few.
+  int S = forced_s();
+  if (!S) {
+    S = 1;
+    while (S < 4 && units * S < (int64_t)CW * dev_info().sm_count * 4) S <<= 1;
+  }
   while (S > 1 && t3 / S < 8) S >>= 1;
   const int nw = t3 / S;
   if (nw < 3) return false;
@@ -641,7 +648,7 @@ bool gemv_tl2_scan_item_supported(int T, int64_t M, int64_t K, const TlGeom& g) 
     return false;
   if (g.tiles2 > 2 || g.three_k > 0x3fffffff) return false;    // more pair tiles than a ring refill pattern assumes
   Shape sh;
-  return launch_shape((int)g.tiles3, T, code_bytes_of(T, (int)g.tiles3, (int)g.tiles2), &sh);
+  return launch_shape((int)g.tiles3, T, code_bytes_of(T, (int)g.tiles3, (int)g.tiles2), M / 32, &sh);
 }
 
 // Launches the scan kernel over `n` supported TL2 items: as few launches as the argument block (NLARGE items,
@@ -653,6 +660,8 @@ int launch_gemv_tl2_scan(const Tl2Linear* items, int64_t n, cudaStream_t st) {
     int t3_min = 1 << 30, tmax = 1;
     size_t code = 0;
     Shape sh{1, 3};
+    int64_t units = 0;
+    for (int64_t k = i; k < n && k - i < NLARGE; ++k) units += items[k].M / 32;   // (an estimate when the run is cut short)
     while (j < n && j - i < NLARGE) {
       const TlGeom& g = items[j].g;
       const int64_t add = (items[j].M / 32) * (g.tiles3 + g.tiles2);
@@ -661,7 +670,7 @@ int launch_gemv_tl2_scan(const Tl2Linear* items, int64_t n, cudaStream_t st) {
       const size_t cm = cb > code ? cb : code;
       const int t3 = (int)g.tiles3 < t3_min ? (int)g.tiles3 : t3_min;
       Shape sj;
-      const bool fits = launch_shape(t3, tm, cm, &sj);
+      const bool fits = launch_shape(t3, tm, cm, units, &sj);
       if (!fits && j == i) return BITNET_ERR_UNSUPPORTED_SHAPE;
       if (!fits || (j > i && w + add > (1ll << 30))) break;
       w += add;
