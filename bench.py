@@ -402,6 +402,43 @@ def time_replays(torch, fn, steps, warmup, dist=None):
     return ms / steps
 
 
+def bench_ceilings(bn, torch, sm_mhz):
+    """Ceilings measured on this GPU with the decode kernels' own access pattern and instruction kinds: a read-only
+    stream over 8 GiB (cp.async rings, no arithmetic), the issue rate of the instructions the decode loops are made
+    of (warp-instructions per clock and SM at the SM clock sampled under load), and the library's dense int8 GEMM
+    at 8192^3 (the prefill denominator next to 2 x the measured bf16 figure)."""
+    dev = torch.device("cuda")
+    out = {}
+    sink = torch.zeros(4, dtype=torch.int32, device=dev)
+    buf = torch.empty(8 << 30, dtype=torch.uint8, device=dev)
+    buf.view(torch.int32).fill_(0x01010101)
+    rs = {}
+    for depth in (4, 6, 8):
+        ms = time_replays(torch, lambda: bn.bitnet_microbench_read_stream(buf, depth, sink), 10, 3)
+        rs[f"ring_{depth}"] = buf.numel() / ms / 1e6
+    out["read_stream_GBps"] = rs
+    del buf
+    torch.cuda.empty_cache()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    clock_hz = (sm_mhz or 1965.0) * 1e6
+    iters = 20000
+    rates = {}
+    for kind in bn.MICROBENCH_KINDS:
+        ms = time_replays(torch, lambda: bn.bitnet_microbench_issue(kind, iters, sink), 5, 3)
+        rates[kind] = 16.0 * iters * 32 / (ms * 1e-3 * clock_hz)
+    out["issue_warp_instr_per_clk_per_sm"] = rates
+    out["issue_note"] = f"16 warps per SM, 32 independent instructions per thread and iteration, at {clock_hz / 1e6:.0f} MHz"
+    try:
+        a = torch.randint(-127, 128, (8192, 8192), dtype=torch.int8, device=dev)
+        b = torch.randint(-1, 2, (8192, 8192), dtype=torch.int8, device=dev).t()
+        ms = time_replays(torch, lambda: torch._int_mm(a, b), 10, 3)
+        out["library_int8_gemm_8192cubed_tops"] = 2.0 * 8192 ** 3 / ms / 1e9
+    except Exception as e:          # noqa: BLE001 - context only
+        out["library_int8_gemm_8192cubed_tops"] = None
+        out["library_int8_gemm_note"] = str(e)[:80]
+    return out
+
+
 def bench_prefill(bn, torch, synth, steps, warmup):
     wl = synth.CONFIGS["prefill"]
     lin, T = wl.linears[0], wl.tokens[0]
@@ -600,10 +637,15 @@ def run_ours(args):
         torch.cuda.empty_cache()
         if not args.skip_small:
             line["small_configs"] = bench_small_configs(bn, torch, synth, max(5, args.steps // 2), 3)
+        if not args.skip_ceilings:
+            line["ceilings"] = bench_ceilings(bn, torch, (clocks or {}).get("sm_mhz"))
         if not args.skip_prefill:
             pf = bench_prefill(bn, torch, synth, max(3, args.steps // 2), 3)
             pf["frac_of_int8_peak"] = pf["int8_tops"] / (2.0 * pk["bf16"])
             pf["int8_peak_used"] = f"2 x {pk['which']} bf16 dense ({pk['bf16']} TFLOP/s)"
+            lib8 = (line.get("ceilings") or {}).get("library_int8_gemm_8192cubed_tops")
+            if lib8:
+                pf["frac_of_library_int8_gemm_8192cubed"] = pf["int8_tops"] / lib8
             line["prefill"] = pf
         print(json.dumps(line))
     if dist is not None:
@@ -623,6 +665,7 @@ def main():
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-batched", action="store_true")
     ap.add_argument("--skip-small", action="store_true", help="skip the timings of the three small workloads")
+    ap.add_argument("--skip-ceilings", action="store_true", help="skip the read-stream / issue-rate / int8 GEMM ceilings")
     ap.add_argument("--no-early-start", action="store_true",
                     help="launch every kernel in plain stream order (no programmatic dependent launch)")
     args = ap.parse_args()

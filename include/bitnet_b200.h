@@ -56,6 +56,8 @@ int bitnet_last_cuda_error(void);
  * to *status_out (0 = no kernel ever gave up).  Not for the hot path.
  */
 int bitnet_device_status(int* status_out);
+/* Synchronises the device and clears the flag (after a reported time-out has been dealt with). */
+int bitnet_device_status_clear(void);
 
 /*
  * Early start (on by default).  The quantiser and the I2_S decode kernel are launched with
@@ -283,7 +285,25 @@ int bitnet_mpgemv_tl_noalloc(bitnet_fmt_t fmt, const void* packed, float w_scale
                              int bk3, const int8_t* q, const float* act_scale, int64_t T, float* y,
                              int32_t* acc_out, void* stream);
 
+/* ---- measurement hooks (not part of the path; the paper has no counterpart) ------------------- */
+/*
+ * The ceilings the decode kernels are judged against, measured rather than assumed (the host times the launches with
+ * CUDA events).
+ *   bitnet_microbench_read_stream: the grouped decode kernel's memory side alone -- persistent CTAs, per-warp rings of
+ *     `depth` (4, 6 or 8) 1-KB chunks filled by 16-byte cp.async copies -- reads `bytes` bytes at buf (device, 16-byte
+ *     aligned) once, no arithmetic.  sink: one device word the kernel may write.
+ *   bitnet_microbench_issue: every warp of one 16-warp CTA per SM issues iters * 32 independent instructions of one
+ *     kind: 0 dp4a, 1 lop3, 2 prmt, 3 32-bit multiply-add, 4 ld.shared.u32, 5 ld.shared.v4.u32,
+ *     6 mma.sync.m16n8k32 (u8 x s8).
+ */
+int bitnet_microbench_read_stream(const void* buf, size_t bytes, int depth, unsigned* sink, void* stream);
+int bitnet_microbench_issue(int kind, int iters, unsigned* sink, void* stream);
+
 /* ---- test hooks (not part of the four operations) ------------------------------------------- */
+/* Launches a one-CTA kernel whose bounded wait (the lookup-table kernel's own) is bound to run out: its barrier
+ * expects bytes that no copy ever delivers.  Nothing is in flight, nothing faults; afterwards
+ * bitnet_device_status reports BITNET_ERR_TIMEOUT until bitnet_device_status_clear. */
+int bitnet_debug_wait_timeout_probe(void* stream);
 /* Inverse of the packers: packed -> w[M][K] int8.  dev_status set if an invalid code is met. */
 int bitnet_unpack_i2s(const void* packed, int64_t M, int64_t K, int8_t* w, int* dev_status,
                       void* stream);

@@ -38,6 +38,7 @@ def lib():
         L.oracle_mpgemm_def.argtypes = [vp, vp, i64, i64, i64, vp]
         L.oracle_dequant.argtypes = [vp, vp, C.c_float, i64, i64, vp]
         L.oracle_dequant.restype = None
+        L.oracle_dequant_segments.argtypes = [vp, vp, i64, vp, vp, i64, i64, vp]
         L.oracle_i2s_packed_bytes.argtypes = [i64, i64]
         L.oracle_i2s_packed_bytes.restype = sz
         L.oracle_pack_i2s.argtypes = [vp, i64, i64, vp]
@@ -98,6 +99,17 @@ def dequant(acc, act_scale, w_scale):
     T, M = acc.shape
     y = np.empty((T, M), np.float64)
     lib().oracle_dequant(_p(acc), _p(act_scale), float(w_scale), T, M, _p(y))
+    return y
+
+
+def dequant_segments(acc, act_scale, seg_end, w_scales):
+    """y[t, m] = acc * act_scale[t] * w_scales[s] for rows m in [seg_end[s-1], seg_end[s])."""
+    acc, act_scale = _c(acc, np.int32), _c(act_scale, np.float32)
+    seg_end, w_scales = _c(np.asarray(seg_end), np.int64), _c(np.asarray(w_scales), np.float32)
+    T, M = acc.shape
+    y = np.empty((T, M), np.float64)
+    _check(lib().oracle_dequant_segments(_p(acc), _p(act_scale), len(seg_end), _p(seg_end), _p(w_scales), T, M, _p(y)),
+           "dequant_segments")
     return y
 
 

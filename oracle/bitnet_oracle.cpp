@@ -10,6 +10,7 @@
 //                         activation quantisation); rounding and operation order: see below.
 //   oracle_mpgemm_def     Alg. 1 Phase 2 / Eq. 1: R[n,m] = sum_k A_q[n,k] * W[m,k].
 //   oracle_dequant        the "Scale" of I2_S (Sec. 3.2.2): y = acc * act_scale * w_scale.
+//   oracle_dequant_segments  the same with one scale per stacked matrix of a fused tensor.
 //   oracle_pack_i2s       I2_S, 2 bits per weight (Table 1); the byte layout is this build's.
 //   oracle_pack_tl        TL1 codes of Table 4 (Alg. 3 PreprocessWeights); TL2 codes of
 //                         Table 5 with the signed-unsigned split (Sec. 3.1.2, Alg. 4
@@ -164,6 +165,22 @@ void oracle_dequant(const int32_t* acc, const float* act_scale, float w_scale, i
   for (int64_t t = 0; t < T; ++t)
     for (int64_t m = 0; m < M; ++m)
       y[t * M + m] = (double)acc[t * M + m] * (double)act_scale[t] * (double)w_scale;
+}
+
+// The same for a tensor made of several matrices stacked by rows (fused Q/K/V, gate and up), each with the scale it
+// was quantised with: rows [seg_end[s-1], seg_end[s]) carry w_scale[s] (seg_end ascending, seg_end[n_seg-1] = M).
+// "Int2 with a Scale" (Sec. 3.2.2) per stacked matrix.
+int oracle_dequant_segments(const int32_t* acc, const float* act_scale, int64_t n_seg, const int64_t* seg_end,
+                            const float* w_scale, int64_t T, int64_t M, double* y) {
+  if (n_seg < 1 || seg_end[n_seg - 1] != M) return 1;
+  for (int64_t t = 0; t < T; ++t) {
+    int64_t row = 0;
+    for (int64_t s = 0; s < n_seg; ++s) {
+      if (seg_end[s] <= row) return 1;
+      for (; row < seg_end[s]; ++row) y[t * M + row] = (double)acc[t * M + row] * (double)act_scale[t] * (double)w_scale[s];
+    }
+  }
+  return 0;
 }
 
 // ---------------------------------------------------------------------------------------------

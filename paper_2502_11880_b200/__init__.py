@@ -26,7 +26,7 @@ SYMBOLS = [
     "bitnet_pack_i2s", "bitnet_tl_packed_bytes", "bitnet_pack_tl", "bitnet_mpgemm_workspace_bytes",
     "bitnet_workspace_init", "bitnet_mpgemm", "bitnet_linear", "bitnet_linear_host", "bitnet_linear_host_batch", "bitnet_unpack_i2s", "bitnet_unpack_tl",
     "bitnet_tl_num_groups", "bitnet_tl_build_lut_debug", "bitnet_mpgemv_tl_noalloc", "bitnet_device_status",
-    "bitnet_set_early_start", "bitnet_set_tl2_lookup", "bitnet_linear_group",
+    "bitnet_set_early_start", "bitnet_set_tl2_lookup", "bitnet_device_status_clear", "bitnet_debug_wait_timeout_probe", "bitnet_linear_group", "bitnet_microbench_read_stream", "bitnet_microbench_issue",
 ]
 
 _lib = None
@@ -49,6 +49,7 @@ def lib():
         L.bitnet_status_string.restype = C.c_char_p
         L.bitnet_last_cuda_error.restype = ci
         L.bitnet_device_status.argtypes = [vp]
+        L.bitnet_debug_wait_timeout_probe.argtypes = [vp]
         L.bitnet_set_early_start.argtypes = [ci]
         L.bitnet_set_early_start.restype = None
         L.bitnet_set_tl2_lookup.argtypes = [ci]
@@ -68,6 +69,8 @@ def lib():
         L.bitnet_linear_host.argtypes = [ci, vp, fl, i64, i64, ci, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp]
         L.bitnet_linear_host_batch.argtypes = [vp, i64, vp]
         L.bitnet_linear_group.argtypes = [vp, i64, vp]
+        L.bitnet_microbench_read_stream.argtypes = [vp, sz, ci, vp, vp]
+        L.bitnet_microbench_issue.argtypes = [ci, ci, vp, vp]
         L.bitnet_unpack_i2s.argtypes = [vp, i64, i64, vp, vp, vp]
         L.bitnet_unpack_tl.argtypes = [ci, vp, i64, i64, ci, vp, vp, vp]
         L.bitnet_tl_num_groups.argtypes = [ci, i64, ci]
@@ -87,6 +90,15 @@ def bitnet_device_status() -> int:
     out = C.c_int(0)
     _check(lib().bitnet_device_status(C.byref(out)), "bitnet_device_status")
     return out.value
+
+
+def bitnet_device_status_clear():
+    _check(lib().bitnet_device_status_clear(), "bitnet_device_status_clear")
+
+
+def bitnet_debug_wait_timeout_probe(stream=None):
+    """Test hook: a kernel whose bounded wait runs out (sets the device status flag to BITNET_ERR_TIMEOUT)."""
+    _check(lib().bitnet_debug_wait_timeout_probe(_stream(stream)), "bitnet_debug_wait_timeout_probe")
 
 
 def bitnet_set_early_start(enable: bool):
@@ -343,6 +355,21 @@ def bitnet_linear_group(group, stream=None):
     """Queues a list of linears made by make_group (device buffers): one persistent kernel per run of I2_S
     decode items, bitnet_linear for the others."""
     _check(lib().bitnet_linear_group(group, C.c_int64(len(group)), _stream(stream)), "bitnet_linear_group")
+
+
+MICROBENCH_KINDS = {"dp4a": 0, "lop3": 1, "prmt": 2, "imad": 3, "lds32": 4, "lds128": 5, "mma_u8s8_m16n8k32": 6}
+
+
+def bitnet_microbench_read_stream(buf, depth, sink, stream=None):
+    """Queues one read of `buf` (CUDA uint8 tensor) with the grouped decode kernel's copy pattern and no arithmetic."""
+    _check(lib().bitnet_microbench_read_stream(_ptr(buf), buf.numel() * buf.element_size(), int(depth), _ptr(sink),
+                                               _stream(stream)), "bitnet_microbench_read_stream")
+
+
+def bitnet_microbench_issue(kind, iters, sink, stream=None):
+    """Queues iters * 32 independent instructions of `kind` (a key of MICROBENCH_KINDS) per thread on every SM."""
+    _check(lib().bitnet_microbench_issue(MICROBENCH_KINDS[kind], int(iters), _ptr(sink), _stream(stream)),
+           "bitnet_microbench_issue")
 
 
 NOALLOC_MAX_M = 32768

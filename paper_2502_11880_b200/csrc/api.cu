@@ -100,6 +100,18 @@ int bitnet_device_status(int* status_out) {
   return BITNET_OK;
 }
 
+int bitnet_device_status_clear(void) {
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return note_cuda_error(e);
+  int rc = gemv_i2s_stream_status_clear();
+  if (rc) return rc;
+  rc = gemm_prefill_status_clear();
+  if (rc) return rc;
+  return gemv_tl_status_clear();
+}
+
+int bitnet_debug_wait_timeout_probe(void* stream) { return launch_wait_timeout_probe((cudaStream_t)stream); }
+
 void bitnet_set_early_start(int enable) { g_early_start = enable ? 1 : 0; }
 void bitnet_set_tl2_lookup(int enable) { bitnet::g_tl2_lookup = enable ? 1 : 0; }
 

@@ -165,5 +165,9 @@ int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int
 
 int gemm_prefill_status(int* out);
 int gemv_tl_status(int* out);
+int gemm_prefill_status_clear();
+int gemv_tl_status_clear();
+int gemv_i2s_stream_status_clear();
+int launch_wait_timeout_probe(cudaStream_t st);
 
 }  // namespace bitnet

@@ -581,5 +581,10 @@ int gemm_prefill_status(int* out) {
   cudaError_t e = cudaMemcpyFromSymbol(out, g_prefill_error, sizeof(int));
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
 }
+int gemm_prefill_status_clear() {
+  const int zero = 0;
+  cudaError_t e = cudaMemcpyToSymbol(g_prefill_error, &zero, sizeof(int));
+  return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
+}
 
 }  // namespace bitnet

@@ -555,6 +555,11 @@ int gemv_i2s_stream_status(int* out) {
   cudaError_t e = cudaMemcpyFromSymbol(out, g_stream_error, sizeof(int));
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
 }
+int gemv_i2s_stream_status_clear() {
+  const int zero = 0;
+  cudaError_t e = cudaMemcpyToSymbol(g_stream_error, &zero, sizeof(int));
+  return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
+}
 
 
 }  // namespace bitnet

@@ -127,6 +127,38 @@ __device__ __forceinline__ uint4 load_row_words(const uint8_t* tp, int r) {
   return make_uint4(__ldg(p), __ldg(p + 4), __ldg(p + 8), __ldg(p + 12));
 }
 
+// Waits for phase 0 of an mbarrier, at most `limit` polls.  A wait that gives up records BITNET_ERR_TIMEOUT in the
+// device flag (read by bitnet_device_status) and returns false: the kernel then returns instead of hanging.
+__device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t limit) {
+  bool got = false;
+  for (uint32_t it = 0; it < limit && !got; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar))
+        : "memory");
+    got = ok != 0;
+  }
+  if (!got && threadIdx.x == 0) atomicExch(&g_tl_error, BITNET_ERR_TIMEOUT);
+  return got;
+}
+
+// Test hook: a barrier that expects 16 bytes which nobody ever copies.  The bounded wait runs out, the flag is set,
+// the kernel returns; nothing is in flight at any point.
+__global__ void wait_timeout_probe_kernel(uint32_t limit) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bar)) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(&bar)), "r"(16u) : "memory");
+  }
+  __syncthreads();
+  bounded_wait(&bar, limit);
+}
+
 __global__ void __launch_bounds__(THREADS, 2) gemv_tl_kernel(const TlArgs a) {
   extern __shared__ __align__(128) int smem[];
   int* tab = smem;                                   // [tiles_per_slice][32][16]
@@ -154,24 +186,7 @@ __global__ void __launch_bounds__(THREADS, 2) gemv_tl_kernel(const TlArgs a) {
                  : "memory");
   }
   __syncthreads();
-  {
-    bool got = false;
-    for (uint32_t it = 0; it < WAIT_LIMIT && !got; ++it) {
-      uint32_t ok;
-      asm volatile(
-          "{\n\t.reg .pred p;\n\t"
-          "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
-          "selp.u32 %0, 1, 0, p;\n\t}"
-          : "=r"(ok)
-          : "r"(smem_u32(bar))
-          : "memory");
-      got = ok != 0;
-    }
-    if (!got) {
-      if (threadIdx.x == 0) atomicExch(&g_tl_error, BITNET_ERR_TIMEOUT);
-      return;
-    }
-  }
+  if (!bounded_wait(bar, WAIT_LIMIT)) return;
 
   const float sc0 = __fmul_rn(a.act_scale[0], a.w_scale);
   const float sc1 = (a.nt == 2) ? __fmul_rn(a.act_scale[1], a.w_scale) : 0.0f;
@@ -392,6 +407,15 @@ int launch_tl_build_lut(int fmt, const int8_t* q_row, int64_t K, const TlGeom& g
 int gemv_tl_status(int* out) {
   cudaError_t e = cudaMemcpyFromSymbol(out, g_tl_error, sizeof(int));
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
+}
+int gemv_tl_status_clear() {
+  const int zero = 0;
+  cudaError_t e = cudaMemcpyToSymbol(g_tl_error, &zero, sizeof(int));
+  return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
+}
+int launch_wait_timeout_probe(cudaStream_t st) {
+  wait_timeout_probe_kernel<<<1, 64, 0, st>>>(1u << 14);
+  return check_launch();
 }
 
 }  // namespace bitnet

@@ -1,0 +1,154 @@
+// Measurement hooks (not part of the path): the ceilings the decode kernels are judged against, measured with
+// the kernels' own access pattern and instruction mix rather than assumed.
+//   - read stream: the grouped decode kernel's memory side alone -- 148 persistent CTAs, 16 warps, per-warp rings
+//     of 1-KB chunks filled by 16-byte cp.async copies (L2 evict-first) -- over a buffer, with no arithmetic;
+//   - issue rates: back-to-back independent instructions of one kind (dp4a, lop3, prmt, imad, 32-bit and 128-bit
+//     shared-memory loads, the int8 mma.sync) on every warp of every SM.
+// The host times the launches with CUDA events; bench.py turns the times into GB/s and warp-instructions per clock
+// and SM.
+#include "common.cuh"
+#include "device_utils.cuh"
+
+namespace bitnet {
+namespace {
+
+constexpr int MB_WARPS = 16, MB_THREADS = MB_WARPS * 32;
+
+template <int DEPTH>
+__global__ void __launch_bounds__(MB_THREADS, 1) read_stream_kernel(const uint8_t* __restrict__ buf, int64_t chunks,
+                                                                     unsigned* __restrict__ sink) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // CTA c owns a contiguous share of the chunks; its 16 warps interleave 8-chunk runs of it
+  const int64_t lo = chunks * blockIdx.x / gridDim.x, hi = chunks * (blockIdx.x + 1) / gridDim.x;
+  const uint64_t pol = policy_evict_first();
+  const uint32_t ring = smem_u32(smem + (size_t)warp * DEPTH * 1024) + lane * 16;
+  // the warp's stream: runs [lo + 8 (warp + 16 r), +8) for r = 0, 1, ...
+  auto chunk_ptr = [&](int64_t k) -> const uint8_t* {     // k-th chunk of the warp's stream, or null past its end
+    const int64_t c = lo + 8 * (warp + 16 * (k >> 3)) + (k & 7);
+    return c < hi ? buf + c * 1024 + lane * 16 : nullptr;
+  };
+  int64_t pfk = 0;
+#pragma unroll
+  for (int d = 0; d < DEPTH; ++d, ++pfk) {
+    const uint8_t* p = chunk_ptr(pfk);
+    if (p) {
+      cp16(ring + d * 1024, p, pol);
+      cp16(ring + d * 1024 + 512, p + 512, pol);
+    }
+    cp_commit();
+  }
+  unsigned acc = 0;
+  uint32_t slot = 0;
+  for (int64_t k = 0; chunk_ptr(k); ++k, ++pfk) {
+    cp_wait<DEPTH - 1>();
+    unsigned v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(ring + slot));
+    acc ^= v;
+    const uint8_t* p = chunk_ptr(pfk);
+    if (p) {
+      cp16(ring + slot, p, pol);
+      cp16(ring + slot + 512, p + 512, pol);
+    }
+    cp_commit();
+    slot = (slot + 1024 == DEPTH * 1024) ? 0 : slot + 1024;
+  }
+  cp_wait<0>();
+  if (acc == 0x9E3779B9u) *sink = acc;   // keeps the loads alive
+}
+
+// kind: 0 dp4a, 1 lop3, 2 prmt, 3 imad, 4 ld.shared.u32, 5 ld.shared.v4, 6 mma.sync m16n8k32 u8*s8
+template <int KIND>
+__global__ void __launch_bounds__(MB_THREADS, 1) issue_kernel(int iters, unsigned* __restrict__ sink) {
+  __shared__ __align__(16) unsigned tab[MB_THREADS * 4];
+  for (int i = threadIdx.x; i < MB_THREADS * 4; i += MB_THREADS) tab[i] = i * 2654435761u;
+  __syncthreads();
+  unsigned r[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) r[i] = threadIdx.x * 97u + i;
+  int c[4][4] = {};
+  const uint32_t a16 = smem_u32(tab) + threadIdx.x * 16;
+  for (int it = 0; it < iters; ++it) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {          // 8 independent chains x 4 = 32 instructions of the kind per iteration
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (KIND == 0) r[i] = __dp4a((int)r[i], 0x01020304, (int)r[(i + 1) & 7]);
+        if (KIND == 1) asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(r[i]) : "r"(r[(i + 1) & 7]), "r"(r[(i + 2) & 7]));
+        if (KIND == 2) asm volatile("prmt.b32 %0, %0, %1, %2;" : "+r"(r[i]) : "r"(r[(i + 1) & 7]), "r"(0x5140u + u));
+        if (KIND == 3) asm volatile("mad.lo.u32 %0, %0, %1, %2;" : "+r"(r[i]) : "r"(r[(i + 1) & 7]), "r"(r[(i + 2) & 7]));
+        // loads: the address comes from a register the loop changes, so no load can be merged with another
+        if (KIND == 4) {
+          unsigned v;
+          asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a16 + ((r[i] >> 7) & 12u)) : "memory");
+          r[i] += v | 1u;
+        }
+        if (KIND == 5) {
+          unsigned v0, v1, v2, v3;
+          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                       : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3)
+                       : "r"(a16 ^ ((r[i] & 1u) << 4))
+                       : "memory");
+          r[i] += (v0 ^ v1 ^ v2 ^ v3) | 1u;
+        }
+        if (KIND == 6) mma_u8s8(c[i & 3], r[0], r[1], r[2], r[3], (int)r[4], (int)r[5]);
+      }
+    }
+  }
+  unsigned acc = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc ^= r[i];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc ^= (unsigned)c[i][j];
+  if (acc == 0x12345u) *sink = acc;
+}
+
+template <int KIND>
+int launch_issue(int iters, unsigned* sink, cudaStream_t st) {
+  issue_kernel<KIND><<<dev_info().sm_count, MB_THREADS, 0, st>>>(iters, sink);
+  return check_launch();
+}
+
+}  // namespace
+}  // namespace bitnet
+
+using namespace bitnet;
+
+extern "C" int bitnet_microbench_read_stream(const void* buf, size_t bytes, int depth, unsigned* sink, void* stream) {
+  if (!buf || !sink || !aligned16(buf) || bytes < 1024) return BITNET_ERR_INVALID_ARG;
+  const int64_t chunks = (int64_t)(bytes / 1024);
+  cudaStream_t st = (cudaStream_t)stream;
+  const int grid = dev_info().sm_count;
+  cudaError_t e;
+  if (depth == 4) {
+    e = cudaFuncSetAttribute(read_stream_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, MB_WARPS * 4 * 1024);
+    if (e == cudaSuccess) read_stream_kernel<4><<<grid, MB_THREADS, MB_WARPS * 4 * 1024, st>>>((const uint8_t*)buf, chunks, sink);
+  } else if (depth == 6) {
+    e = cudaFuncSetAttribute(read_stream_kernel<6>, cudaFuncAttributeMaxDynamicSharedMemorySize, MB_WARPS * 6 * 1024);
+    if (e == cudaSuccess) read_stream_kernel<6><<<grid, MB_THREADS, MB_WARPS * 6 * 1024, st>>>((const uint8_t*)buf, chunks, sink);
+  } else if (depth == 8) {
+    e = cudaFuncSetAttribute(read_stream_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, MB_WARPS * 8 * 1024);
+    if (e == cudaSuccess) read_stream_kernel<8><<<grid, MB_THREADS, MB_WARPS * 8 * 1024, st>>>((const uint8_t*)buf, chunks, sink);
+  } else {
+    return BITNET_ERR_INVALID_ARG;
+  }
+  if (e != cudaSuccess) return note_cuda_error(e);
+  return check_launch();
+}
+
+extern "C" int bitnet_microbench_issue(int kind, int iters, unsigned* sink, void* stream) {
+  if (!sink || iters < 1) return BITNET_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  switch (kind) {
+    case 0: return launch_issue<0>(iters, sink, st);
+    case 1: return launch_issue<1>(iters, sink, st);
+    case 2: return launch_issue<2>(iters, sink, st);
+    case 3: return launch_issue<3>(iters, sink, st);
+    case 4: return launch_issue<4>(iters, sink, st);
+    case 5: return launch_issue<5>(iters, sink, st);
+    case 6: return launch_issue<6>(iters, sink, st);
+    default: return BITNET_ERR_INVALID_ARG;
+  }
+}

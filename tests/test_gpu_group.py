@@ -219,3 +219,49 @@ def test_group_long_rows_walked_in_parts():
     run_group(items)
     for it in items:
         it.check()
+
+
+def test_workload_sweep100b_every_layer_sampled_rows():
+    """All 80 layers of the 100B-shaped sweep, both encodings: weights drawn and packed in device memory as the
+    benchmark does, each layer's eight linears (four per format) in one grouped call; about a hundred output rows
+    per tensor are recomputed by the oracle from host re-draws of the same weights, and the TL2 accumulators must
+    equal the I2_S ones everywhere."""
+    wl = synth.CONFIGS["sweep100b"]
+    nl = len(wl.linears)
+    bufs = {}
+    for fmt in ("i2s", "tl2"):
+        for j, lin in enumerate(wl.linears):
+            bufs[fmt, j] = (torch.empty((1, lin.K), dtype=torch.int8, device="cuda"), torch.empty(1, dtype=torch.float32, device="cuda"),
+                            torch.empty((1, lin.M), dtype=torch.float32, device="cuda"),
+                            torch.empty((1, lin.M), dtype=torch.int32, device="cuda"))
+    for layer in range(wl.layers):
+        rng = np.random.default_rng(7000 + layer)
+        items, xs, blobs = [], [], []
+        for fmt in ("i2s", "tl2"):
+            for j, lin in enumerate(wl.linears):
+                wd = wl.weights(layer, j, device="cuda")
+                blobs.append(bn.pack(fmt, wd, check=False))
+                del wd
+                if fmt == "i2s":
+                    xs.append(wl.activations(layer, j, 1))
+                q, sc, y, acc = bufs[fmt, j]
+                items.append(dict(fmt=fmt, packed=blobs[-1], w_scale=0.625, M=lin.M, K=lin.K, x=xs[j].cuda(), q=q,
+                                  act_scale=sc, y=y, acc_out=acc))
+        bn.bitnet_linear_group(bn.make_group(items))
+        torch.cuda.synchronize()
+        for j, lin in enumerate(wl.linears):
+            rows = np.unique(np.concatenate([[0, 15, 16, 31, 32, lin.M - 1], rng.integers(0, lin.M, 96)]))
+            w_rows = np.stack([wl.weights(layer, j, row_start=int(r), rows=1).numpy()[0] for r in rows])
+            q_ref, sc_ref, _ = oracle.quant_act(xs[j].numpy())
+            acc_ref = oracle.mpgemm_def(q_ref, np.ascontiguousarray(w_rows))
+            rows_d = torch.as_tensor(rows).cuda()
+            for fmt in ("i2s", "tl2"):
+                q, sc, y, acc = bufs[fmt, j]
+                assert np.array_equal(npy(q), q_ref), (layer, j, fmt)
+                assert np.array_equal(npy(sc).view(np.uint32), sc_ref.view(np.uint32))
+                assert np.array_equal(npy(acc[:, rows_d]), acc_ref), (layer, j, fmt)
+                check_y(y[:, rows_d], acc_ref, sc_ref, 0.625)
+            assert torch.equal(bufs["tl2", j][3], bufs["i2s", j][3]), (layer, j)
+            assert torch.equal(bufs["tl2", j][2], bufs["i2s", j][2]), (layer, j)
+        del items, blobs
+    assert bn.bitnet_device_status() == 0

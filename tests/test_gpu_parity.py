@@ -510,7 +510,7 @@ def test_linear_host_batch_matches_single_calls():
     """bitnet_linear_host_batch (overlapped copies) gives what bitnet_linear gives item by item, for a mix
     of formats, shapes and batch sizes, and leaves the stream joined (two batches back to back)."""
     shapes = [("i2s", 512, 2048, 1), ("i2s", 96, 8192, 2), ("tl2", 64, 1536, 1), ("i2s", 1040, 4096, 4), ("tl1", 128, 256, 3)]
-    items, keep, refs = [], [], []
+    items, keep, refs, orc = [], [], [], []
     for n, (fmt, M, K, T) in enumerate(shapes):
         w = synth.ternary(40 + n, 0, M, K, 1 / 3, 1 / 3)
         x = synth.normal(40 + n, 1, T, K)
@@ -530,14 +530,21 @@ def test_linear_host_batch_matches_single_calls():
         y = torch.empty_like(yd)
         bn.bitnet_linear(fmt, blob, 0.75, M, K, x.cuda(), q=q, act_scale=sc, y=y, workspace=bn.new_workspace(fmt, T, M, K))
         refs.append(y.cpu())
+        q_ref, sc_ref, _ = oracle.quant_act(x.numpy())
+        orc.append((q_ref, sc_ref, oracle.mpgemm_def(q_ref, w.numpy())))
     batch = bn.make_host_batch(items)
     for rep in range(2):
         for it in items:
             it["y_host"].zero_()
         bn.bitnet_linear_host_batch(batch)
         torch.cuda.current_stream().synchronize()
-        for it, ref in zip(items, refs):
+        for n, (it, ref) in enumerate(zip(items, refs)):
             assert torch.equal(it["y_host"], ref), (rep, it["fmt"], it["M"], it["K"])
+            # and directly against the oracle: the host result, and the codes and scales left on the device
+            q_ref, sc_ref, acc_ref = orc[n]
+            check_y(it["y_host"], acc_ref, sc_ref, 0.75)
+            assert np.array_equal(npy(it["q_dev"]), q_ref)
+            assert np.array_equal(npy(it["scale_dev"]).view(np.uint32), sc_ref.view(np.uint32))
     assert bn.bitnet_device_status() == 0
 
 
@@ -607,3 +614,65 @@ def test_tl_workspace_shared_by_calls_of_different_shapes(fmt):
         acc_ref = oracle.mpgemm_def(q_ref, w.numpy())
         assert np.array_equal(npy(acc), acc_ref)
         check_y(y, acc_ref, sc_ref, 0.5)
+
+
+def test_bounded_wait_times_out_and_reports():
+    """A device-side wait that cannot complete gives up after its poll limit, sets the status flag and lets the kernel
+    return: the context stays usable, bitnet_device_status reports the time-out, and the flag can be cleared."""
+    assert bn.bitnet_device_status() == 0
+    bn.bitnet_debug_wait_timeout_probe()
+    assert bn.bitnet_device_status() == 6          # BITNET_ERR_TIMEOUT
+    assert "wait" in bn.status_string(6)
+    bn.bitnet_device_status_clear()
+    assert bn.bitnet_device_status() == 0
+    # the device still computes
+    check_linear("tl1", tern(95, 32, 192), synth.normal(95, 1, 1, 192))
+
+
+def _run_child(code, extra_env):
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, "-c", code], cwd=root, env=dict(os.environ, **extra_env), capture_output=True,
+                         text=True, timeout=900)
+    assert out.returncode == 0 and "ok" in out.stdout, (extra_env, out.stderr[-2000:])
+
+
+@pytest.mark.parametrize("extra", [dict(BITNET_PREFILL="simt"), dict(BITNET_PREFILL_TMA_STORE="0"),
+                                   dict(BITNET_I2S_STREAM="ring"), dict(BITNET_QUANT_CLUSTERS="0"),
+                                   dict(BITNET_FUSE_MAX_T="0"), dict(BITNET_I2S_MID_MIN_T="9"),
+                                   dict(BITNET_MID_NS="5"), dict(BITNET_TL2="lut"), dict(BITNET_TL2_S="4", BITNET_TL2_DEPTH="4"),
+                                   dict(BITNET_GROUP="0"), dict(BITNET_GROUP_S="2", BITNET_GROUP_DEPTH="8"),
+                                   dict(BITNET_GROUP_DEPTH="12")])
+def test_read_once_switches_in_child_processes(extra):
+    """Every kernel choice that an environment variable makes (read once per process) against the oracle: the dp4a
+    prefill kernel, plain stores instead of bulk tensor stores in the tensor-core prefill kernel, the bulk-copy ring
+    decode kernel, the quantiser without clusters, no fused quantiser, the mid-batch kernel's lower limit and forced
+    slice count, the lookup-table kernel for TL2, other ring depths and warps per unit in the grouped kernels, and
+    the grouped call switched off."""
+    code = (
+        "import sys; sys.path.insert(0, 'tests'); import numpy as np, torch\n"
+        "import oracle\n"
+        "from paper_2502_11880_b200 import synth\n"
+        "import paper_2502_11880_b200 as bn\n"
+        "from helpers import check_linear, check_y, run_fused, npy\n"
+        "from test_gpu_group import Item, run_group\n"
+        "for (M, K, T) in [(70, 1536, 1), (64, 8192, 2), (33, 28672, 5), (48, 16384, 6), (40, 8192, 8), (200, 4096, 20),\n"
+        "                  (300, 2048, 300)]:\n"
+        "    check_linear('i2s', synth.ternary(62, 1, M, K, 1/3, 1/3), synth.normal(62, T, T, K))\n"
+        "for (M, K, T) in [(64, 3200, 1), (96, 8192, 3), (32, 28672, 8), (64, 130, 2)]:\n"
+        "    check_linear('tl2', synth.ternary(63, 1, M, K, 1/3, 1/3), synth.normal(63, T, T, K))\n"
+        "for (M, K, T) in [(96, 8192, 1), (64, 28672, 4), (32, 16384, 7)]:\n"
+        "    w = synth.ternary(64, 1, M, K, 1/3, 1/3); x = synth.normal(64, T, T, K)\n"
+        "    for fmt in ('i2s', 'tl2'):\n"
+        "        y, q, sc, acc = run_fused(fmt, bn.pack(fmt, w.cuda()), 0.5, M, K, x.cuda(), workspace=bn.new_workspace(fmt, T, M, K))\n"
+        "        q_ref, sc_ref, _ = oracle.quant_act(x.numpy())\n"
+        "        assert np.array_equal(npy(q), q_ref) and np.array_equal(npy(acc), oracle.mpgemm_def(q_ref, w.numpy()))\n"
+        "items = [Item('i2s', 160, 8192, 1, 900), Item('tl2', 64, 8192, 1, 901), Item('i2s', 48, 28672, 8, 902), Item('i2s', 2000, 2048, 3, 903),\n"
+        "         Item('tl2', 640, 3200, 2, 904)]\n"
+        "run_group(items)\n"
+        "for it in items: it.check()\n"
+        "assert bn.bitnet_device_status() == 0\n"
+        "print('ok')\n")
+    _run_child(code, extra)

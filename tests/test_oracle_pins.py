@@ -337,6 +337,19 @@ def test_tl1_documented_byte_positions_and_padding():
     assert np.array_equal(p, expect)
 
 
+def test_dequant_segments_closed_form():
+    """Two stacked matrices with scales 0.5 and 3: powers of two and small integers keep every product exact, so the
+    expected values are written down; a single segment equals oracle.dequant; bad segment lists are refused."""
+    acc = np.array([[2, -4, 6, 8, -10], [1, 1, 1, 1, 1]], np.int32)
+    act_scale = np.array([0.25, 2.0], np.float32)
+    y = oracle.dequant_segments(acc, act_scale, [2, 5], [0.5, 3.0])
+    assert np.array_equal(y, np.array([[0.25, -0.5, 4.5, 6.0, -7.5], [1.0, 1.0, 6.0, 6.0, 6.0]]))
+    assert np.array_equal(oracle.dequant_segments(acc, act_scale, [5], [0.75]), oracle.dequant(acc, act_scale, 0.75))
+    for bad in ([2, 4], [3, 3, 5], [6]):
+        with pytest.raises(Exception):
+            oracle.dequant_segments(acc, act_scale, bad, [1.0] * len(bad))
+
+
 # ----------------------------------------------------------------------------- LUT build (Alg. 3 / Alg. 4 PreCompute)
 def test_lut_identities():
     q = rand_q(1, 96 * 2 + 64)[0]

@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2502_11880_b200 as bn
 from paper_2502_11880_b200 import synth
 
@@ -18,12 +19,12 @@ pytestmark = pytest.mark.gpu
 REL_TOL = 1e-6
 
 
-def _case(fmt, M, K, T, seed):
-    w = synth.ternary(seed, 1, M, K, 1 / 3, 1 / 3).cuda()
-    x = synth.normal(seed, 2, T, K).cuda()
-    q, sc, _ = bn.bitnet_quant_act(x)
-    blob = bn.pack(fmt, w)
-    return blob, q, sc
+def _case(fmt, M, K, T, seed, want_inputs=False):
+    w = synth.ternary(seed, 1, M, K, 1 / 3, 1 / 3)
+    x = synth.normal(seed, 2, T, K)
+    q, sc, _ = bn.bitnet_quant_act(x.cuda())
+    blob = bn.pack(fmt, w.cuda())
+    return (blob, q, sc, w, x) if want_inputs else (blob, q, sc)
 
 
 @pytest.mark.parametrize("fmt,M,K,T", [("tl2", 64, 28672, 1), ("tl2", 96, 8192, 2), ("tl1", 32, 14336, 3),
@@ -31,7 +32,7 @@ def _case(fmt, M, K, T, seed):
 def test_noalloc_matches_workspace_entry_point_twice(fmt, M, K, T):
     w_scale = 0.625
     for call in range(2):                      # two calls in a row share the built-in scratch
-        blob, q, sc = _case(fmt, M, K, T, seed=40 + call)
+        blob, q, sc, w, x = _case(fmt, M, K, T, seed=40 + call, want_inputs=True)
         y_ref, acc_ref = bn.bitnet_mpgemm(fmt, blob, w_scale, M, K, q, sc, want_acc=True)
         y = torch.full((T, M), float("nan"), dtype=torch.float32, device="cuda")
         acc = torch.full((T, M), -7, dtype=torch.int32, device="cuda")
@@ -41,6 +42,12 @@ def test_noalloc_matches_workspace_entry_point_twice(fmt, M, K, T):
         yr = y_ref.double().cpu().numpy()
         err = np.abs(y.double().cpu().numpy() - yr)
         assert np.all(err <= REL_TOL * np.abs(yr))
+        # and directly against the CPU oracle
+        q_ref, sc_ref, _ = oracle.quant_act(x.numpy())
+        acc_ref = oracle.mpgemm_def(q_ref, w.numpy())
+        assert np.array_equal(acc.cpu().numpy(), acc_ref)
+        y_or = oracle.dequant(acc_ref, sc_ref, w_scale)
+        assert np.all(np.abs(y.double().cpu().numpy() - y_or) <= REL_TOL * np.abs(y_or))
 
 
 def test_noalloc_rejects_sizes_beyond_its_scratch():
