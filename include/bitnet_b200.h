@@ -262,6 +262,23 @@ typedef struct bitnet_group_item {
 int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* stream);
 
 /*
+ * One linear layer whose packed tensor is several matrices stacked by rows -- fused Q/K/V, gate and up -- each
+ * quantised with its own scale: "Int2 with a Scale" (Sec. 3.2.2) per stacked matrix.  Same arguments and results
+ * as bitnet_linear, except that rows [seg_end[s-1], seg_end[s]) of the output are rescaled with seg_scale[s]:
+ *     y[t,m] = acc[t,m] * act_scale[t] * seg_scale[s(m)].
+ *   - seg_end[n_seg], seg_scale[n_seg]: HOST arrays, read during the call; 1 <= n_seg <= 16; ends ascending, the
+ *     last one M; every end but the last a multiple of the format's row block (16 for I2_S, 32 for TL), so that a
+ *     segment is a contiguous piece of the blob packed from the stacked matrix.
+ *   - I2_S and TL2 with T <= 8 (shapes the grouped kernels take): ONE persistent kernel, an item per segment, the
+ *     shared input quantised once per CTA.  Otherwise the whole tensor runs with scale 1 and a small kernel
+ *     multiplies every segment's columns by its scale (one more fp32 rounding, inside the 1e-6 relative bound).
+ */
+int bitnet_linear_segments(bitnet_fmt_t fmt, const void* packed, int64_t M, int64_t K, int bk3, int64_t n_seg,
+                           const int64_t* seg_end, const float* seg_scale, const float* x, int64_t T, int8_t* q,
+                           float* act_scale, float* y, int32_t* acc_out, void* workspace, size_t workspace_bytes,
+                           void* stream);
+
+/*
  * Table-lookup mpGEMV without a workspace argument (the paper has no counterpart: this entry point
  * exists for the sake of callers, not of the method).
  *

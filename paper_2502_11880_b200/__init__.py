@@ -26,7 +26,7 @@ SYMBOLS = [
     "bitnet_pack_i2s", "bitnet_tl_packed_bytes", "bitnet_pack_tl", "bitnet_mpgemm_workspace_bytes",
     "bitnet_workspace_init", "bitnet_mpgemm", "bitnet_linear", "bitnet_linear_host", "bitnet_linear_host_batch", "bitnet_unpack_i2s", "bitnet_unpack_tl",
     "bitnet_tl_num_groups", "bitnet_tl_build_lut_debug", "bitnet_mpgemv_tl_noalloc", "bitnet_device_status",
-    "bitnet_set_early_start", "bitnet_set_tl2_lookup", "bitnet_device_status_clear", "bitnet_debug_wait_timeout_probe", "bitnet_linear_group", "bitnet_microbench_read_stream", "bitnet_microbench_issue",
+    "bitnet_set_early_start", "bitnet_set_tl2_lookup", "bitnet_device_status_clear", "bitnet_debug_wait_timeout_probe", "bitnet_linear_group", "bitnet_linear_segments", "bitnet_microbench_read_stream", "bitnet_microbench_issue",
 ]
 
 _lib = None
@@ -69,6 +69,7 @@ def lib():
         L.bitnet_linear_host.argtypes = [ci, vp, fl, i64, i64, ci, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp]
         L.bitnet_linear_host_batch.argtypes = [vp, i64, vp]
         L.bitnet_linear_group.argtypes = [vp, i64, vp]
+        L.bitnet_linear_segments.argtypes = [ci, vp, i64, i64, ci, i64, vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
         L.bitnet_microbench_read_stream.argtypes = [vp, sz, ci, vp, vp]
         L.bitnet_microbench_issue.argtypes = [ci, ci, vp, vp]
         L.bitnet_unpack_i2s.argtypes = [vp, i64, i64, vp, vp, vp]
@@ -326,6 +327,29 @@ def bitnet_linear_host_batch(batch, stream=None):
     """Queues a batch made by make_host_batch: uploads, kernels and downloads overlap; the caller
     synchronises the stream before reading the host results."""
     _check(lib().bitnet_linear_host_batch(batch, C.c_int64(len(batch)), _stream(stream)), "bitnet_linear_host_batch")
+
+
+def bitnet_linear_segments(fmt, packed, M, K, seg_end, seg_scale, x, bk3=0, q=None, act_scale=None, y=None, acc_out=None,
+                           want_acc=False, workspace=None, stream=None):
+    """bitnet_linear for a tensor of row-stacked matrices with one weight scale each: rows [seg_end[s-1], seg_end[s])
+    of y carry seg_scale[s].  Returns (y, q, act_scale, acc or None)."""
+    _dev(x, torch.float32, "x")
+    T = x.shape[0]
+    q = torch.empty((T, K), dtype=torch.int8, device=x.device) if q is None else q
+    act_scale = torch.empty(T, dtype=torch.float32, device=x.device) if act_scale is None else act_scale
+    y = torch.empty((T, M), dtype=torch.float32, device=x.device) if y is None else y
+    if want_acc and acc_out is None:
+        acc_out = torch.empty((T, M), dtype=torch.int32, device=x.device)
+    if workspace is None:
+        workspace = new_workspace(fmt, T, M, K, x.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    n = len(seg_end)
+    ends = (C.c_int64 * n)(*[int(v) for v in seg_end])
+    scales = (C.c_float * n)(*[float(v) for v in seg_scale])
+    _check(lib().bitnet_linear_segments(_fmt(fmt), _ptr(packed), M, K, bk3, n, ends, scales, _ptr(x), T, _ptr(q),
+                                        _ptr(act_scale), _ptr(y), _ptr(acc_out), _ptr(workspace), ws_bytes, _stream(stream)),
+           "bitnet_linear_segments")
+    return y, q, act_scale, acc_out
 
 
 class GroupItem(C.Structure):

@@ -275,6 +275,7 @@ int bitnet_mpgemm(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
       it.T = nt;
       it.M = M;
       it.K = K;
+      it.ldy = 0;
       it.g = g;
       rc = launch_gemv_tl2_scan(&it, 1, st);
     } else {
@@ -326,6 +327,7 @@ int bitnet_linear(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
       it.T = (int)T;
       it.M = M;
       it.K = K;
+      it.ldy = 0;
       it.g = g;
       return launch_gemv_tl2_scan(&it, 1, (cudaStream_t)stream);
     }
@@ -395,6 +397,7 @@ int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* strea
         it.T = (int)d.T;
         it.M = d.M;
         it.K = d.K;
+        it.ldy = 0;
         it.g = g2;
         run2.push_back(it);
       }
@@ -424,12 +427,94 @@ int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* strea
       gl.T = (int)d.T;
       gl.M = d.M;
       gl.K = d.K;
+      gl.ldy = 0;
       run.push_back(gl);
     }
     int rc = launch_gemv_i2s_group(run.data(), (int64_t)run.size(), (cudaStream_t)stream);
     if (rc) return rc;
   }
   return BITNET_OK;
+}
+
+int bitnet_linear_segments(bitnet_fmt_t fmt, const void* packed, int64_t M, int64_t K, int bk3, int64_t n_seg,
+                           const int64_t* seg_end, const float* seg_scale, const float* x, int64_t T, int8_t* q,
+                           float* act_scale, float* y, int32_t* acc_out, void* workspace, size_t workspace_bytes,
+                           void* stream) {
+  if (!packed || !x || !q || !act_scale || !y || !seg_end || !seg_scale || T < 1 || n_seg < 1 || n_seg > 16)
+    return BITNET_ERR_INVALID_ARG;
+  if (!aligned16(packed) || !aligned16(x) || !aligned16(q) || !aligned16(y) || (acc_out && !aligned16(acc_out)) ||
+      (reinterpret_cast<uintptr_t>(act_scale) & 3u))
+    return BITNET_ERR_INVALID_ARG;
+  TlGeom g;
+  int rc = fmt == BITNET_FMT_I2S ? i2s_shape(M, K) : tl_shape(fmt, M, K, bk3, &g);
+  if (rc) return rc;
+  // segments: ascending ends, the last one M; every segment but the last ends on a row block of the format
+  // (16 rows for I2_S, 32 for TL), so that it is a contiguous piece of the blob
+  const int64_t rows_per_block = fmt == BITNET_FMT_I2S ? 16 : 32;
+  int64_t prev = 0;
+  for (int64_t s = 0; s < n_seg; ++s) {
+    if (seg_end[s] <= prev || seg_end[s] > M) return BITNET_ERR_INVALID_ARG;
+    if (s + 1 < n_seg && (seg_end[s] % rows_per_block) != 0) return BITNET_ERR_UNSUPPORTED_SHAPE;
+    prev = seg_end[s];
+  }
+  if (prev != M) return BITNET_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  static const bool grouped = [] { const char* e = getenv("BITNET_GROUP"); return !(e && atoi(e) == 0); }();
+  // one grouped kernel: an item per segment, all sharing the input (quantised once per CTA), each writing its own
+  // columns of y with its own scale
+  if (grouped && fmt == BITNET_FMT_I2S && T <= 8) {
+    bool ok = true;
+    int64_t r0 = 0;
+    for (int64_t s = 0; s < n_seg && ok; r0 = seg_end[s], ++s) ok = gemv_i2s_group_item_supported((int)T, seg_end[s] - r0, K);
+    if (ok) {
+      GroupLinear it[16];
+      r0 = 0;
+      for (int64_t s = 0; s < n_seg; r0 = seg_end[s], ++s) {
+        it[s].packed = (const uint8_t*)packed + (size_t)(r0 / 16) * (size_t)(4 * i2s_kp(K));
+        it[s].x = x;
+        it[s].q = q;
+        it[s].act_scale = act_scale;
+        it[s].y = y + r0;
+        it[s].acc_out = acc_out ? acc_out + r0 : nullptr;
+        it[s].w_scale = seg_scale[s];
+        it[s].T = (int)T;
+        it[s].M = seg_end[s] - r0;
+        it[s].K = K;
+        it[s].ldy = M;
+      }
+      return launch_gemv_i2s_group(it, n_seg, st);
+    }
+  }
+  if (grouped && fmt == BITNET_FMT_TL2 && T <= 8) {
+    bool ok = true;
+    int64_t r0 = 0;
+    TlGeom gs[16];
+    for (int64_t s = 0; s < n_seg && ok; r0 = seg_end[s], ++s)
+      ok = tl_shape(fmt, seg_end[s] - r0, K, bk3, &gs[s]) == BITNET_OK && tl2_scan_takes(fmt, T, seg_end[s] - r0, K, gs[s]);
+    if (ok) {
+      Tl2Linear it[16];
+      r0 = 0;
+      for (int64_t s = 0; s < n_seg; r0 = seg_end[s], ++s) {
+        it[s].packed = (const uint8_t*)packed + (size_t)(r0 / 32) * (size_t)g.block_bytes;
+        it[s].x = x;
+        it[s].q = q;
+        it[s].act_scale = act_scale;
+        it[s].y = y + r0;
+        it[s].acc_out = acc_out ? acc_out + r0 : nullptr;
+        it[s].w_scale = seg_scale[s];
+        it[s].T = (int)T;
+        it[s].M = seg_end[s] - r0;
+        it[s].K = K;
+        it[s].ldy = M;
+        it[s].g = gs[s];
+      }
+      return launch_gemv_tl2_scan(it, n_seg, st);
+    }
+  }
+  // any other shape: the whole tensor with scale 1, then every segment's columns times its scale
+  rc = bitnet_linear(fmt, packed, 1.0f, M, K, bk3, x, T, q, act_scale, y, acc_out, workspace, workspace_bytes, stream);
+  if (rc) return rc;
+  return launch_scale_segments(y, T, M, (int)n_seg, seg_end, seg_scale, st);
 }
 
 }  // extern "C"

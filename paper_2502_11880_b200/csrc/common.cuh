@@ -116,6 +116,7 @@ struct GroupLinear {
   float w_scale;
   int T;
   int64_t M, K;
+  int64_t ldy;         // elements between the token rows of y / acc_out; 0 = M
 };
 bool gemv_i2s_group_item_supported(int T, int64_t M, int64_t K);
 int launch_gemv_i2s_group(const GroupLinear* items, int64_t n, cudaStream_t st);
@@ -131,6 +132,7 @@ struct Tl2Linear {
   float w_scale;
   int T;
   int64_t M, K;
+  int64_t ldy;         // elements between the token rows of y / acc_out; 0 = M
   TlGeom g;
 };
 bool gemv_tl2_scan_item_supported(int T, int64_t M, int64_t K, const TlGeom& g);
@@ -153,6 +155,9 @@ int launch_tl_build_lut(int fmt, const int8_t* q_row, int64_t K, const TlGeom& g
                         cudaStream_t st);
 
 // y = float(sums) * (act_scale[t] * w_scale) over a [T][M] int32 array of finished sums, which is left zeroed.
+// y[t][m] *= scale of the segment row m lies in (n_seg <= 16 segments, ends ascending, the last = M).
+int launch_scale_segments(float* y, int64_t T, int64_t M, int n_seg, const int64_t* seg_end, const float* seg_scale,
+                          cudaStream_t st);
 int launch_rescale_sums(int32_t* sums, const float* act_scale, float w_scale, int64_t T, int64_t M, float* y,
                         int32_t* acc_out, cudaStream_t st);
 

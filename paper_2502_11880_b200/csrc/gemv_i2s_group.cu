@@ -56,7 +56,7 @@ struct GItem {
   int first_unit;      // units of the items before this one
   int first_w;         // 1-KB chunks of the items before this one
   int nparts;          // K is walked in this many parts (1 unless the staged codes of a whole row do not fit)
-  int pad;
+  int ldy;             // elements between the token rows of y and acc_out (M, or more for a slice of a wider output)
 };
 static_assert(sizeof(GItem) == 80, "argument block layout");
 
@@ -304,7 +304,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
     const int qst = ((nch + nparts - 1) / nparts) * 256 + 16;
     const bool owner = jb <= d.first_unit;
     const int jlo = range_lo(ci), jhi = range_hi(ci);
-    const int first = d.first_unit, M = d.M;
+    const int first = d.first_unit, M = d.M, ldy = d.ldy;
     const unsigned has_tok = g < T ? 1u : 0u;
     const float w_scale = d.w_scale;
     float* const y = d.y;
@@ -411,11 +411,11 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
               const int tok = idx >> 4, row = row0 + (idx & 15);
               v -= qsum[tok];
               if (row < M) {
-                float* const yp = y + (int64_t)tok * M + row;
+                float* const yp = y + (int64_t)tok * ldy + row;
                 if (part > 0) v += __ldcg(reinterpret_cast<const int*>(yp));
                 if (last_part) {
                   *yp = __fmul_rn((float)v, __fmul_rn(qscale[tok], w_scale));
-                  if (acc_out) acc_out[(int64_t)tok * M + row] = v;
+                  if (acc_out) acc_out[(int64_t)tok * ldy + row] = v;
                 } else {
                   *reinterpret_cast<int*>(yp) = v;
                 }
@@ -570,7 +570,7 @@ int launch_run(const GroupLinear* items, int n, Shape shape, cudaStream_t st) {
     d.first_unit = (int)units;
     d.first_w = (int)w;
     d.nparts = pl.nparts;
-    d.pad = 0;
+    d.ldy = (int)(s.ldy ? s.ldy : s.M);
     const int64_t nu = ceil_div(s.M, 16), nch = i2s_kp(s.K) / 256;
     units += nu;
     w += nu * nch;

@@ -55,7 +55,7 @@ struct SItem {
   int block_bytes;
   int first_unit;      // 32-row blocks of the items before this one
   int first_w;         // tiles of the items before this one
-  int pad;
+  int ldy;             // elements between the token rows of y and acc_out
 };
 static_assert(sizeof(SItem) == 88, "argument block layout");
 
@@ -354,7 +354,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
     const int n2 = (wk == S - 1) ? tiles2 : 0;
     const int iend = (ci + 1 < a.n) ? a.it[ci + 1].first_unit : a.total_units;
     const int cend = je < iend ? je : iend;
-    const int first = d.first_unit, M = d.M;
+    const int first = d.first_unit, M = d.M, ldy = d.ldy;
     const unsigned has_tok = g < T ? 1u : 0u;
     const uint32_t q_row = smem_u32(qs_mem + min(g, T - 1) * qst);
     const uint32_t q3 = q_row + lo3 * 128 + t * 32;         // B registers of the warp's first triple tile
@@ -494,8 +494,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
           const int tok = idx >> 5, row = row0 + (idx & 31);
           v -= qsum[tok];
           if (row < M) {
-            y[(int64_t)tok * M + row] = __fmul_rn((float)v, __fmul_rn(qscale[tok], w_scale));
-            if (acc_out) acc_out[(int64_t)tok * M + row] = v;
+            y[(int64_t)tok * ldy + row] = __fmul_rn((float)v, __fmul_rn(qscale[tok], w_scale));
+            if (acc_out) acc_out[(int64_t)tok * ldy + row] = v;
           }
         }
       }
@@ -620,7 +620,7 @@ int launch_run(const Tl2Linear* items, int n, Shape shape, cudaStream_t st) {
     d.block_bytes = (int)s.g.block_bytes;
     d.first_unit = (int)units;
     d.first_w = (int)w;
-    d.pad = 0;
+    d.ldy = (int)(s.ldy ? s.ldy : s.M);
     units += s.M / 32;
     w += (s.M / 32) * (s.g.tiles3 + s.g.tiles2);
     if (s.T > a.tmax) a.tmax = s.T;

@@ -265,3 +265,46 @@ def test_workload_sweep100b_every_layer_sampled_rows():
             assert torch.equal(bufs["tl2", j][2], bufs["i2s", j][2]), (layer, j)
         del items, blobs
     assert bn.bitnet_device_status() == 0
+
+
+@pytest.mark.parametrize("fmt,T", [("i2s", 1), ("i2s", 3), ("i2s", 12), ("tl2", 1), ("tl2", 2), ("tl1", 1)])
+def test_linear_segments_fused_qkv_and_gate_up(fmt, T):
+    """The 8B-shaped layer with its fused tensors as the model keeps them: Q/K/V stacked (4096 + 1024 + 1024 rows,
+    three scales) and gate/up stacked (2 x 14336 rows, two scales), one call each; every accumulator against the
+    definition and every output against the oracle's per-segment rescale.  12 tokens and TL1 take the fallback
+    (whole tensor, then a rescale of the segments' columns)."""
+    for (M, K, ends, scales, seed) in [(6144, 4096, [4096, 5120, 6144], [0.5, 0.71875, 0.4375], 1000),
+                                       (28672, 4096, [14336, 28672], [0.625, 0.6875], 1001),
+                                       (200, 2048, [64, 128, 200] if fmt == "i2s" else [64, 128, 192], [1.0, 0.25, 3.0], 1002)]:
+        M = ends[-1]
+        w = tern(seed, M, K, 0.4, 0.3)
+        x = synth.normal(seed, 2000 + T, T, K)
+        blob = bn.pack(fmt, w.cuda())
+        gq, gsc = Guarded((T, K), torch.int8), Guarded((T,), torch.float32)
+        gy, gacc = Guarded((T, M), torch.float32), Guarded((T, M), torch.int32)
+        bn.bitnet_linear_segments(fmt, blob, M, K, ends, scales, x.cuda(), q=gq.t, act_scale=gsc.t, y=gy.t, acc_out=gacc.t)
+        torch.cuda.synchronize()
+        for name, g in (("q", gq), ("act_scale", gsc), ("y", gy), ("acc", gacc)):
+            assert g.intact(), name
+        q_ref, sc_ref, _ = oracle.quant_act(x.numpy())
+        assert np.array_equal(npy(gq.t), q_ref)
+        assert np.array_equal(npy(gsc.t).view(np.uint32), sc_ref.view(np.uint32))
+        acc_ref = oracle.mpgemm_def(q_ref, w.numpy())
+        assert np.array_equal(npy(gacc.t), acc_ref)
+        y_ref = oracle.dequant_segments(acc_ref, sc_ref, ends, scales)
+        y = npy(gy.t).astype(np.float64)
+        assert np.all(np.abs(y - y_ref) <= 1e-6 * np.abs(y_ref))
+        assert np.all(y[acc_ref == 0] == 0.0)
+    assert bn.bitnet_device_status() == 0
+
+
+def test_linear_segments_rejects_bad_lists():
+    w = tern(1100, 64, 1024)
+    blob = bn.pack("i2s", w.cuda())
+    x = synth.normal(1100, 1, 1, 1024).cuda()
+    with pytest.raises(bn.BitnetError, match="shape"):
+        bn.bitnet_linear_segments("i2s", blob, 64, 1024, [24, 64], [1.0, 1.0], x)      # 24 is not a multiple of 16
+    with pytest.raises(bn.BitnetError, match="invalid"):
+        bn.bitnet_linear_segments("i2s", blob, 64, 1024, [32, 48], [1.0, 1.0], x)      # does not end at M
+    with pytest.raises(bn.BitnetError, match="invalid"):
+        bn.bitnet_linear_segments("i2s", blob, 64, 1024, [32, 32, 64], [1.0, 1.0, 1.0], x)   # empty segment
