@@ -308,3 +308,17 @@ def test_linear_segments_rejects_bad_lists():
         bn.bitnet_linear_segments("i2s", blob, 64, 1024, [32, 48], [1.0, 1.0], x)      # does not end at M
     with pytest.raises(bn.BitnetError, match="invalid"):
         bn.bitnet_linear_segments("i2s", blob, 64, 1024, [32, 32, 64], [1.0, 1.0, 1.0], x)   # empty segment
+
+
+def test_group_tl2_long_rows_walked_in_parts():
+    """TL2 batches whose staged codes do not fit beside the decode table: the triple tiles of a row are walked in
+    parts, the pair tiles of the tail with the last part, the integer sums resting in y in between."""
+    shapes = [(64, 14336, 8), (96, 28672, 4), (32, 28672, 8), (160, 96 * 150 + 92, 7), (64, 8192, 8), (320, 28672, 2),
+              (32, 96 * 9, 1)]
+    items = [Item("tl2", M, K, T, 1200 + i) for i, (M, K, T) in enumerate(shapes)]
+    run_group(items)
+    for it in items:
+        it.check()
+    run_group(items)            # y held integer scratch in between: nothing stale may survive
+    for it in items:
+        it.check()
