@@ -165,13 +165,16 @@ class Sweep:
         self.blobs = {f: [] for f in fmts}
         self.w_scale = []
         t0 = time.time()
-        for layer in range(layers):
-            for j, lin in enumerate(self.lin):
-                w = wl.weights(layer, j, device=device)
-                self.w_scale.append(bn.synth.absmean_scale(w))
-                for f in fmts:
+        # one encoding after the other, so that the blobs of an encoding lie together in device memory as they would
+        # in a deployment that keeps a single encoding
+        for fi, f in enumerate(fmts):
+            for layer in range(layers):
+                for j, lin in enumerate(self.lin):
+                    w = wl.weights(layer, j, device=device)
+                    if fi == 0:
+                        self.w_scale.append(bn.synth.absmean_scale(w))
                     self.blobs[f].append(bn.pack(f, w, check=False))
-                del w
+                    del w
         torch.cuda.synchronize()
         self.setup_s = time.time() - t0
         self.bytes = {f: sum(b.numel() for b in self.blobs[f]) for f in fmts}
@@ -297,7 +300,8 @@ class Sweep:
 def bench_batched(sw, torch, T, steps, warmup):
     """The same sweep with T tokens per linear (I2_S) through ONE bitnet_linear_group call per step: quantiser +
     mpGEMM + rescale.  Every linear keeps its own weights; the T activation rows of layer 0's four linears are
-    reused by all layers.  Items the grouped kernel does not take (more than 144 KiB of codes) run as bitnet_linear."""
+    reused by all layers.  Up to 8 tokens the whole list is one persistent kernel; beyond that the call runs every
+    item as bitnet_linear (quantiser + mid-batch mma.sync kernel + rescale, three launches per linear)."""
     bn, dev = sw.bn, sw.x_dev.device
     nl = len(sw.lin)
     xs = [sw.wl.activations(0, j, T).to(dev) for j in range(nl)]
@@ -607,7 +611,7 @@ def run_ours(args):
         if not args.skip_batched:
             line["batched_decode"] = {
                 "note": "the same sweep with T tokens per linear, one bitnet_linear_group call per step, inputs resident",
-                "runs": [bench_batched(sw, torch, T, max(3, args.steps // 5), 3) for T in (2, 4, 8)]}
+                "runs": [bench_batched(sw, torch, T, max(3, args.steps // 5), 3) for T in (2, 4, 8, 16, 64)]}
         if world == 1 and not args.skip_cpu:
             # ---- CPU baseline leg: the oracle, as it stands, on one full layer of the sweep for about 10 s on the
             # host cores; its results then check the y the GPU left in device memory

@@ -149,8 +149,12 @@ int bitnet_pack_tl(bitnet_fmt_t fmt, const int8_t* w, int64_t M, int64_t K, int 
  * I2_S: T <= 8 runs the decode GEMV kernel; 9 <= T <= 64 a scan of the weights on mma.sync tensor-core
  * tiles over K-slices followed by a rescale kernel (when the workspace is missing or too small, the
  * prefill kernel takes the call instead); larger T the tcgen05 prefill kernel (whole tiles per CTA; parts
- * of a tile's K per CTA when there are few tiles and the workspace is there).  TL runs its GEMV kernel
- * over groups of 8 tokens.  The integer results do not depend on which kernel ran.
+ * of a tile's K per CTA when there are few tiles and the workspace is there).  TL runs a decode kernel over
+ * groups of 8 tokens (TL2: the scan kernel, see bitnet_set_tl2_lookup); from 128 tokens on, with K a multiple of
+ * 64 and the workspace bitnet_mpgemm_workspace_bytes asks for, the TL blob is first turned into its I2_S form
+ * inside the workspace (a device-side transcode of the packed codes) and the tcgen05 prefill kernel serves the
+ * call, so that a model kept only in the 1.67-bit TL2 encoding has a tensor-core prefill too.  The integer
+ * results do not depend on which kernel ran.
  */
 size_t bitnet_mpgemm_workspace_bytes(bitnet_fmt_t fmt, int64_t T, int64_t M, int64_t K);
 int bitnet_workspace_init(void* workspace, size_t workspace_bytes, void* stream);

@@ -216,6 +216,10 @@ static bool tl2_scan_takes(int fmt, int64_t T, int64_t M, int64_t K, const TlGeo
   return !bitnet::g_tl2_lookup && fmt == BITNET_FMT_TL2 && T >= 1 && T <= 8 && gemv_tl2_scan_item_supported((int)T, M, K, g);
 }
 
+// From this many tokens on a TL call is cheaper as: transcode the blob to I2_S in the workspace (about 20 us for a
+// 4096 x 14336 tensor), then the tcgen05 prefill kernel -- than as ceil(T / 8) scans of the blob.
+static constexpr int64_t TL_PREFILL_MIN_T = 128;
+
 size_t bitnet_mpgemm_workspace_bytes(bitnet_fmt_t fmt, int64_t T, int64_t M, int64_t K) {
   if (T < 1 || M < 1 || K < 1) return 0;
   if (fmt == BITNET_FMT_I2S) {
@@ -226,7 +230,14 @@ size_t bitnet_mpgemm_workspace_bytes(bitnet_fmt_t fmt, int64_t T, int64_t M, int
     }
     return n;
   }
-  return gemv_tl_workspace_bytes(fmt, T, M, K);
+  size_t n = gemv_tl_workspace_bytes(fmt, T, M, K);
+  // batches of TL_PREFILL_MIN_T tokens or more are served by the tensor-core prefill kernel from an I2_S copy of the
+  // tensor made on the fly in the workspace
+  if (T >= TL_PREFILL_MIN_T && (K % 64) == 0) {
+    const size_t m = bitnet_i2s_packed_bytes(M, K);
+    if (m > n) n = m;
+  }
+  return n;
 }
 
 int bitnet_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
@@ -261,6 +272,13 @@ int bitnet_mpgemm(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
   TlGeom g;
   int rc = tl_shape(fmt, M, K, bk3, &g);
   if (rc) return rc;
+  if (T >= TL_PREFILL_MIN_T && (K % 64) == 0 && workspace && workspace_bytes >= bitnet_i2s_packed_bytes(M, K)) {
+    // many tokens: the packed tensor is turned into its I2_S form in the workspace and the tensor-core prefill
+    // kernel (whole tiles per CTA: it is given no workspace of its own) does the rest; same integers
+    rc = launch_tl_to_i2s((const uint8_t*)packed, M, K, g, (uint8_t*)workspace, st);
+    if (rc) return rc;
+    return launch_gemm_i2s_prefill((const uint8_t*)workspace, w_scale, M, K, q, act_scale, T, y, acc_out, nullptr, 0, st);
+  }
   for (int64_t t0 = 0; t0 < T; t0 += 8) {
     const int nt = (int)((T - t0 < 8) ? (T - t0) : 8);
     if (tl2_scan_takes(fmt, nt, M, K, g)) {

@@ -89,6 +89,8 @@ int launch_pack_tl(int fmt, const int8_t* w, int64_t M, int64_t K, const TlGeom&
                    int* dev_status, cudaStream_t st);
 int launch_unpack_tl(int fmt, const uint8_t* packed, int64_t M, int64_t K, const TlGeom& g, int8_t* w,
                      int* dev_status, cudaStream_t st);
+// TL blob -> I2_S blob of the same matrix (bitnet_i2s_packed_bytes(M, K) bytes), entirely on the device.
+int launch_tl_to_i2s(const uint8_t* tl, int64_t M, int64_t K, const TlGeom& g, uint8_t* i2s, cudaStream_t st);
 
 // Decode GEMV, T <= 8.
 size_t gemv_i2s_workspace_bytes(int64_t T, int64_t M, int64_t K);

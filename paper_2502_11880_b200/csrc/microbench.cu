@@ -67,31 +67,38 @@ __global__ void __launch_bounds__(MB_THREADS, 1) issue_kernel(int iters, unsigne
 #pragma unroll
   for (int i = 0; i < 8; ++i) r[i] = threadIdx.x * 97u + i;
   int c[4][4] = {};
-  const uint32_t a16 = smem_u32(tab) + threadIdx.x * 16;
+  const uint32_t a16 = smem_u32(tab) + threadIdx.x * 16;   // 128-bit loads: a quarter-warp covers all banks once
+  const uint32_t a4 = smem_u32(tab) + threadIdx.x * 4;     // 32-bit loads: one bank per lane, four 2-KB rows
   for (int it = 0; it < iters; ++it) {
 #pragma unroll
     for (int u = 0; u < 4; ++u) {          // 8 independent chains x 4 = 32 instructions of the kind per iteration
+      if (KIND == 4 || KIND == 5) {
+        // loads: all eight are issued before the first result is used (a warp issues in order), and every address
+        // comes from a register the loop changes, so that no load can be merged with another
+        unsigned v[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        if (KIND == 0) r[i] = __dp4a((int)r[i], 0x01020304, (int)r[(i + 1) & 7]);
-        if (KIND == 1) asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(r[i]) : "r"(r[(i + 1) & 7]), "r"(r[(i + 2) & 7]));
-        if (KIND == 2) asm volatile("prmt.b32 %0, %0, %1, %2;" : "+r"(r[i]) : "r"(r[(i + 1) & 7]), "r"(0x5140u + u));
-        if (KIND == 3) asm volatile("mad.lo.u32 %0, %0, %1, %2;" : "+r"(r[i]) : "r"(r[(i + 1) & 7]), "r"(r[(i + 2) & 7]));
-        // loads: the address comes from a register the loop changes, so no load can be merged with another
-        if (KIND == 4) {
-          unsigned v;
-          asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a16 + ((r[i] >> 7) & 12u)) : "memory");
-          r[i] += v | 1u;
+        for (int i = 0; i < 8; ++i) {
+          if (KIND == 4) {
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v[i]) : "r"(a4 + ((r[i] << 4) & 0x1800u)));   // lane l -> bank l
+          } else {
+            unsigned v1, v2, v3;
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                         : "=r"(v[i]), "=r"(v1), "=r"(v2), "=r"(v3)
+                         : "r"(a16 ^ ((r[i] & 1u) << 4)));
+            v[i] ^= v1 ^ v2 ^ v3;
+          }
         }
-        if (KIND == 5) {
-          unsigned v0, v1, v2, v3;
-          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                       : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3)
-                       : "r"(a16 ^ ((r[i] & 1u) << 4))
-                       : "memory");
-          r[i] += (v0 ^ v1 ^ v2 ^ v3) | 1u;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) r[i] += v[i] | 1u;
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (KIND == 0) r[i] = __dp4a((int)r[i], 0x01020304, (int)r[(i + 1) & 7]);
+          if (KIND == 1) asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(r[i]) : "r"(r[(i + 1) & 7]), "r"(r[(i + 2) & 7]));
+          if (KIND == 2) asm volatile("prmt.b32 %0, %0, %1, %2;" : "+r"(r[i]) : "r"(r[(i + 1) & 7]), "r"(0x5140u + u));
+          if (KIND == 3) asm volatile("mad.lo.u32 %0, %0, %1, %2;" : "+r"(r[i]) : "r"(r[(i + 1) & 7]), "r"(r[(i + 2) & 7]));
+          if (KIND == 6) mma_u8s8(c[i & 3], r[0], r[1], r[2], r[3], (int)r[4], (int)r[5]);
         }
-        if (KIND == 6) mma_u8s8(c[i & 3], r[0], r[1], r[2], r[3], (int)r[4], (int)r[5]);
       }
     }
   }

@@ -184,6 +184,91 @@ int launch_unpack_i2s(const uint8_t* packed, int64_t M, int64_t K, int8_t* w, in
   return check_launch();
 }
 
+// TL blob -> I2_S blob of the same matrix, for batches large enough for the tensor-core prefill kernel (which reads
+// I2_S): one thread per 32-bit word of the I2_S blob (16 weights = four runs of four consecutive columns).  A run of
+// four triple-coded columns lies in two neighbouring triples: their (sign, index) pairs go through a 32-entry table
+// to three 2-bit codes each, and a shift picks the run's four codes out of the six; a run of pair-coded columns is
+// one index byte.  A 256-entry table spreads four codes over the four bytes of the word.
+__global__ void __launch_bounds__(256) tl_to_i2s_kernel(const uint8_t* __restrict__ tl, int64_t M, int64_t K, TlGeom g,
+                                                        uint32_t* __restrict__ out) {
+  __shared__ unsigned short lut5[32];   // (sign << 4 | index) -> codes c0 | c1 << 2 | c2 << 4
+  __shared__ unsigned spread[256];      // four 2-bit codes -> one per byte
+  if (threadIdx.x < 32) {
+    int idx = threadIdx.x & 15;
+    const int neg = threadIdx.x >> 4;
+    if (idx > 13) idx = 0;
+    const int d0 = (idx + 4) / 9, rem = idx - 9 * d0, d1 = (rem + 7) / 3 - 2, d2 = rem - 3 * d1, sg = neg ? -1 : 1;
+    lut5[threadIdx.x] = (unsigned short)((sg * d0 + 1) | ((sg * d1 + 1) << 2) | ((sg * d2 + 1) << 4));
+  }
+  {
+    const unsigned x = threadIdx.x;
+    spread[x] = (x & 3u) | (((x >> 2) & 3u) << 8) | (((x >> 4) & 3u) << 16) | (((x >> 6) & 3u) << 24);
+  }
+  __syncthreads();
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int64_t kp = i2s_kp(K), mp = i2s_mp(M);
+  const int64_t nwords = mp * kp / 16;
+  const int64_t wi = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (wi >= nwords) return;
+  // word wi of the blob: 16-row unit, chunk, row in the unit, word j in the row's 64 bytes
+  const int j = (int)(wi & 15), r16 = (int)((wi >> 4) & 15);
+  const int64_t piece = wi >> 8, chunks = kp / 256;
+  const int64_t unit = piece / chunks, chunk = piece - unit * chunks;
+  const int64_t m = unit * 16 + r16;
+  unsigned word = 0x55555555u;          // weight 0 everywhere (padding rows and columns)
+  if (m < M) {
+    const int r = (int)(m & 31);
+    const uint8_t* blk = tl + (m >> 5) * g.block_bytes;
+    word = 0;
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      const int64_t k = chunk * 256 + 32 * (j >> 1) + 8 * s + 4 * (j & 1);      // the run's first column
+      unsigned codes = 0x55u;                                                   // four zeros
+      if (k < g.three_k) {
+        const int tile = (int)(k / 96), c = (int)(k - 96 * (int64_t)tile);
+        const int g0 = c / 3, d0 = c - 3 * g0;                                  // first triple of the run, digit offset
+        const uint8_t* tp = blk + (int64_t)tile * 640;
+        const unsigned signs = *reinterpret_cast<const unsigned*>(tp + tl_sign_off(r));
+        unsigned six = 0;
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const int grp = g0 + q;                                               // (g0 + 1 <= 31: a run never leaves its tile)
+          const unsigned byte = tp[tl_word_off(r, grp >> 3) + ((grp >> 1) & 3)];
+          const unsigned idx = (grp & 1) ? (byte >> 4) : (byte & 15u);
+          const unsigned neg = (signs >> tl_sign_bit(grp)) & 1u;
+          six |= (unsigned)lut5[(neg << 4) | idx] << (6 * q);
+        }
+        codes = (six >> (2 * d0)) & 0xFFu;
+      } else if (k < K) {
+        const int64_t k2 = k - g.three_k;
+        const int tile = (int)(k2 / 64), p = (int)((k2 - 64 * (int64_t)tile) >> 1);   // first pair of the run (even)
+        const uint8_t* tp = blk + g.tiles3 * 640 + (int64_t)tile * 512;
+        const unsigned byte = tp[tl_word_off(r, p >> 3) + ((p >> 1) & 3)];
+        const unsigned lo = byte & 15u, hi = byte >> 4;
+        // pair code i -> (i/3, i%3) as codes w+1; pairs beyond K carry code 4 = (0, 0)
+        codes = (lo / 3) | ((lo % 3) << 2) | ((hi / 3) << 4) | ((hi % 3) << 6);
+      }
+      word |= spread[codes] << (2 * s);
+    }
+  }
+  out[wi] = word;
+}
+
+int launch_tl_to_i2s(const uint8_t* tl, int64_t M, int64_t K, const TlGeom& g, uint8_t* i2s, cudaStream_t st) {
+  const int64_t nwords = i2s_mp(M) * i2s_kp(K) / 16;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(blocks_for(nwords, 256));
+  cfg.blockDim = dim3(256);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = early_start_enabled() ? 1 : 0;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, tl_to_i2s_kernel, tl, M, K, g, reinterpret_cast<uint32_t*>(i2s));
+  return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
+}
+
 int launch_pack_tl(int, const int8_t* w, int64_t M, int64_t K, const TlGeom& g, uint8_t* packed,
                    int* dev_status, cudaStream_t st) {
   pack_tl_kernel<<<blocks_for(M * (g.tiles3 + g.tiles2), 256), 256, 0, st>>>(w, M, K, g, packed, dev_status);

@@ -676,3 +676,26 @@ def test_read_once_switches_in_child_processes(extra):
         "assert bn.bitnet_device_status() == 0\n"
         "print('ok')\n")
     _run_child(code, extra)
+
+
+@pytest.mark.parametrize("fmt", ["tl1", "tl2"])
+def test_tl_prefill_through_the_transcode(fmt):
+    """TL blobs at prefill batch sizes: the blob is turned into its I2_S form in the workspace (device-side transcode
+    of the packed codes) and the tensor-core prefill kernel serves the call; accumulators equal the definition.  The
+    transcoded bytes themselves must equal the I2_S packer's blob of the same matrix."""
+    for i, (M, K, T) in enumerate([(320, 4096, 128), (64, 1536, 200), (160, 8640, 130), (96, 3200, 256), (32, 64, 128)]):
+        w = tern(110 + i, M, K, 0.4, 0.3)
+        x = synth.normal(111, i, T, K)
+        q, sc, _ = bn.bitnet_quant_act(x.cuda())
+        blob = bn.pack(fmt, w.cuda())
+        ws = bn.new_workspace(fmt, T, M, K)
+        assert ws.numel() >= bn.bitnet_i2s_packed_bytes(M, K)
+        y, acc = bn.bitnet_mpgemm(fmt, blob, 0.5, M, K, q, sc, want_acc=True, workspace=ws)
+        torch.cuda.synchronize()
+        q_ref, sc_ref, _ = oracle.quant_act(x.numpy())
+        acc_ref = oracle.mpgemm_def(q_ref, w.numpy())
+        assert np.array_equal(npy(acc), acc_ref), (fmt, M, K, T)
+        check_y(y, acc_ref, sc_ref, 0.5)
+        n = bn.bitnet_i2s_packed_bytes(M, K)
+        assert np.array_equal(npy(ws[:n]), oracle.pack_i2s(w.numpy())), (fmt, M, K)
+    assert bn.bitnet_device_status() == 0
