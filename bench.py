@@ -111,7 +111,7 @@ class ClockSampler:
 
     def __init__(self, gpu_index):
         import threading
-        self.sm, self.reasons, self.sm_max = [], set(), None
+        self.sm, self.mem, self.power, self.reasons, self.sm_max = [], [], [], set(), None
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -130,6 +130,8 @@ class ClockSampler:
         while not self._stop.is_set():
             try:
                 self.sm.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                self.mem.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_MEM)))
+                self.power.append(nv.nvmlDeviceGetPowerUsage(self._h) / 1000.0)
                 bits = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
                 for bit, name in self.REASONS.items():
                     if bits & bit:
@@ -143,6 +145,10 @@ class ClockSampler:
         if self._thread is not None:
             self._thread.join(timeout=2)
         out = {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": sorted(self.reasons), "samples": len(self.sm)}
+        if self.mem:
+            out["mem_mhz"] = statistics.median(self.mem)
+        if self.power:
+            out["power_w"] = statistics.median(self.power)
         if self.sm:
             out["sm_mhz"] = statistics.median(self.sm)
         elif self._nv is None:
