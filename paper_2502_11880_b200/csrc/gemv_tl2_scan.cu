@@ -86,6 +86,11 @@ __device__ __forceinline__ unsigned prmt(unsigned a, unsigned b, unsigned sel) {
   asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
   return d;
 }
+__device__ __forceinline__ unsigned mad_u32(unsigned a, unsigned b, unsigned c) {
+  unsigned d;
+  asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
 __device__ __forceinline__ void lds128(uint32_t addr, unsigned (&v)[4]) {
   asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(addr));
 }
@@ -438,10 +443,11 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
             const unsigned tw = (sg[u] >> (2 * t)) & 0x03030303u;     // sign pair of index byte j in byte j
-            e[u][0] = lds32(tbl2_lane + prmt(iw[u], tw, 0xCC40u) * 128);
-            e[u][1] = lds32(tbl2_lane + prmt(iw[u], tw, 0xDD51u) * 128);
-            e[u][2] = lds32(tbl2_lane + prmt(iw[u], tw, 0xEE62u) * 128);
-            e[u][3] = lds32(tbl2_lane + prmt(iw[u], tw, 0xFF73u) * 128);
+            // (the entry's address by a multiply-add: the FMA pipe has room, the integer pipe is the busy one)
+            e[u][0] = lds32(mad_u32(prmt(iw[u], tw, 0xCC40u), 128u, tbl2_lane));
+            e[u][1] = lds32(mad_u32(prmt(iw[u], tw, 0xDD51u), 128u, tbl2_lane));
+            e[u][2] = lds32(mad_u32(prmt(iw[u], tw, 0xEE62u), 128u, tbl2_lane));
+            e[u][3] = lds32(mad_u32(prmt(iw[u], tw, 0xFF73u), 128u, tbl2_lane));
           }
           constexpr unsigned M0 = 0x03030303u, M1 = 0x0C0C0C0Cu;
           // scale 1: index bytes 0, 1 then 2, 3; scale 4: the s=1 pairs of bytes (0, 2) and (1, 3)
