@@ -57,6 +57,18 @@ def lib():
         L.oracle_tl_build_lut.argtypes = [ci, vp, i64, ci, vp]
         L.oracle_tl_mpgemm.argtypes = [ci, vp, i64, i64, ci, vp, i64, vp]
         L.oracle_num_threads.restype = ci
+        L.oracle_elut_lo.argtypes = [ci]
+        L.oracle_elut_index_bits.argtypes = [ci, ci]
+        L.oracle_elut_bitwise_bits.argtypes = [ci]
+        L.oracle_elut_index.argtypes = [vp, ci, ci]
+        L.oracle_elut_encode.argtypes = [vp, i64, i64, ci, ci, vp]
+        L.oracle_elut_table_setup.argtypes = [vp, i64, ci, ci, vp]
+        L.oracle_elut_mpgemm.argtypes = [vp, i64, i64, ci, ci, vp, i64, vp]
+        L.oracle_elut2_packed_bytes.argtypes = [ci, i64, i64]
+        L.oracle_elut2_packed_bytes.restype = sz
+        L.oracle_pack_elut2.argtypes = [ci, vp, i64, i64, vp]
+        L.oracle_unpack_elut2.argtypes = [ci, vp, i64, i64, vp]
+        L.oracle_elut2_mpgemm.argtypes = [ci, vp, i64, i64, vp, i64, vp]
         _lib = L
     return _lib
 
@@ -199,3 +211,75 @@ def tl_mpgemm(fmt, packed, M, K, q, bk3=0):
 
 def num_threads():
     return lib().oracle_num_threads()
+
+
+# ---- element-wise tables for weights of cardinality C in groups of g (App. A)
+def elut_lo(C):
+    return lib().oracle_elut_lo(C)
+
+
+def elut_index_bits(C, g):
+    return lib().oracle_elut_index_bits(C, g)
+
+
+def elut_bitwise_bits(C):
+    return lib().oracle_elut_bitwise_bits(C)
+
+
+def elut_index(group, C):
+    group = _c(group, np.int8).reshape(-1)
+    return lib().oracle_elut_index(_p(group), C, group.shape[0])
+
+
+def elut_encode(w, C, g):
+    w = _c(w, np.int8)
+    M, K = w.shape
+    idx = np.empty((M, K // g), np.uint16)
+    _check(lib().oracle_elut_encode(_p(w), M, K, C, g, _p(idx)), "elut_encode")
+    return idx
+
+
+def elut_table_setup(q_row, C, g):
+    q_row = _c(q_row, np.int8).reshape(-1)
+    K = q_row.shape[0]
+    lut = np.empty((K // g, C ** g), np.int32)
+    _check(lib().oracle_elut_table_setup(_p(q_row), K, C, g, _p(lut)), "elut_table_setup")
+    return lut
+
+
+def elut_mpgemm(idx, K, C, g, q):
+    idx, q = _c(idx, np.uint16), _c(q, np.int8)
+    M, T = idx.shape[0], q.shape[0]
+    acc = np.empty((T, M), np.int32)
+    _check(lib().oracle_elut_mpgemm(_p(idx), M, K, C, g, _p(q), T, _p(acc)), "elut_mpgemm")
+    return acc
+
+
+def elut2_packed_bytes(C, M, K):
+    return lib().oracle_elut2_packed_bytes(C, M, K)
+
+
+def pack_elut2(C, w):
+    w = _c(w, np.int8)
+    M, K = w.shape
+    n = elut2_packed_bytes(C, M, K)
+    if n == 0:
+        raise ValueError("unsupported ELUT shape")
+    out = np.empty(n, np.uint8)
+    _check(lib().oracle_pack_elut2(C, _p(w), M, K, _p(out)), "pack_elut2")
+    return out
+
+
+def unpack_elut2(C, packed, M, K):
+    packed = _c(packed, np.uint8)
+    w = np.empty((M, K), np.int8)
+    _check(lib().oracle_unpack_elut2(C, _p(packed), M, K, _p(w)), "unpack_elut2")
+    return w
+
+
+def elut2_mpgemm(C, packed, M, K, q):
+    packed, q = _c(packed, np.uint8), _c(q, np.int8)
+    T = q.shape[0]
+    acc = np.empty((T, M), np.int32)
+    _check(lib().oracle_elut2_mpgemm(C, _p(packed), M, K, _p(q), T, _p(acc)), "elut2_mpgemm")
+    return acc

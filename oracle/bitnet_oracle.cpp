@@ -20,6 +20,9 @@
 //   oracle_tl_mpgemm      Alg. 3 / Alg. 4 accumulation by table lookups from the packed blob,
 //                         sign applied per group (caption of Fig. 5).
 //   oracle_i2s_mpgemm     Alg. 1 Phase 2 evaluated straight from the I2_S blob.
+//   oracle_elut_*         App. A: the element-wise table method for weights of any cardinality C in groups of
+//                         g ("ELUT mpGEMM": Tbl-quantization, Table-setup, then one Lookup per group), the
+//                         bits-per-weight figures of Table 3, and a packed form of the g = 2 case.
 //
 // Readings where the paper is silent (all listed in the design notes):
 //   * activations are quantised per token (row of x); per_tensor != 0 gives the paper's
@@ -28,7 +31,11 @@
 //     with round-half-to-even; act_scale = amax / 127 in binary32;
 //   * TL2 code of a triple: v = 9*w0 + 3*w1 + w2, index = |v|, sign = [v < 0] -- this
 //     reproduces every printed row of Table 5;
-//   * TL1 code of a pair: 3*(w0+1) + (w1+1) -- Table 4.
+//   * TL1 code of a pair: 3*(w0+1) + (w1+1) -- Table 4;
+//   * App. A gives weights "of cardinality C" without naming the values: here the C consecutive integers
+//     from -(C/2) (integer division) upwards -- {-1,0,1} for C = 3 (the ternary case), {-2,..,1} for C = 4 (two's
+//     complement int2), {-2,..,2} for C = 5; the index of a group is its weights read as a base-C number, first
+//     weight most significant, each digit = weight + C/2 -- for C = 3, g = 2 exactly the codes of Table 4.
 //
 // Pins (tests/test_oracle_*.py): closed-form quantiser cases, brute-force enumeration on tiny
 // shapes against numpy, one-hot position probes of every packed bit, Tables 4 and 5 as golden
@@ -431,6 +438,199 @@ int oracle_tl_mpgemm(int fmt, const uint8_t* packed, int64_t M, int64_t K, int b
           const uint8_t byte = tile[tl_idx_pos((int)r, grp)];
           const int idx = (grp & 1) ? (byte >> 4) : (byte & 15);
           s += lut[(g.tiles3 * 32 + tile_i * 32 + grp) * 16 + idx];
+        }
+      }
+      acc[t * M + m] = (int32_t)s;
+    }
+  }
+  return 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// ELUT beyond ternary (App. A).  Weights take C consecutive integer values from lo = -(C/2); g of them form a
+// group; a group is stored as its index in [0, C^g) and costs ceil(log2(C^g)) bits (Table 3: bpw_e = that / g,
+// against ceil(log2 C) bits per weight for bit-wise storage).
+static int64_t ipow(int64_t c, int g) {
+  int64_t p = 1;
+  for (int i = 0; i < g; ++i) p *= c;
+  return p;
+}
+static bool elut_ok(int C, int g) { return C >= 2 && C <= 16 && g >= 1 && g <= 8 && ipow(C, g) <= 65536; }
+
+int oracle_elut_lo(int C) { return -(C / 2); }
+// smallest b with 2^b >= n
+static int bits_for(int64_t n) {
+  int b = 0;
+  while (((int64_t)1 << b) < n) ++b;
+  return b;
+}
+int oracle_elut_index_bits(int C, int g) { return elut_ok(C, g) ? bits_for(ipow(C, g)) : -1; }   // bpw_e * g
+int oracle_elut_bitwise_bits(int C) { return (C >= 2 && C <= 16) ? bits_for(C) : -1; }           // bpw_b
+
+// Index of one group: digits w_i - lo, first weight most significant.  -1 if a weight lies outside the alphabet.
+int oracle_elut_index(const int8_t* w, int C, int g) {
+  if (!elut_ok(C, g)) return -1;
+  const int lo = oracle_elut_lo(C);
+  int idx = 0;
+  for (int i = 0; i < g; ++i) {
+    const int d = (int)w[i] - lo;
+    if (d < 0 || d >= C) return -1;
+    idx = idx * C + d;
+  }
+  return idx;
+}
+
+// Offline step: every group of every row -> its index.  idx[M][K/g].
+int oracle_elut_encode(const int8_t* w, int64_t M, int64_t K, int C, int g, uint16_t* idx) {
+  if (!w || !idx || M < 1 || K < 1 || !elut_ok(C, g) || K % g != 0) return 1;
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t k = 0; k < K / g; ++k) {
+      const int v = oracle_elut_index(w + m * K + k * g, C, g);
+      if (v < 0) return 3;
+      idx[m * (K / g) + k] = (uint16_t)v;
+    }
+  return 0;
+}
+
+// Phase 1, "Table-setup": for one token, lut[k][i] = sum_j digit_j(i) * a[g k + j] for every group k and every one
+// of the C^g weight combinations i (digit_j(i) = the j-th weight of the group whose index is i).
+int oracle_elut_table_setup(const int8_t* q, int64_t K, int C, int g, int32_t* lut) {
+  if (!q || !lut || K < 1 || !elut_ok(C, g) || K % g != 0) return 1;
+  const int lo = oracle_elut_lo(C);
+  const int64_t n = ipow(C, g);
+  for (int64_t k = 0; k < K / g; ++k)
+    for (int64_t i = 0; i < n; ++i) {
+      int64_t rest = i, s = 0;
+      for (int j = g - 1; j >= 0; --j) {      // least significant digit = last weight of the group
+        const int wj = (int)(rest % C) + lo;
+        rest /= C;
+        s += (int64_t)wj * q[k * g + j];
+      }
+      lut[k * n + i] = (int32_t)s;
+    }
+  return 0;
+}
+
+// Phase 2, accumulation: R[n, m] = sum over groups k of Lookup(LUT[n, k], W[m, k]).
+int oracle_elut_mpgemm(const uint16_t* idx, int64_t M, int64_t K, int C, int g, const int8_t* q, int64_t T,
+                       int32_t* acc) {
+  if (!idx || !q || !acc || M < 1 || T < 1 || K < 1 || !elut_ok(C, g) || K % g != 0) return 1;
+  const int64_t n = ipow(C, g), ng = K / g;
+  std::vector<int32_t> lut((size_t)(ng * n));
+  for (int64_t t = 0; t < T; ++t) {
+    if (oracle_elut_table_setup(q + t * K, K, C, g, lut.data())) return 1;
+    for (int64_t m = 0; m < M; ++m) {
+      int64_t s = 0;
+      for (int64_t k = 0; k < ng; ++k) {
+        const int64_t i = idx[m * ng + k];
+        if (i >= n) return 3;
+        s += lut[k * n + i];
+      }
+      acc[t * M + m] = (int32_t)s;
+    }
+  }
+  return 0;
+}
+
+// Packed form of the g = 2 case for C = 3, 4, 5 (index of 4 bits for C <= 4, 5 bits for C = 5: Table 3's 2 and 2.5
+// bits per weight).  Same 32-row blocks and tile geometry as the TL blobs: a tile covers 32 pairs (64 columns) of
+// 32 rows; its first 512 bytes hold the low four bits of every index (pair 2i of a row in the low nibble of the
+// row's byte i, pair 2i+1 in the high nibble; bytes placed as tl_idx_pos says); for C = 5 a 128-byte plane follows
+// with the fifth bit (row r's uint32 at tl_sign_pos(r), pair grp at bit tl_sign_bit(grp)).  Columns past K are
+// zero weights.  For C = 3 the blob equals the TL1 blob byte for byte.
+static bool elut2_geom(int C, int64_t M, int64_t K, int64_t* tiles, int64_t* tile_bytes) {
+  if (C < 3 || C > 5 || M < 32 || M % 32 != 0 || K < 2 || K % 2 != 0) return false;
+  *tiles = (K + 63) / 64;
+  *tile_bytes = (C == 5) ? 640 : 512;
+  return true;
+}
+
+size_t oracle_elut2_packed_bytes(int C, int64_t M, int64_t K) {
+  int64_t tiles, tb;
+  if (!elut2_geom(C, M, K, &tiles, &tb)) return 0;
+  return (size_t)(M / 32) * (size_t)(tiles * tb);
+}
+
+int oracle_pack_elut2(int C, const int8_t* w, int64_t M, int64_t K, uint8_t* packed) {
+  int64_t tiles, tb;
+  if (!w || !packed || !elut2_geom(C, M, K, &tiles, &tb)) return 1;
+  std::memset(packed, 0, (size_t)(M / 32) * (size_t)(tiles * tb));
+  const int8_t zero_pair[2] = {0, 0};
+  for (int64_t m = 0; m < M; ++m) {
+    const int64_t rb = m / 32, r = m % 32;
+    for (int64_t t = 0; t < tiles; ++t) {
+      uint8_t* tile = packed + (rb * tiles + t) * tb;
+      uint32_t high = 0;
+      for (int grp = 0; grp < 32; ++grp) {
+        const int64_t k = t * 64 + 2 * grp;
+        const int idx = oracle_elut_index(k < K ? w + m * K + k : zero_pair, C, 2);
+        if (idx < 0) return 3;
+        tile[tl_idx_pos((int)r, grp)] |= (uint8_t)((grp & 1) ? ((idx & 15) << 4) : (idx & 15));
+        if (idx & 16) high |= 1u << tl_sign_bit(grp);
+      }
+      if (tb == 640)
+        for (int b = 0; b < 4; ++b) tile[tl_sign_pos((int)r) + b] = (uint8_t)(high >> (8 * b));
+    }
+  }
+  return 0;
+}
+
+// The index of pair grp of row r of a tile, read back.
+static int elut2_read(const uint8_t* tile, int64_t tb, int r, int grp) {
+  const uint8_t byte = tile[tl_idx_pos(r, grp)];
+  int idx = (grp & 1) ? (byte >> 4) : (byte & 15);
+  if (tb == 640) {
+    uint32_t high = 0;
+    for (int b = 0; b < 4; ++b) high |= (uint32_t)tile[tl_sign_pos(r) + b] << (8 * b);
+    idx |= (int)((high >> tl_sign_bit(grp)) & 1u) << 4;
+  }
+  return idx;
+}
+
+int oracle_unpack_elut2(int C, const uint8_t* packed, int64_t M, int64_t K, int8_t* w) {
+  int64_t tiles, tb;
+  if (!w || !packed || !elut2_geom(C, M, K, &tiles, &tb)) return 1;
+  const int lo = oracle_elut_lo(C);
+  for (int64_t m = 0; m < M; ++m) {
+    const int64_t rb = m / 32, r = m % 32;
+    for (int64_t t = 0; t < tiles; ++t) {
+      const uint8_t* tile = packed + (rb * tiles + t) * tb;
+      for (int grp = 0; grp < 32; ++grp) {
+        const int idx = elut2_read(tile, tb, (int)r, grp);
+        if (idx >= C * C) return 3;
+        const int w0 = idx / C + lo, w1 = idx % C + lo;
+        const int64_t k = t * 64 + 2 * grp;
+        if (k < K) {
+          w[m * K + k] = (int8_t)w0;
+          w[m * K + k + 1] = (int8_t)w1;
+        } else if (w0 != 0 || w1 != 0) {
+          return 3;
+        }
+      }
+    }
+  }
+  return 0;
+}
+
+// "ELUT mpGEMM" straight from the packed blob: tables per token, one lookup per stored index.
+int oracle_elut2_mpgemm(int C, const uint8_t* packed, int64_t M, int64_t K, const int8_t* q, int64_t T, int32_t* acc) {
+  int64_t tiles, tb;
+  if (!packed || !q || !acc || T < 1 || !elut2_geom(C, M, K, &tiles, &tb)) return 1;
+  const int64_t n = (int64_t)C * C, kp = tiles * 64;
+  std::vector<int8_t> qp((size_t)kp);
+  std::vector<int32_t> lut((size_t)(kp / 2 * n));
+  for (int64_t t = 0; t < T; ++t) {
+    for (int64_t k = 0; k < kp; ++k) qp[k] = k < K ? q[t * K + k] : (int8_t)0;
+    if (oracle_elut_table_setup(qp.data(), kp, C, 2, lut.data())) return 1;
+    for (int64_t m = 0; m < M; ++m) {
+      const int64_t rb = m / 32, r = m % 32;
+      int64_t s = 0;
+      for (int64_t ti = 0; ti < tiles; ++ti) {
+        const uint8_t* tile = packed + (rb * tiles + ti) * tb;
+        for (int grp = 0; grp < 32; ++grp) {
+          const int idx = elut2_read(tile, tb, (int)r, grp);
+          if (idx >= n) return 3;
+          s += lut[(ti * 32 + grp) * n + idx];
         }
       }
       acc[t * M + m] = (int32_t)s;

@@ -411,3 +411,160 @@ def test_tl2_one_hot_across_split_and_tile_boundaries():
     for i, k in enumerate(probes):
         assert acc[0, i] == (1 if i % 2 == 0 else -1) * int(q[0, k])
     assert not acc[0, len(probes):].any()
+
+
+# ----------------------------------------------------------------------------- ELUT beyond ternary (App. A)
+def rand_alphabet(M, K, C):
+    return rng.integers(-(C // 2), -(C // 2) + C, size=(M, K)).astype(np.int8)
+
+
+def test_elut_bits_per_weight_match_table3():
+    rows = _read_rows("elut_table3.txt")
+    assert len(rows) == 3
+    for C, g, bpw_b, bpw_e in rows:
+        C, g = int(C), int(g)
+        assert oracle.elut_bitwise_bits(C) == int(bpw_b)
+        assert round(oracle.elut_index_bits(C, g) / g, 2) == float(bpw_e)
+    # a group index needs the smallest b with 2^b >= C^g
+    for C, g in itertools.product(range(2, 9), range(1, 5)):
+        b = oracle.elut_index_bits(C, g)
+        assert 2 ** b >= C ** g > 2 ** (b - 1) or (C ** g == 1 and b == 0)
+
+
+def test_elut_alphabet_and_index_are_base_c_digits():
+    assert [oracle.elut_lo(C) for C in (2, 3, 4, 5, 8)] == [-1, -1, -2, -2, -4]
+    for C, g in [(3, 2), (3, 3), (4, 2), (5, 2), (4, 3), (3, 5)]:
+        lo = -(C // 2)
+        seen = set()
+        for grp in itertools.product(range(lo, lo + C), repeat=g):
+            want = 0
+            for wv in grp:                       # Horner, first weight most significant
+                want = want * C + (wv - lo)
+            got = oracle.elut_index(grp, C)
+            assert got == want
+            seen.add(got)
+        assert seen == set(range(C ** g))        # a bijection onto [0, C^g)
+        assert oracle.elut_index([lo - 1] + [0] * (g - 1), C) == -1
+        assert oracle.elut_index([0] * (g - 1) + [lo + C], C) == -1
+    # the all-zero group sits in the middle of the odd alphabets' range
+    assert oracle.elut_index([0, 0], 5) == 12 and oracle.elut_index([0, 0], 4) == 10 and oracle.elut_index([0, 0], 3) == 4
+
+
+def test_elut_ternary_pairs_are_table4_and_triples_are_table5():
+    for w0, w1, code in _read_rows("tl1_table4.txt"):
+        assert oracle.elut_index([int(w0), int(w1)], 3) == int(code, 2)
+    # Table 5 is the mirror-consolidated form of the 27-entry table: v = index - 13, |v| its index, v < 0 its sign
+    for w0, w1, w2, sign, idx in _read_rows("tl2_table5.txt"):
+        v = oracle.elut_index([int(w0), int(w1), int(w2)], 3) - 13
+        assert abs(v) == int(idx, 2) and int(v < 0) == int(sign)
+
+
+@pytest.mark.parametrize("C,g", [(3, 2), (3, 3), (4, 2), (5, 2), (4, 3), (5, 3), (3, 5), (16, 2)])
+def test_elut_table_setup_entries_by_brute_force(C, g):
+    K = 6 * g
+    q = rand_q(1, K)[0]
+    lut = oracle.elut_table_setup(q, C, g)
+    assert lut.shape == (K // g, C ** g)
+    lo = -(C // 2)
+    for k in range(K // g):
+        a = [int(v) for v in q[g * k: g * k + g]]
+        for i, grp in enumerate(itertools.product(range(lo, lo + C), repeat=g)):   # lexicographic = index order
+            assert lut[k, i] == sum(wv * av for wv, av in zip(grp, a))
+        zero = oracle.elut_index([0] * g, C)
+        assert lut[k, zero] == 0
+        if C % 2 == 1:                           # symmetric alphabet: the table is odd about its middle
+            assert all(lut[k, i] + lut[k, C ** g - 1 - i] == 0 for i in range(C ** g))
+
+
+def test_elut_tables_reduce_to_the_ternary_ones():
+    q = rand_q(1, 96 * 2)[0]
+    pair = oracle.elut_table_setup(q, 3, 2)
+    tl1 = oracle.tl_build_lut("tl1", q)                   # Alg. 3 PreCompute, 9 of 16 slots used
+    assert np.array_equal(pair, tl1[: pair.shape[0], :9])
+    triple = oracle.elut_table_setup(q, 3, 3)
+    tl2 = oracle.tl_build_lut("tl2", q)                   # Alg. 4 PreCompute: the non-negative half
+    for v in range(-13, 14):
+        assert np.array_equal(triple[:, 13 + v], np.sign(v) * tl2[:, abs(v)] if v else tl2[:, 0])
+
+
+@pytest.mark.parametrize("C,g,K", [(3, 2, 64), (3, 3, 96), (4, 2, 130), (5, 2, 70), (5, 3, 99), (4, 4, 64), (3, 5, 80)])
+def test_elut_lookup_accumulation_gives_the_definition(C, g, K):
+    T, M = 3, 40
+    q, w = rand_q(T, K), rand_alphabet(M, K, C)
+    ref = q.astype(np.int64) @ w.astype(np.int64).T
+    assert np.array_equal(oracle.mpgemm_def(q, w), ref)
+    idx = oracle.elut_encode(w, C, g)
+    assert idx.max() < C ** g
+    assert np.array_equal(oracle.elut_mpgemm(idx, K, C, g, q), ref)
+    bad = w.copy()
+    bad[0, 0] = -(C // 2) + C
+    with pytest.raises(ValueError):
+        oracle.elut_encode(bad, C, g)
+
+
+@pytest.mark.parametrize("C", [3, 4, 5])
+def test_elut2_blob_size_round_trip_and_definition(C):
+    # 4 bits per pair for C <= 4, 5 bits for C = 5: 2 and 2.5 bits per weight (Table 3)
+    assert oracle.elut2_packed_bytes(C, 64, 128) * 8 == (5 if C == 5 else 4) * 64 * 128 // 2
+    assert oracle.elut2_packed_bytes(C, 33, 64) == 0 and oracle.elut2_packed_bytes(C, 32, 65) == 0
+    assert oracle.elut2_packed_bytes(6, 32, 64) == 0
+    for K in (64, 130, 2, 192 + 34):
+        T, M = 2, 64
+        q, w = rand_q(T, K), rand_alphabet(M, K, C)
+        p = oracle.pack_elut2(C, w)
+        assert p.size == oracle.elut2_packed_bytes(C, M, K) == (M // 32) * ((K + 63) // 64) * (640 if C == 5 else 512)
+        assert np.array_equal(oracle.unpack_elut2(C, p, M, K), w)
+        assert np.array_equal(oracle.elut2_mpgemm(C, p, M, K, q), q.astype(np.int64) @ w.astype(np.int64).T)
+    with pytest.raises(ValueError):
+        oracle.pack_elut2(C, np.full((32, 64), -(C // 2) - 1, np.int8))
+
+
+def test_elut2_ternary_blob_is_the_tl1_blob():
+    w = rand_ternary(64, 192 + 34)
+    assert np.array_equal(oracle.pack_elut2(3, w), oracle.pack_tl("tl1", w))
+
+
+def test_elut2_documented_byte_positions():
+    """C = 5: pair grp of row r = g + 8u has index 5(w0+2) + (w1+2); its low four bits sit in the nibble of index
+    byte i = grp//2 (grp odd: high nibble) at 64g + 16(i//4) + 4u + i%4, its fifth bit at bit 8(i%4) + 2(i//4) + grp%2
+    of the word at 512 + 16g + 4u.  Zero weights have index 12: every other nibble is 0xC, every other high bit 0."""
+    w = np.zeros((32, 64), np.int8)
+    w[5, 14:16] = (2, 1)        # index 23 = 16 + 7: row 5 = (g 5, u 0), pair 7 -> byte i = 3, high nibble; bit 8*3+0+1
+    w[31, 60:62] = (-2, -1)     # index 1: row 31 = (g 7, u 3), pair 30 -> byte i = 15, low nibble
+    w[9, 0:2] = (1, 2)          # index 19 = 16 + 3: row 9 = (g 1, u 1), pair 0 -> byte 0, low nibble; bit 0
+    p = oracle.pack_elut2(5, w)
+    expect = np.zeros(640, np.uint8)
+    expect[:512] = 0xCC
+    expect[64 * 5 + 3] = 0x7C
+    expect[512 + 16 * 5 + 3] = 1 << 1
+    expect[64 * 7 + 16 * 3 + 4 * 3 + 3] = 0xC1
+    expect[64 * 1 + 4 * 1] = 0xC3
+    expect[512 + 16 * 1 + 4 * 1] = 1
+    assert np.array_equal(p, expect)
+    # C = 4: index 4(w0+2) + (w1+2), four bits, no second plane; zero weights have index 10
+    w4 = np.zeros((32, 34), np.int8)
+    w4[2, 0:2] = (1, -2)        # index 12
+    w4[26, 2:4] = (-2, 1)       # index 3: row 26 = (g 2, u 3), pair 1 -> high nibble of byte 0
+    p4 = oracle.pack_elut2(4, w4)
+    expect4 = np.full(512, 0xAA, np.uint8)
+    expect4[64 * 2] = 0xAC
+    expect4[64 * 2 + 4 * 3] = 0x3A
+    assert np.array_equal(p4, expect4)
+
+
+@pytest.mark.parametrize("C", [4, 5])
+def test_elut2_one_hot_dot_products(C):
+    # a single non-zero weight v at column k against q[k] returns exactly v * q[k], for every column of two tiles
+    K = 128
+    q = ((np.arange(K) * 7) % 251 - 125).astype(np.int8).reshape(1, K)
+    lo = -(C // 2)
+    vals = [v for v in range(lo, lo + C) if v != 0]
+    rows = [(k, v) for k in range(K) for v in vals]
+    M = ((len(rows) + 31) // 32) * 32
+    w = np.zeros((M, K), np.int8)
+    for i, (k, v) in enumerate(rows):
+        w[i, k] = v
+    acc = oracle.elut2_mpgemm(C, oracle.pack_elut2(C, w), M, K, q)
+    for i, (k, v) in enumerate(rows):
+        assert acc[0, i] == v * int(q[0, k])
+    assert not acc[0, len(rows):].any()
