@@ -283,6 +283,50 @@ int bitnet_linear_segments(bitnet_fmt_t fmt, const void* packed, int64_t M, int6
                            void* stream);
 
 /*
+ * Element-wise tables beyond ternary (App. A, "ELUT mpGEMM"; Table 3).  Weights of cardinality C take the C
+ * consecutive integers from -(C/2) (integer division): {-1,0,1} for C = 3, {-2,..,1} for C = 4, {-2,..,2} for
+ * C = 5.  g weights form a group, stored as the group's index = its weights + C/2 read as a base-C number, first
+ * weight most significant, in ceil(log2(C^g)) bits.  Built: g = 2 with C = 3, 4 (4 bits per pair: 2 bits per
+ * weight) and C = 5 (5 bits per pair: 2.5 bits per weight, against 3 for bit-wise storage); other (C, g) return
+ * BITNET_ERR_UNSUPPORTED_SHAPE.
+ *
+ * Blob (M a multiple of 32, K even; the kernels need K a multiple of 4): 32-row blocks, each a sequence of
+ * ceil(K/64) tiles of 32 rows x 32 pairs.  A tile's first 512 bytes hold the low four bits of every index exactly
+ * where a TL1 tile keeps its codes (see bitnet_pack_tl); for C = 5 another 128 bytes follow with the fifth bits,
+ * placed where a TL2 tile keeps its signs.  Columns past K are zero weights.  For C = 3 the blob is the TL1 blob.
+ *
+ * bitnet_pack_elut: w[M][K] int8 in the alphabet -> packed; dev_status (nullable device int) is set to
+ * BITNET_ERR_BAD_WEIGHT if a value outside the alphabet is met.  bitnet_unpack_elut is its inverse (a test hook).
+ *
+ * bitnet_elut_linear_group: a list of linear layers (as bitnet_linear_group: y = acc * act_scale[t] * w_scale,
+ * acc[t,m] = sum_k q[t,k] w[m,k]) over such blobs, 1..8 tokens each, on DEVICE buffers.  Per item x[T][K] fp32 in and
+ * q, act_scale out (Phase 1 runs inside the kernel) -- or x = NULL and q, act_scale are inputs.  Runs of items
+ * with the same C are ONE persistent kernel that reads every blob once: an index byte plus its fifth bits selects
+ * an entry of a shared-memory table that holds the four weights of the two pairs, which go to the int8 tensor cores
+ * as they are (the table is indexed by the packed weights rather than filled from the activations: Phase 1 of the
+ * algorithm then costs nothing per token and the lookups feed 4 weights x 8 tokens each).  Integer results are
+ * exact.  Errors: BITNET_ERR_INVALID_ARG (null or misaligned pointer, T outside 1..8), BITNET_ERR_UNSUPPORTED_SHAPE
+ * ((C, g) not built, M % 32, K % 4, rows too short for the kernel's rings: K < 192); nothing is queued then.
+ */
+size_t bitnet_elut_packed_bytes(int C, int g, int64_t M, int64_t K);
+int bitnet_pack_elut(int C, int g, const int8_t* w, int64_t M, int64_t K, void* packed, size_t packed_bytes,
+                     int* dev_status, void* stream);
+int bitnet_unpack_elut(int C, int g, const void* packed, int64_t M, int64_t K, int8_t* w, int* dev_status,
+                       void* stream);
+typedef struct bitnet_elut_item {
+  int32_t C, g;
+  const void* packed;
+  float w_scale;
+  int64_t M, K, T;
+  const float* x;         /* [T][K] fp32, device; NULL: q and act_scale are inputs */
+  int8_t* q;              /* [T][K] int8, device */
+  float* act_scale;       /* [T] fp32, device */
+  float* y;               /* [T][M] fp32, device, out */
+  int32_t* acc_out;       /* [T][M] int32, device, out, nullable */
+} bitnet_elut_item_t;
+int bitnet_elut_linear_group(const bitnet_elut_item_t* items, int64_t n, void* stream);
+
+/*
  * Table-lookup mpGEMV without a workspace argument (the paper has no counterpart: this entry point
  * exists for the sake of callers, not of the method).
  *

@@ -27,6 +27,7 @@ SYMBOLS = [
     "bitnet_workspace_init", "bitnet_mpgemm", "bitnet_linear", "bitnet_linear_host", "bitnet_linear_host_batch", "bitnet_unpack_i2s", "bitnet_unpack_tl",
     "bitnet_tl_num_groups", "bitnet_tl_build_lut_debug", "bitnet_mpgemv_tl_noalloc", "bitnet_device_status",
     "bitnet_set_early_start", "bitnet_set_tl2_lookup", "bitnet_device_status_clear", "bitnet_debug_wait_timeout_probe", "bitnet_linear_group", "bitnet_linear_segments", "bitnet_microbench_read_stream", "bitnet_microbench_issue",
+    "bitnet_elut_packed_bytes", "bitnet_pack_elut", "bitnet_unpack_elut", "bitnet_elut_linear_group",
 ]
 
 _lib = None
@@ -78,6 +79,11 @@ def lib():
         L.bitnet_tl_num_groups.restype = i64
         L.bitnet_tl_build_lut_debug.argtypes = [ci, vp, i64, ci, vp, vp]
         L.bitnet_mpgemv_tl_noalloc.argtypes = [ci, vp, fl, i64, i64, ci, vp, vp, i64, vp, vp, vp]
+        L.bitnet_elut_packed_bytes.argtypes = [ci, ci, i64, i64]
+        L.bitnet_elut_packed_bytes.restype = sz
+        L.bitnet_pack_elut.argtypes = [ci, ci, vp, i64, i64, vp, sz, vp, vp]
+        L.bitnet_unpack_elut.argtypes = [ci, ci, vp, i64, i64, vp, vp, vp]
+        L.bitnet_elut_linear_group.argtypes = [vp, i64, vp]
         _lib = L
     return _lib
 
@@ -379,6 +385,63 @@ def bitnet_linear_group(group, stream=None):
     """Queues a list of linears made by make_group (device buffers): one persistent kernel per run of I2_S
     decode items, bitnet_linear for the others."""
     _check(lib().bitnet_linear_group(group, C.c_int64(len(group)), _stream(stream)), "bitnet_linear_group")
+
+
+# ---- element-wise tables beyond ternary (App. A): weights of cardinality C in groups of g
+def bitnet_elut_packed_bytes(C_, g, M, K) -> int:
+    return lib().bitnet_elut_packed_bytes(int(C_), int(g), M, K)
+
+
+def bitnet_pack_elut(C_, g, w, check=True, stream=None):
+    """w[M][K] int8 with values -(C//2) .. -(C//2)+C-1 (CUDA) -> uint8 blob of group indices."""
+    _dev(w, torch.int8, "w")
+    M, K = w.shape
+    n = bitnet_elut_packed_bytes(C_, g, M, K)
+    if n == 0:
+        _check(2, "bitnet_pack_elut")
+    out = torch.empty(n, dtype=torch.uint8, device=w.device)
+    st = _status_word(w.device) if check else None
+    _check(lib().bitnet_pack_elut(int(C_), int(g), _ptr(w), M, K, _ptr(out), n, _ptr(st), _stream(stream)),
+           "bitnet_pack_elut")
+    if check:
+        _check(int(st.item()), "bitnet_pack_elut")
+    return out
+
+
+def bitnet_unpack_elut(C_, g, packed, M, K, stream=None):
+    w = torch.empty((M, K), dtype=torch.int8, device=packed.device)
+    st = _status_word(packed.device)
+    _check(lib().bitnet_unpack_elut(int(C_), int(g), _ptr(packed), M, K, _ptr(w), _ptr(st), _stream(stream)),
+           "bitnet_unpack_elut")
+    _check(int(st.item()), "bitnet_unpack_elut")
+    return w
+
+
+class ElutItem(C.Structure):
+    """Mirror of bitnet_elut_item_t."""
+    _fields_ = [("C", C.c_int32), ("g", C.c_int32), ("packed", C.c_void_p), ("w_scale", C.c_float),
+                ("M", C.c_int64), ("K", C.c_int64), ("T", C.c_int64), ("x", C.c_void_p), ("q", C.c_void_p),
+                ("act_scale", C.c_void_p), ("y", C.c_void_p), ("acc_out", C.c_void_p)]
+
+
+def make_elut_group(items):
+    """items: dicts with C, g, packed, w_scale, M, K, q, act_scale, y and optionally x (fp32 activations: q and
+    act_scale are then outputs) and acc_out (CUDA tensors).  Returns the ctypes array for bitnet_elut_linear_group;
+    the caller keeps the tensors alive."""
+    arr = (ElutItem * len(items))()
+    for a, d in zip(arr, items):
+        x, acc = d.get("x"), d.get("acc_out")
+        a.C, a.g, a.packed, a.w_scale = int(d["C"]), int(d["g"]), d["packed"].data_ptr(), float(d["w_scale"])
+        a.M, a.K, a.T = int(d["M"]), int(d["K"]), int(d["q"].shape[0])
+        a.x = None if x is None else x.data_ptr()
+        a.q, a.act_scale, a.y = d["q"].data_ptr(), d["act_scale"].data_ptr(), d["y"].data_ptr()
+        a.acc_out = None if acc is None else acc.data_ptr()
+    return arr
+
+
+def bitnet_elut_linear_group(group, stream=None):
+    """Queues a list made by make_elut_group: one persistent kernel per run of items with the same C."""
+    _check(lib().bitnet_elut_linear_group(group, C.c_int64(len(group)), _stream(stream)), "bitnet_elut_linear_group")
 
 
 MICROBENCH_KINDS = {"dp4a": 0, "lop3": 1, "prmt": 2, "imad": 3, "lds32": 4, "lds128": 5, "mma_u8s8_m16n8k32": 6}

@@ -77,7 +77,7 @@ const char* bitnet_status_string(int status) {
     case BITNET_ERR_INVALID_ARG: return "invalid argument (null or misaligned pointer, bad enum or size)";
     case BITNET_ERR_UNSUPPORTED_SHAPE: return "unsupported shape for this weight format";
     case BITNET_ERR_WORKSPACE: return "workspace missing or too small";
-    case BITNET_ERR_BAD_WEIGHT: return "weight outside {-1,0,+1} or invalid packed code";
+    case BITNET_ERR_BAD_WEIGHT: return "weight outside the format's alphabet or invalid packed code";
     case BITNET_ERR_CUDA: return "CUDA call failed (see bitnet_last_cuda_error)";
     case BITNET_ERR_TIMEOUT: return "bounded device-side wait gave up";
     default: return "unknown status";
@@ -533,6 +533,76 @@ int bitnet_linear_segments(bitnet_fmt_t fmt, const void* packed, int64_t M, int6
   rc = bitnet_linear(fmt, packed, 1.0f, M, K, bk3, x, T, q, act_scale, y, acc_out, workspace, workspace_bytes, stream);
   if (rc) return rc;
   return launch_scale_segments(y, T, M, (int)n_seg, seg_end, seg_scale, st);
+}
+
+// ---- element-wise tables beyond ternary (App. A): g = 2, C = 3, 4, 5
+static int elut_shape(int C, int g, int64_t M, int64_t K, TlGeom* geom) {
+  if (C < 2 || g < 1 || M < 1 || K < 1 || M > 0x7fffffff) return BITNET_ERR_INVALID_ARG;
+  if (g != 2 || !elut2_geom(C, M, K, geom)) return BITNET_ERR_UNSUPPORTED_SHAPE;
+  return BITNET_OK;
+}
+
+size_t bitnet_elut_packed_bytes(int C, int g, int64_t M, int64_t K) {
+  TlGeom geom;
+  if (elut_shape(C, g, M, K, &geom)) return 0;
+  return (size_t)(M / 32) * (size_t)geom.block_bytes;
+}
+
+int bitnet_pack_elut(int C, int g, const int8_t* w, int64_t M, int64_t K, void* packed, size_t packed_bytes,
+                     int* dev_status, void* stream) {
+  if (!w || !packed || !aligned16(packed)) return BITNET_ERR_INVALID_ARG;
+  TlGeom geom;
+  int rc = elut_shape(C, g, M, K, &geom);
+  if (rc) return rc;
+  if (packed_bytes < (size_t)(M / 32) * (size_t)geom.block_bytes) return BITNET_ERR_INVALID_ARG;
+  return launch_pack_elut2(C, w, M, K, geom, (uint8_t*)packed, dev_status, (cudaStream_t)stream);
+}
+
+int bitnet_unpack_elut(int C, int g, const void* packed, int64_t M, int64_t K, int8_t* w, int* dev_status,
+                       void* stream) {
+  if (!w || !packed || !aligned16(packed)) return BITNET_ERR_INVALID_ARG;
+  TlGeom geom;
+  int rc = elut_shape(C, g, M, K, &geom);
+  if (rc) return rc;
+  return launch_unpack_elut2(C, (const uint8_t*)packed, M, K, geom, w, dev_status, (cudaStream_t)stream);
+}
+
+int bitnet_elut_linear_group(const bitnet_elut_item_t* items, int64_t n, void* stream) {
+  if (n < 0 || (n > 0 && !items)) return BITNET_ERR_INVALID_ARG;
+  static thread_local std::vector<Tl2Linear> run;
+  run.clear();
+  for (int64_t i = 0; i < n; ++i) {
+    const bitnet_elut_item_t& d = items[i];
+    if (!d.packed || !d.q || !d.act_scale || !d.y || d.T < 1 || d.T > 8) return BITNET_ERR_INVALID_ARG;
+    if (!aligned16(d.packed) || (d.x && !aligned16(d.x)) || !aligned16(d.q) || !aligned16(d.y) ||
+        (d.acc_out && !aligned16(d.acc_out)) || (reinterpret_cast<uintptr_t>(d.act_scale) & 3u))
+      return BITNET_ERR_INVALID_ARG;
+    Tl2Linear it;
+    int rc = elut_shape(d.C, d.g, d.M, d.K, &it.g);
+    if (rc) return rc;
+    if (!gemv_elut_scan_item_supported((int)d.T, d.M, d.K, it.g)) return BITNET_ERR_UNSUPPORTED_SHAPE;
+    it.packed = (const uint8_t*)d.packed;
+    it.x = d.x;
+    it.q = d.q;
+    it.act_scale = d.act_scale;
+    it.y = d.y;
+    it.acc_out = d.acc_out;
+    it.w_scale = d.w_scale;
+    it.T = (int)d.T;
+    it.M = d.M;
+    it.K = d.K;
+    it.ldy = 0;
+    run.push_back(it);
+  }
+  // one launch per run of items with the same cardinality (one decode table, one tile size per launch)
+  for (int64_t i = 0; i < n;) {
+    int64_t j = i + 1;
+    while (j < n && items[j].C == items[i].C) ++j;
+    int rc = launch_gemv_elut_scan(run.data() + i, j - i, items[i].C, (cudaStream_t)stream);
+    if (rc) return rc;
+    i = j;
+  }
+  return BITNET_OK;
 }
 
 }  // extern "C"

@@ -139,6 +139,16 @@ struct Tl2Linear {
 };
 bool gemv_tl2_scan_item_supported(int T, int64_t M, int64_t K, const TlGeom& g);
 int launch_gemv_tl2_scan(const Tl2Linear* items, int64_t n, cudaStream_t st);
+// App. A beyond ternary, g = 2: weights of cardinality C = 3, 4, 5 as pair indices in 32-row x 32-pair tiles (512
+// bytes of index nibbles; for C = 5 another 128 bytes of fifth bits).  The geometry comes back in a TlGeom whose
+// tiles3 counts those tiles (tiles2 = 0); the same persistent kernel walks them.
+bool elut2_geom(int C, int64_t M, int64_t K, TlGeom* g);
+bool gemv_elut_scan_item_supported(int T, int64_t M, int64_t K, const TlGeom& g);
+int launch_gemv_elut_scan(const Tl2Linear* items, int64_t n, int C, cudaStream_t st);
+int launch_pack_elut2(int C, const int8_t* w, int64_t M, int64_t K, const TlGeom& g, uint8_t* packed, int* dev_status,
+                      cudaStream_t st);
+int launch_unpack_elut2(int C, const uint8_t* packed, int64_t M, int64_t K, const TlGeom& g, int8_t* w, int* dev_status,
+                        cudaStream_t st);
 // Batches of 9 to 64 tokens: mma.sync over K-slices, partial sums through a [T][M] int32 workspace when K is
 // cut into more than one slice (gemv_i2s_mid_workspace_bytes says how much; 0 = none needed).
 bool gemv_i2s_mid_supported(int T, int64_t M, int64_t K);

@@ -3,6 +3,7 @@
 //   TL1  : Table 4 / Alg. 3 PreprocessWeights -- pair -> 3(w0+1)+(w1+1).
 //   TL2  : Table 5 / Alg. 4 PreprocessWeights -- triple -> (|v|, [v<0]), v = 9w0+3w1+w2, index and
 //          sign kept in separate planes (signed-unsigned weight splitting, Sec. 3.1.2).
+//   ELUT : App. A -- weights of cardinality C in pairs, a pair stored as its index C (w0 + C/2) + (w1 + C/2).
 // The byte layouts are documented in bitnet_b200.h.
 #include "common.cuh"
 
@@ -164,6 +165,69 @@ __global__ void unpack_tl_kernel(const uint8_t* __restrict__ packed, int64_t M, 
   if (bad && dev_status) atomicExch(dev_status, BITNET_ERR_BAD_WEIGHT);
 }
 
+// App. A, g = 2: one thread per (row, tile of 32 pairs).  The low four bits of a pair's index go where a TL1 tile
+// keeps its codes; C = 5 adds the plane of fifth bits where a TL2 tile keeps its signs.
+__global__ void pack_elut2_kernel(const int8_t* __restrict__ w, int64_t M, int64_t K, int C, int64_t tiles, int tile_bytes,
+                                  uint8_t* __restrict__ packed, int* dev_status) {
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= M * tiles) return;
+  const int64_t r = gid % 32, tile = (gid / 32) % tiles, rb = gid / (32 * tiles);
+  const int8_t* wr = w + (rb * 32 + r) * K;
+  const int z = C / 2;
+  uint32_t idx_words[4] = {0, 0, 0, 0}, high = 0;
+  bool bad = false;
+  for (int grp = 0; grp < 32; ++grp) {
+    const int64_t k = tile * 64 + 2 * grp;
+    int d0 = z, d1 = z;                          // columns past K: zero weights
+    if (k < K) {
+      d0 = wr[k] + z;
+      d1 = wr[k + 1] + z;
+      if (d0 < 0 || d0 >= C || d1 < 0 || d1 >= C) {
+        bad = true;
+        d0 = d1 = z;
+      }
+    }
+    const uint32_t idx = (uint32_t)(C * d0 + d1);
+    idx_words[grp >> 3] |= (idx & 15u) << (4 * (grp & 7));
+    high |= (idx >> 4) << tl_sign_bit(grp);
+  }
+  uint8_t* tp = packed + (rb * tiles + tile) * tile_bytes;
+#pragma unroll
+  for (int t = 0; t < 4; ++t) *reinterpret_cast<uint32_t*>(tp + tl_word_off((int)r, t)) = idx_words[t];
+  if (tile_bytes == 640) *reinterpret_cast<uint32_t*>(tp + tl_sign_off((int)r)) = high;
+  if (bad && dev_status) atomicExch(dev_status, BITNET_ERR_BAD_WEIGHT);
+}
+
+__global__ void unpack_elut2_kernel(const uint8_t* __restrict__ packed, int64_t M, int64_t K, int C, int64_t tiles,
+                                    int tile_bytes, int8_t* __restrict__ w, int* dev_status) {
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= M * tiles) return;
+  const int64_t r = gid % 32, tile = (gid / 32) % tiles, rb = gid / (32 * tiles);
+  int8_t* wr = w + (rb * 32 + r) * K;
+  const uint8_t* tp = packed + (rb * tiles + tile) * tile_bytes;
+  const int z = C / 2;
+  uint32_t words[4];
+#pragma unroll
+  for (int t = 0; t < 4; ++t) words[t] = *reinterpret_cast<const uint32_t*>(tp + tl_word_off((int)r, t));
+  const uint32_t high = tile_bytes == 640 ? *reinterpret_cast<const uint32_t*>(tp + tl_sign_off((int)r)) : 0u;
+  bool bad = false;
+  for (int grp = 0; grp < 32; ++grp) {
+    const int idx = (int)((words[grp >> 3] >> (4 * (grp & 7))) & 15u) | (int)(((high >> tl_sign_bit(grp)) & 1u) << 4);
+    const int64_t k = tile * 64 + 2 * grp;
+    if (idx >= C * C) {
+      bad = true;
+      continue;
+    }
+    if (k < K) {
+      wr[k] = (int8_t)(idx / C - z);
+      wr[k + 1] = (int8_t)(idx % C - z);
+    } else {
+      bad |= idx != C * z + z;
+    }
+  }
+  if (bad && dev_status) atomicExch(dev_status, BITNET_ERR_BAD_WEIGHT);
+}
+
 inline unsigned blocks_for(int64_t n, int threads) { return (unsigned)ceil_div(n, threads); }
 
 }  // namespace
@@ -267,6 +331,20 @@ int launch_tl_to_i2s(const uint8_t* tl, int64_t M, int64_t K, const TlGeom& g, u
   cfg.numAttrs = early_start_enabled() ? 1 : 0;
   cudaError_t e = cudaLaunchKernelEx(&cfg, tl_to_i2s_kernel, tl, M, K, g, reinterpret_cast<uint32_t*>(i2s));
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
+}
+
+int launch_pack_elut2(int C, const int8_t* w, int64_t M, int64_t K, const TlGeom& g, uint8_t* packed, int* dev_status,
+                      cudaStream_t st) {
+  pack_elut2_kernel<<<blocks_for(M * g.tiles3, 256), 256, 0, st>>>(w, M, K, C, g.tiles3, (int)(g.block_bytes / g.tiles3),
+                                                                 packed, dev_status);
+  return check_launch();
+}
+
+int launch_unpack_elut2(int C, const uint8_t* packed, int64_t M, int64_t K, const TlGeom& g, int8_t* w, int* dev_status,
+                        cudaStream_t st) {
+  unpack_elut2_kernel<<<blocks_for(M * g.tiles3, 256), 256, 0, st>>>(packed, M, K, C, g.tiles3,
+                                                                   (int)(g.block_bytes / g.tiles3), w, dev_status);
+  return check_launch();
 }
 
 int launch_pack_tl(int, const int8_t* w, int64_t M, int64_t K, const TlGeom& g, uint8_t* packed,

@@ -14,6 +14,8 @@ be produced directly in device memory and any row of it re-drawn on the host.
 
 * ternary weights: ``r = u >> 32``; ``w = 0`` if ``r < floor(p0 * 2**32)``,
   ``+1`` if ``r < floor((p0 + p_plus) * 2**32)``, else ``-1``.
+* weights of cardinality C (the formats beyond ternary): ``w = -(C // 2) +
+  ((u >> 32) * C >> 32)``, uniform over the C consecutive integers from -(C // 2).
 * normal activations: Box-Muller in float64 on the two 32-bit halves of ``u``
   (always evaluated on the host so that libm differences cannot split the two
   sides), cast to float32.
@@ -93,6 +95,18 @@ def ternary(seed: int, tensor_id: int, rows: int, cols: int, p0: float, p_plus: 
         r = _lsr(draw_u64(seed, tensor_id, base + s, c, device), 32)
         w = torch.where(r < t0, 0, torch.where(r < t1, 1, -1))
         out[s:s + c] = w.to(torch.int8)
+    return out.view(rows, cols)
+
+
+def uniform_alphabet(seed: int, tensor_id: int, rows: int, cols: int, card: int, device="cpu",
+                     chunk_elems: int = 1 << 27) -> torch.Tensor:
+    """int8 matrix [rows][cols], uniform over the ``card`` consecutive integers from -(card // 2)."""
+    out = torch.empty(rows * cols, dtype=torch.int8, device=device)
+    n = rows * cols
+    for s in range(0, n, chunk_elems):
+        c = min(chunk_elems, n - s)
+        r = _lsr(draw_u64(seed, tensor_id, s, c, device), 32)
+        out[s:s + c] = (_lsr(r * card, 32) - (card // 2)).to(torch.int8)
     return out.view(rows, cols)
 
 
