@@ -215,6 +215,30 @@ static bool mid_takes(int64_t T, int64_t M, int64_t K, const void* workspace, si
 static bool tl2_scan_takes(int fmt, int64_t T, int64_t M, int64_t K, const TlGeom& g) {
   return !bitnet::g_tl2_lookup && fmt == BITNET_FMT_TL2 && T >= 1 && T <= 8 && gemv_tl2_scan_item_supported((int)T, M, K, g);
 }
+// A TL1 blob is the pair-index blob of cardinality 3 (Table 4's code of a pair = 3 (w0+1) + (w1+1)): decode batches
+// go to the scan kernel's pair mode under the same switch.  `pg` receives the geometry that kernel wants.
+static bool tl1_scan_takes(int fmt, int64_t T, int64_t M, int64_t K, TlGeom* pg) {
+  return !bitnet::g_tl2_lookup && fmt == BITNET_FMT_TL1 && T >= 1 && T <= 8 && elut2_geom(3, M, K, pg) &&
+         gemv_elut_scan_item_supported((int)T, M, K, *pg);
+}
+// One decode item for either scan mode.
+static Tl2Linear scan_item(const void* packed, const float* x, int8_t* q, float* act_scale, float* y, int32_t* acc_out,
+                           float w_scale, int64_t T, int64_t M, int64_t K, int64_t ldy, const TlGeom& g) {
+  Tl2Linear it;
+  it.packed = (const uint8_t*)packed;
+  it.x = x;
+  it.q = q;
+  it.act_scale = act_scale;
+  it.y = y;
+  it.acc_out = acc_out;
+  it.w_scale = w_scale;
+  it.T = (int)T;
+  it.M = M;
+  it.K = K;
+  it.ldy = ldy;
+  it.g = g;
+  return it;
+}
 
 // From this many tokens on a TL call is cheaper as: transcode the blob to I2_S in the workspace (about 20 us for a
 // 4096 x 14336 tensor), then the tcgen05 prefill kernel -- than as ceil(T / 8) scans of the blob.
@@ -281,21 +305,15 @@ int bitnet_mpgemm(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
   }
   for (int64_t t0 = 0; t0 < T; t0 += 8) {
     const int nt = (int)((T - t0 < 8) ? (T - t0) : 8);
+    TlGeom pg;
     if (tl2_scan_takes(fmt, nt, M, K, g)) {
-      Tl2Linear it;
-      it.packed = (const uint8_t*)packed;
-      it.x = nullptr;
-      it.q = const_cast<int8_t*>(q + t0 * K);
-      it.act_scale = const_cast<float*>(act_scale + t0);
-      it.y = y + t0 * M;
-      it.acc_out = acc_out ? acc_out + t0 * M : nullptr;
-      it.w_scale = w_scale;
-      it.T = nt;
-      it.M = M;
-      it.K = K;
-      it.ldy = 0;
-      it.g = g;
+      const Tl2Linear it = scan_item(packed, nullptr, const_cast<int8_t*>(q + t0 * K), const_cast<float*>(act_scale + t0),
+                                     y + t0 * M, acc_out ? acc_out + t0 * M : nullptr, w_scale, nt, M, K, 0, g);
       rc = launch_gemv_tl2_scan(&it, 1, st);
+    } else if (tl1_scan_takes(fmt, nt, M, K, &pg)) {
+      const Tl2Linear it = scan_item(packed, nullptr, const_cast<int8_t*>(q + t0 * K), const_cast<float*>(act_scale + t0),
+                                     y + t0 * M, acc_out ? acc_out + t0 * M : nullptr, w_scale, nt, M, K, 0, pg);
+      rc = launch_gemv_elut_scan(&it, 1, 3, st);
     } else {
       rc = launch_gemv_tl(fmt, (const uint8_t*)packed, w_scale, M, K, g, q + t0 * K, act_scale + t0, nt,
                           y + t0 * M, acc_out ? acc_out + t0 * M : nullptr, workspace, workspace_bytes, st);
@@ -334,20 +352,17 @@ int bitnet_linear(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
     int rc = tl_shape(fmt, M, K, bk3, &g);
     if (rc) return rc;
     if (tl2_scan_takes(fmt, T, M, K, g)) {       // one kernel: quantiser fused
-      Tl2Linear it;
-      it.packed = (const uint8_t*)packed;
-      it.x = x;
-      it.q = q;
-      it.act_scale = act_scale;
-      it.y = y;
-      it.acc_out = acc_out;
-      it.w_scale = w_scale;
-      it.T = (int)T;
-      it.M = M;
-      it.K = K;
-      it.ldy = 0;
-      it.g = g;
+      const Tl2Linear it = scan_item(packed, x, q, act_scale, y, acc_out, w_scale, T, M, K, 0, g);
       return launch_gemv_tl2_scan(&it, 1, (cudaStream_t)stream);
+    }
+  }
+  if (fmt == BITNET_FMT_TL1 && T <= 8) {
+    TlGeom g, pg;
+    int rc = tl_shape(fmt, M, K, bk3, &g);
+    if (rc) return rc;
+    if (tl1_scan_takes(fmt, T, M, K, &pg)) {
+      const Tl2Linear it = scan_item(packed, x, q, act_scale, y, acc_out, w_scale, T, M, K, 0, pg);
+      return launch_gemv_elut_scan(&it, 1, 3, (cudaStream_t)stream);
     }
   }
   int rc = bitnet_quant_act(x, T, K, 0, q, act_scale, nullptr, stream);
@@ -398,28 +413,30 @@ int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* strea
     return grouped && d.fmt == BITNET_FMT_TL2 && tl_shape(d.fmt, d.M, d.K, d.bk3, g) == BITNET_OK &&
            tl2_scan_takes(d.fmt, d.T, d.M, d.K, *g);
   };
+  auto takes1 = [&](const bitnet_group_item_t& d, TlGeom* pg) {
+    TlGeom g;
+    return grouped && d.fmt == BITNET_FMT_TL1 && tl_shape(d.fmt, d.M, d.K, d.bk3, &g) == BITNET_OK &&
+           tl1_scan_takes(d.fmt, d.T, d.M, d.K, pg);
+  };
   for (int64_t i = 0; i < n;) {
     TlGeom g2;
     if (takes2(items[i], &g2)) {
       run2.clear();
       for (; i < n && takes2(items[i], &g2); ++i) {
         const bitnet_group_item_t& d = items[i];
-        Tl2Linear it;
-        it.packed = (const uint8_t*)d.packed;
-        it.x = d.x;
-        it.q = d.q;
-        it.act_scale = d.act_scale;
-        it.y = d.y;
-        it.acc_out = d.acc_out;
-        it.w_scale = d.w_scale;
-        it.T = (int)d.T;
-        it.M = d.M;
-        it.K = d.K;
-        it.ldy = 0;
-        it.g = g2;
-        run2.push_back(it);
+        run2.push_back(scan_item(d.packed, d.x, d.q, d.act_scale, d.y, d.acc_out, d.w_scale, d.T, d.M, d.K, 0, g2));
       }
       int rc = launch_gemv_tl2_scan(run2.data(), (int64_t)run2.size(), (cudaStream_t)stream);
+      if (rc) return rc;
+      continue;
+    }
+    if (takes1(items[i], &g2)) {
+      run2.clear();
+      for (; i < n && takes1(items[i], &g2); ++i) {
+        const bitnet_group_item_t& d = items[i];
+        run2.push_back(scan_item(d.packed, d.x, d.q, d.act_scale, d.y, d.acc_out, d.w_scale, d.T, d.M, d.K, 0, g2));
+      }
+      int rc = launch_gemv_elut_scan(run2.data(), (int64_t)run2.size(), 3, (cudaStream_t)stream);
       if (rc) return rc;
       continue;
     }
@@ -512,21 +529,24 @@ int bitnet_linear_segments(bitnet_fmt_t fmt, const void* packed, int64_t M, int6
     if (ok) {
       Tl2Linear it[16];
       r0 = 0;
-      for (int64_t s = 0; s < n_seg; r0 = seg_end[s], ++s) {
-        it[s].packed = (const uint8_t*)packed + (size_t)(r0 / 32) * (size_t)g.block_bytes;
-        it[s].x = x;
-        it[s].q = q;
-        it[s].act_scale = act_scale;
-        it[s].y = y + r0;
-        it[s].acc_out = acc_out ? acc_out + r0 : nullptr;
-        it[s].w_scale = seg_scale[s];
-        it[s].T = (int)T;
-        it[s].M = seg_end[s] - r0;
-        it[s].K = K;
-        it[s].ldy = M;
-        it[s].g = gs[s];
-      }
+      for (int64_t s = 0; s < n_seg; r0 = seg_end[s], ++s)
+        it[s] = scan_item((const uint8_t*)packed + (size_t)(r0 / 32) * (size_t)g.block_bytes, x, q, act_scale, y + r0,
+                          acc_out ? acc_out + r0 : nullptr, seg_scale[s], T, seg_end[s] - r0, K, M, gs[s]);
       return launch_gemv_tl2_scan(it, n_seg, st);
+    }
+  }
+  if (grouped && fmt == BITNET_FMT_TL1 && T <= 8) {
+    bool ok = true;
+    int64_t r0 = 0;
+    TlGeom gs[16];
+    for (int64_t s = 0; s < n_seg && ok; r0 = seg_end[s], ++s) ok = tl1_scan_takes(fmt, T, seg_end[s] - r0, K, &gs[s]);
+    if (ok) {
+      Tl2Linear it[16];
+      r0 = 0;
+      for (int64_t s = 0; s < n_seg; r0 = seg_end[s], ++s)
+        it[s] = scan_item((const uint8_t*)packed + (size_t)(r0 / 32) * (size_t)g.block_bytes, x, q, act_scale, y + r0,
+                          acc_out ? acc_out + r0 : nullptr, seg_scale[s], T, seg_end[s] - r0, K, M, gs[s]);
+      return launch_gemv_elut_scan(it, n_seg, 3, st);
     }
   }
   // any other shape: the whole tensor with scale 1, then every segment's columns times its scale
@@ -581,18 +601,7 @@ int bitnet_elut_linear_group(const bitnet_elut_item_t* items, int64_t n, void* s
     int rc = elut_shape(d.C, d.g, d.M, d.K, &it.g);
     if (rc) return rc;
     if (!gemv_elut_scan_item_supported((int)d.T, d.M, d.K, it.g)) return BITNET_ERR_UNSUPPORTED_SHAPE;
-    it.packed = (const uint8_t*)d.packed;
-    it.x = d.x;
-    it.q = d.q;
-    it.act_scale = d.act_scale;
-    it.y = d.y;
-    it.acc_out = d.acc_out;
-    it.w_scale = d.w_scale;
-    it.T = (int)d.T;
-    it.M = d.M;
-    it.K = d.K;
-    it.ldy = 0;
-    run.push_back(it);
+    run.push_back(scan_item(d.packed, d.x, d.q, d.act_scale, d.y, d.acc_out, d.w_scale, d.T, d.M, d.K, 0, it.g));
   }
   // one launch per run of items with the same cardinality (one decode table, one tile size per launch)
   for (int64_t i = 0; i < n;) {

@@ -77,8 +77,17 @@ def test_host_validation_returns_codes_without_a_gpu(L):
     assert L.bitnet_mpgemm(0, fake, 1.0, 64, 100, 0, fake, fake, 1, fake, null, null, 0, null) == 2
     assert L.bitnet_mpgemm(0, fake, 1.0, 64, 128, 0, fake, fake, 0, fake, null, null, 0, null) == 1
     assert L.bitnet_mpgemm(0, fake, 1.0, 64, 128, 0, odd, fake, 1, fake, null, null, 0, null) == 1
-    # lookup-table kernel (TL1 always runs it) without the workspace it keeps its tables in
-    assert L.bitnet_mpgemm(1, fake, 1.0, 64, 28672, 0, fake, fake, 1, fake, null, null, 0, null) == 3
+    # lookup-table kernel (rows the scan kernel does not take: K not a multiple of 4) without the workspace it keeps
+    # its tables in
+    assert L.bitnet_mpgemm(1, fake, 1.0, 64, 28674, 0, fake, fake, 1, fake, null, null, 0, null) == 3
+    # element-wise tables beyond ternary: only pairs of cardinality 3, 4, 5 are built
+    assert L.bitnet_elut_packed_bytes(5, 2, 64, 128) == 64 * 128 * 5 // 16
+    assert L.bitnet_elut_packed_bytes(5, 3, 64, 126) == 0 and L.bitnet_elut_packed_bytes(6, 2, 64, 128) == 0
+    assert L.bitnet_pack_elut(5, 3, fake, 32, 96, fake, 1 << 20, null, null) == 2
+    assert L.bitnet_pack_elut(5, 2, fake, 48, 96, fake, 1 << 20, null, null) == 2   # M % 32
+    assert L.bitnet_pack_elut(5, 2, null, 32, 96, fake, 1 << 20, null, null) == 1
+    assert L.bitnet_pack_elut(5, 2, fake, 32, 128, fake, 16, null, null) == 1       # blob too small
+    assert L.bitnet_elut_linear_group(null, 1, null) == 1 and L.bitnet_elut_linear_group(null, 0, null) == 0
     # bitnet_linear validates the shape before it plans a launch (K = 0 or negative must not reach a division)
     for T in (1, 6, 8):
         assert L.bitnet_linear(0, fake, 1.0, 64, 0, 0, fake, T, fake, fake, fake, null, fake, 1 << 20, null) == 1

@@ -171,6 +171,21 @@ def test_group_tl2_items_through_the_scan_kernel():
         it.check()
 
 
+def test_group_tl1_items_through_the_scan_kernel():
+    """TL1 items: a TL1 blob is the pair-index blob of cardinality 3, so decode batches run in the scan kernel's pair
+    mode (the index byte of two pairs selects a table entry holding their four weights).  Ragged last tiles, every
+    token count, items sharing an input, a TL2 and an I2_S item in between, a row too short for the kernel."""
+    x = synth.normal(9, 2, 2, 4096)
+    items = [Item("tl1", 64, 64 * 12, 1, 720), Item("tl1", 320, 3200, 3, 721), Item("tl1", 96, 8640, 4, 722),
+             Item("tl1", 4096, 4096, 2, 723, x=x), Item("tl1", 2048, 4096, 2, 724, x=x), Item("tl2", 64, 2048, 1, 725),
+             Item("tl1", 32, 8192, 8, 726), Item("tl1", 160, 28672, 1, 727), Item("i2s", 64, 2048, 1, 728),
+             Item("tl1", 64, 64 * 20 + 36, 5, 729), Item("tl1", 64, 128, 2, 730), Item("tl1", 32, 28672, 8, 731)]
+    items[4].xd = items[3].xd
+    run_group(items)
+    for it in items:
+        it.check()
+
+
 def test_group_tl2_workload_layer():
     """A 100B-shaped decoder layer in the TL2 encoding at one token through the grouped call (one persistent scan
     kernel): sampled rows of every linear against the oracle, and the whole vectors against the I2_S result."""

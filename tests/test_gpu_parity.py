@@ -597,6 +597,14 @@ def test_tl_workspace_shared_by_calls_of_different_shapes(fmt):
     """One workspace serves TL calls of different shapes back to back: the tables of a call with few rows lie
     where a later call with many rows keeps its split-K sums, so every call must clear what it relies on."""
     shapes = [(32, 28672, 2), (4096, 8192, 1), (64, 14336, 3), (2048, 28672, 1), (32, 96 * 40, 1)]
+    bn.bitnet_set_tl2_lookup(True)     # the kernel that keeps tables and sums in the workspace, for both formats
+    try:
+        _shared_workspace_calls(fmt, shapes)
+    finally:
+        bn.bitnet_set_tl2_lookup(False)
+
+
+def _shared_workspace_calls(fmt, shapes):
     n = max(bn.bitnet_mpgemm_workspace_bytes(fmt, T, M, K) for M, K, T in shapes)
     ws = torch.full((n,), 0x5A, dtype=torch.uint8, device="cuda")      # never initialised: garbage on purpose
     cases = []
@@ -649,7 +657,7 @@ def test_read_once_switches_in_child_processes(extra):
     """Every kernel choice that an environment variable makes (read once per process) against the oracle: the dp4a
     prefill kernel, plain stores instead of bulk tensor stores in the tensor-core prefill kernel, the bulk-copy ring
     decode kernel, the quantiser without clusters, no fused quantiser, the mid-batch kernel's lower limit and forced
-    slice count, the lookup-table kernel for TL2, other ring depths and warps per unit in the grouped kernels, and
+    slice count, the lookup-table kernel for TL1 and TL2, other ring depths and warps per unit in the grouped kernels, and
     the grouped call switched off."""
     code = (
         "import sys; sys.path.insert(0, 'tests'); import numpy as np, torch\n"
@@ -662,7 +670,8 @@ def test_read_once_switches_in_child_processes(extra):
         "                  (300, 2048, 300)]:\n"
         "    check_linear('i2s', synth.ternary(62, 1, M, K, 1/3, 1/3), synth.normal(62, T, T, K))\n"
         "for (M, K, T) in [(64, 3200, 1), (96, 8192, 3), (32, 28672, 8), (64, 130, 2)]:\n"
-        "    check_linear('tl2', synth.ternary(63, 1, M, K, 1/3, 1/3), synth.normal(63, T, T, K))\n"
+        "    for fmt in ('tl2', 'tl1'):\n"
+        "        check_linear(fmt, synth.ternary(63, 1, M, K, 1/3, 1/3), synth.normal(63, T, T, K))\n"
         "for (M, K, T) in [(96, 8192, 1), (64, 28672, 4), (32, 16384, 7)]:\n"
         "    w = synth.ternary(64, 1, M, K, 1/3, 1/3); x = synth.normal(64, T, T, K)\n"
         "    for fmt in ('i2s', 'tl2'):\n"
@@ -670,7 +679,7 @@ def test_read_once_switches_in_child_processes(extra):
         "        q_ref, sc_ref, _ = oracle.quant_act(x.numpy())\n"
         "        assert np.array_equal(npy(q), q_ref) and np.array_equal(npy(acc), oracle.mpgemm_def(q_ref, w.numpy()))\n"
         "items = [Item('i2s', 160, 8192, 1, 900), Item('tl2', 64, 8192, 1, 901), Item('i2s', 48, 28672, 8, 902), Item('i2s', 2000, 2048, 3, 903),\n"
-        "         Item('tl2', 640, 3200, 2, 904)]\n"
+        "         Item('tl2', 640, 3200, 2, 904), Item('tl1', 96, 8192, 1, 905), Item('tl1', 320, 4096, 4, 906)]\n"
         "run_group(items)\n"
         "for it in items: it.check()\n"
         "assert bn.bitnet_device_status() == 0\n"
