@@ -485,6 +485,46 @@ def bench_prefill(bn, torch, synth, steps, warmup):
     return out
 
 
+def bench_elut(bn, torch, synth, wl, layers, card, steps, warmup, check):
+    """The sweep's shapes with weights of cardinality `card` (App. A, Table 3) stored as pair indices: one
+    bitnet_elut_linear_group call per step (quantiser + scan kernel in pair mode + rescale).  With `check`, sampled rows
+    of every linear of layer 0 are compared with the oracle."""
+    import numpy as np
+    dev = torch.device("cuda")
+    items, kept, nbytes = [], [], 0
+    for layer in range(layers):
+        for j, lin in enumerate(wl.linears):
+            w = synth.uniform_alphabet(wl.seed, 1000 + layer * 8 + j, lin.M, lin.K, card, device=dev)
+            x = wl.activations(layer, j, 1)
+            if layer == 0:
+                rows = np.unique(np.concatenate([[0, lin.M - 1], np.random.default_rng(j).integers(0, lin.M, 30)]))
+                kept.append((rows, w[torch.as_tensor(rows, device=dev)].cpu().numpy(), x.numpy()))
+            blob = bn.bitnet_pack_elut(card, 2, w, check=False)
+            del w
+            items.append(dict(C=card, g=2, packed=blob, w_scale=0.5, M=lin.M, K=lin.K, x=x.to(dev),
+                              q=torch.empty((1, lin.K), dtype=torch.int8, device=dev),
+                              act_scale=torch.empty(1, dtype=torch.float32, device=dev),
+                              y=torch.empty((1, lin.M), dtype=torch.float32, device=dev)))
+            nbytes += blob.numel()
+    grp = bn.make_elut_group(items)
+    ms = time_replays(torch, lambda: bn.bitnet_elut_linear_group(grp), steps, warmup)
+    out = {"cardinality": card, "group": 2, "bits_per_weight": 8.0 * nbytes / sum(l.M * l.K for l in wl.linears) / layers,
+           "packed_bytes": nbytes, "ms_per_step": ms, "value": nbytes / ms / 1e6, "unit": UNIT,
+           "frac_of_hbm_peak": nbytes / ms / 1e6 / peaks()["hbm"],
+           "kernel": "gemv_tl2_scan_kernel in pair mode (one bitnet_elut_linear_group call per step)"}
+    if check:
+        import oracle
+        ok = True
+        for (rows, w_rows, x), d in zip(kept, items):
+            q, sc, _ = oracle.quant_act(x)
+            acc = oracle.mpgemm_def(q, np.ascontiguousarray(w_rows))
+            y_ref = oracle.dequant(acc, sc, 0.5)[0]
+            y = d["y"].cpu().numpy()[0, rows].astype(np.float64)
+            ok &= bool(np.all(np.abs(y - y_ref) <= 1e-6 * np.abs(y_ref)) and np.all(y[acc[0] == 0] == 0.0))
+        out["verified"] = ok
+    return out
+
+
 def verify_against_oracle(oracle, sw, wl, torch, ys_layer0, rows_per_linear=8):
     """Part of the CPU-baseline leg: the y the GPU produced in the timed steps against the oracle -- every row of
     layer 0 (whose oracle results `ys_layer0` come from the timed CPU run) and `rows_per_linear` sampled rows of
@@ -544,7 +584,7 @@ def run_ours(args):
     pk = peaks()
     wl = synth.CONFIGS["sweep100b"]
     layers = args.layers or wl.layers
-    fmts = ["i2s", "tl2"] if not args.skip_tl2 else ["i2s"]
+    fmts = ["i2s", "tl2", "tl1"] if not args.skip_tl2 else ["i2s"]
     sw = Sweep(bn, torch, wl, fmts, layers, torch.device("cuda", local))
     n_lin = sw.n_linears()
 
@@ -613,6 +653,11 @@ def run_ours(args):
                            "lookup_table_kernel": {"ms_per_step": ms_lut, "value": sw.bytes["tl2"] / ms_lut / 1e6,
                                                    "frac_of_hbm_peak": sw.bytes["tl2"] / ms_lut / 1e6 / pk["hbm"],
                                                    "kernel": "quantiser + tl_table_kernel + gemv_tl_kernel per linear"}}
+            # TL1 (2 bits per weight, Table 4): the scan kernel's pair mode
+            ms_tl1 = time_replays(torch, lambda: sw.step_group("tl1"), max(5, args.steps // 2), args.warmup)
+            line["tl1"] = {"packed_bytes": sw.bytes["tl1"], "ms_per_step": ms_tl1, "value": sw.bytes["tl1"] / ms_tl1 / 1e6,
+                           "unit": UNIT, "frac_of_hbm_peak": sw.bytes["tl1"] / ms_tl1 / 1e6 / pk["hbm"],
+                           "kernel": "gemv_tl2_scan_kernel in pair mode (one bitnet_linear_group call per step)"}
             sw.step_group("tl2")        # the verification below sees the scan kernel's y
         if not args.skip_batched:
             line["batched_decode"] = {
@@ -645,6 +690,11 @@ def run_ours(args):
                 line["verify_failures"] = failures
         del sw
         torch.cuda.empty_cache()
+        if not args.skip_elut:
+            # beyond ternary (App. A): the same shapes with weights of cardinality 5 (2.5 bits per weight) and 4 (2 bits)
+            line["elut"] = [bench_elut(bn, torch, synth, wl, layers, card, max(5, args.steps // 2), args.warmup,
+                                       world == 1 and not args.skip_cpu) for card in (5, 4)]
+            torch.cuda.empty_cache()
         if not args.skip_small:
             line["small_configs"] = bench_small_configs(bn, torch, synth, max(5, args.steps // 2), 3)
         if not args.skip_ceilings:
@@ -674,6 +724,7 @@ def main():
     ap.add_argument("--skip-prefill", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-batched", action="store_true")
+    ap.add_argument("--skip-elut", action="store_true", help="skip the sweeps with weights of cardinality 5 and 4")
     ap.add_argument("--skip-small", action="store_true", help="skip the timings of the three small workloads")
     ap.add_argument("--skip-ceilings", action="store_true", help="skip the read-stream / issue-rate / int8 GEMM ceilings")
     ap.add_argument("--no-early-start", action="store_true",
