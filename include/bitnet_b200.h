@@ -71,14 +71,15 @@ int bitnet_device_status_clear(void);
 void bitnet_set_early_start(int enable);
 
 /*
- * Which kernel serves TL2 batches of up to 8 tokens (process-wide; also set by BITNET_TL2=lut in the environment).
- *   0 (default): the scan kernel -- every packed index byte plus its sign bits is resolved by one shared-memory
- *      table lookup into the weights it stands for (Table 5), which go through the int8 tensor cores; about
- *      3.5 times the rate of the other form on a B200.  Shapes it does not take (K not a multiple of 4, fewer
- *      than three 96-column tiles per warp, more codes than fit beside its 128 KB table) fall back to the other form.
+ * Which kernel serves TL1 and TL2 batches of up to 8 tokens (process-wide; also set by BITNET_TL2=lut in the
+ * environment).
+ *   0 (default): the scan kernel -- every packed index byte (TL2: plus its sign bits) is resolved by one
+ *      shared-memory table lookup into the weights it stands for (Tables 4, 5), which go through the int8 tensor
+ *      cores; 4 to 5 times the rate of the other form on a B200.  Shapes it does not take (K not a multiple of 4,
+ *      fewer than three tiles per warp, more codes than fit beside its 128 KB table) fall back to the other form.
  *   1: the element-wise lookup-table kernel of Alg. 2 / Alg. 4 as the paper states it -- per-token tables of
  *      activation partial sums, one lookup, conditional negate and add per packed index.
- * Both give the same integers.  TL1 always runs the lookup-table kernel.
+ * Both give the same integers.
  */
 void bitnet_set_tl2_lookup(int enable);
 
@@ -150,7 +151,7 @@ int bitnet_pack_tl(bitnet_fmt_t fmt, const int8_t* w, int64_t M, int64_t K, int 
  * tiles over K-slices followed by a rescale kernel (when the workspace is missing or too small, the
  * prefill kernel takes the call instead); larger T the tcgen05 prefill kernel (whole tiles per CTA; parts
  * of a tile's K per CTA when there are few tiles and the workspace is there).  TL runs a decode kernel over
- * groups of 8 tokens (TL2: the scan kernel, see bitnet_set_tl2_lookup); from 128 tokens on, with K a multiple of
+ * groups of 8 tokens (the scan kernel, see bitnet_set_tl2_lookup); from 128 tokens on, with K a multiple of
  * 64 and the workspace bitnet_mpgemm_workspace_bytes asks for, the TL blob is first turned into its I2_S form
  * inside the workspace (a device-side transcode of the packed codes) and the tcgen05 prefill kernel serves the
  * call, so that a model kept only in the 1.67-bit TL2 encoding has a tensor-core prefill too.  The integer
