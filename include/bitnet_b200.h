@@ -64,9 +64,12 @@ int bitnet_device_status_clear(void);
  * programmatic dependent launch: their prologue may run while the previous kernel queued on the same
  * stream is finishing, and the decode kernel starts copying the PACKED WEIGHTS into shared memory
  * before that kernel has finished (activations, scales and outputs are touched only after it has).
- * Packed weights are treated as read-only model state: if a blob was written by work queued earlier on
- * the same stream, synchronise (or record/wait an event) before the first bitnet_mpgemm that reads it,
- * or switch early start off.  enable = 0 restores plain stream order for every later call.
+ * Packed weights are treated as read-only model state.  A blob written by this library's own packers is
+ * safe to use at once: the first kernel the library launches on a stream after a packer was queued on it
+ * starts in plain stream order (the library remembers such streams; a few words of host state).  If a
+ * blob was written by other work queued earlier on the same stream (a copy, a kernel of the caller),
+ * synchronise (or record/wait an event) before the first call that reads it, or switch early start off.
+ * enable = 0 restores plain stream order for every later call.
  */
 void bitnet_set_early_start(int enable);
 

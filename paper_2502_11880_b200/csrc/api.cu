@@ -4,6 +4,7 @@
 #include <cstring>
 #include <cstdarg>
 #include <cstdio>
+#include <atomic>
 #include <mutex>
 
 #include <vector>
@@ -21,7 +22,29 @@ int note_cuda_error(cudaError_t e) {
 
 static int g_early_start = 1;
 static int g_tl2_lookup = [] { const char* e = getenv("BITNET_TL2"); return (e && strcmp(e, "lut") == 0) ? 1 : 0; }();
-bool early_start_enabled() { return g_early_start != 0; }
+// Streams on which a packer (or the TL -> I2_S transcode) has been queued and no kernel of this library since.
+static std::mutex g_written_mu;
+static std::vector<cudaStream_t> g_written;
+static std::atomic<int> g_written_n{0};
+void note_blob_written(cudaStream_t st) {
+  std::lock_guard<std::mutex> lock(g_written_mu);
+  for (cudaStream_t s : g_written)
+    if (s == st) return;
+  g_written.push_back(st);
+  g_written_n.store((int)g_written.size(), std::memory_order_release);
+}
+bool early_start_enabled(cudaStream_t st) {
+  if (!g_early_start) return false;
+  if (g_written_n.load(std::memory_order_acquire) == 0) return true;
+  std::lock_guard<std::mutex> lock(g_written_mu);
+  for (size_t i = 0; i < g_written.size(); ++i)
+    if (g_written[i] == st) {
+      g_written.erase(g_written.begin() + (long)i);
+      g_written_n.store((int)g_written.size(), std::memory_order_release);
+      return false;
+    }
+  return true;
+}
 
 bool log_enabled() {
   static const bool on = [] { const char* e = getenv("BITNET_LOG"); return e && atoi(e) != 0; }();

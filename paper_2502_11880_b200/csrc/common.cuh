@@ -157,8 +157,12 @@ int launch_gemv_i2s_mid(const uint8_t* packed, float w_scale, int64_t M, int64_t
                         const float* act_scale, int T, float* y, int32_t* acc_out, void* ws, size_t ws_bytes,
                         cudaStream_t st);
 // Programmatic dependent launch (kernels may start their prologue, and prefetch weights, before the
-// previous kernel in the stream has finished); process-wide switch, on by default.
-bool early_start_enabled();
+// previous kernel in the stream has finished); process-wide switch, on by default.  early_start_enabled(st) is asked
+// once per launch on `st`: it answers no for the first launch after a kernel of this library wrote a packed blob
+// on that stream (note_blob_written), so that this launch begins only when the blob is complete and everything
+// queued behind it is ordered after it.
+bool early_start_enabled(cudaStream_t st);
+void note_blob_written(cudaStream_t st);
 size_t gemv_tl_workspace_bytes(int fmt, int64_t T, int64_t M, int64_t K);
 int launch_gemv_tl(int fmt, const uint8_t* packed, float w_scale, int64_t M, int64_t K, const TlGeom& g,
                    const int8_t* q, const float* act_scale, int T, float* y, int32_t* acc_out, void* ws,

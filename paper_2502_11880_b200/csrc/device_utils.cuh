@@ -55,6 +55,11 @@ __device__ __forceinline__ int quant4_packed(const float4& v, float s) {
   asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(a1), "r"(a0), "r"(hi));
   return w;
 }
+// The same word from four separate clamps (kept where the compiler schedules it better than the pack).
+__device__ __forceinline__ int quant4(const float4& v, float s) {
+  return (quant1(v.x, s) & 255) | ((quant1(v.y, s) & 255) << 8) | ((quant1(v.z, s) & 255) << 16) |
+         ((quant1(v.w, s) & 255) << 24);
+}
 __device__ __forceinline__ float absmax4(const float4& v) {
   return fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
 }

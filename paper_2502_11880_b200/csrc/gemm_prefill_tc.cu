@@ -30,6 +30,7 @@
 #include <cstring>
 
 #include "common.cuh"
+#include "device_utils.cuh"
 
 namespace bitnet {
 namespace {
@@ -91,7 +92,6 @@ struct __align__(8) Barriers {
   int abort_flag;
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
@@ -569,7 +569,7 @@ int launch_gemm_i2s_prefill(const uint8_t* packed, float w_scale, int64_t M, int
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = early_start_enabled() ? 1 : 0;
+  cfg.numAttrs = early_start_enabled(st) ? 1 : 0;
   cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_i2s_tc_kernel, qmap, ymap, a);
   int rc = le == cudaSuccess ? BITNET_OK : note_cuda_error(le);
   if (rc || ksplit == 1) return rc;

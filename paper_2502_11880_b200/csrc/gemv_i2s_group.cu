@@ -515,7 +515,7 @@ int launch_group(const GArgs<NMAX>& a, int grid, size_t smem, cudaStream_t st) {
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = early_start_enabled() ? 1 : 0;
+  cfg.numAttrs = early_start_enabled(st) ? 1 : 0;
   cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_i2s_group_kernel<DEPTH, NMAX>, a);
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
 }

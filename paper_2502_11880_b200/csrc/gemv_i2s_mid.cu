@@ -22,6 +22,7 @@
 #include <stdlib.h>
 
 #include "common.cuh"
+#include "device_utils.cuh"
 
 namespace bitnet {
 namespace {
@@ -51,26 +52,6 @@ struct MArgs {
   int qst;               // bytes between staged token rows
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void cp16_stream(uint32_t dst, const void* src, uint64_t pol) {
-  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(pol)
-               : "memory");
-}
-__device__ __forceinline__ void cp16_keep(uint32_t dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-// D(16x8, s32) += A(16x32, u8, row) * B(32x8, s8, col); fragment layout as in the decode kernel.
-__device__ __forceinline__ void mma_u8s8(int (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, int b0,
-                                         int b1) {
-  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
-               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
 
 // NT token tiles of 8; RU 16-row units per item; DEPTH ring slots (of RU KB) per warp;
 // NSL accumulator sets per token tile: 4 = one per 2-bit slot (fields used in place, weights 1, 4, 16, 64),
@@ -114,8 +95,8 @@ __global__ void __launch_bounds__(MTHREADS, 1) gemv_i2s_mid_kernel(const MArgs a
       const int u = p * RU + r;
       if (u < a.nunits) {
         const uint8_t* src = base + (int64_t)u * a.unit_bytes + (int64_t)c * 1024;
-        cp16_stream(slot_addr + r * 1024, src, pol);
-        cp16_stream(slot_addr + r * 1024 + 512, src + 512, pol);
+        cp16(slot_addr + r * 1024, src, pol);
+        cp16(slot_addr + r * 1024 + 512, src + 512, pol);
       }
     }
   };
@@ -429,7 +410,7 @@ int launch_mid(const MArgs& a, const MidPlan& p, cudaStream_t st) {
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = early_start_enabled() ? 1 : 0;
+  cfg.numAttrs = early_start_enabled(st) ? 1 : 0;
   cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_i2s_mid_kernel<NT, RU, DEPTH, NSL>, a);
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
 }
@@ -449,7 +430,7 @@ int launch_rescale_sums(int32_t* sums, const float* act_scale, float w_scale, in
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = early_start_enabled() ? 1 : 0;
+  cfg.numAttrs = early_start_enabled(st) ? 1 : 0;
   cudaError_t e = cudaLaunchKernelEx(&cfg, finish_mid_kernel, sums, act_scale, w_scale, (int)T, (int)M, y, acc_out);
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
 }

@@ -35,6 +35,7 @@
 #include <cstring>
 
 #include "common.cuh"
+#include "device_utils.cuh"
 
 namespace bitnet {
 namespace {
@@ -66,46 +67,6 @@ struct WArgs {
   int nunits;            // ceil(M / 16)
   int pre;               // ring slots requested before waiting for the previous kernel
 };
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void cp16(uint32_t dst, const void* src, uint64_t pol) {
-  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(pol)
-               : "memory");
-}
-__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void group_barrier(int id, int nthreads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
-}
-// D(16x8, s32) += A(16x32, u8, row) * B(32x8, s8, col).  Lane (g = lane/4, t = lane%4):
-// a0 = row g, k 4t..4t+3; a1 = row g+8, same k; a2, a3 = the same rows, k 16+4t..; b0 = k 4t..4t+3 of
-// column g, b1 = k 16+4t..; c0,c1 = row g, columns 2t, 2t+1; c2,c3 = row g+8.
-__device__ __forceinline__ void mma_u8s8(int (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, int b0,
-                                         int b1) {
-  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
-               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ int quant1(float x, float s) {
-  return max(-128, min(127, __float2int_rn(__fmul_rn(x, s))));
-}
-// Four codes in one word: round to nearest even, then the saturating pack does the clamp to [-128, 127]
-// (which never fires for |x| <= amax; same result as quant1 on every input).
-__device__ __forceinline__ int quant4_packed(const float4& v, float s) {
-  const int a0 = __float2int_rn(__fmul_rn(v.x, s)), a1 = __float2int_rn(__fmul_rn(v.y, s));
-  const int a2 = __float2int_rn(__fmul_rn(v.z, s)), a3 = __float2int_rn(__fmul_rn(v.w, s));
-  int hi, w;
-  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(a3), "r"(a2), "r"(0));
-  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(a1), "r"(a0), "r"(hi));
-  return w;
-}
-__device__ __forceinline__ int quant4(const float4& v, float s) {
-  return (quant1(v.x, s) & 255) | ((quant1(v.y, s) & 255) << 8) | ((quant1(v.z, s) & 255) << 16) |
-         ((quant1(v.w, s) & 255) << 24);
-}
 
 // shared memory: [unit counter, unit queues, quantiser scratch: 2 KB][partials][codes][rings]
 __host__ __device__ inline size_t red_bytes(int T) { return (size_t)CW * 2 * T * 16 * 4; }
@@ -496,7 +457,7 @@ int launch_wring(const WArgs& a, const Plan& p, cudaStream_t st) {
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = early_start_enabled() ? 1 : 0;
+  cfg.numAttrs = early_start_enabled(st) ? 1 : 0;
   cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_i2s_wring_kernel<DEPTH, XREG>, a);
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
 }

@@ -21,6 +21,7 @@
 // memory, and K-slices of different CTAs meet in an int32 workspace by atomicAdd, finalised by
 // whichever slice arrives last (no waiting).
 #include "common.cuh"
+#include "device_utils.cuh"
 
 namespace bitnet {
 namespace {
@@ -113,7 +114,6 @@ __global__ void tl_table_kernel(const int8_t* __restrict__ q, int T, int64_t K, 
   table[(int64_t)blockIdx.y * nslots + e] = v;
 }
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ int sign_mask(unsigned sg, int bit) {   // 0 or -1 from one bit
   int m;
@@ -344,7 +344,7 @@ int launch_gemv_tl(int fmt, const uint8_t* packed, float w_scale, int64_t M, int
   tcfg.blockDim = dim3(256);
   tcfg.stream = st;
   tcfg.attrs = pdl;
-  tcfg.numAttrs = early_start_enabled() ? 1 : 0;
+  tcfg.numAttrs = early_start_enabled(st) ? 1 : 0;
   cudaError_t le = cudaLaunchKernelEx(&tcfg, tl_table_kernel, q, T, K, g, table, nslots, reinterpret_cast<int*>(ws),
                                       (int64_t)T * M + M);
   int rc = le == cudaSuccess ? BITNET_OK : note_cuda_error(le);
@@ -388,7 +388,7 @@ int launch_gemv_tl(int fmt, const uint8_t* packed, float w_scale, int64_t M, int
     gcfg.dynamicSmemBytes = smem;
     gcfg.stream = st;
     gcfg.attrs = pdl;
-    gcfg.numAttrs = early_start_enabled() ? 1 : 0;
+    gcfg.numAttrs = early_start_enabled(st) ? 1 : 0;
     le = cudaLaunchKernelEx(&gcfg, gemv_tl_kernel, a);
     rc = le == cudaSuccess ? BITNET_OK : note_cuda_error(le);
     if (rc != BITNET_OK) return rc;

@@ -237,6 +237,7 @@ int launch_pack_i2s(const int8_t* w, int64_t M, int64_t K, uint8_t* packed, int*
   const int64_t kp = i2s_kp(K), nwords = i2s_mp(M) * kp / 16;
   pack_i2s_kernel<<<blocks_for(nwords, 256), 256, 0, st>>>(w, M, K, kp, nwords, reinterpret_cast<uint32_t*>(packed),
                                                          dev_status);
+  note_blob_written(st);
   return check_launch();
 }
 
@@ -328,8 +329,9 @@ int launch_tl_to_i2s(const uint8_t* tl, int64_t M, int64_t K, const TlGeom& g, u
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = early_start_enabled() ? 1 : 0;
+  cfg.numAttrs = early_start_enabled(st) ? 1 : 0;
   cudaError_t e = cudaLaunchKernelEx(&cfg, tl_to_i2s_kernel, tl, M, K, g, reinterpret_cast<uint32_t*>(i2s));
+  note_blob_written(st);     // the prefill kernel that follows reads this blob before it waits for earlier kernels
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
 }
 
@@ -337,6 +339,7 @@ int launch_pack_elut2(int C, const int8_t* w, int64_t M, int64_t K, const TlGeom
                       cudaStream_t st) {
   pack_elut2_kernel<<<blocks_for(M * g.tiles3, 256), 256, 0, st>>>(w, M, K, C, g.tiles3, (int)(g.block_bytes / g.tiles3),
                                                                  packed, dev_status);
+  note_blob_written(st);
   return check_launch();
 }
 
@@ -350,6 +353,7 @@ int launch_unpack_elut2(int C, const uint8_t* packed, int64_t M, int64_t K, cons
 int launch_pack_tl(int, const int8_t* w, int64_t M, int64_t K, const TlGeom& g, uint8_t* packed,
                    int* dev_status, cudaStream_t st) {
   pack_tl_kernel<<<blocks_for(M * (g.tiles3 + g.tiles2), 256), 256, 0, st>>>(w, M, K, g, packed, dev_status);
+  note_blob_written(st);
   return check_launch();
 }
 

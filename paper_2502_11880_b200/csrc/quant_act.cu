@@ -8,6 +8,7 @@
 #include <stdlib.h>
 
 #include "common.cuh"
+#include "device_utils.cuh"
 
 namespace bitnet {
 namespace {
@@ -25,10 +26,6 @@ __device__ __forceinline__ int warp_sum(int v) {
   return v;
 }
 
-__device__ __forceinline__ int quant1(float x, float s) {
-  int v = __float2int_rn(__fmul_rn(x, s));
-  return max(-128, min(127, v));
-}
 
 // amax over a [rows][K] slab starting at x; result in every thread.
 __device__ float block_amax(const float* __restrict__ x, int64_t n, float* red) {
@@ -284,7 +281,7 @@ cudaError_t launch_cluster(const float* x, int64_t T, int64_t K, int8_t* q, floa
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = early_start_enabled() ? 2 : 1;
+  cfg.numAttrs = early_start_enabled(st) ? 2 : 1;
   return cudaLaunchKernelEx(&cfg, quant_act_cluster_kernel<NT, C>, x, K, q, act_scale, act_sum);
 }
 
@@ -298,7 +295,7 @@ cudaError_t launch_reg(const float* x, int64_t T, int64_t K, int8_t* q, float* a
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = early_start_enabled() ? 1 : 0;
+  cfg.numAttrs = early_start_enabled(st) ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, quant_act_reg_kernel<NT>, x, K, q, act_scale, act_sum);
 }
 
@@ -348,7 +345,7 @@ int launch_quant_act(const float* x, int64_t T, int64_t K, int per_tensor, int8_
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = early_start_enabled() ? 1 : 0;
+    cfg.numAttrs = early_start_enabled(st) ? 1 : 0;
     const unsigned* no_amax = nullptr;
     cudaError_t e = cudaLaunchKernelEx(&cfg, quant_act_kernel, x, K, q, act_scale, act_sum, no_amax);
     if (e != cudaSuccess) return note_cuda_error(e);

@@ -706,7 +706,7 @@ int launch_scan(const SArgs<NMAX>& a, int grid, size_t smem, cudaStream_t st) {
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = early_start_enabled() ? 1 : 0;
+  cfg.numAttrs = early_start_enabled(st) ? 1 : 0;
   cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_tl2_scan_kernel<DEPTH, NMAX, F>, a);
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
 }

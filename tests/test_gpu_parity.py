@@ -708,3 +708,30 @@ def test_tl_prefill_through_the_transcode(fmt):
         n = bn.bitnet_i2s_packed_bytes(M, K)
         assert np.array_equal(npy(ws[:n]), oracle.pack_i2s(w.numpy())), (fmt, M, K)
     assert bn.bitnet_device_status() == 0
+
+
+@pytest.mark.parametrize("fmt", ["i2s", "tl1", "tl2"])
+def test_pack_then_compute_back_to_back_on_one_stream(fmt):
+    """A blob packed and used at once -- no host synchronisation between the packer and the first kernel that reads
+    it, early start on: the decode and prefill kernels copy packed weights before they wait for earlier kernels, so
+    the library itself must order the first launch after a packer behind it.  1, 16 and 256 tokens, through the
+    quantiser (the launch that follows the packer is then not the one that reads the blob) and without it."""
+    for i, (M, K, T) in enumerate([(4096, 8192, 1), (2048, 4096, 16), (1024, 4096, 256), (8192, 8192, 3)]):
+        w = tern(130 + i, M, K)
+        x = synth.normal(131, i, T, K)
+        wd, xd = w.cuda(), x.cuda()
+        q0, sc0, _ = bn.bitnet_quant_act(xd)
+        ws = bn.new_workspace(fmt, T, M, K)
+        ws2 = bn.new_workspace(fmt, T, M, K)
+        torch.cuda.synchronize()
+        blob = bn.pack(fmt, wd, check=False)
+        y, acc = bn.bitnet_mpgemm(fmt, blob, 0.5, M, K, q0, sc0, want_acc=True, workspace=ws)
+        blob2 = bn.pack(fmt, wd, check=False)
+        y2, q2, sc2, acc2 = bn.bitnet_linear(fmt, blob2, 0.5, M, K, xd, want_acc=True, workspace=ws2)
+        torch.cuda.synchronize()
+        q_ref, sc_ref, _ = oracle.quant_act(x.numpy())
+        acc_ref = oracle.mpgemm_def(q_ref, w.numpy())
+        assert np.array_equal(npy(acc), acc_ref), (fmt, M, K, T)
+        assert np.array_equal(npy(acc2), acc_ref), (fmt, M, K, T)
+        check_y(y, acc_ref, sc_ref, 0.5)
+        check_y(y2, acc_ref, sc_ref, 0.5)
