@@ -511,7 +511,7 @@ def bench_elut(bn, torch, synth, wl, layers, card, steps, warmup, check):
     out = {"cardinality": card, "group": 2, "bits_per_weight": 8.0 * nbytes / sum(l.M * l.K for l in wl.linears) / layers,
            "packed_bytes": nbytes, "ms_per_step": ms, "value": nbytes / ms / 1e6, "unit": UNIT,
            "frac_of_hbm_peak": nbytes / ms / 1e6 / peaks()["hbm"],
-           "kernel": "gemv_tl2_scan_kernel in pair mode (one bitnet_elut_linear_group call per step)"}
+           "kernel": "gemv_tl2_scan_kernel, " + ("mask mode" if card == 4 else "pair mode") + " (one bitnet_elut_linear_group call per step)"}
     if check:
         import oracle
         ok = True

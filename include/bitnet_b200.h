@@ -308,7 +308,8 @@ int bitnet_linear_segments(bitnet_fmt_t fmt, const void* packed, int64_t M, int6
  * with the same C are ONE persistent kernel that reads every blob once: an index byte plus its fifth bits selects
  * an entry of a shared-memory table that holds the four weights of the two pairs, which go to the int8 tensor cores
  * as they are (the table is indexed by the packed weights rather than filled from the activations: Phase 1 of the
- * algorithm then costs nothing per token and the lookups feed 4 weights x 8 tokens each).  Integer results are
+ * algorithm then costs nothing per token and the lookups feed 4 weights x 8 tokens each).  At C = 4 the index is two
+ * 2-bit codes side by side and is taken apart by masks instead (BITNET_ELUT4=table: through the table).  Integer results are
  * exact.  Errors: BITNET_ERR_INVALID_ARG (null or misaligned pointer, T outside 1..8), BITNET_ERR_UNSUPPORTED_SHAPE
  * ((C, g) not built, M % 32, K % 4, rows too short for the kernel's rings: K < 192); nothing is queued then.
  */

@@ -1,7 +1,7 @@
 // Element-wise tables beyond ternary (App. A, Table 3) in their g = 2 form, 1..8 tokens: weights of cardinality
 // C = 3, 4, 5 stored as pair indices (2 or 2.5 bits per weight), served by the scan kernel of scan_kernel.cuh in its
 // pair mode -- an index byte and its fifth bits select a table entry holding the four weights of two pairs, which
-// go to the int8 tensor cores as they are.
+// go to the int8 tensor cores as they are; C = 4, whose index is two 2-bit codes, is decoded by masks instead.
 #include "scan_kernel.cuh"
 
 namespace bitnet {
@@ -21,6 +21,10 @@ bool gemv_elut_scan_item_supported(int T, int64_t M, int64_t K, const TlGeom& g)
 }
 
 int launch_gemv_elut_scan(const Tl2Linear* items, int64_t n, int C, cudaStream_t st) {
+  // Cardinality 4: the index is two 2-bit codes, decoded by masks; BITNET_ELUT4=table sends it through the decode
+  // table like the other cardinalities.
+  static const bool table4 = [] { const char* e = getenv("BITNET_ELUT4"); return e && strcmp(e, "table") == 0; }();
+  if (C == 4 && !table4) return scan::launch_items<2>(items, n, C, st);
   return scan::launch_items<1>(items, n, C, st);
 }
 

@@ -33,8 +33,12 @@
 // table entry that IS the A register -- four weights as bytes w + C/2 -- so a tile is 16 lookups and four MMAs per
 // lane with no masking, against activations staged in their natural order; sum(code*q) - (C/2) sum(q) = sum(w*q).
 //
+// For C = 4 the pair index is the two 2-bit codes side by side (at a power of two, bit-wise and element-wise storage
+// coincide: Table 3), so no table is needed (F = 2): one shift and four masks per index word give the A registers of
+// two MMAs at the scales 1 and 16, against activations staged in the matching byte order.
+//
 // This header is the whole kernel and its launcher as templates over F; gemv_tl2_scan.cu and gemv_elut_scan.cu
-// instantiate one each.
+// instantiate them.
 #pragma once
 #include <cstdlib>
 #include <cstring>
@@ -142,6 +146,19 @@ __device__ __forceinline__ bool store_codes(int8_t* row, int i, int word, const 
     const int tile = k >> 6;
     if (tile < pt.t0 || tile >= pt.t1) return false;
     *reinterpret_cast<int*>(row + (k - 64 * pt.t0)) = word;
+    return true;
+  }
+  if (F == 2) {
+    // pair tiles decoded by masks: the 16 columns of lane quarter t are four words, word s holding the columns
+    // 16t + 4j + p(s), j = 0..3, p = (1, 0, 3, 2): bit pair s of index byte j is the code of exactly that column
+    const int tile = k >> 6;
+    if (tile < pt.t0 || tile >= pt.t1) return false;
+    const int c = k & 63, j = (c >> 2) & 3;
+    int8_t* blk = row + (tile - pt.t0) * 64 + (c & 48);
+    blk[4 + j] = (int8_t)word;
+    blk[j] = (int8_t)(word >> 8);
+    blk[12 + j] = (int8_t)(word >> 16);
+    blk[8 + j] = (int8_t)(word >> 24);
     return true;
   }
   if (k < 96 * pt.tiles3) {
@@ -384,7 +401,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
   }
 
   // ---------------- the decode tables (they depend on nothing either)
-  for (int e = warp; e < 1024; e += CW) {
+  for (int e = warp; e < (F == 2 ? 0 : 1024); e += CW) {
     const int byte = e & 255;
     if (F == 1) {
       // pair index i < C^2 -> the weights (i / C, i % C) + lo as codes i / C, i % C; an index that does not occur
@@ -465,8 +482,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
           const uint32_t sl = ring + slot * SLOT;
           unsigned iw[4], sg[4] = {0u, 0u, 0u, 0u};
           lds128(sl + lane * 16, iw);            // index word t of rows g, g+8, g+16, g+24
-          if (hb) lds128(sl + 512 + g * 16, sg); // their sign words (fifth index bits)
-          if (F == 1)
+          if (F != 2 && hb) lds128(sl + 512 + g * 16, sg); // their sign words (fifth index bits)
+          if (F != 0)
             asm volatile(
                 "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %5, 0;\n\t"
                 "@p ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n\t}"
@@ -482,7 +499,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
                 : "r"(qp), "r"(has_tok));
           unsigned e[4][4];                      // [row u][index byte j]
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
+          for (int u = 0; u < (F == 2 ? 0 : 4); ++u) {
             const unsigned tw = (sg[u] >> (2 * t)) & 0x03030303u;     // sign pair of index byte j in byte j
             // (the entry's address by a multiply-add: the FMA pipe has room, the integer pipe is the busy one)
             e[u][0] = lds32(mad_u32(prmt(iw[u], tw, 0xCC40u), 128u, tbl2_lane));
@@ -490,7 +507,17 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
             e[u][2] = lds32(mad_u32(prmt(iw[u], tw, 0xEE62u), 128u, tbl2_lane));
             e[u][3] = lds32(mad_u32(prmt(iw[u], tw, 0xFF73u), 128u, tbl2_lane));
           }
-          if (F == 1) {
+          if (F == 2) {
+            // bit pairs 0, 1 of the index bytes at scale 1 (in place, shifted down by two), pairs 2, 3 at scale 16
+            constexpr unsigned M0 = 0x03030303u, M2 = 0x30303030u;
+            unsigned hi[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) hi[u] = iw[u] >> 2;
+            mma_u8s8(C0[0], iw[0] & M0, iw[1] & M0, hi[0] & M0, hi[1] & M0, qr[0], qr[1]);
+            mma_u8s8(C1[0], iw[2] & M0, iw[3] & M0, hi[2] & M0, hi[3] & M0, qr[0], qr[1]);
+            mma_u8s8(C0[1], iw[0] & M2, iw[1] & M2, hi[0] & M2, hi[1] & M2, qr[2], qr[3]);
+            mma_u8s8(C1[1], iw[2] & M2, iw[3] & M2, hi[2] & M2, hi[3] & M2, qr[2], qr[3]);
+          } else if (F == 1) {
             // entry of index byte j = the codes of columns 16t + 4j .. + 3, the activation word j of the lane's quarter
             mma_u8s8(C0[0], e[0][0], e[1][0], e[0][1], e[1][1], qr[0], qr[1]);
             mma_u8s8(C1[0], e[2][0], e[3][0], e[2][1], e[3][1], qr[0], qr[1]);
@@ -572,7 +599,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
         for (int u = 0; u < 2; ++u) {
           int c[4];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) c[i] = u == 0 ? C0[0][i] + (C0[1][i] >> 2) : C1[0][i] + (C1[1][i] >> 2);
+          for (int i = 0; i < 4; ++i)
+            c[i] = u == 0 ? C0[0][i] + (C0[1][i] >> (F == 2 ? 4 : 2)) : C1[0][i] + (C1[1][i] >> (F == 2 ? 4 : 2));
           if (2 * t < T) {
             mine[(2 * t) * 32 + 16 * u + g] = c[0];
             mine[(2 * t) * 32 + 16 * u + g + 8] = c[2];

@@ -141,3 +141,21 @@ def test_elut_malformed_items_are_refused():
     with pytest.raises(bn.BitnetError, match="invalid"):
         bn.bitnet_elut_linear_group(bn.make_elut_group([dict(base, q=q9)]))       # more than 8 tokens
     bn.bitnet_elut_linear_group(bn.make_elut_group([]))                           # an empty list is fine
+
+
+def test_cardinality4_through_the_decode_table_in_a_child_process():
+    """Cardinality 4 is decoded by masks by default (its pair index is two 2-bit codes); BITNET_ELUT4=table, read once
+    per process, sends it through the decode table like cardinality 3 and 5.  Same integers either way."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = ("import sys; sys.path.insert(0, 'tests')\n"
+            "from test_gpu_elut import _run, _check\n"
+            "for fused in (False, True):\n"
+            "    for M, K, T in [(32, 192, 1), (64, 1028, 1), (96, 4096, 3), (2048, 4100, 1), (160, 8192, 8), (64, 28672, 2)]:\n"
+            "        _check(*_run([(4, M, K, T, 20 + T)], fused))\n"
+            "print('ok')\n")
+    out = subprocess.run([sys.executable, "-c", code], cwd=root, env=dict(os.environ, BITNET_ELUT4="table"),
+                         capture_output=True, text=True, timeout=900)
+    assert out.returncode == 0 and "ok" in out.stdout, out.stderr[-2000:]
