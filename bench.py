@@ -657,7 +657,7 @@ def run_ours(args):
             ms_tl1 = time_replays(torch, lambda: sw.step_group("tl1"), max(5, args.steps // 2), args.warmup)
             line["tl1"] = {"packed_bytes": sw.bytes["tl1"], "ms_per_step": ms_tl1, "value": sw.bytes["tl1"] / ms_tl1 / 1e6,
                            "unit": UNIT, "frac_of_hbm_peak": sw.bytes["tl1"] / ms_tl1 / 1e6 / pk["hbm"],
-                           "kernel": "gemv_tl2_scan_kernel in pair mode (one bitnet_linear_group call per step)"}
+                           "kernel": "gemv_tl2_scan_kernel, arithmetic mode (one bitnet_linear_group call per step)"}
             sw.step_group("tl2")        # the verification below sees the scan kernel's y
         if not args.skip_batched:
             line["batched_decode"] = {

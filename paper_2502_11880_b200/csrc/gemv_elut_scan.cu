@@ -25,6 +25,10 @@ int launch_gemv_elut_scan(const Tl2Linear* items, int64_t n, int C, cudaStream_t
   // table like the other cardinalities.
   static const bool table4 = [] { const char* e = getenv("BITNET_ELUT4"); return e && strcmp(e, "table") == 0; }();
   if (C == 4 && !table4) return scan::launch_items<2>(items, n, C, st);
+  // Cardinality 3 (TL1 blobs): the pair code 3 a + b is taken apart by byte-wise arithmetic; BITNET_TL1=table sends it
+  // through the decode table.
+  static const bool table3 = [] { const char* e = getenv("BITNET_TL1"); return e && strcmp(e, "table") == 0; }();
+  if (C == 3 && !table3) return scan::launch_items<3>(items, n, C, st);
   return scan::launch_items<1>(items, n, C, st);
 }
 

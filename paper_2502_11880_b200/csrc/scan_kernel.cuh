@@ -36,6 +36,10 @@
 // For C = 4 the pair index is the two 2-bit codes side by side (at a power of two, bit-wise and element-wise storage
 // coincide: Table 3), so no table is needed (F = 2): one shift and four masks per index word give the A registers of
 // two MMAs at the scales 1 and 16, against activations staged in the matching byte order.
+// For C = 3 (TL1: Table 4's code of a pair is 3 a + b with a, b the weights + 1) the index is taken apart by byte-wise
+// arithmetic (F = 3): the index nibbles of a word spread over two words of bytes x; bits 5, 6 of 11 x are a = x / 3
+// (x <= 8, and 11 x stays inside its byte), so 32 a = (11 x) & 0x60 and 32 b = 32 x - 3 (32 a): four A registers of
+// byte codes per index word at the scale 32, more than half of the instructions on the multiply-add pipe.
 //
 // This header is the whole kernel and its launcher as templates over F; gemv_tl2_scan.cu and gemv_elut_scan.cu
 // instantiate them.
@@ -159,6 +163,18 @@ __device__ __forceinline__ bool store_codes(int8_t* row, int i, int word, const 
     blk[j] = (int8_t)(word >> 8);
     blk[12 + j] = (int8_t)(word >> 16);
     blk[8 + j] = (int8_t)(word >> 24);
+    return true;
+  }
+  if (F == 3) {
+    // pair tiles decoded by arithmetic: word d of a lane quarter's 16 bytes holds the columns 16t + 4j + d, j = 0..3
+    const int tile = k >> 6;
+    if (tile < pt.t0 || tile >= pt.t1) return false;
+    const int c = k & 63, j = (c >> 2) & 3;
+    int8_t* blk = row + (tile - pt.t0) * 64 + (c & 48);
+    blk[j] = (int8_t)word;
+    blk[4 + j] = (int8_t)(word >> 8);
+    blk[8 + j] = (int8_t)(word >> 16);
+    blk[12 + j] = (int8_t)(word >> 24);
     return true;
   }
   if (k < 96 * pt.tiles3) {
@@ -401,7 +417,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
   }
 
   // ---------------- the decode tables (they depend on nothing either)
-  for (int e = warp; e < (F == 2 ? 0 : 1024); e += CW) {
+  for (int e = warp; e < (F >= 2 ? 0 : 1024); e += CW) {
     const int byte = e & 255;
     if (F == 1) {
       // pair index i < C^2 -> the weights (i / C, i % C) + lo as codes i / C, i % C; an index that does not occur
@@ -482,7 +498,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
           const uint32_t sl = ring + slot * SLOT;
           unsigned iw[4], sg[4] = {0u, 0u, 0u, 0u};
           lds128(sl + lane * 16, iw);            // index word t of rows g, g+8, g+16, g+24
-          if (F != 2 && hb) lds128(sl + 512 + g * 16, sg); // their sign words (fifth index bits)
+          if (F < 2 && hb) lds128(sl + 512 + g * 16, sg); // their sign words (fifth index bits)
           if (F != 0)
             asm volatile(
                 "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %5, 0;\n\t"
@@ -499,7 +515,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
                 : "r"(qp), "r"(has_tok));
           unsigned e[4][4];                      // [row u][index byte j]
 #pragma unroll
-          for (int u = 0; u < (F == 2 ? 0 : 4); ++u) {
+          for (int u = 0; u < (F >= 2 ? 0 : 4); ++u) {
             const unsigned tw = (sg[u] >> (2 * t)) & 0x03030303u;     // sign pair of index byte j in byte j
             // (the entry's address by a multiply-add: the FMA pipe has room, the integer pipe is the busy one)
             e[u][0] = lds32(mad_u32(prmt(iw[u], tw, 0xCC40u), 128u, tbl2_lane));
@@ -507,7 +523,25 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
             e[u][2] = lds32(mad_u32(prmt(iw[u], tw, 0xEE62u), 128u, tbl2_lane));
             e[u][3] = lds32(mad_u32(prmt(iw[u], tw, 0xFF73u), 128u, tbl2_lane));
           }
-          if (F == 2) {
+          if (F == 3) {
+            // x = index nibbles as bytes (0..8); a = x / 3 = (11 x) >> 5, b = x - 3 a: the codes of the pair's weights
+            // Both kept at the scale 32 where bits 5, 6 of 11 x hold a: 32 a = (11 x) & 0x60, 32 b = 32 x - 3 (32 a)
+            // (multiply-adds; every byte of the result is at most 64, so the word arithmetic is exact).
+            constexpr unsigned MB = 0x0F0F0F0Fu, MA = 0x60606060u;
+            unsigned alo[4], blo[4], ahi[4], bhi[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const unsigned xl = iw[u] & MB, xh = (iw[u] >> 4) & MB;
+              alo[u] = mad_u32(xl, 11u, 0u) & MA;
+              ahi[u] = mad_u32(xh, 11u, 0u) & MA;
+              blo[u] = mad_u32(xl, 32u, mad_u32(alo[u], 0xFFFFFFFDu, 0u));
+              bhi[u] = mad_u32(xh, 32u, mad_u32(ahi[u], 0xFFFFFFFDu, 0u));
+            }
+            mma_u8s8(C0[0], alo[0], alo[1], blo[0], blo[1], qr[0], qr[1]);
+            mma_u8s8(C1[0], alo[2], alo[3], blo[2], blo[3], qr[0], qr[1]);
+            mma_u8s8(C0[0], ahi[0], ahi[1], bhi[0], bhi[1], qr[2], qr[3]);
+            mma_u8s8(C1[0], ahi[2], ahi[3], bhi[2], bhi[3], qr[2], qr[3]);
+          } else if (F == 2) {
             // bit pairs 0, 1 of the index bytes at scale 1 (in place, shifted down by two), pairs 2, 3 at scale 16
             constexpr unsigned M0 = 0x03030303u, M2 = 0x30303030u;
             unsigned hi[4];
@@ -600,7 +634,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
           int c[4];
 #pragma unroll
           for (int i = 0; i < 4; ++i)
-            c[i] = u == 0 ? C0[0][i] + (C0[1][i] >> (F == 2 ? 4 : 2)) : C1[0][i] + (C1[1][i] >> (F == 2 ? 4 : 2));
+            c[i] = u == 0 ? (C0[0][i] >> (F == 3 ? 5 : 0)) + (C0[1][i] >> (F == 2 ? 4 : 2))
+                          : (C1[0][i] >> (F == 3 ? 5 : 0)) + (C1[1][i] >> (F == 2 ? 4 : 2));
           if (2 * t < T) {
             mine[(2 * t) * 32 + 16 * u + g] = c[0];
             mine[(2 * t) * 32 + 16 * u + g + 8] = c[2];

@@ -652,13 +652,13 @@ def _run_child(code, extra_env):
                                    dict(BITNET_FUSE_MAX_T="0"), dict(BITNET_I2S_MID_MIN_T="9"),
                                    dict(BITNET_MID_NS="5"), dict(BITNET_TL2="lut"), dict(BITNET_TL2_S="4", BITNET_TL2_DEPTH="4"),
                                    dict(BITNET_GROUP="0"), dict(BITNET_GROUP_S="2", BITNET_GROUP_DEPTH="8"),
-                                   dict(BITNET_GROUP_DEPTH="12")])
+                                   dict(BITNET_GROUP_DEPTH="12"), dict(BITNET_TL1="table")])
 def test_read_once_switches_in_child_processes(extra):
     """Every kernel choice that an environment variable makes (read once per process) against the oracle: the dp4a
     prefill kernel, plain stores instead of bulk tensor stores in the tensor-core prefill kernel, the bulk-copy ring
     decode kernel, the quantiser without clusters, no fused quantiser, the mid-batch kernel's lower limit and forced
-    slice count, the lookup-table kernel for TL1 and TL2, other ring depths and warps per unit in the grouped kernels, and
-    the grouped call switched off."""
+    slice count, the lookup-table kernel for TL1 and TL2, other ring depths and warps per unit in the grouped kernels,
+    the grouped call switched off, and TL1 through the scan kernel's decode table instead of its arithmetic decode."""
     code = (
         "import sys; sys.path.insert(0, 'tests'); import numpy as np, torch\n"
         "import oracle\n"
