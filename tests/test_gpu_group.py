@@ -107,6 +107,16 @@ def test_group_more_items_than_the_small_argument_block():
         it.check()
 
 
+@pytest.mark.parametrize("fmt,count", [("i2s", 430), ("tl2", 360), ("tl1", 350)])
+def test_group_more_items_than_one_launch_takes(fmt, count):
+    """More items than the largest argument block holds (409 for I2_S, 340 for the scan kernel): the call is cut into
+    several launches, in list order."""
+    items = [Item(fmt, 32 * (1 + i % 3), 1024 + 256 * (i % 3), 1 + i % 3, 3000 + i) for i in range(count)]
+    run_group(items)
+    for it in items:
+        it.check()
+
+
 def test_group_equals_single_calls_and_given_workload_layer():
     """A 100B-shaped decoder layer (8192->10240, 8192->8192, 8192->57344, 28672->8192) at one token through the
     grouped call: every output row against the oracle."""
