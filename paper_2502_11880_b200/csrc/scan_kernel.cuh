@@ -564,10 +564,13 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
             mma_u8s8(C1[0], e[2][0] & M0, e[3][0] & M0, e[2][1] & M0, e[3][1] & M0, qr[0], qr[1]);
             mma_u8s8(C0[0], e[0][2] & M0, e[1][2] & M0, e[0][3] & M0, e[1][3] & M0, qr[2], qr[3]);
             mma_u8s8(C1[0], e[2][2] & M0, e[3][2] & M0, e[2][3] & M0, e[3][3] & M0, qr[2], qr[3]);
-            mma_u8s8(C0[1], prmt(e[0][0], e[0][2], 0x5410u) & M1, prmt(e[1][0], e[1][2], 0x5410u) & M1,
-                     prmt(e[0][1], e[0][3], 0x5410u) & M1, prmt(e[1][1], e[1][3], 0x5410u) & M1, qr[4], qr[5]);
-            mma_u8s8(C1[1], prmt(e[2][0], e[2][2], 0x5410u) & M1, prmt(e[3][0], e[3][2], 0x5410u) & M1,
-                     prmt(e[2][1], e[2][3], 0x5410u) & M1, prmt(e[3][1], e[3][3], 0x5410u) & M1, qr[4], qr[5]);
+            // (bytes 2, 3 of an entry carry nothing under M1, so the second entry shifted up by a multiply-add and
+            // one three-input logic operation join the pairs: one integer-pipe instruction per register)
+            auto join = [](unsigned ea, unsigned eb) { return (ea | mad_u32(eb, 65536u, 0u)) & M1; };
+            mma_u8s8(C0[1], join(e[0][0], e[0][2]), join(e[1][0], e[1][2]), join(e[0][1], e[0][3]), join(e[1][1], e[1][3]),
+                     qr[4], qr[5]);
+            mma_u8s8(C1[1], join(e[2][0], e[2][2]), join(e[3][0], e[3][2]), join(e[2][1], e[2][3]), join(e[3][1], e[3][3]),
+                     qr[4], qr[5]);
           }
           qp += COLS;
           __syncwarp();                          // every lane has read the slot's sign plane
