@@ -242,14 +242,19 @@ int bitnet_linear_host_batch(const bitnet_host_linear_t* items, int64_t n, void*
  *     x[T][K] fp32 in, q[T][K] int8 and act_scale[T] fp32 out, y[T][M] fp32 out, acc_out nullable.
  *     Items that share an input may share x, q and act_scale (neighbouring I2_S items with the same x, K and
  *     T are quantised once per CTA).
- *   - I2_S items with T <= 8, K >= 1024 and T*(K+16) <= 144 KiB run in ONE persistent kernel per run of
- *     up to 454 consecutive such items: the packed weights of the whole run are one stream, cut into equal
- *     shares per SM at 16-row borders; a CTA's asynchronous copies run on across the borders between
- *     linears, and each activation row is quantised by the two or three CTAs whose share touches its linear
- *     instead of by every CTA of a launch of its own.  The per-launch fixed cost of a decode GEMV (about
- *     3 us of the 5-20 us a 100B-shaped linear takes) is paid once per run.
- *   - Every other item (TL formats, more tokens, short K) is run by bitnet_linear in list order, with the
- *     item's workspace.
+ *   - I2_S items with T <= 8 and K >= 1024 run in ONE persistent kernel per run of up to 409 consecutive
+ *     such items: the packed weights of the whole run are one stream, cut into equal shares per SM at
+ *     16-row borders; a CTA's asynchronous copies run on across the borders between linears, and each
+ *     activation row is quantised by the two or three CTAs whose share touches its linear instead of by
+ *     every CTA of a launch of its own (rows whose codes do not fit shared memory are walked in parts of K).
+ *     The per-launch fixed cost of a decode GEMV (about 3 us of the 5-20 us a 100B-shaped linear takes) is
+ *     paid once per run.  Items with 9 to 16 tokens join such a run as two items over the same weights
+ *     (tokens 0..7, then the rest).
+ *   - TL2 and TL1 items with T <= 8 (K a multiple of 4, at least three tiles per row) likewise run in one
+ *     persistent kernel per run of up to 340 consecutive items of the same format (the scan kernel, see
+ *     bitnet_set_tl2_lookup).
+ *   - Every other item (more tokens, short K) is run by bitnet_linear in list order, with the item's
+ *     workspace.
  * Results are identical to calling bitnet_linear per item.  Errors: BITNET_ERR_INVALID_ARG for a null or
  * malformed item (nothing is queued), otherwise the status of the first failing launch.
  */

@@ -427,8 +427,13 @@ int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* strea
     }
   }
   static const bool grouped = [] { const char* e = getenv("BITNET_GROUP"); return !(e && atoi(e) == 0); }();
+  // 9 to 16 tokens: two passes of the grouped kernel (tokens 0..7, then the rest) beat the mid-batch kernel's
+  // launch per linear on lists (6.4 against 8.4 ms on the 100B sweep at 16 tokens); BITNET_GROUP_MAX_T lowers the limit.
+  static const int group_max_t = [] { const char* e = getenv("BITNET_GROUP_MAX_T"); const int v = e ? atoi(e) : 16; return v < 8 ? 8 : (v > 16 ? 16 : v); }();
   auto takes = [&](const bitnet_group_item_t& d) {
-    return grouped && d.fmt == BITNET_FMT_I2S && d.T <= 8 && gemv_i2s_group_item_supported((int)d.T, d.M, d.K);
+    if (!grouped || d.fmt != BITNET_FMT_I2S || d.T > group_max_t) return false;
+    if (d.T <= 8) return gemv_i2s_group_item_supported((int)d.T, d.M, d.K);
+    return gemv_i2s_group_item_supported(8, d.M, d.K) && gemv_i2s_group_item_supported((int)d.T - 8, d.M, d.K);
   };
   static thread_local std::vector<GroupLinear> run;
   static thread_local std::vector<Tl2Linear> run2;
@@ -482,11 +487,20 @@ int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* strea
       gl.y = d.y;
       gl.acc_out = d.acc_out;
       gl.w_scale = d.w_scale;
-      gl.T = (int)d.T;
+      gl.T = (int)(d.T > 8 ? 8 : d.T);
       gl.M = d.M;
       gl.K = d.K;
       gl.ldy = 0;
       run.push_back(gl);
+      if (d.T > 8) {                       // the remaining tokens: a second item over the same weights
+        gl.x = d.x + 8 * d.K;
+        gl.q = d.q + 8 * d.K;
+        gl.act_scale = d.act_scale + 8;
+        gl.y = d.y + 8 * d.M;
+        gl.acc_out = d.acc_out ? d.acc_out + 8 * d.M : nullptr;
+        gl.T = (int)d.T - 8;
+        run.push_back(gl);
+      }
     }
     int rc = launch_gemv_i2s_group(run.data(), (int64_t)run.size(), (cudaStream_t)stream);
     if (rc) return rc;

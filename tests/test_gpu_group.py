@@ -67,6 +67,17 @@ def test_group_small_ragged_list():
         it.check()
 
 
+def test_group_nine_to_sixteen_tokens_in_two_passes():
+    """Items with 9 to 16 tokens run as two items over the same weights (tokens 0..7, then the rest); ragged rows, a
+    long row walked in parts, neighbours with fewer tokens, and an item with 17 tokens (left to the mid-batch kernel)."""
+    shapes = [(40, 2048, 9), (300, 8192, 16), (33, 28672, 12), (64, 4096, 3), (1000, 3200, 13), (64, 4096, 17),
+              (17, 1536, 10)]
+    items = [Item("i2s", M, K, T, 150 + i) for i, (M, K, T) in enumerate(shapes)]
+    run_group(items)
+    for it in items:
+        it.check()
+
+
 def test_group_many_units_per_cta_and_shared_inputs():
     """More units than warp groups (every group walks several units and crosses item borders), Q/K/V-like items
     that share one activation buffer (quantised once, each item still gets its codes), and an item whose token
