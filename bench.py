@@ -306,8 +306,9 @@ class Sweep:
 def bench_batched(sw, torch, T, steps, warmup):
     """The same sweep with T tokens per linear (I2_S) through ONE bitnet_linear_group call per step: quantiser +
     mpGEMM + rescale.  Every linear keeps its own weights; the T activation rows of layer 0's four linears are
-    reused by all layers.  Up to 8 tokens the whole list is one persistent kernel; beyond that the call runs every
-    item as bitnet_linear (quantiser + mid-batch mma.sync kernel + rescale, three launches per linear)."""
+    reused by all layers.  Up to 8 tokens the whole list is one persistent kernel; 9 to 16 tokens are two items of that
+    kernel per linear (tokens 0..7, then the rest: two launches of 320 items each); beyond that the call runs every item
+    as bitnet_linear (quantiser + mid-batch mma.sync kernel + rescale, three launches per linear)."""
     bn, dev = sw.bn, sw.x_dev.device
     nl = len(sw.lin)
     xs = [sw.wl.activations(0, j, T).to(dev) for j in range(nl)]
@@ -596,7 +597,7 @@ def run_ours(args):
     clocks = sampler.stop() if sampler else None
     value = whole_job_value(sw.bytes["i2s"], world, ms_step)
     achieved = sw.bytes["i2s"] / ms_step / 1e6
-    launches_per_step = -(-n_lin // 454)      # the grouped kernel takes up to 454 items per launch
+    launches_per_step = -(-n_lin // 409)      # the grouped kernel takes up to 409 items per launch
 
     # ---- end to end through the host-buffer entry point
     ms_e2e = time_replays(torch, lambda: (sw.step_host("i2s"), torch.cuda.current_stream().synchronize()),
@@ -662,7 +663,7 @@ def run_ours(args):
         if not args.skip_batched:
             line["batched_decode"] = {
                 "note": "the same sweep with T tokens per linear, one bitnet_linear_group call per step, inputs resident",
-                "runs": [bench_batched(sw, torch, T, max(3, args.steps // 5), 3) for T in (2, 4, 8, 16, 64)]}
+                "runs": [bench_batched(sw, torch, T, max(3, args.steps // 5), 3) for T in (2, 4, 8, 16, 32, 64)]}
         if world == 1 and not args.skip_cpu:
             # ---- CPU baseline leg: the oracle, as it stands, on one full layer of the sweep for about 10 s on the
             # host cores; its results then check the y the GPU left in device memory
