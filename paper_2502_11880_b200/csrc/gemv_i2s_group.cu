@@ -73,6 +73,11 @@ __device__ __forceinline__ bool same_input(const GItem& p, const GItem& d) {
          (d.x ? p.x == d.x : (p.x == nullptr && p.q == d.q && p.act_scale == d.act_scale));
 }
 
+// Where word r (four columns) of a staged row lies: within every 256-column chunk the 16-byte pieces are kept as
+// [piece p][lane quarter t] instead of [t][p], so that the four quarters' loads of one piece (and, with the row
+// stride of 64 bytes modulo 128, the rows of two tokens) cover the 32 banks exactly once.
+__device__ __forceinline__ int staged_word(int r) { return (r & ~63) | ((r & 12) << 2) | ((r & 48) >> 2) | (r & 3); }
+
 // Stages the activation codes of the item's columns [256 c0, 256 c1) (T rows, qst bytes apart, zero beyond K) and,
 // per token, the scale and the sum of the staged codes.  `first` = the item's first part: the row maximum is taken
 // (Alg. 1 Phase 1) and, in the CTA that owns the item, codes and scales of the WHOLE row go to the caller; later
@@ -121,7 +126,7 @@ __device__ __forceinline__ void stage_item(const GItem& d, bool owner, bool firs
         if (r < nrow && i < kw) {
           const int word = quant4_packed(xv[r], sq);  // columns K..Kp-1 came in as zeros
           if (i >= w0 && i < w1) {
-            reinterpret_cast<int*>(qs_mem + tok * qst)[i - w0] = word;
+            reinterpret_cast<int*>(qs_mem + tok * qst)[staged_word(i - w0)] = word;
             s = __dp4a(word, 0x01010101, s);
           }
           if (owner && i < n4) reinterpret_cast<int*>(d.q + (int64_t)tok * d.K)[i] = word;
@@ -167,7 +172,7 @@ __device__ __forceinline__ void stage_item(const GItem& d, bool owner, bool firs
           if (owner && first) reinterpret_cast<int*>(d.q + (int64_t)tok * d.K)[i] = word;
         }
         if (i >= w0 && i < w1) {
-          reinterpret_cast<int*>(qs_mem + tok * qst)[i - w0] = word;
+          reinterpret_cast<int*>(qs_mem + tok * qst)[staged_word(i - w0)] = word;
           s = __dp4a(word, 0x01010101, s);
         }
       }
@@ -183,7 +188,7 @@ __device__ __forceinline__ void stage_item(const GItem& d, bool owner, bool firs
       int s = 0;
       for (int i = w0 + threadIdx.x; i < w1; i += THREADS) {
         const int word = (i < n4) ? __ldcg(qrow + i) : 0;
-        reinterpret_cast<int*>(qs_mem + tok * qst)[i - w0] = word;
+        reinterpret_cast<int*>(qs_mem + tok * qst)[staged_word(i - w0)] = word;
         s = __dp4a(word, 0x01010101, s);
       }
 #pragma unroll
@@ -301,7 +306,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
   for (int ci = item0; ci <= item1; ++ci) {
     const GItem& d = a.it[ci];
     const int T = d.T, kp = (int)i2s_kp(d.K), nch = kp / 256, nparts = d.nparts;
-    const int qst = ((nch + nparts - 1) / nparts) * 256 + 16;
+    const int qst = ((nch + nparts - 1) / nparts) * 256 + 64;
     const bool owner = jb <= d.first_unit;
     const int jlo = range_lo(ci), jhi = range_hi(ci);
     const int first = d.first_unit, M = d.M, ldy = d.ldy;
@@ -320,11 +325,11 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
         // same input as the previous item but its own output buffers for the codes
         for (int tok = 0; tok < T; ++tok)
           for (int i = threadIdx.x; i < d.K / 4; i += THREADS)
-            reinterpret_cast<int*>(d.q + (int64_t)tok * d.K)[i] = reinterpret_cast<const int*>(qs_mem + tok * qst)[i];
+            reinterpret_cast<int*>(d.q + (int64_t)tok * d.K)[i] = reinterpret_cast<const int*>(qs_mem + tok * qst)[staged_word(i)];
         if (threadIdx.x < T) d.act_scale[threadIdx.x] = qscale[threadIdx.x];
       }
       const int s_lo = wk * npc / S, nw = (wk + 1) * npc / S - s_lo;
-      const uint32_t q_lane = smem_u32(qs_mem + min(g, T - 1) * qst + s_lo * 256 + t * 64);
+      const uint32_t q_lane = smem_u32(qs_mem + min(g, T - 1) * qst + s_lo * 256 + t * 16);
       const bool last_part = part + 1 == nparts;
 
       for (int cj = jlo; cj < jhi; cj += G, ++nloc) {
@@ -352,9 +357,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
             asm volatile(
                 "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %9, 0;\n\t"
                 "@p ld.shared.v4.u32 {%0,%1,%2,%3}, [%8];\n\t"
-                "@p ld.shared.v4.u32 {%4,%5,%6,%7}, [%8+16];\n\t}"
+                "@p ld.shared.v4.u32 {%4,%5,%6,%7}, [%8+64];\n\t}"
                 : "+r"(qr[0]), "+r"(qr[1]), "+r"(qr[2]), "+r"(qr[3]), "+r"(qr[4]), "+r"(qr[5]), "+r"(qr[6]), "+r"(qr[7])
-                : "r"(qp + h * 32), "r"(has_tok));
+                : "r"(qp + h * 128), "r"(has_tok));
 #pragma unroll
             for (int s = 0; s < 4; ++s) {
               const unsigned m = 0x03030303u << (2 * s);
@@ -493,7 +498,7 @@ bool plan_item(int T, int64_t M, int64_t K, ItemPlan* out) {
     for (int n = 1; n <= 8; ++n) {
       const int64_t big = ceil_div(nch, n), small = nch / n;
       if (small < 4) break;
-      const size_t code = ((size_t)T * (size_t)(big * 256 + 16) + 127) & ~(size_t)127;
+      const size_t code = ((size_t)T * (size_t)(big * 256 + 64) + 127) & ~(size_t)127;
       if (code <= MAX_CODE_BYTES && smem_of(T, code, want_depth) <= cap) {
         *out = ItemPlan{n, code, small};
         return true;

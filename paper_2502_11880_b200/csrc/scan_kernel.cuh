@@ -60,6 +60,14 @@ constexpr int NSMALL = 42, NLARGE = 340;   // items per launch: argument blocks 
 constexpr int SLOT = 640;                  // ring slot = one tile
 constexpr int TBL2_BYTES = 1024 * 32 * 4;
 
+// Bytes between the staged rows of two tokens: the columns of the largest part (+ a pair-coded tail) rounded up to
+// 96 (triple tiles) or 64 (pair tiles) modulo 128, so that the activation loads of a quarter- or half-warp -- the
+// lane quarters of one token 24 or 16 bytes apart, the tokens one row apart -- cover the 32 banks exactly once.
+__host__ __device__ inline int staged_stride(int cols, int big, int tiles2) {
+  const int raw = big * cols + tiles2 * 64 + 16, want = cols == 96 ? 96 : 64;
+  return ((raw - want + 127) / 128) * 128 + want;
+}
+
 struct SItem {
   const uint8_t* packed;
   const float* x;      // fp32 activations [T][K]; null: q and act_scale are inputs
@@ -330,7 +338,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
   unsigned* tbl1 = reinterpret_cast<unsigned*>(smem + 1024);     // [256] index byte of two pairs -> four codes
   int* red = reinterpret_cast<int*>(smem + 2048);                // [CW][2][tmax][32] partial sums
   unsigned* tbl2 = reinterpret_cast<unsigned*>(smem + 2048 + CW * 2 * a.tmax * 32 * 4);   // [1024][32 lanes]
-  int8_t* qs_mem = reinterpret_cast<int8_t*>(tbl2) + TBL2_BYTES;
+  int8_t* qs_mem = reinterpret_cast<int8_t*>(tbl2) + (F >= 2 ? 0 : TBL2_BYTES);   // (the mask and arithmetic modes have no table)
   uint8_t* rings = reinterpret_cast<uint8_t*>(qs_mem) + a.code_bytes;
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -453,7 +461,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
   for (int ci = item0; ci <= item1; ++ci) {
     const SItem& d = a.it[ci];
     const int T = d.T, tiles3 = d.tiles3, tiles2 = d.tiles2, nparts = d.nparts;
-    const int qst = ((tiles3 + nparts - 1) / nparts) * COLS + tiles2 * 64 + 16;
+    const int qst = staged_stride(COLS, (tiles3 + nparts - 1) / nparts, tiles2);
     const bool owner = jb <= d.first_unit;
     const int jlo = range_lo(ci), jhi = range_hi(ci);
     const int first = d.first_unit, M = d.M, ldy = d.ldy;
@@ -698,8 +706,8 @@ inline int forced_s() {
   return s;
 }
 
-inline size_t smem_of(int tmax, size_t code_bytes, int depth) {
-  return 2048 + (size_t)CW * 2 * tmax * 32 * 4 + TBL2_BYTES + code_bytes + (size_t)CW * depth * SLOT;
+inline size_t smem_of(int tmax, size_t code_bytes, int depth, int F) {
+  return 2048 + (size_t)CW * 2 * tmax * 32 * 4 + (F >= 2 ? 0 : TBL2_BYTES) + code_bytes + (size_t)CW * depth * SLOT;
 }
 
 // How one item is walked: its triple tiles in `nparts` parts (as few as let the staged codes of a part fit beside
@@ -710,15 +718,15 @@ struct ItemPlan {
   size_t code;
   int t3;
 };
-inline bool plan_item(int T, const TlGeom& g, int cols, ItemPlan* out) {
+inline bool plan_item(int T, const TlGeom& g, int cols, int F, ItemPlan* out) {
   const size_t cap = (size_t)dev_info().max_smem_optin;
   const int tiles3 = (int)g.tiles3, tiles2 = (int)g.tiles2;
   for (int want_depth = 4; want_depth >= 3; --want_depth)
     for (int n = 1; n <= 16; ++n) {
       const int big = (tiles3 + n - 1) / n, small = tiles3 / n;
       if (small < 3) break;
-      const size_t code = ((size_t)T * (size_t)(big * cols + tiles2 * 64 + 16) + 127) & ~(size_t)127;
-      if (smem_of(T, code, want_depth) <= cap) {
+      const size_t code = ((size_t)T * (size_t)staged_stride(cols, big, tiles2) + 127) & ~(size_t)127;
+      if (smem_of(T, code, want_depth, F) <= cap) {
         *out = ItemPlan{n, code, small};
         return true;
       }
@@ -731,7 +739,7 @@ struct Shape {
 };
 // S and ring depth for a launch whose shortest rows have `t3` triple tiles: every warp's run of triple tiles is at
 // least as long as its ring; the ring is made shallower until everything fits one SM's shared memory.
-inline bool launch_shape(int t3, int tmax, size_t code, int64_t units, Shape* out) {
+inline bool launch_shape(int t3, int tmax, size_t code, int64_t units, int F, Shape* out) {
   // Warps per 32-row block: one when the launch has enough blocks to keep the 16 warps of every SM busy with
   // blocks of their own (no partial sums to join: 3.4 TB/s against 3.1 with four on the 100B sweep), more when
   // it has few.
@@ -746,8 +754,8 @@ inline bool launch_shape(int t3, int tmax, size_t code, int64_t units, Shape* ou
   const size_t cap = (size_t)dev_info().max_smem_optin;
   int depth = depth_cap();
   auto lower = [](int d) { return d == 8 ? 6 : d - 1; };
-  while (depth > 3 && (depth > nw || smem_of(tmax, code, depth) > cap)) depth = lower(depth);
-  if (depth > nw || smem_of(tmax, code, depth) > cap) return false;
+  while (depth > 3 && (depth > nw || smem_of(tmax, code, depth, F) > cap)) depth = lower(depth);
+  if (depth > nw || smem_of(tmax, code, depth, F) > cap) return false;
   *out = Shape{S, depth};
   return true;
 }
@@ -802,7 +810,7 @@ int launch_run(const Tl2Linear* items, int n, int card, Shape shape, cudaStream_
     const Tl2Linear& s = items[i];
     SItem& d = a.it[i];
     ItemPlan pl;
-    if (!plan_item(s.T, s.g, COLS, &pl)) return BITNET_ERR_UNSUPPORTED_SHAPE;
+    if (!plan_item(s.T, s.g, COLS, F, &pl)) return BITNET_ERR_UNSUPPORTED_SHAPE;
     d.packed = s.packed;
     d.x = s.x;
     d.q = s.q;
@@ -831,7 +839,7 @@ int launch_run(const Tl2Linear* items, int n, int card, Shape shape, cudaStream_
   a.code_bytes = (int)code;
   a.card = card;
   a.tile_bytes = (F && n > 0) ? (int)(items[0].g.block_bytes / items[0].g.tiles3) : SLOT;
-  const size_t smem = smem_of(a.tmax, code, shape.depth);
+  const size_t smem = smem_of(a.tmax, code, shape.depth, F);
   if (smem > (size_t)dev_info().max_smem_optin) return BITNET_ERR_UNSUPPORTED_SHAPE;
   const int G = CW / a.S;
   int grid = dev_info().sm_count;
@@ -849,7 +857,7 @@ bool item_supported(int T, int64_t M, int64_t K, const TlGeom& g) {
   if (g.tiles2 > 2 || g.three_k > 0x3fffffff) return false;    // more pair tiles than a ring refill pattern assumes
   ItemPlan pl;
   Shape sh;
-  return plan_item(T, g, F ? 64 : 96, &pl) && launch_shape(pl.t3, T, pl.code, M / 32, &sh);
+  return plan_item(T, g, F ? 64 : 96, F, &pl) && launch_shape(pl.t3, T, pl.code, M / 32, F, &sh);
 }
 
 // Launches the scan kernel over `n` supported items of one format (and, F = 1, one cardinality and tile size): as
@@ -868,13 +876,13 @@ int launch_items(const Tl2Linear* items, int64_t n, int card, cudaStream_t st) {
     while (j < n && j - i < NLARGE) {
       const TlGeom& g = items[j].g;
       ItemPlan pl;
-      if (!plan_item(items[j].T, g, COLS, &pl)) return BITNET_ERR_UNSUPPORTED_SHAPE;
+      if (!plan_item(items[j].T, g, COLS, F, &pl)) return BITNET_ERR_UNSUPPORTED_SHAPE;
       const int64_t add = (items[j].M / 32) * (g.tiles3 + g.tiles2);
       const int tm = items[j].T > tmax ? items[j].T : tmax;
       const size_t cm = pl.code > code ? pl.code : code;
       const int t3 = pl.t3 < t3_min ? pl.t3 : t3_min;
       Shape sj;
-      const bool fits = launch_shape(t3, tm, cm, units, &sj);
+      const bool fits = launch_shape(t3, tm, cm, units, F, &sj);
       if (!fits && j == i) return BITNET_ERR_UNSUPPORTED_SHAPE;
       if (!fits || (j > i && w + add > (1ll << 30))) break;
       w += add;
