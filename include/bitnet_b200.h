@@ -172,7 +172,7 @@ int bitnet_mpgemm(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
  *   x[T][K] fp32 in; q[T][K] int8 and act_scale[T] fp32 are OUTPUTS (the quantised activations, as
  *   bitnet_quant_act would give them); y[T][M] fp32 out; acc_out nullable; workspace as for
  *   bitnet_mpgemm.
- * For I2_S with T <= 8 (and T*(K+16) up to 144 KiB) this is ONE kernel: every CTA of the decode kernel
+ * For I2_S with T <= 8 (and T*(K+64) up to 144 KiB) this is ONE kernel: every CTA of the decode kernel
  * quantises the activation rows itself while its first weight tiles are in flight.  Exception: with 6 or
  * more tokens, or more than 96 KiB of codes (T * K padded to 256), and a workspace of the size
  * bitnet_mpgemm_workspace_bytes reports, the stand-alone quantiser and the mid-batch kernel run instead

@@ -60,6 +60,10 @@ __device__ __forceinline__ int quant4(const float4& v, float s) {
   return (quant1(v.x, s) & 255) | ((quant1(v.y, s) & 255) << 8) | ((quant1(v.z, s) & 255) << 16) |
          ((quant1(v.w, s) & 255) << 24);
 }
+// Where word r (four columns) of a staged activation row lies in the I2_S decode kernels: within every 256-column
+// chunk the 16-byte pieces are kept as [piece p][lane quarter t] instead of [t][p], so that the four quarters' loads
+// of one piece (and, with a row stride of 64 bytes modulo 128, the rows of two tokens) cover the 32 banks exactly once.
+__device__ __forceinline__ int staged_word(int r) { return (r & ~63) | ((r & 12) << 2) | ((r & 48) >> 2) | (r & 3); }
 __device__ __forceinline__ float absmax4(const float4& v) {
   return fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
 }

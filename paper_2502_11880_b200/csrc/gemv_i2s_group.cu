@@ -73,11 +73,6 @@ __device__ __forceinline__ bool same_input(const GItem& p, const GItem& d) {
          (d.x ? p.x == d.x : (p.x == nullptr && p.q == d.q && p.act_scale == d.act_scale));
 }
 
-// Where word r (four columns) of a staged row lies: within every 256-column chunk the 16-byte pieces are kept as
-// [piece p][lane quarter t] instead of [t][p], so that the four quarters' loads of one piece (and, with the row
-// stride of 64 bytes modulo 128, the rows of two tokens) cover the 32 banks exactly once.
-__device__ __forceinline__ int staged_word(int r) { return (r & ~63) | ((r & 12) << 2) | ((r & 48) >> 2) | (r & 3); }
-
 // Stages the activation codes of the item's columns [256 c0, 256 c1) (T rows, qst bytes apart, zero beyond K) and,
 // per token, the scale and the sum of the staged codes.  `first` = the item's first part: the row maximum is taken
 // (Alg. 1 Phase 1) and, in the CTA that owns the item, codes and scales of the WHOLE row go to the caller; later

@@ -82,9 +82,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
   int* red = reinterpret_cast<int*>(smem + 2048);              // [CW][2][T][16] partial sums
   const int kp = a.nchunks * 256;
   int8_t* qs_mem = reinterpret_cast<int8_t*>(smem + 2048 + red_bytes(a.T));
-  // Token rows are kp + 16 bytes apart: the B loads of one MMA pair read 16 bytes of every token at the same
-  // column, and rows a multiple of 128 bytes apart would all hit the same shared-memory banks.
-  const int qst = kp + 16;
+  // Token rows are kp + 64 bytes apart and the 16-byte pieces of a chunk are kept [piece][lane quarter]
+  // (staged_word): the B loads of one MMA pair -- the four lane quarters of every token at the same piece -- then
+  // cover the 32 shared-memory banks exactly once per eight lanes.
+  const int qst = kp + 64;
   uint8_t* rings = reinterpret_cast<uint8_t*>(qs_mem) + (((size_t)a.T * qst + 127) & ~(size_t)127);
 
   const int lane = threadIdx.x & 31;
@@ -190,7 +191,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
         const int i = threadIdx.x + r * THREADS;
         if (r < nrow && i < kp / 4) {
           const int word = quant4_packed(xv[r], sq);          // columns K..Kp-1 came in as zeros
-          reinterpret_cast<int*>(qs_mem + tok * qst)[i] = word;
+          reinterpret_cast<int*>(qs_mem + tok * qst)[staged_word(i)] = word;
           if (blockIdx.x == 0 && a.q_out && i < n4) reinterpret_cast<int*>(a.q_out + (int64_t)tok * a.K)[i] = word;
         }
       }
@@ -233,7 +234,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
           word = quant4(__ldcg(x4 + i), sq);
           if (blockIdx.x == 0 && a.q_out) reinterpret_cast<int*>(a.q_out + (int64_t)tok * a.K)[i] = word;
         }
-        reinterpret_cast<int*>(qs_mem + tok * qst)[i] = word;
+        reinterpret_cast<int*>(qs_mem + tok * qst)[staged_word(i)] = word;
       }
     }
   } else {
@@ -252,11 +253,11 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
 #pragma unroll
     for (int r = 0; r < QREG; ++r) {
       const int i = threadIdx.x + r * THREADS;
-      if (i < total4) reinterpret_cast<int*>(qs_mem + (i / (kp / 4)) * qst)[i % (kp / 4)] = qv[r];
+      if (i < total4) reinterpret_cast<int*>(qs_mem + (i / (kp / 4)) * qst)[staged_word(i % (kp / 4))] = qv[r];
     }
     for (int i = threadIdx.x + QREG * THREADS; i < total4; i += THREADS) {
       const int tok = i / (kp / 4), col = i - tok * (kp / 4);
-      reinterpret_cast<int*>(qs_mem + tok * qst)[col] = (col < nq4) ? __ldcg(reinterpret_cast<const int*>(a.q + (int64_t)tok * a.K) + col) : 0;
+      reinterpret_cast<int*>(qs_mem + tok * qst)[staged_word(col)] = (col < nq4) ? __ldcg(reinterpret_cast<const int*>(a.q + (int64_t)tok * a.K) + col) : 0;
     }
     if (threadIdx.x < a.T) qscale[threadIdx.x] = my_scale;
   }
@@ -283,7 +284,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
   }
   // token g's codes under this lane's 16-byte weight column: 64 bytes per chunk
   const unsigned has_tok = g < a.T ? 1u : 0u;
-  const uint32_t q_lane = smem_u32(qs_mem + min(g, a.T - 1) * qst + c_lo * 256 + t * 64);
+  const uint32_t q_lane = smem_u32(qs_mem + min(g, a.T - 1) * qst + c_lo * 256 + t * 16);
   const int bar_id = 1 + gi, bar_threads = a.S * 32;
 
   // One step: wait for the oldest chunk of the ring, put it through the tensor cores, then refill its slot
@@ -309,9 +310,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_wring_kernel(const WArgs 
       asm volatile(
           "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %9, 0;\n\t"
           "@p ld.shared.v4.u32 {%0,%1,%2,%3}, [%8];\n\t"
-          "@p ld.shared.v4.u32 {%4,%5,%6,%7}, [%8+16];\n\t}"
+          "@p ld.shared.v4.u32 {%4,%5,%6,%7}, [%8+64];\n\t}"
           : "+r"(qr[0]), "+r"(qr[1]), "+r"(qr[2]), "+r"(qr[3]), "+r"(qr[4]), "+r"(qr[5]), "+r"(qr[6]), "+r"(qr[7])
-          : "r"(qp + h * 32), "r"(has_tok));
+          : "r"(qp + h * 128), "r"(has_tok));
 #pragma unroll
       for (int s = 0; s < 4; ++s) {
         const unsigned m = 0x03030303u << (2 * s);
@@ -415,7 +416,7 @@ bool make_plan(int T, int64_t M, int64_t K, Plan* p) {
   p->nchunks = (int)(i2s_kp(K) / 256);
   const int forced = tuning().depth;
   int depth = (forced == 12 || forced == 8 || forced == 6 || forced == 4) ? forced : 8;
-  while (depth > 4 && 2048 + red_bytes(T) + (((size_t)T * (p->nchunks * 256 + 16) + 127) & ~(size_t)127) +
+  while (depth > 4 && 2048 + red_bytes(T) + (((size_t)T * (p->nchunks * 256 + 64) + 127) & ~(size_t)127) +
                               (size_t)CW * depth * 1024 > (size_t)dev_info().max_smem_optin)
     depth -= 2;
   if (depth == 10) depth = 8;
@@ -430,7 +431,7 @@ bool make_plan(int T, int64_t M, int64_t K, Plan* p) {
   p->nunits = (int)ceil_div(M, 16);
   const int ctas = dev_info().sm_count * tuning().ctas;
   p->grid = ctas < p->nunits ? ctas : p->nunits;
-  const size_t qs_bytes = ((size_t)T * (p->nchunks * 256 + 16) + 127) & ~(size_t)127;
+  const size_t qs_bytes = ((size_t)T * (p->nchunks * 256 + 64) + 127) & ~(size_t)127;
   if (qs_bytes > MAX_QS_BYTES) return false;
   p->depth = depth;
   p->smem = 2048 + red_bytes(T) + qs_bytes + (size_t)CW * depth * 1024;
