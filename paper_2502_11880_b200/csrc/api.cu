@@ -119,7 +119,10 @@ int bitnet_device_status(int* status_out) {
   int c = 0;
   rc = gemv_tl_status(&c);
   if (rc) return rc;
-  *status_out = a ? a : (b ? b : c);
+  int d = 0;
+  rc = gemm_i2s_stream_tc_status(&d);
+  if (rc) return rc;
+  *status_out = a ? a : (b ? b : (c ? c : d));
   return BITNET_OK;
 }
 
@@ -129,6 +132,8 @@ int bitnet_device_status_clear(void) {
   int rc = gemv_i2s_stream_status_clear();
   if (rc) return rc;
   rc = gemm_prefill_status_clear();
+  if (rc) return rc;
+  rc = gemm_i2s_stream_tc_status_clear();
   if (rc) return rc;
   return gemv_tl_status_clear();
 }
@@ -435,6 +440,13 @@ int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* strea
     if (d.T <= 8) return gemv_i2s_group_item_supported((int)d.T, d.M, d.K);
     return gemv_i2s_group_item_supported(8, d.M, d.K) && gemv_i2s_group_item_supported((int)d.T - 8, d.M, d.K);
   };
+  // 17 to 64 tokens: the stand-alone quantiser per item, then ONE streaming tensor-core kernel over the run
+  // (BITNET_I2S_STREAM_TC=0: every such item as bitnet_linear)
+  static const bool stream_tc = [] { const char* e = getenv("BITNET_I2S_STREAM_TC"); return !(e && atoi(e) == 0); }();
+  auto takes_tc = [&](const bitnet_group_item_t& d) {
+    return grouped && stream_tc && d.fmt == BITNET_FMT_I2S && d.T > group_max_t && gemm_i2s_stream_tc_item_supported(d.T, d.M, d.K);
+  };
+  static thread_local std::vector<StreamTcLinear> run3;
   static thread_local std::vector<GroupLinear> run;
   static thread_local std::vector<Tl2Linear> run2;
   auto takes2 = [&](const bitnet_group_item_t& d, TlGeom* g) {
@@ -465,6 +477,29 @@ int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* strea
         run2.push_back(scan_item(d.packed, d.x, d.q, d.act_scale, d.y, d.acc_out, d.w_scale, d.T, d.M, d.K, 0, g2));
       }
       int rc = launch_gemv_elut_scan(run2.data(), (int64_t)run2.size(), 3, (cudaStream_t)stream);
+      if (rc) return rc;
+      continue;
+    }
+    if (takes_tc(items[i])) {
+      run3.clear();
+      for (; i < n && takes_tc(items[i]); ++i) {
+        const bitnet_group_item_t& d = items[i];
+        int rc = launch_quant_act(d.x, d.T, d.K, 0, d.q, d.act_scale, nullptr, (cudaStream_t)stream);
+        if (rc) return rc;
+        StreamTcLinear t;
+        t.packed = (const uint8_t*)d.packed;
+        t.q = d.q;
+        t.act_scale = d.act_scale;
+        t.y = d.y;
+        t.acc_out = d.acc_out;
+        t.w_scale = d.w_scale;
+        t.T = (int)d.T;
+        t.M = d.M;
+        t.K = d.K;
+        t.ldy = 0;
+        run3.push_back(t);
+      }
+      int rc = launch_gemm_i2s_stream_tc(run3.data(), (int64_t)run3.size(), (cudaStream_t)stream);
       if (rc) return rc;
       continue;
     }

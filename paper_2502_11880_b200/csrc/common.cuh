@@ -156,6 +156,23 @@ size_t gemv_i2s_mid_workspace_bytes(int T, int64_t M, int64_t K);
 int launch_gemv_i2s_mid(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const int8_t* q,
                         const float* act_scale, int T, float* y, int32_t* acc_out, void* ws, size_t ws_bytes,
                         cudaStream_t st);
+// 9 to 64 tokens over a list of I2_S linears whose codes exist (q, act_scale): the weights streamed once, unpacked
+// into tensor memory, tcgen05 MMAs (gemm_i2s_stream_tc.cu).
+struct StreamTcLinear {
+  const uint8_t* packed;
+  const int8_t* q;
+  const float* act_scale;
+  float* y;
+  int32_t* acc_out;    // nullable
+  float w_scale;
+  int T;
+  int64_t M, K;
+  int64_t ldy;         // elements between the token rows of y / acc_out; 0 = M
+};
+bool gemm_i2s_stream_tc_item_supported(int64_t T, int64_t M, int64_t K);
+int launch_gemm_i2s_stream_tc(const StreamTcLinear* items, int64_t n, cudaStream_t st);
+int gemm_i2s_stream_tc_status(int* out);
+int gemm_i2s_stream_tc_status_clear();
 // Programmatic dependent launch (kernels may start their prologue, and prefetch weights, before the
 // previous kernel in the stream has finished); process-wide switch, on by default.  early_start_enabled(st) is asked
 // once per launch on `st`: it answers no for the first launch after a kernel of this library wrote a packed blob

@@ -1,0 +1,39 @@
+"""17 to 64 tokens per linear through the list call: the streaming tensor-core kernel (weights read once, unpacked
+into tensor memory, tcgen05 MMAs with unsigned codes, sum(q) taken off in the epilogue) against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2502_11880_b200 as bn
+from paper_2502_11880_b200 import synth
+from test_gpu_group import Item, run_group
+
+pytestmark = pytest.mark.gpu
+
+
+def test_stream_tc_one_small_item():
+    items = [Item("i2s", 128, 2048, 17, 800)]
+    run_group(items)
+    items[0].check()
+
+
+def test_stream_tc_ragged_rows_token_counts_and_long_rows():
+    """Rows that are no multiple of the 128-row tile, K with a padded last chunk (K % 256 = 64), 17..64 tokens, a
+    28672-column row, neighbours the other grouped kernels take (1 and 12 tokens) in the same list."""
+    shapes = [(300, 4096, 24), (1000, 8192, 64), (64, 28672, 33), (5, 2112, 40), (129, 3200, 17), (160, 8192, 1),
+              (96, 4096, 12), (2048, 2048, 63)]
+    items = [Item("i2s", M, K, T, 810 + i) for i, (M, K, T) in enumerate(shapes)]
+    run_group(items)
+    for it in items:
+        it.check()
+
+
+def test_stream_tc_many_tiles_per_cta_and_repeat():
+    """More tiles than CTAs (every CTA walks several tiles and both accumulators), run twice in a row."""
+    items = [Item("i2s", 24576, 2048, 32, 830), Item("i2s", 8192, 4096, 48, 831)]
+    rng = np.random.default_rng(3)
+    for _ in range(2):
+        run_group(items)
+        for it in items:
+            it.check(rows=np.sort(rng.choice(it.M, 300, replace=False)))
