@@ -307,8 +307,8 @@ def bench_batched(sw, torch, T, steps, warmup):
     """The same sweep with T tokens per linear (I2_S) through ONE bitnet_linear_group call per step: quantiser +
     mpGEMM + rescale.  Every linear keeps its own weights; the T activation rows of layer 0's four linears are
     reused by all layers.  Up to 8 tokens the whole list is one persistent kernel; 9 to 16 tokens are two items of that
-    kernel per linear (tokens 0..7, then the rest: two launches of 320 items each); beyond that the call runs every item
-    as bitnet_linear (quantiser + mid-batch mma.sync kernel + rescale, three launches per linear)."""
+    kernel per linear (tokens 0..7, then the rest: two launches of 320 items each); 17 to 64 tokens: the quantiser per
+    linear, then one launch of the streaming tcgen05 kernel over all 320 linears."""
     bn, dev = sw.bn, sw.x_dev.device
     nl = len(sw.lin)
     xs = [sw.wl.activations(0, j, T).to(dev) for j in range(nl)]
