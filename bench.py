@@ -307,7 +307,7 @@ def bench_batched(sw, torch, T, steps, warmup):
     """The same sweep with T tokens per linear (I2_S) through ONE bitnet_linear_group call per step: quantiser +
     mpGEMM + rescale.  Every linear keeps its own weights; the T activation rows of layer 0's four linears are
     reused by all layers.  Up to 8 tokens the whole list is one persistent kernel; 9 to 16 tokens are two items of that
-    kernel per linear (tokens 0..7, then the rest: two launches of 320 items each); 17 to 64 tokens: the quantiser per
+    kernel per linear (tokens 0..7, then the rest: two launches of 320 items each); 17 to 128 tokens: the quantiser per
     linear, then one launch of the streaming tcgen05 kernel over all 320 linears."""
     bn, dev = sw.bn, sw.x_dev.device
     nl = len(sw.lin)
@@ -663,7 +663,7 @@ def run_ours(args):
         if not args.skip_batched:
             line["batched_decode"] = {
                 "note": "the same sweep with T tokens per linear, one bitnet_linear_group call per step, inputs resident",
-                "runs": [bench_batched(sw, torch, T, max(3, args.steps // 5), 3) for T in (2, 4, 8, 16, 32, 64)]}
+                "runs": [bench_batched(sw, torch, T, max(3, args.steps // 5), 3) for T in (2, 4, 8, 16, 32, 64, 128)]}
         if world == 1 and not args.skip_cpu:
             # ---- CPU baseline leg: the oracle, as it stands, on one full layer of the sweep for about 10 s on the
             # host cores; its results then check the y the GPU left in device memory

@@ -253,9 +253,9 @@ int bitnet_linear_host_batch(const bitnet_host_linear_t* items, int64_t n, void*
  *   - TL2 and TL1 items with T <= 8 (K a multiple of 4, at least three tiles per row) likewise run in one
  *     persistent kernel per run of up to 340 consecutive items of the same format (the scan kernel, see
  *     bitnet_set_tl2_lookup).
- *   - I2_S items with 17 to 64 tokens and K >= 2048: the stand-alone quantiser per item, then ONE
- *     persistent kernel per run of up to 400 such items that reads every blob once, unpacks the codes into
- *     tensor memory and multiplies on the tcgen05 tensor cores.
+ *   - I2_S items with 17 to 128 tokens and K >= 2048: the stand-alone quantiser per item, then ONE
+ *     persistent kernel per run of up to 400 such items of the same class (up to 64 tokens, 65 to 128) that
+ *     reads every blob once, unpacks the codes into tensor memory and multiplies on the tcgen05 tensor cores.
  *   - Every other item (more tokens, short K) is run by bitnet_linear in list order, with the item's
  *     workspace.
  * Results are identical to calling bitnet_linear per item.  Errors: BITNET_ERR_INVALID_ARG for a null or

@@ -440,7 +440,7 @@ int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* strea
     if (d.T <= 8) return gemv_i2s_group_item_supported((int)d.T, d.M, d.K);
     return gemv_i2s_group_item_supported(8, d.M, d.K) && gemv_i2s_group_item_supported((int)d.T - 8, d.M, d.K);
   };
-  // 17 to 64 tokens: the stand-alone quantiser per item, then ONE streaming tensor-core kernel over the run
+  // 17 to 128 tokens: the stand-alone quantiser per item, then the streaming tensor-core kernel over the run
   // (BITNET_I2S_STREAM_TC=0: every such item as bitnet_linear)
   static const bool stream_tc = [] { const char* e = getenv("BITNET_I2S_STREAM_TC"); return !(e && atoi(e) == 0); }();
   auto takes_tc = [&](const bitnet_group_item_t& d) {

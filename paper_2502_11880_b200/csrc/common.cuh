@@ -156,7 +156,7 @@ size_t gemv_i2s_mid_workspace_bytes(int T, int64_t M, int64_t K);
 int launch_gemv_i2s_mid(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const int8_t* q,
                         const float* act_scale, int T, float* y, int32_t* acc_out, void* ws, size_t ws_bytes,
                         cudaStream_t st);
-// 9 to 64 tokens over a list of I2_S linears whose codes exist (q, act_scale): the weights streamed once, unpacked
+// 9 to 128 tokens over a list of I2_S linears whose codes exist (q, act_scale): the weights streamed once, unpacked
 // into tensor memory, tcgen05 MMAs (gemm_i2s_stream_tc.cu).
 struct StreamTcLinear {
   const uint8_t* packed;

@@ -1,4 +1,4 @@
-// I2_S mpGEMM for 17 to 64 tokens over a list of linears: Alg. 1 Phase 2 with the weights streamed from HBM once
+// I2_S mpGEMM for 17 to 128 tokens over a list of linears: Alg. 1 Phase 2 with the weights streamed from HBM once
 // and multiplied on the fifth-generation tensor cores (tcgen05.mma kind::i8, accumulators in tensor memory).
 //
 //   acc[t,m] = sum_k q[t,k] * w[m,k],   y[t,m] = acc[t,m] * act_scale[t] * w_scale
@@ -25,7 +25,9 @@
 //   * warps 20-23: epilogue -- tcgen05.ld the finished 128 x 64 accumulator, zero it, subtract sum(q), rescale,
 //     store y.
 // Two accumulators (2 x 64 columns) overlap a tile's epilogue with the next tile's MMAs; the A ring takes 12 x 32
-// columns.  What binds is the writers' instruction stream (about 100 per warp and step: 7.6 ms per 100B sweep at any
+// columns.  Items with 65 to 128 tokens run the same kernel with 128-token tiles (template TN = 128: two activation
+// pieces per writer thread and K block, accumulators of 128 columns, 8 stages): 11 ms per 100B sweep against 22 ms
+// for the prefill kernel, which such lists fell to before.  What binds is the writers' instruction stream (about 100 per warp and step: 7.6 ms per 100B sweep at any
 // token count from 17 to 64, against 9.6 to 19.4 ms for the mma.sync kernel of gemv_i2s_mid.cu).  Every mbarrier wait is bounded; a wait that gives up sets a CTA-wide abort flag and the device status
 // word, all roles leave their loops, and the CTA frees its tensor memory before it exits.
 #include <cstdlib>
@@ -38,13 +40,12 @@ namespace bitnet {
 namespace {
 
 constexpr int TILE_M = 128;     // out-features per tile (MMA M, tensor-memory lanes)
-constexpr int TILE_N = 64;      // tokens per tile (MMA N, tensor-memory columns of an accumulator)
+// tokens per tile (MMA N, tensor-memory columns of an accumulator): the kernel template's TN, 64 or 128
 constexpr int KBLK = 128;       // K columns per pipeline stage = one 128-byte swizzle row of int8
-constexpr int STAGES = 12;
+constexpr int MAX_STAGES = 12;               // stages: 12 at 64 tokens, 8 at 128 (tensor memory: 2 TN + 32 stages = 512 columns)
 constexpr int NACC = 2;
-constexpr int A_COL0 = NACC * TILE_N;        // first tensor-memory column of the A ring (32 columns per stage)
-constexpr int TMEM_COLS = 512;               // allocation: 128 + 12 * 32 columns
-constexpr int B_BYTES = TILE_N * KBLK;       // 8 KB per stage
+constexpr int TMEM_COLS = 512;
+constexpr int MAX_N = 128;
 constexpr int WRITER_WARPS = 16;
 constexpr int MMA_WARPS = 4;                 // issuers: warp i takes the steps i, i + 4, ... of a tile
 constexpr int THREADS = (WRITER_WARPS + MMA_WARPS + 4) * 32;   // + 4 epilogue warps
@@ -77,7 +78,7 @@ struct TArgs {
 static_assert(sizeof(TArgs) <= 32764, "kernel parameter limit");
 
 struct __align__(8) Bars {
-  uint64_t full[STAGES], empty[STAGES], tmem_full[NACC], tmem_empty[NACC], qsum_ready[NACC];
+  uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[NACC], tmem_empty[NACC], qsum_ready[NACC];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -120,21 +121,22 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
   return d;
 }
 
-// Instruction descriptor: D = s32, A = u8 (the codes 0, 1, 2), B = s8, both K-major, N = 64, M = 128.
-constexpr uint32_t IDESC = (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(TILE_N >> 3) << 17) |
-                           ((uint32_t)(TILE_M >> 4) << 24);
+// Instruction descriptor: D = s32, A = u8 (the codes 0, 1, 2), B = s8, both K-major, N tokens, M = 128.
+__host__ __device__ constexpr uint32_t idesc_of(int n) {
+  return (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+}
 
 // operand A in tensor memory (lane = row, 8 columns = 32 codes along K), operand B through a descriptor.  The
 // whole warp runs the issuing loop and one elected lane issues (`leader` != 0): with warp-uniform operands the
 // compiler keeps addresses and descriptors in uniform registers instead of moving them there per instruction.
-__device__ __forceinline__ void umma_u8s8_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t accumulate,
-                                             uint32_t leader) {
+__device__ __forceinline__ void umma_u8s8_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate, uint32_t leader) {
   asm volatile(
       "{\n\t.reg .pred p, q;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "setp.ne.b32 q, %5, 0;\n\t"
       "@q tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(IDESC), "r"(accumulate), "r"(leader)
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(leader)
       : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar, uint32_t leader) {
@@ -165,15 +167,22 @@ __device__ __forceinline__ int locate(const TArgs& a, int job) {
   return lo;
 }
 
+template <int TN>
 __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __grid_constant__ TArgs a) {
+  constexpr int TILE_N = TN;
+  constexpr int STAGES = TN == 64 ? 12 : 8;
+  constexpr int A_COL0 = NACC * TILE_N;        // first tensor-memory column of the A ring (32 columns per stage)
+  constexpr int B_BYTES = TILE_N * KBLK;       // 8 or 16 KB per stage
+  constexpr int NP = TN / 64;                  // activation pieces per writer thread and K block (tokens tb, tb + 64)
+  constexpr uint32_t IDESC = idesc_of(TN);
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* tileB = smem;                                   // STAGES x 8 KB
   uint8_t* ringA = smem + STAGES * B_BYTES;                // SLOTS_A x 512 x 16 bytes
   Bars* bars = reinterpret_cast<Bars*>(smem + STAGES * B_BYTES + RING_A_BYTES);
   volatile int* abort_flag = &bars->abort_flag;
-  __shared__ int qsum_s[NACC][TILE_N];                     // sum of a token's codes over K, per accumulator in flight
-  __shared__ float ep_scale[4][TILE_N];                    // epilogue: act_scale[t] * w_scale of the current tile
+  __shared__ int qsum_s[NACC][MAX_N];                      // sum of a token's codes over K, per accumulator in flight
+  __shared__ float ep_scale[4][MAX_N];                     // epilogue: act_scale[t] * w_scale of the current tile
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -243,9 +252,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
       // chunk s of the row: 64 bytes; K block 2s + grp2 = its half grp2 (32 bytes), of which this thread takes 16
       // (rows beyond M read the last row: their sums are never stored)
       const uint8_t* rowp = d.packed + i2s_row_chunk_offset(m < d.M ? m : d.M - 1, 0, kp) + grp2 * 32 + hf * 16;
-      const int8_t* qrow = d.q + (int64_t)(tb < d.T ? tb : 0) * d.K + cb * 16;
-      const bool tok_ok = tb < d.T;
       const int K = d.K;
+      const int8_t* qrow = d.q + (int64_t)(tb < d.T ? tb : 0) * K + cb * 16;
+      const int8_t* qrow2 = d.q + (int64_t)(tb + 64 < d.T ? tb + 64 : 0) * K + cb * 16;   // (TN = 128: the thread's second token)
+      const bool tok_ok = tb < d.T, tok2_ok = NP == 2 && tb + 64 < d.T;
       // the thread's two activation pieces of step s into stage pair stb (zeros beyond T, K), once that pair is free:
       // the stages are released in order, so the later one being free means both are
       auto issue_b = [&](int s, int stb, uint32_t phb) -> bool {
@@ -257,6 +267,13 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(by0 ? src : qrow), "r"(by0) : "memory");
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + B_BYTES), "l"(by1 ? src + KBLK : qrow), "r"(by1)
                      : "memory");
+        if (NP == 2) {                             // tokens 64..127 lie 8 row groups (8 KB) further down the tile
+          const uint32_t cy0 = (tok2_ok && col + 16 <= K) ? 16u : 0u, cy1 = (tok2_ok && col + KBLK + 16 <= K) ? 16u : 0u;
+          const int8_t* src2 = qrow2 + 2 * s * KBLK;
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + 8192), "l"(cy0 ? src2 : qrow), "r"(cy0) : "memory");
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + B_BYTES + 8192), "l"(cy1 ? src2 + KBLK : qrow), "r"(cy1)
+                       : "memory");
+        }
         return true;
       };
       // prologue: packed words of the first DA steps (slots slot .. slot + DA - 1); activation pieces of the first DB
@@ -274,7 +291,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
         if (ok && p < nsteps) ok = issue_b(p, stb, phb);
         cp_commit();
       }
-      int qs = 0;
+      int qs = 0, qs2 = 0;
       const uint8_t* pa = rowp + (int64_t)DA * 1024;   // packed words of step s + DA
       for (int s = 0; s < nsteps && ok; ++s, pa += 1024) {
         if (s + DB < nsteps) {
@@ -302,6 +319,19 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
           qs = __dp4a((int)b1.y, 0x01010101, qs);
           qs = __dp4a((int)b1.z, 0x01010101, qs);
           qs = __dp4a((int)b1.w, 0x01010101, qs);
+        }
+        if (NP == 2) {
+          uint4 b0, b1;
+          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b0.x), "=r"(b0.y), "=r"(b0.z), "=r"(b0.w) : "r"(tile_b + st0 * B_BYTES + 8192));
+          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b1.x), "=r"(b1.y), "=r"(b1.z), "=r"(b1.w) : "r"(tile_b + (st0 + 1) * B_BYTES + 8192));
+          qs2 = __dp4a((int)b0.x, 0x01010101, qs2);
+          qs2 = __dp4a((int)b0.y, 0x01010101, qs2);
+          qs2 = __dp4a((int)b0.z, 0x01010101, qs2);
+          qs2 = __dp4a((int)b0.w, 0x01010101, qs2);
+          qs2 = __dp4a((int)b1.x, 0x01010101, qs2);
+          qs2 = __dp4a((int)b1.y, 0x01010101, qs2);
+          qs2 = __dp4a((int)b1.z, 0x01010101, qs2);
+          qs2 = __dp4a((int)b1.w, 0x01010101, qs2);
         }
         {
           // 64 codes of the row in K order = 16 tensor-memory columns: columns 4 c4 .. 4 c4 + 3 take the words
@@ -342,6 +372,12 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
       qs += __shfl_xor_sync(0xffffffffu, qs, 2);
       qs += __shfl_xor_sync(0xffffffffu, qs, 4);
       if (cb == 0) qsum_s[nt % NACC][tb] = qs;
+      if (NP == 2) {
+        qs2 += __shfl_xor_sync(0xffffffffu, qs2, 1);
+        qs2 += __shfl_xor_sync(0xffffffffu, qs2, 2);
+        qs2 += __shfl_xor_sync(0xffffffffu, qs2, 4);
+        if (cb == 0) qsum_s[nt % NACC][tb + 64] = qs2;
+      }
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->qsum_ready[nt % NACC]);
     }
@@ -375,7 +411,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
 #pragma unroll
           for (int k4 = 0; k4 < 2 * (KBLK / 32); ++k4)   // 32 bytes further along K: +2 in the address field, +8 columns
             umma_u8s8_ta(d_tmem, tmem_base + A_COL0 + st * 32 + 8 * k4, bdesc + (uint64_t)((k4 >> 2) * (B_BYTES >> 4) + 2 * (k4 & 3)),
-                         1u, leader);
+                         IDESC, 1u, leader);
           umma_commit(&bars->empty[st + 1], leader);   // the pair is reusable once these MMAs have read it
         }
         if (!ok) break;
@@ -434,8 +470,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
         }
       }
       // the accumulator and the sums have been read: clear it and hand the buffer back
-      zero32(taddr);
-      zero32(taddr + 32);
+#pragma unroll
+      for (int c0 = 0; c0 < TILE_N; c0 += 32) zero32(taddr + c0);
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
@@ -456,18 +492,40 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
 // Shapes the kernel takes: 9 to 64 tokens; rows long enough that a tile's K blocks outnumber the ring by far (the
 // hand-over of the per-token sums between tiles relies on it).
 bool gemm_i2s_stream_tc_item_supported(int64_t T, int64_t M, int64_t K) {
-  return T >= 9 && T <= TILE_N && M >= 1 && M <= 0x7fffffff && K >= 2048 && (K % 64) == 0 && K <= 0x3fffffff;
+  return T >= 9 && T <= MAX_N && M >= 1 && M <= 0x7fffffff && K >= 2048 && (K % 64) == 0 && K <= 0x3fffffff;
 }
 
+namespace {
+template <int TN>
+int launch_tn(const TArgs& a, int grid, cudaStream_t st) {
+  constexpr int STAGES = TN == 64 ? 12 : 8;
+  const size_t smem = (size_t)STAGES * TN * KBLK + RING_A_BYTES + sizeof(Bars) + 1024;
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (!attr_set[dev & 63]) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_i2s_stream_tc_kernel<TN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return note_cuda_error(e);
+    attr_set[dev & 63] = true;
+  }
+  gemm_i2s_stream_tc_kernel<TN><<<grid, THREADS, smem, st>>>(a);
+  return check_launch();
+}
+}  // namespace
+
+// One launch per run of up to NITEMS items whose token counts fall into the same class (up to 64: 64-token tiles;
+// 65 to 128: 128-token tiles).
 int launch_gemm_i2s_stream_tc(const StreamTcLinear* items, int64_t n, cudaStream_t st) {
   static thread_local TArgs a;      // 26 KB: off the stack
-  for (int64_t i0 = 0; i0 < n; i0 += NITEMS) {
-    const int cnt = (int)((n - i0 < NITEMS) ? n - i0 : NITEMS);
+  for (int64_t i0 = 0; i0 < n;) {
+    const bool wide = items[i0].T > 64;
+    int cnt = 0;
     int64_t tiles = 0;
-    for (int i = 0; i < cnt; ++i) {
-      const StreamTcLinear& s = items[i0 + i];
+    while (i0 + cnt < n && cnt < NITEMS && (items[i0 + cnt].T > 64) == wide) {
+      const StreamTcLinear& s = items[i0 + cnt];
       if (!gemm_i2s_stream_tc_item_supported(s.T, s.M, s.K)) return BITNET_ERR_UNSUPPORTED_SHAPE;
-      TItem& d = a.it[i];
+      if (tiles + ceil_div(s.M, TILE_M) > 0x3fffffff) break;
+      TItem& d = a.it[cnt];
       d.packed = s.packed;
       d.q = s.q;
       d.act_scale = s.act_scale;
@@ -480,25 +538,17 @@ int launch_gemm_i2s_stream_tc(const StreamTcLinear* items, int64_t n, cudaStream
       d.first_tile = (int)tiles;
       d.ldy = (int)(s.ldy ? s.ldy : s.M);
       tiles += ceil_div(s.M, TILE_M);
-      if (tiles > 0x3fffffff) return BITNET_ERR_UNSUPPORTED_SHAPE;
+      ++cnt;
     }
+    if (cnt == 0) return BITNET_ERR_UNSUPPORTED_SHAPE;
     a.n = cnt;
     a.total_tiles = (int)tiles;
-    const size_t smem = (size_t)STAGES * B_BYTES + RING_A_BYTES + sizeof(Bars) + 1024;
-    static bool attr_set[64] = {false};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (!attr_set[dev & 63]) {
-      cudaError_t e = cudaFuncSetAttribute(gemm_i2s_stream_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e != cudaSuccess) return note_cuda_error(e);
-      attr_set[dev & 63] = true;
-    }
     int grid = dev_info().sm_count;
     if (grid > tiles) grid = (int)tiles;
-    log_launch("gemm_i2s_stream_tc_kernel items=%d tiles=%lld grid=%d", cnt, (long long)tiles, grid);
-    gemm_i2s_stream_tc_kernel<<<grid, THREADS, smem, st>>>(a);
-    int rc = check_launch();
+    log_launch("gemm_i2s_stream_tc_kernel<%d> items=%d tiles=%lld grid=%d", wide ? 128 : 64, cnt, (long long)tiles, grid);
+    const int rc = wide ? launch_tn<128>(a, grid, st) : launch_tn<64>(a, grid, st);
     if (rc) return rc;
+    i0 += cnt;
   }
   return BITNET_OK;
 }

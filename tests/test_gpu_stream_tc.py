@@ -1,4 +1,4 @@
-"""17 to 64 tokens per linear through the list call: the streaming tensor-core kernel (weights read once, unpacked
+"""17 to 128 tokens per linear through the list call: the streaming tensor-core kernel (weights read once, unpacked
 into tensor memory, tcgen05 MMAs with unsigned codes, sum(q) taken off in the epilogue) against the CPU oracle."""
 import numpy as np
 import pytest
@@ -37,3 +37,14 @@ def test_stream_tc_many_tiles_per_cta_and_repeat():
         run_group(items)
         for it in items:
             it.check(rows=np.sort(rng.choice(it.M, 300, replace=False)))
+
+
+def test_stream_tc_sixty_five_to_128_tokens():
+    """The 128-token tile variant (two activation pieces per writer thread and K block, 8 stages), mixed with
+    64-token items in one list (separate launches per class), ragged rows and a long row."""
+    shapes = [(128, 2048, 65), (300, 4096, 100), (1000, 8192, 128), (64, 28672, 77), (129, 3200, 33), (2048, 2048, 127),
+              (96, 4096, 128)]
+    items = [Item("i2s", M, K, T, 850 + i) for i, (M, K, T) in enumerate(shapes)]
+    run_group(items)
+    for it in items:
+        it.check()
