@@ -310,6 +310,28 @@ int bitnet_mpgemm(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
   if (fmt == BITNET_FMT_I2S) {
     int rc = i2s_shape(M, K);
     if (rc) return rc;
+    // A single tensor with enough 128-row tiles for the SMs: the streaming tcgen05 kernel (weights read once, codes
+    // unpacked into tensor memory).  Measured crossovers on 100B- and 8B-shaped tensors: 33 to 64 tokens from two
+    // thirds of a tile per SM on (72 against 112 us at 57344 x 8192, 18 against 32 at 14336 x 4096); 65 to 128 tokens
+    // from two tiles per SM on (104 against 121 us); up to 32 tokens the mma.sync kernel is as fast or faster on one
+    // tensor (lists are another matter: bitnet_linear_group).
+    static const bool stream_tc = [] { const char* e = getenv("BITNET_I2S_STREAM_TC"); return !(e && atoi(e) == 0); }();
+    const int64_t tiles128 = ceil_div(M, 128), sms = dev_info().sm_count;
+    if (stream_tc && gemm_i2s_stream_tc_item_supported(T, M, K) &&
+        ((T >= 33 && T <= 64 && tiles128 * 3 >= sms * 2) || (T >= 65 && T <= 128 && tiles128 >= sms * 2))) {
+      StreamTcLinear t;
+      t.packed = (const uint8_t*)packed;
+      t.q = q;
+      t.act_scale = act_scale;
+      t.y = y;
+      t.acc_out = acc_out;
+      t.w_scale = w_scale;
+      t.T = (int)T;
+      t.M = M;
+      t.K = K;
+      t.ldy = 0;
+      return launch_gemm_i2s_stream_tc(&t, 1, st);
+    }
     // 9 to 64 tokens (and crowded decode batches): the weight scan on mma.sync; the prefill (or decode) kernel
     // takes the call when the caller's workspace is smaller than bitnet_mpgemm_workspace_bytes asked for
     if (mid_takes(T, M, K, workspace, workspace_bytes))

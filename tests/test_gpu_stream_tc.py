@@ -48,3 +48,22 @@ def test_stream_tc_sixty_five_to_128_tokens():
     run_group(items)
     for it in items:
         it.check()
+
+
+def test_stream_tc_serves_large_single_calls():
+    """bitnet_mpgemm / bitnet_linear on one tensor with many 128-row tiles and 33 to 128 tokens take the same kernel
+    (sampled rows against the oracle); the same call with the switch off must give identical bits."""
+    from helpers import check_y, npy
+    for M, K, T in [(14336, 4096, 48), (40000, 2048, 100)]:
+        w = synth.ternary(870, 1, M, K, 1 / 3, 1 / 3)
+        x = synth.normal(871, T, T, K)
+        blob = bn.pack("i2s", w.cuda())
+        y, q, sc, acc = bn.bitnet_linear("i2s", blob, 0.5, M, K, x.cuda(), want_acc=True)
+        torch.cuda.synchronize()
+        rows = np.sort(np.random.default_rng(7).choice(M, 400, replace=False))
+        q_ref, sc_ref, _ = oracle.quant_act(x.numpy())
+        assert np.array_equal(npy(q), q_ref)
+        acc_ref = oracle.mpgemm_def(q_ref, np.ascontiguousarray(w.numpy()[rows]))
+        assert np.array_equal(npy(acc)[:, rows], acc_ref)
+        check_y(y[:, torch.as_tensor(rows).cuda()], acc_ref, sc_ref, 0.5)
+    assert bn.bitnet_device_status() == 0
