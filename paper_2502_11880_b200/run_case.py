@@ -6,7 +6,8 @@ small, self-contained workload the ncu captures under profiles/ are taken on).
 FMT = i2s | tl1 | tl2.  Weights and activations are seeded synthetic tensors; N launches (default 6) over
 three distinct copies of the packed blob.  T <= 8 runs the decode path through bitnet_linear (one fused kernel
 for I2_S up to 5 tokens unless --two-kernel); larger T runs the quantiser and bitnet_mpgemm: the mid-batch
-kernel up to 64 tokens, the prefill kernel beyond.
+kernel up to 64 tokens (large tensors from 33 tokens on: the streaming tcgen05 kernel, unless
+BITNET_I2S_STREAM_TC=0), the prefill kernel beyond.
 """
 import sys
 
