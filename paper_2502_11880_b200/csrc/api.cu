@@ -454,12 +454,18 @@ int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* strea
     }
   }
   static const bool grouped = [] { const char* e = getenv("BITNET_GROUP"); return !(e && atoi(e) == 0); }();
-  // 9 to 16 tokens: two passes of the grouped kernel (tokens 0..7, then the rest) beat the mid-batch kernel's
-  // launch per linear on lists (6.4 against 8.4 ms on the 100B sweep at 16 tokens); BITNET_GROUP_MAX_T lowers the limit.
+  // 9 to 16 tokens: the grouped kernel's two-group form (every A register feeds an MMA per group of eight tokens;
+  // the weights cross HBM once); BITNET_GROUP_WIDE=0 or a shape that form does not take: two items of the
+  // one-group kernel (tokens 0..7, then the rest), which still beat the mid-batch kernel's launch per linear on
+  // lists (5.5 against 8.4 ms on the 100B sweep at 16 tokens).  BITNET_GROUP_MAX_T lowers the limit.
+  static const bool group_wide = [] { const char* e = getenv("BITNET_GROUP_WIDE"); return !(e && atoi(e) == 0); }();
   static const int group_max_t = [] { const char* e = getenv("BITNET_GROUP_MAX_T"); const int v = e ? atoi(e) : 16; return v < 8 ? 8 : (v > 16 ? 16 : v); }();
   auto takes = [&](const bitnet_group_item_t& d) {
     if (!grouped || d.fmt != BITNET_FMT_I2S || d.T > group_max_t) return false;
-    if (d.T <= 8) return gemv_i2s_group_item_supported((int)d.T, d.M, d.K);
+    if (d.T <= 8 || group_wide) {
+      if (gemv_i2s_group_item_supported((int)d.T, d.M, d.K)) return true;
+      if (d.T <= 8) return false;
+    }
     return gemv_i2s_group_item_supported(8, d.M, d.K) && gemv_i2s_group_item_supported((int)d.T - 8, d.M, d.K);
   };
   // 17 to 128 tokens: the stand-alone quantiser per item, then the streaming tensor-core kernel over the run
@@ -469,6 +475,7 @@ int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* strea
     return grouped && stream_tc && d.fmt == BITNET_FMT_I2S && d.T > group_max_t && gemm_i2s_stream_tc_item_supported(d.T, d.M, d.K);
   };
   static thread_local std::vector<StreamTcLinear> run3;
+  static thread_local std::vector<QuantListItem> qrun;
   static thread_local std::vector<GroupLinear> run;
   static thread_local std::vector<Tl2Linear> run2;
   auto takes2 = [&](const bitnet_group_item_t& d, TlGeom* g) {
@@ -504,10 +511,12 @@ int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* strea
     }
     if (takes_tc(items[i])) {
       run3.clear();
+      qrun.clear();
       for (; i < n && takes_tc(items[i]); ++i) {
         const bitnet_group_item_t& d = items[i];
-        int rc = launch_quant_act(d.x, d.T, d.K, 0, d.q, d.act_scale, nullptr, (cudaStream_t)stream);
-        if (rc) return rc;
+        if (qrun.empty() || qrun.back().x != d.x || qrun.back().q != d.q || qrun.back().act_scale != d.act_scale ||
+            qrun.back().K != d.K || qrun.back().T != (int)d.T)
+          qrun.push_back(QuantListItem{d.x, d.q, d.act_scale, d.K, (int)d.T});
         StreamTcLinear t;
         t.packed = (const uint8_t*)d.packed;
         t.q = d.q;
@@ -521,7 +530,9 @@ int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* strea
         t.ldy = 0;
         run3.push_back(t);
       }
-      int rc = launch_gemm_i2s_stream_tc(run3.data(), (int64_t)run3.size(), (cudaStream_t)stream);
+      int rc = launch_quant_act_list(qrun.data(), (int64_t)qrun.size(), (cudaStream_t)stream);   // the codes of the whole run
+      if (rc) return rc;
+      rc = launch_gemm_i2s_stream_tc(run3.data(), (int64_t)run3.size(), (cudaStream_t)stream);
       if (rc) return rc;
       continue;
     }
@@ -534,6 +545,7 @@ int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* strea
       continue;
     }
     run.clear();
+    qrun.clear();
     for (; i < n && takes(items[i]); ++i) {
       const bitnet_group_item_t& d = items[i];
       GroupLinear gl;
@@ -544,12 +556,21 @@ int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* strea
       gl.y = d.y;
       gl.acc_out = d.acc_out;
       gl.w_scale = d.w_scale;
-      gl.T = (int)(d.T > 8 ? 8 : d.T);
+      const bool split = d.T > 8 && !(group_wide && gemv_i2s_group_item_supported((int)d.T, d.M, d.K));
+      gl.T = (int)(split ? 8 : d.T);
       gl.M = d.M;
       gl.K = d.K;
       gl.ldy = 0;
+      if (d.T > 8 && !split) {
+        // 9 to 16 tokens in one item: the codes come from one quantiser launch over all such items of the run (a CTA
+        // of the grouped kernel would quantise 16 rows per linear it touches: more L2 reads than weight bytes)
+        if (qrun.empty() || qrun.back().x != d.x || qrun.back().q != d.q || qrun.back().act_scale != d.act_scale ||
+            qrun.back().K != d.K || qrun.back().T != (int)d.T)
+          qrun.push_back(QuantListItem{d.x, d.q, d.act_scale, d.K, (int)d.T});
+        gl.x = nullptr;
+      }
       run.push_back(gl);
-      if (d.T > 8) {                       // the remaining tokens: a second item over the same weights
+      if (split) {                         // the remaining tokens: a second item over the same weights
         gl.x = d.x + 8 * d.K;
         gl.q = d.q + 8 * d.K;
         gl.act_scale = d.act_scale + 8;
@@ -558,6 +579,10 @@ int bitnet_linear_group(const bitnet_group_item_t* items, int64_t n, void* strea
         gl.T = (int)d.T - 8;
         run.push_back(gl);
       }
+    }
+    if (!qrun.empty()) {
+      int rc = launch_quant_act_list(qrun.data(), (int64_t)qrun.size(), (cudaStream_t)stream);
+      if (rc) return rc;
     }
     int rc = launch_gemv_i2s_group(run.data(), (int64_t)run.size(), (cudaStream_t)stream);
     if (rc) return rc;

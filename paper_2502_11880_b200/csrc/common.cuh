@@ -81,6 +81,15 @@ const DevInfo& dev_info();
 // ---- kernel launchers (one per .cu file) ----------------------------------------------------
 int launch_quant_act(const float* x, int64_t T, int64_t K, int per_tensor, int8_t* q, float* act_scale,
                      int32_t* act_sum, cudaStream_t st);
+// per-token quantiser over a list of matrices x[T][K] -> q[T][K], act_scale[T], in one launch per 800 matrices
+struct QuantListItem {
+  const float* x;
+  int8_t* q;
+  float* act_scale;
+  int64_t K;
+  int T;
+};
+int launch_quant_act_list(const QuantListItem* items, int64_t n, cudaStream_t st);
 int launch_pack_i2s(const int8_t* w, int64_t M, int64_t K, uint8_t* packed, int* dev_status,
                     cudaStream_t st);
 int launch_unpack_i2s(const uint8_t* packed, int64_t M, int64_t K, int8_t* w, int* dev_status,

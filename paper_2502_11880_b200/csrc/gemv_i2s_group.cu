@@ -68,6 +68,10 @@ struct GArgs {
 };
 static_assert(sizeof(GArgs<NSMALL>) <= 4096 && sizeof(GArgs<NLARGE>) <= 32764, "kernel parameter limits");
 
+// bytes of the kernel's shared-memory header (range, per-token scales, sums and partial maxima) for batches of up to
+// `tmax` tokens
+__host__ __device__ constexpr int header_bytes(int tmax) { return tmax > 8 ? 2048 : 1024; }
+
 __device__ __forceinline__ bool same_input(const GItem& p, const GItem& d) {
   return p.nparts == 1 && d.nparts == 1 && p.K == d.K && p.T == d.T &&
          (d.x ? p.x == d.x : (p.x == nullptr && p.q == d.q && p.act_scale == d.act_scale));
@@ -77,11 +81,12 @@ __device__ __forceinline__ bool same_input(const GItem& p, const GItem& d) {
 // per token, the scale and the sum of the staged codes.  `first` = the item's first part: the row maximum is taken
 // (Alg. 1 Phase 1) and, in the CTA that owns the item, codes and scales of the WHOLE row go to the caller; later
 // parts reuse the multiplier kept in qmul.  Called by all threads; contains barriers.
+template <int NT>
 __device__ __forceinline__ void stage_item(const GItem& d, bool owner, bool first, int c0, int c1, int qst, int8_t* qs_mem,
                                            float* qscale, float* qmul, int* qsum, float* qred) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int n4 = d.K / 4, w0 = c0 * 64, w1 = c1 * 64;       // staged words [w0, w1) of a row
-  if (threadIdx.x < 8) qsum[threadIdx.x] = 0;
+  if (threadIdx.x < 8 * NT) qsum[threadIdx.x] = 0;
   if (d.x && first && d.K <= 4 * XREG * THREADS) {
     // one round trip per token: s = 127 / max(amax, 1e-5), q = clamp(rint(x * s)); the row stays in registers
     const int kw = (int)(i2s_kp(d.K) / 4);
@@ -176,15 +181,19 @@ __device__ __forceinline__ void stage_item(const GItem& d, bool owner, bool firs
       if (lane == 0) atomicAdd(qsum + tok, s);
     }
   } else {
-    // given codes
+    // given codes: 16 at a time (K % 64 == 0 and the parts begin on chunks: a row's words come in whole fours, and
+    // staged_word keeps four consecutive words together)
     __syncthreads();  // qsum is zero before the first atomicAdd
     for (int tok = 0; tok < d.T; ++tok) {
-      const int* qrow = reinterpret_cast<const int*>(d.q + (int64_t)tok * d.K);
+      const int4* qrow = reinterpret_cast<const int4*>(d.q + (int64_t)tok * d.K);
       int s = 0;
-      for (int i = w0 + threadIdx.x; i < w1; i += THREADS) {
-        const int word = (i < n4) ? __ldcg(qrow + i) : 0;
-        reinterpret_cast<int*>(qs_mem + tok * qst)[staged_word(i - w0)] = word;
-        s = __dp4a(word, 0x01010101, s);
+      for (int i = w0 / 4 + threadIdx.x; i < w1 / 4; i += THREADS) {
+        const int4 v = (4 * i < n4) ? __ldcg(qrow + i) : make_int4(0, 0, 0, 0);
+        *reinterpret_cast<int4*>(reinterpret_cast<int*>(qs_mem + tok * qst) + staged_word(4 * i - w0)) = v;
+        s = __dp4a(v.x, 0x01010101, s);
+        s = __dp4a(v.y, 0x01010101, s);
+        s = __dp4a(v.z, 0x01010101, s);
+        s = __dp4a(v.w, 0x01010101, s);
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
@@ -194,16 +203,19 @@ __device__ __forceinline__ void stage_item(const GItem& d, bool owner, bool firs
   }
 }
 
-template <int DEPTH, int NMAX>
+// NT = groups of eight tokens an item may have (1: up to 8 tokens; 2: up to 16 -- every A register then feeds two
+// MMAs, one per group, and the weights of a 9-to-16-token batch still cross HBM once).
+template <int DEPTH, int NMAX, int NT>
 __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid_constant__ GArgs<NMAX> a) {
   extern __shared__ __align__(128) uint8_t smem[];
+  constexpr int HB = header_bytes(8 * NT);
   int* hdr = reinterpret_cast<int*>(smem);             // [0] first unit, [1] end unit, [2] first item, [3] last item
-  float* qscale = reinterpret_cast<float*>(smem + 64);  // [8] act_scale per token
-  int* qsum = reinterpret_cast<int*>(smem + 96);        // [8] sum of the staged codes per token
-  float* qred = reinterpret_cast<float*>(smem + 128);   // [8][16] partial maxima
-  float* qmul = reinterpret_cast<float*>(smem + 640);   // [8] 127 / amax per token
-  int* red = reinterpret_cast<int*>(smem + 1024);       // [CW][2][tmax][16] partial sums
-  int8_t* qs_mem = reinterpret_cast<int8_t*>(smem + 1024 + CW * 2 * a.tmax * 16 * 4);
+  float* qscale = reinterpret_cast<float*>(smem + 64);            // [8 NT] act_scale per token
+  int* qsum = reinterpret_cast<int*>(smem + 64 + 32 * NT);        // [8 NT] sum of the staged codes per token
+  float* qred = reinterpret_cast<float*>(smem + 64 + 64 * NT);    // [8 NT][16] partial maxima
+  float* qmul = reinterpret_cast<float*>(smem + 64 + 576 * NT);   // [8 NT] 127 / amax per token
+  int* red = reinterpret_cast<int*>(smem + HB);                   // [CW][2][tmax][16] partial sums
+  int8_t* qs_mem = reinterpret_cast<int8_t*>(smem + HB + CW * 2 * a.tmax * 16 * 4);
   uint8_t* rings = reinterpret_cast<uint8_t*>(qs_mem) + a.code_bytes;
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -305,7 +317,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
     const bool owner = jb <= d.first_unit;
     const int jlo = range_lo(ci), jhi = range_hi(ci);
     const int first = d.first_unit, M = d.M, ldy = d.ldy;
-    const unsigned has_tok = g < T ? 1u : 0u;
+    const unsigned has_tok = g < T ? 1u : 0u, has_tok2 = g + 8 < T ? 1u : 0u;
     const float w_scale = d.w_scale;
     float* const y = d.y;
     int32_t* const acc_out = d.acc_out;
@@ -313,7 +325,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
       const int c0 = part * nch / nparts, c1 = (part + 1) * nch / nparts, npc = c1 - c0;
       if (!staged_any || part > 0 || !same_input(a.it[ci - 1], d)) {
         if (staged_any) __syncthreads();  // everyone is done with the codes staged before (and with y as scratch)
-        stage_item(d, owner, part == 0, c0, c1, qst, qs_mem, qscale, qmul, qsum, qred);
+        stage_item<NT>(d, owner, part == 0, c0, c1, qst, qs_mem, qscale, qmul, qsum, qred);
         __syncthreads();
         staged_any = true;
       } else if (owner && d.x && d.q != a.it[ci - 1].q) {
@@ -325,16 +337,22 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
       }
       const int s_lo = wk * npc / S, nw = (wk + 1) * npc / S - s_lo;
       const uint32_t q_lane = smem_u32(qs_mem + min(g, T - 1) * qst + s_lo * 256 + t * 16);
+      const uint32_t q_grp2 = (uint32_t)((min(g + 8, T - 1) - min(g, T - 1)) * qst);   // (NT = 2) on to token g + 8
       const bool last_part = part + 1 == nparts;
 
       for (int cj = jlo; cj < jhi; cj += G, ++nloc) {
-        int C[4][4];
+        int C[NT][4][4];
+        int qr[NT][8];                         // B registers; lanes beyond the batch keep their zeros
 #pragma unroll
-        for (int s = 0; s < 4; ++s)
+        for (int n = 0; n < NT; ++n) {
 #pragma unroll
-          for (int i = 0; i < 4; ++i) C[s][i] = 0;
+          for (int s = 0; s < 4; ++s)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) C[n][s][i] = 0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) qr[n][i] = 0;
+        }
         uint32_t qp = q_lane;
-        int qr[8] = {0, 0, 0, 0, 0, 0, 0, 0};  // B registers; lanes beyond the batch keep these zeros
         // One step: wait for the oldest chunk of the ring, put it through the tensor cores, then refill its slot
         // from `pf` (the chunk DEPTH places further down the warp's stream), if there is one.
         auto step = [&](const uint8_t* pf, bool do_pf) {
@@ -353,12 +371,23 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
                 "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %9, 0;\n\t"
                 "@p ld.shared.v4.u32 {%0,%1,%2,%3}, [%8];\n\t"
                 "@p ld.shared.v4.u32 {%4,%5,%6,%7}, [%8+64];\n\t}"
-                : "+r"(qr[0]), "+r"(qr[1]), "+r"(qr[2]), "+r"(qr[3]), "+r"(qr[4]), "+r"(qr[5]), "+r"(qr[6]), "+r"(qr[7])
+                : "+r"(qr[0][0]), "+r"(qr[0][1]), "+r"(qr[0][2]), "+r"(qr[0][3]), "+r"(qr[0][4]), "+r"(qr[0][5]), "+r"(qr[0][6]),
+                  "+r"(qr[0][7])
                 : "r"(qp + h * 128), "r"(has_tok));
+            if (NT == 2)
+              asm volatile(
+                  "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %9, 0;\n\t"
+                  "@p ld.shared.v4.u32 {%0,%1,%2,%3}, [%8];\n\t"
+                  "@p ld.shared.v4.u32 {%4,%5,%6,%7}, [%8+64];\n\t}"
+                  : "+r"(qr[NT - 1][0]), "+r"(qr[NT - 1][1]), "+r"(qr[NT - 1][2]), "+r"(qr[NT - 1][3]), "+r"(qr[NT - 1][4]),
+                    "+r"(qr[NT - 1][5]), "+r"(qr[NT - 1][6]), "+r"(qr[NT - 1][7])
+                  : "r"(qp + q_grp2 + h * 128), "r"(has_tok2));
 #pragma unroll
             for (int s = 0; s < 4; ++s) {
               const unsigned m = 0x03030303u << (2 * s);
-              mma_u8s8(C[s], w4[2 * h] & m, v4[2 * h] & m, w4[2 * h + 1] & m, v4[2 * h + 1] & m, qr[2 * s], qr[2 * s + 1]);
+              const unsigned a0 = w4[2 * h] & m, a1 = v4[2 * h] & m, a2 = w4[2 * h + 1] & m, a3 = v4[2 * h + 1] & m;
+#pragma unroll
+              for (int n = 0; n < NT; ++n) mma_u8s8(C[n][s], a0, a1, a2, a3, qr[n][2 * s], qr[n][2 * s + 1]);
             }
           }
           qp += 256;
@@ -383,17 +412,22 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
         cur = nxt;
 
         // fragment: c[0] = (row g, token 2t), c[1] = (row g, token 2t+1), c[2], c[3] = the same for row g+8
-        int c[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) c[i] = C[0][i] + (C[1][i] >> 2) + (C[2][i] >> 4) + (C[3][i] >> 6);
+        // (token group n: the tokens 8 n + 2t, 8 n + 2t + 1)
         int* mine = red + ((warp * 2 + (nloc & 1)) * tmax) * 16;
-        if (2 * t < T) {
-          mine[(2 * t) * 16 + g] = c[0];
-          mine[(2 * t) * 16 + g + 8] = c[2];
-        }
-        if (2 * t + 1 < T) {
-          mine[(2 * t + 1) * 16 + g] = c[1];
-          mine[(2 * t + 1) * 16 + g + 8] = c[3];
+#pragma unroll
+        for (int n = 0; n < NT; ++n) {
+          int c[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) c[i] = C[n][0][i] + (C[n][1][i] >> 2) + (C[n][2][i] >> 4) + (C[n][3][i] >> 6);
+          const int tk = 8 * n + 2 * t;
+          if (tk < T) {
+            mine[tk * 16 + g] = c[0];
+            mine[tk * 16 + g + 8] = c[2];
+          }
+          if (tk + 1 < T) {
+            mine[(tk + 1) * 16 + g] = c[1];
+            mine[(tk + 1) * 16 + g + 8] = c[3];
+          }
         }
         if (S > 1) group_barrier(1 + gi, S * 32);
         else __syncwarp();
@@ -403,7 +437,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
           const int row0 = (cj - first) * 16;
           const int* grp = red + (((gi * S) * 2 + (nloc & 1)) * tmax) * 16;
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
+          for (int i = 0; i < 4 * NT; ++i) {
             const int idx = lane + 32 * i;
             if (idx < T * 16) {
               int v = 0;
@@ -474,7 +508,7 @@ Shape shape_for(int64_t nch, int64_t units) {
 }
 
 size_t smem_of(int tmax, size_t code_bytes, int depth) {
-  return 1024 + (size_t)CW * 2 * tmax * 16 * 4 + code_bytes + (size_t)CW * depth * 1024;
+  return (size_t)header_bytes(tmax) + (size_t)CW * 2 * tmax * 16 * 4 + code_bytes + (size_t)CW * depth * 1024;
 }
 
 // How one item is walked: in `nparts` parts of its K (as few as let the staged codes of a part, T rows of at most
@@ -486,11 +520,11 @@ struct ItemPlan {
   int64_t npc;
 };
 bool plan_item(int T, int64_t M, int64_t K, ItemPlan* out) {
-  if (T < 1 || T > 8 || M < 1 || K < 1 || (K % 64) != 0 || M > 0x7fffffff) return false;
+  if (T < 1 || T > 16 || M < 1 || K < 1 || (K % 64) != 0 || M > 0x7fffffff) return false;
   const int64_t nch = i2s_kp(K) / 256;
   const size_t cap = (size_t)dev_info().max_smem_optin;
   for (int want_depth = 6; want_depth >= 4; want_depth -= 2)
-    for (int n = 1; n <= 8; ++n) {
+    for (int n = 1; n <= 16; ++n) {
       const int64_t big = ceil_div(nch, n), small = nch / n;
       if (small < 4) break;
       const size_t code = ((size_t)T * (size_t)(big * 256 + 64) + 127) & ~(size_t)127;
@@ -502,13 +536,13 @@ bool plan_item(int T, int64_t M, int64_t K, ItemPlan* out) {
   return false;
 }
 
-template <int DEPTH, int NMAX>
+template <int DEPTH, int NMAX, int NT>
 int launch_group(const GArgs<NMAX>& a, int grid, size_t smem, cudaStream_t st) {
   static bool attr_set[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
   if (!attr_set[dev & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(gemv_i2s_group_kernel<DEPTH, NMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(gemv_i2s_group_kernel<DEPTH, NMAX, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          dev_info().max_smem_optin);
     if (e != cudaSuccess) return note_cuda_error(e);
     attr_set[dev & 63] = true;
@@ -523,17 +557,17 @@ int launch_group(const GArgs<NMAX>& a, int grid, size_t smem, cudaStream_t st) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = early_start_enabled(st) ? 1 : 0;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_i2s_group_kernel<DEPTH, NMAX>, a);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_i2s_group_kernel<DEPTH, NMAX, NT>, a);
   return e == cudaSuccess ? BITNET_OK : note_cuda_error(e);
 }
 
-template <int NMAX>
+template <int NMAX, int NT>
 int launch_depth(const GArgs<NMAX>& a, int depth, int grid, size_t smem, cudaStream_t st) {
   switch (depth) {
-    case 4: return launch_group<4, NMAX>(a, grid, smem, st);
-    case 6: return launch_group<6, NMAX>(a, grid, smem, st);
-    case 8: return launch_group<8, NMAX>(a, grid, smem, st);
-    case 12: return launch_group<12, NMAX>(a, grid, smem, st);
+    case 4: return launch_group<4, NMAX, NT>(a, grid, smem, st);
+    case 6: return launch_group<6, NMAX, NT>(a, grid, smem, st);
+    case 8: return launch_group<8, NMAX, NT>(a, grid, smem, st);
+    case 12: return launch_group<12, NMAX, NT>(a, grid, smem, st);
     default: return BITNET_ERR_UNSUPPORTED_SHAPE;
   }
 }
@@ -596,7 +630,11 @@ int launch_run(const GroupLinear* items, int n, Shape shape, cudaStream_t st) {
   if ((int64_t)grid * G > units) grid = (int)ceil_div(units, G);
   log_launch("gemv_i2s_group_kernel items=%d units=%lld chunks=%lld grid=%d warps/unit=%d ring=%d tmax=%d smem=%zu", n,
              (long long)units, (long long)w, grid, a.S, depth, a.tmax, smem);
-  return launch_depth<NMAX>(a, depth, grid, smem, st);
+  if (a.tmax > 8) {                        // 9 to 16 tokens: the two-group kernel, built for the large block only
+    if (NMAX != NLARGE) return BITNET_ERR_UNSUPPORTED_SHAPE;
+    return launch_depth<NMAX, NMAX == NLARGE ? 2 : 1>(a, depth, grid, smem, st);
+  }
+  return launch_depth<NMAX, 1>(a, depth, grid, smem, st);
 }
 
 }  // namespace
@@ -618,8 +656,10 @@ int launch_gemv_i2s_group(const GroupLinear* items, int64_t n, cudaStream_t st) 
     size_t code = 0;
     Shape sh{1, 4};
     int64_t units = 0;
-    for (int64_t k = i; k < n && k - i < NLARGE; ++k) units += ceil_div(items[k].M, 16);   // (an estimate when the run is cut short)
-    while (j < n && j - i < NLARGE) {
+    const bool wide = items[i].T > 8;      // a launch holds items of one class: up to 8 tokens, or 9 to 16
+    for (int64_t k = i; k < n && k - i < NLARGE && (items[k].T > 8) == wide; ++k)
+      units += ceil_div(items[k].M, 16);   // (an estimate when the run is cut short)
+    while (j < n && j - i < NLARGE && (items[j].T > 8) == wide) {
       ItemPlan pl;
       if (!plan_item(items[j].T, items[j].M, items[j].K, &pl)) return BITNET_ERR_UNSUPPORTED_SHAPE;
       const int64_t add = ceil_div(items[j].M, 16) * (i2s_kp(items[j].K) / 256);
@@ -638,7 +678,7 @@ int launch_gemv_i2s_group(const GroupLinear* items, int64_t n, cudaStream_t st) 
       ++j;
     }
     const int cnt = (int)(j - i);
-    const int rc = cnt <= NSMALL ? launch_run<NSMALL>(items + i, cnt, sh, st) : launch_run<NLARGE>(items + i, cnt, sh, st);
+    const int rc = (cnt <= NSMALL && !wide) ? launch_run<NSMALL>(items + i, cnt, sh, st) : launch_run<NLARGE>(items + i, cnt, sh, st);
     if (rc != BITNET_OK) return rc;
     i = j;
   }

@@ -299,6 +299,48 @@ cudaError_t launch_reg(const float* x, int64_t T, int64_t K, int8_t* q, float* a
   return cudaLaunchKernelEx(&cfg, quant_act_reg_kernel<NT>, x, K, q, act_scale, act_sum);
 }
 
+// The rows of a LIST of activation matrices in one launch (Alg. 1 Phase 1 for every linear of a grouped call whose
+// kernel wants the codes ready): one CTA per row, the row's matrix found by a binary search over the items' first
+// rows.  Same operations in the same order as quant_act_kernel: the bytes are identical.
+constexpr int QLIST_ITEMS = 800;
+struct QListEntry {
+  const float* x;
+  int8_t* q;
+  float* act_scale;
+  int K, first_row;
+};
+struct QListArgs {
+  int n, rows;
+  QListEntry it[QLIST_ITEMS];
+};
+static_assert(sizeof(QListArgs) <= 32764, "kernel parameter limit");
+
+__global__ void __launch_bounds__(QTHREADS) quant_act_list_kernel(const __grid_constant__ QListArgs a) {
+  __shared__ float red[32];
+  const int tid = threadIdx.x;
+  if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  int lo = 0, hi = a.n - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (a.it[mid].first_row <= (int)blockIdx.x) lo = mid; else hi = mid - 1;
+  }
+  const QListEntry& d = a.it[lo];
+  const int64_t t = (int)blockIdx.x - d.first_row, K = d.K;
+  const float* xr = d.x + t * K;
+  int8_t* qr = d.q + t * K;
+  const float amax_c = fmaxf(block_amax(xr, K, red), 1e-5f);
+  const float s = __fdiv_rn(127.0f, amax_c);
+  if ((K & 3) == 0 && ((reinterpret_cast<uintptr_t>(xr) & 15u) == 0) && ((reinterpret_cast<uintptr_t>(qr) & 3u) == 0)) {
+    const float4* x4 = reinterpret_cast<const float4*>(xr);
+    int* q4 = reinterpret_cast<int*>(qr);
+    for (int64_t i = tid; i < K / 4; i += blockDim.x) q4[i] = quant4_packed(__ldcg(x4 + i), s);
+  } else {
+    for (int64_t i = tid; i < K; i += blockDim.x) qr[i] = (int8_t)quant1(__ldcg(xr + i), s);
+  }
+  if (tid == 0) d.act_scale[t] = __fdiv_rn(amax_c, 127.0f);
+}
+
 __global__ void fill_scale_kernel(float* act_scale, int64_t T) {
   __shared__ float sc;
   if (threadIdx.x == 0) {
@@ -310,6 +352,38 @@ __global__ void fill_scale_kernel(float* act_scale, int64_t T) {
 }
 
 }  // namespace
+
+int launch_quant_act_list(const QuantListItem* items, int64_t n, cudaStream_t st) {
+  static thread_local QListArgs a;   // 19 KB: off the stack
+  for (int64_t i0 = 0; i0 < n;) {
+    int cnt = 0;
+    int64_t rows = 0;
+    while (i0 + cnt < n && cnt < QLIST_ITEMS && rows + items[i0 + cnt].T <= 0x3fffffff) {
+      const QuantListItem& s = items[i0 + cnt];
+      if (!s.x || !s.q || !s.act_scale || s.T < 1 || s.K < 1 || s.K > 0x7fffffff) return BITNET_ERR_INVALID_ARG;
+      a.it[cnt] = QListEntry{s.x, s.q, s.act_scale, (int)s.K, (int)rows};
+      rows += s.T;
+      ++cnt;
+    }
+    if (cnt == 0) return BITNET_ERR_INVALID_ARG;
+    a.n = cnt;
+    a.rows = (int)rows;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)rows);
+    cfg.blockDim = dim3(QTHREADS);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = early_start_enabled(st) ? 1 : 0;
+    log_launch("quant_act_list_kernel items=%d rows=%lld", cnt, (long long)rows);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, quant_act_list_kernel, a);
+    if (e != cudaSuccess) return note_cuda_error(e);
+    i0 += cnt;
+  }
+  return check_launch();
+}
 
 int launch_quant_act(const float* x, int64_t T, int64_t K, int per_tensor, int8_t* q, float* act_scale,
                      int32_t* act_sum, cudaStream_t st) {

@@ -67,15 +67,51 @@ def test_group_small_ragged_list():
         it.check()
 
 
-def test_group_nine_to_sixteen_tokens_in_two_passes():
-    """Items with 9 to 16 tokens run as two items over the same weights (tokens 0..7, then the rest); ragged rows, a
-    long row walked in parts, neighbours with fewer tokens, and an item with 17 tokens (left to the mid-batch kernel)."""
-    shapes = [(40, 2048, 9), (300, 8192, 16), (33, 28672, 12), (64, 4096, 3), (1000, 3200, 13), (64, 4096, 17),
-              (17, 1536, 10)]
-    items = [Item("i2s", M, K, T, 150 + i) for i, (M, K, T) in enumerate(shapes)]
+WIDE_SHAPES = [(40, 2048, 9), (300, 8192, 16), (33, 28672, 12), (64, 4096, 3), (1000, 3200, 13), (64, 4096, 17),
+               (17, 1536, 10), (2000, 1024, 11), (160, 28672, 16), (48, 16384, 14), (16, 8192, 15), (640, 4096, 8)]
+
+
+def test_group_nine_to_sixteen_tokens():
+    """Items with 9 to 16 tokens run through the grouped kernel's two-group form (launches of their own, between those
+    of the neighbours with up to 8 tokens): every token count, ragged rows, long rows walked in parts, an item with 17
+    tokens (left to the streaming or mid-batch kernel) in between."""
+    items = [Item("i2s", M, K, T, 150 + i) for i, (M, K, T) in enumerate(WIDE_SHAPES)]
     run_group(items)
     for it in items:
         it.check()
+
+
+def test_group_nine_to_sixteen_tokens_shared_input_and_many_units():
+    """Two-group form: linears that share their input (quantised once per CTA, codes stored per item), and enough units
+    that every warp takes whole units and walks several of them."""
+    x = synth.normal(170, 3, 12, 4096)
+    items = [Item("i2s", 4096, 4096, 12, 171, x=x), Item("i2s", 1024, 4096, 12, 172, x=x), Item("i2s", 11008, 4096, 12, 173, x=x),
+             Item("i2s", 40000, 2048, 16, 174)]
+    items[1].xd = items[2].xd = items[0].xd
+    run_group(items)
+    for it in items:
+        it.check(rows=np.unique(np.concatenate([[0, 15, 16, it.M - 1], np.random.default_rng(it.M).integers(0, it.M, 200)])))
+
+
+def test_group_nine_to_sixteen_tokens_in_two_passes_in_a_child_process():
+    """BITNET_GROUP_WIDE=0 (read once per process): such items run as two items of the one-group kernel over the same
+    weights (tokens 0..7, then the rest)."""
+    import os
+    import subprocess
+    import sys
+    code = (
+        "import sys; sys.path.insert(0, 'tests')\n"
+        "import paper_2502_11880_b200 as bn\n"
+        "from test_gpu_group import Item, run_group, WIDE_SHAPES\n"
+        "items = [Item('i2s', M, K, T, 150 + i) for i, (M, K, T) in enumerate(WIDE_SHAPES)]\n"
+        "run_group(items)\n"
+        "for it in items: it.check()\n"
+        "assert bn.bitnet_device_status() == 0\n"
+        "print('ok')\n")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, "-c", code], cwd=root, env=dict(os.environ, BITNET_GROUP_WIDE="0"), capture_output=True,
+                         text=True, timeout=900)
+    assert out.returncode == 0 and "ok" in out.stdout, out.stderr[-2000:]
 
 
 def test_group_many_units_per_cta_and_shared_inputs():
