@@ -47,12 +47,19 @@ constexpr int NACC = 2;
 constexpr int TMEM_COLS = 512;
 constexpr int MAX_N = 128;
 constexpr int WRITER_WARPS = 16;
-constexpr int MMA_WARPS = 4;                 // issuers: warp i takes the steps i, i + 4, ... of a tile
-constexpr int THREADS = (WRITER_WARPS + MMA_WARPS + 4) * 32;   // + 4 epilogue warps
-constexpr int DA = 8;                        // steps (pairs of K blocks) of packed words in flight per thread
-constexpr int DB = 2;                        // steps by which the activation copies run ahead
-constexpr int SLOTS_A = DA + 1;              // ring slots: the copy for step s + DA never lands in the slot step s reads
-constexpr int RING_A_BYTES = SLOTS_A * WRITER_WARPS * 32 * 16;   // 72 KB: one 16-byte slot per writer thread and step
+constexpr int MMA_WARPS = 4;                 // issuer warps (NISS of them at work: see the kernel)
+constexpr int PRODUCER_WARP = WRITER_WARPS + MMA_WARPS + 4;    // after the 4 epilogue warps
+constexpr int THREADS = (PRODUCER_WARP + 1) * 32;
+// A step = CPS 256-column chunks of a tile's rows (2 CPS K blocks = 2 CPS stages): two chunks per step at 64-token
+// tiles (12 stages = 3 steps in the ring), one at 128-token tiles (8 stages = 4 steps).  Per step a writer thread
+// unpacks 16 bytes of packed words per chunk; the waits, fences and barrier arrivals are paid once per step.
+__host__ __device__ constexpr int cps_of(int tn) { return tn == 64 ? 2 : 1; }
+// slots of the packed-word ring = steps the producer runs ahead (8 chunks of the tile's 128 rows either way: 64 KB)
+__host__ __device__ constexpr int da_of(int tn) { return 8 / cps_of(tn); }
+__host__ __device__ constexpr int ring_a_bytes(int tn) { return da_of(tn) * cps_of(tn) * 8192; }
+constexpr int MAX_SLOTS_A = 8;
+// steps by which the activation copies run ahead (the stages they go to must have been read by the MMAs)
+__host__ __device__ constexpr int db_of(int tn) { return tn == 64 ? 1 : 2; }
 constexpr int NITEMS = 400;                  // items per launch (argument block of 32 KB)
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
@@ -68,23 +75,36 @@ struct TItem {
   int M, K, T;
   int first_tile;         // tiles of the items before this one
   int ldy;
+  int64_t first_w;        // steps of the tiles of the items before this one (the measure of work the CTAs share)
 };
-static_assert(sizeof(TItem) == 64, "argument block layout");
+static_assert(sizeof(TItem) == 72, "argument block layout");
 
 struct TArgs {
   int n, total_tiles;
+  int64_t total_w;
   TItem it[NITEMS];
 };
 static_assert(sizeof(TArgs) <= 32764, "kernel parameter limit");
 
 struct __align__(8) Bars {
   uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[NACC], tmem_empty[NACC], qsum_ready[NACC];
+  uint64_t a_full[MAX_SLOTS_A], a_empty[MAX_SLOTS_A];   // packed-word ring: bytes landed / slot read by every writer warp
   uint32_t tmem_base;
   int abort_flag;
 };
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// bulk asynchronous copy global -> shared (16-byte aligned, a multiple of 16 bytes), bytes counted on `bar`
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint64_t* bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+      ::"r"(dst), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol)
+      : "memory");
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -167,10 +187,35 @@ __device__ __forceinline__ int locate(const TArgs& a, int job) {
   return lo;
 }
 
+// steps of one tile of an item with K columns
+__host__ __device__ __forceinline__ int steps_of(int K, int cps) { return (int)((i2s_kp(K) / 256 + cps - 1) / cps); }
+
+// first tile (of the list's tile sequence) whose first step lies at or after position w of the list's step sequence
+__device__ __forceinline__ int tile_at(const TArgs& a, int64_t w, int cps) {
+  if (w >= a.total_w) return a.total_tiles;
+  int lo = 0, hi = a.n - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (a.it[mid].first_w <= w) lo = mid; else hi = mid - 1;
+  }
+  const int ns = steps_of(a.it[lo].K, cps);
+  return a.it[lo].first_tile + (int)((w - a.it[lo].first_w + ns - 1) / ns);
+}
+
 template <int TN>
 __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __grid_constant__ TArgs a) {
   constexpr int TILE_N = TN;
   constexpr int STAGES = TN == 64 ? 12 : 8;
+  constexpr int CPS = cps_of(TN), GST = 2 * CPS;   // chunks and stages per step
+  constexpr int DA = da_of(TN), DB = db_of(TN), SLOTS_A = DA;
+  constexpr uint32_t SLOT_BYTES = CPS * 8192;      // a step's packed words of the tile: 8 units x CPS KB
+  constexpr int RING_A_BYTES = ring_a_bytes(TN);
+  // Issuers at work: as many as the ring holds steps, issuer i taking the steps i, i + NISS, ... of the CTA's whole
+  // step sequence (counted across tiles), i.e. always the same stages.  A wait for a barrier's phase k is only
+  // meaningful once phase k - 1 is known to be complete (a barrier still in phase k - 1 answers "done" to a probe
+  // for the parity of k); an issuer that meets every phase of its own barriers in order knows that.
+  constexpr int NISS = STAGES / GST;
+  static_assert(NISS <= MMA_WARPS, "an issuer warp per step of the ring");
   constexpr int A_COL0 = NACC * TILE_N;        // first tensor-memory column of the A ring (32 columns per stage)
   constexpr int B_BYTES = TILE_N * KBLK;       // 8 or 16 KB per stage
   constexpr int NP = TN / 64;                  // activation pieces per writer thread and K block (tokens tb, tb + 64)
@@ -185,14 +230,24 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
   __shared__ float ep_scale[4][MAX_N];                     // epilogue: act_scale[t] * w_scale of the current tile
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // this CTA's tiles: a contiguous range of the list's tile sequence holding an equal share of its steps (a CTA
+  // then meets few items, and the per-token sums of an item are taken once per CTA, not once per tile)
+  const int jb = tile_at(a, a.total_w * blockIdx.x / gridDim.x, CPS);
+  const int je = tile_at(a, a.total_w * (blockIdx.x + 1) / gridDim.x, CPS);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(&bars->full[s], WRITER_WARPS);   // every writer warp: its pieces of B, and of A where it has some
+      // a step's last stage: every writer warp once its codes are in tensor memory, and every writer thread's
+      // asynchronous arrival once its activation pieces have landed
+      mbar_init(&bars->full[s], WRITER_WARPS + WRITER_WARPS * 32);
       mbar_init(&bars->empty[s], 1);             // tcgen05.commit (used on the odd stages: one per stage pair)
     }
+    for (int sl = 0; sl < SLOTS_A; ++sl) {
+      mbar_init(&bars->a_full[sl], 1);           // the producer's arrival with the byte count
+      mbar_init(&bars->a_empty[sl], WRITER_WARPS);
+    }
     for (int b = 0; b < NACC; ++b) {
-      mbar_init(&bars->tmem_full[b], MMA_WARPS); // one tcgen05.commit per issuer
+      mbar_init(&bars->tmem_full[b], NISS);      // one tcgen05.commit per issuer at work
       mbar_init(&bars->tmem_empty[b], 4);        // one arrival per epilogue warp
       mbar_init(&bars->qsum_ready[b], WRITER_WARPS);
     }
@@ -218,7 +273,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
         ::"r"(taddr), "r"(0u)
         : "memory");
   };
-  if (warp >= WRITER_WARPS + MMA_WARPS) {
+  if (warp >= WRITER_WARPS + MMA_WARPS && warp < PRODUCER_WARP) {
     for (int c0 = 0; c0 < NACC * TILE_N; c0 += 32) zero32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + c0);
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
   }
@@ -234,112 +289,123 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
     const int r = quarter * 32 + lane;
     const int tb = threadIdx.x >> 3, cb = threadIdx.x & 7;   // activation piece: token, 16-byte piece of the 128-byte row
     const uint32_t b_off = (uint32_t)((tb >> 3) * 1024 + (tb & 7) * 128 + ((cb ^ (tb & 7)) << 4));
-    const uint32_t ring_a = smem_u32(ringA) + threadIdx.x * 16;
+    // this thread's 16 bytes of a chunk in a ring slot: the slot holds the tile's 8 units, CPS KB each, as the blob does
+    const uint32_t ring_a = smem_u32(ringA) + (r >> 4) * (CPS * 1024) + (r & 15) * 64 + grp2 * 32 + hf * 16;
     const uint32_t tile_b = smem_u32(tileB) + b_off;
-    // Running positions instead of divisions: st0 = stage of the current step's first K block (even; its second K
-    // block sits in st0 + 1), ph = how often the stage ring has been passed (mod 2), slot = the step's ring slot.
+    // Running positions instead of divisions: st0 = first stage of the current step (a multiple of GST), ph = how
+    // often the stage ring has been passed (mod 2), slot = the step's ring slot.
     int st0 = 0, slot = 0;
-    uint32_t ph = 0;
-    constexpr uint32_t SLOT_BYTES = WRITER_WARPS * 32 * 16;
+    uint32_t ph = 0, pha = 0;                      // (pha: passes of the packed-word ring, mod 2)
     uint32_t nt = 0;
     bool ok = true;
-    for (int job = blockIdx.x; ok && job < a.total_tiles && !*abort_flag; job += gridDim.x, ++nt) {
-      const int ii = locate(a, job);
+    int ii = jb < je ? locate(a, jb) : 0, prev_item = -1;
+    int qtot = 0, qtot2 = 0;                       // sums of the codes of this thread's tokens over K, current item
+    for (int job = jb; ok && job < je && !*abort_flag; ++job, ++nt) {
+      while (ii + 1 < a.n && a.it[ii + 1].first_tile <= job) ++ii;
       const TItem& d = a.it[ii];
+      const bool need_q = ii != prev_item;         // first tile of the item in this CTA: take the sums of the codes
+      prev_item = ii;
       const int64_t kp = i2s_kp(d.K);
-      const int nsteps = (int)(kp / 256);          // a step = the two K blocks of a 256-column chunk
-      const int m = (job - d.first_tile) * TILE_M + r;
-      // chunk s of the row: 64 bytes; K block 2s + grp2 = its half grp2 (32 bytes), of which this thread takes 16
-      // (rows beyond M read the last row: their sums are never stored)
-      const uint8_t* rowp = d.packed + i2s_row_chunk_offset(m < d.M ? m : d.M - 1, 0, kp) + grp2 * 32 + hf * 16;
+      const int nch = (int)(kp / 256), nsteps = (nch + CPS - 1) / CPS;
+      // chunk c of a row: 64 bytes; K block 2c + grp2 = its half grp2 (32 bytes), of which this thread takes 16
       const int K = d.K;
+      const int nfull = K / (GST * KBLK);          // steps whose K blocks all lie inside K
       const int8_t* qrow = d.q + (int64_t)(tb < d.T ? tb : 0) * K + cb * 16;
       const int8_t* qrow2 = d.q + (int64_t)(tb + 64 < d.T ? tb + 64 : 0) * K + cb * 16;   // (TN = 128: the thread's second token)
-      const bool tok_ok = tb < d.T, tok2_ok = NP == 2 && tb + 64 < d.T;
-      // the thread's two activation pieces of step s into stage pair stb (zeros beyond T, K), once that pair is free:
-      // the stages are released in order, so the later one being free means both are
-      auto issue_b = [&](int s, int stb, uint32_t phb) -> bool {
-        if (!mbar_wait(&bars->empty[stb + 1], phb ^ 1u, abort_flag, 20)) return false;
-        const int col = 2 * s * KBLK + cb * 16;
-        const uint32_t by0 = (tok_ok && col + 16 <= K) ? 16u : 0u, by1 = (tok_ok && col + KBLK + 16 <= K) ? 16u : 0u;
-        const int8_t* src = qrow + 2 * s * KBLK;
+      const uint32_t tok_sz = tb < d.T ? 16u : 0u, tok2_sz = (NP == 2 && tb + 64 < d.T) ? 16u : 0u;
+      // the thread's activation pieces of step s into the stages stb .. stb + GST - 1 (zeros beyond T, K), once they
+      // are free: the stages are released in order, so the last one being free means all are
+      auto issue_b = [&](int s2, int stb, uint32_t phb) -> bool {
+        if (!mbar_wait(&bars->empty[stb + GST - 1], phb ^ 1u, abort_flag, 20)) return false;
         const uint32_t dst = tile_b + stb * B_BYTES;
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(by0 ? src : qrow), "r"(by0) : "memory");
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + B_BYTES), "l"(by1 ? src + KBLK : qrow), "r"(by1)
-                     : "memory");
-        if (NP == 2) {                             // tokens 64..127 lie 8 row groups (8 KB) further down the tile
-          const uint32_t cy0 = (tok2_ok && col + 16 <= K) ? 16u : 0u, cy1 = (tok2_ok && col + KBLK + 16 <= K) ? 16u : 0u;
-          const int8_t* src2 = qrow2 + 2 * s * KBLK;
-          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + 8192), "l"(cy0 ? src2 : qrow), "r"(cy0) : "memory");
-          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + B_BYTES + 8192), "l"(cy1 ? src2 + KBLK : qrow), "r"(cy1)
-                       : "memory");
+        const int8_t* src = qrow + (int64_t)s2 * (GST * KBLK);
+        const int8_t* src2 = qrow2 + (int64_t)s2 * (GST * KBLK);
+        if (s2 < nfull) {
+#pragma unroll
+          for (int j = 0; j < GST; ++j) {
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + j * B_BYTES), "l"(src + j * KBLK), "r"(tok_sz) : "memory");
+            if (NP == 2)                             // tokens 64..127 lie 8 row groups (8 KB) further down the tile
+              asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + j * B_BYTES + 8192), "l"(src2 + j * KBLK), "r"(tok2_sz)
+                           : "memory");
+          }
+        } else {
+          const int col = s2 * (GST * KBLK) + cb * 16;
+#pragma unroll
+          for (int j = 0; j < GST; ++j) {
+            const bool in = col + j * KBLK + 16 <= K;
+            const uint32_t by = in ? tok_sz : 0u;
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + j * B_BYTES), "l"(in ? src + j * KBLK : qrow), "r"(by) : "memory");
+            if (NP == 2) {
+              const uint32_t cy = in ? tok2_sz : 0u;
+              asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + j * B_BYTES + 8192), "l"(in ? src2 + j * KBLK : qrow), "r"(cy)
+                           : "memory");
+            }
+          }
         }
+        // this thread's arrival on the step's barrier, made by the copy unit when the pieces (and every copy issued
+        // before them) have landed: no thread waits for activation bytes, the issuer does
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&bars->full[stb + GST - 1])) : "memory");
         return true;
       };
-      // prologue: packed words of the first DA steps (slots slot .. slot + DA - 1); activation pieces of the first DB
-#pragma unroll
-      for (int p = 0; p < DA; ++p) {
-        const int sl = slot + p >= SLOTS_A ? slot + p - SLOTS_A : slot + p;
-        if (p < nsteps) cp16_keep(ring_a + sl * SLOT_BYTES, rowp + (int64_t)p * 1024);
-      }
-      cp_commit();
+      // prologue: activation pieces of the first DB steps, a copy group per step
 #pragma unroll
       for (int p = 0; p < DB; ++p) {
-        int stb = st0 + 2 * p;
+        int stb = st0 + GST * p;
         uint32_t phb = ph;
         if (stb >= STAGES) stb -= STAGES, phb ^= 1u;
         if (ok && p < nsteps) ok = issue_b(p, stb, phb);
         cp_commit();
       }
       int qs = 0, qs2 = 0;
-      const uint8_t* pa = rowp + (int64_t)DA * 1024;   // packed words of step s + DA
-      for (int s = 0; s < nsteps && ok; ++s, pa += 1024) {
-        if (s + DB < nsteps) {
-          int stb = st0 + 2 * DB;
+      for (int s2 = 0; s2 < nsteps && ok; ++s2) {
+        if (s2 + DB < nsteps) {
+          int stb = st0 + GST * DB;
           uint32_t phb = ph;
           if (stb >= STAGES) stb -= STAGES, phb ^= 1u;
-          ok = issue_b(s + DB, stb, phb);
+          ok = issue_b(s2 + DB, stb, phb);
           if (!ok) break;
         }
-        // step s + DA goes to the slot before this step's (DA = SLOTS_A - 1 places on)
-        if (s + DA < nsteps) cp16_keep(ring_a + (slot ? slot - 1 : SLOTS_A - 1) * SLOT_BYTES, pa);
         cp_commit();
-        cp_wait<DB>();                             // everything but the last DB groups has landed: step s is complete
-        // the landed activation bytes go to the tensor core through the async proxy
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        {
-          uint4 b0, b1;                            // this thread's own pieces, for the row sums
-          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b0.x), "=r"(b0.y), "=r"(b0.z), "=r"(b0.w) : "r"(tile_b + st0 * B_BYTES));
-          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b1.x), "=r"(b1.y), "=r"(b1.z), "=r"(b1.w) : "r"(tile_b + (st0 + 1) * B_BYTES));
-          qs = __dp4a((int)b0.x, 0x01010101, qs);
-          qs = __dp4a((int)b0.y, 0x01010101, qs);
-          qs = __dp4a((int)b0.z, 0x01010101, qs);
-          qs = __dp4a((int)b0.w, 0x01010101, qs);
-          qs = __dp4a((int)b1.x, 0x01010101, qs);
-          qs = __dp4a((int)b1.y, 0x01010101, qs);
-          qs = __dp4a((int)b1.z, 0x01010101, qs);
-          qs = __dp4a((int)b1.w, 0x01010101, qs);
+        // No thread waits for activation bytes (the issuer does, through the step's barrier), except in a tile that
+        // takes the sums of the codes: there the pieces committed DB steps ago are read back.
+        if (need_q) {
+          cp_wait<DB>();
+#pragma unroll
+          for (int j = 0; j < GST; ++j) {
+            uint4 b0;                              // this thread's own pieces, for the row sums
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b0.x), "=r"(b0.y), "=r"(b0.z), "=r"(b0.w) : "r"(tile_b + (st0 + j) * B_BYTES));
+            qs = __dp4a((int)b0.x, 0x01010101, qs);
+            qs = __dp4a((int)b0.y, 0x01010101, qs);
+            qs = __dp4a((int)b0.z, 0x01010101, qs);
+            qs = __dp4a((int)b0.w, 0x01010101, qs);
+            if (NP == 2) {
+              uint4 b1;
+              asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b1.x), "=r"(b1.y), "=r"(b1.z), "=r"(b1.w) : "r"(tile_b + (st0 + j) * B_BYTES + 8192));
+              qs2 = __dp4a((int)b1.x, 0x01010101, qs2);
+              qs2 = __dp4a((int)b1.y, 0x01010101, qs2);
+              qs2 = __dp4a((int)b1.z, 0x01010101, qs2);
+              qs2 = __dp4a((int)b1.w, 0x01010101, qs2);
+            }
+          }
         }
-        if (NP == 2) {
-          uint4 b0, b1;
-          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b0.x), "=r"(b0.y), "=r"(b0.z), "=r"(b0.w) : "r"(tile_b + st0 * B_BYTES + 8192));
-          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b1.x), "=r"(b1.y), "=r"(b1.z), "=r"(b1.w) : "r"(tile_b + (st0 + 1) * B_BYTES + 8192));
-          qs2 = __dp4a((int)b0.x, 0x01010101, qs2);
-          qs2 = __dp4a((int)b0.y, 0x01010101, qs2);
-          qs2 = __dp4a((int)b0.z, 0x01010101, qs2);
-          qs2 = __dp4a((int)b0.w, 0x01010101, qs2);
-          qs2 = __dp4a((int)b1.x, 0x01010101, qs2);
-          qs2 = __dp4a((int)b1.y, 0x01010101, qs2);
-          qs2 = __dp4a((int)b1.z, 0x01010101, qs2);
-          qs2 = __dp4a((int)b1.w, 0x01010101, qs2);
-        }
-        {
+        // the step's packed words have landed (bulk copies of the producer warp); once they are in registers the slot
+        // goes back to the producer.  (A chunk beyond the row's last, or a row beyond M, is not copied: what the
+        // slot holds then meets activation codes that are all zero, or sums that are never stored.)
+        ok = mbar_wait(&bars->a_full[slot], pha, abort_flag, 20);
+        if (!ok) break;
+        uint32_t wa[CPS][4];
+#pragma unroll
+        for (int c = 0; c < CPS; ++c)
+          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                       : "=r"(wa[c][0]), "=r"(wa[c][1]), "=r"(wa[c][2]), "=r"(wa[c][3])
+                       : "r"(ring_a + slot * SLOT_BYTES + c * 1024));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->a_empty[slot]);
+#pragma unroll
+        for (int c = 0; c < CPS; ++c) {
           // 64 codes of the row in K order = 16 tensor-memory columns: columns 4 c4 .. 4 c4 + 3 take the words
           // 2 (c4 / 2), 2 (c4 / 2) + 1 of the 16 packed bytes under the slots 2h, 2h + 1 (h = c4 % 2)
-          uint32_t w[4];
-          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                       : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3])
-                       : "r"(ring_a + slot * SLOT_BYTES));
+          const uint32_t* w = wa[c];
           uint32_t o[16];
 #pragma unroll
           for (int c4 = 0; c4 < 4; ++c4) {
@@ -350,33 +416,39 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
             o[4 * c4 + 2] = (w0 >> (4 * h + 2)) & 0x03030303u;
             o[4 * c4 + 3] = (w1 >> (4 * h + 2)) & 0x03030303u;
           }
-          const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 + (st0 + grp2) * 32 + hf * 16;
+          const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 + (st0 + 2 * c + grp2) * 32 + hf * 16;
           asm volatile(
               "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, "
               "%14, %15, %16};"
               ::"r"(taddr), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]),
                 "r"(o[8]), "r"(o[9]), "r"(o[10]), "r"(o[11]), "r"(o[12]), "r"(o[13]), "r"(o[14]), "r"(o[15])
               : "memory");
-          asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         }
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();
-        if (lane == 0) mbar_arrive(&bars->full[st0 + 1]);   // one barrier per stage pair (the odd stage's)
-        st0 += 2;
+        if (lane == 0) mbar_arrive(&bars->full[st0 + GST - 1]);   // one barrier per step (its last stage's)
+        st0 += GST;
         if (st0 == STAGES) st0 = 0, ph ^= 1u;
-        slot = slot + 1 == SLOTS_A ? 0 : slot + 1;
+        if (++slot == SLOTS_A) slot = 0, pha ^= 1u;
       }
       if (!ok) break;
-      // sum of the codes of token tb over all of K: the 8 threads that carry the token's pieces
-      qs += __shfl_xor_sync(0xffffffffu, qs, 1);
-      qs += __shfl_xor_sync(0xffffffffu, qs, 2);
-      qs += __shfl_xor_sync(0xffffffffu, qs, 4);
-      if (cb == 0) qsum_s[nt % NACC][tb] = qs;
-      if (NP == 2) {
-        qs2 += __shfl_xor_sync(0xffffffffu, qs2, 1);
-        qs2 += __shfl_xor_sync(0xffffffffu, qs2, 2);
-        qs2 += __shfl_xor_sync(0xffffffffu, qs2, 4);
-        if (cb == 0) qsum_s[nt % NACC][tb + 64] = qs2;
+      if (need_q) {
+        // sum of the codes of token tb over all of K: the 8 threads that carry the token's pieces
+        qs += __shfl_xor_sync(0xffffffffu, qs, 1);
+        qs += __shfl_xor_sync(0xffffffffu, qs, 2);
+        qs += __shfl_xor_sync(0xffffffffu, qs, 4);
+        qtot = qs;
+        if (NP == 2) {
+          qs2 += __shfl_xor_sync(0xffffffffu, qs2, 1);
+          qs2 += __shfl_xor_sync(0xffffffffu, qs2, 2);
+          qs2 += __shfl_xor_sync(0xffffffffu, qs2, 4);
+          qtot2 = qs2;
+        }
+      }
+      if (cb == 0) {
+        qsum_s[nt % NACC][tb] = qtot;
+        if (NP == 2) qsum_s[nt % NACC][tb + 64] = qtot2;
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->qsum_ready[nt % NACC]);
@@ -392,30 +464,34 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
       const uint32_t leader = elect_one();
       uint32_t it0 = 0, nt = 0;                   // pipeline index of the tile's K block 0; tiles done
       bool ok = true;
-      for (int job = blockIdx.x; ok && job < a.total_tiles && !*abort_flag; job += gridDim.x, ++nt) {
-        const TItem& d = a.it[locate(a, job)];
-        const int nsteps = (int)(i2s_kp(d.K) / 256);
+      int ii = jb < je ? locate(a, jb) : 0;
+      for (int job = jb; me < NISS && ok && job < je && !*abort_flag; ++job, ++nt) {
+        while (ii + 1 < a.n && a.it[ii + 1].first_tile <= job) ++ii;
+        const int nsteps = steps_of(a.it[ii].K, CPS);
         const int buf = (int)(nt % NACC);
         ok = mbar_wait(&bars->tmem_empty[buf], ((nt / NACC) & 1u) ^ 1u, abort_flag, 1000);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t d_tmem = tmem_base + buf * TILE_N;
-        // a step = two K blocks = a stage pair: one wait, one fence and one commit per step (the writers signal and
-        // wait on the pair's later stage only)
-        for (int sidx = me; ok && sidx < nsteps; sidx += MMA_WARPS) {
-          const uint32_t it = it0 + 2u * (uint32_t)sidx;
+        // a step = GST K blocks = GST stages: one wait, one fence and one commit per step (the writers signal and
+        // wait on the step's last stage only)
+        for (int sidx = (int)((me + NISS - (it0 / GST) % NISS) % NISS); ok && sidx < nsteps; sidx += NISS) {
+          const uint32_t it = it0 + (uint32_t)GST * (uint32_t)sidx;
           const int st = (int)(it % STAGES);
-          ok = mbar_wait(&bars->full[st + 1], (it / STAGES) & 1u, abort_flag, 20);   // codes in tensor memory, activations landed
+          ok = mbar_wait(&bars->full[st + GST - 1], (it / STAGES) & 1u, abort_flag, 20);   // codes in tensor memory, activations landed
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          // the activation bytes were written through the generic proxy (cp.async) by the writer threads, whose
+          // arrivals this wait has observed; the tensor core reads them through the async proxy
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           const uint64_t bdesc = make_desc(smem_u32(tileB + st * B_BYTES));
 #pragma unroll
-          for (int k4 = 0; k4 < 2 * (KBLK / 32); ++k4)   // 32 bytes further along K: +2 in the address field, +8 columns
+          for (int k4 = 0; k4 < GST * (KBLK / 32); ++k4)   // 32 bytes further along K: +2 in the address field, +8 columns
             umma_u8s8_ta(d_tmem, tmem_base + A_COL0 + st * 32 + 8 * k4, bdesc + (uint64_t)((k4 >> 2) * (B_BYTES >> 4) + 2 * (k4 & 3)),
                          IDESC, 1u, leader);
-          umma_commit(&bars->empty[st + 1], leader);   // the pair is reusable once these MMAs have read it
+          umma_commit(&bars->empty[st + GST - 1], leader);   // the stages are reusable once these MMAs have read them
         }
         if (!ok) break;
-        it0 += 2u * (uint32_t)nsteps;
+        it0 += (uint32_t)GST * (uint32_t)nsteps;
         umma_commit(&bars->tmem_full[buf], leader);   // this issuer's share of the accumulator is complete
       }
       if (!ok && leader) {
@@ -423,12 +499,47 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
         bars->abort_flag = 1;
       }
     }
+  } else if (warp == PRODUCER_WARP) {
+    // ------------------------------------------------------------ producer of the packed-word ring
+    // Per step one bulk copy per 16-row unit of the tile (a unit's chunks are contiguous in the blob: CPS KB), issued
+    // by one lane each, SLOTS_A steps ahead of the writers: whole 32-byte sectors, no copy instructions in the
+    // writers' instruction stream.
+    const uint64_t pol = policy_evict_first();
+    int slot = 0;
+    uint32_t php = 0;
+    bool ok = true;
+    int ii = jb < je ? locate(a, jb) : 0;
+    for (int job = jb; ok && job < je && !*abort_flag; ++job) {
+      while (ii + 1 < a.n && a.it[ii + 1].first_tile <= job) ++ii;
+      const TItem& d = a.it[ii];
+      const int64_t kp = i2s_kp(d.K);
+      const int nch = (int)(kp / 256), nsteps = (nch + CPS - 1) / CPS;
+      const int row0 = (job - d.first_tile) * TILE_M;
+      const int left = (d.M - row0 + 15) >> 4, nunits = left < 8 ? left : 8;
+      const uint8_t* src = d.packed + ((int64_t)(row0 >> 4) + lane) * (4 * kp);
+      const uint32_t dst = smem_u32(ringA) + lane * (CPS * 1024);
+      for (int s2 = 0; s2 < nsteps && ok; ++s2) {
+        ok = mbar_wait(&bars->a_empty[slot], php ^ 1u, abort_flag, 20);   // every writer warp has read the slot
+        if (!ok) break;
+        const int nc = nch - s2 * CPS < CPS ? nch - s2 * CPS : CPS;
+        if (lane == 0) mbar_expect_tx(&bars->a_full[slot], (uint32_t)(nunits * nc) * 1024u);
+        __syncwarp();
+        if (lane < nunits) bulk_g2s(dst + slot * SLOT_BYTES, src + (int64_t)s2 * (CPS * 1024), (uint32_t)nc * 1024u, &bars->a_full[slot], pol);
+        if (++slot == SLOTS_A) slot = 0, php ^= 1u;
+      }
+    }
+    if (!ok && lane == 0) {
+      atomicExch(&g_stream_tc_error, BITNET_ERR_TIMEOUT);
+      bars->abort_flag = 1;
+    }
   } else {
     // ------------------------------------------------------------ epilogue
     const int quarter = warp & 3;                  // tensor-memory lanes 32*quarter .. 32*quarter+31
     uint32_t nt = 0;
-    for (int job = blockIdx.x; job < a.total_tiles && !*abort_flag; job += gridDim.x, ++nt) {
-      const TItem& d = a.it[locate(a, job)];
+    int ii = jb < je ? locate(a, jb) : 0;
+    for (int job = jb; job < je && !*abort_flag; ++job, ++nt) {
+      while (ii + 1 < a.n && a.it[ii + 1].first_tile <= job) ++ii;
+      const TItem& d = a.it[ii];
       const int buf = (int)(nt % NACC);
       const int m = (job - d.first_tile) * TILE_M + quarter * 32 + lane;
       float* const my_scale = ep_scale[quarter];
@@ -499,7 +610,7 @@ namespace {
 template <int TN>
 int launch_tn(const TArgs& a, int grid, cudaStream_t st) {
   constexpr int STAGES = TN == 64 ? 12 : 8;
-  const size_t smem = (size_t)STAGES * TN * KBLK + RING_A_BYTES + sizeof(Bars) + 1024;
+  const size_t smem = (size_t)STAGES * TN * KBLK + ring_a_bytes(TN) + sizeof(Bars) + 1024;
   static bool attr_set[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
@@ -520,7 +631,8 @@ int launch_gemm_i2s_stream_tc(const StreamTcLinear* items, int64_t n, cudaStream
   for (int64_t i0 = 0; i0 < n;) {
     const bool wide = items[i0].T > 64;
     int cnt = 0;
-    int64_t tiles = 0;
+    int64_t tiles = 0, work = 0;
+    const int cps = cps_of(wide ? 128 : 64);
     while (i0 + cnt < n && cnt < NITEMS && (items[i0 + cnt].T > 64) == wide) {
       const StreamTcLinear& s = items[i0 + cnt];
       if (!gemm_i2s_stream_tc_item_supported(s.T, s.M, s.K)) return BITNET_ERR_UNSUPPORTED_SHAPE;
@@ -537,12 +649,15 @@ int launch_gemm_i2s_stream_tc(const StreamTcLinear* items, int64_t n, cudaStream
       d.T = s.T;
       d.first_tile = (int)tiles;
       d.ldy = (int)(s.ldy ? s.ldy : s.M);
+      d.first_w = work;
+      work += ceil_div(s.M, TILE_M) * steps_of((int)s.K, cps);
       tiles += ceil_div(s.M, TILE_M);
       ++cnt;
     }
     if (cnt == 0) return BITNET_ERR_UNSUPPORTED_SHAPE;
     a.n = cnt;
     a.total_tiles = (int)tiles;
+    a.total_w = work;
     int grid = dev_info().sm_count;
     if (grid > tiles) grid = (int)tiles;
     log_launch("gemm_i2s_stream_tc_kernel<%d> items=%d tiles=%lld grid=%d", wide ? 128 : 64, cnt, (long long)tiles, grid);
