@@ -58,8 +58,13 @@ __host__ __device__ constexpr int cps_of(int tn) { return tn == 64 ? 2 : 1; }
 __host__ __device__ constexpr int da_of(int tn) { return 8 / cps_of(tn); }
 __host__ __device__ constexpr int ring_a_bytes(int tn) { return da_of(tn) * cps_of(tn) * 8192; }
 constexpr int MAX_SLOTS_A = 8;
-// steps by which the activation copies run ahead (the stages they go to must have been read by the MMAs)
+// Steps in the ring of the activation tiles (operand B, shared memory), of operand A (tensor memory) and of the step
+// barriers: 3 at 64-token tiles (12 stages of 32 columns beside two accumulators), 4 at 128-token tiles; and steps
+// by which the activation copies run ahead (into the tiles the MMAs of step s + DB - RB have read).  A longer B
+// ring with its own barriers (4 steps, copies two steps ahead) measured no faster and costs a wait per step.
+__host__ __device__ constexpr int rb_of(int tn) { return tn == 64 ? 3 : 4; }
 __host__ __device__ constexpr int db_of(int tn) { return tn == 64 ? 1 : 2; }
+__host__ __device__ constexpr int b_stages(int tn) { return rb_of(tn) * 2 * cps_of(tn); }
 constexpr int NITEMS = 400;                  // items per launch (argument block of 32 KB)
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
@@ -207,24 +212,26 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
   constexpr int TILE_N = TN;
   constexpr int STAGES = TN == 64 ? 12 : 8;
   constexpr int CPS = cps_of(TN), GST = 2 * CPS;   // chunks and stages per step
-  constexpr int DA = da_of(TN), DB = db_of(TN), SLOTS_A = DA;
+  constexpr int DA = da_of(TN), SLOTS_A = DA, RB = rb_of(TN), DB = db_of(TN);
+  constexpr int RA = STAGES / GST;                 // steps in the tensor-memory ring of operand A
+  constexpr int STAGES_B = RB * GST;               // activation tiles (one per K block) in shared memory
   constexpr uint32_t SLOT_BYTES = CPS * 8192;      // a step's packed words of the tile: 8 units x CPS KB
   constexpr int RING_A_BYTES = ring_a_bytes(TN);
   // Issuers at work: as many as the ring holds steps, issuer i taking the steps i, i + NISS, ... of the CTA's whole
   // step sequence (counted across tiles), i.e. always the same stages.  A wait for a barrier's phase k is only
   // meaningful once phase k - 1 is known to be complete (a barrier still in phase k - 1 answers "done" to a probe
   // for the parity of k); an issuer that meets every phase of its own barriers in order knows that.
-  constexpr int NISS = STAGES / GST;
-  static_assert(NISS <= MMA_WARPS, "an issuer warp per step of the ring");
+  constexpr int NISS = RB;
+  static_assert(NISS <= MMA_WARPS && RA <= RB, "an issuer warp per step of the barrier ring");
   constexpr int A_COL0 = NACC * TILE_N;        // first tensor-memory column of the A ring (32 columns per stage)
   constexpr int B_BYTES = TILE_N * KBLK;       // 8 or 16 KB per stage
   constexpr int NP = TN / 64;                  // activation pieces per writer thread and K block (tokens tb, tb + 64)
   constexpr uint32_t IDESC = idesc_of(TN);
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* tileB = smem;                                   // STAGES x 8 KB
-  uint8_t* ringA = smem + STAGES * B_BYTES;                // SLOTS_A x 512 x 16 bytes
-  Bars* bars = reinterpret_cast<Bars*>(smem + STAGES * B_BYTES + RING_A_BYTES);
+  uint8_t* tileB = smem;                                   // STAGES_B x 8 or 16 KB
+  uint8_t* ringA = smem + STAGES_B * B_BYTES;              // SLOTS_A steps of packed words
+  Bars* bars = reinterpret_cast<Bars*>(smem + STAGES_B * B_BYTES + RING_A_BYTES);
   volatile int* abort_flag = &bars->abort_flag;
   __shared__ int qsum_s[NACC][MAX_N];                      // sum of a token's codes over K, per accumulator in flight
   __shared__ float ep_scale[4][MAX_N];                     // epilogue: act_scale[t] * w_scale of the current tile
@@ -236,11 +243,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
   const int je = tile_at(a, a.total_w * (blockIdx.x + 1) / gridDim.x, CPS);
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) {
-      // a step's last stage: every writer warp once its codes are in tensor memory, and every writer thread's
-      // asynchronous arrival once its activation pieces have landed
-      mbar_init(&bars->full[s], WRITER_WARPS + WRITER_WARPS * 32);
-      mbar_init(&bars->empty[s], 1);             // tcgen05.commit (used on the odd stages: one per stage pair)
+    for (int s = 0; s < RB; ++s) {            // (per step of the barrier ring)
+      // every writer warp: its codes are in tensor memory and its activation pieces have landed
+      mbar_init(&bars->full[s], WRITER_WARPS);
+      mbar_init(&bars->empty[s], 1);             // tcgen05.commit: the step's MMAs have read their operands
     }
     for (int sl = 0; sl < SLOTS_A; ++sl) {
       mbar_init(&bars->a_full[sl], 1);           // the producer's arrival with the byte count
@@ -294,8 +300,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
     const uint32_t tile_b = smem_u32(tileB) + b_off;
     // Running positions instead of divisions: st0 = first stage of the current step (a multiple of GST), ph = how
     // often the stage ring has been passed (mod 2), slot = the step's ring slot.
-    int st0 = 0, slot = 0;
+    int bs = 0, tg = 0, slot = 0;                  // (bs: position in the B and barrier ring; tg: in the tensor-memory ring)
     uint32_t ph = 0, pha = 0;                      // (pha: passes of the packed-word ring, mod 2)
+    uint32_t g = 0;                                // steps done by this CTA
     uint32_t nt = 0;
     bool ok = true;
     int ii = jb < je ? locate(a, jb) : 0, prev_item = -1;
@@ -316,8 +323,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
       // the thread's activation pieces of step s into the stages stb .. stb + GST - 1 (zeros beyond T, K), once they
       // are free: the stages are released in order, so the last one being free means all are
       auto issue_b = [&](int s2, int stb, uint32_t phb) -> bool {
-        if (!mbar_wait(&bars->empty[stb + GST - 1], phb ^ 1u, abort_flag, 20)) return false;
-        const uint32_t dst = tile_b + stb * B_BYTES;
+        if (!mbar_wait(&bars->empty[stb], phb ^ 1u, abort_flag, 20)) return false;
+        const uint32_t dst = tile_b + stb * (GST * B_BYTES);
         const int8_t* src = qrow + (int64_t)s2 * (GST * KBLK);
         const int8_t* src2 = qrow2 + (int64_t)s2 * (GST * KBLK);
         if (s2 < nfull) {
@@ -342,45 +349,42 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
             }
           }
         }
-        // this thread's arrival on the step's barrier, made by the copy unit when the pieces (and every copy issued
-        // before them) have landed: no thread waits for activation bytes, the issuer does
-        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&bars->full[stb + GST - 1])) : "memory");
         return true;
       };
       // prologue: activation pieces of the first DB steps, a copy group per step
 #pragma unroll
       for (int p = 0; p < DB; ++p) {
-        int stb = st0 + GST * p;
+        int stb = bs + p;
         uint32_t phb = ph;
-        if (stb >= STAGES) stb -= STAGES, phb ^= 1u;
+        if (stb >= RB) stb -= RB, phb ^= 1u;
         if (ok && p < nsteps) ok = issue_b(p, stb, phb);
         cp_commit();
       }
       int qs = 0, qs2 = 0;
       for (int s2 = 0; s2 < nsteps && ok; ++s2) {
         if (s2 + DB < nsteps) {
-          int stb = st0 + GST * DB;
+          int stb = bs + DB;
           uint32_t phb = ph;
-          if (stb >= STAGES) stb -= STAGES, phb ^= 1u;
+          if (stb >= RB) stb -= RB, phb ^= 1u;
           ok = issue_b(s2 + DB, stb, phb);
           if (!ok) break;
         }
         cp_commit();
-        // No thread waits for activation bytes (the issuer does, through the step's barrier), except in a tile that
-        // takes the sums of the codes: there the pieces committed DB steps ago are read back.
+        // this thread's activation pieces of step s (committed DB steps ago; the copy groups hold nothing else) have
+        // landed; the issuer makes them visible to the tensor core's proxy after the step's barrier
+        cp_wait<DB>();
         if (need_q) {
-          cp_wait<DB>();
 #pragma unroll
           for (int j = 0; j < GST; ++j) {
             uint4 b0;                              // this thread's own pieces, for the row sums
-            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b0.x), "=r"(b0.y), "=r"(b0.z), "=r"(b0.w) : "r"(tile_b + (st0 + j) * B_BYTES));
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b0.x), "=r"(b0.y), "=r"(b0.z), "=r"(b0.w) : "r"(tile_b + (bs * GST + j) * B_BYTES));
             qs = __dp4a((int)b0.x, 0x01010101, qs);
             qs = __dp4a((int)b0.y, 0x01010101, qs);
             qs = __dp4a((int)b0.z, 0x01010101, qs);
             qs = __dp4a((int)b0.w, 0x01010101, qs);
             if (NP == 2) {
               uint4 b1;
-              asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b1.x), "=r"(b1.y), "=r"(b1.z), "=r"(b1.w) : "r"(tile_b + (st0 + j) * B_BYTES + 8192));
+              asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b1.x), "=r"(b1.y), "=r"(b1.z), "=r"(b1.w) : "r"(tile_b + (bs * GST + j) * B_BYTES + 8192));
               qs2 = __dp4a((int)b1.x, 0x01010101, qs2);
               qs2 = __dp4a((int)b1.y, 0x01010101, qs2);
               qs2 = __dp4a((int)b1.z, 0x01010101, qs2);
@@ -393,6 +397,12 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
         // slot holds then meets activation codes that are all zero, or sums that are never stored.)
         ok = mbar_wait(&bars->a_full[slot], pha, abort_flag, 20);
         if (!ok) break;
+        // the tensor-memory columns of this step were last read by the MMAs of step g - RA (with a B ring as long,
+        // the wait before the copies of this step's activation pieces covered that)
+        if (RA < RB && g >= (uint32_t)RA) {
+          ok = mbar_wait(&bars->empty[(g - RA) % RB], ((g - RA) / RB) & 1u, abort_flag, 20);
+          if (!ok) break;
+        }
         uint32_t wa[CPS][4];
 #pragma unroll
         for (int c = 0; c < CPS; ++c)
@@ -416,7 +426,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
             o[4 * c4 + 2] = (w0 >> (4 * h + 2)) & 0x03030303u;
             o[4 * c4 + 3] = (w1 >> (4 * h + 2)) & 0x03030303u;
           }
-          const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 + (st0 + 2 * c + grp2) * 32 + hf * 16;
+          const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 + (tg * GST + 2 * c + grp2) * 32 + hf * 16;
           asm volatile(
               "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, "
               "%14, %15, %16};"
@@ -427,9 +437,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();
-        if (lane == 0) mbar_arrive(&bars->full[st0 + GST - 1]);   // one barrier per step (its last stage's)
-        st0 += GST;
-        if (st0 == STAGES) st0 = 0, ph ^= 1u;
+        if (lane == 0) mbar_arrive(&bars->full[bs]);
+        ++g;
+        if (++bs == RB) bs = 0, ph ^= 1u;
+        if (++tg == RA) tg = 0;
         if (++slot == SLOTS_A) slot = 0, pha ^= 1u;
       }
       if (!ok) break;
@@ -462,7 +473,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
     {
       const int me = warp - WRITER_WARPS;
       const uint32_t leader = elect_one();
-      uint32_t it0 = 0, nt = 0;                   // pipeline index of the tile's K block 0; tiles done
+      uint32_t g0 = 0, nt = 0;                    // steps before this tile; tiles done
       bool ok = true;
       int ii = jb < je ? locate(a, jb) : 0;
       for (int job = jb; me < NISS && ok && job < je && !*abort_flag; ++job, ++nt) {
@@ -474,10 +485,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
         const uint32_t d_tmem = tmem_base + buf * TILE_N;
         // a step = GST K blocks = GST stages: one wait, one fence and one commit per step (the writers signal and
         // wait on the step's last stage only)
-        for (int sidx = (int)((me + NISS - (it0 / GST) % NISS) % NISS); ok && sidx < nsteps; sidx += NISS) {
-          const uint32_t it = it0 + (uint32_t)GST * (uint32_t)sidx;
-          const int st = (int)(it % STAGES);
-          ok = mbar_wait(&bars->full[st + GST - 1], (it / STAGES) & 1u, abort_flag, 20);   // codes in tensor memory, activations landed
+        for (int sidx = (int)((me + NISS - g0 % NISS) % NISS); ok && sidx < nsteps; sidx += NISS) {
+          const uint32_t g = g0 + (uint32_t)sidx;        // the step's number in the CTA's step sequence
+          const int pos = (int)(g % RB), st = pos * GST, sta = (int)(g % RA) * GST;
+          ok = mbar_wait(&bars->full[pos], (g / RB) & 1u, abort_flag, 20);   // codes in tensor memory, activations landed
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           // the activation bytes were written through the generic proxy (cp.async) by the writer threads, whose
@@ -486,12 +497,12 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
           const uint64_t bdesc = make_desc(smem_u32(tileB + st * B_BYTES));
 #pragma unroll
           for (int k4 = 0; k4 < GST * (KBLK / 32); ++k4)   // 32 bytes further along K: +2 in the address field, +8 columns
-            umma_u8s8_ta(d_tmem, tmem_base + A_COL0 + st * 32 + 8 * k4, bdesc + (uint64_t)((k4 >> 2) * (B_BYTES >> 4) + 2 * (k4 & 3)),
+            umma_u8s8_ta(d_tmem, tmem_base + A_COL0 + sta * 32 + 8 * k4, bdesc + (uint64_t)((k4 >> 2) * (B_BYTES >> 4) + 2 * (k4 & 3)),
                          IDESC, 1u, leader);
-          umma_commit(&bars->empty[st + GST - 1], leader);   // the stages are reusable once these MMAs have read them
+          umma_commit(&bars->empty[pos], leader);   // the step's tiles and columns are reusable once these MMAs have read them
         }
         if (!ok) break;
-        it0 += (uint32_t)GST * (uint32_t)nsteps;
+        g0 += (uint32_t)nsteps;
         umma_commit(&bars->tmem_full[buf], leader);   // this issuer's share of the accumulator is complete
       }
       if (!ok && leader) {
@@ -609,8 +620,7 @@ bool gemm_i2s_stream_tc_item_supported(int64_t T, int64_t M, int64_t K) {
 namespace {
 template <int TN>
 int launch_tn(const TArgs& a, int grid, cudaStream_t st) {
-  constexpr int STAGES = TN == 64 ? 12 : 8;
-  const size_t smem = (size_t)STAGES * TN * KBLK + ring_a_bytes(TN) + sizeof(Bars) + 1024;
+  const size_t smem = (size_t)b_stages(TN) * TN * KBLK + ring_a_bytes(TN) + sizeof(Bars) + 1024;
   static bool attr_set[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
