@@ -392,9 +392,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
             }
           }
         }
-        // the step's packed words have landed (bulk copies of the producer warp); once they are in registers the slot
-        // goes back to the producer.  (A chunk beyond the row's last, or a row beyond M, is not copied: what the
-        // slot holds then meets activation codes that are all zero, or sums that are never stored.)
+        // the step's packed words have landed (bulk copies of the producer warp).  (A chunk beyond the row's last, or a
+        // row beyond M, is not copied: what the slot holds then meets activation codes that are all zero, or sums that
+        // are never stored.)
         ok = mbar_wait(&bars->a_full[slot], pha, abort_flag, 20);
         if (!ok) break;
         // the tensor-memory columns of this step were last read by the MMAs of step g - RA (with a B ring as long,
@@ -409,8 +409,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
           asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
                        : "=r"(wa[c][0]), "=r"(wa[c][1]), "=r"(wa[c][2]), "=r"(wa[c][3])
                        : "r"(ring_a + slot * SLOT_BYTES + c * 1024));
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&bars->a_empty[slot]);
 #pragma unroll
         for (int c = 0; c < CPS; ++c) {
           // 64 codes of the row in K order = 16 tensor-memory columns: columns 4 c4 .. 4 c4 + 3 take the words
@@ -421,10 +419,12 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
           for (int c4 = 0; c4 < 4; ++c4) {
             const uint32_t w0 = w[2 * (c4 >> 1)], w1 = w[2 * (c4 >> 1) + 1];
             const int h = c4 & 1;
-            o[4 * c4 + 0] = (w0 >> (4 * h)) & 0x03030303u;
-            o[4 * c4 + 1] = (w1 >> (4 * h)) & 0x03030303u;
-            o[4 * c4 + 2] = (w0 >> (4 * h + 2)) & 0x03030303u;
-            o[4 * c4 + 3] = (w1 >> (4 * h + 2)) & 0x03030303u;
+            // the code moves to the top two bits of its byte (64 x code: one scale for all four fields, taken out in
+            // the epilogue): left shifts, which the multiply-add pipe can do beside the integer pipe's masks
+            o[4 * c4 + 0] = (w0 << (6 - 4 * h)) & 0xC0C0C0C0u;
+            o[4 * c4 + 1] = (w1 << (6 - 4 * h)) & 0xC0C0C0C0u;
+            o[4 * c4 + 2] = (w0 << (4 - 4 * h)) & 0xC0C0C0C0u;
+            o[4 * c4 + 3] = (w1 << (4 - 4 * h)) & 0xC0C0C0C0u;
           }
           const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL0 + (tg * GST + 2 * c + grp2) * 32 + hf * 16;
           asm volatile(
@@ -437,7 +437,13 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();
-        if (lane == 0) mbar_arrive(&bars->full[bs]);
+        // The ring slot goes back to the producer only here, after the codes made from its words have been stored: an
+        // arrival right behind the shared-memory loads is not held back until they have read (measured: a refill
+        // overtook them), the loads' results having been used is.
+        if (lane == 0) {
+          mbar_arrive(&bars->a_empty[slot]);
+          mbar_arrive(&bars->full[bs]);
+        }
         ++g;
         if (++bs == RB) bs = 0, ph ^= 1u;
         if (++tg == RA) tg = 0;
@@ -584,7 +590,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
           for (int j = 0; j < 32; ++j) {
             const int t = c0 + j;
             if (t < d.T) {
-              const int acc = (int)v[j] - qsum_s[buf][t];          // sum(code * q) - sum(q) = sum(w * q)
+              const int acc = ((int)v[j] >> 6) - qsum_s[buf][t];   // sum(64 code * q) / 64 - sum(q) = sum(w * q)
               d.y[(int64_t)t * d.ldy + m] = __fmul_rn((float)acc, my_scale[t]);
               if (d.acc_out) d.acc_out[(int64_t)t * d.ldy + m] = acc;
             }
@@ -614,7 +620,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
 // Shapes the kernel takes: 9 to 64 tokens; rows long enough that a tile's K blocks outnumber the ring by far (the
 // hand-over of the per-token sums between tiles relies on it).
 bool gemm_i2s_stream_tc_item_supported(int64_t T, int64_t M, int64_t K) {
-  return T >= 9 && T <= MAX_N && M >= 1 && M <= 0x7fffffff && K >= 2048 && (K % 64) == 0 && K <= 0x3fffffff;
+  // (K: the accumulators hold 64 x sum(code * q), at most 64 * 2 * 127 * K in magnitude)
+  return T >= 9 && T <= MAX_N && M >= 1 && M <= 0x7fffffff && K >= 2048 && (K % 64) == 0 && K <= 131072;
 }
 
 namespace {
