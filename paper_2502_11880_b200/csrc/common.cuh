@@ -179,6 +179,9 @@ struct StreamTcLinear {
   int64_t ldy;         // elements between the token rows of y / acc_out; 0 = M
 };
 bool gemm_i2s_stream_tc_item_supported(int64_t T, int64_t M, int64_t K);
+// Tensor map of the codes q[T][K] (int8) for tensor copies of 128 columns x `box_t` tokens into the 128-byte-swizzled
+// K-major layout of an MMA operand; columns and tokens beyond the matrix read as zeros (gemm_prefill_tc.cu).
+int encode_q_tile_map(void* out /* CUtensorMap */, const int8_t* q, int64_t K, int64_t T, int box_t);
 int launch_gemm_i2s_stream_tc(const StreamTcLinear* items, int64_t n, cudaStream_t st);
 int gemm_i2s_stream_tc_status(int* out);
 int gemm_i2s_stream_tc_status_clear();

@@ -30,6 +30,8 @@
 // for the prefill kernel, which such lists fell to before.  What binds is the writers' instruction stream (about 100 per warp and step: 7.6 ms per 100B sweep at any
 // token count from 17 to 64, against 9.6 to 19.4 ms for the mma.sync kernel of gemv_i2s_mid.cu).  Every mbarrier wait is bounded; a wait that gives up sets a CTA-wide abort flag and the device status
 // word, all roles leave their loops, and the CTA frees its tensor memory before it exits.
+#include <cuda.h>
+
 #include <cstdlib>
 #include <cstring>
 
@@ -48,8 +50,9 @@ constexpr int TMEM_COLS = 512;
 constexpr int MAX_N = 128;
 constexpr int WRITER_WARPS = 16;
 constexpr int MMA_WARPS = 4;                 // issuer warps (NISS of them at work: see the kernel)
-constexpr int PRODUCER_WARP = WRITER_WARPS + MMA_WARPS + 4;    // after the 4 epilogue warps
-constexpr int THREADS = (PRODUCER_WARP + 1) * 32;
+constexpr int PRODUCER_WARP = WRITER_WARPS + MMA_WARPS + 4;    // packed words (operand A's source); after the 4 epilogue warps
+constexpr int PRODUCER_B_WARP = PRODUCER_WARP + 1;             // activation tiles (operand B)
+constexpr int THREADS = (PRODUCER_B_WARP + 1) * 32;
 // A step = CPS 256-column chunks of a tile's rows (2 CPS K blocks = 2 CPS stages): two chunks per step at 64-token
 // tiles (12 stages = 3 steps in the ring), one at 128-token tiles (8 stages = 4 steps).  Per step a writer thread
 // unpacks 16 bytes of packed words per chunk; the waits, fences and barrier arrivals are paid once per step.
@@ -65,7 +68,7 @@ constexpr int MAX_SLOTS_A = 8;
 __host__ __device__ constexpr int rb_of(int tn) { return tn == 64 ? 3 : 4; }
 __host__ __device__ constexpr int db_of(int tn) { return tn == 64 ? 1 : 2; }
 __host__ __device__ constexpr int b_stages(int tn) { return rb_of(tn) * 2 * cps_of(tn); }
-constexpr int NITEMS = 400;                  // items per launch (argument block of 32 KB)
+constexpr int NITEMS = 160;                  // items per launch (argument block of 32 KB: a tensor map and 72 bytes each)
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 static __device__ int g_stream_tc_error = 0;
@@ -85,6 +88,7 @@ struct TItem {
 static_assert(sizeof(TItem) == 72, "argument block layout");
 
 struct TArgs {
+  CUtensorMap qmap[NITEMS];   // the item's codes q[T][K] as tiles of 128 columns x TN tokens, 128-byte swizzle, zero fill
   int n, total_tiles;
   int64_t total_w;
   TItem it[NITEMS];
@@ -93,6 +97,7 @@ static_assert(sizeof(TArgs) <= 32764, "kernel parameter limit");
 
 struct __align__(8) Bars {
   uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[NACC], tmem_empty[NACC], qsum_ready[NACC];
+  uint64_t b_full[4];                                   // a step's activation tiles have landed
   uint64_t a_full[MAX_SLOTS_A], a_empty[MAX_SLOTS_A];   // packed-word ring: bytes landed / slot read by every writer warp
   uint32_t tmem_base;
   int abort_flag;
@@ -244,8 +249,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < RB; ++s) {            // (per step of the barrier ring)
-      // every writer warp: its codes are in tensor memory and its activation pieces have landed
+      // every writer warp: its codes are in tensor memory
       mbar_init(&bars->full[s], WRITER_WARPS);
+      mbar_init(&bars->b_full[s], 1);            // the producer's arrival with the byte count
       mbar_init(&bars->empty[s], 1);             // tcgen05.commit: the step's MMAs have read their operands
     }
     for (int sl = 0; sl < SLOTS_A; ++sl) {
@@ -315,64 +321,13 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
       const int64_t kp = i2s_kp(d.K);
       const int nch = (int)(kp / 256), nsteps = (nch + CPS - 1) / CPS;
       // chunk c of a row: 64 bytes; K block 2c + grp2 = its half grp2 (32 bytes), of which this thread takes 16
-      const int K = d.K;
-      const int nfull = K / (GST * KBLK);          // steps whose K blocks all lie inside K
-      const int8_t* qrow = d.q + (int64_t)(tb < d.T ? tb : 0) * K + cb * 16;
-      const int8_t* qrow2 = d.q + (int64_t)(tb + 64 < d.T ? tb + 64 : 0) * K + cb * 16;   // (TN = 128: the thread's second token)
-      const uint32_t tok_sz = tb < d.T ? 16u : 0u, tok2_sz = (NP == 2 && tb + 64 < d.T) ? 16u : 0u;
-      // the thread's activation pieces of step s into the stages stb .. stb + GST - 1 (zeros beyond T, K), once they
-      // are free: the stages are released in order, so the last one being free means all are
-      auto issue_b = [&](int s2, int stb, uint32_t phb) -> bool {
-        if (!mbar_wait(&bars->empty[stb], phb ^ 1u, abort_flag, 20)) return false;
-        const uint32_t dst = tile_b + stb * (GST * B_BYTES);
-        const int8_t* src = qrow + (int64_t)s2 * (GST * KBLK);
-        const int8_t* src2 = qrow2 + (int64_t)s2 * (GST * KBLK);
-        if (s2 < nfull) {
-#pragma unroll
-          for (int j = 0; j < GST; ++j) {
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + j * B_BYTES), "l"(src + j * KBLK), "r"(tok_sz) : "memory");
-            if (NP == 2)                             // tokens 64..127 lie 8 row groups (8 KB) further down the tile
-              asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + j * B_BYTES + 8192), "l"(src2 + j * KBLK), "r"(tok2_sz)
-                           : "memory");
-          }
-        } else {
-          const int col = s2 * (GST * KBLK) + cb * 16;
-#pragma unroll
-          for (int j = 0; j < GST; ++j) {
-            const bool in = col + j * KBLK + 16 <= K;
-            const uint32_t by = in ? tok_sz : 0u;
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + j * B_BYTES), "l"(in ? src + j * KBLK : qrow), "r"(by) : "memory");
-            if (NP == 2) {
-              const uint32_t cy = in ? tok2_sz : 0u;
-              asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + j * B_BYTES + 8192), "l"(in ? src2 + j * KBLK : qrow), "r"(cy)
-                           : "memory");
-            }
-          }
-        }
-        return true;
-      };
-      // prologue: activation pieces of the first DB steps, a copy group per step
-#pragma unroll
-      for (int p = 0; p < DB; ++p) {
-        int stb = bs + p;
-        uint32_t phb = ph;
-        if (stb >= RB) stb -= RB, phb ^= 1u;
-        if (ok && p < nsteps) ok = issue_b(p, stb, phb);
-        cp_commit();
-      }
       int qs = 0, qs2 = 0;
       for (int s2 = 0; s2 < nsteps && ok; ++s2) {
-        if (s2 + DB < nsteps) {
-          int stb = bs + DB;
-          uint32_t phb = ph;
-          if (stb >= RB) stb -= RB, phb ^= 1u;
-          ok = issue_b(s2 + DB, stb, phb);
+        // a tile that takes the sums of the codes reads this thread's pieces of the landed activation tiles
+        if (need_q) {
+          ok = mbar_wait(&bars->b_full[bs], ph, abort_flag, 20);
           if (!ok) break;
         }
-        cp_commit();
-        // this thread's activation pieces of step s (committed DB steps ago; the copy groups hold nothing else) have
-        // landed; the issuer makes them visible to the tensor core's proxy after the step's barrier
-        cp_wait<DB>();
         if (need_q) {
 #pragma unroll
           for (int j = 0; j < GST; ++j) {
@@ -397,12 +352,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
         // are never stored.)
         ok = mbar_wait(&bars->a_full[slot], pha, abort_flag, 20);
         if (!ok) break;
-        // the tensor-memory columns of this step were last read by the MMAs of step g - RA (with a B ring as long,
-        // the wait before the copies of this step's activation pieces covered that)
-        if (RA < RB && g >= (uint32_t)RA) {
-          ok = mbar_wait(&bars->empty[(g - RA) % RB], ((g - RA) / RB) & 1u, abort_flag, 20);
-          if (!ok) break;
-        }
+        // the tensor-memory columns of this step were last read by the MMAs of step g - RA
+        static_assert(RA == RB, "one barrier ring for both operands");
+        ok = mbar_wait(&bars->empty[bs], ph ^ 1u, abort_flag, 20);
+        if (!ok) break;
         uint32_t wa[CPS][4];
 #pragma unroll
         for (int c = 0; c < CPS; ++c)
@@ -496,10 +449,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
           const int pos = (int)(g % RB), st = pos * GST, sta = (int)(g % RA) * GST;
           ok = mbar_wait(&bars->full[pos], (g / RB) & 1u, abort_flag, 20);   // codes in tensor memory, activations landed
           if (!ok) break;
+          ok = mbar_wait(&bars->b_full[pos], (g / RB) & 1u, abort_flag, 20);      // the step's activation tiles have landed
+          if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          // the activation bytes were written through the generic proxy (cp.async) by the writer threads, whose
-          // arrivals this wait has observed; the tensor core reads them through the async proxy
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           const uint64_t bdesc = make_desc(smem_u32(tileB + st * B_BYTES));
 #pragma unroll
           for (int k4 = 0; k4 < GST * (KBLK / 32); ++k4)   // 32 bytes further along K: +2 in the address field, +8 columns
@@ -515,6 +467,39 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
         atomicExch(&g_stream_tc_error, BITNET_ERR_TIMEOUT);
         bars->abort_flag = 1;
       }
+    }
+  } else if (warp == PRODUCER_B_WARP) {
+    // ------------------------------------------------------------ producer of the activation tiles (operand B)
+    // Per step GST tiles of 128 columns x TN tokens (tensor copies: 128-byte swizzle, zeros beyond T and K), as far
+    // ahead as the ring allows: a step's tiles are free once the MMAs of the step RB before have read them.
+    int bs = 0;
+    uint32_t ph = 0;
+    bool ok = true;
+    int ii = jb < je ? locate(a, jb) : 0;
+    for (int job = jb; ok && job < je && !*abort_flag; ++job) {
+      while (ii + 1 < a.n && a.it[ii + 1].first_tile <= job) ++ii;
+      const int nsteps = steps_of(a.it[ii].K, CPS);
+      const CUtensorMap* map = &a.qmap[ii];
+      for (int s2 = 0; s2 < nsteps && ok; ++s2) {
+        ok = mbar_wait(&bars->empty[bs], ph ^ 1u, abort_flag, 20);
+        if (!ok) break;
+        if (lane == 0) {
+          mbar_expect_tx(&bars->b_full[bs], (uint32_t)(GST * B_BYTES));
+#pragma unroll
+          for (int j = 0; j < GST; ++j)
+            asm volatile(
+                "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                ::"r"(smem_u32(tileB + (bs * GST + j) * B_BYTES)), "l"(map), "r"((s2 * GST + j) * KBLK), "r"(0),
+                  "r"(smem_u32(&bars->b_full[bs]))
+                : "memory");
+        }
+        __syncwarp();
+        if (++bs == RB) bs = 0, ph ^= 1u;
+      }
+    }
+    if (!ok && lane == 0) {
+      atomicExch(&g_stream_tc_error, BITNET_ERR_TIMEOUT);
+      bars->abort_flag = 1;
     }
   } else if (warp == PRODUCER_WARP) {
     // ------------------------------------------------------------ producer of the packed-word ring
@@ -667,6 +652,7 @@ int launch_gemm_i2s_stream_tc(const StreamTcLinear* items, int64_t n, cudaStream
       d.first_tile = (int)tiles;
       d.ldy = (int)(s.ldy ? s.ldy : s.M);
       d.first_w = work;
+      if (int rc = encode_q_tile_map(&a.qmap[cnt], s.q, s.K, s.T, wide ? 128 : 64)) return rc;
       work += ceil_div(s.M, TILE_M) * steps_of((int)s.K, cps);
       tiles += ceil_div(s.M, TILE_M);
       ++cnt;

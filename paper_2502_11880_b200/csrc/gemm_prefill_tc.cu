@@ -468,6 +468,19 @@ EncodeTiledFn encode_fn() {
 
 }  // namespace
 
+int encode_q_tile_map(void* out, const int8_t* q, int64_t K, int64_t T, int box_t) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return note_cuda_error(cudaErrorNotSupported);
+  const cuuint64_t gdim[2] = {(cuuint64_t)K, (cuuint64_t)T};
+  const cuuint64_t gstride[1] = {(cuuint64_t)K};            // bytes between token rows
+  const cuuint32_t box[2] = {KBLK, (cuuint32_t)box_t};
+  const cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(static_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(q), gdim, gstride, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? BITNET_OK : note_cuda_error(cudaErrorInvalidValue);
+}
+
 int launch_gemm_i2s_simt(const uint8_t* packed, float w_scale, int64_t M, int64_t K, const int8_t* q,
                          const float* act_scale, int64_t T, float* y, int32_t* acc_out, cudaStream_t st);
 
