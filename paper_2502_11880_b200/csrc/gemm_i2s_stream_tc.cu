@@ -6,30 +6,36 @@
 // Between decode (1..8 tokens: the weight stream is everything, mma.sync keeps up) and prefill (hundreds of tokens:
 // the tensor cores are everything) the work per weight byte is small enough that the blob should cross HBM once,
 // yet too large for mma.sync: m16n8k32 needs 2 T MMAs per 1-KB chunk.  The paper treats neither stage; the design
-// is this build's.  One persistent CTA per SM walks tiles of 128 out-features x all of K, tile j of the list's
-// tile sequence going to CTA j mod grid:
-//   * warps 0-15 (writers): thread = (row of the tile, half of a 128-column K block).  It keeps the row's packed
-//     words of the next eight steps in flight (16-byte cp.async copies into a private ring slot: 64 KB per SM),
-//     turns the 2-bit codes into bytes 0/1/2 (a shift and a mask per word: the codes go to the tensor core as
-//     UNSIGNED 8-bit values, the "- sum(q)" of code = w + 1 is applied in the epilogue) and writes them straight
-//     into tensor memory (tcgen05.st): operand A never touches shared memory as bytes.  The same threads copy the
-//     activation tile (64 tokens x 128 codes) of each K block, two steps ahead, into shared memory in the
-//     128-byte-swizzled K-major layout (operand B; cp.async with zero fill beyond T and K) and add up the codes of
-//     their own pieces once landed, which gives sum(q) per token;
-//   * warps 16-19: issuers, taking the steps in turn.  Per step (two K blocks) one elected lane issues eight
-//     tcgen05.mma (M = 128, N = 64, K = 32; A from tensor memory, B from shared memory) and releases the stage pair
-//     with one tcgen05.commit.  An issuer's wait-fence-issue-commit round costs about 500 cycles whatever the MMAs
-//     do (at 64 tokens they occupy the tensor pipe for 32 cycles each: measured 22 cycles of issue per MMA, over
-//     200 for the wait, fence and commit around them), so several warps share the steps; every MMA accumulates (the
-//     epilogue leaves the accumulators zeroed), so their order does not matter;
-//   * warps 20-23: epilogue -- tcgen05.ld the finished 128 x 64 accumulator, zero it, subtract sum(q), rescale,
-//     store y.
-// Two accumulators (2 x 64 columns) overlap a tile's epilogue with the next tile's MMAs; the A ring takes 12 x 32
-// columns.  Items with 65 to 128 tokens run the same kernel with 128-token tiles (template TN = 128: two activation
-// pieces per writer thread and K block, accumulators of 128 columns, 8 stages): 11 ms per 100B sweep against 22 ms
-// for the prefill kernel, which such lists fell to before.  What binds is the writers' instruction stream (about 100 per warp and step: 7.6 ms per 100B sweep at any
-// token count from 17 to 64, against 9.6 to 19.4 ms for the mma.sync kernel of gemv_i2s_mid.cu).  Every mbarrier wait is bounded; a wait that gives up sets a CTA-wide abort flag and the device status
-// word, all roles leave their loops, and the CTA frees its tensor memory before it exits.
+// is this build's.  One persistent CTA per SM walks tiles of 128 out-features x all of K; the list's tiles form one
+// sequence, of which a CTA takes the contiguous range that holds its equal share of the work (steps).  A step is two
+// 256-column chunks of the tile's rows (four K blocks of 128) at 64-token tiles, one chunk at 128-token tiles.
+//   * warp 24 (producer of packed words): per step one bulk copy per 16-row unit of the tile (a unit's chunks are
+//     contiguous in the blob) into a ring of shared memory, 8 chunks ahead of the writers;
+//   * warp 25 (producer of activation tiles): per K block one tensor copy of 128 codes x 64 (128) tokens of q into the
+//     128-byte-swizzled K-major layout of operand B, zeros beyond T and K (the tensor maps, one per item, travel in
+//     the argument block), as far ahead as the ring of 3 (4) steps allows;
+//   * warps 0-15 (writers): thread = (row of the tile, 16 bytes of a chunk's 64).  It turns the 2-bit codes into bytes
+//     whose top two bits are the code (a left shift and a mask per word: 64 x code as UNSIGNED 8-bit values; the
+//     factor 64 and the "- sum(q)" of code = w + 1 are taken out in the epilogue) and writes them straight into
+//     tensor memory (tcgen05.st): operand A never touches shared memory as bytes.  In the first tile of an item the
+//     writers also add up the codes of the landed activation tiles: sum(q) per token, kept for the item's other tiles;
+//   * warps 16-19: issuers.  Issuer i takes the steps i, i + R, ... of the CTA's whole step sequence (R = steps in
+//     the ring = issuers at work), so it always meets the same barriers, phase after phase.  Per step one elected
+//     lane issues 16 (8) tcgen05.mma (M = 128, N = 64 or 128, K = 32; A from tensor memory, B from shared memory) and
+//     releases the step's stages with one tcgen05.commit; every MMA accumulates (the epilogue leaves the accumulators
+//     zeroed), so their order does not matter;
+//   * warps 20-23: epilogue -- tcgen05.ld the finished 128 x 64 accumulator, zero it, divide by 64, subtract sum(q),
+//     rescale, store y.
+// Two accumulators (2 x 64 or 2 x 128 columns) overlap a tile's epilogue with the next tile's MMAs; the A ring takes
+// the other 12 (8) x 32 columns.  Measured on the 100B-shaped sweep (17.1 GB of packed weights, inputs fp32, the
+// list quantiser included): 4.7 ms at 32 tokens, 5.2 at 64, 8.0 at 128, against 9.6 to 19.4 ms for the mma.sync
+// kernel of gemv_i2s_mid.cu and 22 ms for the prefill kernel at 128.  What binds: the writers -- about 500 cycles
+// of integer work and 400 of barrier probes per step against the 712 the HBM stream allows -- then, at 128 tokens,
+// the tensor pipe.  Two rules learnt by measurement: a wait for phase k of a barrier means nothing unless phase
+// k - 1 is known to be over (hence issuers bound to their own stages), and a ring slot may be handed back only
+// after the values loaded from it have been used, not right behind the loads.  Every mbarrier wait is bounded; a wait
+// that gives up sets a CTA-wide abort flag and the device status word, all roles leave their loops, and the CTA frees
+// its tensor memory before it exits.
 #include <cuda.h>
 
 #include <cstdlib>
@@ -62,11 +68,9 @@ __host__ __device__ constexpr int da_of(int tn) { return 8 / cps_of(tn); }
 __host__ __device__ constexpr int ring_a_bytes(int tn) { return da_of(tn) * cps_of(tn) * 8192; }
 constexpr int MAX_SLOTS_A = 8;
 // Steps in the ring of the activation tiles (operand B, shared memory), of operand A (tensor memory) and of the step
-// barriers: 3 at 64-token tiles (12 stages of 32 columns beside two accumulators), 4 at 128-token tiles; and steps
-// by which the activation copies run ahead (into the tiles the MMAs of step s + DB - RB have read).  A longer B
-// ring with its own barriers (4 steps, copies two steps ahead) measured no faster and costs a wait per step.
+// barriers: 3 at 64-token tiles (12 stages of 32 columns beside two accumulators), 4 at 128-token tiles.  A longer B
+// ring with its own barriers (4 steps at 64-token tiles) measured no faster and costs the writers a wait per step.
 __host__ __device__ constexpr int rb_of(int tn) { return tn == 64 ? 3 : 4; }
-__host__ __device__ constexpr int db_of(int tn) { return tn == 64 ? 1 : 2; }
 __host__ __device__ constexpr int b_stages(int tn) { return rb_of(tn) * 2 * cps_of(tn); }
 constexpr int NITEMS = 160;                  // items per launch (argument block of 32 KB: a tensor map and 72 bytes each)
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
@@ -217,7 +221,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
   constexpr int TILE_N = TN;
   constexpr int STAGES = TN == 64 ? 12 : 8;
   constexpr int CPS = cps_of(TN), GST = 2 * CPS;   // chunks and stages per step
-  constexpr int DA = da_of(TN), SLOTS_A = DA, RB = rb_of(TN), DB = db_of(TN);
+  constexpr int DA = da_of(TN), SLOTS_A = DA, RB = rb_of(TN);
   constexpr int RA = STAGES / GST;                 // steps in the tensor-memory ring of operand A
   constexpr int STAGES_B = RB * GST;               // activation tiles (one per K block) in shared memory
   constexpr uint32_t SLOT_BYTES = CPS * 8192;      // a step's packed words of the tile: 8 units x CPS KB

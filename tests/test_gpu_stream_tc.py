@@ -39,6 +39,27 @@ def test_stream_tc_many_tiles_per_cta_and_repeat():
             it.check(rows=np.sort(rng.choice(it.M, 300, replace=False)))
 
 
+def test_stream_tc_more_items_than_one_launch_takes():
+    """More items than one argument block holds (160: a tensor map per item): several launches in list order; every
+    CTA meets several items (the per-token sums are taken anew at each), K with an odd number of 256-column chunks."""
+    items = [Item("i2s", 128 * (1 + i % 2) - (i % 5), 2048 + 256 * (i % 4), 17 + i % 20, 3500 + i) for i in range(170)]
+    run_group(items)
+    for it in items:
+        it.check()
+
+
+def test_stream_tc_same_list_ten_times():
+    """One tile per CTA, cold and warm: the packed-word ring must not be refilled before every warp has used its
+    words, whatever the timing (ten runs, every accumulator each time)."""
+    it = Item("i2s", 1000, 8192, 64, 811)
+    q_ref, _, _ = oracle.quant_act(it.x.numpy())
+    acc_ref = oracle.mpgemm_def(q_ref, it.w.numpy())
+    for _ in range(10):
+        it.gacc.t.zero_()
+        run_group([it])
+        assert np.array_equal(it.gacc.t.cpu().numpy(), acc_ref)
+
+
 def test_stream_tc_sixty_five_to_128_tokens():
     """The 128-token tile variant (two activation pieces per writer thread and K block, 8 stages), mixed with
     64-token items in one list (separate launches per class), ragged rows and a long row."""
