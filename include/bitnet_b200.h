@@ -250,14 +250,16 @@ int bitnet_linear_host_batch(const bitnet_host_linear_t* items, int64_t n, void*
  *     activation row is quantised by the two or three CTAs whose share touches its linear instead of by
  *     every CTA of a launch of its own (rows whose codes do not fit shared memory are walked in parts of K).
  *     The per-launch fixed cost of a decode GEMV (about 3 us of the 5-20 us a 100B-shaped linear takes) is
- *     paid once per run.  Items with 9 to 16 tokens join such a run as two items over the same weights
- *     (tokens 0..7, then the rest).
+ *     paid once per run.  Items with 9 to 16 tokens run in launches of their own of the same kernel's
+ *     two-group form (an MMA per group of eight tokens and weight register; the weights still cross HBM
+ *     once), their codes coming from one quantiser launch over the run's activation matrices.
  *   - TL2 and TL1 items with T <= 8 (K a multiple of 4, at least three tiles per row) likewise run in one
  *     persistent kernel per run of up to 340 consecutive items of the same format (the scan kernel, see
  *     bitnet_set_tl2_lookup).
- *   - I2_S items with 17 to 128 tokens and K >= 2048: the stand-alone quantiser per item, then ONE
- *     persistent kernel per run of up to 400 such items of the same class (up to 64 tokens, 65 to 128) that
- *     reads every blob once, unpacks the codes into tensor memory and multiplies on the tcgen05 tensor cores.
+ *   - I2_S items with 17 to 128 tokens and 2048 <= K <= 131072: one quantiser launch over the run's
+ *     activation matrices, then ONE persistent kernel per run of up to 160 such items of the same class (up to
+ *     64 tokens, 65 to 128) that reads every blob once, unpacks the codes into tensor memory and multiplies on
+ *     the tcgen05 tensor cores.
  *   - Every other item (more tokens, short K) is run by bitnet_linear in list order, with the item's
  *     workspace.
  * Results are identical to calling bitnet_linear per item.  Errors: BITNET_ERR_INVALID_ARG for a null or
