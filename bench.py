@@ -620,7 +620,7 @@ def run_ours(args):
                    "pct_of_8TBps": 100.0 * (value / world) / 8000.0},
         "e2e": {"value": e2e_val, "unit": UNIT, "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": int(sw.x_host.numel() * 4), "d2h_bytes_per_step": int(sw.y_host.numel() * 4),
-                "note": "one bitnet_linear_host_batch call per step: pinned fp32 x -> device, grouped kernels (quantiser + mpGEMV + rescale), fp32 y -> pinned host, in about eight groups whose copies overlap the neighbouring groups' kernels; weights resident"},
+                "note": "one bitnet_linear_host_batch call per step: pinned fp32 x -> device, grouped kernels (quantiser + mpGEMV + rescale), fp32 y -> pinned host, in five groups (1, 4, 6, 4 and 1 sixteenths of the linears) whose copies overlap the neighbouring groups' kernels; weights resident"},
         "gpu_launches": launches_per_step * args.steps,
         "roofline": {"bound": "hbm", "kernel": "gemv_i2s_group_kernel (quantiser fused)", "achieved": achieved,
                      "peak": pk["hbm"], "unit": "GB/s", "frac": achieved / pk["hbm"], "peak_source": pk["which"],

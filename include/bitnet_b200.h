@@ -199,8 +199,9 @@ int bitnet_linear_host(bitnet_fmt_t fmt, const void* packed, float w_scale, int6
 
 /*
  * A batch of linear layers with HOST activations and HOST results (Alg. 1 end to end per item), with the
- * copies overlapped with the kernels.  The batch is cut into about eight groups of consecutive items (one group
- * up to 16 items); a group's x_host are uploaded on an internal stream, the group runs as one bitnet_linear_group
+ * copies overlapped with the kernels.  The batch is cut into five groups of consecutive items, of 1, 4, 6, 4 and 1
+ * sixteenths of the items (one group below 32 items): only the first group's uploads and the last group's
+ * downloads are not hidden behind a kernel.  A group's x_host are uploaded on an internal stream, the group runs as one bitnet_linear_group
  * call on `stream` (one persistent kernel for I2_S decode items) once those uploads are complete, and its y_host
  * are downloaded on a second internal stream once the group is complete, while the next groups' uploads and
  * kernels proceed.  The items of a batch must therefore be independent of one another, as for

@@ -551,9 +551,10 @@ def test_linear_host_batch_matches_single_calls():
 @pytest.mark.gpu
 def test_linear_host_batch_merges_neighbouring_buffers():
     """Items whose host and device buffers continue one another (one pinned block, one device block) travel as
-    one copy per group; items 3 and 4 break the chain on the host side only, item 11 has 24 tokens (mid-batch
-    kernel).  Same results as item-by-item calls, nothing outside the buffers touched."""
-    specs = [(256, 1024, 1)] * 3 + [(512, 2048, 2)] * 8 + [(320, 4096, 24)]
+    one copy per group (40 items: five groups, the copies of one under the kernels of its
+    neighbour); items 3 and 4 break the chain on the host side only, the last item has 24 tokens (streaming or
+    mid-batch kernel).  Same results as item-by-item calls, nothing outside the buffers touched."""
+    specs = [(256, 1024, 1)] * 3 + [(512, 2048, 2)] * 36 + [(320, 4096, 24)]
     nx = sum(T * K for M, K, T in specs)
     ny = sum(T * M for M, K, T in specs)
     xh_all = torch.empty(nx + 64, dtype=torch.float32).pin_memory()
