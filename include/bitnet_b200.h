@@ -153,7 +153,7 @@ int bitnet_pack_tl(bitnet_fmt_t fmt, const int8_t* w, int64_t M, int64_t K, int 
  * I2_S: T <= 8 runs the decode GEMV kernel; 9 <= T <= 64 a scan of the weights on mma.sync tensor-core
  * tiles over K-slices followed by a rescale kernel (when the workspace is missing or too small, the
  * prefill kernel takes the call instead) -- except that a tensor with many 128-row tiles (two thirds of a
- * tile per SM at 33..64 tokens, two tiles per SM at 65..128) goes to the streaming tcgen05 kernel of
+ * tile per SM at 25..64 tokens, one tile per SM at 65..128) goes to the streaming tcgen05 kernel of
  * bitnet_linear_group, which needs no workspace; larger T the tcgen05 prefill kernel (whole tiles per CTA; parts
  * of a tile's K per CTA when there are few tiles and the workspace is there).  TL runs a decode kernel over
  * groups of 8 tokens (the scan kernel, see bitnet_set_tl2_lookup); from 128 tokens on, with K a multiple of

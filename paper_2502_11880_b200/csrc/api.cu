@@ -311,14 +311,14 @@ int bitnet_mpgemm(bitnet_fmt_t fmt, const void* packed, float w_scale, int64_t M
     int rc = i2s_shape(M, K);
     if (rc) return rc;
     // A single tensor with enough 128-row tiles for the SMs: the streaming tcgen05 kernel (weights read once, codes
-    // unpacked into tensor memory).  Measured crossovers on 100B- and 8B-shaped tensors: 33 to 64 tokens from two
-    // thirds of a tile per SM on (72 against 112 us at 57344 x 8192, 18 against 32 at 14336 x 4096); 65 to 128 tokens
-    // from two tiles per SM on (104 against 121 us); up to 32 tokens the mma.sync kernel is as fast or faster on one
-    // tensor (lists are another matter: bitnet_linear_group).
+    // unpacked into tensor memory).  Measured crossovers against the mma.sync and prefill kernels, quantiser
+    // included (us): 57344 x 8192 at 24 / 32 / 64 / 128 tokens 57 / 56 / 59 / 85 against 54 / 66 / 114 / 125;
+    // 28672 x 8192: 36 / 36 / 38 / 53 against 35 / 40 / 65 / 70; with fewer tiles than two thirds of the SMs
+    // (8192 x 28672: 56 / 56 / 58 / 75 against 34 / 40 / 62 / 72) the kernels that split K stay ahead up to 64 tokens.
     static const bool stream_tc = [] { const char* e = getenv("BITNET_I2S_STREAM_TC"); return !(e && atoi(e) == 0); }();
     const int64_t tiles128 = ceil_div(M, 128), sms = dev_info().sm_count;
     if (stream_tc && gemm_i2s_stream_tc_item_supported(T, M, K) &&
-        ((T >= 33 && T <= 64 && tiles128 * 3 >= sms * 2) || (T >= 65 && T <= 128 && tiles128 >= sms * 2))) {
+        ((T >= 25 && T <= 64 && tiles128 * 3 >= sms * 2) || (T >= 65 && T <= 128 && tiles128 >= sms))) {
       StreamTcLinear t;
       t.packed = (const uint8_t*)packed;
       t.q = q;
