@@ -443,7 +443,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
         while (ii + 1 < a.n && a.it[ii + 1].first_tile <= job) ++ii;
         const int nsteps = steps_of(a.it[ii].K, CPS);
         const int buf = (int)(nt % NACC);
-        ok = mbar_wait(&bars->tmem_empty[buf], ((nt / NACC) & 1u) ^ 1u, abort_flag, 1000);
+        ok = mbar_wait(&bars->tmem_empty[buf], ((nt / NACC) & 1u) ^ 1u, abort_flag, 200);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t d_tmem = tmem_base + buf * TILE_N;
         // a step = GST K blocks = GST stages: one wait, one fence and one commit per step (the writers signal and
@@ -451,7 +451,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
         for (int sidx = (int)((me + NISS - g0 % NISS) % NISS); ok && sidx < nsteps; sidx += NISS) {
           const uint32_t g = g0 + (uint32_t)sidx;        // the step's number in the CTA's step sequence
           const int pos = (int)(g % RB), st = pos * GST, sta = (int)(g % RA) * GST;
-          ok = mbar_wait(&bars->full[pos], (g / RB) & 1u, abort_flag, 20);   // codes in tensor memory, activations landed
+          ok = mbar_wait(&bars->full[pos], (g / RB) & 1u, abort_flag, 200);   // codes in tensor memory, activations landed
           if (!ok) break;
           ok = mbar_wait(&bars->b_full[pos], (g / RB) & 1u, abort_flag, 20);      // the step's activation tiles have landed
           if (!ok) break;
@@ -485,7 +485,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
       const int nsteps = steps_of(a.it[ii].K, CPS);
       const CUtensorMap* map = &a.qmap[ii];
       for (int s2 = 0; s2 < nsteps && ok; ++s2) {
-        ok = mbar_wait(&bars->empty[bs], ph ^ 1u, abort_flag, 20);
+        ok = mbar_wait(&bars->empty[bs], ph ^ 1u, abort_flag, 200);
         if (!ok) break;
         if (lane == 0) {
           mbar_expect_tx(&bars->b_full[bs], (uint32_t)(GST * B_BYTES));
@@ -525,7 +525,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
       const uint8_t* src = d.packed + ((int64_t)(row0 >> 4) + lane) * (4 * kp);
       const uint32_t dst = smem_u32(ringA) + lane * (CPS * 1024);
       for (int s2 = 0; s2 < nsteps && ok; ++s2) {
-        ok = mbar_wait(&bars->a_empty[slot], php ^ 1u, abort_flag, 20);   // every writer warp has read the slot
+        ok = mbar_wait(&bars->a_empty[slot], php ^ 1u, abort_flag, 200);   // every writer warp has read the slot
         if (!ok) break;
         const int nc = nch - s2 * CPS < CPS ? nch - s2 * CPS : CPS;
         if (lane == 0) mbar_expect_tx(&bars->a_full[slot], (uint32_t)(nunits * nc) * 1024u);
