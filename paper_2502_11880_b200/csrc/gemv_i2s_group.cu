@@ -214,8 +214,11 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
   int* qsum = reinterpret_cast<int*>(smem + 64 + 32 * NT);        // [8 NT] sum of the staged codes per token
   float* qred = reinterpret_cast<float*>(smem + 64 + 64 * NT);    // [8 NT][16] partial maxima
   float* qmul = reinterpret_cast<float*>(smem + 64 + 576 * NT);   // [8 NT] 127 / amax per token
-  int* red = reinterpret_cast<int*>(smem + HB);                   // [CW][2][tmax][16] partial sums
-  int8_t* qs_mem = reinterpret_cast<int8_t*>(smem + HB + CW * 2 * a.tmax * 16 * 4);
+  // partial sums [CW][RD][tmax][16]: two buffers per warp, so that a warp may start its next unit while its group
+  // still adds up the last one; one when every warp finishes its own units (two-group form, one warp per unit)
+  const int RD = a.r0;                                 // (set by the host: 1 or 2)
+  int* red = reinterpret_cast<int*>(smem + HB);
+  int8_t* qs_mem = reinterpret_cast<int8_t*>(smem + HB + CW * RD * a.tmax * 16 * 4);
   uint8_t* rings = reinterpret_cast<uint8_t*>(qs_mem) + a.code_bytes;
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -413,7 +416,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
 
         // fragment: c[0] = (row g, token 2t), c[1] = (row g, token 2t+1), c[2], c[3] = the same for row g+8
         // (token group n: the tokens 8 n + 2t, 8 n + 2t + 1)
-        int* mine = red + ((warp * 2 + (nloc & 1)) * tmax) * 16;
+        const int rbuf = RD == 2 ? (nloc & 1) : 0;
+        int* mine = red + ((warp * RD + rbuf) * tmax) * 16;
 #pragma unroll
         for (int n = 0; n < NT; ++n) {
           int c[4];
@@ -435,13 +439,13 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_i2s_group_kernel(const __grid
           // this unit's turn to be finished by this warp: add the group's partials; the sums of an item walked in
           // parts rest in y (as integers) between the parts; the last part rescales and stores 16 rows
           const int row0 = (cj - first) * 16;
-          const int* grp = red + (((gi * S) * 2 + (nloc & 1)) * tmax) * 16;
+          const int* grp = red + (((gi * S) * RD + rbuf) * tmax) * 16;
 #pragma unroll
           for (int i = 0; i < 4 * NT; ++i) {
             const int idx = lane + 32 * i;
             if (idx < T * 16) {
               int v = 0;
-              for (int w2 = 0; w2 < S; ++w2) v += grp[w2 * 2 * tmax * 16 + idx];
+              for (int w2 = 0; w2 < S; ++w2) v += grp[w2 * RD * tmax * 16 + idx];
               const int tok = idx >> 4, row = row0 + (idx & 15);
               v -= qsum[tok];
               if (row < M) {
@@ -490,6 +494,7 @@ int depth_cap() {
 // unit, then shallower rings.
 struct Shape {
   int S, depth;
+  int rd = 2;      // buffers of partial sums per warp (1: two-group form with one warp per unit)
 };
 // `units` = 16-row units of the whole launch: with at least four units per warp of the GPU every warp takes whole
 // units (no partial sums to join, no group barriers: 2.52 ms per 100B sweep against 2.72 with four warps per unit,
@@ -504,11 +509,20 @@ Shape shape_for(int64_t nch, int64_t units) {
   const int64_t nw = nch / S;      // the shortest slice
   int depth = depth_cap();
   while (depth > 4 && depth > nw) depth = depth == 12 ? 8 : depth - 2;
-  return Shape{S, depth};
+  Shape sh;
+  sh.S = S;
+  sh.depth = depth;
+  return sh;
 }
 
-size_t smem_of(int tmax, size_t code_bytes, int depth) {
-  return (size_t)header_bytes(tmax) + (size_t)CW * 2 * tmax * 16 * 4 + code_bytes + (size_t)CW * depth * 1024;
+// true if a launch over `units` units runs with one warp per unit
+bool one_warp_per_unit(int64_t units) {
+  const int f = forced_s();
+  return f ? f == 1 : units >= (int64_t)CW * dev_info().sm_count * 4;
+}
+
+size_t smem_of(int tmax, size_t code_bytes, int depth, int rd) {
+  return (size_t)header_bytes(tmax) + (size_t)CW * rd * tmax * 16 * 4 + code_bytes + (size_t)CW * depth * 1024;
 }
 
 // How one item is walked: in `nparts` parts of its K (as few as let the staged codes of a part, T rows of at most
@@ -519,19 +533,30 @@ struct ItemPlan {
   size_t code;
   int64_t npc;
 };
-bool plan_item(int T, int64_t M, int64_t K, ItemPlan* out) {
+// (`rd`: buffers of partial sums per warp the launch will have.  With 9 to 16 tokens fewer parts come before a deeper
+// ring: a part costs a staging pass over 16 rows of codes and a round trip of the sums through y.)
+bool plan_item(int T, int64_t M, int64_t K, ItemPlan* out, int rd = 2) {
   if (T < 1 || T > 16 || M < 1 || K < 1 || (K % 64) != 0 || M > 0x7fffffff) return false;
   const int64_t nch = i2s_kp(K) / 256;
   const size_t cap = (size_t)dev_info().max_smem_optin;
+  auto fits = [&](int n, int depth, ItemPlan* pl) {
+    const int64_t big = ceil_div(nch, n), small = nch / n;
+    if (small < 4) return false;
+    const size_t code = ((size_t)T * (size_t)(big * 256 + 64) + 127) & ~(size_t)127;
+    if (code > MAX_CODE_BYTES || smem_of(T, code, depth, rd) > cap) return false;
+    *pl = ItemPlan{n, code, small};
+    return true;
+  };
+  if (T > 8) {
+    for (int n = 1; n <= 16; ++n)
+      for (int want_depth = 6; want_depth >= 4; want_depth -= 2)
+        if (fits(n, want_depth, out)) return true;
+    return false;
+  }
   for (int want_depth = 6; want_depth >= 4; want_depth -= 2)
     for (int n = 1; n <= 16; ++n) {
-      const int64_t big = ceil_div(nch, n), small = nch / n;
-      if (small < 4) break;
-      const size_t code = ((size_t)T * (size_t)(big * 256 + 64) + 127) & ~(size_t)127;
-      if (code <= MAX_CODE_BYTES && smem_of(T, code, want_depth) <= cap) {
-        *out = ItemPlan{n, code, small};
-        return true;
-      }
+      if (nch / n < 4) break;
+      if (fits(n, want_depth, out)) return true;
     }
   return false;
 }
@@ -574,12 +599,14 @@ int launch_depth(const GArgs<NMAX>& a, int depth, int grid, size_t smem, cudaStr
 
 // S and ring depth for a launch whose shortest part has `npc` chunks, whose largest batch is `tmax` tokens and
 // whose largest staged codes take `code` bytes; false if they do not fit one SM's shared memory.
-bool launch_shape(int64_t npc, int tmax, size_t code, int64_t units, Shape* out) {
+bool launch_shape(int64_t npc, int tmax, size_t code, int64_t units, int rd, Shape* out) {
   if (npc < 4 || code > MAX_CODE_BYTES) return false;
   Shape sh = shape_for(npc, units);
+  if (rd == 1 && sh.S != 1) return false;     // (one buffer of partial sums per warp needs one warp per unit)
+  sh.rd = rd;
   const size_t cap = (size_t)dev_info().max_smem_optin;
-  while (sh.depth > 4 && smem_of(tmax, code, sh.depth) > cap) sh.depth = sh.depth == 12 ? 8 : sh.depth - 2;
-  if (smem_of(tmax, code, sh.depth) > cap) return false;
+  while (sh.depth > 4 && smem_of(tmax, code, sh.depth, sh.rd) > cap) sh.depth = sh.depth == 12 ? 8 : sh.depth - 2;
+  if (smem_of(tmax, code, sh.depth, sh.rd) > cap) return false;
   *out = sh;
   return true;
 }
@@ -597,7 +624,7 @@ int launch_run(const GroupLinear* items, int n, Shape shape, cudaStream_t st) {
     const GroupLinear& s = items[i];
     GItem& d = a.it[i];
     ItemPlan pl;
-    if (!plan_item(s.T, s.M, s.K, &pl)) return BITNET_ERR_UNSUPPORTED_SHAPE;
+    if (!plan_item(s.T, s.M, s.K, &pl, shape.rd)) return BITNET_ERR_UNSUPPORTED_SHAPE;
     d.packed = s.packed;
     d.x = s.x;
     d.q = s.q;
@@ -621,9 +648,10 @@ int launch_run(const GroupLinear* items, int n, Shape shape, cudaStream_t st) {
   a.total_units = (int)units;
   a.total_w = (int)w;
   a.code_bytes = (int)code;
-  a.r0 = a.r1 = 0;
+  a.r0 = shape.rd;
+  a.r1 = 0;
   const int depth = shape.depth;
-  const size_t smem = smem_of(a.tmax, code, depth);
+  const size_t smem = smem_of(a.tmax, code, depth, shape.rd);
   if (smem > (size_t)dev_info().max_smem_optin) return BITNET_ERR_UNSUPPORTED_SHAPE;
   const int G = CW / a.S;
   int grid = dev_info().sm_count;
@@ -642,7 +670,7 @@ int launch_run(const GroupLinear* items, int n, Shape shape, cudaStream_t st) {
 bool gemv_i2s_group_item_supported(int T, int64_t M, int64_t K) {
   ItemPlan pl;
   Shape sh;
-  return plan_item(T, M, K, &pl) && launch_shape(pl.npc, T, pl.code, ceil_div(M, 16), &sh);
+  return plan_item(T, M, K, &pl) && launch_shape(pl.npc, T, pl.code, ceil_div(M, 16), 2, &sh);
 }
 
 // Launches the grouped kernel over `n` supported items: as few launches as the argument block (NLARGE items,
@@ -659,15 +687,16 @@ int launch_gemv_i2s_group(const GroupLinear* items, int64_t n, cudaStream_t st) 
     const bool wide = items[i].T > 8;      // a launch holds items of one class: up to 8 tokens, or 9 to 16
     for (int64_t k = i; k < n && k - i < NLARGE && (items[k].T > 8) == wide; ++k)
       units += ceil_div(items[k].M, 16);   // (an estimate when the run is cut short)
+    const int rd = (wide && one_warp_per_unit(units)) ? 1 : 2;   // buffers of partial sums per warp
     while (j < n && j - i < NLARGE && (items[j].T > 8) == wide) {
       ItemPlan pl;
-      if (!plan_item(items[j].T, items[j].M, items[j].K, &pl)) return BITNET_ERR_UNSUPPORTED_SHAPE;
+      if (!plan_item(items[j].T, items[j].M, items[j].K, &pl, rd)) return BITNET_ERR_UNSUPPORTED_SHAPE;
       const int64_t add = ceil_div(items[j].M, 16) * (i2s_kp(items[j].K) / 256);
       const int tm = items[j].T > tmax ? items[j].T : tmax;
       const size_t cm = pl.code > code ? pl.code : code;
       const int64_t nm = pl.npc < npc_min ? pl.npc : npc_min;
       Shape sj;
-      const bool fits = launch_shape(nm, tm, cm, units, &sj);
+      const bool fits = launch_shape(nm, tm, cm, units, rd, &sj);
       if (!fits && j == i) return BITNET_ERR_UNSUPPORTED_SHAPE;
       if (!fits || (j > i && w + add > (1ll << 30))) break;
       w += add;
