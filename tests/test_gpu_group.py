@@ -93,9 +93,13 @@ def test_group_nine_to_sixteen_tokens_shared_input_and_many_units():
         it.check(rows=np.unique(np.concatenate([[0, 15, 16, it.M - 1], np.random.default_rng(it.M).integers(0, it.M, 200)])))
 
 
-def test_group_nine_to_sixteen_tokens_in_two_passes_in_a_child_process():
-    """BITNET_GROUP_WIDE=0 (read once per process): such items run as two items of the one-group kernel over the same
-    weights (tokens 0..7, then the rest)."""
+@pytest.mark.parametrize("extra", [dict(BITNET_GROUP_WIDE="0"), dict(BITNET_GROUP_S="1"),
+                                   dict(BITNET_GROUP_S="2", BITNET_GROUP_DEPTH="8")])
+def test_group_nine_to_sixteen_tokens_switches_in_child_processes(extra):
+    """Read-once switches on the list of 9-to-16-token items: BITNET_GROUP_WIDE=0 runs such items as two items of the
+    one-group kernel over the same weights (tokens 0..7, then the rest); BITNET_GROUP_S=1 forces one warp per unit
+    (the form with one buffer of partial sums per warp and the fewest parts of K, which otherwise only launches with
+    thousands of units take); two warps per unit with rings of eight chunks."""
     import os
     import subprocess
     import sys
@@ -109,9 +113,18 @@ def test_group_nine_to_sixteen_tokens_in_two_passes_in_a_child_process():
         "assert bn.bitnet_device_status() == 0\n"
         "print('ok')\n")
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    out = subprocess.run([sys.executable, "-c", code], cwd=root, env=dict(os.environ, BITNET_GROUP_WIDE="0"), capture_output=True,
+    out = subprocess.run([sys.executable, "-c", code], cwd=root, env=dict(os.environ, **extra), capture_output=True,
                          text=True, timeout=900)
-    assert out.returncode == 0 and "ok" in out.stdout, out.stderr[-2000:]
+    assert out.returncode == 0 and "ok" in out.stdout, (extra, out.stderr[-2000:])
+
+
+def test_group_nine_to_sixteen_tokens_one_warp_per_unit():
+    """Enough units that the launch runs with one warp per unit by itself: the two-group form with one buffer of
+    partial sums per warp, K = 8192 in one part at 16 tokens."""
+    items = [Item("i2s", 160000, 1024, 12, 176), Item("i2s", 4096, 8192, 16, 177), Item("i2s", 1024, 28672, 16, 178)]
+    run_group(items)
+    for it in items:
+        it.check(rows=np.unique(np.concatenate([[0, 15, 16, it.M - 1], np.random.default_rng(it.M).integers(0, it.M, 150)])))
 
 
 def test_group_many_units_per_cta_and_shared_inputs():
