@@ -100,7 +100,8 @@ struct TArgs {
 static_assert(sizeof(TArgs) <= 32764, "kernel parameter limit");
 
 struct __align__(8) Bars {
-  uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[NACC], tmem_empty[NACC], qsum_ready[NACC];
+  uint64_t full[MAX_STAGES], empty[MAX_STAGES];         // per step of the ring: codes written / operands read by the MMAs
+  uint64_t tmem_full[NACC], tmem_empty[NACC], qsum_ready[NACC];
   uint64_t b_full[4];                                   // a step's activation tiles have landed
   uint64_t a_full[MAX_SLOTS_A], a_empty[MAX_SLOTS_A];   // packed-word ring: bytes landed / slot read by every writer warp
   uint32_t tmem_base;
@@ -155,7 +156,7 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
   return d;
 }
 
-// Instruction descriptor: D = s32, A = u8 (the codes 0, 1, 2), B = s8, both K-major, N tokens, M = 128.
+// Instruction descriptor: D = s32, A = u8 (64 x the codes 0, 1, 2), B = s8, both K-major, N tokens, M = 128.
 __host__ __device__ constexpr uint32_t idesc_of(int n) {
   return (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
 }
