@@ -1,4 +1,4 @@
-"""Seeded random shapes through the list calls against the oracle: every format, 1..8 tokens, ragged row and column
+"""Seeded random shapes through the list calls against the oracle: every format at 1..8 tokens, I2_S up to 128, ragged row and column
 counts, short and long rows, lists that mix formats and shapes in one call.  The shapes are drawn so that each case
 stays small enough for the oracle to finish in well under a second."""
 import numpy as np
@@ -70,3 +70,23 @@ def test_random_lists_beyond_ternary(seed):
         acc_ref = oracle.mpgemm_def(q_ref, w.numpy())
         assert np.array_equal(npy(d["acc_out"]), acc_ref), (d["C"], d["M"], d["K"], x.shape[0])
         check_y(d["y"], acc_ref, sc_ref, 0.75)
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_random_i2s_lists_from_nine_to_128_tokens(seed):
+    """I2_S lists whose items have 1 to 128 tokens in random order: neighbouring items change between the grouped
+    kernel's one- and two-group forms, the streaming tensor-core kernel's 64- and 128-token tiles and the single-call
+    kernels (rows shorter than 2048 columns), ragged row counts, K with odd numbers of 256-column chunks."""
+    rng = np.random.default_rng(3000 + seed)
+    items = []
+    for i in range(12):
+        T = int(rng.choice([int(rng.integers(1, 9)), int(rng.integers(9, 17)), int(rng.integers(17, 65)),
+                            int(rng.integers(65, 129))]))
+        M = int(rng.integers(1, 300))
+        K = 64 * int(rng.integers(8, 130))
+        if rng.random() < 0.12:
+            M, K = int(rng.integers(1, 64)), 28672
+        items.append(Item("i2s", M, K, T, 7000 + 100 * seed + i, w_scale=float(rng.choice([0.5, 0.625, 1.0]))))
+    run_group(items)
+    for it in items:
+        it.check()
