@@ -326,8 +326,14 @@ def bench_batched(sw, torch, T, steps, warmup):
     grp = bn.make_group(items)
     ms = time_replays(torch, lambda: bn.bitnet_linear_group(grp), steps, warmup)
     weights = sw.bytes["i2s"] * 4.0          # four weights per packed byte
+    # roofline of the line: the weights once over HBM, or the multiply-adds on the int8 tensor cores (2 x the measured
+    # bf16 rate), whichever takes longer
+    pk = peaks()
+    ms_hbm, ms_tensor = sw.bytes["i2s"] / pk["hbm"] / 1e6, 2.0 * T * weights / (2.0 * pk["bf16"]) / 1e9
     return {"tokens": T, "ms_per_step": ms, "tokens_per_s": T / ms * 1e3, "weight_GBps": sw.bytes["i2s"] / ms / 1e6,
-            "frac_of_hbm_peak": sw.bytes["i2s"] / ms / 1e6 / peaks()["hbm"], "int8_tops": 2.0 * T * weights / ms / 1e9}
+            "frac_of_hbm_peak": sw.bytes["i2s"] / ms / 1e6 / pk["hbm"], "int8_tops": 2.0 * T * weights / ms / 1e9,
+            "roofline_ms": max(ms_hbm, ms_tensor), "roofline_bound": "hbm" if ms_hbm >= ms_tensor else "tensor",
+            "frac_of_roofline": max(ms_hbm, ms_tensor) / ms}
 
 
 def bench_small_configs(bn, torch, synth, steps, warmup):
