@@ -328,7 +328,18 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
       // chunk c of a row: 64 bytes; K block 2c + grp2 = its half grp2 (32 bytes), of which this thread takes 16
       int qs = 0, qs2 = 0;
       for (int s2 = 0; s2 < nsteps && ok; ++s2) {
-        // a tile that takes the sums of the codes reads this thread's pieces of the landed activation tiles
+        // the step's packed words have landed (bulk copies of the producer warp).  (A chunk beyond the row's last, or a
+        // row beyond M, is not copied: what the slot holds then meets activation codes that are all zero, or sums that
+        // are never stored.)
+        ok = mbar_wait(&bars->a_full[slot], pha, abort_flag, 20);
+        if (!ok) break;
+        // the tensor-memory columns of this step were last read by the MMAs of step g - RA
+        static_assert(RA == RB, "one barrier ring for both operands");
+        ok = mbar_wait(&bars->empty[bs], ph ^ 1u, abort_flag, 20);
+        if (!ok) break;
+        // A tile that takes the sums of the codes reads this thread's pieces of the landed activation tiles.  (After
+        // the wait above: the MMAs of step g - RB being over means the barrier of the activation tiles has left the
+        // phase of that step, so a probe for this step's phase cannot be answered by the one before.)
         if (need_q) {
           ok = mbar_wait(&bars->b_full[bs], ph, abort_flag, 20);
           if (!ok) break;
@@ -352,15 +363,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_i2s_stream_tc_kernel(const __
             }
           }
         }
-        // the step's packed words have landed (bulk copies of the producer warp).  (A chunk beyond the row's last, or a
-        // row beyond M, is not copied: what the slot holds then meets activation codes that are all zero, or sums that
-        // are never stored.)
-        ok = mbar_wait(&bars->a_full[slot], pha, abort_flag, 20);
-        if (!ok) break;
-        // the tensor-memory columns of this step were last read by the MMAs of step g - RA
-        static_assert(RA == RB, "one barrier ring for both operands");
-        ok = mbar_wait(&bars->empty[bs], ph ^ 1u, abort_flag, 20);
-        if (!ok) break;
         uint32_t wa[CPS][4];
 #pragma unroll
         for (int c = 0; c < CPS; ++c)
