@@ -482,9 +482,11 @@ int forced_s() {
 }
 int depth_cap() {
   static const int d = [] {
-    // six chunks per warp in flight measured fastest on the 100B sweep (2.45 ms per step against 2.59 with eight)
-    const int v = env_int_once("BITNET_GROUP_DEPTH", 6);
-    return (v == 4 || v == 6 || v == 8 || v == 12) ? v : 6;
+    // Four chunks per warp in flight (64 KB per SM) measured fastest on the 100B sweep with one warp per unit: 2.42 ms
+    // per step against 2.47 with three, 2.46 with five, 2.56 with six and 2.63 with eight (with four warps per unit,
+    // before units went to single warps, six had been best: 2.45 against 2.59 with eight).
+    const int v = env_int_once("BITNET_GROUP_DEPTH", 4);
+    return (v == 4 || v == 6 || v == 8 || v == 12) ? v : 4;
   }();
   return d;
 }
@@ -547,13 +549,14 @@ bool plan_item(int T, int64_t M, int64_t K, ItemPlan* out, int rd = 2) {
     *pl = ItemPlan{n, code, small};
     return true;
   };
+  const int top = depth_cap() >= 6 ? 6 : 4;      // (rings deeper than the launch will use need no room)
   if (T > 8) {
     for (int n = 1; n <= 16; ++n)
-      for (int want_depth = 6; want_depth >= 4; want_depth -= 2)
+      for (int want_depth = top; want_depth >= 4; want_depth -= 2)
         if (fits(n, want_depth, out)) return true;
     return false;
   }
-  for (int want_depth = 6; want_depth >= 4; want_depth -= 2)
+  for (int want_depth = top; want_depth >= 4; want_depth -= 2)
     for (int n = 1; n <= 16; ++n) {
       if (nch / n < 4) break;
       if (fits(n, want_depth, out)) return true;
