@@ -528,7 +528,7 @@ size_t smem_of(int tmax, size_t code_bytes, int depth, int rd) {
 }
 
 // How one item is walked: in `nparts` parts of its K (as few as let the staged codes of a part, T rows of at most
-// ceil(nch / nparts) chunks, fit beside a ring of at least 6 chunks per warp -- 4 if nothing else fits); `code` =
+// ceil(nch / nparts) chunks, fit beside the warps' rings, 4 chunks each unless BITNET_GROUP_DEPTH asks for more); `code` =
 // bytes of the staged codes of its largest part, `npc` = chunks of its smallest part.
 struct ItemPlan {
   int nparts;
