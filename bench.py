@@ -303,29 +303,32 @@ class Sweep:
         return replay
 
 
-def bench_batched(sw, torch, T, steps, warmup):
-    """The same sweep with T tokens per linear (I2_S) through ONE bitnet_linear_group call per step: quantiser +
-    mpGEMM + rescale.  Every linear keeps its own weights; the T activation rows of layer 0's four linears are
-    reused by all layers.  Up to 8 tokens the whole list is one persistent kernel; 9 to 16 tokens are two items of that
-    kernel per linear (tokens 0..7, then the rest: two launches of 320 items each); 17 to 128 tokens: the quantiser per
-    linear, then one launch of the streaming tcgen05 kernel over all 320 linears."""
+def bench_batched(sw, torch, T, steps, warmup, fmt="i2s"):
+    """The same sweep with T tokens per linear through ONE bitnet_linear_group call per step: quantiser + mpGEMM +
+    rescale.  Every linear keeps its own weights; the T activation rows of layer 0's four linears are reused by all
+    layers.  I2_S: up to 8 tokens the whole list is one persistent kernel; 9 to 16 tokens its two-group form after one
+    quantiser launch over the list; 17 to 128 tokens one quantiser launch, then the streaming tcgen05 kernel (160
+    linears per launch).  TL1, TL2 (up to 8 tokens): the scan kernel over the whole list."""
     bn, dev = sw.bn, sw.x_dev.device
     nl = len(sw.lin)
     xs = [sw.wl.activations(0, j, T).to(dev) for j in range(nl)]
     qs = [torch.empty((T, l.K), dtype=torch.int8, device=dev) for l in sw.lin]
     scs = [torch.empty(T, dtype=torch.float32, device=dev) for l in sw.lin]
     ys = [torch.empty((T, l.M), dtype=torch.float32, device=dev) for l in sw.lin]
-    ws = torch.zeros(max(16, max(bn.bitnet_mpgemm_workspace_bytes("i2s", T, l.M, l.K) for l in sw.lin)),
+    ws = torch.zeros(max(16, max(bn.bitnet_mpgemm_workspace_bytes(fmt, T, l.M, l.K) for l in sw.lin)),
                      dtype=torch.uint8, device=dev)
     items = []
     for i in range(sw.n_linears()):
         j = i % nl
         lin = sw.lin[j]
-        items.append(dict(fmt="i2s", packed=sw.blobs["i2s"][i], w_scale=sw.w_scale[i], M=lin.M, K=lin.K, x=xs[j], q=qs[j],
+        items.append(dict(fmt=fmt, packed=sw.blobs[fmt][i], w_scale=sw.w_scale[i], M=lin.M, K=lin.K, x=xs[j], q=qs[j],
                           act_scale=scs[j], y=ys[j], workspace=ws))
     grp = bn.make_group(items)
     ms = time_replays(torch, lambda: bn.bitnet_linear_group(grp), steps, warmup)
-    weights = sw.bytes["i2s"] * 4.0          # four weights per packed byte
+    weights = sw.bytes["i2s"] * 4.0          # four weights per packed byte of the I2_S blob
+    if fmt != "i2s":
+        return {"tokens": T, "ms_per_step": ms, "tokens_per_s": T / ms * 1e3, "weight_GBps": sw.bytes[fmt] / ms / 1e6,
+                "frac_of_hbm_peak": sw.bytes[fmt] / ms / 1e6 / peaks()["hbm"], "int8_tops": 2.0 * T * weights / ms / 1e9}
     # roofline of the line: the weights once over HBM, or the multiply-adds on the int8 tensor cores (2 x the measured
     # bf16 rate), whichever takes longer
     pk = peaks()
@@ -665,6 +668,10 @@ def run_ours(args):
             line["tl1"] = {"packed_bytes": sw.bytes["tl1"], "ms_per_step": ms_tl1, "value": sw.bytes["tl1"] / ms_tl1 / 1e6,
                            "unit": UNIT, "frac_of_hbm_peak": sw.bytes["tl1"] / ms_tl1 / 1e6 / pk["hbm"],
                            "kernel": "gemv_tl2_scan_kernel, arithmetic mode (one bitnet_linear_group call per step)"}
+            if not args.skip_batched:
+                nb = max(3, args.steps // 10)
+                line["tl2"]["batched"] = [bench_batched(sw, torch, T, nb, 3, "tl2") for T in (2, 4, 8)]
+                line["tl1"]["batched"] = [bench_batched(sw, torch, T, nb, 3, "tl1") for T in (2, 4, 8)]
             sw.step_group("tl2")        # the verification below sees the scan kernel's y
         if not args.skip_batched:
             line["batched_decode"] = {

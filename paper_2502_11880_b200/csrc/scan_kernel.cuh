@@ -336,13 +336,16 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
   float* qred = reinterpret_cast<float*>(smem + 128);
   float* qmul = reinterpret_cast<float*>(smem + 640);            // [8] 127 / amax per token
   unsigned* tbl1 = reinterpret_cast<unsigned*>(smem + 1024);     // [256] index byte of two pairs -> four codes
-  int* red = reinterpret_cast<int*>(smem + 2048);                // [CW][2][tmax][32] partial sums
-  unsigned* tbl2 = reinterpret_cast<unsigned*>(smem + 2048 + CW * 2 * a.tmax * 32 * 4);   // [1024][32 lanes]
+  // partial sums [CW][RD][tmax][32]: two buffers per warp, so that a warp may start its next block while its group
+  // still adds up the last one; one (bit 8 of a.S) when every warp finishes its own blocks
+  const int RD = (a.S & 0x100) ? 1 : 2;
+  int* red = reinterpret_cast<int*>(smem + 2048);
+  unsigned* tbl2 = reinterpret_cast<unsigned*>(smem + 2048 + CW * RD * a.tmax * 32 * 4);   // [1024][32 lanes]
   int8_t* qs_mem = reinterpret_cast<int8_t*>(tbl2) + (F >= 2 ? 0 : TBL2_BYTES);   // (the mask and arithmetic modes have no table)
   uint8_t* rings = reinterpret_cast<uint8_t*>(qs_mem) + a.code_bytes;
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int S = a.S, G = CW / S, gi = warp / S, wk = warp % S;
+  const int S = a.S & 0xff, G = CW / S, gi = warp / S, wk = warp % S;
   const int g = lane >> 2, t = lane & 3;
 
   if (threadIdx.x == 0) {
@@ -639,7 +642,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
         cur = nxt;
 
         // fragments: c[0] = (row g, token 2t), c[1] = (row g, token 2t+1), c[2], c[3] = the same for row g+8
-        int* mine = red + ((warp * 2 + (nloc & 1)) * tmax) * 32;
+        const int rbuf = RD == 2 ? (nloc & 1) : 0;
+        int* mine = red + ((warp * RD + rbuf) * tmax) * 32;
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
           int c[4];
@@ -662,10 +666,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemv_tl2_scan_kernel(const __grid_
           // this block's turn to be finished by this warp: add the group's partials; the sums of an item walked in
           // parts rest in y (as integers) between the parts; the last part rescales and stores 32 rows
           const int row0 = (cj - first) * 32;
-          const int* grp = red + (((gi * S) * 2 + (nloc & 1)) * tmax) * 32;
+          const int* grp = red + (((gi * S) * RD + rbuf) * tmax) * 32;
           for (int idx = lane; idx < T * 32; idx += 32) {
             int v = 0;
-            for (int w2 = 0; w2 < S; ++w2) v += grp[w2 * 2 * tmax * 32 + idx];
+            for (int w2 = 0; w2 < S; ++w2) v += grp[w2 * RD * tmax * 32 + idx];
             const int tok = idx >> 5, row = row0 + (idx & 31);
             v -= (F ? a.card >> 1 : 1) * qsum[tok];     // codes are weights + 1 (+ C/2)
             if (row < M) {
@@ -706,8 +710,14 @@ inline int forced_s() {
   return s;
 }
 
-inline size_t smem_of(int tmax, size_t code_bytes, int depth, int F) {
-  return 2048 + (size_t)CW * 2 * tmax * 32 * 4 + (F >= 2 ? 0 : TBL2_BYTES) + code_bytes + (size_t)CW * depth * SLOT;
+// (`rd`: buffers of partial sums per warp: 1 when the launch runs with one warp per block, else 2)
+inline size_t smem_of(int tmax, size_t code_bytes, int depth, int F, int rd) {
+  return 2048 + (size_t)CW * rd * tmax * 32 * 4 + (F >= 2 ? 0 : TBL2_BYTES) + code_bytes + (size_t)CW * depth * SLOT;
+}
+// true if a launch over `units` blocks runs with one warp per block
+inline bool one_warp_per_block(int64_t units) {
+  const int f = forced_s();
+  return f ? f == 1 : units >= (int64_t)CW * dev_info().sm_count * 4;
 }
 
 // How one item is walked: its triple tiles in `nparts` parts (as few as let the staged codes of a part fit beside
@@ -718,28 +728,40 @@ struct ItemPlan {
   size_t code;
   int t3;
 };
-inline bool plan_item(int T, const TlGeom& g, int cols, int F, ItemPlan* out) {
+inline bool plan_item(int T, const TlGeom& g, int cols, int F, ItemPlan* out, int rd = 2) {
   const size_t cap = (size_t)dev_info().max_smem_optin;
   const int tiles3 = (int)g.tiles3, tiles2 = (int)g.tiles2;
+  auto fits = [&](int n, int depth) {
+    const int big = (tiles3 + n - 1) / n, small = tiles3 / n;
+    if (small < 3) return false;
+    const size_t code = ((size_t)T * (size_t)staged_stride(cols, big, tiles2) + 127) & ~(size_t)127;
+    if (smem_of(T, code, depth, F, rd) > cap) return false;
+    *out = ItemPlan{n, code, small};
+    return true;
+  };
+  if (F < 2 && T > 4) {
+    // table modes with many tokens: fewer parts before deeper rings (the decode binds, not the weight stream, and a
+    // part costs a staging pass and a round trip of the sums through y)
+    for (int n = 1; n <= 16; ++n)
+      for (int want_depth = 4; want_depth >= 3; --want_depth)
+        if (fits(n, want_depth)) return true;
+    return false;
+  }
   for (int want_depth = 4; want_depth >= 3; --want_depth)
     for (int n = 1; n <= 16; ++n) {
-      const int big = (tiles3 + n - 1) / n, small = tiles3 / n;
-      if (small < 3) break;
-      const size_t code = ((size_t)T * (size_t)staged_stride(cols, big, tiles2) + 127) & ~(size_t)127;
-      if (smem_of(T, code, want_depth, F) <= cap) {
-        *out = ItemPlan{n, code, small};
-        return true;
-      }
+      if (tiles3 / n < 3) break;
+      if (fits(n, want_depth)) return true;
     }
   return false;
 }
 
 struct Shape {
   int S, depth;
+  int rd = 2;
 };
 // S and ring depth for a launch whose shortest rows have `t3` triple tiles: every warp's run of triple tiles is at
 // least as long as its ring; the ring is made shallower until everything fits one SM's shared memory.
-inline bool launch_shape(int t3, int tmax, size_t code, int64_t units, int F, Shape* out) {
+inline bool launch_shape(int t3, int tmax, size_t code, int64_t units, int F, Shape* out, int rd = 2) {
   // Warps per 32-row block: one when the launch has enough blocks to keep the 16 warps of every SM busy with
   // blocks of their own (no partial sums to join: 3.4 TB/s against 3.1 with four on the 100B sweep), more when
   // it has few.
@@ -754,9 +776,14 @@ inline bool launch_shape(int t3, int tmax, size_t code, int64_t units, int F, Sh
   const size_t cap = (size_t)dev_info().max_smem_optin;
   int depth = depth_cap();
   auto lower = [](int d) { return d == 8 ? 6 : d - 1; };
-  while (depth > 3 && (depth > nw || smem_of(tmax, code, depth, F) > cap)) depth = lower(depth);
-  if (depth > nw || smem_of(tmax, code, depth, F) > cap) return false;
-  *out = Shape{S, depth};
+  if (rd == 1 && S != 1) return false;          // (one buffer of partial sums per warp needs one warp per block)
+  while (depth > 3 && (depth > nw || smem_of(tmax, code, depth, F, rd) > cap)) depth = lower(depth);
+  if (depth > nw || smem_of(tmax, code, depth, F, rd) > cap) return false;
+  Shape sh;
+  sh.S = S;
+  sh.depth = depth;
+  sh.rd = rd;
+  *out = sh;
   return true;
 }
 
@@ -802,7 +829,7 @@ int launch_run(const Tl2Linear* items, int n, int card, Shape shape, cudaStream_
   constexpr int COLS = F ? 64 : 96;
   static thread_local SArgs<NMAX> a;
   a.n = n;
-  a.S = shape.S;
+  a.S = shape.S | (shape.rd == 1 ? 0x100 : 0);
   a.tmax = 1;
   size_t code = 0;
   int64_t units = 0, w = 0;
@@ -810,7 +837,7 @@ int launch_run(const Tl2Linear* items, int n, int card, Shape shape, cudaStream_
     const Tl2Linear& s = items[i];
     SItem& d = a.it[i];
     ItemPlan pl;
-    if (!plan_item(s.T, s.g, COLS, F, &pl)) return BITNET_ERR_UNSUPPORTED_SHAPE;
+    if (!plan_item(s.T, s.g, COLS, F, &pl, shape.rd)) return BITNET_ERR_UNSUPPORTED_SHAPE;
     d.packed = s.packed;
     d.x = s.x;
     d.q = s.q;
@@ -839,14 +866,14 @@ int launch_run(const Tl2Linear* items, int n, int card, Shape shape, cudaStream_
   a.code_bytes = (int)code;
   a.card = card;
   a.tile_bytes = (F && n > 0) ? (int)(items[0].g.block_bytes / items[0].g.tiles3) : SLOT;
-  const size_t smem = smem_of(a.tmax, code, shape.depth, F);
+  const size_t smem = smem_of(a.tmax, code, shape.depth, F, shape.rd);
   if (smem > (size_t)dev_info().max_smem_optin) return BITNET_ERR_UNSUPPORTED_SHAPE;
-  const int G = CW / a.S;
+  const int G = CW / shape.S;
   int grid = dev_info().sm_count;
   if ((int64_t)grid * G > units) grid = (int)ceil_div(units, G);
   log_launch(F ? "gemv_tl2_scan_kernel<pairs> items=%d blocks=%lld tiles=%lld grid=%d warps/block=%d ring=%d tmax=%d smem=%zu"
                : "gemv_tl2_scan_kernel items=%d blocks=%lld tiles=%lld grid=%d warps/block=%d ring=%d tmax=%d smem=%zu", n,
-             (long long)units, (long long)w, grid, a.S, shape.depth, a.tmax, smem);
+             (long long)units, (long long)w, grid, shape.S, shape.depth, a.tmax, smem);
   return launch_depth<NMAX, F>(a, shape.depth, grid, smem, st);
 }
 
@@ -873,16 +900,17 @@ int launch_items(const Tl2Linear* items, int64_t n, int card, cudaStream_t st) {
     Shape sh{1, 3};
     int64_t units = 0;
     for (int64_t k = i; k < n && k - i < NLARGE; ++k) units += items[k].M / 32;   // (an estimate when the run is cut short)
+    const int rd = one_warp_per_block(units) ? 1 : 2;   // buffers of partial sums per warp
     while (j < n && j - i < NLARGE) {
       const TlGeom& g = items[j].g;
       ItemPlan pl;
-      if (!plan_item(items[j].T, g, COLS, F, &pl)) return BITNET_ERR_UNSUPPORTED_SHAPE;
+      if (!plan_item(items[j].T, g, COLS, F, &pl, rd)) return BITNET_ERR_UNSUPPORTED_SHAPE;
       const int64_t add = (items[j].M / 32) * (g.tiles3 + g.tiles2);
       const int tm = items[j].T > tmax ? items[j].T : tmax;
       const size_t cm = pl.code > code ? pl.code : code;
       const int t3 = pl.t3 < t3_min ? pl.t3 : t3_min;
       Shape sj;
-      const bool fits = launch_shape(t3, tm, cm, units, F, &sj);
+      const bool fits = launch_shape(t3, tm, cm, units, F, &sj, rd);
       if (!fits && j == i) return BITNET_ERR_UNSUPPORTED_SHAPE;
       if (!fits || (j > i && w + add > (1ll << 30))) break;
       w += add;
