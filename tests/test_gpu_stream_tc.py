@@ -60,6 +60,15 @@ def test_stream_tc_same_list_ten_times():
         assert np.array_equal(it.gacc.t.cpu().numpy(), acc_ref)
 
 
+def test_stream_tc_leaves_very_long_rows_to_other_kernels():
+    """K beyond 131072 (64 x the sums would leave 32 bits) is not taken by the streaming kernel: the list call hands
+    such items to the single-call kernels, K = 131072 itself still runs here; both agree with the oracle."""
+    items = [Item("i2s", 96, 131072, 20, 890), Item("i2s", 64, 131072 + 64, 20, 891)]
+    run_group(items)
+    for it in items:
+        it.check()
+
+
 def test_stream_tc_sixty_five_to_128_tokens():
     """The 128-token tile variant (two activation pieces per writer thread and K block, 8 stages), mixed with
     64-token items in one list (separate launches per class), ragged rows and a long row."""
